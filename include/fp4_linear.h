@@ -1,0 +1,170 @@
+/*
+ * fp4_linear.h -- C ABI of the FP4-quantized linear layer for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the linear-layer hot path of "Optimizing Large Language Model
+ * Training Using FP4 Quantization": vector-wise absmax quantisation to E2M1 (Eq. 1 with the
+ * look-up quantiser of Appendix A), outlier clamping at a quantile with a sparse residual
+ * (Section 3.2), the FP4 GEMM with the two de-scales applied to its result (Fig. 2,
+ * Appendix C.2), the compensation product, and the backward pass with the differentiable
+ * gradient estimator (Eq. 6-8).
+ *
+ * Conventions shared by every entry point
+ * ---------------------------------------
+ *  - Every tensor pointer is a DEVICE pointer unless the parameter is documented as host.
+ *    Tensors are dense, row-major and 16-byte aligned.  The caller owns every tensor; the
+ *    context owns only its workspace.  Nothing is allocated after fp4_create().
+ *  - Notation: A[M x K] activations, W[K x N] weights (input channels x output channels),
+ *    Y[M x N] = A W.  M, K and N must be multiples of 128.
+ *  - E2M1 codes are sign-magnitude nibbles (bit 3 sign; 0..7 -> 0, .5, 1, 1.5, 2, 3, 4, 6),
+ *    two per byte with the even element in bits 3:0.  A negative zero code is never written.
+ *  - Calls are asynchronous on `stream` (a cudaStream_t passed as void*).  They return 0 or
+ *    a negative FP4_ERR_* code for errors found on the host before anything is enqueued.
+ *  - Conditions found on the device are OR-ed into the caller's device word `*status`
+ *    (FP4_DEV_* bits).  When a bit is set the outputs are unspecified but every write stayed
+ *    inside the caller's buffers.  Every device-side wait is bounded: a stalled pipeline
+ *    sets FP4_DEV_TIMEOUT and the kernel returns.
+ */
+#ifndef FP4_LINEAR_H_
+#define FP4_LINEAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* host-side return codes */
+#define FP4_OK              0
+#define FP4_ERR_NULL       (-1)   /* a required pointer is NULL                              */
+#define FP4_ERR_SHAPE      (-2)   /* a dimension is not a positive multiple of 128           */
+#define FP4_ERR_ALPHA      (-3)   /* alpha outside (0.5, 1]                                  */
+#define FP4_ERR_ALIGN      (-4)   /* a tensor pointer is not 16-byte aligned                 */
+#define FP4_ERR_WORKSPACE  (-5)   /* the context's workspace is too small for this call      */
+#define FP4_ERR_CUDA       (-6)   /* a CUDA runtime / driver call failed                     */
+#define FP4_ERR_ARG        (-7)   /* an argument has an unsupported value                    */
+#define FP4_ERR_CAPACITY   (-8)   /* sparse_cap is below the guaranteed bound 2 * n_tail     */
+
+/* bits of the device status word */
+#define FP4_DEV_SPARSE_OVERFLOW  1   /* more residual entries than sparse_cap                */
+#define FP4_DEV_NONFINITE        2   /* reserved: a non-finite input was seen                */
+#define FP4_DEV_TIMEOUT          4   /* a bounded wait inside a kernel ran out               */
+
+/* gemm_kind: which tcgen05.mma flavour multiplies the E2M1 codes */
+#define FP4_GEMM_MXF4    0   /* packed nibbles, K = 64 per instruction, unit block scales    */
+#define FP4_GEMM_F8F6F4  1   /* nibbles in byte containers, K = 32 per instruction           */
+
+typedef struct fp4_ctx fp4_ctx;   /* opaque: device id, SM count, workspace */
+
+/* One quantised operand.  Every buffer is allocated by the caller; pointers that are not
+ * needed may be NULL (then that output is skipped).                                        */
+typedef struct fp4_qtensor {
+  int64_t  rows, cols;     /* logical shape of the source tensor                              */
+  uint8_t* codes;          /* [rows x cols/2]  (r, 2j) low nibble, (r, 2j+1) high nibble      */
+  uint8_t* codes_t;        /* [cols x rows/2]  (2i, c) low nibble, (2i+1, c) high nibble      */
+  float*   amax;           /* [rows] if scale_axis == 0 else [cols]: exact max |x| of each
+                              vector (after the clamp and the optional prescale); the scale
+                              of Eq. 1 is gamma = 6 / amax and the de-scale amax / 6, each
+                              rounded once to float                                           */
+  float*   thresholds;     /* [2] = {lo, hi}: the (1-alpha)- and alpha-quantile (OCC only)    */
+  int32_t* csr_rowptr;     /* [rows + 1]                                                      */
+  int32_t* csr_col;        /* [sparse_cap] column index, ascending within a row               */
+  float*   csr_val;        /* [sparse_cap] x - clamp(x)                                       */
+  int32_t* csc_colptr;     /* [cols + 1]                                                      */
+  int32_t* csc_row;        /* [sparse_cap] row index, ascending within a column               */
+  float*   csc_val;        /* [sparse_cap]                                                    */
+  int64_t  sparse_cap;     /* capacity in entries; 2 * round((1-alpha) * rows * cols) always
+                              suffices                                                        */
+  int32_t* nnz;            /* [1] number of residual entries                                  */
+} fp4_qtensor;
+
+/* Create a context on `device` with a workspace of `workspace_bytes` (cudaMalloc'ed here,
+ * freed by fp4_destroy).  fp4_workspace_bytes() gives a sufficient size.  `out` is host.   */
+int fp4_create(fp4_ctx** out, int device, size_t workspace_bytes);
+int fp4_destroy(fp4_ctx* ctx);
+
+/* Workspace that fp4_quantize / fp4_linear_fwd / fp4_linear_bwd need for these sizes.      */
+size_t fp4_workspace_bytes(int64_t M, int64_t K, int64_t N);
+
+/* Text of a host return code (static string).                                              */
+const char* fp4_status_string(int code);
+
+/*
+ * fp4_quantize -- vector-wise absmax quantisation to E2M1 (Eq. 1; quantiser Q: Appendix A;
+ * granularity: Section 4.1), optionally preceded by outlier clamping with the sparse
+ * residual emitted alongside (Section 3.2).
+ *
+ *   x_bf16      [rows x cols] BF16
+ *   scale_axis  0: one scale per row (token-wise, activations)
+ *               1: one scale per column (channel-wise, weights W[c_i x c_o])
+ *   alpha       1.0: no clamp.  Otherwise 0.5 < alpha < 1: with n = rows*cols and
+ *               n_tail = llround((1-alpha)*n), lo and hi are the order statistics
+ *               sorted[n_tail] and sorted[n-1-n_tail] of the whole tensor; x is clamped to
+ *               [lo, hi] BEFORE the absmax, and every x outside [lo, hi] yields a residual
+ *               entry x - clamp(x).  Requires scale_axis == 0 and prescale == NULL.
+ *   prescale    optional float vector along the OTHER axis ([cols] for scale_axis 0,
+ *               [rows] for scale_axis 1): x is replaced by float(x * prescale) first.
+ *   out         destination buffers (host struct of device pointers); amax is required,
+ *               at least one of codes / codes_t is required; with alpha < 1 thresholds,
+ *               nnz, csr_* and csc_* are required.
+ * Scaled value: v = float(x) * gamma with one float rounding; code = Q(v), where a value
+ * equal to a threshold of the chain goes to the larger neighbour.  A zero vector gets
+ * amax = 0 and all-zero codes.
+ */
+int fp4_quantize(fp4_ctx* ctx, void* stream, const void* x_bf16, int64_t rows, int64_t cols,
+                 int scale_axis, double alpha, const float* prescale,
+                 fp4_qtensor* out, int32_t* status);
+
+/*
+ * fp4_gemm -- the FP4 GEMM of Fig. 2 on E2M1 codes with the two de-scales applied to the
+ * result (Appendix C.2: the GEMM consumes the scaled quantised tensors, the de-scale comes
+ * afterwards):
+ *     out[i, j] = (acc[i, j] * d_row[i]) * d_col[j],
+ *     acc[i, j] = sum_c val(a_codes[i, c]) * val(b_codes[j, c])   (fp32 accumulation),
+ *     d = amax / 6 rounded to float; a NULL amax vector means d = 1.
+ *   a_codes [I x C/2], b_codes [J x C/2]: both operands have the contraction contiguous.
+ *   out     [I x J], float if out_f32 != 0 else BF16.
+ *   I, J, C multiples of 128.  gemm_kind: FP4_GEMM_MXF4 or FP4_GEMM_F8F6F4.
+ */
+int fp4_gemm(fp4_ctx* ctx, void* stream, const uint8_t* a_codes, const uint8_t* b_codes,
+             int64_t I, int64_t J, int64_t C, const float* row_amax, const float* col_amax,
+             void* out, int out_f32, int gemm_kind, int32_t* status);
+
+/*
+ * fp4_linear_fwd -- forward of the FP4 linear layer (Fig. 2, Section 3.2):
+ *     Y = bf16( (Q(A_c) Q(W)) (.) d_A[m] (.) d_W[n]  +  (A - A_c) W )
+ * A is clamped at the alpha-quantiles and quantised token-wise, W channel-wise; the residual
+ * A - A_c multiplies the BF16 weight in fp32; both branches meet in fp32 and are rounded once.
+ *   A_bf16 [M x K], W_bf16 [K x N], Y [M x N] (BF16, or float if out_f32 != 0).
+ *   savedA, savedW: caller-allocated fp4_qtensor buffers that receive the quantised operands
+ *   and are handed to fp4_linear_bwd.  savedA needs codes, codes_t, amax, thresholds, nnz,
+ *   csr_*, csc_*; savedW needs codes, codes_t, amax.  If reuse_w != 0, savedW already holds
+ *   this weight's codes (weights change once per optimizer step) and is not recomputed.
+ */
+int fp4_linear_fwd(fp4_ctx* ctx, void* stream, const void* A_bf16, const void* W_bf16,
+                   int64_t M, int64_t K, int64_t N, double alpha, int reuse_w, int gemm_kind,
+                   void* Y, int out_f32, fp4_qtensor* savedA, fp4_qtensor* savedW,
+                   int32_t* status);
+
+/*
+ * fp4_linear_bwd -- backward of the FP4 linear layer (Eq. 3, Eq. 6, Appendix C.2):
+ *     dA = bf16( dY W_q^T )                         with the forward's W_q,
+ *     dW = bf16( (Q(A_c)^T dY + (A - A_c)^T dY) (.) Q'(W (.) sf) )
+ * where Q' is the DGE derivative of Eq. 8 with exponent parameter dge_k (paper: 5) capped at
+ * dge_clip (paper: 3.0), evaluated on the scaled weights the forward quantised; dge_on == 0
+ * selects the straight-through estimator (Q' = 1).  Both GEMMs take E2M1 operands: dY is
+ * quantised token-wise after multiplication by d_W[n] (dgrad) and channel-wise after
+ * multiplication by d_A[m] (wgrad), so that the forward's codes of W and A are re-used.
+ *   dY_bf16 [M x N], W_bf16 [K x N], dA [M x K], dW [K x N] (BF16, or float if out_f32).
+ *   dA or dW may be NULL to skip that gradient.
+ */
+int fp4_linear_bwd(fp4_ctx* ctx, void* stream, const void* dY_bf16, const void* W_bf16,
+                   const fp4_qtensor* savedA, const fp4_qtensor* savedW,
+                   int64_t M, int64_t K, int64_t N,
+                   int dge_on, float dge_k, float dge_clip, int gemm_kind,
+                   void* dA, void* dW, int out_f32, int32_t* status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FP4_LINEAR_H_ */

@@ -1,0 +1,13 @@
+"""FP4-quantized linear layer for NVIDIA B200 (sm_100a): Python binding of libfp4linear.so.
+
+The library is the product; this package marshals arguments to its C ABI
+(include/fp4_linear.h).  Importing the package does not load the library, so the
+seeded workload generators stay usable on a machine without CUDA; every compute
+entry point loads it on first use and raises if it has not been built.
+"""
+from .binding import (  # noqa: F401
+    FP4_DEV_NONFINITE, FP4_DEV_SPARSE_OVERFLOW, FP4_DEV_TIMEOUT, FP4_GEMM_F8F6F4, FP4_GEMM_MXF4, EXPORTS,
+    Context, Fp4Error, QTensor, fp4_gemm, fp4_linear_bwd, fp4_linear_fwd, fp4_quantize, load_library,
+    tail_capacity,
+)
+from . import workloads  # noqa: F401

@@ -1,0 +1,218 @@
+"""Thin ctypes binding of libfp4linear.so: argument marshalling only.
+
+Function names and argument order follow include/fp4_linear.h.  PyTorch is used for device
+memory and the current stream; every step of the path runs inside the library's kernels.
+There is no CPU fallback: if the shared library is missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from .build import LIB_PATH
+
+FP4_GEMM_MXF4 = 0
+FP4_GEMM_F8F6F4 = 1
+FP4_DEV_SPARSE_OVERFLOW = 1
+FP4_DEV_NONFINITE = 2
+FP4_DEV_TIMEOUT = 4
+
+EXPORTS = ("fp4_create", "fp4_destroy", "fp4_workspace_bytes", "fp4_status_string", "fp4_quantize",
+           "fp4_gemm", "fp4_linear_fwd", "fp4_linear_bwd")
+
+
+class fp4_qtensor(C.Structure):
+    _fields_ = [
+        ("rows", C.c_int64), ("cols", C.c_int64),
+        ("codes", C.c_void_p), ("codes_t", C.c_void_p), ("amax", C.c_void_p), ("thresholds", C.c_void_p),
+        ("csr_rowptr", C.c_void_p), ("csr_col", C.c_void_p), ("csr_val", C.c_void_p),
+        ("csc_colptr", C.c_void_p), ("csc_row", C.c_void_p), ("csc_val", C.c_void_p),
+        ("sparse_cap", C.c_int64), ("nnz", C.c_void_p),
+    ]
+
+
+_lib = None
+
+
+def load_library(path: str | None = None) -> C.CDLL:
+    """dlopen the in-tree library and declare its prototypes.  Raises if it was not built."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    path = path or LIB_PATH
+    if not os.path.exists(path):
+        raise RuntimeError(
+            f"{path} is missing: build it with `python -m paper_2501_17116_b200.build` "
+            "(there is no fallback path)")
+    lib = C.CDLL(path)
+    vp, i64, i32p = C.c_void_p, C.c_int64, C.c_void_p
+    lib.fp4_create.argtypes = [C.POINTER(vp), C.c_int, C.c_size_t]
+    lib.fp4_create.restype = C.c_int
+    lib.fp4_destroy.argtypes = [vp]
+    lib.fp4_destroy.restype = C.c_int
+    lib.fp4_workspace_bytes.argtypes = [i64, i64, i64]
+    lib.fp4_workspace_bytes.restype = C.c_size_t
+    lib.fp4_status_string.argtypes = [C.c_int]
+    lib.fp4_status_string.restype = C.c_char_p
+    lib.fp4_quantize.argtypes = [vp, vp, vp, i64, i64, C.c_int, C.c_double, vp, C.POINTER(fp4_qtensor), i32p]
+    lib.fp4_quantize.restype = C.c_int
+    lib.fp4_gemm.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp, vp, vp, C.c_int, C.c_int, i32p]
+    lib.fp4_gemm.restype = C.c_int
+    lib.fp4_linear_fwd.argtypes = [vp, vp, vp, vp, i64, i64, i64, C.c_double, C.c_int, C.c_int, vp, C.c_int,
+                                   C.POINTER(fp4_qtensor), C.POINTER(fp4_qtensor), i32p]
+    lib.fp4_linear_fwd.restype = C.c_int
+    lib.fp4_linear_bwd.argtypes = [vp, vp, vp, vp, C.POINTER(fp4_qtensor), C.POINTER(fp4_qtensor), i64, i64, i64,
+                                   C.c_int, C.c_float, C.c_float, C.c_int, vp, vp, C.c_int, i32p]
+    lib.fp4_linear_bwd.restype = C.c_int
+    if path == LIB_PATH:
+        _lib = lib
+    return lib
+
+
+class Fp4Error(RuntimeError):
+    def __init__(self, code: int):
+        self.code = code
+        super().__init__(f"fp4 error {code}: {load_library().fp4_status_string(code).decode()}")
+
+
+def _check(rc: int):
+    if rc != 0:
+        raise Fp4Error(rc)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+class Context:
+    """fp4_create / fp4_destroy.  Owns the workspace and a device status word."""
+
+    def __init__(self, device: int = 0, workspace_bytes: int = 0):
+        self.lib = load_library()
+        self.device = device
+        self.handle = C.c_void_p()
+        torch.cuda.set_device(device)
+        _check(self.lib.fp4_create(C.byref(self.handle), device, workspace_bytes))
+        self.workspace_bytes = workspace_bytes
+        self.status = torch.zeros(1, dtype=torch.int32, device=f"cuda:{device}")
+
+    @classmethod
+    def for_shape(cls, M: int, K: int, N: int, device: int = 0):
+        return cls(device, int(load_library().fp4_workspace_bytes(M, K, N)))
+
+    def close(self):
+        if self.handle:
+            self.lib.fp4_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def read_status(self) -> int:
+        """Device status word (synchronises)."""
+        return int(self.status.item())
+
+
+class QTensor:
+    """Caller-owned buffers of one quantised operand (struct fp4_qtensor)."""
+
+    def __init__(self, rows: int, cols: int, scale_axis: int, device, sparse_cap: int = 0,
+                 codes: bool = True, codes_t: bool = True):
+        dev = device
+        self.rows, self.cols, self.scale_axis = rows, cols, scale_axis
+        self.codes = torch.empty((rows, cols // 2), dtype=torch.uint8, device=dev) if codes else None
+        self.codes_t = torch.empty((cols, rows // 2), dtype=torch.uint8, device=dev) if codes_t else None
+        self.amax = torch.empty(rows if scale_axis == 0 else cols, dtype=torch.float32, device=dev)
+        self.sparse_cap = int(sparse_cap)
+        if sparse_cap > 0:
+            cap = max(int(sparse_cap), 1)
+            self.thresholds = torch.zeros(2, dtype=torch.float32, device=dev)
+            self.csr_rowptr = torch.zeros(rows + 1, dtype=torch.int32, device=dev)
+            self.csr_col = torch.zeros(cap, dtype=torch.int32, device=dev)
+            self.csr_val = torch.zeros(cap, dtype=torch.float32, device=dev)
+            self.csc_colptr = torch.zeros(cols + 1, dtype=torch.int32, device=dev)
+            self.csc_row = torch.zeros(cap, dtype=torch.int32, device=dev)
+            self.csc_val = torch.zeros(cap, dtype=torch.float32, device=dev)
+            self.nnz = torch.zeros(1, dtype=torch.int32, device=dev)
+        else:
+            self.thresholds = self.csr_rowptr = self.csr_col = self.csr_val = None
+            self.csc_colptr = self.csc_row = self.csc_val = self.nnz = None
+        self.struct = fp4_qtensor(
+            rows, cols, _ptr(self.codes), _ptr(self.codes_t), _ptr(self.amax), _ptr(self.thresholds),
+            _ptr(self.csr_rowptr), _ptr(self.csr_col), _ptr(self.csr_val),
+            _ptr(self.csc_colptr), _ptr(self.csc_row), _ptr(self.csc_val), self.sparse_cap, _ptr(self.nnz))
+
+
+def tail_capacity(rows: int, cols: int, alpha: float) -> int:
+    """2 * n_tail: the guaranteed bound on the number of residual entries."""
+    if alpha >= 1.0:
+        return 0
+    import math
+    return 2 * int(math.floor((1.0 - alpha) * rows * cols + 0.5))
+
+
+def fp4_quantize(ctx: Context, x: torch.Tensor, scale_axis: int, alpha: float = 1.0, prescale=None,
+                 codes: bool = True, codes_t: bool = True, out: QTensor | None = None) -> QTensor:
+    assert x.dtype == torch.bfloat16 and x.is_cuda and x.is_contiguous() and x.dim() == 2
+    rows, cols = x.shape
+    if out is None:
+        out = QTensor(rows, cols, scale_axis, x.device, tail_capacity(rows, cols, alpha), codes, codes_t)
+    _check(ctx.lib.fp4_quantize(ctx.handle, _stream(), _ptr(x), rows, cols, scale_axis, float(alpha),
+                                _ptr(prescale), C.byref(out.struct), _ptr(ctx.status)))
+    return out
+
+
+def fp4_gemm(ctx: Context, a_codes: torch.Tensor, b_codes: torch.Tensor, row_amax=None, col_amax=None,
+             out_f32: bool = True, gemm_kind: int = FP4_GEMM_MXF4, out: torch.Tensor | None = None):
+    I, c2 = a_codes.shape
+    J = b_codes.shape[0]
+    assert b_codes.shape[1] == c2
+    if out is None:
+        out = torch.empty((I, J), dtype=torch.float32 if out_f32 else torch.bfloat16, device=a_codes.device)
+    _check(ctx.lib.fp4_gemm(ctx.handle, _stream(), _ptr(a_codes), _ptr(b_codes), I, J, 2 * c2, _ptr(row_amax),
+                            _ptr(col_amax), _ptr(out), int(out_f32), gemm_kind, _ptr(ctx.status)))
+    return out
+
+
+def fp4_linear_fwd(ctx: Context, A: torch.Tensor, W: torch.Tensor, alpha: float, saved_a: QTensor | None = None,
+                   saved_w: QTensor | None = None, reuse_w: bool = False, gemm_kind: int = FP4_GEMM_MXF4,
+                   out_f32: bool = False, out: torch.Tensor | None = None):
+    M, K = A.shape
+    K2, N = W.shape
+    assert K == K2 and A.dtype == torch.bfloat16 and W.dtype == torch.bfloat16
+    if saved_a is None:
+        saved_a = QTensor(M, K, 0, A.device, tail_capacity(M, K, alpha))
+    if saved_w is None:
+        saved_w = QTensor(K, N, 1, A.device)
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float32 if out_f32 else torch.bfloat16, device=A.device)
+    _check(ctx.lib.fp4_linear_fwd(ctx.handle, _stream(), _ptr(A), _ptr(W), M, K, N, float(alpha), int(reuse_w),
+                                  gemm_kind, _ptr(out), int(out_f32), C.byref(saved_a.struct),
+                                  C.byref(saved_w.struct), _ptr(ctx.status)))
+    return out, saved_a, saved_w
+
+
+def fp4_linear_bwd(ctx: Context, dY: torch.Tensor, W: torch.Tensor, saved_a: QTensor, saved_w: QTensor,
+                   dge_on: bool = True, dge_k: float = 5.0, dge_clip: float = 3.0,
+                   gemm_kind: int = FP4_GEMM_MXF4, out_f32: bool = False, dA=None, dW=None,
+                   want_da: bool = True, want_dw: bool = True):
+    M, N = dY.shape
+    K = W.shape[0]
+    dt = torch.float32 if out_f32 else torch.bfloat16
+    if dA is None and want_da:
+        dA = torch.empty((M, K), dtype=dt, device=dY.device)
+    if dW is None and want_dw:
+        dW = torch.empty((K, N), dtype=dt, device=dY.device)
+    _check(ctx.lib.fp4_linear_bwd(ctx.handle, _stream(), _ptr(dY), _ptr(W), C.byref(saved_a.struct),
+                                  C.byref(saved_w.struct), M, K, N, int(dge_on), float(dge_k), float(dge_clip),
+                                  gemm_kind, _ptr(dA), _ptr(dW), int(out_f32), _ptr(ctx.status)))
+    return dA, dW

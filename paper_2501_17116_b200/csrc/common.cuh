@@ -1,0 +1,65 @@
+// Shared declarations of the CUDA sources (internal; the public ABI is include/fp4_linear.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "fp4_linear.h"
+
+struct fp4_ctx {
+  int      device;
+  int      num_sms;
+  char*    workspace;
+  size_t   workspace_bytes;
+  void*    encode_tiled;       // cuTensorMapEncodeTiled, fetched through the runtime
+};
+
+#define FP4_CUDA_TRY(expr)                         \
+  do {                                             \
+    cudaError_t e__ = (expr);                      \
+    if (e__ != cudaSuccess) return FP4_ERR_CUDA;   \
+  } while (0)
+
+// Bump allocator over the context's workspace; every block is 256-byte aligned.
+struct Arena {
+  char*  base;
+  size_t size;
+  size_t off = 0;
+  bool   ok = true;
+  Arena(char* b, size_t s) : base(b), size(s) {}
+  template <typename T>
+  T* take(size_t count) {
+    size_t bytes = (count * sizeof(T) + 255) & ~size_t(255);
+    if (off + bytes > size) { ok = false; return nullptr; }
+    T* p = reinterpret_cast<T*>(base + off);
+    off += bytes;
+    return p;
+  }
+};
+
+// ---- internal launchers (each enqueues on `stream`, returns an FP4_* host code) -------------
+
+// out[i,j] = (sum_c a[i,c] b[j,c]) * (row_amax[i]/6) * (col_amax[j]/6)
+int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, const uint8_t* b_codes,
+                    int64_t I, int64_t J, int64_t C, const float* row_amax, const float* col_amax,
+                    void* out, int out_f32, int gemm_kind, int32_t* status);
+
+// Quantiser pieces (quantize.cu)
+// `prescale_is_amax`: the prescale vector holds amax values and stands for amax / 6.
+size_t quantize_scratch_bytes(int64_t rows, int64_t cols);
+int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void* x_bf16, int64_t rows,
+                    int64_t cols, int scale_axis, double alpha, const float* prescale,
+                    int prescale_is_amax, fp4_qtensor* out, int32_t* status);
+
+// Sparse compensation and epilogues (compensate.cu)
+// y[m,:] = store( y1[m,:] + sum_{entries of row m} val * dense[col,:] )
+int launch_comp_fwd(fp4_ctx* ctx, cudaStream_t stream, const float* y1, const int32_t* rowptr,
+                    const int32_t* col, const float* val, const void* w_bf16, int64_t M, int64_t K,
+                    int64_t N, void* y, int out_f32);
+// dw[k,:] = store( (s[k,:] + sum_{entries of column k} val * dy[row,:]) * Q'(w[k,:] * gamma[:]) )
+int launch_comp_wgrad_dge(fp4_ctx* ctx, cudaStream_t stream, const float* s, const int32_t* colptr,
+                          const int32_t* row, const float* val, const void* dy_bf16,
+                          const void* w_bf16, const float* w_amax, int64_t M, int64_t K, int64_t N,
+                          int dge_on, float dge_k, float dge_clip, void* dw, int out_f32);

@@ -1,0 +1,151 @@
+// Outlier compensation (Section 3.2: the sparse residual times a dense high-precision matrix)
+// fused with the final store, and the DGE factor of the weight gradient (Eq. 6, Eq. 8).
+//
+//   forward   Y[m, :]  = store( Y1[m, :] + sum_{(m,k) in dA} dA[m,k] * W[k, :] )
+//   wgrad     dW[k, :] = store( (S[k, :] + sum_{(m,k) in dA} dA[m,k] * dY[m, :]) * Q'(W[k,:] * gamma[:]) )
+//
+// Both are "sparse row times dense BF16 matrix" with fp32 accumulation on the plain ALUs: a warp
+// owns one output row and 256 of its columns (8 per lane); the sparse entries of that row (CSR
+// for the forward, CSC for the weight gradient) are walked in order, so the result is
+// deterministic.  The FP4 branch and the compensation meet in fp32 and are rounded once.
+#include "common.cuh"
+
+namespace {
+
+constexpr int COMP_THREADS = 256;          // 8 warps = 8 output rows per block
+constexpr int COMP_COLS = 256;             // columns per block (8 per lane)
+
+__device__ __forceinline__ void fma8(float (&acc)[8], float v, const uint4& d) {
+  const uint32_t w[4] = {d.x, d.y, d.z, d.w};
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    acc[2 * q] = fmaf(v, __uint_as_float(w[q] << 16), acc[2 * q]);
+    acc[2 * q + 1] = fmaf(v, __uint_as_float(w[q] & 0xFFFF0000u), acc[2 * q + 1]);
+  }
+}
+
+__device__ __forceinline__ void store8(void* out, int out_f32, long long off, const float (&y)[8]) {
+  if (out_f32) {
+    float4* dst = reinterpret_cast<float4*>(static_cast<float*>(out) + off);
+    dst[0] = make_float4(y[0], y[1], y[2], y[3]);
+    dst[1] = make_float4(y[4], y[5], y[6], y[7]);
+  } else {
+    uint32_t w[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      __nv_bfloat162 h = __floats2bfloat162_rn(y[2 * q], y[2 * q + 1]);
+      w[q] = *reinterpret_cast<uint32_t*>(&h);
+    }
+    *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(out) + off) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
+// acc[0..7] += sum over the entries [e0, e1) of val[e] * dense[idx[e], col .. col+7]
+__device__ __forceinline__ void sparse_row_times_dense(float (&acc)[8], const int* __restrict__ idx,
+                                                       const float* __restrict__ val, int e0, int e1,
+                                                       const uint4* __restrict__ dense, int vec_per_row, int vcol) {
+  int e = e0;
+  for (; e + 4 <= e1; e += 4) {                 // four independent loads in flight
+    int r[4];
+    float v[4];
+    uint4 d[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      r[u] = __ldg(&idx[e + u]);
+      v[u] = __ldg(&val[e + u]);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) d[u] = __ldg(&dense[(long long)r[u] * vec_per_row + vcol]);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) fma8(acc, v[u], d[u]);
+  }
+  for (; e < e1; ++e) {
+    const uint4 d = __ldg(&dense[(long long)__ldg(&idx[e]) * vec_per_row + vcol]);
+    fma8(acc, __ldg(&val[e]), d);
+  }
+}
+
+__global__ void __launch_bounds__(COMP_THREADS)
+comp_fwd_kernel(const float* __restrict__ y1, const int* __restrict__ rowptr, const int* __restrict__ col,
+                const float* __restrict__ val, const uint4* __restrict__ w, int M, int N, void* y, int out_f32) {
+  const int m = blockIdx.y * 8 + (threadIdx.x >> 5);
+  const int n0 = blockIdx.x * COMP_COLS + 8 * (threadIdx.x & 31);
+  if (m >= M || n0 >= N) return;
+  float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  sparse_row_times_dense(acc, col, val, rowptr[m], rowptr[m + 1], w, N >> 3, n0 >> 3);
+  const long long off = (long long)m * N + n0;
+  const float4 a = *reinterpret_cast<const float4*>(y1 + off);
+  const float4 b = *reinterpret_cast<const float4*>(y1 + off + 4);
+  const float y8[8] = {a.x + acc[0], a.y + acc[1], a.z + acc[2], a.w + acc[3],
+                       b.x + acc[4], b.y + acc[5], b.z + acc[6], b.w + acc[7]};
+  store8(y, out_f32, off, y8);
+}
+
+// DGE derivative of Eq. 8 on a scaled weight, capped at `clip`.  The E2M1 grid has steps of 0.5
+// below 2, 1 on [2, 4) and 2 from 4 up; u = 2 (|w| - g) / delta - 1 is the position inside the
+// interval [g, g + delta] mapped to [-1, 1].
+__device__ __forceinline__ float dge_factor(float ws, float expo, float inv_k, float clip) {
+  const float a = fabsf(ws);
+  float g, two_over_delta;
+  if (a < 2.0f) { g = 0.5f * floorf(2.0f * a); two_over_delta = 4.0f; }
+  else if (a < 4.0f) { g = floorf(a); two_over_delta = 2.0f; }
+  else { g = 4.0f; two_over_delta = 1.0f; }
+  const float u = fabsf((a - g) * two_over_delta - 1.0f);
+  // |u|^(1/k - 1) = 2^((1/k - 1) log2 |u|); u = 0 gives +inf, which the cap turns into `clip`
+  const float d = inv_k * exp2f(expo * __log2f(u));
+  return fminf(d, clip);
+}
+
+__global__ void __launch_bounds__(COMP_THREADS)
+comp_wgrad_dge_kernel(const float* __restrict__ s, const int* __restrict__ colptr, const int* __restrict__ row,
+                      const float* __restrict__ val, const uint4* __restrict__ dy, const uint4* __restrict__ w,
+                      const float* __restrict__ w_amax, int K, int N, int dge_on, float dge_k, float dge_clip,
+                      void* dw, int out_f32) {
+  const int k = blockIdx.y * 8 + (threadIdx.x >> 5);
+  const int n0 = blockIdx.x * COMP_COLS + 8 * (threadIdx.x & 31);
+  if (k >= K || n0 >= N) return;
+  float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  if (colptr) sparse_row_times_dense(acc, row, val, colptr[k], colptr[k + 1], dy, N >> 3, n0 >> 3);
+  const long long off = (long long)k * N + n0;
+  const float4 a = *reinterpret_cast<const float4*>(s + off);
+  const float4 b = *reinterpret_cast<const float4*>(s + off + 4);
+  float y8[8] = {a.x + acc[0], a.y + acc[1], a.z + acc[2], a.w + acc[3],
+                 b.x + acc[4], b.y + acc[5], b.z + acc[6], b.w + acc[7]};
+  if (dge_on) {
+    const uint4 wv = __ldg(&w[off >> 3]);
+    const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
+    const float inv_k = 1.0f / dge_k;
+    const float expo = inv_k - 1.0f;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      const float wf = __uint_as_float((c & 1) ? (ww[c >> 1] & 0xFFFF0000u) : (ww[c >> 1] << 16));
+      const float amax = __ldg(&w_amax[n0 + c]);
+      const float gamma = amax > 0.0f ? __fdiv_rn(6.0f, amax) : 0.0f;
+      const float ws = __fmul_rn(wf, gamma);          // the value the forward quantised
+      y8[c] *= dge_factor(ws, expo, inv_k, dge_clip);
+    }
+  }
+  store8(dw, out_f32, off, y8);
+}
+
+}  // namespace
+
+int launch_comp_fwd(fp4_ctx*, cudaStream_t stream, const float* y1, const int32_t* rowptr, const int32_t* col,
+                    const float* val, const void* w_bf16, int64_t M, int64_t, int64_t N, void* y, int out_f32) {
+  const dim3 grid(unsigned((N + COMP_COLS - 1) / COMP_COLS), unsigned((M + 7) / 8));
+  comp_fwd_kernel<<<grid, COMP_THREADS, 0, stream>>>(y1, rowptr, col, val, static_cast<const uint4*>(w_bf16), int(M),
+                                                     int(N), y, out_f32);
+  FP4_CUDA_TRY(cudaGetLastError());
+  return FP4_OK;
+}
+
+int launch_comp_wgrad_dge(fp4_ctx*, cudaStream_t stream, const float* s, const int32_t* colptr, const int32_t* row,
+                          const float* val, const void* dy_bf16, const void* w_bf16, const float* w_amax, int64_t,
+                          int64_t K, int64_t N, int dge_on, float dge_k, float dge_clip, void* dw, int out_f32) {
+  const dim3 grid(unsigned((N + COMP_COLS - 1) / COMP_COLS), unsigned((K + 7) / 8));
+  comp_wgrad_dge_kernel<<<grid, COMP_THREADS, 0, stream>>>(s, colptr, row, val, static_cast<const uint4*>(dy_bf16),
+                                                           static_cast<const uint4*>(w_bf16), w_amax, int(K), int(N),
+                                                           dge_on, dge_k, dge_clip, dw, out_f32);
+  FP4_CUDA_TRY(cudaGetLastError());
+  return FP4_OK;
+}

@@ -1,0 +1,443 @@
+// FP4 GEMM on the 5th-generation tensor cores (tcgen05.mma) for sm_100a.
+//
+//   out[i, j] = ( sum_c val(a[i, c]) * val(b[j, c]) ) * (row_amax[i] / 6) * (col_amax[j] / 6)
+//
+// Both operands are E2M1 nibbles with the contraction contiguous ("K-major"), which is the
+// form of all three GEMMs of the layer (Fig. 2; Eq. 3; Appendix C.2).  The two de-scales are
+// applied to the accumulators in the epilogue, after the GEMM, as Appendix C.2 prescribes.
+//
+// Structure: persistent CTAs (one per SM), 128 x 256 output tile per CTA, six warps:
+//   warp 0      TMA producer: cp.async.bulk.tensor loads into 128-byte-swizzled shared memory,
+//               a ring of STAGES stages guarded by full/empty mbarriers;
+//   warp 1      allocates tensor memory and issues tcgen05.mma from one thread, fp32
+//               accumulators in tensor memory; tcgen05.commit releases stages and publishes tiles;
+//   warps 2..5  epilogue: tcgen05.ld the accumulators (one row per thread), de-scale, store.
+// Two MMA flavours are compiled:
+//   MXF4    kind::mxf4.block_scale, packed nibbles, K = 64 per instruction.  The method has no
+//           block scales, so every UE8M0 scale in tensor memory is 2^0: the product is unchanged.
+//   F8F6F4  kind::f8f6f4, TMA expands the packed nibbles to one per byte-container group
+//           (16 nibbles + 8 bytes of padding), K = 32 per instruction.
+// Every wait is bounded: on a timeout the CTA raises FP4_DEV_TIMEOUT, drains its own copies,
+// frees its tensor memory and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BN = 256;
+constexpr int STAGES = 4;
+constexpr int A_STAGE_BYTES = BM * 128;
+constexpr int B_STAGE_BYTES = BN * 128;
+constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int NUM_THREADS = 192;
+constexpr int TMEM_COLS = 512;
+constexpr int SF_COL_A = 256;            // MXF4 only: unit block scales live past the accumulator
+constexpr int SF_COL_B = 288;
+constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
+constexpr size_t SMEM_BYTES = 1024 + size_t(STAGES) * STAGE_BYTES + 256;
+
+struct GemmArgs {
+  int I, J;
+  int num_k_blocks;
+  int num_m_blocks, num_n_blocks;
+  uint32_t tx_bytes;
+  const float* row_amax;
+  const float* col_amax;
+  void* out;
+  int out_f32;
+  int32_t* status;
+};
+
+// ------------------------------------------------------------------ PTX wrappers ------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the wait ran out or another role already gave up.
+__device__ __noinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                       int32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  uint32_t spins = 0;
+  for (;;) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((++spins & 31u) == 0u) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > WAIT_LIMIT_NS) {
+        *abort_flag = 1;
+        atomicOr(status, FP4_DEV_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void mma_f8f6f4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                           uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void mma_mxf4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                         uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%4], [%5], p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate)
+      : "memory");
+}
+// 32 lanes x 32 consecutive columns of 32-bit cells: thread t gets row t of the warp's lane quarter.
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_32x8(uint32_t taddr, uint32_t x) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1};" ::"r"(taddr), "r"(x)
+               : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes, 128-byte swizzle:
+// 8-row groups are 1024 bytes apart (stride offset); the leading offset is unused in this mode.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= uint64_t((smem_addr & 0x3FFFFu) >> 4);
+  d |= uint64_t(1) << 16;
+  d |= uint64_t(1024 >> 4) << 32;
+  d |= uint64_t(1) << 46;   // descriptor version of this architecture
+  d |= uint64_t(2) << 61;   // 128-byte swizzle
+  return d;
+}
+// Instruction descriptors: M = 128, N = BN, both operands K-major, E2M1 x E2M1 -> fp32.
+__host__ __device__ constexpr uint32_t idesc_f8f6f4() {
+  return (1u << 4) | (5u << 7) | (5u << 10) | (uint32_t(BN >> 3) << 17) | (uint32_t(BM >> 4) << 24);
+}
+__host__ __device__ constexpr uint32_t idesc_mxf4() {
+  return (1u << 7) | (1u << 10) | (uint32_t(BN >> 3) << 17) | (1u << 23) | (uint32_t(BM >> 4) << 24);
+}
+
+template <int KIND>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                const GemmArgs args) {
+  constexpr int NACC = (KIND == FP4_GEMM_F8F6F4) ? 2 : 1;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* smem_a = smem;
+  uint8_t* smem_b = smem + STAGES * A_STAGE_BYTES;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+  uint64_t* empty_bar = full_bar + STAGES;
+  uint64_t* acc_full = empty_bar + STAGES;
+  uint64_t* acc_empty = acc_full + 2;
+  uint64_t* final_bar = acc_empty + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(final_bar + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int num_tiles = args.num_m_blocks * args.num_n_blocks;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(&acc_full[a], 1);
+      mbar_init(&acc_empty[a], 4);
+    }
+    mbar_init(final_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (KIND == FP4_GEMM_MXF4) {
+    // Unit block scales: every byte of the scale columns is 0x7F (UE8M0 2^0), so the layout the
+    // instruction expects inside these columns does not matter.
+    if (warp >= 2) {
+      const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
+      for (int c = 0; c < 64; c += 8) tmem_st_32x8(tmem_base + lane_base + SF_COL_A + c, 0x7F7F7F7Fu);
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+  }
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer -------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      uint32_t fills = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+        const int m_blk = t % args.num_m_blocks;
+        const int n_blk = t / args.num_m_blocks;
+        for (int kb = 0; kb < args.num_k_blocks; ++kb) {
+          ok = mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, args.status);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&full_bar[stage], args.tx_bytes);
+          tma_load_2d(smem_a + stage * A_STAGE_BYTES, &map_a, &full_bar[stage], kb * 128, m_blk * BM);
+          tma_load_2d(smem_b + stage * B_STAGE_BYTES, &map_b, &full_bar[stage], kb * 128, n_blk * BN);
+          ++fills;
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // Gave up: let the copies already in flight land before shared memory is released.
+        const uint32_t last = fills < uint32_t(STAGES) ? fills : uint32_t(STAGES);
+        for (uint32_t back = 1; back <= last; ++back) {
+          const uint32_t f = fills - back;                 // global index of that fill
+          const uint64_t t0 = global_timer_ns();
+          while (!mbar_try_wait(&full_bar[f % STAGES], (f / STAGES) & 1u)) {
+            if (global_timer_ns() - t0 > 1000000ull) break;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer ---------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      const uint32_t idesc = (KIND == FP4_GEMM_F8F6F4) ? idesc_f8f6f4() : idesc_mxf4();
+      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+        ok = mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, args.status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + uint32_t(acc * BN);
+        for (int kb = 0; kb < args.num_k_blocks; ++kb) {
+          ok = mbar_wait(&full_bar[stage], phase, abort_flag, args.status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t a_desc = make_smem_desc(smem_u32(smem_a + stage * A_STAGE_BYTES));
+          const uint64_t b_desc = make_smem_desc(smem_u32(smem_b + stage * B_STAGE_BYTES));
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            // 32 bytes of the swizzled 128-byte row per instruction: +2 in the (>>4) address field
+            const uint32_t accumulate = (kb | k) != 0 ? 1u : 0u;
+            if (KIND == FP4_GEMM_F8F6F4) {
+              mma_f8f6f4(d_tmem, a_desc + uint64_t(2 * k), b_desc + uint64_t(2 * k), idesc, accumulate);
+            } else {
+              mma_mxf4(d_tmem, a_desc + uint64_t(2 * k), b_desc + uint64_t(2 * k), idesc, tmem_base + SF_COL_A,
+                       tmem_base + SF_COL_B, accumulate);
+            }
+          }
+          tc_commit(&empty_bar[stage]);       // frees the stage once these MMAs have read it
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(&acc_full[acc]);            // accumulators of this tile are complete
+        if (++acc == NACC) { acc = 0; acc_phase ^= 1u; }
+      }
+      // All MMAs issued by this thread must have retired before tensor memory is freed.
+      tc_commit(final_bar);
+      const uint64_t t0 = global_timer_ns();
+      while (!mbar_try_wait(final_bar, 0)) {
+        if (global_timer_ns() - t0 > WAIT_LIMIT_NS) {
+          atomicOr(args.status, FP4_DEV_TIMEOUT);
+          break;
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue -----------
+    const int quarter = warp & 3;               // the lane quarter of tensor memory this warp may read
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
+      const int m_blk = t % args.num_m_blocks;
+      const int n_blk = t / args.num_m_blocks;
+      bool ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, args.status);
+      ok = __all_sync(0xFFFFFFFFu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const int row = m_blk * BM + quarter * 32 + lane;
+      const float d_row = args.row_amax ? __fdiv_rn(args.row_amax[row], 6.0f) : 1.0f;
+#pragma unroll 1
+      for (int chunk = 0; chunk < BN / 32; ++chunk) {
+        const int col0 = n_blk * BN + chunk * 32;
+        if (col0 >= args.J) break;                // warp-uniform: ragged last tile in N
+        uint32_t v[32];
+        tmem_ld_32x32(tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * BN + chunk * 32), v);
+        const float d_col_lane = args.col_amax ? __fdiv_rn(args.col_amax[col0 + lane], 6.0f) : 1.0f;
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        float y[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float d_col = __shfl_sync(0xFFFFFFFFu, d_col_lane, j);
+          y[j] = __fmul_rn(__fmul_rn(__uint_as_float(v[j]), d_row), d_col);
+        }
+        const size_t off = size_t(row) * size_t(args.J) + size_t(col0);
+        if (args.out_f32) {
+          float4* dst = reinterpret_cast<float4*>(static_cast<float*>(args.out) + off);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) dst[j] = make_float4(y[4 * j], y[4 * j + 1], y[4 * j + 2], y[4 * j + 3]);
+        } else {
+          uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(args.out) + off);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            uint32_t w[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              __nv_bfloat162 h = __floats2bfloat162_rn(y[8 * j + 2 * q], y[8 * j + 2 * q + 1]);
+              w[q] = *reinterpret_cast<uint32_t*>(&h);
+            }
+            dst[j] = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[acc]);
+      if (++acc == NACC) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// Tensor map over packed codes [rows x C/2 bytes] with a box of 128 bytes x box_rows.
+int make_codes_map(fp4_ctx* ctx, CUtensorMap* map, const uint8_t* codes, int64_t rows, int64_t C, int box_rows,
+                   int gemm_kind) {
+  EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
+  if (!encode) return FP4_ERR_CUDA;
+  const cuuint64_t strides[1] = {cuuint64_t(C / 2)};
+  const cuuint32_t elem_strides[2] = {1, 1};
+  CUresult r;
+  if (gemm_kind == FP4_GEMM_F8F6F4) {
+    // global memory packed, shared memory 16 nibbles + 8 bytes of padding per 16 bytes
+    const cuuint64_t dims[2] = {cuuint64_t(C), cuuint64_t(rows)};
+    const cuuint32_t box[2] = {128, cuuint32_t(box_rows)};
+    r = encode(map, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, 2, const_cast<uint8_t*>(codes), dims, strides, box,
+               elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else {
+    const cuuint64_t dims[2] = {cuuint64_t(C / 2), cuuint64_t(rows)};
+    const cuuint32_t box[2] = {128, cuuint32_t(box_rows)};
+    r = encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(codes), dims, strides, box, elem_strides,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  }
+  return r == CUDA_SUCCESS ? FP4_OK : FP4_ERR_CUDA;
+}
+
+}  // namespace
+
+int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, const uint8_t* b_codes, int64_t I,
+                    int64_t J, int64_t C, const float* row_amax, const float* col_amax, void* out, int out_f32,
+                    int gemm_kind, int32_t* status) {
+  if (gemm_kind != FP4_GEMM_MXF4 && gemm_kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;
+  // The byte-container form expands 32 bytes of a packed row into 64, so its rows must start on
+  // 32-byte boundaries (C/2 a multiple of 32 holds for every multiple of 128).
+  const uintptr_t need = gemm_kind == FP4_GEMM_F8F6F4 ? 31 : 15;
+  if ((reinterpret_cast<uintptr_t>(a_codes) & need) || (reinterpret_cast<uintptr_t>(b_codes) & need))
+    return FP4_ERR_ALIGN;
+  CUtensorMap map_a, map_b;
+  int rc = make_codes_map(ctx, &map_a, a_codes, I, C, BM, gemm_kind);
+  if (rc != FP4_OK) return rc;
+  rc = make_codes_map(ctx, &map_b, b_codes, J, C, BN, gemm_kind);
+  if (rc != FP4_OK) return rc;
+
+  GemmArgs args;
+  args.I = int(I);
+  args.J = int(J);
+  const int k_per_stage = gemm_kind == FP4_GEMM_F8F6F4 ? 128 : 256;   // elements per 128-byte row
+  args.num_k_blocks = int((C + k_per_stage - 1) / k_per_stage);
+  args.num_m_blocks = int(I / BM);
+  args.num_n_blocks = int((J + BN - 1) / BN);
+  // The transaction count of a copy is in bytes read from global memory: the byte-container form
+  // fills a 48 KB stage from 24 KB of packed nibbles.
+  args.tx_bytes = gemm_kind == FP4_GEMM_F8F6F4 ? STAGE_BYTES / 2 : STAGE_BYTES;
+  args.row_amax = row_amax;
+  args.col_amax = col_amax;
+  args.out = out;
+  args.out_f32 = out_f32;
+  args.status = status;
+  const int tiles = args.num_m_blocks * args.num_n_blocks;
+  const int grid = tiles < ctx->num_sms ? tiles : ctx->num_sms;
+
+  if (gemm_kind == FP4_GEMM_F8F6F4) {
+    FP4_CUDA_TRY(cudaFuncSetAttribute(gemm_fp4_kernel<FP4_GEMM_F8F6F4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      int(SMEM_BYTES)));
+    gemm_fp4_kernel<FP4_GEMM_F8F6F4><<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(map_a, map_b, args);
+  } else {
+    FP4_CUDA_TRY(cudaFuncSetAttribute(gemm_fp4_kernel<FP4_GEMM_MXF4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      int(SMEM_BYTES)));
+    gemm_fp4_kernel<FP4_GEMM_MXF4><<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(map_a, map_b, args);
+  }
+  FP4_CUDA_TRY(cudaGetLastError());
+  return FP4_OK;
+}

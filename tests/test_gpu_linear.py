@@ -1,0 +1,135 @@
+"""GPU parity of fp4_linear_fwd / fp4_linear_bwd against the oracle.
+
+Tolerance (fp32-accumulated results against the double oracle): an output that is the sum of
+an FP4 branch and a compensation branch must satisfy
+    |gpu - oracle| <= 1e-3 * (|fp4 branch| + |compensation branch|)
+in float output mode.  In BF16 output mode the stored value must be the BF16 rounding of the
+oracle value, or a neighbouring BF16 number where the oracle value lies within 1e-3 (relative)
+of a rounding boundary.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import fp4_oracle as O
+from paper_2501_17116_b200 import workloads as WL
+
+pytestmark = pytest.mark.gpu
+RTOL = 1e-3
+
+
+@pytest.fixture(scope="module")
+def ctx(lib):
+    c = lib.Context(0, 1 << 30)
+    yield c
+    c.close()
+
+
+def _dev(bits):
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def assert_close_f32(got, want, branch_a, branch_b=None, what=""):
+    scale = np.abs(branch_a) + (0 if branch_b is None else np.abs(branch_b))
+    err = np.abs(got.astype(np.float64) - want)
+    bad = err > RTOL * scale + 1e-300
+    assert not bad.any(), f"{what}: {bad.sum()} of {bad.size} outside tolerance, worst {np.max(err / (scale + 1e-300))}"
+
+
+def assert_bf16_rounding(got_bf16: torch.Tensor, want, what=""):
+    got = got_bf16.float().cpu().numpy().astype(np.float64)
+    r = O.f64_to_bf16_f64(want)
+    exact = got == r
+    # a neighbouring BF16 value is accepted only if the oracle value is within RTOL of the midpoint
+    near = np.abs(got - want) <= np.abs(r - want) + RTOL * np.abs(want)
+    ok = exact | near
+    assert ok.all(), f"{what}: {np.sum(~ok)} of {ok.size} values are not the BF16 rounding of the oracle"
+    assert exact.mean() > 0.99, f"{what}: only {exact.mean():.4f} match the rounding exactly"
+
+
+def _saved_matches(sa, sw, f: O.Forward):
+    np.testing.assert_array_equal(sa.codes.cpu().numpy(), f.qa.packed())
+    np.testing.assert_array_equal(sa.codes_t.cpu().numpy(), f.qa.packed_t())
+    np.testing.assert_array_equal(sa.amax.cpu().numpy(), f.qa.amax)
+    np.testing.assert_array_equal(sw.codes.cpu().numpy(), f.qw.packed())
+    np.testing.assert_array_equal(sw.codes_t.cpu().numpy(), f.qw.packed_t())
+    np.testing.assert_array_equal(sw.amax.cpu().numpy(), f.qw.amax)
+
+
+CASES = [
+    # M, K, N, alpha, gemm kind
+    (128, 128, 128, 0.99, 0),
+    (256, 384, 640, 0.97, 0),
+    (384, 640, 384, 0.999, 1),
+    (128, 256, 128, 1.0, 0),
+    (256, 1152, 256, 0.99, 1),
+]
+
+
+@pytest.mark.parametrize("M,K,N,alpha,kind", CASES)
+def test_forward_and_backward_match_oracle(lib, ctx, M, K, N, alpha, kind):
+    a_bits, w_bits, dy_bits = WL.small_case(M, K, N, seed=M + K + N)
+    f = O.linear_fwd(a_bits, w_bits, alpha)
+    b = O.linear_bwd(dy_bits, w_bits, f)
+    A, W, dY = _dev(a_bits), _dev(w_bits), _dev(dy_bits)
+    ctx.status.zero_()
+    y32, sa, sw = lib.fp4_linear_fwd(ctx, A, W, alpha, gemm_kind=kind, out_f32=True)
+    da32, dw32 = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, gemm_kind=kind, out_f32=True)
+    y16, _, _ = lib.fp4_linear_fwd(ctx, A, W, alpha, gemm_kind=kind)
+    da16, dw16 = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, gemm_kind=kind)
+    torch.cuda.synchronize()
+    assert ctx.read_status() == 0
+    _saved_matches(sa, sw, f)
+    assert_close_f32(y32.cpu().numpy(), f.y, f.y_fp4, f.y_comp, "Y")
+    assert_close_f32(da32.cpu().numpy(), b.da, b.da, None, "dA")
+    assert_close_f32(dw32.cpu().numpy(), b.dw, b.s_fp4 * b.dge, b.s_comp * b.dge, "dW")
+    assert_bf16_rounding(y16, f.y, "Y")
+    assert_bf16_rounding(da16, b.da, "dA")
+    assert_bf16_rounding(dw16, b.dw, "dW")
+
+
+def test_ste_switch_and_dge_parameters(lib, ctx):
+    a_bits, w_bits, dy_bits = WL.small_case(128, 256, 128, seed=21)
+    f = O.linear_fwd(a_bits, w_bits, 0.99)
+    A, W, dY = _dev(a_bits), _dev(w_bits), _dev(dy_bits)
+    _, sa, sw = lib.fp4_linear_fwd(ctx, A, W, 0.99)
+    for dge_on, k, clip in ((False, 5.0, 3.0), (True, 3.0, 2.0), (True, 7.0, 10.0)):
+        b = O.linear_bwd(dy_bits, w_bits, f, dge_on=dge_on, k=k, clip=clip)
+        _, dw = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, dge_on=dge_on, dge_k=k, dge_clip=clip, out_f32=True,
+                                   want_da=False)
+        torch.cuda.synchronize()
+        assert_close_f32(dw.cpu().numpy(), b.dw, b.s_fp4 * b.dge, b.s_comp * b.dge, f"dW dge={dge_on} k={k}")
+
+
+def test_reuse_quantised_weight(lib, ctx):
+    a_bits, w_bits, _ = WL.small_case(128, 256, 256, seed=5)
+    a2_bits, _, _ = WL.small_case(128, 256, 256, seed=6)
+    W = _dev(w_bits)
+    y1, sa, sw = lib.fp4_linear_fwd(ctx, _dev(a_bits), W, 0.99)
+    y2, _, _ = lib.fp4_linear_fwd(ctx, _dev(a2_bits), W, 0.99, saved_w=sw, reuse_w=True)
+    y2_fresh, _, _ = lib.fp4_linear_fwd(ctx, _dev(a2_bits), W, 0.99)
+    torch.cuda.synchronize()
+    assert torch.equal(y2, y2_fresh)
+
+
+def test_config0_full_layer(lib, ctx):
+    """The small configuration in full: X[256 x 1024] with 8 outlier channels, alpha = 0.99, DGE on."""
+    cfg = WL.CONFIGS[0]
+    a_bits = WL.activations(cfg, 1024)
+    w_bits = WL.weights(cfg, 1024, 1024)
+    dy_bits = WL.output_grads(cfg, 1024)
+    f = O.linear_fwd(a_bits, w_bits, 0.99)
+    b = O.linear_bwd(dy_bits, w_bits, f)
+    A, W, dY = _dev(a_bits), _dev(w_bits), _dev(dy_bits)
+    for kind in (0, 1):
+        ctx.status.zero_()
+        y32, sa, sw = lib.fp4_linear_fwd(ctx, A, W, 0.99, gemm_kind=kind, out_f32=True)
+        da32, dw32 = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, gemm_kind=kind, out_f32=True)
+        y16, _, _ = lib.fp4_linear_fwd(ctx, A, W, 0.99, gemm_kind=kind)
+        torch.cuda.synchronize()
+        assert ctx.read_status() == 0
+        _saved_matches(sa, sw, f)
+        assert_close_f32(y32.cpu().numpy(), f.y, f.y_fp4, f.y_comp, "Y")
+        assert_close_f32(da32.cpu().numpy(), b.da, b.da, None, "dA")
+        assert_close_f32(dw32.cpu().numpy(), b.dw, b.s_fp4 * b.dge, b.s_comp * b.dge, "dW")
+        assert_bf16_rounding(y16, f.y, "Y")

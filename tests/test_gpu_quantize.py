@@ -1,0 +1,192 @@
+"""GPU parity of fp4_quantize against the oracle: codes (both layouts), amax, thresholds and
+the sparse residual are compared bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import fp4_oracle as O
+from paper_2501_17116_b200 import workloads as WL
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx(lib):
+    c = lib.Context(0, 512 << 20)
+    yield c
+    c.close()
+
+
+def _dev(bits):
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def _check_dense(q, ref: O.Quantized):
+    np.testing.assert_array_equal(q.amax.cpu().numpy(), ref.amax)
+    if q.codes is not None:
+        np.testing.assert_array_equal(q.codes.cpu().numpy(), ref.packed())
+    if q.codes_t is not None:
+        np.testing.assert_array_equal(q.codes_t.cpu().numpy(), ref.packed_t())
+
+
+def _check_sparse(q, ref: O.Quantized):
+    th = q.thresholds.cpu().numpy()
+    assert (float(th[0]), float(th[1])) == (ref.lo, ref.hi)
+    assert not (np.signbit(th) & (th == 0)).any()        # a zero threshold is +0
+    nnz = int(q.nnz.item())
+    rowptr, col, val = ref.csr
+    colptr, row, cval = ref.csc
+    assert nnz == rowptr[-1]
+    np.testing.assert_array_equal(q.csr_rowptr.cpu().numpy(), rowptr)
+    np.testing.assert_array_equal(q.csr_col.cpu().numpy()[:nnz], col)
+    np.testing.assert_array_equal(q.csr_val.cpu().numpy()[:nnz], val)
+    np.testing.assert_array_equal(q.csc_colptr.cpu().numpy(), colptr)
+    np.testing.assert_array_equal(q.csc_row.cpu().numpy()[:nnz], row)
+    np.testing.assert_array_equal(q.csc_val.cpu().numpy()[:nnz], cval)
+
+
+@pytest.mark.parametrize("axis", [0, 1])
+@pytest.mark.parametrize("shape", [(128, 128), (256, 384), (384, 1152), (1024, 640)])
+def test_absmax_quantize_matches_oracle(lib, ctx, axis, shape):
+    rng = np.random.default_rng(shape[0] + shape[1] + axis)
+    bits = WL.to_bf16_bits(rng.standard_normal(shape).astype(np.float32) * np.float32(0.02))
+    bits[3, :] = 0                                    # a zero row: amax 0 when axis == 0
+    bits[:, 5] = 0 if axis == 1 else bits[:, 5]       # a zero column when axis == 1
+    bits[7, 9] = 0x8000                               # negative zero input
+    ctx.status.zero_()
+    q = lib.fp4_quantize(ctx, _dev(bits), axis)
+    torch.cuda.synchronize()
+    assert ctx.read_status() == 0
+    _check_dense(q, O.absmax_quantize(O.bf16_bits_to_f64(bits), axis))
+
+
+@pytest.mark.parametrize("axis", [0, 1])
+def test_prescaled_quantize_matches_oracle(lib, ctx, axis):
+    rng = np.random.default_rng(17 + axis)
+    rows, cols = 256, 384
+    bits = WL.to_bf16_bits(rng.standard_normal((rows, cols)).astype(np.float32) * np.float32(1e-3))
+    p = (rng.random(cols if axis == 0 else rows).astype(np.float32) * 3 + np.float32(0.01))
+    q = lib.fp4_quantize(ctx, _dev(bits), axis, prescale=torch.from_numpy(p).cuda())
+    torch.cuda.synchronize()
+    _check_dense(q, O.absmax_quantize(O.bf16_bits_to_f64(bits), axis, prescale=p))
+
+
+def test_Q_on_chosen_float32_values(lib, ctx):
+    """Drive the encoder with arbitrary float32 inputs: x = 1 and a prescale vector of the probe
+    values; one probe is 6 so that gamma = 1 and the scaled value is the probe itself.  Probes:
+    every threshold of the chain, its float32 neighbours, grid points, zeros, tiny and large."""
+    probes = [6.0]
+    for t in O.LUT_THRESHOLDS:
+        t32 = np.float32(t)
+        probes += [t32, np.nextafter(t32, np.float32(-np.inf)), np.nextafter(t32, np.float32(np.inf)),
+                   np.nextafter(np.nextafter(t32, np.float32(-np.inf)), np.float32(-np.inf)),
+                   np.nextafter(np.nextafter(t32, np.float32(np.inf)), np.float32(np.inf))]
+    probes += list(O.LUT_VALUES) + [0.0, -0.0, 1e-30, -1e-30, 1e-42, -1e-42, 5.9999995, -5.9999995, 0.1, -0.1]
+    rng = np.random.default_rng(3)
+    probes += list(rng.uniform(-6, 6, 384 - len(probes)))
+    p = np.array(probes, dtype=np.float32)
+    assert p.size == 384 and np.abs(p).max() == 6.0
+    ones = np.full((128, 384), 0x3F80, dtype=np.uint16)
+    q = lib.fp4_quantize(ctx, _dev(ones), 0, prescale=torch.from_numpy(p).cuda())
+    torch.cuda.synchronize()
+    got = O.unpack_nibbles(q.codes.cpu().numpy())
+    want = O.lut_quantize(p)
+    np.testing.assert_array_equal(got[0], want)
+    np.testing.assert_array_equal(got, np.broadcast_to(want, got.shape))
+    assert not (got == 8).any()
+
+
+def test_Q_on_every_bf16_value(lib, ctx):
+    """All finite BF16 patterns of magnitude <= 6 in one tensor whose rows all have amax 6."""
+    bits = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    v = O.bf16_bits_to_f64(bits)
+    keep = bits[np.isfinite(v) & (np.abs(v) <= 6.0)]
+    cols = 256
+    rows = -(-keep.size // (cols - 1))
+    rows = -(-rows // 128) * 128
+    x = np.zeros((rows, cols), dtype=np.uint16)
+    x[:, 0] = 0x40C0                                   # 6.0 in every row -> gamma = 1
+    body = np.zeros(rows * (cols - 1), dtype=np.uint16)
+    body[:keep.size] = keep
+    x[:, 1:] = body.reshape(rows, cols - 1)
+    q = lib.fp4_quantize(ctx, _dev(x), 0)
+    torch.cuda.synchronize()
+    _check_dense(q, O.absmax_quantize(O.bf16_bits_to_f64(x), 0))
+
+
+@pytest.mark.parametrize("shape,alpha,dist", [((128, 128), 0.99, "normal"), ((256, 384), 0.97, "student_t3"),
+                                              ((384, 1152), 0.999, "laplace"), ((1024, 640), 0.99, "normal")])
+def test_occ_quantize_matches_oracle(lib, ctx, shape, alpha, dist):
+    cfg = WL.Config(50, "t", shape[0], (), dist, 3, 40.0, "channels_count", (alpha,))
+    bits = WL.activations(cfg, shape[1], seed=1, layer=shape[0])
+    ctx.status.zero_()
+    q = lib.fp4_quantize(ctx, _dev(bits), 0, alpha=alpha)
+    torch.cuda.synchronize()
+    assert ctx.read_status() == 0
+    ref = O.occ_quantize(O.bf16_bits_to_f64(bits), alpha)
+    _check_sparse(q, ref)
+    _check_dense(q, ref)
+
+
+def test_occ_with_heavy_ties_and_zeros(lib, ctx):
+    """Few distinct values: thresholds sit on big ties (entries equal to a threshold carry no
+    residual), one bin holds far more than 2^16 entries, and lo is a zero."""
+    rng = np.random.default_rng(8)
+    vals = np.array([0.0, -0.0, 0.5, 1.0, -1.0, 2.5, -3.0, 64.0], dtype=np.float32)
+    prob = np.array([0.86, 0.05, 0.03, 0.02, 0.005, 0.02, 0.005, 0.01])
+    a = rng.choice(vals, size=(512, 1024), p=prob)
+    bits = WL.to_bf16_bits(a)
+    for alpha in (0.99, 0.97):
+        q = lib.fp4_quantize(ctx, _dev(bits), 0, alpha=alpha)
+        torch.cuda.synchronize()
+        ref = O.occ_quantize(O.bf16_bits_to_f64(bits), alpha)
+        _check_sparse(q, ref)
+        _check_dense(q, ref)
+
+
+def test_config0_activation_and_weight(lib, ctx):
+    cfg = WL.CONFIGS[0]
+    a_bits = WL.activations(cfg, 1024)
+    w_bits = WL.weights(cfg, 1024, 1024)
+    qa = lib.fp4_quantize(ctx, _dev(a_bits), 0, alpha=0.99)
+    qw = lib.fp4_quantize(ctx, _dev(w_bits), 1)
+    torch.cuda.synchronize()
+    ra = O.occ_quantize(O.bf16_bits_to_f64(a_bits), 0.99)
+    assert ra.n_tail == 2621
+    _check_sparse(qa, ra)
+    _check_dense(qa, ra)
+    _check_dense(qw, O.absmax_quantize(O.bf16_bits_to_f64(w_bits), 1))
+    # the bound that sizes the sparse buffers
+    assert int(qa.nnz.item()) <= 2 * ra.n_tail == qa.sparse_cap
+
+
+def test_run_to_run_determinism(lib, ctx):
+    cfg = WL.CONFIGS[0]
+    x = _dev(WL.activations(cfg, 1024))
+    a = lib.fp4_quantize(ctx, x, 0, alpha=0.99)
+    b = lib.fp4_quantize(ctx, x, 0, alpha=0.99)
+    torch.cuda.synchronize()
+    for name in ("codes", "codes_t", "amax", "thresholds", "csr_rowptr", "csr_col", "csr_val", "csc_colptr",
+                 "csc_row", "csc_val", "nnz"):
+        assert torch.equal(getattr(a, name), getattr(b, name)), name
+
+
+def test_host_side_argument_errors(lib, ctx):
+    x = torch.zeros((128, 128), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(lib.Fp4Error) as e:
+        lib.fp4_quantize(ctx, x[:, :64].contiguous(), 0)
+    assert e.value.code == -2                                   # shape
+    with pytest.raises(lib.Fp4Error) as e:
+        lib.fp4_quantize(ctx, x, 0, alpha=0.4, out=lib.QTensor(128, 128, 0, x.device, 64))
+    assert e.value.code == -3                                   # alpha
+    with pytest.raises(lib.Fp4Error) as e:
+        lib.fp4_quantize(ctx, x, 1, alpha=0.99, out=lib.QTensor(128, 128, 1, x.device, 1000))
+    assert e.value.code == -7                                   # clamp needs token-wise scaling
+    with pytest.raises(lib.Fp4Error) as e:
+        lib.fp4_quantize(ctx, x, 0, alpha=0.99, out=lib.QTensor(128, 128, 0, x.device, 10))
+    assert e.value.code == -8                                   # capacity below 2 * n_tail
+    small = lib.Context(0, 1024)
+    with pytest.raises(lib.Fp4Error) as e:
+        lib.fp4_quantize(small, x, 0)
+    assert e.value.code == -5                                   # workspace
+    small.close()
