@@ -1,0 +1,343 @@
+#!/usr/bin/env python
+"""Benchmark of the FP4 linear layer, forward + backward, on synthetic LLaMA-shaped layers.
+
+One step = one pass of the whole hot path (quantile select, clamp, quantise, FP4 GEMM,
+compensation; dY quantisation, dgrad, wgrad, compensation, DGE) over every linear of the
+workload.  The workload is the LLaMA-1.3B-shaped layer set at 4096 tokens (the second entry of
+the configuration list); inputs are seeded and synthetic.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config I]
+
+Prints ONE JSON line.  `value` = sum over linears of 6 M K N flop / device time of the step,
+inputs resident in HBM.  `e2e` = the same through fp4_linear_step_host with pinned host buffers,
+host<->device copies inside the timed region.  `roofline` describes the kernel class that takes
+the largest share of the step, timed live with CUDA events on the launching stream; `kernels`
+lists every class.  With `--impl reference` the CPU oracle is timed on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "fp4_linear_fwd_bwd_tflops"
+UNIT = "TFLOP/s"
+# fallback peaks (an earlier measurement on this machine), used only if MEASURED_PEAKS.json is absent
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS_SUSTAINED = 1400.0
+FP4_OVER_BF16 = 4.0                 # nominal dense ratio 9 : 2.25 PFLOP/s
+SM_COUNT, FMA_LANES = 148, 128      # plain fp32 pipe: 148 SMs x 128 FMA lanes x 2 flop
+
+# DRAM bytes per launch of the dominant kernel from the committed ncu summaries
+# (profiles/*.md); None where no capture exists for the class.
+NCU_TRAFFIC_PER_UNIT = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops_sustained"]),
+                    sm_max_mhz=float(p.get("sm_max_mhz", 1965.0)), source="measured")
+    return dict(hbm_gbs=FALLBACK_HBM_GBS, bf16_tflops=FALLBACK_BF16_TFLOPS_SUSTAINED, sm_max_mhz=1965.0,
+                source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0]))
+                smax.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def layer_inputs(cfg, WL, seed=0):
+    """Per linear: (name, K, N, A bits, W bits, dY bits).  q/k/v and gate/up read the same activation."""
+    groups = {"q": 0, "k": 0, "v": 0, "o": 1, "gate": 2, "up": 2, "down": 3, "fc": 0}
+    acts = {}
+    out = []
+    for li, lin in enumerate(cfg.linears):
+        g = (groups[lin.name], lin.K)
+        if g not in acts:
+            acts[g] = WL.activations(cfg, lin.K, seed, layer=groups[lin.name])
+        out.append((lin.name, lin.K, lin.N, acts[g], WL.weights(cfg, lin.K, lin.N, seed, layer=li),
+                    WL.output_grads(cfg, lin.N, seed, layer=li)))
+    return out
+
+
+def oracle_sample_tflops(cfg, WL, reps: int, m_rows: int):
+    """The oracle as it stands on the first linear of the workload, `m_rows` tokens; TFLOP/s."""
+    from oracle import fp4_oracle as O
+    lin = cfg.linears[0]
+    a = WL.activations(cfg, lin.K, M=m_rows)
+    w = WL.weights(cfg, lin.K, lin.N)
+    dy = WL.output_grads(cfg, lin.N, M=m_rows)
+    alpha = cfg.alphas[0]
+    times = []
+    for _ in range(reps):
+        t0 = time.perf_counter()
+        f = O.linear_fwd(a, w, alpha)
+        O.linear_bwd(dy, w, f)
+        times.append(time.perf_counter() - t0)
+    flop = 6.0 * m_rows * lin.K * lin.N
+    return flop / 1e12, times
+
+
+def run_reference(args):
+    """CPU oracle on the host cores; rank 0 alone works and prints."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from paper_2501_17116_b200 import workloads as WL
+    cfg = WL.CONFIGS[args.config]
+    m_rows = 1024
+    tf, times = oracle_sample_tflops(cfg, WL, args.warmup + args.steps, m_rows)
+    timed = times[args.warmup:]
+    sec = float(np.sum(timed))
+    value = tf * len(timed) / sec
+    cores = os.cpu_count()
+    lin = cfg.linears[0]
+    sample = f"oracle fwd+bwd of linear '{lin.name}' ({lin.K}x{lin.N}) on the first {m_rows} tokens per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sec / len(timed),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "tokens": cfg.M, "alpha": cfg.alphas[0], "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=1)
+    ap.add_argument("--gemm-kind", type=int, default=0, help="0 mxf4 (K=64), 1 f8f6f4 (K=32)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+
+    import torch
+    import paper_2501_17116_b200 as fp4
+    from paper_2501_17116_b200 import harness, workloads as WL
+
+    rank, local_rank, world = harness.rank_info()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    harness.init_process_group("nccl")
+    peaks = load_peaks()
+    cfg = WL.CONFIGS[args.config]
+    alpha = cfg.alphas[0]
+    M = cfg.M
+    kind = args.gemm_kind
+
+    # ------------------------------------------------------------------ inputs ------------
+    def pinned(bits):
+        return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+
+    layers = []
+    ws_bytes = 0
+    lib = fp4.load_library()
+    for name, K, N, a_bits, w_bits, dy_bits in layer_inputs(cfg, WL, seed=rank):
+        hA, hW, hG = pinned(a_bits), pinned(w_bits), pinned(dy_bits)
+        L = dict(name=name, K=K, N=N, hA=hA, hW=hW, hG=hG, A=hA.to(dev), W=hW.to(dev), G=hG.to(dev),
+                 Y=torch.empty((M, N), dtype=torch.bfloat16, device=dev),
+                 dA=torch.empty((M, K), dtype=torch.bfloat16, device=dev),
+                 dW=torch.empty((K, N), dtype=torch.bfloat16, device=dev),
+                 sa=fp4.QTensor(M, K, 0, dev, fp4.tail_capacity(M, K, alpha)), sw=fp4.QTensor(K, N, 1, dev),
+                 hY=torch.empty((M, N), dtype=torch.bfloat16).pin_memory(),
+                 hdA=torch.empty((M, K), dtype=torch.bfloat16).pin_memory(),
+                 hdW=torch.empty((K, N), dtype=torch.bfloat16).pin_memory())
+        layers.append(L)
+        ws_bytes = max(ws_bytes, int(lib.fp4_step_host_workspace_bytes(M, K, N, alpha)))
+    ctx = fp4.Context(local_rank, ws_bytes)
+    flop_step = sum(6.0 * M * L["K"] * L["N"] for L in layers)
+    resident_bytes = sum(2 * (M * L["K"] + L["K"] * L["N"] + M * L["N"]) * 2 for L in layers)
+
+    def step():
+        for L in layers:
+            fp4.fp4_linear_fwd(ctx, L["A"], L["W"], alpha, L["sa"], L["sw"], gemm_kind=kind, out=L["Y"])
+            fp4.fp4_linear_bwd(ctx, L["G"], L["W"], L["sa"], L["sw"], gemm_kind=kind, dA=L["dA"], dW=L["dW"])
+
+    def step_host():
+        for L in layers:
+            fp4.fp4_linear_step_host(ctx, L["hA"], L["hW"], L["hG"], alpha, L["hY"], L["hdA"], L["hdW"],
+                                     gemm_kind=kind, read_status=False)
+
+    # ------------------------------------------------------------------ device-resident ---
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    assert ctx.read_status() == 0, "device status word is set"
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ctx.profile_reset()
+    ctx.profile_enable(True)
+    harness.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    harness.barrier()
+    ms = e0.elapsed_time(e1)
+    launches = ctx.launch_count()
+    prof = ctx.profile_read()
+    ctx.profile_enable(False)
+    ctx.profile_reset()
+    nnz = [int(L["sa"].nnz.item()) if L["sa"].nnz is not None else 0 for L in layers]
+    assert ctx.read_status() == 0, "device status word is set"
+
+    # ------------------------------------------------------------------ end to end ---------
+    for _ in range(3):
+        step_host()
+    torch.cuda.synchronize()
+    harness.barrier()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        step_host()
+    t1.record()
+    torch.cuda.synchronize()
+    harness.barrier()
+    ms_e2e = t0.elapsed_time(t1)
+    clocks = sampler.stop()
+
+    sec = harness.max_over_ranks(ms / 1e3, dev)
+    sec_e2e = harness.max_over_ranks(ms_e2e / 1e3, dev)
+    total_flop = harness.sum_over_ranks(flop_step * args.steps, dev)
+    value = total_flop / sec / 1e12
+    value_e2e = total_flop / sec_e2e / 1e12
+    h2d = sum((M * L["K"] + L["K"] * L["N"] + M * L["N"]) * 2 for L in layers)
+    d2h = h2d
+
+    # ------------------------------------------------------------------ rooflines ----------
+    fp4_peak = FP4_OVER_BF16 * peaks["bf16_tflops"]
+    alu_peak = SM_COUNT * FMA_LANES * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+    steps = args.steps
+    elems_a = sum(M * L["K"] for L in layers)
+    elems_w = sum(L["K"] * L["N"] for L in layers)
+    elems_g = sum(M * L["N"] for L in layers)
+    nnz_total = sum(nnz)
+    work = {
+        # class: (bound, algorithmic work per step, unit of the rate)
+        "gemm": ("tensor", flop_step, "TFLOP/s"),
+        "select": ("hbm", 2.0 * elems_a, "GB/s"),                                   # one read of A
+        "encode": ("hbm", 3.125 * elems_a + 3.0 * elems_w + 2 * 2.5 * elems_g, "GB/s"),
+        "absmax": ("hbm", 2.0 * elems_w + 2 * 2.0 * elems_g, "GB/s"),                # one read each
+        "sparse": ("hbm", 2 * 8.0 * nnz_total + 3 * elems_a / 8.0, "GB/s"),           # entries + 3 mask sweeps
+        "comp_fwd": ("alu", sum(2.0 * z * L["N"] for z, L in zip(nnz, layers)), "TFLOP/s"),
+        "comp_wgrad_dge": ("alu", sum(2.0 * z * L["N"] + 8.0 * L["K"] * L["N"] for z, L in zip(nnz, layers)),
+                           "TFLOP/s"),
+    }
+    kernels = {}
+    total_ms = sum(v[0] for v in prof.values()) or 1.0
+    for name, (t_ms, n) in prof.items():
+        bound, w_step, unit = work[name]
+        peak = {"tensor": fp4_peak, "hbm": peaks["hbm_gbs"], "alu": alu_peak}[bound]
+        scale = 1e12 if unit == "TFLOP/s" else 1e9
+        achieved = (w_step * steps / (t_ms / 1e3) / scale) if t_ms > 0 else 0.0
+        kernels[name] = {"bound": bound, "achieved": round(achieved, 2), "peak": round(peak, 1), "unit": unit,
+                         "frac": round(achieved / peak, 4), "ms_per_step": round(t_ms / steps, 4),
+                         "share": round(t_ms / total_ms, 4), "launches_per_step": n // steps}
+    dominant = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
+    dk = kernels[dominant]
+    roofline = {"kernel": dominant, "bound": dk["bound"], "achieved": dk["achieved"], "peak": dk["peak"],
+                "unit": dk["unit"], "frac": dk["frac"], "traffic": NCU_TRAFFIC_PER_UNIT.get(dominant),
+                "peak_source": ("of measured" if peaks["source"] == "measured" else "of fallback")
+                + (": 4 x sustained bf16 cuBLAS" if dk["bound"] == "tensor" else
+                   ": copy bandwidth" if dk["bound"] == "hbm" else ": 148 SMs x 128 FMA x 2 x max clock")}
+
+    # ------------------------------------------------------------------ CPU baseline -------
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        tf, times = oracle_sample_tflops(cfg, WL, 2, M)
+        lin = cfg.linears[0]
+        cpu_baseline = {"value": tf / min(times), "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+                        "sample": f"fwd+bwd of linear '{lin.name}' ({lin.K}x{lin.N}) at {M} tokens, best of 2",
+                        "seconds": round(min(times), 3)}
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * sec / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "fp4_e2m1", "data": "synthetic",
+            "config": {"workload": cfg.name, "tokens": M, "linears": [f"{L['name']}:{L['K']}x{L['N']}" for L in layers],
+                       "alpha": alpha, "dge": True, "gemm_kind": "mxf4" if kind == 0 else "f8f6f4",
+                       "l2": f"inputs exceed L2: {resident_bytes / 1e6:.0f} MB touched per step",
+                       "replicas": world},
+            "e2e": {"value": value_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": 1e3 * sec_e2e / args.steps},
+            "gpu_launches": launches,
+            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu_baseline, "clocks": clocks,
+            "residual_nnz": nnz_total,
+        }))
+    ctx.close()
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -164,6 +164,41 @@ int fp4_linear_bwd(fp4_ctx* ctx, void* stream, const void* dY_bf16, const void* 
                    int dge_on, float dge_k, float dge_clip, int gemm_kind,
                    void* dA, void* dW, int out_f32, int32_t* status);
 
+/*
+ * fp4_linear_step_host -- one forward + backward of the layer with HOST buffers (pinned memory
+ * recommended): copies A, W, dY to the device, runs fp4_linear_fwd and fp4_linear_bwd with
+ * BF16 outputs, and copies Y, dA, dW back, all on `stream`.  It is the same path as the two
+ * calls above (Fig. 2, Eq. 3, Eq. 6); only the staging is added.  Device staging and the saved
+ * quantised operands live in the context's workspace: fp4_step_host_workspace_bytes() gives
+ * the size needed.  `status_host` (host int32, may be NULL) receives the device status word;
+ * reading it makes the call wait for the stream.  All six tensor pointers are HOST pointers.
+ */
+size_t fp4_step_host_workspace_bytes(int64_t M, int64_t K, int64_t N, double alpha);
+int fp4_linear_step_host(fp4_ctx* ctx, void* stream, const void* A_host, const void* W_host,
+                         const void* dY_host, int64_t M, int64_t K, int64_t N, double alpha,
+                         int dge_on, float dge_k, float dge_clip, int gemm_kind,
+                         void* Y_host, void* dA_host, void* dW_host, int32_t* status_host);
+
+/*
+ * Measurement support (no counterpart in the paper).  With profiling on, every kernel class the
+ * library enqueues is bracketed by CUDA events on the launching stream; fp4_profile_read waits
+ * for them and returns the summed device time and the number of kernels of one class since the
+ * last fp4_profile_reset.  fp4_launch_count returns the kernels enqueued since the last reset,
+ * whether profiling is on or not.
+ */
+#define FP4_KC_GEMM        0   /* tcgen05 FP4 GEMM                                            */
+#define FP4_KC_SELECT      1   /* histogram + row extremes + order statistics                 */
+#define FP4_KC_ENCODE      2   /* clamp / scale / Q / pack, both layouts                      */
+#define FP4_KC_ABSMAX      3   /* absmax pre-pass of tensors that are not clamped             */
+#define FP4_KC_SPARSE      4   /* mask -> CSR / CSC                                           */
+#define FP4_KC_COMP_FWD    5   /* residual x W + final store of Y                             */
+#define FP4_KC_COMP_WGRAD  6   /* residual^T x dY + DGE factor + final store of dW            */
+#define FP4_KC_COUNT       7
+int fp4_profile_enable(fp4_ctx* ctx, int on);
+int fp4_profile_reset(fp4_ctx* ctx);
+int fp4_profile_read(fp4_ctx* ctx, int kernel_class, double* total_ms, int64_t* launches);
+int64_t fp4_launch_count(fp4_ctx* ctx);
+
 #ifdef __cplusplus
 }
 #endif

@@ -20,7 +20,10 @@ FP4_DEV_NONFINITE = 2
 FP4_DEV_TIMEOUT = 4
 
 EXPORTS = ("fp4_create", "fp4_destroy", "fp4_workspace_bytes", "fp4_status_string", "fp4_quantize",
-           "fp4_gemm", "fp4_linear_fwd", "fp4_linear_bwd")
+           "fp4_gemm", "fp4_linear_fwd", "fp4_linear_bwd", "fp4_step_host_workspace_bytes",
+           "fp4_linear_step_host", "fp4_profile_enable", "fp4_profile_reset", "fp4_profile_read",
+           "fp4_launch_count")
+KERNEL_CLASSES = ("gemm", "select", "encode", "absmax", "sparse", "comp_fwd", "comp_wgrad_dge")
 
 
 class fp4_qtensor(C.Structure):
@@ -66,6 +69,19 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.fp4_linear_bwd.argtypes = [vp, vp, vp, vp, C.POINTER(fp4_qtensor), C.POINTER(fp4_qtensor), i64, i64, i64,
                                    C.c_int, C.c_float, C.c_float, C.c_int, vp, vp, C.c_int, i32p]
     lib.fp4_linear_bwd.restype = C.c_int
+    lib.fp4_step_host_workspace_bytes.argtypes = [i64, i64, i64, C.c_double]
+    lib.fp4_step_host_workspace_bytes.restype = C.c_size_t
+    lib.fp4_linear_step_host.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, C.c_double, C.c_int, C.c_float,
+                                         C.c_float, C.c_int, vp, vp, vp, C.POINTER(C.c_int32)]
+    lib.fp4_linear_step_host.restype = C.c_int
+    lib.fp4_profile_enable.argtypes = [vp, C.c_int]
+    lib.fp4_profile_enable.restype = C.c_int
+    lib.fp4_profile_reset.argtypes = [vp]
+    lib.fp4_profile_reset.restype = C.c_int
+    lib.fp4_profile_read.argtypes = [vp, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+    lib.fp4_profile_read.restype = C.c_int
+    lib.fp4_launch_count.argtypes = [vp]
+    lib.fp4_launch_count.restype = C.c_int64
     if path == LIB_PATH:
         _lib = lib
     return lib
@@ -120,6 +136,25 @@ class Context:
     def read_status(self) -> int:
         """Device status word (synchronises)."""
         return int(self.status.item())
+
+    # measurement support -------------------------------------------------------------------
+    def profile_enable(self, on: bool = True):
+        _check(self.lib.fp4_profile_enable(self.handle, int(on)))
+
+    def profile_reset(self):
+        _check(self.lib.fp4_profile_reset(self.handle))
+
+    def profile_read(self) -> dict:
+        """{kernel class: (total device ms, kernels)} since the last reset (waits for the events)."""
+        out = {}
+        for kc, name in enumerate(KERNEL_CLASSES):
+            ms, n = C.c_double(), C.c_int64()
+            _check(self.lib.fp4_profile_read(self.handle, kc, C.byref(ms), C.byref(n)))
+            out[name] = (ms.value, n.value)
+        return out
+
+    def launch_count(self) -> int:
+        return int(self.lib.fp4_launch_count(self.handle))
 
 
 class QTensor:
@@ -216,3 +251,20 @@ def fp4_linear_bwd(ctx: Context, dY: torch.Tensor, W: torch.Tensor, saved_a: QTe
                                   C.byref(saved_w.struct), M, K, N, int(dge_on), float(dge_k), float(dge_clip),
                                   gemm_kind, _ptr(dA), _ptr(dW), int(out_f32), _ptr(ctx.status)))
     return dA, dW
+
+
+def fp4_linear_step_host(ctx: Context, A_host: torch.Tensor, W_host: torch.Tensor, dY_host: torch.Tensor,
+                         alpha: float, Y_host: torch.Tensor, dA_host: torch.Tensor, dW_host: torch.Tensor,
+                         dge_on: bool = True, dge_k: float = 5.0, dge_clip: float = 3.0,
+                         gemm_kind: int = FP4_GEMM_MXF4, read_status: bool = True) -> int:
+    """Forward + backward with host (pinned) BF16 tensors; returns the device status word."""
+    M, K = A_host.shape
+    N = W_host.shape[1]
+    for t in (A_host, W_host, dY_host, Y_host, dA_host, dW_host):
+        assert not t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+    st = C.c_int32(0)
+    _check(ctx.lib.fp4_linear_step_host(ctx.handle, _stream(), _ptr(A_host), _ptr(W_host), _ptr(dY_host), M, K, N,
+                                        float(alpha), int(dge_on), float(dge_k), float(dge_clip), gemm_kind,
+                                        _ptr(Y_host), _ptr(dA_host), _ptr(dW_host),
+                                        C.byref(st) if read_status else None))
+    return st.value

@@ -32,6 +32,13 @@ int check_qtensor_dense(const fp4_qtensor* q) {
   return FP4_OK;
 }
 
+int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf16, const void* W_bf16, int64_t M,
+                    int64_t K, int64_t N, double alpha, int reuse_w, int gemm_kind, void* Y, int out_f32,
+                    fp4_qtensor* savedA, fp4_qtensor* savedW, int32_t* status);
+int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_bf16, const void* W_bf16,
+                    const fp4_qtensor* savedA, const fp4_qtensor* savedW, int64_t M, int64_t K, int64_t N, int dge_on,
+                    float dge_k, float dge_clip, int gemm_kind, void* dA, void* dW, int out_f32, int32_t* status);
+
 int check_qtensor_sparse(const fp4_qtensor* q, int64_t n_tail) {
   if (!q->thresholds || !q->nnz || !q->csr_rowptr || !q->csr_col || !q->csr_val || !q->csc_colptr || !q->csc_row ||
       !q->csc_val)
@@ -79,19 +86,28 @@ int fp4_create(fp4_ctx** out, int device, size_t workspace_bytes) {
   ctx->workspace = nullptr;
   ctx->workspace_bytes = 0;
   ctx->encode_tiled = nullptr;
+  ctx->profile = 0;
+  ctx->launch_count = 0;
+  ctx->records = new (std::nothrow) std::vector<ProfRecord>();
   cudaDeviceProp prop;
-  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return FP4_ERR_CUDA; }
+  if (!ctx->records || cudaGetDeviceProperties(&prop, device) != cudaSuccess) {
+    delete ctx->records;
+    delete ctx;
+    return FP4_ERR_CUDA;
+  }
   ctx->num_sms = prop.multiProcessorCount;
   cudaDriverEntryPointQueryResult qres;
   void* fn = nullptr;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
       qres != cudaDriverEntryPointSuccess || !fn) {
+    delete ctx->records;
     delete ctx;
     return FP4_ERR_CUDA;
   }
   ctx->encode_tiled = fn;
   if (workspace_bytes) {
     if (cudaMalloc(reinterpret_cast<void**>(&ctx->workspace), workspace_bytes) != cudaSuccess) {
+      delete ctx->records;
       delete ctx;
       return FP4_ERR_CUDA;
     }
@@ -105,6 +121,10 @@ int fp4_destroy(fp4_ctx* ctx) {
   if (!ctx) return FP4_ERR_NULL;
   cudaSetDevice(ctx->device);
   if (ctx->workspace) cudaFree(ctx->workspace);
+  if (ctx->records) {
+    fp4_profile_reset(ctx);
+    delete ctx->records;
+  }
   delete ctx;
   return FP4_OK;
 }
@@ -164,12 +184,21 @@ int fp4_linear_fwd(fp4_ctx* ctx, void* stream, const void* A_bf16, const void* W
     if (rc != FP4_OK) return rc;
   }
   if (fp4_workspace_bytes(M, K, N) > ctx->workspace_bytes) return FP4_ERR_WORKSPACE;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return linear_fwd_impl(ctx, static_cast<cudaStream_t>(stream), Arena(ctx->workspace, ctx->workspace_bytes), A_bf16,
+                         W_bf16, M, K, N, alpha, reuse_w, gemm_kind, Y, out_f32, savedA, savedW, status);
+}
 
-  Arena arena(ctx->workspace, ctx->workspace_bytes);
+}  // extern "C"
+
+namespace {
+
+int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf16, const void* W_bf16, int64_t M,
+                    int64_t K, int64_t N, double alpha, int reuse_w, int gemm_kind, void* Y, int out_f32,
+                    fp4_qtensor* savedA, fp4_qtensor* savedW, int32_t* status) {
+  const bool occ = alpha < 1.0;
   float* y1 = occ ? arena.take<float>(size_t(M) * size_t(N)) : nullptr;
   if (!arena.ok) return FP4_ERR_WORKSPACE;
-  Arena qa_arena(ctx->workspace + arena.off, ctx->workspace_bytes - arena.off);
+  Arena qa_arena(arena.base + arena.off, arena.size - arena.off);
 
   int rc;
   if (!reuse_w) {
@@ -199,6 +228,10 @@ int fp4_linear_fwd(fp4_ctx* ctx, void* stream, const void* A_bf16, const void* W
                          out_f32);
 }
 
+}  // namespace
+
+extern "C" {
+
 int fp4_linear_bwd(fp4_ctx* ctx, void* stream, const void* dY_bf16, const void* W_bf16, const fp4_qtensor* savedA,
                    const fp4_qtensor* savedW, int64_t M, int64_t K, int64_t N, int dge_on, float dge_k,
                    float dge_clip, int gemm_kind, void* dA, void* dW, int out_f32, int32_t* status) {
@@ -211,14 +244,22 @@ int fp4_linear_bwd(fp4_ctx* ctx, void* stream, const void* dY_bf16, const void* 
   if (!savedA->codes_t || !savedA->amax || !savedW->codes || !savedW->amax) return FP4_ERR_NULL;
   if (!aligned16(dY_bf16) || !aligned16(W_bf16) || !aligned16(dA) || !aligned16(dW)) return FP4_ERR_ALIGN;
   if (fp4_workspace_bytes(M, K, N) > ctx->workspace_bytes) return FP4_ERR_WORKSPACE;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return linear_bwd_impl(ctx, static_cast<cudaStream_t>(stream), Arena(ctx->workspace, ctx->workspace_bytes), dY_bf16,
+                         W_bf16, savedA, savedW, M, K, N, dge_on, dge_k, dge_clip, gemm_kind, dA, dW, out_f32, status);
+}
 
-  Arena arena(ctx->workspace, ctx->workspace_bytes);
+}  // extern "C"
+
+namespace {
+
+int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_bf16, const void* W_bf16,
+                    const fp4_qtensor* savedA, const fp4_qtensor* savedW, int64_t M, int64_t K, int64_t N, int dge_on,
+                    float dge_k, float dge_clip, int gemm_kind, void* dA, void* dW, int out_f32, int32_t* status) {
   float* s = arena.take<float>(size_t(K) * size_t(N));
   uint8_t* g_codes = arena.take<uint8_t>(size_t(M) * size_t(N) / 2);
   float* g_amax = arena.take<float>(size_t(M > N ? M : N));
   if (!arena.ok) return FP4_ERR_WORKSPACE;
-  Arena q_arena(ctx->workspace + arena.off, ctx->workspace_bytes - arena.off);
+  Arena q_arena(arena.base + arena.off, arena.size - arena.off);
   int rc;
 
   if (dA) {
@@ -247,5 +288,130 @@ int fp4_linear_bwd(fp4_ctx* ctx, void* stream, const void* dY_bf16, const void* 
   }
   return FP4_OK;
 }
+
+// Buffers of one saved operand carved from the workspace (fp4_linear_step_host).
+void carve_qtensor(Arena& a, fp4_qtensor* q, int64_t rows, int64_t cols, int scale_axis, int64_t cap) {
+  *q = fp4_qtensor();
+  q->rows = rows;
+  q->cols = cols;
+  q->codes = a.take<uint8_t>(size_t(rows) * size_t(cols) / 2);
+  q->codes_t = a.take<uint8_t>(size_t(rows) * size_t(cols) / 2);
+  q->amax = a.take<float>(size_t(scale_axis == 0 ? rows : cols));
+  q->sparse_cap = cap;
+  if (cap > 0) {
+    q->thresholds = a.take<float>(2);
+    q->nnz = a.take<int32_t>(1);
+    q->csr_rowptr = a.take<int32_t>(size_t(rows) + 1);
+    q->csr_col = a.take<int32_t>(size_t(cap));
+    q->csr_val = a.take<float>(size_t(cap));
+    q->csc_colptr = a.take<int32_t>(size_t(cols) + 1);
+    q->csc_row = a.take<int32_t>(size_t(cap));
+    q->csc_val = a.take<float>(size_t(cap));
+  }
+}
+
+int64_t step_capacity(int64_t M, int64_t K, double alpha) {
+  return alpha < 1.0 ? 2 * llround((1.0 - alpha) * double(M * K)) : 0;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t fp4_step_host_workspace_bytes(int64_t M, int64_t K, int64_t N, double alpha) {
+  if (M <= 0 || K <= 0 || N <= 0) return 0;
+  const size_t cap = size_t(step_capacity(M, K, alpha));
+  size_t b = 0;
+  b += 2 * (round256(size_t(M) * K * 2) + round256(size_t(K) * N * 2) + round256(size_t(M) * N * 2));  // in + out
+  b += 2 * round256(size_t(M) * K / 2) + 2 * round256(size_t(K) * N / 2);                                // codes
+  b += round256(size_t(M) * 4) + round256(size_t(N) * 4);                                                // amax
+  b += 4 * round256(cap * 4) + round256((size_t(M) + 1) * 4) + round256((size_t(K) + 1) * 4) + 3 * 256;   // sparse
+  b += 256;                                                                                              // status
+  return b + fp4_workspace_bytes(M, K, N);
+}
+
+int fp4_linear_step_host(fp4_ctx* ctx, void* stream, const void* A_host, const void* W_host, const void* dY_host,
+                         int64_t M, int64_t K, int64_t N, double alpha, int dge_on, float dge_k, float dge_clip,
+                         int gemm_kind, void* Y_host, void* dA_host, void* dW_host, int32_t* status_host) {
+  if (!ctx || !A_host || !W_host || !dY_host || !Y_host || !dA_host || !dW_host) return FP4_ERR_NULL;
+  if (!mult128(M) || !mult128(K) || !mult128(N)) return FP4_ERR_SHAPE;
+  if (M * K >= (int64_t(1) << 31) || K * N >= (int64_t(1) << 31) || M * N >= (int64_t(1) << 31)) return FP4_ERR_SHAPE;
+  if (!(alpha > 0.5 && alpha <= 1.0)) return FP4_ERR_ALPHA;
+  if (gemm_kind != FP4_GEMM_MXF4 && gemm_kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;
+  if (dge_on && !(dge_k > 1.0f && dge_clip > 0.0f)) return FP4_ERR_ARG;
+  if (alpha < 1.0 && step_capacity(M, K, alpha) >= M * K) return FP4_ERR_ALPHA;
+  if (fp4_step_host_workspace_bytes(M, K, N, alpha) > ctx->workspace_bytes) return FP4_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  Arena arena(ctx->workspace, ctx->workspace_bytes);
+  const size_t a_bytes = size_t(M) * K * 2, w_bytes = size_t(K) * N * 2, y_bytes = size_t(M) * N * 2;
+  char* dA_in = arena.take<char>(a_bytes);
+  char* dW_in = arena.take<char>(w_bytes);
+  char* dG_in = arena.take<char>(y_bytes);
+  char* dY_out = arena.take<char>(y_bytes);
+  char* dA_out = arena.take<char>(a_bytes);
+  char* dW_out = arena.take<char>(w_bytes);
+  int32_t* status = arena.take<int32_t>(1);
+  fp4_qtensor qa, qw;
+  carve_qtensor(arena, &qa, M, K, 0, step_capacity(M, K, alpha));
+  carve_qtensor(arena, &qw, K, N, 1, 0);
+  if (!arena.ok) return FP4_ERR_WORKSPACE;
+  Arena rest(arena.base + arena.off, arena.size - arena.off);
+
+  FP4_CUDA_TRY(cudaMemsetAsync(status, 0, 4, st));
+  FP4_CUDA_TRY(cudaMemcpyAsync(dA_in, A_host, a_bytes, cudaMemcpyHostToDevice, st));
+  FP4_CUDA_TRY(cudaMemcpyAsync(dW_in, W_host, w_bytes, cudaMemcpyHostToDevice, st));
+  FP4_CUDA_TRY(cudaMemcpyAsync(dG_in, dY_host, y_bytes, cudaMemcpyHostToDevice, st));
+  int rc = linear_fwd_impl(ctx, st, rest, dA_in, dW_in, M, K, N, alpha, 0, gemm_kind, dY_out, 0, &qa, &qw, status);
+  if (rc != FP4_OK) return rc;
+  rc = linear_bwd_impl(ctx, st, rest, dG_in, dW_in, &qa, &qw, M, K, N, dge_on, dge_k, dge_clip, gemm_kind, dA_out,
+                       dW_out, 0, status);
+  if (rc != FP4_OK) return rc;
+  FP4_CUDA_TRY(cudaMemcpyAsync(Y_host, dY_out, y_bytes, cudaMemcpyDeviceToHost, st));
+  FP4_CUDA_TRY(cudaMemcpyAsync(dA_host, dA_out, a_bytes, cudaMemcpyDeviceToHost, st));
+  FP4_CUDA_TRY(cudaMemcpyAsync(dW_host, dW_out, w_bytes, cudaMemcpyDeviceToHost, st));
+  if (status_host) {
+    FP4_CUDA_TRY(cudaMemcpyAsync(status_host, status, 4, cudaMemcpyDeviceToHost, st));
+    FP4_CUDA_TRY(cudaStreamSynchronize(st));
+  }
+  return FP4_OK;
+}
+
+int fp4_profile_enable(fp4_ctx* ctx, int on) {
+  if (!ctx) return FP4_ERR_NULL;
+  ctx->profile = on ? 1 : 0;
+  return FP4_OK;
+}
+
+int fp4_profile_reset(fp4_ctx* ctx) {
+  if (!ctx) return FP4_ERR_NULL;
+  for (ProfRecord& r : *ctx->records) {
+    cudaEventDestroy(r.start);
+    cudaEventDestroy(r.stop);
+  }
+  ctx->records->clear();
+  ctx->launch_count = 0;
+  return FP4_OK;
+}
+
+int fp4_profile_read(fp4_ctx* ctx, int kernel_class, double* total_ms, int64_t* launches) {
+  if (!ctx || !total_ms || !launches) return FP4_ERR_NULL;
+  if (kernel_class < 0 || kernel_class >= FP4_KC_COUNT) return FP4_ERR_ARG;
+  double ms = 0.0;
+  int64_t n = 0;
+  for (ProfRecord& r : *ctx->records) {
+    if (r.kc != kernel_class) continue;
+    FP4_CUDA_TRY(cudaEventSynchronize(r.stop));
+    float t = 0.f;
+    FP4_CUDA_TRY(cudaEventElapsedTime(&t, r.start, r.stop));
+    ms += t;
+    n += r.launches;
+  }
+  *total_ms = ms;
+  *launches = n;
+  return FP4_OK;
+}
+
+int64_t fp4_launch_count(fp4_ctx* ctx) { return ctx ? ctx->launch_count : -1; }
 
 }  // extern "C"

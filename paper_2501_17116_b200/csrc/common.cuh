@@ -6,7 +6,27 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "fp4_linear.h"
+
+// Kernel classes reported by fp4_profile_read (values are part of the ABI, see fp4_linear.h).
+enum KernelClass {
+  KC_GEMM = FP4_KC_GEMM,
+  KC_SELECT = FP4_KC_SELECT,
+  KC_ENCODE = FP4_KC_ENCODE,
+  KC_ABSMAX = FP4_KC_ABSMAX,
+  KC_SPARSE = FP4_KC_SPARSE,
+  KC_COMP_FWD = FP4_KC_COMP_FWD,
+  KC_COMP_WGRAD = FP4_KC_COMP_WGRAD,
+  KC_COUNT = FP4_KC_COUNT
+};
+
+struct ProfRecord {
+  int kc;
+  int launches;
+  cudaEvent_t start, stop;
+};
 
 struct fp4_ctx {
   int      device;
@@ -14,6 +34,33 @@ struct fp4_ctx {
   char*    workspace;
   size_t   workspace_bytes;
   void*    encode_tiled;       // cuTensorMapEncodeTiled, fetched through the runtime
+  int      profile;            // record CUDA events around every kernel class
+  long long launch_count;      // kernels enqueued since the last reset
+  std::vector<ProfRecord>* records;
+};
+
+// Counts the kernels a launcher enqueues and, in profiling mode, brackets them with CUDA events
+// on the launching stream.
+struct KernelScope {
+  fp4_ctx* c;
+  cudaStream_t s;
+  cudaEvent_t stop = nullptr;
+  KernelScope(fp4_ctx* ctx, cudaStream_t stream, int kc, int launches) : c(ctx), s(stream) {
+    c->launch_count += launches;
+    if (c->profile && c->records) {
+      ProfRecord r;
+      r.kc = kc;
+      r.launches = launches;
+      if (cudaEventCreate(&r.start) != cudaSuccess) return;
+      if (cudaEventCreate(&r.stop) != cudaSuccess) { cudaEventDestroy(r.start); return; }
+      cudaEventRecord(r.start, s);
+      stop = r.stop;
+      c->records->push_back(r);
+    }
+  }
+  ~KernelScope() {
+    if (stop) cudaEventRecord(stop, s);
+  }
 };
 
 #define FP4_CUDA_TRY(expr)                         \

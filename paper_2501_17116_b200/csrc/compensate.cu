@@ -130,19 +130,21 @@ comp_wgrad_dge_kernel(const float* __restrict__ s, const int* __restrict__ colpt
 
 }  // namespace
 
-int launch_comp_fwd(fp4_ctx*, cudaStream_t stream, const float* y1, const int32_t* rowptr, const int32_t* col,
+int launch_comp_fwd(fp4_ctx* ctx, cudaStream_t stream, const float* y1, const int32_t* rowptr, const int32_t* col,
                     const float* val, const void* w_bf16, int64_t M, int64_t, int64_t N, void* y, int out_f32) {
   const dim3 grid(unsigned((N + COMP_COLS - 1) / COMP_COLS), unsigned((M + 7) / 8));
+  KernelScope scope(ctx, stream, KC_COMP_FWD, 1);
   comp_fwd_kernel<<<grid, COMP_THREADS, 0, stream>>>(y1, rowptr, col, val, static_cast<const uint4*>(w_bf16), int(M),
                                                      int(N), y, out_f32);
   FP4_CUDA_TRY(cudaGetLastError());
   return FP4_OK;
 }
 
-int launch_comp_wgrad_dge(fp4_ctx*, cudaStream_t stream, const float* s, const int32_t* colptr, const int32_t* row,
+int launch_comp_wgrad_dge(fp4_ctx* ctx, cudaStream_t stream, const float* s, const int32_t* colptr, const int32_t* row,
                           const float* val, const void* dy_bf16, const void* w_bf16, const float* w_amax, int64_t,
                           int64_t K, int64_t N, int dge_on, float dge_k, float dge_clip, void* dw, int out_f32) {
   const dim3 grid(unsigned((N + COMP_COLS - 1) / COMP_COLS), unsigned((K + 7) / 8));
+  KernelScope scope(ctx, stream, KC_COMP_WGRAD, 1);
   comp_wgrad_dge_kernel<<<grid, COMP_THREADS, 0, stream>>>(s, colptr, row, val, static_cast<const uint4*>(dy_bf16),
                                                            static_cast<const uint4*>(w_bf16), w_amax, int(K), int(N),
                                                            dge_on, dge_k, dge_clip, dw, out_f32);

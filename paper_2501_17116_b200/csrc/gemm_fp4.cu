@@ -429,6 +429,7 @@ int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, c
   const int tiles = args.num_m_blocks * args.num_n_blocks;
   const int grid = tiles < ctx->num_sms ? tiles : ctx->num_sms;
 
+  KernelScope scope(ctx, stream, KC_GEMM, 1);
   if (gemm_kind == FP4_GEMM_F8F6F4) {
     FP4_CUDA_TRY(cudaFuncSetAttribute(gemm_fp4_kernel<FP4_GEMM_F8F6F4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       int(SMEM_BYTES)));

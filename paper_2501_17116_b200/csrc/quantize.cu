@@ -569,6 +569,7 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
   if (!arena.ok) return FP4_ERR_WORKSPACE;
   if (prescale && prescale_is_amax) {
     const int np = scale_axis == 0 ? cols : rows;
+    KernelScope scope(ctx, stream, KC_ABSMAX, 1);
     descale_kernel<<<(np + 255) / 256, 256, 0, stream>>>(prescale, np, pre_d);
     prescale = pre_d;
   }
@@ -590,6 +591,8 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
 
   if (occ) {
     const long long n_tail = llround((1.0 - alpha) * double(n));
+    {
+    KernelScope scope(ctx, stream, KC_SELECT, 3);
     FP4_CUDA_TRY(cudaMemsetAsync(hist, 0, 65536 * 4, stream));
     init_row_extremes_kernel<<<(rows + 255) / 256, 256, 0, stream>>>(row_max, row_min, rows);
     FP4_CUDA_TRY(cudaFuncSetAttribute(hist_rowminmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -599,7 +602,12 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
     hist_rowminmax_kernel<<<int(blocks), HIST_THREADS, HIST_WORDS * 4, stream>>>(x, n_vec, vec_per_row, hist, row_max,
                                                                                 row_min);
     select_thresholds_kernel<<<1, 1024, 0, stream>>>(hist, n, n_tail, out->thresholds);
-    encode_kernel<0, true, false><<<enc_grid, ENC_THREADS, 0, stream>>>(ea);
+    }
+    {
+      KernelScope scope(ctx, stream, KC_ENCODE, 1);
+      encode_kernel<0, true, false><<<enc_grid, ENC_THREADS, 0, stream>>>(ea);
+    }
+    KernelScope scope(ctx, stream, KC_SPARSE, 7);
 
     const uint32_t* mask32 = reinterpret_cast<const uint32_t*>(mask);
     const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x_bf16);
@@ -622,10 +630,14 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
     if (scale_axis == 0) {
       long long blocks = (n_vec + 255) / 256;
       if (blocks > 8LL * ctx->num_sms) blocks = 8LL * ctx->num_sms;
-      if (prescale)
-        absmax_rows_kernel<true><<<int(blocks), 256, 0, stream>>>(x, n_vec, vec_per_row, prescale, vec_amax);
-      else
-        absmax_rows_kernel<false><<<int(blocks), 256, 0, stream>>>(x, n_vec, vec_per_row, nullptr, vec_amax);
+      {
+        KernelScope scope(ctx, stream, KC_ABSMAX, 1);
+        if (prescale)
+          absmax_rows_kernel<true><<<int(blocks), 256, 0, stream>>>(x, n_vec, vec_per_row, prescale, vec_amax);
+        else
+          absmax_rows_kernel<false><<<int(blocks), 256, 0, stream>>>(x, n_vec, vec_per_row, nullptr, vec_amax);
+      }
+      KernelScope scope(ctx, stream, KC_ENCODE, 1);
       if (prescale)
         encode_kernel<0, false, true><<<enc_grid, ENC_THREADS, 0, stream>>>(ea);
       else
@@ -637,10 +649,16 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
       if (strips < 1) strips = 1;
       const int rows_per_strip = (rows + strips - 1) / strips;
       const dim3 agrid(col_blocks, (rows + rows_per_strip - 1) / rows_per_strip);
-      if (prescale)
-        absmax_cols_kernel<true><<<agrid, 256, 0, stream>>>(x, rows, vec_per_row, rows_per_strip, prescale, vec_amax);
-      else
-        absmax_cols_kernel<false><<<agrid, 256, 0, stream>>>(x, rows, vec_per_row, rows_per_strip, nullptr, vec_amax);
+      {
+        KernelScope scope(ctx, stream, KC_ABSMAX, 1);
+        if (prescale)
+          absmax_cols_kernel<true><<<agrid, 256, 0, stream>>>(x, rows, vec_per_row, rows_per_strip, prescale,
+                                                              vec_amax);
+        else
+          absmax_cols_kernel<false><<<agrid, 256, 0, stream>>>(x, rows, vec_per_row, rows_per_strip, nullptr,
+                                                               vec_amax);
+      }
+      KernelScope scope(ctx, stream, KC_ENCODE, 1);
       if (prescale)
         encode_kernel<1, false, true><<<enc_grid, ENC_THREADS, 0, stream>>>(ea);
       else
