@@ -106,7 +106,7 @@ int launch_comp_fwd(fp4_ctx* ctx, cudaStream_t stream, const float* y1, const in
                     const int32_t* col, const float* val, const void* w_bf16, int64_t M, int64_t K,
                     int64_t N, void* y, int out_f32);
 // dw[k,:] = store( (s[k,:] + sum_{entries of column k} val * dy[row,:]) * Q'(w[k,:] * gamma[:]) )
-int launch_comp_wgrad_dge(fp4_ctx* ctx, cudaStream_t stream, const float* s, const int32_t* colptr,
+int launch_comp_wgrad_dge(fp4_ctx* ctx, cudaStream_t stream, float* s, const int32_t* colptr,
                           const int32_t* row, const float* val, const void* dy_bf16,
                           const void* w_bf16, const float* w_amax, int64_t M, int64_t K, int64_t N,
                           int dge_on, float dge_k, float dge_clip, void* dw, int out_f32);

@@ -96,36 +96,94 @@ __device__ __forceinline__ float dge_factor(float ws, float expo, float inv_k, f
   return fminf(d, clip);
 }
 
+// Weight-gradient compensation, step 1: S[k, n-block] += sum over the entries of column k of
+// dA[m,k] * dY[m, n-block].  One block per (column, 256 output columns).  Outliers sit in a few
+// channels (Appendix D), so a handful of columns hold thousands of entries and most hold none:
+// empty columns leave at once, and the eight warps of a block take the entries of a long column
+// round-robin.  Their partial sums are added in warp order, so the result does not depend on
+// scheduling.
 __global__ void __launch_bounds__(COMP_THREADS)
-comp_wgrad_dge_kernel(const float* __restrict__ s, const int* __restrict__ colptr, const int* __restrict__ row,
-                      const float* __restrict__ val, const uint4* __restrict__ dy, const uint4* __restrict__ w,
-                      const float* __restrict__ w_amax, int K, int N, int dge_on, float dge_k, float dge_clip,
-                      void* dw, int out_f32) {
-  const int k = blockIdx.y * 8 + (threadIdx.x >> 5);
-  const int n0 = blockIdx.x * COMP_COLS + 8 * (threadIdx.x & 31);
-  if (k >= K || n0 >= N) return;
+comp_wgrad_accum_kernel(float* __restrict__ s, const int* __restrict__ colptr, const int* __restrict__ row,
+                        const float* __restrict__ val, const uint4* __restrict__ dy, int K, int N) {
+  __shared__ float part[8][32][9];                  // [warp][lane][8 (+1 pad)]
+  const int k = blockIdx.y;
+  const int e0 = colptr[k], e1 = colptr[k + 1];
+  if (e0 == e1) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n0 = blockIdx.x * COMP_COLS + 8 * lane;
+  const bool in_cols = n0 < N;
+  const int vcol = n0 >> 3, vec_per_row = N >> 3;
   float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  if (colptr) sparse_row_times_dense(acc, row, val, colptr[k], colptr[k + 1], dy, N >> 3, n0 >> 3);
-  const long long off = (long long)k * N + n0;
-  const float4 a = *reinterpret_cast<const float4*>(s + off);
-  const float4 b = *reinterpret_cast<const float4*>(s + off + 4);
-  float y8[8] = {a.x + acc[0], a.y + acc[1], a.z + acc[2], a.w + acc[3],
-                 b.x + acc[4], b.y + acc[5], b.z + acc[6], b.w + acc[7]};
-  if (dge_on) {
-    const uint4 wv = __ldg(&w[off >> 3]);
-    const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
-    const float inv_k = 1.0f / dge_k;
-    const float expo = inv_k - 1.0f;
+  if (in_cols) {
+    int e = e0 + warp;
+    for (; e + 24 < e1; e += 32) {                  // four entries of this warp in flight
+      int r[4];
+      float v[4];
+      uint4 d[4];
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      const float wf = __uint_as_float((c & 1) ? (ww[c >> 1] & 0xFFFF0000u) : (ww[c >> 1] << 16));
-      const float amax = __ldg(&w_amax[n0 + c]);
-      const float gamma = amax > 0.0f ? __fdiv_rn(6.0f, amax) : 0.0f;
-      const float ws = __fmul_rn(wf, gamma);          // the value the forward quantised
-      y8[c] *= dge_factor(ws, expo, inv_k, dge_clip);
+      for (int u = 0; u < 4; ++u) {
+        r[u] = __ldg(&row[e + 8 * u]);
+        v[u] = __ldg(&val[e + 8 * u]);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) d[u] = __ldg(&dy[(long long)r[u] * vec_per_row + vcol]);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) fma8(acc, v[u], d[u]);
+    }
+    for (; e < e1; e += 8) {
+      const uint4 d = __ldg(&dy[(long long)__ldg(&row[e]) * vec_per_row + vcol]);
+      fma8(acc, __ldg(&val[e]), d);
     }
   }
-  store8(dw, out_f32, off, y8);
+#pragma unroll
+  for (int c = 0; c < 8; ++c) part[warp][lane][c] = acc[c];
+  __syncthreads();
+  if (warp == 0 && in_cols) {
+    float* dst = s + (long long)k * N + n0;
+    float4 a = *reinterpret_cast<float4*>(dst);
+    float4 b = *reinterpret_cast<float4*>(dst + 4);
+    float t[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    for (int w = 0; w < 8; ++w) {
+#pragma unroll
+      for (int c = 0; c < 8; ++c) t[c] += part[w][lane][c];
+    }
+    a.x += t[0]; a.y += t[1]; a.z += t[2]; a.w += t[3];
+    b.x += t[4]; b.y += t[5]; b.z += t[6]; b.w += t[7];
+    *reinterpret_cast<float4*>(dst) = a;
+    *reinterpret_cast<float4*>(dst + 4) = b;
+  }
+}
+
+// Weight-gradient step 2: dW = store( S (.) Q'(W (.) gamma) ), element-wise (Eq. 6 with the DGE
+// derivative of Eq. 8 evaluated on the scaled weights the forward quantised).
+__global__ void __launch_bounds__(256)
+dge_store_kernel(const float* __restrict__ s, const uint4* __restrict__ w, const float* __restrict__ w_amax,
+                 long long n_vec, int vec_per_row, int dge_on, float dge_k, float dge_clip, void* dw, int out_f32) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  const float inv_k = 1.0f / dge_k;
+  const float expo = inv_k - 1.0f;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += stride) {
+    const long long off = i * 8;
+    const float4 a = __ldg(reinterpret_cast<const float4*>(s + off));
+    const float4 b = __ldg(reinterpret_cast<const float4*>(s + off + 4));
+    float y8[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    if (dge_on) {
+      const int n0 = int(i % vec_per_row) * 8;
+      const uint4 wv = __ldg(&w[i]);
+      const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
+      const float4 m0 = __ldg(reinterpret_cast<const float4*>(w_amax + n0));
+      const float4 m1 = __ldg(reinterpret_cast<const float4*>(w_amax + n0 + 4));
+      const float amax[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const float wf = __uint_as_float((c & 1) ? (ww[c >> 1] & 0xFFFF0000u) : (ww[c >> 1] << 16));
+        const float gamma = amax[c] > 0.0f ? __fdiv_rn(6.0f, amax[c]) : 0.0f;
+        const float ws = __fmul_rn(wf, gamma);        // the value the forward quantised
+        y8[c] *= dge_factor(ws, expo, inv_k, dge_clip);
+      }
+    }
+    store8(dw, out_f32, off, y8);
+  }
 }
 
 }  // namespace
@@ -140,14 +198,20 @@ int launch_comp_fwd(fp4_ctx* ctx, cudaStream_t stream, const float* y1, const in
   return FP4_OK;
 }
 
-int launch_comp_wgrad_dge(fp4_ctx* ctx, cudaStream_t stream, const float* s, const int32_t* colptr, const int32_t* row,
+int launch_comp_wgrad_dge(fp4_ctx* ctx, cudaStream_t stream, float* s, const int32_t* colptr, const int32_t* row,
                           const float* val, const void* dy_bf16, const void* w_bf16, const float* w_amax, int64_t,
                           int64_t K, int64_t N, int dge_on, float dge_k, float dge_clip, void* dw, int out_f32) {
-  const dim3 grid(unsigned((N + COMP_COLS - 1) / COMP_COLS), unsigned((K + 7) / 8));
-  KernelScope scope(ctx, stream, KC_COMP_WGRAD, 1);
-  comp_wgrad_dge_kernel<<<grid, COMP_THREADS, 0, stream>>>(s, colptr, row, val, static_cast<const uint4*>(dy_bf16),
-                                                           static_cast<const uint4*>(w_bf16), w_amax, int(K), int(N),
-                                                           dge_on, dge_k, dge_clip, dw, out_f32);
+  KernelScope scope(ctx, stream, KC_COMP_WGRAD, colptr ? 2 : 1);
+  if (colptr) {
+    const dim3 grid(unsigned((N + COMP_COLS - 1) / COMP_COLS), unsigned(K));
+    comp_wgrad_accum_kernel<<<grid, COMP_THREADS, 0, stream>>>(s, colptr, row, val, static_cast<const uint4*>(dy_bf16),
+                                                               int(K), int(N));
+  }
+  const long long n_vec = (long long)K * N / 8;
+  long long blocks = (n_vec + 255) / 256;
+  if (blocks > 16LL * ctx->num_sms) blocks = 16LL * ctx->num_sms;
+  dge_store_kernel<<<int(blocks), 256, 0, stream>>>(s, static_cast<const uint4*>(w_bf16), w_amax, n_vec, int(N / 8),
+                                                    dge_on, dge_k, dge_clip, dw, out_f32);
   FP4_CUDA_TRY(cudaGetLastError());
   return FP4_OK;
 }

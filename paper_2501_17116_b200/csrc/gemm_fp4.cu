@@ -6,12 +6,15 @@
 // form of all three GEMMs of the layer (Fig. 2; Eq. 3; Appendix C.2).  The two de-scales are
 // applied to the accumulators in the epilogue, after the GEMM, as Appendix C.2 prescribes.
 //
-// Structure: persistent CTAs (one per SM), 128 x 256 output tile per CTA, six warps:
+// Structure: persistent CTAs (one per SM), 128 x BN output tile per CTA, six warps:
 //   warp 0      TMA producer: cp.async.bulk.tensor loads into 128-byte-swizzled shared memory,
 //               a ring of STAGES stages guarded by full/empty mbarriers;
 //   warp 1      allocates tensor memory and issues tcgen05.mma from one thread, fp32
 //               accumulators in tensor memory; tcgen05.commit releases stages and publishes tiles;
 //   warps 2..5  epilogue: tcgen05.ld the accumulators (one row per thread), de-scale, store.
+// Tensor memory holds two accumulator stages, so the epilogue of one tile runs under the MMAs of
+// the next.  512 columns are 2 x 256; the MXF4 flavour also needs a few columns for its block
+// scales, so its tile is 128 x 240 (2 x 240 accumulator columns + 16 scale columns).
 // Two MMA flavours are compiled:
 //   MXF4    kind::mxf4.block_scale, packed nibbles, K = 64 per instruction.  The method has no
 //           block scales, so every UE8M0 scale in tensor memory is 2^0: the product is unchanged.
@@ -26,17 +29,20 @@
 namespace {
 
 constexpr int BM = 128;
-constexpr int BN = 256;
 constexpr int STAGES = 4;
 constexpr int A_STAGE_BYTES = BM * 128;
-constexpr int B_STAGE_BYTES = BN * 128;
-constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr int NUM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
-constexpr int SF_COL_A = 256;            // MXF4 only: unit block scales live past the accumulator
-constexpr int SF_COL_B = 288;
+constexpr int ACC_STRIDE = 256;          // tensor-memory columns between the two accumulator stages
+constexpr int SF_COL_B = 240;            // MXF4 only: unit block scales in the gap behind stage 0
+constexpr int SF_COL_A = 248;
+constexpr int CHUNK = 16;                // accumulator columns per tcgen05.ld of the epilogue
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
-constexpr size_t SMEM_BYTES = 1024 + size_t(STAGES) * STAGE_BYTES + 256;
+
+__host__ __device__ constexpr int tile_n(int kind) { return kind == FP4_GEMM_F8F6F4 ? 256 : 240; }
+__host__ __device__ constexpr int b_stage_bytes(int kind) { return tile_n(kind) * 128; }
+__host__ __device__ constexpr int stage_bytes(int kind) { return A_STAGE_BYTES + b_stage_bytes(kind); }
+constexpr size_t smem_bytes(int kind) { return 1024 + size_t(STAGES) * stage_bytes(kind) + 256 + 2 * 256 * 4; }
 
 struct GemmArgs {
   int I, J;
@@ -126,18 +132,28 @@ __device__ __forceinline__ void mma_mxf4(uint32_t d_tmem, uint64_t a_desc, uint6
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate)
       : "memory");
 }
-// 32 lanes x 32 consecutive columns of 32-bit cells: thread t gets row t of the warp's lane quarter.
-__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&v)[32]) {
+// 32 lanes x 16 consecutive columns of 32-bit cells: thread t gets row t of the warp's lane quarter.
+__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&v)[16]) {
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
       : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
       : "r"(taddr)
       : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Barrier over the 128 epilogue threads that also ORs a flag, so that all four warps take the
+// same decision to give up (a warp must never be left alone at this barrier).
+__device__ __forceinline__ bool epilogue_bar_any(bool flag) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.or.pred p, 1, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"(uint32_t(flag))
+      : "memory");
+  return r != 0;
 }
 __device__ __forceinline__ void tmem_st_32x8(uint32_t taddr, uint32_t x) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1};" ::"r"(taddr), "r"(x)
@@ -155,19 +171,55 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
   d |= uint64_t(2) << 61;   // 128-byte swizzle
   return d;
 }
-// Instruction descriptors: M = 128, N = BN, both operands K-major, E2M1 x E2M1 -> fp32.
+// Instruction descriptors: M = 128, N = tile_n, both operands K-major, E2M1 x E2M1 -> fp32.
 __host__ __device__ constexpr uint32_t idesc_f8f6f4() {
-  return (1u << 4) | (5u << 7) | (5u << 10) | (uint32_t(BN >> 3) << 17) | (uint32_t(BM >> 4) << 24);
+  return (1u << 4) | (5u << 7) | (5u << 10) | (uint32_t(tile_n(FP4_GEMM_F8F6F4) >> 3) << 17) |
+         (uint32_t(BM >> 4) << 24);
 }
 __host__ __device__ constexpr uint32_t idesc_mxf4() {
-  return (1u << 7) | (1u << 10) | (uint32_t(BN >> 3) << 17) | (1u << 23) | (uint32_t(BM >> 4) << 24);
+  return (1u << 7) | (1u << 10) | (uint32_t(tile_n(FP4_GEMM_MXF4) >> 3) << 17) | (1u << 23) |
+         (uint32_t(BM >> 4) << 24);
+}
+
+// De-scale 16 accumulators of one row and store them (BF16: 32 bytes, float: 64 bytes).
+__device__ __forceinline__ void scale_store16(const uint32_t (&v)[16], float d_row, const float* s_dcol, void* out,
+                                              int out_f32, size_t off) {
+  float y[16];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const float4 dc = *reinterpret_cast<const float4*>(s_dcol + 4 * q);     // same address in every lane
+    y[4 * q + 0] = __fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 0]), d_row), dc.x);
+    y[4 * q + 1] = __fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 1]), d_row), dc.y);
+    y[4 * q + 2] = __fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 2]), d_row), dc.z);
+    y[4 * q + 3] = __fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 3]), d_row), dc.w);
+  }
+  if (out_f32) {
+    float4* dst = reinterpret_cast<float4*>(static_cast<float*>(out) + off);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) dst[j] = make_float4(y[4 * j], y[4 * j + 1], y[4 * j + 2], y[4 * j + 3]);
+  } else {
+    uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(out) + off);
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      uint32_t w[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(y[8 * j + 2 * q], y[8 * j + 2 * q + 1]);
+        w[q] = *reinterpret_cast<uint32_t*>(&h);
+      }
+      dst[j] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
 }
 
 template <int KIND>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const GemmArgs args) {
-  constexpr int NACC = (KIND == FP4_GEMM_F8F6F4) ? 2 : 1;
+  constexpr int NACC = 2;
+  constexpr int BN = tile_n(KIND);
+  constexpr int B_STAGE_BYTES = b_stage_bytes(KIND);
+  constexpr int STAGE_BYTES = stage_bytes(KIND);
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* smem_a = smem;
@@ -179,6 +231,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   uint64_t* final_bar = acc_empty + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(final_bar + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* s_dcol = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES + 256);   // [2][256] column de-scales
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -216,7 +269,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     // instruction expects inside these columns does not matter.
     if (warp >= 2) {
       const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
-      for (int c = 0; c < 64; c += 8) tmem_st_32x8(tmem_base + lane_base + SF_COL_A + c, 0x7F7F7F7Fu);
+      for (int c = 0; c < 16; c += 8) tmem_st_32x8(tmem_base + lane_base + SF_COL_B + c, 0x7F7F7F7Fu);
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -269,7 +322,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         ok = mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, args.status);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + uint32_t(acc * BN);
+        const uint32_t d_tmem = tmem_base + uint32_t(acc * ACC_STRIDE);
         for (int kb = 0; kb < args.num_k_blocks; ++kb) {
           ok = mbar_wait(&full_bar[stage], phase, abort_flag, args.status);
           if (!ok) break;
@@ -307,54 +360,46 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   } else {
     // ------------------------------------------------------------------ epilogue -----------
     const int quarter = warp & 3;               // the lane quarter of tensor memory this warp may read
+    const int et = threadIdx.x - 64;            // 0..127 among the epilogue threads
     int acc = 0;
     uint32_t acc_phase = 0;
+    uint32_t tile_parity = 0;
     for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
       const int m_blk = t % args.num_m_blocks;
       const int n_blk = t / args.num_m_blocks;
-      bool ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, args.status);
-      ok = __all_sync(0xFFFFFFFFu, ok);
-      if (!ok) break;
-      tc_fence_after();
+      // De-scales of this tile are fetched before the accumulators are awaited, under the MMAs.
       const int row = m_blk * BM + quarter * 32 + lane;
-      const float d_row = args.row_amax ? __fdiv_rn(args.row_amax[row], 6.0f) : 1.0f;
+      const float d_row = args.row_amax ? __fdiv_rn(__ldg(&args.row_amax[row]), 6.0f) : 1.0f;
+      float* dcol = s_dcol + tile_parity * 256;
+      for (int c = et; c < BN; c += 128) {
+        const int col = n_blk * BN + c;
+        dcol[c] = (args.col_amax && col < args.J) ? __fdiv_rn(__ldg(&args.col_amax[col]), 6.0f) : 1.0f;
+      }
+      const bool ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, args.status);
+      if (epilogue_bar_any(!ok)) break;            // also publishes dcol to the other warps
+      tc_fence_after();
+      const uint32_t t_base = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * ACC_STRIDE);
+      const size_t row_off = size_t(row) * size_t(args.J) + size_t(n_blk) * BN;
+      const int n_chunks = min(BN, args.J - n_blk * BN) / CHUNK;   // ragged last tile in N
+      uint32_t va[16], vb[16];
+      tmem_ld_32x16(t_base, va);
 #pragma unroll 1
-      for (int chunk = 0; chunk < BN / 32; ++chunk) {
-        const int col0 = n_blk * BN + chunk * 32;
-        if (col0 >= args.J) break;                // warp-uniform: ragged last tile in N
-        uint32_t v[32];
-        tmem_ld_32x32(tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * BN + chunk * 32), v);
-        const float d_col_lane = args.col_amax ? __fdiv_rn(args.col_amax[col0 + lane], 6.0f) : 1.0f;
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        float y[32];
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float d_col = __shfl_sync(0xFFFFFFFFu, d_col_lane, j);
-          y[j] = __fmul_rn(__fmul_rn(__uint_as_float(v[j]), d_row), d_col);
-        }
-        const size_t off = size_t(row) * size_t(args.J) + size_t(col0);
-        if (args.out_f32) {
-          float4* dst = reinterpret_cast<float4*>(static_cast<float*>(args.out) + off);
-#pragma unroll
-          for (int j = 0; j < 8; ++j) dst[j] = make_float4(y[4 * j], y[4 * j + 1], y[4 * j + 2], y[4 * j + 3]);
-        } else {
-          uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(args.out) + off);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            uint32_t w[4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              __nv_bfloat162 h = __floats2bfloat162_rn(y[8 * j + 2 * q], y[8 * j + 2 * q + 1]);
-              w[q] = *reinterpret_cast<uint32_t*>(&h);
-            }
-            dst[j] = make_uint4(w[0], w[1], w[2], w[3]);
-          }
+      for (int c = 0; c < n_chunks; c += 2) {
+        tmem_ld_wait();
+        if (c + 1 < n_chunks) tmem_ld_32x16(t_base + uint32_t((c + 1) * CHUNK), vb);
+        scale_store16(va, d_row, dcol + c * CHUNK, args.out, args.out_f32, row_off + size_t(c * CHUNK));
+        if (c + 1 < n_chunks) {
+          tmem_ld_wait();
+          if (c + 2 < n_chunks) tmem_ld_32x16(t_base + uint32_t((c + 2) * CHUNK), va);
+          scale_store16(vb, d_row, dcol + (c + 1) * CHUNK, args.out, args.out_f32,
+                        row_off + size_t((c + 1) * CHUNK));
         }
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[acc]);
       if (++acc == NACC) { acc = 0; acc_phase ^= 1u; }
+      tile_parity ^= 1u;
     }
   }
 
@@ -408,6 +453,7 @@ int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, c
   CUtensorMap map_a, map_b;
   int rc = make_codes_map(ctx, &map_a, a_codes, I, C, BM, gemm_kind);
   if (rc != FP4_OK) return rc;
+  const int BN = tile_n(gemm_kind);
   rc = make_codes_map(ctx, &map_b, b_codes, J, C, BN, gemm_kind);
   if (rc != FP4_OK) return rc;
 
@@ -420,7 +466,7 @@ int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, c
   args.num_n_blocks = int((J + BN - 1) / BN);
   // The transaction count of a copy is in bytes read from global memory: the byte-container form
   // fills a 48 KB stage from 24 KB of packed nibbles.
-  args.tx_bytes = gemm_kind == FP4_GEMM_F8F6F4 ? STAGE_BYTES / 2 : STAGE_BYTES;
+  args.tx_bytes = gemm_kind == FP4_GEMM_F8F6F4 ? stage_bytes(gemm_kind) / 2 : stage_bytes(gemm_kind);
   args.row_amax = row_amax;
   args.col_amax = col_amax;
   args.out = out;
@@ -431,13 +477,15 @@ int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, c
 
   KernelScope scope(ctx, stream, KC_GEMM, 1);
   if (gemm_kind == FP4_GEMM_F8F6F4) {
+    constexpr size_t kSmem = smem_bytes(FP4_GEMM_F8F6F4);
     FP4_CUDA_TRY(cudaFuncSetAttribute(gemm_fp4_kernel<FP4_GEMM_F8F6F4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      int(SMEM_BYTES)));
-    gemm_fp4_kernel<FP4_GEMM_F8F6F4><<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(map_a, map_b, args);
+                                      int(kSmem)));
+    gemm_fp4_kernel<FP4_GEMM_F8F6F4><<<grid, NUM_THREADS, kSmem, stream>>>(map_a, map_b, args);
   } else {
+    constexpr size_t kSmem = smem_bytes(FP4_GEMM_MXF4);
     FP4_CUDA_TRY(cudaFuncSetAttribute(gemm_fp4_kernel<FP4_GEMM_MXF4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      int(SMEM_BYTES)));
-    gemm_fp4_kernel<FP4_GEMM_MXF4><<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(map_a, map_b, args);
+                                      int(kSmem)));
+    gemm_fp4_kernel<FP4_GEMM_MXF4><<<grid, NUM_THREADS, kSmem, stream>>>(map_a, map_b, args);
   }
   FP4_CUDA_TRY(cudaGetLastError());
   return FP4_OK;
