@@ -44,6 +44,7 @@ extern "C" {
 #define FP4_ERR_CUDA       (-6)   /* a CUDA runtime / driver call failed                     */
 #define FP4_ERR_ARG        (-7)   /* an argument has an unsupported value                    */
 #define FP4_ERR_CAPACITY   (-8)   /* sparse_cap is below the guaranteed bound 2 * n_tail     */
+#define FP4_ERR_STATIC_LIMIT (-9) /* input larger than the fixed scratch of a *_static call  */
 
 /* bits of the device status word */
 #define FP4_DEV_SPARSE_OVERFLOW  1   /* more residual entries than sparse_cap                */
@@ -198,6 +199,34 @@ int fp4_profile_enable(fp4_ctx* ctx, int on);
 int fp4_profile_reset(fp4_ctx* ctx);
 int fp4_profile_read(fp4_ctx* ctx, int kernel_class, double* total_ms, int64_t* launches);
 int64_t fp4_launch_count(fp4_ctx* ctx);
+
+/*
+ * fp4_quantile_thresholds_static -- the two clamp thresholds of a tensor, for callers that
+ * must not allocate.  (The paper has no counterpart: this is a packaging variant of the
+ * threshold selection that fp4_quantize performs.)
+ *
+ * Who needs it: code that runs where device allocation is off limits -- inside a region that
+ * forbids cudaMalloc (a memory-pool-only framework, a real-time loop, a plugin that is handed
+ * tensors but no allocator) -- and that therefore cannot create an fp4_ctx, whose workspace is
+ * cudaMalloc'ed.  This call takes no context.  Its scratch (the 65536-bin histogram and the
+ * per-row extremes) is a fixed array inside the library image, 768 KB on every GPU that loads
+ * the library, held until the process exits.  The call itself performs no cudaMalloc, no
+ * cudaFree and calls no allocating library routine.
+ *
+ *   x_bf16      [rows x cols] BF16, device, 16-byte aligned; rows and cols multiples of 128
+ *   rows        at most FP4_STATIC_MAX_ROWS, else FP4_ERR_STATIC_LIMIT is returned and nothing
+ *               is enqueued
+ *   alpha       0.5 < alpha < 1
+ *   thresholds  device float[2]: receives {lo, hi}, bit-identical to what fp4_quantize writes
+ * The work is enqueued on `stream` for the current device.  The first call on each device also
+ * looks up the device address of the scratch array and sets a kernel attribute; make that first
+ * call before any stream capture begins.  All calls on a device share the one scratch array
+ * (it is cleared at the start of each call): two calls whose work overlaps on the GPU -- issued
+ * to different streams without ordering between them -- race and give wrong thresholds.
+ */
+#define FP4_STATIC_MAX_ROWS 65536
+int fp4_quantile_thresholds_static(void* stream, const void* x_bf16, int64_t rows, int64_t cols,
+                                   double alpha, float* thresholds);
 
 #ifdef __cplusplus
 }

@@ -22,7 +22,8 @@ FP4_DEV_TIMEOUT = 4
 EXPORTS = ("fp4_create", "fp4_destroy", "fp4_workspace_bytes", "fp4_status_string", "fp4_quantize",
            "fp4_gemm", "fp4_linear_fwd", "fp4_linear_bwd", "fp4_step_host_workspace_bytes",
            "fp4_linear_step_host", "fp4_profile_enable", "fp4_profile_reset", "fp4_profile_read",
-           "fp4_launch_count")
+           "fp4_launch_count", "fp4_quantile_thresholds_static")
+FP4_STATIC_MAX_ROWS = 65536
 KERNEL_CLASSES = ("gemm", "select", "encode", "absmax", "sparse", "comp_fwd", "comp_wgrad_dge")
 
 
@@ -82,6 +83,8 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.fp4_profile_read.restype = C.c_int
     lib.fp4_launch_count.argtypes = [vp]
     lib.fp4_launch_count.restype = C.c_int64
+    lib.fp4_quantile_thresholds_static.argtypes = [vp, vp, i64, i64, C.c_double, vp]
+    lib.fp4_quantile_thresholds_static.restype = C.c_int
     if path == LIB_PATH:
         _lib = lib
     return lib
@@ -268,3 +271,18 @@ def fp4_linear_step_host(ctx: Context, A_host: torch.Tensor, W_host: torch.Tenso
                                         _ptr(Y_host), _ptr(dA_host), _ptr(dW_host),
                                         C.byref(st) if read_status else None))
     return st.value
+
+
+def fp4_quantile_thresholds_static(x: torch.Tensor, alpha: float, out: torch.Tensor | None = None) -> torch.Tensor:
+    """{lo, hi} of `x` through the entry point that allocates nothing on the device.
+
+    For callers that may not call cudaMalloc (and so cannot own a Context): the scratch is a
+    fixed array inside the library.  `out` (float32[2] on the device) may be passed so that this
+    wrapper does not allocate either.  Calls on one device must not overlap on the GPU.
+    """
+    assert x.dtype == torch.bfloat16 and x.is_cuda and x.is_contiguous() and x.dim() == 2
+    if out is None:
+        out = torch.empty(2, dtype=torch.float32, device=x.device)
+    _check(load_library().fp4_quantile_thresholds_static(_stream(), _ptr(x), x.shape[0], x.shape[1], float(alpha),
+                                                         _ptr(out)))
+    return out

@@ -62,6 +62,7 @@ const char* fp4_status_string(int code) {
     case FP4_ERR_CUDA: return "a CUDA call failed";
     case FP4_ERR_ARG: return "an argument has an unsupported value";
     case FP4_ERR_CAPACITY: return "sparse_cap is below 2 * n_tail";
+    case FP4_ERR_STATIC_LIMIT: return "input exceeds the fixed scratch of the allocation-free entry point";
     default: return "unknown status";
   }
 }

@@ -668,3 +668,65 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
   FP4_CUDA_TRY(cudaGetLastError());
   return FP4_OK;
 }
+
+// ------------------------------------------------------------------------------------------
+// Quantile thresholds without any allocation
+// ------------------------------------------------------------------------------------------
+// Scratch of fp4_quantile_thresholds_static: the 65536-bin histogram followed by the row
+// extremes of up to FP4_STATIC_MAX_ROWS rows.  It lives in the library image: every GPU that
+// loads the library holds these 768 KB until the process exits.
+namespace {
+constexpr size_t STATIC_HIST_BYTES = 65536 * sizeof(uint32_t);
+constexpr size_t STATIC_SCRATCH_BYTES = STATIC_HIST_BYTES + 2 * size_t(FP4_STATIC_MAX_ROWS) * sizeof(int);
+constexpr int STATIC_MAX_DEVICES = 64;
+}  // namespace
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
+
+extern "C" int fp4_quantile_thresholds_static(void* stream, const void* x_bf16, int64_t rows, int64_t cols,
+                                              double alpha, float* thresholds) {
+  // In host code `g_static_scratch` is only a handle; the device address of this device's copy
+  // is looked up once per device and cached.
+  static void* scratch_of_device[STATIC_MAX_DEVICES] = {};
+  static int sms_of_device[STATIC_MAX_DEVICES] = {};
+  if (!x_bf16 || !thresholds) return FP4_ERR_NULL;
+  if (rows <= 0 || cols <= 0 || (rows % 128) || (cols % 128) || rows * cols >= (int64_t(1) << 31))
+    return FP4_ERR_SHAPE;
+  if (rows > FP4_STATIC_MAX_ROWS) return FP4_ERR_STATIC_LIMIT;
+  if (!(alpha > 0.5 && alpha < 1.0)) return FP4_ERR_ALPHA;
+  if (reinterpret_cast<uintptr_t>(x_bf16) & 15) return FP4_ERR_ALIGN;
+  const long long n = (long long)rows * cols;
+  const long long n_tail = llround((1.0 - alpha) * double(n));
+  if (2 * n_tail >= n) return FP4_ERR_ALPHA;
+
+  int device = -1;
+  FP4_CUDA_TRY(cudaGetDevice(&device));
+  if (device < 0 || device >= STATIC_MAX_DEVICES) return FP4_ERR_ARG;
+  if (!scratch_of_device[device]) {
+    void* ptr = nullptr;
+    FP4_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
+    int sms = 0;
+    FP4_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+    FP4_CUDA_TRY(cudaFuncSetAttribute(hist_rowminmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      HIST_WORDS * 4));
+    sms_of_device[device] = sms;
+    scratch_of_device[device] = ptr;
+  }
+  unsigned char* base = static_cast<unsigned char*>(scratch_of_device[device]);
+  uint32_t* hist = reinterpret_cast<uint32_t*>(base);
+  int* row_max = reinterpret_cast<int*>(base + STATIC_HIST_BYTES);
+  int* row_min = row_max + FP4_STATIC_MAX_ROWS;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // The array keeps what the previous call left: the histogram must start from zero and the
+  // row extremes from their identities.
+  FP4_CUDA_TRY(cudaMemsetAsync(hist, 0, STATIC_HIST_BYTES, st));
+  init_row_extremes_kernel<<<int((rows + 255) / 256), 256, 0, st>>>(row_max, row_min, int(rows));
+  const long long n_vec = n / 8;
+  long long blocks = (n_vec + HIST_THREADS - 1) / HIST_THREADS;
+  if (blocks > sms_of_device[device]) blocks = sms_of_device[device];
+  hist_rowminmax_kernel<<<int(blocks), HIST_THREADS, HIST_WORDS * 4, st>>>(static_cast<const uint4*>(x_bf16), n_vec,
+                                                                          int(cols / 8), hist, row_max, row_min);
+  select_thresholds_kernel<<<1, 1024, 0, st>>>(hist, n, n_tail, thresholds);
+  FP4_CUDA_TRY(cudaGetLastError());
+  return FP4_OK;
+}
