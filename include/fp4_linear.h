@@ -209,7 +209,7 @@ int64_t fp4_launch_count(fp4_ctx* ctx);
  * forbids cudaMalloc (a memory-pool-only framework, a real-time loop, a plugin that is handed
  * tensors but no allocator) -- and that therefore cannot create an fp4_ctx, whose workspace is
  * cudaMalloc'ed.  This call takes no context.  Its scratch (the 65536-bin histogram and the
- * per-row extremes) is a fixed array inside the library image, 768 KB on every GPU that loads
+ * per-row extremes) is a fixed array inside the library image, 769 KB on every GPU that loads
  * the library, held until the process exits.  The call itself performs no cudaMalloc, no
  * cudaFree and calls no allocating library routine.
  *

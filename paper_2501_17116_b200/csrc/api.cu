@@ -256,32 +256,43 @@ namespace {
 int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_bf16, const void* W_bf16,
                     const fp4_qtensor* savedA, const fp4_qtensor* savedW, int64_t M, int64_t K, int64_t N, int dge_on,
                     float dge_k, float dge_clip, int gemm_kind, void* dA, void* dW, int out_f32, int32_t* status) {
-  float* s = arena.take<float>(size_t(K) * size_t(N));
-  uint8_t* g_codes = arena.take<uint8_t>(size_t(M) * size_t(N) / 2);
-  float* g_amax = arena.take<float>(size_t(M > N ? M : N));
+  float* s = dW ? arena.take<float>(size_t(K) * size_t(N)) : nullptr;
+  uint8_t* g1_codes = dA ? arena.take<uint8_t>(size_t(M) * size_t(N) / 2) : nullptr;   // dY (.) d_W, token-wise
+  uint8_t* g2_codes = dW ? arena.take<uint8_t>(size_t(M) * size_t(N) / 2) : nullptr;   // dY (.) d_A, channel-wise
+  float* g1_amax = arena.take<float>(size_t(M));
+  float* g2_amax = arena.take<float>(size_t(N));
   if (!arena.ok) return FP4_ERR_WORKSPACE;
   Arena q_arena(arena.base + arena.off, arena.size - arena.off);
   int rc;
 
-  if (dA) {
-    // dgrad: G' = dY (.) d_W[n], token-wise codes [M x N/2]; dA = d_G'[m] * sum_n G'[m,n] Wq[k,n].
+  // dgrad operand: G' = dY (.) d_W[n], token-wise codes [M x N/2].
+  // wgrad operand: G'' = dY (.) d_A[m], channel-wise codes transposed [N x M/2].
+  if (dA && dW) {
+    Arena a = q_arena;
+    rc = launch_quantize_dual(ctx, st, a, dY_bf16, M, N, savedW->amax, savedA->amax, g1_codes, g1_amax, g2_codes,
+                              g2_amax);
+    if (rc != FP4_OK) return rc;
+  } else if (dA) {
     fp4_qtensor g = {};
-    g.rows = M; g.cols = N; g.codes = g_codes; g.amax = g_amax;
+    g.rows = M; g.cols = N; g.codes = g1_codes; g.amax = g1_amax;
     Arena a = q_arena;
     rc = launch_quantize(ctx, st, a, dY_bf16, M, N, /*scale_axis=*/0, 1.0, savedW->amax, 1, &g, status);
     if (rc != FP4_OK) return rc;
-    rc = launch_gemm_fp4(ctx, st, g_codes, savedW->codes, M, K, N, g_amax, nullptr, dA, out_f32, gemm_kind, status);
-    if (rc != FP4_OK) return rc;
-  }
-  if (dW) {
-    // wgrad: G'' = dY (.) d_A[m], channel-wise codes transposed [N x M/2];
-    // S[k,n] = d_G''[n] * sum_m Aq[m,k] G''[m,n], then the compensation and the DGE factor.
+  } else {
     fp4_qtensor g = {};
-    g.rows = M; g.cols = N; g.codes_t = g_codes; g.amax = g_amax;
+    g.rows = M; g.cols = N; g.codes_t = g2_codes; g.amax = g2_amax;
     Arena a = q_arena;
     rc = launch_quantize(ctx, st, a, dY_bf16, M, N, /*scale_axis=*/1, 1.0, savedA->amax, 1, &g, status);
     if (rc != FP4_OK) return rc;
-    rc = launch_gemm_fp4(ctx, st, savedA->codes_t, g_codes, K, N, M, nullptr, g_amax, s, 1, gemm_kind, status);
+  }
+  if (dA) {
+    // dA = d_G'[m] * sum_n G'[m,n] Wq[k,n]
+    rc = launch_gemm_fp4(ctx, st, g1_codes, savedW->codes, M, K, N, g1_amax, nullptr, dA, out_f32, gemm_kind, status);
+    if (rc != FP4_OK) return rc;
+  }
+  if (dW) {
+    // S[k,n] = d_G''[n] * sum_m Aq[m,k] G''[m,n], then the compensation and the DGE factor.
+    rc = launch_gemm_fp4(ctx, st, savedA->codes_t, g2_codes, K, N, M, nullptr, g2_amax, s, 1, gemm_kind, status);
     if (rc != FP4_OK) return rc;
     rc = launch_comp_wgrad_dge(ctx, st, s, savedA->csc_colptr, savedA->csc_row, savedA->csc_val, dY_bf16, W_bf16,
                                savedW->amax, M, K, N, dge_on, dge_k, dge_clip, dW, out_f32);

@@ -100,6 +100,13 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
                     int64_t cols, int scale_axis, double alpha, const float* prescale,
                     int prescale_is_amax, fp4_qtensor* out, int32_t* status);
 
+// dY for both backward GEMMs in one read: row-scaled codes of x (.) (amax_col_pre / 6) with their
+// row amax, and column-scaled transposed codes of x (.) (amax_row_pre / 6) with their column amax.
+int launch_quantize_dual(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void* x_bf16, int64_t rows,
+                         int64_t cols, const float* amax_col_pre, const float* amax_row_pre,
+                         uint8_t* codes_rows, float* amax_rows_out, uint8_t* codes_t_cols,
+                         float* amax_cols_out);
+
 // Sparse compensation and epilogues (compensate.cu)
 // y[m,:] = store( y1[m,:] + sum_{entries of row m} val * dense[col,:] )
 int launch_comp_fwd(fp4_ctx* ctx, cudaStream_t stream, const float* y1, const int32_t* rowptr,

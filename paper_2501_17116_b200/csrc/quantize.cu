@@ -7,22 +7,27 @@
 //                         memory) + signed max / min of every row
 //     2. select           cumulative counts -> the two order statistics lo, hi (bit exact)
 //     3. encode           one read: clamp, per-row scale from the clamped row extremes, Q, both
-//                         nibble layouts, and a 1-bit-per-element mask of the clamped entries
-//     4. mask -> CSR/CSC  counts, prefix sums and ordered fills driven by the mask (1/16 of the
-//                         tensor); values are gathered from the few marked entries
+//                         nibble layouts, a 1-bit-per-element mask of the clamped entries, and
+//                         the number of clamped entries per row and per (64-row strip, column)
+//     4. mask -> CSR/CSC  prefix sums of those counts and ordered fills driven by the mask (1/16
+//                         of the tensor); values are gathered from the few marked entries
 //   without clamping (weights, output gradients)
-//     1. absmax           one read: max |x| per row or per column (after the optional prescale)
+//     1. absmax           one read: max |x| per row and / or per column (after the prescale)
 //     2. encode           one read
+// The "dual" mode serves the backward pass: one read of dY yields the token-wise codes of
+// dY (.) d_W[n] and the channel-wise codes of dY (.) d_A[m].
 #include "common.cuh"
 
 namespace {
 
 constexpr int HIST_THREADS = 1024;
 constexpr int HIST_WORDS = 32768;                 // two 16-bit counters per word
-constexpr int ENC_TM = 64;                        // tile rows of the encoder
+constexpr int ENC_TM = 64;                        // tile rows of the encoder (= one strip)
 constexpr int ENC_TK = 256;                       // tile columns
 constexpr int ENC_THREADS = 256;
-constexpr int MAX_SPLITS = 64;
+constexpr int SELECT_BLOCKS = 64;                 // 64 x 1024 histogram positions
+
+enum Mode { MODE_ROWS = 0, MODE_COLS = 1, MODE_DUAL = 2 };
 
 __device__ __forceinline__ int float_to_ordered(float f) {
   const int b = __float_as_int(f);
@@ -45,6 +50,20 @@ __global__ void init_row_extremes_kernel(int* row_max, int* row_min, int rows) {
   }
 }
 
+// Everything the clamping path accumulates into starts from its identity.
+__global__ void init_occ_kernel(uint32_t* hist, int* row_max, int* row_min, int* row_cnt, int rows,
+                                unsigned* ticket) {
+  const int stride = gridDim.x * blockDim.x;
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  for (int i = t; i < 65536; i += stride) hist[i] = 0;
+  for (int i = t; i < rows; i += stride) {
+    row_max[i] = INT_MIN;
+    row_min[i] = INT_MAX;
+    row_cnt[i] = 0;
+  }
+  if (t == 0) *ticket = 0;
+}
+
 // Shared-memory counters are 16-bit pairs.  A counter that reaches 0x8000 is moved to the global
 // histogram by the thread that made it so.  Between two block barriers the block adds at most
 // 8192 elements, so a counter stays below 0xC000 and never carries into its neighbour.
@@ -58,16 +77,20 @@ __device__ __forceinline__ void bump(uint32_t* h, uint32_t* ghist, uint32_t bits
 }
 
 __global__ void __launch_bounds__(HIST_THREADS, 1)
-hist_rowminmax_kernel(const uint4* __restrict__ x, long long n_vec, int vec_per_row, uint32_t* __restrict__ ghist,
+hist_rowminmax_kernel(const uint4* __restrict__ x, long long n_vec_ll, int vec_per_row, uint32_t* __restrict__ ghist,
                       int* __restrict__ row_max, int* __restrict__ row_min) {
   extern __shared__ uint32_t h[];
   for (int i = threadIdx.x; i < HIST_WORDS; i += HIST_THREADS) h[i] = 0;
   __syncthreads();
-  const long long stride = (long long)gridDim.x * HIST_THREADS;
-  long long i = (long long)blockIdx.x * HIST_THREADS + threadIdx.x;
+  const int n_vec = int(n_vec_ll);                 // rows * cols < 2^31
+  const int stride = gridDim.x * HIST_THREADS;
+  int i = blockIdx.x * HIST_THREADS + threadIdx.x;
+  // row of vector i, advanced incrementally (one division per thread)
+  int row = i / vec_per_row, rem = i - row * vec_per_row;
+  const int row_step = stride / vec_per_row, rem_step = stride - row_step * vec_per_row;
   uint4 nxt = make_uint4(0, 0, 0, 0);
   if (i < n_vec) nxt = __ldg(&x[i]);
-  for (long long base = (long long)blockIdx.x * HIST_THREADS; base < n_vec; base += stride, i += stride) {
+  for (int base = blockIdx.x * HIST_THREADS; base < n_vec; base += stride) {
     const uint4 v = nxt;
     const bool valid = i < n_vec;
     if (i + stride < n_vec) nxt = __ldg(&x[i + stride]);
@@ -88,11 +111,14 @@ hist_rowminmax_kernel(const uint4* __restrict__ x, long long n_vec, int vec_per_
       kmax = __reduce_max_sync(group, kmax);
       kmin = __reduce_min_sync(group, kmin);
       if ((threadIdx.x & 15) == 0) {
-        const int row = int(i / vec_per_row);
         atomicMax(&row_max[row], kmax);
         atomicMin(&row_min[row], kmin);
       }
     }
+    i += stride;
+    row += row_step;
+    rem += rem_step;
+    if (rem >= vec_per_row) { rem -= vec_per_row; ++row; }
     __syncthreads();
   }
   for (int idx = threadIdx.x; idx < HIST_WORDS; idx += HIST_THREADS) {
@@ -109,104 +135,162 @@ hist_rowminmax_kernel(const uint4* __restrict__ x, long long n_vec, int vec_per_
 // 0x8000 (-0), p >= 32768 the non-negative patterns from 0x0000 up.
 __device__ __forceinline__ uint32_t pos_to_bits(int p) { return p < 32768 ? uint32_t(0xFFFF - p) : uint32_t(p - 32768); }
 
-__global__ void __launch_bounds__(1024, 1)
-select_thresholds_kernel(const uint32_t* __restrict__ ghist, long long n, long long n_tail, float* thresholds) {
-  __shared__ long long part[1024];
-  __shared__ int found[2];
-  const int t = threadIdx.x;
-  long long s = 0;
-  for (int p = 64 * t; p < 64 * t + 64; ++p) s += ghist[pos_to_bits(p)];
-  part[t] = s;
-  __syncthreads();
-  // inclusive scan over the 1024 partial sums (Hillis-Steele; runs once per call)
-  for (int off = 1; off < 1024; off <<= 1) {
-    const long long add = t >= off ? part[t - off] : 0;
-    __syncthreads();
-    part[t] += add;
-    __syncthreads();
+// Inclusive scan of one value per thread over a block of 1024 threads.
+__device__ __forceinline__ long long block_scan_1024(long long v, long long* warp_tot /*[32] shared*/) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const long long up = __shfl_up_sync(0xFFFFFFFFu, v, off);
+    if (lane >= off) v += up;
   }
-  const long long before = part[t] - s;            // entries in positions below 64 t
+  if (lane == 31) warp_tot[warp] = v;
+  __syncthreads();
+  if (warp == 0) {
+    long long t = warp_tot[lane];
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const long long up = __shfl_up_sync(0xFFFFFFFFu, t, off);
+      if (lane >= off) t += up;
+    }
+    warp_tot[lane] = t;
+  }
+  __syncthreads();
+  if (warp > 0) v += warp_tot[warp - 1];
+  return v;
+}
+
+// 64 blocks sum 1024 positions each; the block that finishes last (a ticket, no waiting) locates
+// the two ranks among the segment sums and then inside their segments.
+__global__ void __launch_bounds__(1024, 1)
+select_thresholds_kernel(const uint32_t* __restrict__ ghist, long long n, long long n_tail, float* thresholds,
+                         unsigned long long* seg_sum, unsigned* ticket) {
+  __shared__ long long warp_tot[32];
+  __shared__ long long s_before[2];
+  __shared__ int s_seg[2];
+  __shared__ int s_last;
+  const int t = threadIdx.x;
+  const long long c = ghist[pos_to_bits(blockIdx.x * 1024 + t)];
+  const long long incl = block_scan_1024(c, warp_tot);
+  if (t == 1023) {
+    seg_sum[blockIdx.x] = (unsigned long long)incl;
+    __threadfence();
+    s_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
   const long long rank[2] = {n_tail, n - 1 - n_tail};
-  for (int q = 0; q < 2; ++q) {
-    if (rank[q] >= before && rank[q] < before + s) {
-      long long cum = before;
-      for (int p = 64 * t; p < 64 * t + 64; ++p) {
-        cum += ghist[pos_to_bits(p)];
-        if (cum > rank[q]) { found[q] = p; break; }
+  if (t == 0) {
+    long long run = 0;
+    int q = 0;
+    for (int sgm = 0; sgm < int(gridDim.x) && q < 2; ++sgm) {
+      const long long sz = (long long)reinterpret_cast<volatile unsigned long long*>(seg_sum)[sgm];
+      while (q < 2 && rank[q] < run + sz) {
+        s_seg[q] = sgm;
+        s_before[q] = run;
+        ++q;
       }
+      run += sz;
     }
   }
   __syncthreads();
-  if (t < 2) {
-    uint32_t bits = pos_to_bits(found[t]);
-    if (bits == 0x8000u) bits = 0;                 // thresholds are real numbers: -0 is +0
-    thresholds[t] = __uint_as_float(bits << 16);
+  for (int q = 0; q < 2; ++q) {
+    const int p = s_seg[q] * 1024 + t;
+    const long long cq = ghist[pos_to_bits(p)];
+    __syncthreads();                                  // warp_tot is reused
+    const long long iq = s_before[q] + block_scan_1024(cq, warp_tot);
+    if (rank[q] >= iq - cq && rank[q] < iq) {         // exactly one thread
+      uint32_t bits = pos_to_bits(p);
+      if (bits == 0x8000u) bits = 0;                  // thresholds are real numbers: -0 is +0
+      thresholds[q] = __uint_as_float(bits << 16);
+    }
   }
 }
 
 // ------------------------------------------------------------------------------------------
 // absmax without clamping
 // ------------------------------------------------------------------------------------------
-__device__ __forceinline__ float prescale_value(const float* p, int idx) { return __ldg(&p[idx]); }
-
 // d[i] = amax[i] / 6 rounded once: the de-scale vector of a quantised operand, used as a prescale
 __global__ void descale_kernel(const float* __restrict__ amax, int n, float* __restrict__ d) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) d[i] = __fdiv_rn(amax[i], 6.0f);
 }
 
-// one scale per row: flat sweep, 16-lane groups cover 128 consecutive elements of one row
-template <bool PRESCALE>
-__global__ void __launch_bounds__(256)
-absmax_rows_kernel(const uint4* __restrict__ x, long long n_vec, int vec_per_row, const float* __restrict__ prescale,
-                   uint32_t* __restrict__ vec_amax) {
-  const long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += stride) {
-    const uint4 v = __ldg(&x[i]);
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    const int row = int(i / vec_per_row);
-    const int c0 = int(i - (long long)row * vec_per_row) * 8;
-    float m = 0.0f;
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      float a = bf16_lo(w[q]), b = bf16_hi(w[q]);
-      if (PRESCALE) {
-        a = __fmul_rn(a, prescale_value(prescale, c0 + 2 * q));
-        b = __fmul_rn(b, prescale_value(prescale, c0 + 2 * q + 1));
-      }
-      m = fmaxf(m, fmaxf(fabsf(a), fabsf(b)));
-    }
-    const unsigned group = (threadIdx.x & 16) ? 0xFFFF0000u : 0x0000FFFFu;
-    const uint32_t gm = __reduce_max_sync(group, __float_as_uint(m));   // non-negative floats order as integers
-    if ((threadIdx.x & 15) == 0) atomicMax(&vec_amax[row], gm);
-  }
-}
+struct AbsmaxArgs {
+  const uint4* x;
+  int rows, cols;
+  const float* pre_col;         // multiplies along columns before the row-wise maximum (or null)
+  const float* pre_row;         // multiplies along rows before the column-wise maximum (or null)
+  int pre_is_amax;              // the two vectors hold amax values: use amax / 6 and store it
+  float* d_col_out;             // dual mode: the de-scale vectors actually used, for the encoder
+  float* d_row_out;
+  uint32_t* amax_rows;          // float bits, zero-initialised (non-negative floats order as integers)
+  uint32_t* amax_cols;
+};
 
-// one scale per column: each thread owns 8 adjacent columns over a strip of rows
-template <bool PRESCALE>
-__global__ void __launch_bounds__(256)
-absmax_cols_kernel(const uint4* __restrict__ x, int rows, int vec_per_row, int rows_per_strip,
-                   const float* __restrict__ prescale, uint32_t* __restrict__ vec_amax) {
-  const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= vec_per_row) return;
-  const int r0 = blockIdx.y * rows_per_strip;
-  const int r1 = min(rows, r0 + rows_per_strip);
-  float m[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-#pragma unroll 4
-  for (int r = r0; r < r1; ++r) {
-    const uint4 v = __ldg(&x[(long long)r * vec_per_row + j]);
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    const float p = PRESCALE ? prescale_value(prescale, r) : 1.0f;
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      float a = bf16_lo(w[q]), b = bf16_hi(w[q]);
-      if (PRESCALE) { a = __fmul_rn(a, p); b = __fmul_rn(b, p); }
-      m[2 * q] = fmaxf(m[2 * q], fabsf(a));
-      m[2 * q + 1] = fmaxf(m[2 * q + 1], fabsf(b));
+// Tile of 64 rows x 256 columns per block, same thread mapping as the encoder: warp w owns rows
+// 8w..8w+7, lane l the 8 columns 8l..8l+7.
+template <int MODE>
+__global__ void __launch_bounds__(ENC_THREADS)
+absmax_tile_kernel(const AbsmaxArgs a) {
+  __shared__ float s_pcol[ENC_TK];
+  __shared__ float s_prow[ENC_TM];
+  __shared__ uint32_t s_cmax[8][ENC_TK];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int row0 = blockIdx.y * ENC_TM, col0 = blockIdx.x * ENC_TK;
+  const int vec_per_row = a.cols >> 3;
+  constexpr bool want_rows = MODE != MODE_COLS, want_cols = MODE != MODE_ROWS;
+  if (want_rows && a.pre_col) {
+    const int c = col0 + tid;
+    if (c < a.cols) {
+      const float v = __ldg(&a.pre_col[c]);
+      s_pcol[tid] = a.pre_is_amax ? __fdiv_rn(v, 6.0f) : v;
+      if (a.d_col_out && blockIdx.y == 0) a.d_col_out[c] = s_pcol[tid];
     }
   }
+  if (want_cols && a.pre_row && tid < ENC_TM) {
+    const float v = __ldg(&a.pre_row[row0 + tid]);
+    s_prow[tid] = a.pre_is_amax ? __fdiv_rn(v, 6.0f) : v;
+    if (a.d_row_out && blockIdx.x == 0) a.d_row_out[row0 + tid] = s_prow[tid];
+  }
+  __syncthreads();
+  const int col = col0 + 8 * lane;
+  const bool in_cols = col < a.cols;
+  uint4 v[8];
 #pragma unroll
-  for (int c = 0; c < 8; ++c) atomicMax(&vec_amax[8 * j + c], __float_as_uint(m[c]));
+  for (int r = 0; r < 8; ++r) {
+    v[r] = make_uint4(0, 0, 0, 0);
+    if (in_cols) v[r] = __ldg(&a.x[(long long)(row0 + 8 * warp + r) * vec_per_row + (col >> 3)]);
+  }
+  float pc[8];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) pc[c] = (want_rows && a.pre_col && in_cols) ? s_pcol[8 * lane + c] : 1.0f;
+  float cm[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+    const uint32_t w[4] = {v[r].x, v[r].y, v[r].z, v[r].w};
+    const float pr = (want_cols && a.pre_row) ? s_prow[8 * warp + r] : 1.0f;
+    float rm = 0.0f;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      const float f = (c & 1) ? bf16_hi(w[c >> 1]) : bf16_lo(w[c >> 1]);
+      if (want_rows) rm = fmaxf(rm, fabsf(a.pre_col ? __fmul_rn(f, pc[c]) : f));
+      if (want_cols) cm[c] = fmaxf(cm[c], fabsf(a.pre_row ? __fmul_rn(f, pr) : f));
+    }
+    if (want_rows) {
+      const uint32_t g = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(rm));
+      if (lane == 0) atomicMax(&a.amax_rows[row0 + 8 * warp + r], g);
+    }
+  }
+  if (want_cols) {
+#pragma unroll
+    for (int c = 0; c < 8; ++c) s_cmax[warp][8 * lane + c] = __float_as_uint(cm[c]);
+    __syncthreads();
+    uint32_t m = 0;
+#pragma unroll
+    for (int w8 = 0; w8 < 8; ++w8) m = max(m, s_cmax[w8][tid]);
+    if (col0 + tid < a.cols) atomicMax(&a.amax_cols[col0 + tid], m);
+  }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -264,54 +348,68 @@ __device__ __forceinline__ void transpose8x8_nibbles(uint32_t (&r)[8]) {
 struct EncodeArgs {
   const uint4* x;
   int rows, cols;
-  const float* prescale;
-  const uint32_t* vec_amax;     // no clamp: max |x| per scaled vector (float bits)
+  const float* pre_col;         // prescale along columns (row-scaled output) or null
+  const float* pre_row;         // prescale along rows (column-scaled output) or null
+  const uint32_t* amax_rows;    // no clamp: max |x| per row (float bits)
+  const uint32_t* amax_cols;    // max |x| per column
   const int* row_max;           // clamp: ordered-int row extremes
   const int* row_min;
   const float* thresholds;      // clamp: lo, hi
-  uint32_t* codes;              // [rows x cols/8] words or null
-  uint32_t* codes_t;            // [cols x rows/8] words or null
-  float* amax_out;
+  uint32_t* codes;              // [rows x cols/8] words or null   (row-scaled in dual mode)
+  uint32_t* codes_t;            // [cols x rows/8] words or null   (column-scaled in dual mode)
+  float* amax_out_rows;
+  float* amax_out_cols;
   uint8_t* mask;                // clamp: [rows x cols/8] bytes
+  int* row_cnt;                 // clamp: clamped entries per row (zero-initialised)
+  uint8_t* strip_cnt;           // clamp: [rows/64 x cols] clamped entries per (strip, column)
 };
 
-// AXIS 0: one scale per row; AXIS 1: one per column.  OCC implies AXIS 0 and no prescale.
-template <int AXIS, bool OCC, bool PRESCALE>
+// MODE_ROWS: one scale per row -> codes and / or codes_t.  MODE_COLS: one scale per column.
+// MODE_DUAL: codes hold the row-scaled tensor x (.) pre_col, codes_t the column-scaled tensor
+// x (.) pre_row.  OCC (clamping) implies MODE_ROWS without prescale.
+template <int MODE, bool OCC, bool PRESCALE>
 __global__ void __launch_bounds__(ENC_THREADS)
 encode_kernel(const EncodeArgs a) {
-  __shared__ float s_gamma[ENC_TK];
-  __shared__ float s_pre[ENC_TM];
+  __shared__ float s_gcol[ENC_TK];
+  __shared__ float s_grow[ENC_TM];
+  __shared__ float s_prow[ENC_TM];
   __shared__ uint32_t tile_t[8 * 8 * 32];
+  __shared__ int s_colcnt[OCC ? ENC_TK : 1];
   const int tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31;
   const int row0 = blockIdx.y * ENC_TM;
   const int col0 = blockIdx.x * ENC_TK;
   const int vec_per_row = a.cols >> 3;
+  constexpr bool ROW_SCALED = MODE != MODE_COLS;      // a row-scaled output exists
+  constexpr bool COL_SCALED = MODE != MODE_ROWS;
   float lo = 0.f, hi = 0.f;
-  if (OCC) { lo = a.thresholds[0]; hi = a.thresholds[1]; }
+  if (OCC) {
+    lo = a.thresholds[0];
+    hi = a.thresholds[1];
+    s_colcnt[tid] = 0;
+  }
 
-  if (AXIS == 0) {
-    if (tid < ENC_TM) {
-      const int r = row0 + tid;
-      float amax;
-      if (OCC) {
-        const float mx = fminf(fmaxf(ordered_to_float(a.row_max[r]), lo), hi);
-        const float mn = fminf(fmaxf(ordered_to_float(a.row_min[r]), lo), hi);
-        amax = fmaxf(fabsf(mx), fabsf(mn));
-      } else {
-        amax = __uint_as_float(a.vec_amax[r]);
-      }
-      s_gamma[tid] = amax > 0.0f ? __fdiv_rn(6.0f, amax) : 0.0f;
-      if (blockIdx.x == 0) a.amax_out[r] = amax;
+  if (ROW_SCALED && tid < ENC_TM) {
+    const int r = row0 + tid;
+    float amax;
+    if (OCC) {
+      const float mx = fminf(fmaxf(ordered_to_float(a.row_max[r]), lo), hi);
+      const float mn = fminf(fmaxf(ordered_to_float(a.row_min[r]), lo), hi);
+      amax = fmaxf(fabsf(mx), fabsf(mn));
+    } else {
+      amax = __uint_as_float(a.amax_rows[r]);
     }
-  } else {
+    s_grow[tid] = amax > 0.0f ? __fdiv_rn(6.0f, amax) : 0.0f;
+    if (blockIdx.x == 0) a.amax_out_rows[r] = amax;
+  }
+  if (COL_SCALED) {
     const int c = col0 + tid;
     if (c < a.cols) {
-      const float amax = __uint_as_float(a.vec_amax[c]);
-      s_gamma[tid] = amax > 0.0f ? __fdiv_rn(6.0f, amax) : 0.0f;
-      if (blockIdx.y == 0) a.amax_out[c] = amax;
+      const float amax = __uint_as_float(a.amax_cols[c]);
+      s_gcol[tid] = amax > 0.0f ? __fdiv_rn(6.0f, amax) : 0.0f;
+      if (blockIdx.y == 0) a.amax_out_cols[c] = amax;
     }
-    if (PRESCALE && tid < ENC_TM) s_pre[tid] = prescale_value(a.prescale, row0 + tid);
+    if (PRESCALE && tid < ENC_TM) s_prow[tid] = __ldg(&a.pre_row[row0 + tid]);
   }
   __syncthreads();
 
@@ -323,54 +421,81 @@ encode_kernel(const EncodeArgs a) {
     v[r] = make_uint4(0, 0, 0, 0);
     if (in_cols) v[r] = __ldg(&a.x[(long long)(row0 + 8 * warp + r) * vec_per_row + (col >> 3)]);
   }
-  float g[8], p[8];
-  if (AXIS == 1) {
+  float gc[8], pc[8];
+  if (COL_SCALED) {
 #pragma unroll
-    for (int c = 0; c < 8; ++c) g[c] = s_gamma[8 * lane + c];
+    for (int c = 0; c < 8; ++c) gc[c] = in_cols ? s_gcol[8 * lane + c] : 0.0f;
   }
-  if (AXIS == 0 && PRESCALE && in_cols) {
+  if (ROW_SCALED && PRESCALE) {
 #pragma unroll
-    for (int c = 0; c < 8; ++c) p[c] = prescale_value(a.prescale, col + c);
+    for (int c = 0; c < 8; ++c) pc[c] = in_cols ? __ldg(&a.pre_col[col + c]) : 0.0f;
   }
 
-  uint32_t word[8];
+  uint32_t word[8];                                   // codes of the row-major output
+  uint32_t word_t[MODE == MODE_DUAL ? 8 : 1];         // dual: codes of the column-scaled tensor
+  uint32_t any_bits = 0, lo4 = 0, hi4 = 0;            // clamp: mask bytes of rows 0..3 / 4..7
 #pragma unroll
   for (int r = 0; r < 8; ++r) {
     const uint32_t w[4] = {v[r].x, v[r].y, v[r].z, v[r].w};
-    float f[8];
+    float f[8], f2[8];
     uint32_t obits = 0;
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      f[2 * q] = bf16_lo(w[q]);
-      f[2 * q + 1] = bf16_hi(w[q]);
-    }
-    const float grow = AXIS == 0 ? s_gamma[8 * warp + r] : 0.0f;
-    const float prow = (AXIS == 1 && PRESCALE) ? s_pre[8 * warp + r] : 1.0f;
+    const float grow = ROW_SCALED ? s_grow[8 * warp + r] : 0.0f;
+    const float prow = (COL_SCALED && PRESCALE) ? s_prow[8 * warp + r] : 1.0f;
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
-      float xv = f[c];
-      if (PRESCALE) xv = __fmul_rn(xv, AXIS == 0 ? p[c] : prow);
+      float xv = (c & 1) ? bf16_hi(w[c >> 1]) : bf16_lo(w[c >> 1]);
       if (OCC) {
         const float xc = fminf(fmaxf(xv, lo), hi);
         obits |= (xc != xv ? 1u : 0u) << c;
         xv = xc;
       }
-      // + 0.0f turns a -0 product into +0 (the nudge below needs a non-negative zero)
-      f[c] = __fmaf_rn(xv, AXIS == 0 ? grow : g[c], 0.0f);
+      // "+ 0.0f" turns a -0 product into +0 (the nudge needs a non-negative zero)
+      if constexpr (MODE == MODE_ROWS) {
+        f[c] = __fmaf_rn(PRESCALE ? __fmul_rn(xv, pc[c]) : xv, grow, 0.0f);
+      } else if constexpr (MODE == MODE_COLS) {
+        f[c] = __fmaf_rn(PRESCALE ? __fmul_rn(xv, prow) : xv, gc[c], 0.0f);
+      } else {
+        f[c] = __fmaf_rn(__fmul_rn(xv, pc[c]), grow, 0.0f);
+        f2[c] = __fmaf_rn(__fmul_rn(xv, prow), gc[c], 0.0f);
+      }
     }
     word[r] = encode8(f);
+    if constexpr (MODE == MODE_DUAL) word_t[r] = encode8(f2);
     if (in_cols) {
       const long long o = (long long)(row0 + 8 * warp + r) * vec_per_row + (col >> 3);
       if (a.codes) a.codes[o] = word[r];
       if (OCC) a.mask[o] = uint8_t(obits);
     }
+    if (OCC) {
+      any_bits |= obits;
+      if (r < 4) lo4 |= obits << (8 * r); else hi4 |= obits << (8 * (r - 4));
+      const int cnt = __reduce_add_sync(0xFFFFFFFFu, __popc(obits));
+      if (lane == 0 && cnt) atomicAdd(&a.row_cnt[row0 + 8 * warp + r], cnt);
+    }
+  }
+  if (OCC) {
+    // per-column counts of this 64-row strip: only threads that saw a clamped entry take part
+    while (any_bits) {
+      const int c = __ffs(any_bits) - 1;
+      any_bits &= any_bits - 1;
+      const uint32_t sel = 0x01010101u << c;
+      atomicAdd(&s_colcnt[8 * lane + c], __popc(lo4 & sel) + __popc(hi4 & sel));
+    }
   }
 
   if (a.codes_t) {
+    if constexpr (MODE == MODE_DUAL) {
+#pragma unroll
+      for (int r = 0; r < 8; ++r) word[r] = word_t[r];
+    }
     transpose8x8_nibbles(word);
 #pragma unroll
     for (int c = 0; c < 8; ++c) tile_t[(c * 8 + warp) * 32 + lane] = word[c];
-    __syncthreads();
+  }
+  __syncthreads();
+  if (OCC && col0 + tid < a.cols)
+    a.strip_cnt[(long long)blockIdx.y * a.cols + col0 + tid] = uint8_t(s_colcnt[tid]);
+  if (a.codes_t) {
     // thread (c = warp, j = lane) owns column col0 + 8 j + c: 64 rows = 8 words = 32 bytes
     const int k = col0 + 8 * lane + warp;
     if (k < a.cols) {
@@ -387,45 +512,27 @@ encode_kernel(const EncodeArgs a) {
 // ------------------------------------------------------------------------------------------
 // 4. mask -> CSR / CSC
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
-csr_count_kernel(const uint32_t* __restrict__ mask, int rows, int words_per_row, int* __restrict__ row_cnt) {
-  const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
-  const int lane = threadIdx.x & 31;
-  if (row >= rows) return;
-  int c = 0;
-  for (int w = lane; w < words_per_row; w += 32) c += __popc(mask[(long long)row * words_per_row + w]);
-  c = __reduce_add_sync(0xFFFFFFFFu, c);
-  if (lane == 0) row_cnt[row] = c;
-}
-
 // Exclusive prefix sum of n counts by one block; ptr[n] = total.  Also publishes nnz and raises
 // the overflow flag when the total exceeds the caller's capacity.
 __global__ void __launch_bounds__(1024, 1)
 scan_counts_kernel(const int* __restrict__ cnt, int n, int* __restrict__ ptr, int* nnz_out, long long cap,
                    int32_t* status) {
-  __shared__ int part[1024];
+  __shared__ long long warp_tot[32];
   const int t = threadIdx.x;
   const int per = (n + 1023) / 1024;
   const int b = min(n, t * per), e = min(n, b + per);
   int s = 0;
   for (int i = b; i < e; ++i) s += cnt[i];
-  part[t] = s;
-  __syncthreads();
-  for (int off = 1; off < 1024; off <<= 1) {
-    const int add = t >= off ? part[t - off] : 0;
-    __syncthreads();
-    part[t] += add;
-    __syncthreads();
-  }
-  int run = part[t] - s;
+  const long long incl = block_scan_1024(s, warp_tot);
+  int run = int(incl) - s;
   for (int i = b; i < e; ++i) {
     ptr[i] = run;
     run += cnt[i];
   }
   if (t == 1023) {
-    ptr[n] = part[1023];
-    if (nnz_out) *nnz_out = part[1023];
-    if (status && (long long)part[1023] > cap) atomicOr(status, FP4_DEV_SPARSE_OVERFLOW);
+    ptr[n] = int(incl);
+    if (nnz_out) *nnz_out = int(incl);
+    if (status && incl > cap) atomicOr(status, FP4_DEV_SPARSE_OVERFLOW);
   }
 }
 
@@ -441,9 +548,10 @@ csr_fill_kernel(const uint32_t* __restrict__ mask, const __nv_bfloat16* __restri
   const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= rows) return;
+  int base = rowptr[row];
+  if (rowptr[row + 1] == base) return;                // nothing clamped in this row
   const int words_per_row = cols >> 5;
   const float lo = thresholds[0], hi = thresholds[1];
-  int base = rowptr[row];
   for (int w0 = 0; w0 < words_per_row; w0 += 32) {
     const int w = w0 + lane;
     uint32_t m = w < words_per_row ? mask[(long long)row * words_per_row + w] : 0u;
@@ -469,81 +577,114 @@ csr_fill_kernel(const uint32_t* __restrict__ mask, const __nv_bfloat16* __restri
   }
 }
 
-// Column direction: warp <-> one 32-column word of the mask, lane <-> one column, a strip of rows.
+// Per column: running offsets of the strips inside the column, total -> col_cnt.
 __global__ void __launch_bounds__(256)
-csc_count_kernel(const uint32_t* __restrict__ mask, int rows, int cols, int rows_per_split,
-                 int* __restrict__ split_cnt) {
-  const int q = blockIdx.x * 8 + (threadIdx.x >> 5);
-  const int lane = threadIdx.x & 31;
-  const int words_per_row = cols >> 5;
-  if (q >= words_per_row) return;
-  const int r0 = blockIdx.y * rows_per_split, r1 = min(rows, r0 + rows_per_split);
-  int c = 0;
-  for (int r = r0; r < r1; ++r) c += (mask[(long long)r * words_per_row + q] >> lane) & 1u;
-  split_cnt[(long long)blockIdx.y * cols + 32 * q + lane] = c;
-}
-
-// Per column: turn the per-strip counts into running offsets inside the column, total -> col_cnt.
-__global__ void __launch_bounds__(256)
-csc_split_prefix_kernel(int* __restrict__ split_cnt, int cols, int splits, int* __restrict__ col_cnt) {
+csc_strip_prefix_kernel(const uint8_t* __restrict__ strip_cnt, int cols, int strips, int* __restrict__ strip_off,
+                        int* __restrict__ col_cnt) {
   const int k = blockIdx.x * blockDim.x + threadIdx.x;
   if (k >= cols) return;
   int run = 0;
-  for (int s = 0; s < splits; ++s) {
-    const int c = split_cnt[(long long)s * cols + k];
-    split_cnt[(long long)s * cols + k] = run;
+#pragma unroll 8
+  for (int s = 0; s < strips; ++s) {
+    const int c = strip_cnt[(long long)s * cols + k];
+    strip_off[(long long)s * cols + k] = run;
     run += c;
   }
   col_cnt[k] = run;
 }
 
+// Column direction: one warp per (64-row strip, 32-column word of the mask); lane <-> row while
+// loading, lane <-> column while writing.  Strips without a marked entry in the word leave at once.
 __global__ void __launch_bounds__(256)
 csc_fill_kernel(const uint32_t* __restrict__ mask, const __nv_bfloat16* __restrict__ x, int rows, int cols,
-                int rows_per_split, const float* __restrict__ thresholds, const int* __restrict__ colptr,
-                const int* __restrict__ split_off, long long cap, int* __restrict__ csc_row,
+                const float* __restrict__ thresholds, const int* __restrict__ colptr,
+                const int* __restrict__ strip_off, long long cap, int* __restrict__ csc_row,
                 float* __restrict__ csc_val) {
   const int q = blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   const int words_per_row = cols >> 5;
   if (q >= words_per_row) return;
+  const int r0 = blockIdx.y * ENC_TM;
+  const uint32_t w0 = mask[(long long)(r0 + lane) * words_per_row + q];
+  const uint32_t w1 = mask[(long long)(r0 + 32 + lane) * words_per_row + q];
+  uint32_t nz0 = __ballot_sync(0xFFFFFFFFu, w0 != 0);
+  uint32_t nz1 = __ballot_sync(0xFFFFFFFFu, w1 != 0);
+  if (!(nz0 | nz1)) return;
   const int col = 32 * q + lane;
-  const int r0 = blockIdx.y * rows_per_split, r1 = min(rows, r0 + rows_per_split);
   const float lo = thresholds[0], hi = thresholds[1];
-  int pos = colptr[col] + split_off[(long long)blockIdx.y * cols + col];
-  for (int r = r0; r < r1; ++r) {
-    if ((mask[(long long)r * words_per_row + q] >> lane) & 1u) {
-      if (pos < cap) {
-        csc_row[pos] = r;
-        csc_val[pos] = residual_of(x, (long long)r * cols + col, lo, hi);
+  int pos = colptr[col] + strip_off[(long long)blockIdx.y * cols + col];
+#pragma unroll
+  for (int half = 0; half < 2; ++half) {
+    uint32_t nz = half ? nz1 : nz0;
+    const uint32_t mine = half ? w1 : w0;
+    while (nz) {
+      const int rr = __ffs(nz) - 1;
+      nz &= nz - 1;
+      const uint32_t w = __shfl_sync(0xFFFFFFFFu, mine, rr);
+      if ((w >> lane) & 1u) {
+        const int r = r0 + 32 * half + rr;
+        if (pos < cap) {
+          csc_row[pos] = r;
+          csc_val[pos] = residual_of(x, (long long)r * cols + col, lo, hi);
+        }
+        ++pos;
       }
-      ++pos;
     }
   }
 }
 
-int pick_splits(int rows, int cols, int num_sms) {
-  // enough (column-block x strip) CTAs to fill the machine, strips of at least 64 rows
-  const int col_blocks = (cols / 32 + 7) / 8;
-  int splits = (4 * num_sms + col_blocks - 1) / col_blocks;
-  if (splits > rows / 64) splits = rows / 64;
-  if (splits > MAX_SPLITS) splits = MAX_SPLITS;
-  if (splits < 1) splits = 1;
-  return splits;
-}
-
 size_t r256(size_t b) { return (b + 255) & ~size_t(255); }
+
+struct Scratch {
+  uint32_t* hist;
+  int* row_max;
+  int* row_min;
+  uint32_t* amax_rows;
+  uint32_t* amax_cols;
+  uint8_t* mask;
+  int* row_cnt;
+  int* col_cnt;
+  uint8_t* strip_cnt;
+  int* strip_off;
+  float* pre_rows;
+  float* pre_cols;
+  unsigned long long* seg_sum;
+  unsigned* ticket;
+  bool ok;
+};
+
+Scratch carve(Arena& arena, int rows, int cols, bool occ) {
+  Scratch s = {};
+  s.hist = arena.take<uint32_t>(65536);
+  s.row_max = arena.take<int>(rows);
+  s.row_min = arena.take<int>(rows);
+  s.amax_rows = arena.take<uint32_t>(rows);
+  s.amax_cols = arena.take<uint32_t>(cols);
+  s.row_cnt = arena.take<int>(rows);
+  s.col_cnt = arena.take<int>(cols);
+  s.pre_rows = arena.take<float>(rows);
+  s.pre_cols = arena.take<float>(cols);
+  s.seg_sum = arena.take<unsigned long long>(SELECT_BLOCKS);
+  s.ticket = arena.take<unsigned>(1);
+  if (occ) {
+    s.mask = arena.take<uint8_t>(size_t(rows) * cols / 8);
+    s.strip_cnt = arena.take<uint8_t>(size_t(rows / ENC_TM) * cols);
+    s.strip_off = arena.take<int>(size_t(rows / ENC_TM) * cols);
+  }
+  s.ok = arena.ok;
+  return s;
+}
 
 }  // namespace
 
 size_t quantize_scratch_bytes(int64_t rows, int64_t cols) {
   size_t b = 0;
-  b += r256(65536 * 4);                                        // histogram
-  b += 2 * r256(size_t(rows) * 4);                             // row extremes
-  b += r256(size_t(rows > cols ? rows : cols) * 4);            // absmax per vector
-  b += r256(size_t(rows) * size_t(cols) / 8);                  // outlier mask
-  b += r256(size_t(rows) * 4) + r256(size_t(cols) * 4);        // counts
-  b += r256(size_t(MAX_SPLITS) * size_t(cols) * 4);            // per-strip column counts
-  b += r256(size_t(rows > cols ? rows : cols) * 4);            // de-scale vector used as prescale
+  b += r256(65536 * 4);                                          // histogram
+  b += 5 * r256(size_t(rows) * 4) + 4 * r256(size_t(cols) * 4);   // per-row / per-column vectors
+  b += r256(SELECT_BLOCKS * 8) + 256;                            // segment sums, ticket
+  b += r256(size_t(rows) * size_t(cols) / 8);                    // outlier mask
+  b += r256(size_t(rows / ENC_TM) * size_t(cols));               // per-strip column counts (bytes)
+  b += r256(size_t(rows / ENC_TM) * size_t(cols) * 4);           // per-strip column offsets
   return b;
 }
 
@@ -552,119 +693,147 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
                     fp4_qtensor* out, int32_t* status) {
   const int rows = int(rows64), cols = int(cols64);
   const long long n = (long long)rows * cols;
-  const long long n_vec = n / 8;
-  const int vec_per_row = cols / 8;
   const bool occ = alpha < 1.0;
   const uint4* x = static_cast<const uint4*>(x_bf16);
-
-  uint32_t* hist = arena.take<uint32_t>(65536);
-  int* row_max = arena.take<int>(rows);
-  int* row_min = arena.take<int>(rows);
-  uint32_t* vec_amax = arena.take<uint32_t>(rows > cols ? rows : cols);
-  uint8_t* mask = arena.take<uint8_t>(size_t(n / 8));
-  int* row_cnt = arena.take<int>(rows);
-  int* col_cnt = arena.take<int>(cols);
-  int* split_cnt = arena.take<int>(size_t(MAX_SPLITS) * cols);
-  float* pre_d = arena.take<float>(rows > cols ? rows : cols);
-  if (!arena.ok) return FP4_ERR_WORKSPACE;
-  if (prescale && prescale_is_amax) {
-    const int np = scale_axis == 0 ? cols : rows;
-    KernelScope scope(ctx, stream, KC_ABSMAX, 1);
-    descale_kernel<<<(np + 255) / 256, 256, 0, stream>>>(prescale, np, pre_d);
-    prescale = pre_d;
-  }
+  Scratch sc = carve(arena, rows, cols, occ);
+  if (!sc.ok) return FP4_ERR_WORKSPACE;
 
   EncodeArgs ea = {};
   ea.x = x;
   ea.rows = rows;
   ea.cols = cols;
-  ea.prescale = prescale;
-  ea.vec_amax = vec_amax;
-  ea.row_max = row_max;
-  ea.row_min = row_min;
+  ea.amax_rows = sc.amax_rows;
+  ea.amax_cols = sc.amax_cols;
+  ea.row_max = sc.row_max;
+  ea.row_min = sc.row_min;
   ea.thresholds = out->thresholds;
   ea.codes = reinterpret_cast<uint32_t*>(out->codes);
   ea.codes_t = reinterpret_cast<uint32_t*>(out->codes_t);
-  ea.amax_out = out->amax;
-  ea.mask = mask;
-  const dim3 enc_grid((cols + ENC_TK - 1) / ENC_TK, rows / ENC_TM);
+  ea.amax_out_rows = out->amax;
+  ea.amax_out_cols = out->amax;
+  ea.mask = sc.mask;
+  ea.row_cnt = sc.row_cnt;
+  ea.strip_cnt = sc.strip_cnt;
+  const dim3 tile_grid((cols + ENC_TK - 1) / ENC_TK, rows / ENC_TM);
 
   if (occ) {
     const long long n_tail = llround((1.0 - alpha) * double(n));
+    const long long n_vec = n / 8;
     {
-    KernelScope scope(ctx, stream, KC_SELECT, 3);
-    FP4_CUDA_TRY(cudaMemsetAsync(hist, 0, 65536 * 4, stream));
-    init_row_extremes_kernel<<<(rows + 255) / 256, 256, 0, stream>>>(row_max, row_min, rows);
-    FP4_CUDA_TRY(cudaFuncSetAttribute(hist_rowminmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      HIST_WORDS * 4));
-    long long blocks = (n_vec + HIST_THREADS - 1) / HIST_THREADS;
-    if (blocks > ctx->num_sms) blocks = ctx->num_sms;
-    hist_rowminmax_kernel<<<int(blocks), HIST_THREADS, HIST_WORDS * 4, stream>>>(x, n_vec, vec_per_row, hist, row_max,
-                                                                                row_min);
-    select_thresholds_kernel<<<1, 1024, 0, stream>>>(hist, n, n_tail, out->thresholds);
+      KernelScope scope(ctx, stream, KC_SELECT, 3);
+      init_occ_kernel<<<64, 1024, 0, stream>>>(sc.hist, sc.row_max, sc.row_min, sc.row_cnt, rows, sc.ticket);
+      FP4_CUDA_TRY(cudaFuncSetAttribute(hist_rowminmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        HIST_WORDS * 4));
+      long long blocks = (n_vec + HIST_THREADS - 1) / HIST_THREADS;
+      if (blocks > ctx->num_sms) blocks = ctx->num_sms;
+      hist_rowminmax_kernel<<<int(blocks), HIST_THREADS, HIST_WORDS * 4, stream>>>(x, n_vec, cols / 8, sc.hist,
+                                                                                  sc.row_max, sc.row_min);
+      select_thresholds_kernel<<<SELECT_BLOCKS, 1024, 0, stream>>>(sc.hist, n, n_tail, out->thresholds, sc.seg_sum,
+                                                                   sc.ticket);
     }
     {
       KernelScope scope(ctx, stream, KC_ENCODE, 1);
-      encode_kernel<0, true, false><<<enc_grid, ENC_THREADS, 0, stream>>>(ea);
+      encode_kernel<MODE_ROWS, true, false><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
     }
-    KernelScope scope(ctx, stream, KC_SPARSE, 7);
-
-    const uint32_t* mask32 = reinterpret_cast<const uint32_t*>(mask);
+    KernelScope scope(ctx, stream, KC_SPARSE, 5);
+    const uint32_t* mask32 = reinterpret_cast<const uint32_t*>(sc.mask);
     const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x_bf16);
-    csr_count_kernel<<<(rows + 7) / 8, 256, 0, stream>>>(mask32, rows, cols / 32, row_cnt);
-    scan_counts_kernel<<<1, 1024, 0, stream>>>(row_cnt, rows, out->csr_rowptr, out->nnz, out->sparse_cap, status);
+    const int strips = rows / ENC_TM;
+    scan_counts_kernel<<<1, 1024, 0, stream>>>(sc.row_cnt, rows, out->csr_rowptr, out->nnz, out->sparse_cap, status);
     csr_fill_kernel<<<(rows + 7) / 8, 256, 0, stream>>>(mask32, xb, rows, cols, out->thresholds, out->csr_rowptr,
                                                         out->sparse_cap, out->csr_col, out->csr_val);
-    const int splits = pick_splits(rows, cols, ctx->num_sms);
-    const int rows_per_split = (rows + splits - 1) / splits;
-    const dim3 cgrid((cols / 32 + 7) / 8, splits);
-    csc_count_kernel<<<cgrid, 256, 0, stream>>>(mask32, rows, cols, rows_per_split, split_cnt);
-    csc_split_prefix_kernel<<<(cols + 255) / 256, 256, 0, stream>>>(split_cnt, cols, splits, col_cnt);
-    scan_counts_kernel<<<1, 1024, 0, stream>>>(col_cnt, cols, out->csc_colptr, nullptr, out->sparse_cap, nullptr);
-    csc_fill_kernel<<<cgrid, 256, 0, stream>>>(mask32, xb, rows, cols, rows_per_split, out->thresholds,
-                                               out->csc_colptr, split_cnt, out->sparse_cap, out->csc_row,
-                                               out->csc_val);
+    csc_strip_prefix_kernel<<<(cols + 255) / 256, 256, 0, stream>>>(sc.strip_cnt, cols, strips, sc.strip_off,
+                                                                    sc.col_cnt);
+    scan_counts_kernel<<<1, 1024, 0, stream>>>(sc.col_cnt, cols, out->csc_colptr, nullptr, out->sparse_cap, nullptr);
+    const dim3 cgrid((cols / 32 + 7) / 8, strips);
+    csc_fill_kernel<<<cgrid, 256, 0, stream>>>(mask32, xb, rows, cols, out->thresholds, out->csc_colptr, sc.strip_off,
+                                               out->sparse_cap, out->csc_row, out->csc_val);
   } else {
-    const int n_amax = scale_axis == 0 ? rows : cols;
-    FP4_CUDA_TRY(cudaMemsetAsync(vec_amax, 0, size_t(n_amax) * 4, stream));
+    if (prescale && prescale_is_amax) {
+      float* d = scale_axis == 0 ? sc.pre_cols : sc.pre_rows;
+      const int np = scale_axis == 0 ? cols : rows;
+      KernelScope scope(ctx, stream, KC_ABSMAX, 1);
+      descale_kernel<<<(np + 255) / 256, 256, 0, stream>>>(prescale, np, d);
+      prescale = d;
+    }
+    AbsmaxArgs aa = {};
+    aa.x = x;
+    aa.rows = rows;
+    aa.cols = cols;
+    aa.amax_rows = sc.amax_rows;
+    aa.amax_cols = sc.amax_cols;
     if (scale_axis == 0) {
-      long long blocks = (n_vec + 255) / 256;
-      if (blocks > 8LL * ctx->num_sms) blocks = 8LL * ctx->num_sms;
+      aa.pre_col = prescale;
+      ea.pre_col = prescale;
+      FP4_CUDA_TRY(cudaMemsetAsync(sc.amax_rows, 0, size_t(rows) * 4, stream));
       {
         KernelScope scope(ctx, stream, KC_ABSMAX, 1);
-        if (prescale)
-          absmax_rows_kernel<true><<<int(blocks), 256, 0, stream>>>(x, n_vec, vec_per_row, prescale, vec_amax);
-        else
-          absmax_rows_kernel<false><<<int(blocks), 256, 0, stream>>>(x, n_vec, vec_per_row, nullptr, vec_amax);
+        absmax_tile_kernel<MODE_ROWS><<<tile_grid, ENC_THREADS, 0, stream>>>(aa);
       }
       KernelScope scope(ctx, stream, KC_ENCODE, 1);
       if (prescale)
-        encode_kernel<0, false, true><<<enc_grid, ENC_THREADS, 0, stream>>>(ea);
+        encode_kernel<MODE_ROWS, false, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
       else
-        encode_kernel<0, false, false><<<enc_grid, ENC_THREADS, 0, stream>>>(ea);
+        encode_kernel<MODE_ROWS, false, false><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
     } else {
-      const int col_blocks = (vec_per_row + 255) / 256;
-      int strips = (8 * ctx->num_sms + col_blocks - 1) / col_blocks;
-      if (strips > rows / 16) strips = rows / 16;
-      if (strips < 1) strips = 1;
-      const int rows_per_strip = (rows + strips - 1) / strips;
-      const dim3 agrid(col_blocks, (rows + rows_per_strip - 1) / rows_per_strip);
+      aa.pre_row = prescale;
+      ea.pre_row = prescale;
+      FP4_CUDA_TRY(cudaMemsetAsync(sc.amax_cols, 0, size_t(cols) * 4, stream));
       {
         KernelScope scope(ctx, stream, KC_ABSMAX, 1);
-        if (prescale)
-          absmax_cols_kernel<true><<<agrid, 256, 0, stream>>>(x, rows, vec_per_row, rows_per_strip, prescale,
-                                                              vec_amax);
-        else
-          absmax_cols_kernel<false><<<agrid, 256, 0, stream>>>(x, rows, vec_per_row, rows_per_strip, nullptr,
-                                                               vec_amax);
+        absmax_tile_kernel<MODE_COLS><<<tile_grid, ENC_THREADS, 0, stream>>>(aa);
       }
       KernelScope scope(ctx, stream, KC_ENCODE, 1);
       if (prescale)
-        encode_kernel<1, false, true><<<enc_grid, ENC_THREADS, 0, stream>>>(ea);
+        encode_kernel<MODE_COLS, false, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
       else
-        encode_kernel<1, false, false><<<enc_grid, ENC_THREADS, 0, stream>>>(ea);
+        encode_kernel<MODE_COLS, false, false><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
     }
   }
+  FP4_CUDA_TRY(cudaGetLastError());
+  return FP4_OK;
+}
+
+// One read of dY for both backward GEMMs: row-scaled codes of dY (.) (amax_col_pre / 6) and
+// column-scaled transposed codes of dY (.) (amax_row_pre / 6).
+int launch_quantize_dual(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void* x_bf16, int64_t rows64,
+                         int64_t cols64, const float* amax_col_pre, const float* amax_row_pre, uint8_t* codes_rows,
+                         float* amax_rows_out, uint8_t* codes_t_cols, float* amax_cols_out) {
+  const int rows = int(rows64), cols = int(cols64);
+  Scratch sc = carve(arena, rows, cols, false);
+  if (!sc.ok) return FP4_ERR_WORKSPACE;
+  const dim3 tile_grid((cols + ENC_TK - 1) / ENC_TK, rows / ENC_TM);
+  AbsmaxArgs aa = {};
+  aa.x = static_cast<const uint4*>(x_bf16);
+  aa.rows = rows;
+  aa.cols = cols;
+  aa.pre_col = amax_col_pre;
+  aa.pre_row = amax_row_pre;
+  aa.pre_is_amax = 1;
+  aa.d_col_out = sc.pre_cols;
+  aa.d_row_out = sc.pre_rows;
+  aa.amax_rows = sc.amax_rows;
+  aa.amax_cols = sc.amax_cols;
+  FP4_CUDA_TRY(cudaMemsetAsync(sc.amax_rows, 0, size_t(rows) * 4, stream));
+  FP4_CUDA_TRY(cudaMemsetAsync(sc.amax_cols, 0, size_t(cols) * 4, stream));
+  {
+    KernelScope scope(ctx, stream, KC_ABSMAX, 1);
+    absmax_tile_kernel<MODE_DUAL><<<tile_grid, ENC_THREADS, 0, stream>>>(aa);
+  }
+  EncodeArgs ea = {};
+  ea.x = aa.x;
+  ea.rows = rows;
+  ea.cols = cols;
+  ea.pre_col = sc.pre_cols;
+  ea.pre_row = sc.pre_rows;
+  ea.amax_rows = sc.amax_rows;
+  ea.amax_cols = sc.amax_cols;
+  ea.codes = reinterpret_cast<uint32_t*>(codes_rows);
+  ea.codes_t = reinterpret_cast<uint32_t*>(codes_t_cols);
+  ea.amax_out_rows = amax_rows_out;
+  ea.amax_out_cols = amax_cols_out;
+  KernelScope scope(ctx, stream, KC_ENCODE, 1);
+  encode_kernel<MODE_DUAL, false, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
   FP4_CUDA_TRY(cudaGetLastError());
   return FP4_OK;
 }
@@ -672,12 +841,14 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
 // ------------------------------------------------------------------------------------------
 // Quantile thresholds without any allocation
 // ------------------------------------------------------------------------------------------
-// Scratch of fp4_quantile_thresholds_static: the 65536-bin histogram followed by the row
-// extremes of up to FP4_STATIC_MAX_ROWS rows.  It lives in the library image: every GPU that
-// loads the library holds these 768 KB until the process exits.
+// Scratch of fp4_quantile_thresholds_static: the 65536-bin histogram, the select kernel's segment
+// sums and ticket, and the row extremes of up to FP4_STATIC_MAX_ROWS rows.  It lives in the
+// library image: every GPU that loads the library holds these 769 KB until the process exits.
 namespace {
 constexpr size_t STATIC_HIST_BYTES = 65536 * sizeof(uint32_t);
-constexpr size_t STATIC_SCRATCH_BYTES = STATIC_HIST_BYTES + 2 * size_t(FP4_STATIC_MAX_ROWS) * sizeof(int);
+constexpr size_t STATIC_SELECT_BYTES = 1024;      // 64 segment sums (512 B) + ticket, padded
+constexpr size_t STATIC_SCRATCH_BYTES =
+    STATIC_HIST_BYTES + STATIC_SELECT_BYTES + 2 * size_t(FP4_STATIC_MAX_ROWS) * sizeof(int);
 constexpr int STATIC_MAX_DEVICES = 64;
 }  // namespace
 static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
@@ -713,20 +884,22 @@ extern "C" int fp4_quantile_thresholds_static(void* stream, const void* x_bf16, 
   }
   unsigned char* base = static_cast<unsigned char*>(scratch_of_device[device]);
   uint32_t* hist = reinterpret_cast<uint32_t*>(base);
-  int* row_max = reinterpret_cast<int*>(base + STATIC_HIST_BYTES);
+  unsigned long long* seg_sum = reinterpret_cast<unsigned long long*>(base + STATIC_HIST_BYTES);
+  unsigned* ticket = reinterpret_cast<unsigned*>(base + STATIC_HIST_BYTES + 512);
+  int* row_max = reinterpret_cast<int*>(base + STATIC_HIST_BYTES + STATIC_SELECT_BYTES);
   int* row_min = row_max + FP4_STATIC_MAX_ROWS;
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // The array keeps what the previous call left: the histogram must start from zero and the
-  // row extremes from their identities.
-  FP4_CUDA_TRY(cudaMemsetAsync(hist, 0, STATIC_HIST_BYTES, st));
+  // The array keeps what the previous call left: the histogram and the ticket must start from
+  // zero and the row extremes from their identities.
+  FP4_CUDA_TRY(cudaMemsetAsync(base, 0, STATIC_HIST_BYTES + STATIC_SELECT_BYTES, st));
   init_row_extremes_kernel<<<int((rows + 255) / 256), 256, 0, st>>>(row_max, row_min, int(rows));
   const long long n_vec = n / 8;
   long long blocks = (n_vec + HIST_THREADS - 1) / HIST_THREADS;
   if (blocks > sms_of_device[device]) blocks = sms_of_device[device];
   hist_rowminmax_kernel<<<int(blocks), HIST_THREADS, HIST_WORDS * 4, st>>>(static_cast<const uint4*>(x_bf16), n_vec,
                                                                           int(cols / 8), hist, row_max, row_min);
-  select_thresholds_kernel<<<1, 1024, 0, st>>>(hist, n, n_tail, thresholds);
+  select_thresholds_kernel<<<SELECT_BLOCKS, 1024, 0, st>>>(hist, n, n_tail, thresholds, seg_sum, ticket);
   FP4_CUDA_TRY(cudaGetLastError());
   return FP4_OK;
 }
