@@ -23,6 +23,7 @@ size_t linear_scratch_bytes(int64_t M, int64_t K, int64_t N) {
   b += 2 * round256(size_t(M) * size_t(N) / 2);       // dY codes, both scalings
   b += round256(size_t(M) * 4) + round256(size_t(N) * 4);   // their amax vectors
   b += 2 * round256(size_t(M > N ? M : N) * 4);       // de-scale vectors used as prescale
+  b += round256((2 * size_t(K) + 2) * 4);             // lists of columns that hold residual entries
   return b;
 }
 
@@ -261,6 +262,7 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
   uint8_t* g2_codes = dW ? arena.take<uint8_t>(size_t(M) * size_t(N) / 2) : nullptr;   // dY (.) d_A, channel-wise
   float* g1_amax = arena.take<float>(size_t(M));
   float* g2_amax = arena.take<float>(size_t(N));
+  int* col_list = arena.take<int>(2 * size_t(K) + 2);
   if (!arena.ok) return FP4_ERR_WORKSPACE;
   Arena q_arena(arena.base + arena.off, arena.size - arena.off);
   int rc;
@@ -295,7 +297,7 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
     rc = launch_gemm_fp4(ctx, st, savedA->codes_t, g2_codes, K, N, M, nullptr, g2_amax, s, 1, gemm_kind, status);
     if (rc != FP4_OK) return rc;
     rc = launch_comp_wgrad_dge(ctx, st, s, savedA->csc_colptr, savedA->csc_row, savedA->csc_val, dY_bf16, W_bf16,
-                               savedW->amax, M, K, N, dge_on, dge_k, dge_clip, dW, out_f32);
+                               savedW->amax, col_list, M, K, N, dge_on, dge_k, dge_clip, dW, out_f32);
     if (rc != FP4_OK) return rc;
   }
   return FP4_OK;

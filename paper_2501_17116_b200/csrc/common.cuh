@@ -115,5 +115,6 @@ int launch_comp_fwd(fp4_ctx* ctx, cudaStream_t stream, const float* y1, const in
 // dw[k,:] = store( (s[k,:] + sum_{entries of column k} val * dy[row,:]) * Q'(w[k,:] * gamma[:]) )
 int launch_comp_wgrad_dge(fp4_ctx* ctx, cudaStream_t stream, float* s, const int32_t* colptr,
                           const int32_t* row, const float* val, const void* dy_bf16,
-                          const void* w_bf16, const float* w_amax, int64_t M, int64_t K, int64_t N,
-                          int dge_on, float dge_k, float dge_clip, void* dw, int out_f32);
+                          const void* w_bf16, const float* w_amax, int* col_list /*[2 K + 2] scratch*/,
+                          int64_t M, int64_t K, int64_t N, int dge_on, float dge_k, float dge_clip,
+                          void* dw, int out_f32);

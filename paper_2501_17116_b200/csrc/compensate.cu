@@ -96,61 +96,146 @@ __device__ __forceinline__ float dge_factor(float ws, float expo, float inv_k, f
   return fminf(d, clip);
 }
 
+constexpr int LONG_COLUMN = 64;            // entries from which a column gets a whole 1024-thread block
+constexpr int LONG_THREADS = 1024;
+
+// Two ascending lists of the columns that hold residual entries: "long" columns (at least
+// LONG_COLUMN entries: the outlier channels) and "short" ones; counts[0], counts[1] their sizes.
+__global__ void __launch_bounds__(1024, 1)
+nonempty_columns_kernel(const int* __restrict__ colptr, int K, int* __restrict__ list_long,
+                        int* __restrict__ list_short, int* __restrict__ counts) {
+  __shared__ unsigned long long warp_tot[32];
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  const int per = (K + 1023) / 1024;
+  const int b = min(K, t * per), e = min(K, b + per);
+  unsigned long long c = 0;                          // low word: long columns, high word: short columns
+  for (int k = b; k < e; ++k) {
+    const int n = colptr[k + 1] - colptr[k];
+    if (n >= LONG_COLUMN) c += 1ull;
+    else if (n > 0) c += 1ull << 32;
+  }
+  unsigned long long incl = c;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+    if (lane >= off) incl += up;
+  }
+  if (lane == 31) warp_tot[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    unsigned long long v = warp_tot[lane];
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, v, off);
+      if (lane >= off) v += up;
+    }
+    warp_tot[lane] = v;
+  }
+  __syncthreads();
+  const unsigned long long before = incl - c + (warp ? warp_tot[warp - 1] : 0ull);
+  int pos_long = int(before & 0xFFFFFFFFull), pos_short = int(before >> 32);
+  for (int k = b; k < e; ++k) {
+    const int n = colptr[k + 1] - colptr[k];
+    if (n >= LONG_COLUMN) list_long[pos_long++] = k;
+    else if (n > 0) list_short[pos_short++] = k;
+  }
+  if (t == 1023) {
+    counts[0] = int(warp_tot[31] & 0xFFFFFFFFull);
+    counts[1] = int(warp_tot[31] >> 32);
+  }
+}
+
+// acc[0..7] += sum of val[e] * dense[idx[e], vcol] over e = first, first + step, ... < e1, eight
+// gathers in flight and the indices of the next round fetched under them.
+__device__ __forceinline__ void strided_entries_times_dense(float (&acc)[8], const int* __restrict__ idx,
+                                                            const float* __restrict__ val, int first, int e1,
+                                                            int step, const uint4* __restrict__ dense,
+                                                            int vec_per_row, int vcol) {
+  int r[8];
+  float v[8];
+#pragma unroll
+  for (int u = 0; u < 8; ++u) {
+    const bool live = first + step * u < e1;          // past the end: value 0 times row 0
+    r[u] = live ? __ldg(&idx[first + step * u]) : 0;
+    v[u] = live ? __ldg(&val[first + step * u]) : 0.0f;
+  }
+  for (int e = first; e < e1; e += 8 * step) {
+    uint4 d[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) d[u] = __ldg(&dense[(long long)r[u] * vec_per_row + vcol]);
+    int rn[8];
+    float vn[8];
+    const int nxt = e + 8 * step;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const bool live = nxt + step * u < e1;
+      rn[u] = live ? __ldg(&idx[nxt + step * u]) : 0;
+      vn[u] = live ? __ldg(&val[nxt + step * u]) : 0.0f;
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) fma8(acc, v[u], d[u]);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) { r[u] = rn[u]; v[u] = vn[u]; }
+  }
+}
+
+__device__ __forceinline__ void add8_to(float* dst, const float (&t)[8]) {
+  float4 a = *reinterpret_cast<float4*>(dst);
+  float4 b = *reinterpret_cast<float4*>(dst + 4);
+  a.x += t[0]; a.y += t[1]; a.z += t[2]; a.w += t[3];
+  b.x += t[4]; b.y += t[5]; b.z += t[6]; b.w += t[7];
+  *reinterpret_cast<float4*>(dst) = a;
+  *reinterpret_cast<float4*>(dst + 4) = b;
+}
+
 // Weight-gradient compensation, step 1: S[k, n-block] += sum over the entries of column k of
-// dA[m,k] * dY[m, n-block].  One block per (column, 256 output columns).  Outliers sit in a few
-// channels (Appendix D), so a handful of columns hold thousands of entries and most hold none:
-// empty columns leave at once, and the eight warps of a block take the entries of a long column
-// round-robin.  Their partial sums are added in warp order, so the result does not depend on
-// scheduling.
-__global__ void __launch_bounds__(COMP_THREADS)
-comp_wgrad_accum_kernel(float* __restrict__ s, const int* __restrict__ colptr, const int* __restrict__ row,
-                        const float* __restrict__ val, const uint4* __restrict__ dy, int K, int N) {
-  __shared__ float part[8][32][9];                  // [warp][lane][8 (+1 pad)]
-  const int k = blockIdx.y;
-  const int e0 = colptr[k], e1 = colptr[k + 1];
-  if (e0 == e1) return;
+// dA[m,k] * dY[m, n-block].  Outliers sit in a few channels (Appendix D): a handful of columns
+// hold thousands of entries, a few hundred hold one or two, most hold none.
+// Long columns: one 1024-thread block per (column, 256 outputs); its 32 warps take the entries
+// round-robin and their partial sums are added in warp order (independent of scheduling).
+__global__ void __launch_bounds__(LONG_THREADS, 1)
+comp_wgrad_long_kernel(float* __restrict__ s, const int* __restrict__ colptr, const int* __restrict__ row,
+                       const float* __restrict__ val, const uint4* __restrict__ dy, const int* __restrict__ list,
+                       const int* __restrict__ count, int N) {
+  __shared__ float part[32][32][9];                 // [warp][lane][8 (+1 pad)]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n0 = blockIdx.x * COMP_COLS + 8 * lane;
   const bool in_cols = n0 < N;
-  const int vcol = n0 >> 3, vec_per_row = N >> 3;
-  float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  if (in_cols) {
-    int e = e0 + warp;
-    for (; e + 24 < e1; e += 32) {                  // four entries of this warp in flight
-      int r[4];
-      float v[4];
-      uint4 d[4];
+  const int n_cols = *count;
+  for (int slot = blockIdx.y; slot < n_cols; slot += gridDim.y) {
+    const int k = list[slot];
+    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (in_cols)
+      strided_entries_times_dense(acc, row, val, colptr[k] + warp, colptr[k + 1], 32, dy, N >> 3, n0 >> 3);
+    __syncthreads();                                // the previous column's partials have been read
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        r[u] = __ldg(&row[e + 8 * u]);
-        v[u] = __ldg(&val[e + 8 * u]);
+    for (int c = 0; c < 8; ++c) part[warp][lane][c] = acc[c];
+    __syncthreads();
+    if (warp == 0 && in_cols) {
+      float t[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+      for (int w = 0; w < 32; ++w) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) t[c] += part[w][lane][c];
       }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) d[u] = __ldg(&dy[(long long)r[u] * vec_per_row + vcol]);
-#pragma unroll
-      for (int u = 0; u < 4; ++u) fma8(acc, v[u], d[u]);
-    }
-    for (; e < e1; e += 8) {
-      const uint4 d = __ldg(&dy[(long long)__ldg(&row[e]) * vec_per_row + vcol]);
-      fma8(acc, __ldg(&val[e]), d);
+      add8_to(s + (long long)k * N + n0, t);
     }
   }
-#pragma unroll
-  for (int c = 0; c < 8; ++c) part[warp][lane][c] = acc[c];
-  __syncthreads();
-  if (warp == 0 && in_cols) {
-    float* dst = s + (long long)k * N + n0;
-    float4 a = *reinterpret_cast<float4*>(dst);
-    float4 b = *reinterpret_cast<float4*>(dst + 4);
-    float t[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    for (int w = 0; w < 8; ++w) {
-#pragma unroll
-      for (int c = 0; c < 8; ++c) t[c] += part[w][lane][c];
-    }
-    a.x += t[0]; a.y += t[1]; a.z += t[2]; a.w += t[3];
-    b.x += t[4]; b.y += t[5]; b.z += t[6]; b.w += t[7];
-    *reinterpret_cast<float4*>(dst) = a;
-    *reinterpret_cast<float4*>(dst + 4) = b;
+}
+
+// Short columns: one warp per (column, 256 outputs), entries in order.
+__global__ void __launch_bounds__(COMP_THREADS)
+comp_wgrad_short_kernel(float* __restrict__ s, const int* __restrict__ colptr, const int* __restrict__ row,
+                        const float* __restrict__ val, const uint4* __restrict__ dy, const int* __restrict__ list,
+                        const int* __restrict__ count, int N) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n0 = blockIdx.x * COMP_COLS + 8 * lane;
+  if (n0 >= N) return;
+  const int n_cols = *count;
+  for (int slot = blockIdx.y * 8 + warp; slot < n_cols; slot += gridDim.y * 8) {
+    const int k = list[slot];
+    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    strided_entries_times_dense(acc, row, val, colptr[k], colptr[k + 1], 1, dy, N >> 3, n0 >> 3);
+    add8_to(s + (long long)k * N + n0, acc);
   }
 }
 
@@ -199,13 +284,26 @@ int launch_comp_fwd(fp4_ctx* ctx, cudaStream_t stream, const float* y1, const in
 }
 
 int launch_comp_wgrad_dge(fp4_ctx* ctx, cudaStream_t stream, float* s, const int32_t* colptr, const int32_t* row,
-                          const float* val, const void* dy_bf16, const void* w_bf16, const float* w_amax, int64_t,
-                          int64_t K, int64_t N, int dge_on, float dge_k, float dge_clip, void* dw, int out_f32) {
-  KernelScope scope(ctx, stream, KC_COMP_WGRAD, colptr ? 2 : 1);
+                          const float* val, const void* dy_bf16, const void* w_bf16, const float* w_amax,
+                          int* col_list, int64_t, int64_t K, int64_t N, int dge_on, float dge_k, float dge_clip,
+                          void* dw, int out_f32) {
+  KernelScope scope(ctx, stream, KC_COMP_WGRAD, colptr ? 4 : 1);
   if (colptr) {
-    const dim3 grid(unsigned((N + COMP_COLS - 1) / COMP_COLS), unsigned(K));
-    comp_wgrad_accum_kernel<<<grid, COMP_THREADS, 0, stream>>>(s, colptr, row, val, static_cast<const uint4*>(dy_bf16),
-                                                               int(K), int(N));
+    // col_list: [K] long columns, [K] short columns, two counters
+    int* list_long = col_list;
+    int* list_short = col_list + K;
+    int* counts = col_list + 2 * K;
+    nonempty_columns_kernel<<<1, 1024, 0, stream>>>(colptr, int(K), list_long, list_short, counts);
+    const unsigned n_blocks = unsigned((N + COMP_COLS - 1) / COMP_COLS);
+    const uint4* dy = static_cast<const uint4*>(dy_bf16);
+    unsigned gy = unsigned(4 * ctx->num_sms) / n_blocks;          // long columns: 2 resident blocks per SM
+    gy = gy < 1 ? 1 : (gy > unsigned(K) ? unsigned(K) : gy);
+    comp_wgrad_long_kernel<<<dim3(n_blocks, gy), LONG_THREADS, 0, stream>>>(s, colptr, row, val, dy, list_long, counts,
+                                                                           int(N));
+    gy = unsigned(32 * ctx->num_sms) / n_blocks;                   // short columns: 8 per block
+    gy = gy < 1 ? 1 : (gy > unsigned((K + 7) / 8) ? unsigned((K + 7) / 8) : gy);
+    comp_wgrad_short_kernel<<<dim3(n_blocks, gy), COMP_THREADS, 0, stream>>>(s, colptr, row, val, dy, list_short,
+                                                                             counts + 1, int(N));
   }
   const long long n_vec = (long long)K * N / 8;
   long long blocks = (n_vec + 255) / 256;

@@ -180,11 +180,14 @@ select_thresholds_kernel(const uint32_t* __restrict__ ghist, long long n, long l
   if (!s_last) return;
   __threadfence();
   const long long rank[2] = {n_tail, n - 1 - n_tail};
+  __shared__ long long s_sum[SELECT_BLOCKS];
+  if (t < int(gridDim.x)) s_sum[t] = (long long)reinterpret_cast<volatile unsigned long long*>(seg_sum)[t];
+  __syncthreads();
   if (t == 0) {
     long long run = 0;
     int q = 0;
     for (int sgm = 0; sgm < int(gridDim.x) && q < 2; ++sgm) {
-      const long long sz = (long long)reinterpret_cast<volatile unsigned long long*>(seg_sum)[sgm];
+      const long long sz = s_sum[sgm];
       while (q < 2 && rank[q] < run + sz) {
         s_seg[q] = sgm;
         s_before[q] = run;
@@ -593,8 +596,10 @@ csc_strip_prefix_kernel(const uint8_t* __restrict__ strip_cnt, int cols, int str
   col_cnt[k] = run;
 }
 
-// Column direction: one warp per (64-row strip, 32-column word of the mask); lane <-> row while
-// loading, lane <-> column while writing.  Strips without a marked entry in the word leave at once.
+// Column direction: one warp per (64-row strip, 32-column word of the mask).  Lane <-> row: each
+// lane keeps the mask word of its row.  For every column of the word that holds a marked entry
+// (usually one or two: the outlier channels), a ballot gives each marked row its rank inside the
+// column, so all gathers of a column are issued at once and the order is by row by construction.
 __global__ void __launch_bounds__(256)
 csc_fill_kernel(const uint32_t* __restrict__ mask, const __nv_bfloat16* __restrict__ x, int rows, int cols,
                 const float* __restrict__ thresholds, const int* __restrict__ colptr,
@@ -607,28 +612,32 @@ csc_fill_kernel(const uint32_t* __restrict__ mask, const __nv_bfloat16* __restri
   const int r0 = blockIdx.y * ENC_TM;
   const uint32_t w0 = mask[(long long)(r0 + lane) * words_per_row + q];
   const uint32_t w1 = mask[(long long)(r0 + 32 + lane) * words_per_row + q];
-  uint32_t nz0 = __ballot_sync(0xFFFFFFFFu, w0 != 0);
-  uint32_t nz1 = __ballot_sync(0xFFFFFFFFu, w1 != 0);
-  if (!(nz0 | nz1)) return;
-  const int col = 32 * q + lane;
+  const uint32_t any0 = __reduce_or_sync(0xFFFFFFFFu, w0);
+  const uint32_t any1 = __reduce_or_sync(0xFFFFFFFFu, w1);
+  if (!(any0 | any1)) return;
   const float lo = thresholds[0], hi = thresholds[1];
-  int pos = colptr[col] + strip_off[(long long)blockIdx.y * cols + col];
+  // lane c holds the next free position of column 32 q + c
+  int next = colptr[32 * q + lane] + strip_off[(long long)blockIdx.y * cols + 32 * q + lane];
+  const uint32_t lt_mask = (1u << lane) - 1u;
 #pragma unroll
   for (int half = 0; half < 2; ++half) {
-    uint32_t nz = half ? nz1 : nz0;
-    const uint32_t mine = half ? w1 : w0;
-    while (nz) {
-      const int rr = __ffs(nz) - 1;
-      nz &= nz - 1;
-      const uint32_t w = __shfl_sync(0xFFFFFFFFu, mine, rr);
-      if ((w >> lane) & 1u) {
-        const int r = r0 + 32 * half + rr;
+    const uint32_t w = half ? w1 : w0;
+    uint32_t any = half ? any1 : any0;
+    const int r = r0 + 32 * half + lane;
+    while (any) {
+      const int c = __ffs(any) - 1;
+      any &= any - 1;
+      const bool mine = (w >> c) & 1u;
+      const uint32_t b = __ballot_sync(0xFFFFFFFFu, mine);
+      const int base = __shfl_sync(0xFFFFFFFFu, next, c);
+      if (mine) {
+        const int pos = base + __popc(b & lt_mask);
         if (pos < cap) {
           csc_row[pos] = r;
-          csc_val[pos] = residual_of(x, (long long)r * cols + col, lo, hi);
+          csc_val[pos] = residual_of(x, (long long)r * cols + 32 * q + c, lo, hi);
         }
-        ++pos;
       }
+      if (lane == c) next += __popc(b);
     }
   }
 }
