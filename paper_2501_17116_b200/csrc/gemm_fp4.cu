@@ -36,13 +36,15 @@ constexpr int TMEM_COLS = 512;
 constexpr int ACC_STRIDE = 256;          // tensor-memory columns between the two accumulator stages
 constexpr int SF_COL_B = 240;            // MXF4 only: unit block scales in the gap behind stage 0
 constexpr int SF_COL_A = 248;
-constexpr int CHUNK = 16;                // accumulator columns per tcgen05.ld of the epilogue
+constexpr int STAGE_OUT_BYTES = 4 * 4096; // epilogue: 32 rows x 128 bytes of output per warp
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
 
 __host__ __device__ constexpr int tile_n(int kind) { return kind == FP4_GEMM_F8F6F4 ? 256 : 240; }
 __host__ __device__ constexpr int b_stage_bytes(int kind) { return tile_n(kind) * 128; }
 __host__ __device__ constexpr int stage_bytes(int kind) { return A_STAGE_BYTES + b_stage_bytes(kind); }
-constexpr size_t smem_bytes(int kind) { return 1024 + size_t(STAGES) * stage_bytes(kind) + 256 + 2 * 256 * 4; }
+constexpr size_t smem_bytes(int kind) {
+  return 1024 + size_t(STAGES) * stage_bytes(kind) + 256 + 2 * 256 * 4 + STAGE_OUT_BYTES;
+}
 
 struct GemmArgs {
   int I, J;
@@ -132,8 +134,21 @@ __device__ __forceinline__ void mma_mxf4(uint32_t d_tmem, uint64_t a_desc, uint6
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate)
       : "memory");
 }
-// 32 lanes x 16 consecutive columns of 32-bit cells: thread t gets row t of the warp's lane quarter.
-__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&v)[16]) {
+// 32 lanes x 32 (or 16) consecutive columns of 32-bit cells: thread t gets row t of the warp's
+// lane quarter.
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&v)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
@@ -181,35 +196,59 @@ __host__ __device__ constexpr uint32_t idesc_mxf4() {
          (uint32_t(BM >> 4) << 24);
 }
 
-// De-scale 16 accumulators of one row and store them (BF16: 32 bytes, float: 64 bytes).
-__device__ __forceinline__ void scale_store16(const uint32_t (&v)[16], float d_row, const float* s_dcol, void* out,
-                                              int out_f32, size_t off) {
-  float y[16];
+// De-scale W accumulators of this thread's row, then store the warp's 32 x W block through a
+// shared staging tile so that every store instruction writes whole row segments: the thread-per-
+// row layout of tensor memory would otherwise touch 32 different lines per instruction.
+// The staging tile holds 32 rows of SPR 16-byte slots; slot s of row r sits at s ^ f(r), which
+// keeps both the row-wise writes and the segment-wise reads free of bank conflicts.
+template <int W, bool F32>
+__device__ __forceinline__ void scale_stage_store(uint32_t (&v)[32], float d_row, const float* dcol, uint8_t* stage,
+                                                  void* out, size_t elem_off, int J, int lane, uint32_t next_taddr,
+                                                  int next_width) {
+  constexpr int SPR = F32 ? W / 4 : W / 8;          // 16-byte slots per row: 8, 4 or 2
+  constexpr int SH = SPR == 8 ? 0 : (SPR == 4 ? 1 : 2);
+  float y[W];
 #pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const float4 dc = *reinterpret_cast<const float4*>(s_dcol + 4 * q);     // same address in every lane
+  for (int q = 0; q < W / 4; ++q) {
+    const float4 dc = *reinterpret_cast<const float4*>(dcol + 4 * q);     // same address in every lane
     y[4 * q + 0] = __fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 0]), d_row), dc.x);
     y[4 * q + 1] = __fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 1]), d_row), dc.y);
     y[4 * q + 2] = __fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 2]), d_row), dc.z);
     y[4 * q + 3] = __fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 3]), d_row), dc.w);
   }
-  if (out_f32) {
-    float4* dst = reinterpret_cast<float4*>(static_cast<float*>(out) + off);
+  // v is dead now: fetch the next chunk of accumulators under the staging and the stores
+  if (next_width >= 32) tmem_ld_32x32(next_taddr, v);
+  else if (next_width > 0) tmem_ld_32x16(next_taddr, v);
+  uint8_t* my_row = stage + lane * (SPR * 16);
+  const int fx = (lane >> SH) & (SPR - 1);
 #pragma unroll
-    for (int j = 0; j < 4; ++j) dst[j] = make_float4(y[4 * j], y[4 * j + 1], y[4 * j + 2], y[4 * j + 3]);
-  } else {
-    uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(out) + off);
-#pragma unroll
-    for (int j = 0; j < 2; ++j) {
+  for (int j = 0; j < SPR; ++j) {
+    uint4 pk;
+    if (F32) {
+      pk = make_uint4(__float_as_uint(y[4 * j]), __float_as_uint(y[4 * j + 1]), __float_as_uint(y[4 * j + 2]),
+                      __float_as_uint(y[4 * j + 3]));
+    } else {
       uint32_t w[4];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         __nv_bfloat162 h = __floats2bfloat162_rn(y[8 * j + 2 * q], y[8 * j + 2 * q + 1]);
         w[q] = *reinterpret_cast<uint32_t*>(&h);
       }
-      dst[j] = make_uint4(w[0], w[1], w[2], w[3]);
+      pk = make_uint4(w[0], w[1], w[2], w[3]);
     }
+    *reinterpret_cast<uint4*>(my_row + ((j ^ fx) * 16)) = pk;
   }
+  __syncwarp();
+  constexpr int ELT = F32 ? 4 : 2;
+  uint8_t* gbase = static_cast<uint8_t*>(out) + elem_off * ELT;
+#pragma unroll
+  for (int i = 0; i < SPR; ++i) {
+    const int row = i * (32 / SPR) + lane / SPR;
+    const int sl = lane % SPR;
+    const uint4 pk = *reinterpret_cast<const uint4*>(stage + row * (SPR * 16) + ((sl ^ ((row >> SH) & (SPR - 1))) * 16));
+    *reinterpret_cast<uint4*>(gbase + size_t(row) * size_t(J) * ELT + sl * 16) = pk;
+  }
+  __syncwarp();
 }
 
 template <int KIND>
@@ -232,6 +271,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(final_bar + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* s_dcol = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES + 256);   // [2][256] column de-scales
+  uint8_t* s_out = smem + STAGES * STAGE_BYTES + 256 + 2 * 256 * 4;              // [4 warps][4096] staging
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -379,20 +419,30 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       if (epilogue_bar_any(!ok)) break;            // also publishes dcol to the other warps
       tc_fence_after();
       const uint32_t t_base = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * ACC_STRIDE);
-      const size_t row_off = size_t(row) * size_t(args.J) + size_t(n_blk) * BN;
-      const int n_chunks = min(BN, args.J - n_blk * BN) / CHUNK;   // ragged last tile in N
-      uint32_t va[16], vb[16];
-      tmem_ld_32x16(t_base, va);
+      // first element of this warp's 32 rows in this tile
+      const size_t warp_off = size_t(m_blk * BM + quarter * 32) * size_t(args.J) + size_t(n_blk) * BN;
+      const int n_valid = min(BN, args.J - n_blk * BN);           // ragged last tile in N (multiple of 16)
+      uint8_t* stage = s_out + quarter * 4096;
+      uint32_t v[32];
+      if (n_valid >= 32) tmem_ld_32x32(t_base, v); else tmem_ld_32x16(t_base, v);
 #pragma unroll 1
-      for (int c = 0; c < n_chunks; c += 2) {
+      for (int c0 = 0; c0 < n_valid; c0 += 32) {
+        const int width = min(32, n_valid - c0);
+        const int next_width = n_valid - (c0 + 32);                // <= 0: this is the last chunk
+        const uint32_t next_taddr = t_base + uint32_t(c0 + 32);
         tmem_ld_wait();
-        if (c + 1 < n_chunks) tmem_ld_32x16(t_base + uint32_t((c + 1) * CHUNK), vb);
-        scale_store16(va, d_row, dcol + c * CHUNK, args.out, args.out_f32, row_off + size_t(c * CHUNK));
-        if (c + 1 < n_chunks) {
-          tmem_ld_wait();
-          if (c + 2 < n_chunks) tmem_ld_32x16(t_base + uint32_t((c + 2) * CHUNK), va);
-          scale_store16(vb, d_row, dcol + (c + 1) * CHUNK, args.out, args.out_f32,
-                        row_off + size_t((c + 1) * CHUNK));
+        if (width == 32) {
+          if (args.out_f32)
+            scale_stage_store<32, true>(v, d_row, dcol + c0, stage, args.out, warp_off + c0, args.J, lane, next_taddr,
+                                        next_width);
+          else
+            scale_stage_store<32, false>(v, d_row, dcol + c0, stage, args.out, warp_off + c0, args.J, lane, next_taddr,
+                                         next_width);
+        } else {
+          if (args.out_f32)
+            scale_stage_store<16, true>(v, d_row, dcol + c0, stage, args.out, warp_off + c0, args.J, lane, next_taddr, 0);
+          else
+            scale_stage_store<16, false>(v, d_row, dcol + c0, stage, args.out, warp_off + c0, args.J, lane, next_taddr, 0);
         }
       }
       tc_fence_before();
