@@ -70,10 +70,9 @@ const char* fp4_status_string(int code) {
 
 size_t fp4_workspace_bytes(int64_t M, int64_t K, int64_t N) {
   if (M <= 0 || K <= 0 || N <= 0) return 0;
-  size_t q = quantize_scratch_bytes(M, K);
-  const size_t qw = quantize_scratch_bytes(K, N);
+  // forward: A and W are quantised concurrently, each in its own scratch; backward: dY alone
+  size_t q = quantize_scratch_bytes(M, K) + quantize_scratch_bytes(K, N);
   const size_t qg = quantize_scratch_bytes(M, N);
-  if (qw > q) q = qw;
   if (qg > q) q = qg;
   return q + linear_scratch_bytes(M, K, N) + 4096;
 }
@@ -91,6 +90,8 @@ int fp4_create(fp4_ctx** out, int device, size_t workspace_bytes) {
   ctx->profile = 0;
   ctx->launch_count = 0;
   ctx->records = new (std::nothrow) std::vector<ProfRecord>();
+  for (auto& s : ctx->side) s = nullptr;
+  for (auto& e : ctx->ev) e = nullptr;
   cudaDeviceProp prop;
   if (!ctx->records || cudaGetDeviceProperties(&prop, device) != cudaSuccess) {
     delete ctx->records;
@@ -115,6 +116,13 @@ int fp4_create(fp4_ctx** out, int device, size_t workspace_bytes) {
     }
     ctx->workspace_bytes = workspace_bytes;
   }
+  bool ok = true;
+  for (auto& s : ctx->side) ok = ok && cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) == cudaSuccess;
+  for (auto& e : ctx->ev) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) {
+    fp4_destroy(ctx);
+    return FP4_ERR_CUDA;
+  }
   *out = ctx;
   return FP4_OK;
 }
@@ -122,6 +130,10 @@ int fp4_create(fp4_ctx** out, int device, size_t workspace_bytes) {
 int fp4_destroy(fp4_ctx* ctx) {
   if (!ctx) return FP4_ERR_NULL;
   cudaSetDevice(ctx->device);
+  for (auto& s : ctx->side)
+    if (s) cudaStreamDestroy(s);
+  for (auto& e : ctx->ev)
+    if (e) cudaEventDestroy(e);
   if (ctx->workspace) cudaFree(ctx->workspace);
   if (ctx->records) {
     fp4_profile_reset(ctx);
@@ -199,24 +211,34 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
                     fp4_qtensor* savedA, fp4_qtensor* savedW, int32_t* status) {
   const bool occ = alpha < 1.0;
   float* y1 = occ ? arena.take<float>(size_t(M) * size_t(N)) : nullptr;
+  char* scratch_a = arena.take<char>(quantize_scratch_bytes(M, K));
+  char* scratch_w = reuse_w ? nullptr : arena.take<char>(quantize_scratch_bytes(K, N));
   if (!arena.ok) return FP4_ERR_WORKSPACE;
-  Arena qa_arena(arena.base + arena.off, arena.size - arena.off);
-
   int rc;
+
+  // Three independent chains: W (side stream 0), A up to its codes (caller's stream), and the
+  // mask -> CSR / CSC stage of A (side stream 1), which only the compensation and the backward need.
   if (!reuse_w) {
-    Arena a = qa_arena;
+    FP4_CUDA_TRY(cudaEventRecord(ctx->ev[0], st));
+    FP4_CUDA_TRY(cudaStreamWaitEvent(ctx->side[0], ctx->ev[0], 0));
+    Arena a(scratch_w, quantize_scratch_bytes(K, N));
     savedW->rows = K;
     savedW->cols = N;
-    rc = launch_quantize(ctx, st, a, W_bf16, K, N, /*scale_axis=*/1, 1.0, nullptr, 0, savedW, status);
+    rc = launch_quantize(ctx, ctx->side[0], a, W_bf16, K, N, /*scale_axis=*/1, 1.0, nullptr, 0, savedW, status);
     if (rc != FP4_OK) return rc;
+    FP4_CUDA_TRY(cudaEventRecord(ctx->ev[1], ctx->side[0]));
   }
   {
-    Arena a = qa_arena;
+    Arena a(scratch_a, quantize_scratch_bytes(M, K));
     savedA->rows = M;
     savedA->cols = K;
-    rc = launch_quantize(ctx, st, a, A_bf16, M, K, /*scale_axis=*/0, alpha, nullptr, 0, savedA, status);
+    const SparseOverlap so = {ctx->side[1], ctx->ev[2], ctx->ev[3]};
+    rc = launch_quantize(ctx, st, a, A_bf16, M, K, /*scale_axis=*/0, alpha, nullptr, 0, savedA, status,
+                         occ ? &so : nullptr);
     if (rc != FP4_OK) return rc;
+    if (occ) FP4_CUDA_TRY(cudaEventRecord(ctx->ev[4], ctx->side[1]));       // CSR and CSC complete
   }
+  if (!reuse_w) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[1], 0));
   // Y1 = (Q(A_c) Q(W)) * d_A[m] * d_W[n]: A codes [M x K/2], W codes transposed [N x K/2].
   if (!occ) {
     return launch_gemm_fp4(ctx, st, savedA->codes, savedW->codes_t, M, N, K, savedA->amax, savedW->amax, Y, out_f32,
@@ -225,9 +247,12 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
   rc = launch_gemm_fp4(ctx, st, savedA->codes, savedW->codes_t, M, N, K, savedA->amax, savedW->amax, y1, 1, gemm_kind,
                        status);
   if (rc != FP4_OK) return rc;
-  // Y = store(Y1 + (A - A_c) W): one rounding of the fp32 sum.
-  return launch_comp_fwd(ctx, st, y1, savedA->csr_rowptr, savedA->csr_col, savedA->csr_val, W_bf16, M, K, N, Y,
-                         out_f32);
+  // Y = store(Y1 + (A - A_c) W): one rounding of the fp32 sum.  Needs the CSR.
+  FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[3], 0));
+  rc = launch_comp_fwd(ctx, st, y1, savedA->csr_rowptr, savedA->csr_col, savedA->csr_val, W_bf16, M, K, N, Y, out_f32);
+  if (rc != FP4_OK) return rc;
+  FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[4], 0));                      // savedA is complete on return
+  return FP4_OK;
 }
 
 }  // namespace
@@ -287,18 +312,29 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
     rc = launch_quantize(ctx, st, a, dY_bf16, M, N, /*scale_axis=*/1, 1.0, savedA->amax, 1, &g, status);
     if (rc != FP4_OK) return rc;
   }
+  // The two gradients are independent from here on: the weight-gradient chain runs on a side stream.
+  cudaStream_t sw = st;
+  if (dA && dW) {
+    sw = ctx->side[0];
+    FP4_CUDA_TRY(cudaEventRecord(ctx->ev[5], st));
+    FP4_CUDA_TRY(cudaStreamWaitEvent(sw, ctx->ev[5], 0));
+  }
+  if (dW) {
+    // S[k,n] = d_G''[n] * sum_m Aq[m,k] G''[m,n], then the compensation and the DGE factor.
+    rc = launch_gemm_fp4(ctx, sw, savedA->codes_t, g2_codes, K, N, M, nullptr, g2_amax, s, 1, gemm_kind, status);
+    if (rc != FP4_OK) return rc;
+    rc = launch_comp_wgrad_dge(ctx, sw, s, savedA->csc_colptr, savedA->csc_row, savedA->csc_val, dY_bf16, W_bf16,
+                               savedW->amax, col_list, M, K, N, dge_on, dge_k, dge_clip, dW, out_f32);
+    if (rc != FP4_OK) return rc;
+  }
   if (dA) {
     // dA = d_G'[m] * sum_n G'[m,n] Wq[k,n]
     rc = launch_gemm_fp4(ctx, st, g1_codes, savedW->codes, M, K, N, g1_amax, nullptr, dA, out_f32, gemm_kind, status);
     if (rc != FP4_OK) return rc;
   }
-  if (dW) {
-    // S[k,n] = d_G''[n] * sum_m Aq[m,k] G''[m,n], then the compensation and the DGE factor.
-    rc = launch_gemm_fp4(ctx, st, savedA->codes_t, g2_codes, K, N, M, nullptr, g2_amax, s, 1, gemm_kind, status);
-    if (rc != FP4_OK) return rc;
-    rc = launch_comp_wgrad_dge(ctx, st, s, savedA->csc_colptr, savedA->csc_row, savedA->csc_val, dY_bf16, W_bf16,
-                               savedW->amax, col_list, M, K, N, dge_on, dge_k, dge_clip, dW, out_f32);
-    if (rc != FP4_OK) return rc;
+  if (sw != st) {
+    FP4_CUDA_TRY(cudaEventRecord(ctx->ev[6], sw));
+    FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[6], 0));
   }
   return FP4_OK;
 }

@@ -34,6 +34,8 @@ struct fp4_ctx {
   char*    workspace;
   size_t   workspace_bytes;
   void*    encode_tiled;       // cuTensorMapEncodeTiled, fetched through the runtime
+  cudaStream_t side[2];        // side streams for independent kernel chains inside one call
+  cudaEvent_t  ev[8];          // fork / join events of those chains
   int      profile;            // record CUDA events around every kernel class
   long long launch_count;      // kernels enqueued since the last reset
   std::vector<ProfRecord>* records;
@@ -93,12 +95,22 @@ int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, c
                     int64_t I, int64_t J, int64_t C, const float* row_amax, const float* col_amax,
                     void* out, int out_f32, int gemm_kind, int32_t* status);
 
+// Lets the mask -> CSR / CSC stage of a clamping quantisation run on a side stream: it starts
+// after `encoded` (recorded on the main stream), `csr_done` is recorded on the side stream once
+// the CSR is complete.  The caller joins the side stream (the CSC follows the CSR on it).
+struct SparseOverlap {
+  cudaStream_t stream;
+  cudaEvent_t encoded;
+  cudaEvent_t csr_done;
+};
+
 // Quantiser pieces (quantize.cu)
 // `prescale_is_amax`: the prescale vector holds amax values and stands for amax / 6.
 size_t quantize_scratch_bytes(int64_t rows, int64_t cols);
 int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void* x_bf16, int64_t rows,
                     int64_t cols, int scale_axis, double alpha, const float* prescale,
-                    int prescale_is_amax, fp4_qtensor* out, int32_t* status);
+                    int prescale_is_amax, fp4_qtensor* out, int32_t* status,
+                    const SparseOverlap* overlap = nullptr);
 
 // dY for both backward GEMMs in one read: row-scaled codes of x (.) (amax_col_pre / 6) with their
 // row amax, and column-scaled transposed codes of x (.) (amax_row_pre / 6) with their column amax.

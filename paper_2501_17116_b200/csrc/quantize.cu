@@ -699,7 +699,7 @@ size_t quantize_scratch_bytes(int64_t rows, int64_t cols) {
 
 int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void* x_bf16, int64_t rows64,
                     int64_t cols64, int scale_axis, double alpha, const float* prescale, int prescale_is_amax,
-                    fp4_qtensor* out, int32_t* status) {
+                    fp4_qtensor* out, int32_t* status, const SparseOverlap* overlap) {
   const int rows = int(rows64), cols = int(cols64);
   const long long n = (long long)rows * cols;
   const bool occ = alpha < 1.0;
@@ -744,19 +744,25 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
       KernelScope scope(ctx, stream, KC_ENCODE, 1);
       encode_kernel<MODE_ROWS, true, false><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
     }
-    KernelScope scope(ctx, stream, KC_SPARSE, 5);
+    cudaStream_t sp = stream;
+    if (overlap && overlap->stream) {
+      sp = overlap->stream;
+      FP4_CUDA_TRY(cudaEventRecord(overlap->encoded, stream));
+      FP4_CUDA_TRY(cudaStreamWaitEvent(sp, overlap->encoded, 0));
+    }
+    KernelScope scope(ctx, sp, KC_SPARSE, 5);
     const uint32_t* mask32 = reinterpret_cast<const uint32_t*>(sc.mask);
     const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x_bf16);
     const int strips = rows / ENC_TM;
-    scan_counts_kernel<<<1, 1024, 0, stream>>>(sc.row_cnt, rows, out->csr_rowptr, out->nnz, out->sparse_cap, status);
-    csr_fill_kernel<<<(rows + 7) / 8, 256, 0, stream>>>(mask32, xb, rows, cols, out->thresholds, out->csr_rowptr,
-                                                        out->sparse_cap, out->csr_col, out->csr_val);
-    csc_strip_prefix_kernel<<<(cols + 255) / 256, 256, 0, stream>>>(sc.strip_cnt, cols, strips, sc.strip_off,
-                                                                    sc.col_cnt);
-    scan_counts_kernel<<<1, 1024, 0, stream>>>(sc.col_cnt, cols, out->csc_colptr, nullptr, out->sparse_cap, nullptr);
+    scan_counts_kernel<<<1, 1024, 0, sp>>>(sc.row_cnt, rows, out->csr_rowptr, out->nnz, out->sparse_cap, status);
+    csr_fill_kernel<<<(rows + 7) / 8, 256, 0, sp>>>(mask32, xb, rows, cols, out->thresholds, out->csr_rowptr,
+                                                    out->sparse_cap, out->csr_col, out->csr_val);
+    if (sp != stream) FP4_CUDA_TRY(cudaEventRecord(overlap->csr_done, sp));
+    csc_strip_prefix_kernel<<<(cols + 255) / 256, 256, 0, sp>>>(sc.strip_cnt, cols, strips, sc.strip_off, sc.col_cnt);
+    scan_counts_kernel<<<1, 1024, 0, sp>>>(sc.col_cnt, cols, out->csc_colptr, nullptr, out->sparse_cap, nullptr);
     const dim3 cgrid((cols / 32 + 7) / 8, strips);
-    csc_fill_kernel<<<cgrid, 256, 0, stream>>>(mask32, xb, rows, cols, out->thresholds, out->csc_colptr, sc.strip_off,
-                                               out->sparse_cap, out->csc_row, out->csc_val);
+    csc_fill_kernel<<<cgrid, 256, 0, sp>>>(mask32, xb, rows, cols, out->thresholds, out->csc_colptr, sc.strip_off,
+                                           out->sparse_cap, out->csc_row, out->csc_val);
   } else {
     if (prescale && prescale_is_amax) {
       float* d = scale_axis == 0 ? sc.pre_cols : sc.pre_rows;
