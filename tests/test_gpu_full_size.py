@@ -1,0 +1,147 @@
+"""Parity at the full sizes of the workload list, through the same calls bench.py times.
+
+The oracle cannot produce whole outputs at these sizes in seconds, so it is evaluated on
+samples: thresholds, every amax, the residual count and the CSR row pointer are compared in
+full (they are cheap vector operations), while codes, sparse entries and the outputs of the
+three GEMMs are compared on sampled rows / columns / entries, each computed by the oracle's own
+functions on the slice that determines it (a row of A with the tensor-wide thresholds, a column
+of W, a row or column of dY with the folded de-scale vector).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import fp4_oracle as O
+from paper_2501_17116_b200 import workloads as WL
+
+pytestmark = pytest.mark.gpu
+RTOL = 1e-3
+
+# (config index, linear name, alpha)
+CASES = [(1, "q", 0.999), (1, "down", 0.999), (2, "down", 0.99), (3, "q", 0.9999), (4, "gate", 0.99)]
+
+
+def _dev(bits):
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def _f32(bits):
+    return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+def _nibbles_of_rows(packed_t_dev, rows):
+    """codes_t is [cols x rows/2]: gather the codes of the given source rows -> [len(rows), cols]."""
+    r = torch.as_tensor(rows, device="cuda")
+    b = packed_t_dev[:, r // 2].cpu().numpy()                       # [cols, len(rows)]
+    odd = (np.asarray(rows) % 2 == 1)[None, :]
+    return np.where(odd, b >> 4, b & 0xF).T.astype(np.uint8)
+
+
+def _close(got, want, scale, what):
+    err = np.abs(np.asarray(got, dtype=np.float64) - want)
+    bad = err > RTOL * scale + 1e-300
+    assert not bad.any(), f"{what}: {bad.sum()} of {bad.size} outside tolerance"
+
+
+@pytest.mark.parametrize("ci,lname,alpha", CASES)
+def test_full_size_layer_matches_sampled_oracle(lib, ci, lname, alpha):
+    cfg = WL.CONFIGS[ci]
+    lin = next(l for l in cfg.linears if l.name == lname)
+    M, K, N = cfg.M, lin.K, lin.N
+    rng = np.random.default_rng(ci * 100 + K)
+    a_bits = WL.activations(cfg, K)
+    w_bits = WL.weights(cfg, K, N)
+    dy_bits = WL.output_grads(cfg, N)
+    A, W, dY = _dev(a_bits), _dev(w_bits), _dev(dy_bits)
+
+    ctx = lib.Context.for_shape(M, K, N)
+    y32, sa, sw = lib.fp4_linear_fwd(ctx, A, W, alpha, out_f32=True)
+    da32, dw32 = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, out_f32=True)
+    torch.cuda.synchronize()
+    assert ctx.read_status() == 0
+
+    # ---- thresholds, counts, amax: in full -------------------------------------------------
+    a32, w32, dy32 = _f32(a_bits), _f32(w_bits), _f32(dy_bits)
+    n = M * K
+    n_tail = O.tail_count(n, alpha)
+    srt = np.sort(a32, axis=None)                                    # the order statistics of R7
+    lo, hi = float(srt[n_tail]) + 0.0, float(srt[n - 1 - n_tail]) + 0.0
+    del srt
+    th = sa.thresholds.cpu().numpy()
+    assert (float(th[0]), float(th[1])) == (lo, hi)
+    out_mask = (a32 > hi) | (a32 < lo)
+    assert int(sa.nnz.item()) == int(out_mask.sum()) <= 2 * n_tail
+    rowptr = np.concatenate([[0], np.cumsum(out_mask.sum(axis=1))]).astype(np.int32)
+    colptr = np.concatenate([[0], np.cumsum(out_mask.sum(axis=0))]).astype(np.int32)
+    np.testing.assert_array_equal(sa.csr_rowptr.cpu().numpy(), rowptr)
+    np.testing.assert_array_equal(sa.csc_colptr.cpu().numpy(), colptr)
+    amax_a = np.abs(np.clip(a32, np.float32(lo), np.float32(hi))).max(axis=1)
+    amax_w = np.abs(w32).max(axis=0)
+    np.testing.assert_array_equal(sa.amax.cpu().numpy(), amax_a)
+    np.testing.assert_array_equal(sw.amax.cpu().numpy(), amax_w)
+    _, d_a = O.absmax_scales(amax_a)
+    _, d_w = O.absmax_scales(amax_w)
+
+    # ---- sampled rows of A: codes (both layouts), CSR entries ---------------------------------
+    hot_cols = np.argsort(out_mask.sum(axis=0))[-4:]
+    rows = np.unique(np.concatenate([rng.choice(M, 24, replace=False), [0, M - 1, 63, 64]]))
+    a_rows = O.bf16_bits_to_f64(a_bits[rows])
+    a_c, resid = O.occ_split(a_rows, lo, hi)
+    qa = O.absmax_quantize(a_c, 0)
+    np.testing.assert_array_equal(sa.codes[torch.as_tensor(rows, device="cuda")].cpu().numpy(), qa.packed())
+    np.testing.assert_array_equal(_nibbles_of_rows(sa.codes_t, rows), qa.codes)
+    csr_col, csr_val = sa.csr_col.cpu().numpy(), sa.csr_val.cpu().numpy()
+    for i, m in enumerate(rows):
+        seg = slice(rowptr[m], rowptr[m + 1])
+        cols_ref = np.nonzero(resid[i])[0]
+        np.testing.assert_array_equal(csr_col[seg], cols_ref)
+        np.testing.assert_array_equal(csr_val[seg], resid[i, cols_ref].astype(np.float32))
+    # ---- sampled columns of A: CSC entries -----------------------------------------------------
+    csc_row, csc_val = sa.csc_row.cpu().numpy(), sa.csc_val.cpu().numpy()
+    cols_a = np.unique(np.concatenate([rng.choice(K, 12, replace=False), hot_cols, [0, K - 1]]))
+    a_cols = O.bf16_bits_to_f64(a_bits[:, cols_a])
+    ac_cols, resid_cols = O.occ_split(a_cols, lo, hi)
+    for j, k in enumerate(cols_a):
+        seg = slice(colptr[k], colptr[k + 1])
+        rows_ref = np.nonzero(resid_cols[:, j])[0]
+        np.testing.assert_array_equal(csc_row[seg], rows_ref)
+        np.testing.assert_array_equal(csc_val[seg], resid_cols[rows_ref, j].astype(np.float32))
+
+    # ---- sampled columns of W: codes (both layouts) -------------------------------------------
+    cols_w = np.unique(np.concatenate([rng.choice(N, 28, replace=False), [0, N - 1, 239, 240]]))
+    qw = O.absmax_quantize(O.bf16_bits_to_f64(w_bits[:, cols_w]), 1)
+    np.testing.assert_array_equal(sw.codes_t[torch.as_tensor(cols_w, device="cuda")].cpu().numpy(), qw.packed_t())
+    # the row-major layout of W holds the same codes: rows of W are pairs of nibbles along n
+    w_codes_rows = O.unpack_nibbles(sw.codes[:, torch.as_tensor(cols_w // 2, device="cuda")].cpu().numpy())
+    pick = np.arange(len(cols_w)) * 2 + (cols_w % 2)
+    np.testing.assert_array_equal(w_codes_rows[:, pick], qw.codes)
+
+    # ---- forward: Y on rows x cols_w -------------------------------------------------------------
+    w_cols = O.bf16_bits_to_f64(w_bits[:, cols_w])
+    y_fp4 = (O.gemm_codes(qa.codes, qw.codes.T) * d_a[rows].astype(np.float64)[:, None]) \
+        * d_w[cols_w].astype(np.float64)[None, :]
+    y_comp = resid @ w_cols
+    got = y32[torch.as_tensor(rows, device="cuda")][:, torch.as_tensor(cols_w, device="cuda")].cpu().numpy()
+    _close(got, y_fp4 + y_comp, np.abs(y_fp4) + np.abs(y_comp), "Y")
+
+    # ---- dgrad: dA on rows x cols_a ----------------------------------------------------------------
+    qg1 = O.absmax_quantize(O.bf16_bits_to_f64(dy_bits[rows]), 0, prescale=d_w)
+    # codes of W rows cols_a (all N): scaled by the per-column gamma of the full tensor
+    gamma_w, _ = O.absmax_scales(amax_w)
+    w_sel = O.bf16_bits_to_f64(w_bits[cols_a])                       # [len(cols_a), N]
+    w_sel_codes = O.lut_quantize((w_sel * gamma_w.astype(np.float64)[None, :]).astype(np.float32))
+    da_ref = O.gemm_codes(qg1.codes, w_sel_codes) * qg1.descale.astype(np.float64)[:, None]
+    got = da32[torch.as_tensor(rows, device="cuda")][:, torch.as_tensor(cols_a, device="cuda")].cpu().numpy()
+    _close(got, da_ref, np.abs(da_ref), "dA")
+
+    # ---- wgrad: dW on cols_a x cols_w ----------------------------------------------------------------
+    gamma_a, _ = O.absmax_scales(amax_a)
+    a_sel_codes = O.lut_quantize((ac_cols * gamma_a.astype(np.float64)[:, None]).astype(np.float32))   # [M, len(cols_a)]
+    qg2 = O.absmax_quantize(O.bf16_bits_to_f64(dy_bits[:, cols_w]), 1, prescale=d_a)
+    s_fp4 = O.gemm_codes(a_sel_codes.T, qg2.codes.T) * qg2.descale.astype(np.float64)[None, :]
+    s_comp = resid_cols.T @ O.bf16_bits_to_f64(dy_bits[:, cols_w])
+    w_scaled = (O.bf16_bits_to_f64(w_bits[np.ix_(cols_a, cols_w)]) * gamma_w[cols_w].astype(np.float64)[None, :]).astype(np.float32)
+    factor = O.dge_fprime(w_scaled.astype(np.float64))
+    got = dw32[torch.as_tensor(cols_a, device="cuda")][:, torch.as_tensor(cols_w, device="cuda")].cpu().numpy()
+    _close(got, (s_fp4 + s_comp) * factor, (np.abs(s_fp4) + np.abs(s_comp)) * factor, "dW")
+    ctx.close()
