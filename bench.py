@@ -224,30 +224,51 @@ def main():
                                      gemm_kind=kind, read_status=False)
 
     # ------------------------------------------------------------------ device-resident ---
+    # The step is captured once into a CUDA graph (the library's side streams fork from and
+    # rejoin the capturing stream) and replayed: the timed region is K replays back to back.
     for _ in range(args.warmup):
         step()
     torch.cuda.synchronize()
     assert ctx.read_status() == 0, "device status word is set"
+    ctx.profile_reset()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    launches_per_step = ctx.launch_count()
+    for _ in range(args.warmup):
+        graph.replay()
+    torch.cuda.synchronize()
     sampler = ClockSampler(local_rank)
     sampler.start()
-    ctx.profile_reset()
-    ctx.profile_enable(True)
     harness.barrier()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.steps):
-        step()
+        graph.replay()
     e1.record()
     torch.cuda.synchronize()
     harness.barrier()
     ms = e0.elapsed_time(e1)
-    launches = ctx.launch_count()
+    launches = launches_per_step * args.steps
+    assert ctx.read_status() == 0, "device status word is set"
+
+    # Per-kernel-class device times: the same K steps again, launched plainly with a CUDA event
+    # pair around every kernel class on its launching stream (events cannot sit inside a graph).
+    ctx.profile_reset()
+    ctx.profile_enable(True)
+    torch.cuda.synchronize()
+    p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    p0.record()
+    for _ in range(args.steps):
+        step()
+    p1.record()
+    torch.cuda.synchronize()
+    ms_profiled = p0.elapsed_time(p1)
     prof = ctx.profile_read()
     ctx.profile_enable(False)
     ctx.profile_reset()
     nnz = [int(L["sa"].nnz.item()) if L["sa"].nnz is not None else 0 for L in layers]
-    assert ctx.read_status() == 0, "device status word is set"
 
     # ------------------------------------------------------------------ end to end ---------
     for _ in range(3):
@@ -326,6 +347,9 @@ def main():
             "config": {"workload": cfg.name, "tokens": M, "linears": [f"{L['name']}:{L['K']}x{L['N']}" for L in layers],
                        "alpha": alpha, "dge": True, "gemm_kind": "mxf4" if kind == 0 else "f8f6f4",
                        "l2": f"inputs exceed L2: {resident_bytes / 1e6:.0f} MB touched per step",
+                       "launch": "one CUDA graph per step, replayed",
+                       "kernel_timing": f"CUDA events per kernel class over {args.steps} plainly launched steps "
+                                        f"({ms_profiled / args.steps:.3f} ms/step with the events)",
                        "replicas": world},
             "e2e": {"value": value_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": 1e3 * sec_e2e / args.steps},
