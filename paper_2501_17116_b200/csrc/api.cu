@@ -23,7 +23,7 @@ size_t linear_scratch_bytes(int64_t M, int64_t K, int64_t N) {
   b += 2 * round256(size_t(M) * size_t(N) / 2);       // dY codes, both scalings
   b += round256(size_t(M) * 4) + round256(size_t(N) * 4);   // their amax vectors
   b += 2 * round256(size_t(M > N ? M : N) * 4);       // de-scale vectors used as prescale
-  b += round256((2 * size_t(K) + 2) * 4);             // lists of columns that hold residual entries
+  b += round256((2 * size_t(K) + 2) * 4) + round256(size_t(K) * 4);   // non-empty residual columns, their slots
   return b;
 }
 
@@ -282,15 +282,31 @@ namespace {
 int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_bf16, const void* W_bf16,
                     const fp4_qtensor* savedA, const fp4_qtensor* savedW, int64_t M, int64_t K, int64_t N, int dge_on,
                     float dge_k, float dge_clip, int gemm_kind, void* dA, void* dW, int out_f32, int32_t* status) {
-  float* s = dW ? arena.take<float>(size_t(K) * size_t(N)) : nullptr;
+  const bool has_comp = dW && savedA->csc_colptr != nullptr;
+  float* comp = has_comp ? arena.take<float>(size_t(K) * size_t(N)) : nullptr;   // compact: one row per non-empty column
   uint8_t* g1_codes = dA ? arena.take<uint8_t>(size_t(M) * size_t(N) / 2) : nullptr;   // dY (.) d_W, token-wise
   uint8_t* g2_codes = dW ? arena.take<uint8_t>(size_t(M) * size_t(N) / 2) : nullptr;   // dY (.) d_A, channel-wise
   float* g1_amax = arena.take<float>(size_t(M));
   float* g2_amax = arena.take<float>(size_t(N));
-  int* col_list = arena.take<int>(2 * size_t(K) + 2);
+  int* col_lists = arena.take<int>(2 * size_t(K) + 2);
+  int* slot_of_col = arena.take<int>(size_t(K));
   if (!arena.ok) return FP4_ERR_WORKSPACE;
   Arena q_arena(arena.base + arena.off, arena.size - arena.off);
   int rc;
+
+  // The weight-gradient chain runs on a side stream when both gradients are wanted.  Its first
+  // part, the compensation dA^T dY of the non-empty residual columns, needs neither GEMM operand.
+  cudaStream_t sw = st;
+  if (dA && dW) {
+    sw = ctx->side[0];
+    FP4_CUDA_TRY(cudaEventRecord(ctx->ev[5], st));
+    FP4_CUDA_TRY(cudaStreamWaitEvent(sw, ctx->ev[5], 0));
+  }
+  if (has_comp) {
+    rc = launch_comp_wgrad(ctx, sw, savedA->csc_colptr, savedA->csc_row, savedA->csc_val, dY_bf16, col_lists,
+                           slot_of_col, comp, K, N);
+    if (rc != FP4_OK) return rc;
+  }
 
   // dgrad operand: G' = dY (.) d_W[n], token-wise codes [M x N/2].
   // wgrad operand: G'' = dY (.) d_A[m], channel-wise codes transposed [N x M/2].
@@ -299,6 +315,8 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
     rc = launch_quantize_dual(ctx, st, a, dY_bf16, M, N, savedW->amax, savedA->amax, g1_codes, g1_amax, g2_codes,
                               g2_amax);
     if (rc != FP4_OK) return rc;
+    FP4_CUDA_TRY(cudaEventRecord(ctx->ev[6], st));
+    FP4_CUDA_TRY(cudaStreamWaitEvent(sw, ctx->ev[6], 0));
   } else if (dA) {
     fp4_qtensor g = {};
     g.rows = M; g.cols = N; g.codes = g1_codes; g.amax = g1_amax;
@@ -312,19 +330,18 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
     rc = launch_quantize(ctx, st, a, dY_bf16, M, N, /*scale_axis=*/1, 1.0, savedA->amax, 1, &g, status);
     if (rc != FP4_OK) return rc;
   }
-  // The two gradients are independent from here on: the weight-gradient chain runs on a side stream.
-  cudaStream_t sw = st;
-  if (dA && dW) {
-    sw = ctx->side[0];
-    FP4_CUDA_TRY(cudaEventRecord(ctx->ev[5], st));
-    FP4_CUDA_TRY(cudaStreamWaitEvent(sw, ctx->ev[5], 0));
-  }
   if (dW) {
-    // S[k,n] = d_G''[n] * sum_m Aq[m,k] G''[m,n], then the compensation and the DGE factor.
-    rc = launch_gemm_fp4(ctx, sw, savedA->codes_t, g2_codes, K, N, M, nullptr, g2_amax, s, 1, gemm_kind, status);
-    if (rc != FP4_OK) return rc;
-    rc = launch_comp_wgrad_dge(ctx, sw, s, savedA->csc_colptr, savedA->csc_row, savedA->csc_val, dY_bf16, W_bf16,
-                               savedW->amax, col_list, M, K, N, dge_on, dge_k, dge_clip, dW, out_f32);
+    // dW[k,n] = store( (d_G''[n] * sum_m Aq[m,k] G''[m,n] + comp[k,n]) * Q'(W[k,n] * 6 / amax_W[n]) ):
+    // the compensation rows and the DGE factor are applied in the GEMM's epilogue.
+    GemmEpilogue epi = {};
+    epi.addend = comp;
+    epi.slot_of_row = slot_of_col;
+    epi.w_bf16 = dge_on ? W_bf16 : nullptr;
+    epi.w_amax = savedW->amax;
+    epi.dge_k = dge_k;
+    epi.dge_clip = dge_clip;
+    rc = launch_gemm_fp4(ctx, sw, savedA->codes_t, g2_codes, K, N, M, nullptr, g2_amax, dW, out_f32, gemm_kind, status,
+                         &epi);
     if (rc != FP4_OK) return rc;
   }
   if (dA) {
@@ -333,8 +350,8 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
     if (rc != FP4_OK) return rc;
   }
   if (sw != st) {
-    FP4_CUDA_TRY(cudaEventRecord(ctx->ev[6], sw));
-    FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[6], 0));
+    FP4_CUDA_TRY(cudaEventRecord(ctx->ev[7], sw));
+    FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[7], 0));
   }
   return FP4_OK;
 }

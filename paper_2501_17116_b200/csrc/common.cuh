@@ -88,12 +88,41 @@ struct Arena {
   }
 };
 
+// DGE derivative of Eq. 8 on a scaled weight, capped at `clip`.  The E2M1 grid has steps of 0.5
+// below 2, 1 on [2, 4) and 2 from 4 up, i.e. delta = 2^(max(e, 0) - 1) with e the binary exponent
+// of |w| (capped at the last interval, whose formula continues past 6).  With t = |w| / delta the
+// position inside the interval [g, g + delta], mapped to [-1, 1], is u = 2 (t - floor(t)) - 1.
+// Branch-free: the exponent arithmetic is done on the float's bit pattern.
+__device__ __forceinline__ float dge_factor(float ws, float expo, float inv_k, float clip) {
+  const float a = fabsf(ws);
+  int em = int(__float_as_uint(a) >> 23);
+  em = min(max(em, 127), 129);                                   // exponent 0, 1 or 2
+  const float inv_delta = __uint_as_float(uint32_t(255 - em) << 23);    // 2, 1 or 1/2
+  const float t = a * inv_delta;                                 // exact: a power of two
+  const float g = em == 129 ? 2.0f : floorf(t);                  // last interval starts at 4 = 2 delta
+  const float u = fabsf(fmaf(t - g, 2.0f, -1.0f));
+  // |u|^(1/k - 1) = 2^((1/k - 1) log2 |u|); u = 0 gives +inf, which the cap turns into `clip`
+  const float d = inv_k * exp2f(expo * __log2f(u));
+  return fminf(d, clip);
+}
+
+// Work fused into the epilogue of the weight-gradient GEMM (all null / zero: plain epilogue):
+//   out[k, n] = store( (acc * d_col[n] + addend[slot_of_row[k], n]) * Q'(w[k, n] * 6 / w_amax[n]) )
+struct GemmEpilogue {
+  const float* addend;        // compact [slots x J] fp32 rows, added before the DGE factor (or null)
+  const int*   slot_of_row;   // [I]: row of `addend` that belongs to output row i, -1 for none
+  const void*  w_bf16;        // [I x J] BF16 weights whose scaled values drive the DGE factor (or null)
+  const float* w_amax;        // [J]
+  float dge_k, dge_clip;
+};
+
 // ---- internal launchers (each enqueues on `stream`, returns an FP4_* host code) -------------
 
 // out[i,j] = (sum_c a[i,c] b[j,c]) * (row_amax[i]/6) * (col_amax[j]/6)
 int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, const uint8_t* b_codes,
                     int64_t I, int64_t J, int64_t C, const float* row_amax, const float* col_amax,
-                    void* out, int out_f32, int gemm_kind, int32_t* status);
+                    void* out, int out_f32, int gemm_kind, int32_t* status,
+                    const GemmEpilogue* epilogue = nullptr);
 
 // Lets the mask -> CSR / CSC stage of a clamping quantisation run on a side stream: it starts
 // after `encoded` (recorded on the main stream), `csr_done` is recorded on the side stream once
@@ -124,9 +153,10 @@ int launch_quantize_dual(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const 
 int launch_comp_fwd(fp4_ctx* ctx, cudaStream_t stream, const float* y1, const int32_t* rowptr,
                     const int32_t* col, const float* val, const void* w_bf16, int64_t M, int64_t K,
                     int64_t N, void* y, int out_f32);
-// dw[k,:] = store( (s[k,:] + sum_{entries of column k} val * dy[row,:]) * Q'(w[k,:] * gamma[:]) )
-int launch_comp_wgrad_dge(fp4_ctx* ctx, cudaStream_t stream, float* s, const int32_t* colptr,
-                          const int32_t* row, const float* val, const void* dy_bf16,
-                          const void* w_bf16, const float* w_amax, int* col_list /*[2 K + 2] scratch*/,
-                          int64_t M, int64_t K, int64_t N, int dge_on, float dge_k, float dge_clip,
-                          void* dw, int out_f32);
+// Weight-gradient compensation into a compact buffer: for every column k of the residual that
+// holds entries, comp[slot_of_col[k], :] = sum_{entries of column k} val * dy[row, :].
+// `lists`: scratch of 2 K + 2 ints; `slot_of_col`: [K] ints (-1 where the column is empty).
+int launch_comp_wgrad(fp4_ctx* ctx, cudaStream_t stream, const int32_t* colptr, const int32_t* row,
+                      const float* val, const void* dy_bf16, int* lists, int* slot_of_col, float* comp,
+                      int64_t K, int64_t N);
+

@@ -2,7 +2,8 @@
 // fused with the final store, and the DGE factor of the weight gradient (Eq. 6, Eq. 8).
 //
 //   forward   Y[m, :]  = store( Y1[m, :] + sum_{(m,k) in dA} dA[m,k] * W[k, :] )
-//   wgrad     dW[k, :] = store( (S[k, :] + sum_{(m,k) in dA} dA[m,k] * dY[m, :]) * Q'(W[k,:] * gamma[:]) )
+//   wgrad     C[slot(k), :] = sum_{(m,k) in dA} dA[m,k] * dY[m, :]   for the columns k that hold entries;
+//             the weight-gradient GEMM adds C and applies the DGE factor in its epilogue
 //
 // Both are "sparse row times dense BF16 matrix" with fp32 accumulation on the plain ALUs: a warp
 // owns one output row and 256 of its columns (8 per lane); the sparse entries of that row (CSR
@@ -81,21 +82,6 @@ comp_fwd_kernel(const float* __restrict__ y1, const int* __restrict__ rowptr, co
   store8(y, out_f32, off, y8);
 }
 
-// DGE derivative of Eq. 8 on a scaled weight, capped at `clip`.  The E2M1 grid has steps of 0.5
-// below 2, 1 on [2, 4) and 2 from 4 up; u = 2 (|w| - g) / delta - 1 is the position inside the
-// interval [g, g + delta] mapped to [-1, 1].
-__device__ __forceinline__ float dge_factor(float ws, float expo, float inv_k, float clip) {
-  const float a = fabsf(ws);
-  float g, two_over_delta;
-  if (a < 2.0f) { g = 0.5f * floorf(2.0f * a); two_over_delta = 4.0f; }
-  else if (a < 4.0f) { g = floorf(a); two_over_delta = 2.0f; }
-  else { g = 4.0f; two_over_delta = 1.0f; }
-  const float u = fabsf((a - g) * two_over_delta - 1.0f);
-  // |u|^(1/k - 1) = 2^((1/k - 1) log2 |u|); u = 0 gives +inf, which the cap turns into `clip`
-  const float d = inv_k * exp2f(expo * __log2f(u));
-  return fminf(d, clip);
-}
-
 constexpr int LONG_COLUMN = 64;            // entries from which a column gets a whole 1024-thread block
 constexpr int LONG_THREADS = 1024;
 
@@ -103,7 +89,7 @@ constexpr int LONG_THREADS = 1024;
 // LONG_COLUMN entries: the outlier channels) and "short" ones; counts[0], counts[1] their sizes.
 __global__ void __launch_bounds__(1024, 1)
 nonempty_columns_kernel(const int* __restrict__ colptr, int K, int* __restrict__ list_long,
-                        int* __restrict__ list_short, int* __restrict__ counts) {
+                        int* __restrict__ list_short, int* __restrict__ counts, int* __restrict__ slot_of_col) {
   __shared__ unsigned long long warp_tot[32];
   const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
   const int per = (K + 1023) / 1024;
@@ -133,11 +119,15 @@ nonempty_columns_kernel(const int* __restrict__ colptr, int K, int* __restrict__
   }
   __syncthreads();
   const unsigned long long before = incl - c + (warp ? warp_tot[warp - 1] : 0ull);
+  // rows of the compact buffer: long columns first (in list order), then the short ones
+  const int n_long = int(warp_tot[31] & 0xFFFFFFFFull);
   int pos_long = int(before & 0xFFFFFFFFull), pos_short = int(before >> 32);
   for (int k = b; k < e; ++k) {
     const int n = colptr[k + 1] - colptr[k];
-    if (n >= LONG_COLUMN) list_long[pos_long++] = k;
-    else if (n > 0) list_short[pos_short++] = k;
+    int slot = -1;
+    if (n >= LONG_COLUMN) { slot = pos_long; list_long[pos_long++] = k; }
+    else if (n > 0) { slot = n_long + pos_short; list_short[pos_short++] = k; }
+    slot_of_col[k] = slot;
   }
   if (t == 1023) {
     counts[0] = int(warp_tot[31] & 0xFFFFFFFFull);
@@ -179,13 +169,9 @@ __device__ __forceinline__ void strided_entries_times_dense(float (&acc)[8], con
   }
 }
 
-__device__ __forceinline__ void add8_to(float* dst, const float (&t)[8]) {
-  float4 a = *reinterpret_cast<float4*>(dst);
-  float4 b = *reinterpret_cast<float4*>(dst + 4);
-  a.x += t[0]; a.y += t[1]; a.z += t[2]; a.w += t[3];
-  b.x += t[4]; b.y += t[5]; b.z += t[6]; b.w += t[7];
-  *reinterpret_cast<float4*>(dst) = a;
-  *reinterpret_cast<float4*>(dst + 4) = b;
+__device__ __forceinline__ void store8_f32(float* dst, const float (&t)[8]) {
+  *reinterpret_cast<float4*>(dst) = make_float4(t[0], t[1], t[2], t[3]);
+  *reinterpret_cast<float4*>(dst + 4) = make_float4(t[4], t[5], t[6], t[7]);
 }
 
 // Weight-gradient compensation, step 1: S[k, n-block] += sum over the entries of column k of
@@ -194,7 +180,7 @@ __device__ __forceinline__ void add8_to(float* dst, const float (&t)[8]) {
 // Long columns: one 1024-thread block per (column, 256 outputs); its 32 warps take the entries
 // round-robin and their partial sums are added in warp order (independent of scheduling).
 __global__ void __launch_bounds__(LONG_THREADS, 1)
-comp_wgrad_long_kernel(float* __restrict__ s, const int* __restrict__ colptr, const int* __restrict__ row,
+comp_wgrad_long_kernel(float* __restrict__ comp, const int* __restrict__ colptr, const int* __restrict__ row,
                        const float* __restrict__ val, const uint4* __restrict__ dy, const int* __restrict__ list,
                        const int* __restrict__ count, int N) {
   __shared__ float part[32][32][9];                 // [warp][lane][8 (+1 pad)]
@@ -217,57 +203,25 @@ comp_wgrad_long_kernel(float* __restrict__ s, const int* __restrict__ colptr, co
 #pragma unroll
         for (int c = 0; c < 8; ++c) t[c] += part[w][lane][c];
       }
-      add8_to(s + (long long)k * N + n0, t);
+      store8_f32(comp + (long long)slot * N + n0, t);
     }
   }
 }
 
 // Short columns: one warp per (column, 256 outputs), entries in order.
 __global__ void __launch_bounds__(COMP_THREADS)
-comp_wgrad_short_kernel(float* __restrict__ s, const int* __restrict__ colptr, const int* __restrict__ row,
+comp_wgrad_short_kernel(float* __restrict__ comp, const int* __restrict__ colptr, const int* __restrict__ row,
                         const float* __restrict__ val, const uint4* __restrict__ dy, const int* __restrict__ list,
-                        const int* __restrict__ count, int N) {
+                        const int* __restrict__ counts, int N) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n0 = blockIdx.x * COMP_COLS + 8 * lane;
   if (n0 >= N) return;
-  const int n_cols = *count;
+  const int n_long = counts[0], n_cols = counts[1];
   for (int slot = blockIdx.y * 8 + warp; slot < n_cols; slot += gridDim.y * 8) {
     const int k = list[slot];
     float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     strided_entries_times_dense(acc, row, val, colptr[k], colptr[k + 1], 1, dy, N >> 3, n0 >> 3);
-    add8_to(s + (long long)k * N + n0, acc);
-  }
-}
-
-// Weight-gradient step 2: dW = store( S (.) Q'(W (.) gamma) ), element-wise (Eq. 6 with the DGE
-// derivative of Eq. 8 evaluated on the scaled weights the forward quantised).
-__global__ void __launch_bounds__(256)
-dge_store_kernel(const float* __restrict__ s, const uint4* __restrict__ w, const float* __restrict__ w_amax,
-                 long long n_vec, int vec_per_row, int dge_on, float dge_k, float dge_clip, void* dw, int out_f32) {
-  const long long stride = (long long)gridDim.x * blockDim.x;
-  const float inv_k = 1.0f / dge_k;
-  const float expo = inv_k - 1.0f;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += stride) {
-    const long long off = i * 8;
-    const float4 a = __ldg(reinterpret_cast<const float4*>(s + off));
-    const float4 b = __ldg(reinterpret_cast<const float4*>(s + off + 4));
-    float y8[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-    if (dge_on) {
-      const int n0 = int(i % vec_per_row) * 8;
-      const uint4 wv = __ldg(&w[i]);
-      const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
-      const float4 m0 = __ldg(reinterpret_cast<const float4*>(w_amax + n0));
-      const float4 m1 = __ldg(reinterpret_cast<const float4*>(w_amax + n0 + 4));
-      const float amax[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
-#pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        const float wf = __uint_as_float((c & 1) ? (ww[c >> 1] & 0xFFFF0000u) : (ww[c >> 1] << 16));
-        const float gamma = amax[c] > 0.0f ? __fdiv_rn(6.0f, amax[c]) : 0.0f;
-        const float ws = __fmul_rn(wf, gamma);        // the value the forward quantised
-        y8[c] *= dge_factor(ws, expo, inv_k, dge_clip);
-      }
-    }
-    store8(dw, out_f32, off, y8);
+    store8_f32(comp + (long long)(n_long + slot) * N + n0, acc);
   }
 }
 
@@ -283,33 +237,24 @@ int launch_comp_fwd(fp4_ctx* ctx, cudaStream_t stream, const float* y1, const in
   return FP4_OK;
 }
 
-int launch_comp_wgrad_dge(fp4_ctx* ctx, cudaStream_t stream, float* s, const int32_t* colptr, const int32_t* row,
-                          const float* val, const void* dy_bf16, const void* w_bf16, const float* w_amax,
-                          int* col_list, int64_t, int64_t K, int64_t N, int dge_on, float dge_k, float dge_clip,
-                          void* dw, int out_f32) {
-  KernelScope scope(ctx, stream, KC_COMP_WGRAD, colptr ? 4 : 1);
-  if (colptr) {
-    // col_list: [K] long columns, [K] short columns, two counters
-    int* list_long = col_list;
-    int* list_short = col_list + K;
-    int* counts = col_list + 2 * K;
-    nonempty_columns_kernel<<<1, 1024, 0, stream>>>(colptr, int(K), list_long, list_short, counts);
-    const unsigned n_blocks = unsigned((N + COMP_COLS - 1) / COMP_COLS);
-    const uint4* dy = static_cast<const uint4*>(dy_bf16);
-    unsigned gy = unsigned(4 * ctx->num_sms) / n_blocks;          // long columns: 2 resident blocks per SM
-    gy = gy < 1 ? 1 : (gy > unsigned(K) ? unsigned(K) : gy);
-    comp_wgrad_long_kernel<<<dim3(n_blocks, gy), LONG_THREADS, 0, stream>>>(s, colptr, row, val, dy, list_long, counts,
-                                                                           int(N));
-    gy = unsigned(32 * ctx->num_sms) / n_blocks;                   // short columns: 8 per block
-    gy = gy < 1 ? 1 : (gy > unsigned((K + 7) / 8) ? unsigned((K + 7) / 8) : gy);
-    comp_wgrad_short_kernel<<<dim3(n_blocks, gy), COMP_THREADS, 0, stream>>>(s, colptr, row, val, dy, list_short,
-                                                                             counts + 1, int(N));
-  }
-  const long long n_vec = (long long)K * N / 8;
-  long long blocks = (n_vec + 255) / 256;
-  if (blocks > 16LL * ctx->num_sms) blocks = 16LL * ctx->num_sms;
-  dge_store_kernel<<<int(blocks), 256, 0, stream>>>(s, static_cast<const uint4*>(w_bf16), w_amax, n_vec, int(N / 8),
-                                                    dge_on, dge_k, dge_clip, dw, out_f32);
+int launch_comp_wgrad(fp4_ctx* ctx, cudaStream_t stream, const int32_t* colptr, const int32_t* row, const float* val,
+                      const void* dy_bf16, int* lists, int* slot_of_col, float* comp, int64_t K, int64_t N) {
+  KernelScope scope(ctx, stream, KC_COMP_WGRAD, 3);
+  // lists: [K] long columns, [K] short columns, two counters
+  int* list_long = lists;
+  int* list_short = lists + K;
+  int* counts = lists + 2 * K;
+  nonempty_columns_kernel<<<1, 1024, 0, stream>>>(colptr, int(K), list_long, list_short, counts, slot_of_col);
+  const unsigned n_blocks = unsigned((N + COMP_COLS - 1) / COMP_COLS);
+  const uint4* dy = static_cast<const uint4*>(dy_bf16);
+  unsigned gy = unsigned(4 * ctx->num_sms) / n_blocks;          // long columns: 2 resident blocks per SM
+  gy = gy < 1 ? 1 : (gy > unsigned(K) ? unsigned(K) : gy);
+  comp_wgrad_long_kernel<<<dim3(n_blocks, gy), LONG_THREADS, 0, stream>>>(comp, colptr, row, val, dy, list_long,
+                                                                         counts, int(N));
+  gy = unsigned(32 * ctx->num_sms) / n_blocks;                   // short columns: 8 per block
+  gy = gy < 1 ? 1 : (gy > unsigned((K + 7) / 8) ? unsigned((K + 7) / 8) : gy);
+  comp_wgrad_short_kernel<<<dim3(n_blocks, gy), COMP_THREADS, 0, stream>>>(comp, colptr, row, val, dy, list_short,
+                                                                           counts, int(N));
   FP4_CUDA_TRY(cudaGetLastError());
   return FP4_OK;
 }

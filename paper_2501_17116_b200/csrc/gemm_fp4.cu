@@ -42,8 +42,9 @@ constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
 __host__ __device__ constexpr int tile_n(int kind) { return kind == FP4_GEMM_F8F6F4 ? 256 : 240; }
 __host__ __device__ constexpr int b_stage_bytes(int kind) { return tile_n(kind) * 128; }
 __host__ __device__ constexpr int stage_bytes(int kind) { return A_STAGE_BYTES + b_stage_bytes(kind); }
+// operand ring, barriers, column de-scales [2][256], staging [4][4096], DGE column scales [2][256], slots [2][128]
 constexpr size_t smem_bytes(int kind) {
-  return 1024 + size_t(STAGES) * stage_bytes(kind) + 256 + 2 * 256 * 4 + STAGE_OUT_BYTES;
+  return 1024 + size_t(STAGES) * stage_bytes(kind) + 256 + 2 * 256 * 4 + STAGE_OUT_BYTES + 2 * 256 * 4 + 2 * 128 * 4;
 }
 
 struct GemmArgs {
@@ -56,7 +57,15 @@ struct GemmArgs {
   void* out;
   int out_f32;
   int32_t* status;
+  // fused weight-gradient epilogue (EPI_WGRAD)
+  const float* addend;
+  const int* slot_of_row;
+  const uint4* w;
+  const float* w_amax;
+  float inv_k, expo, clip;
 };
+
+enum { EPI_PLAIN = 0, EPI_WGRAD = 1 };
 
 // ------------------------------------------------------------------ PTX wrappers ------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -196,17 +205,51 @@ __host__ __device__ constexpr uint32_t idesc_mxf4() {
          (uint32_t(BM >> 4) << 24);
 }
 
+// Global operands of the fused weight-gradient epilogue for one 32 x 32 chunk, in the layout of
+// the store phase (iteration i, lane -> row i * RPI + lane / LPR, 8 columns from 8 * (lane % LPR)).
+// They are fetched one chunk ahead so that their latency hides under the previous chunk.
+struct EpiPrefetch {
+  uint4 w[4];            // 8 BF16 weights
+  float4 add[4][2];      // 8 compensation values (zeros for rows without a compensation row)
+};
+template <int EPI>
+__device__ __forceinline__ void epi_prefetch(EpiPrefetch& pf, const GemmArgs& args, size_t elem_off, int col0,
+                                             int width, int lane, const int* slot_rows) {
+  if (EPI != EPI_WGRAD) return;
+  const int lpr = width / 8, rpi = 32 / lpr;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    pf.w[i] = make_uint4(0, 0, 0, 0);
+    pf.add[i][0] = pf.add[i][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i < lpr) {
+      const int row = i * rpi + lane / lpr;
+      const int p = lane % lpr;
+      const size_t o = elem_off + size_t(row) * size_t(args.J) + size_t(8 * p);
+      if (args.w) pf.w[i] = __ldg(&args.w[o >> 3]);
+      const int slot = slot_rows[row];
+      if (slot >= 0) {
+        const float* src = args.addend + size_t(slot) * size_t(args.J) + size_t(col0 + 8 * p);
+        pf.add[i][0] = __ldg(reinterpret_cast<const float4*>(src));
+        pf.add[i][1] = __ldg(reinterpret_cast<const float4*>(src + 4));
+      }
+    }
+  }
+}
+
 // De-scale W accumulators of this thread's row, then store the warp's 32 x W block through a
 // shared staging tile so that every store instruction writes whole row segments: the thread-per-
 // row layout of tensor memory would otherwise touch 32 different lines per instruction.
-// The staging tile holds 32 rows of SPR 16-byte slots; slot s of row r sits at s ^ f(r), which
-// keeps both the row-wise writes and the segment-wise reads free of bank conflicts.
-template <int W, bool F32>
+// The staging tile holds 32 rows of W floats in 16-byte slots; slot s of row r sits at s ^ f(r),
+// which keeps both the row-wise writes and the segment-wise reads free of bank conflicts.  In the
+// store phase a lane owns 8 consecutive columns of one row; the fused weight-gradient epilogue
+// adds the compensation row and applies the DGE factor there, with coalesced reads of W.
+template <int W, int EPI>
 __device__ __forceinline__ void scale_stage_store(uint32_t (&v)[32], float d_row, const float* dcol, uint8_t* stage,
-                                                  void* out, size_t elem_off, int J, int lane, uint32_t next_taddr,
-                                                  int next_width) {
-  constexpr int SPR = F32 ? W / 4 : W / 8;          // 16-byte slots per row: 8, 4 or 2
-  constexpr int SH = SPR == 8 ? 0 : (SPR == 4 ? 1 : 2);
+                                                  const GemmArgs& args, size_t elem_off, int lane,
+                                                  uint32_t next_taddr, int next_width, const EpiPrefetch& pf,
+                                                  const float* gcol) {
+  constexpr int SPR = W / 4;                        // 16-byte slots per staged row: 8 or 4
+  constexpr int SH = SPR == 8 ? 0 : 1;
   float y[W];
 #pragma unroll
   for (int q = 0; q < W / 4; ++q) {
@@ -222,36 +265,54 @@ __device__ __forceinline__ void scale_stage_store(uint32_t (&v)[32], float d_row
   uint8_t* my_row = stage + lane * (SPR * 16);
   const int fx = (lane >> SH) & (SPR - 1);
 #pragma unroll
-  for (int j = 0; j < SPR; ++j) {
-    uint4 pk;
-    if (F32) {
-      pk = make_uint4(__float_as_uint(y[4 * j]), __float_as_uint(y[4 * j + 1]), __float_as_uint(y[4 * j + 2]),
-                      __float_as_uint(y[4 * j + 3]));
+  for (int j = 0; j < SPR; ++j)
+    *reinterpret_cast<float4*>(my_row + ((j ^ fx) * 16)) = make_float4(y[4 * j], y[4 * j + 1], y[4 * j + 2], y[4 * j + 3]);
+  __syncwarp();
+  constexpr int LPR = W / 8;                        // lanes per row in the store phase: 4 or 2
+  constexpr int RPI = 32 / LPR;                     // rows per store instruction: 8 or 16
+#pragma unroll
+  for (int i = 0; i < LPR; ++i) {
+    const int row = i * RPI + lane / LPR;
+    const int p = lane % LPR;
+    const int fr = (row >> SH) & (SPR - 1);
+    const uint8_t* srow = stage + row * (SPR * 16);
+    const float4 a = *reinterpret_cast<const float4*>(srow + (((2 * p) ^ fr) * 16));
+    const float4 b = *reinterpret_cast<const float4*>(srow + (((2 * p + 1) ^ fr) * 16));
+    float f[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    const size_t o = elem_off + size_t(row) * size_t(args.J) + size_t(8 * p);
+    if (EPI == EPI_WGRAD) {
+      f[0] += pf.add[i][0].x; f[1] += pf.add[i][0].y; f[2] += pf.add[i][0].z; f[3] += pf.add[i][0].w;
+      f[4] += pf.add[i][1].x; f[5] += pf.add[i][1].y; f[6] += pf.add[i][1].z; f[7] += pf.add[i][1].w;
+      if (args.w) {
+        const uint32_t ww[4] = {pf.w[i].x, pf.w[i].y, pf.w[i].z, pf.w[i].w};
+        const float4 g0 = *reinterpret_cast<const float4*>(gcol + 8 * p);
+        const float4 g1 = *reinterpret_cast<const float4*>(gcol + 8 * p + 4);
+        const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const float wf = __uint_as_float((c & 1) ? (ww[c >> 1] & 0xFFFF0000u) : (ww[c >> 1] << 16));
+          f[c] *= dge_factor(__fmul_rn(wf, g[c]), args.expo, args.inv_k, args.clip);
+        }
+      }
+    }
+    if (args.out_f32) {
+      float4* dst = reinterpret_cast<float4*>(static_cast<float*>(args.out) + o);
+      dst[0] = make_float4(f[0], f[1], f[2], f[3]);
+      dst[1] = make_float4(f[4], f[5], f[6], f[7]);
     } else {
-      uint32_t w[4];
+      uint32_t w4[4];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        __nv_bfloat162 h = __floats2bfloat162_rn(y[8 * j + 2 * q], y[8 * j + 2 * q + 1]);
-        w[q] = *reinterpret_cast<uint32_t*>(&h);
+        __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * q], f[2 * q + 1]);
+        w4[q] = *reinterpret_cast<uint32_t*>(&h);
       }
-      pk = make_uint4(w[0], w[1], w[2], w[3]);
+      *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(args.out) + o) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
     }
-    *reinterpret_cast<uint4*>(my_row + ((j ^ fx) * 16)) = pk;
-  }
-  __syncwarp();
-  constexpr int ELT = F32 ? 4 : 2;
-  uint8_t* gbase = static_cast<uint8_t*>(out) + elem_off * ELT;
-#pragma unroll
-  for (int i = 0; i < SPR; ++i) {
-    const int row = i * (32 / SPR) + lane / SPR;
-    const int sl = lane % SPR;
-    const uint4 pk = *reinterpret_cast<const uint4*>(stage + row * (SPR * 16) + ((sl ^ ((row >> SH) & (SPR - 1))) * 16));
-    *reinterpret_cast<uint4*>(gbase + size_t(row) * size_t(J) * ELT + sl * 16) = pk;
   }
   __syncwarp();
 }
 
-template <int KIND>
+template <int KIND, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const GemmArgs args) {
@@ -272,6 +333,8 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* s_dcol = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES + 256);   // [2][256] column de-scales
   uint8_t* s_out = smem + STAGES * STAGE_BYTES + 256 + 2 * 256 * 4;              // [4 warps][4096] staging
+  float* s_gcol = reinterpret_cast<float*>(s_out + STAGE_OUT_BYTES);             // [2][256] 6 / w_amax (DGE)
+  int* s_slot = reinterpret_cast<int*>(s_gcol + 2 * 256);                        // [2][128] compensation rows
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -411,13 +474,26 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const int row = m_blk * BM + quarter * 32 + lane;
       const float d_row = args.row_amax ? __fdiv_rn(__ldg(&args.row_amax[row]), 6.0f) : 1.0f;
       float* dcol = s_dcol + tile_parity * 256;
+      float* gcol = s_gcol + tile_parity * 256;
+      int* slot_rows = s_slot + tile_parity * 128;
       for (int c = et; c < BN; c += 128) {
         const int col = n_blk * BN + c;
         dcol[c] = (args.col_amax && col < args.J) ? __fdiv_rn(__ldg(&args.col_amax[col]), 6.0f) : 1.0f;
+        if (EPI == EPI_WGRAD && args.w) {
+          const float am = col < args.J ? __ldg(&args.w_amax[col]) : 0.0f;
+          gcol[c] = am > 0.0f ? __fdiv_rn(6.0f, am) : 0.0f;
+        }
       }
+      if (EPI == EPI_WGRAD) slot_rows[et] = args.slot_of_row ? __ldg(&args.slot_of_row[m_blk * BM + et]) : -1;
       const bool ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, args.status);
       if (epilogue_bar_any(!ok)) break;            // also publishes dcol to the other warps
       tc_fence_after();
+      EpiPrefetch pf;
+      {
+        const int nv = min(BN, args.J - n_blk * BN);
+        epi_prefetch<EPI>(pf, args, size_t(m_blk * BM + quarter * 32) * size_t(args.J) + size_t(n_blk) * BN, n_blk * BN,
+                          min(32, nv), lane, slot_rows + quarter * 32);
+      }
       const uint32_t t_base = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * ACC_STRIDE);
       // first element of this warp's 32 rows in this tile
       const size_t warp_off = size_t(m_blk * BM + quarter * 32) * size_t(args.J) + size_t(n_blk) * BN;
@@ -430,20 +506,17 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const int width = min(32, n_valid - c0);
         const int next_width = n_valid - (c0 + 32);                // <= 0: this is the last chunk
         const uint32_t next_taddr = t_base + uint32_t(c0 + 32);
+        const EpiPrefetch cur = pf;
+        if (next_width > 0)
+          epi_prefetch<EPI>(pf, args, warp_off + c0 + 32, n_blk * BN + c0 + 32, min(32, next_width), lane,
+                            slot_rows + quarter * 32);
         tmem_ld_wait();
-        if (width == 32) {
-          if (args.out_f32)
-            scale_stage_store<32, true>(v, d_row, dcol + c0, stage, args.out, warp_off + c0, args.J, lane, next_taddr,
-                                        next_width);
-          else
-            scale_stage_store<32, false>(v, d_row, dcol + c0, stage, args.out, warp_off + c0, args.J, lane, next_taddr,
-                                         next_width);
-        } else {
-          if (args.out_f32)
-            scale_stage_store<16, true>(v, d_row, dcol + c0, stage, args.out, warp_off + c0, args.J, lane, next_taddr, 0);
-          else
-            scale_stage_store<16, false>(v, d_row, dcol + c0, stage, args.out, warp_off + c0, args.J, lane, next_taddr, 0);
-        }
+        if (width == 32)
+          scale_stage_store<32, EPI>(v, d_row, dcol + c0, stage, args, warp_off + c0, lane, next_taddr, next_width, cur,
+                                     gcol + c0);
+        else
+          scale_stage_store<16, EPI>(v, d_row, dcol + c0, stage, args, warp_off + c0, lane, next_taddr, 0, cur,
+                                     gcol + c0);
       }
       tc_fence_before();
       __syncwarp();
@@ -489,11 +562,21 @@ int make_codes_map(fp4_ctx* ctx, CUtensorMap* map, const uint8_t* codes, int64_t
   return r == CUDA_SUCCESS ? FP4_OK : FP4_ERR_CUDA;
 }
 
+template <int KIND, int EPI>
+int launch_kernel(int grid, cudaStream_t stream, const CUtensorMap& map_a, const CUtensorMap& map_b,
+                  const GemmArgs& args) {
+  constexpr size_t kSmem = smem_bytes(KIND);
+  FP4_CUDA_TRY(cudaFuncSetAttribute(gemm_fp4_kernel<KIND, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    int(kSmem)));
+  gemm_fp4_kernel<KIND, EPI><<<grid, NUM_THREADS, kSmem, stream>>>(map_a, map_b, args);
+  return FP4_OK;
+}
+
 }  // namespace
 
 int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, const uint8_t* b_codes, int64_t I,
                     int64_t J, int64_t C, const float* row_amax, const float* col_amax, void* out, int out_f32,
-                    int gemm_kind, int32_t* status) {
+                    int gemm_kind, int32_t* status, const GemmEpilogue* epi) {
   if (gemm_kind != FP4_GEMM_MXF4 && gemm_kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;
   // The byte-container form expands 32 bytes of a packed row into 64, so its rows must start on
   // 32-byte boundaries (C/2 a multiple of 32 holds for every multiple of 128).
@@ -525,18 +608,23 @@ int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, c
   const int tiles = args.num_m_blocks * args.num_n_blocks;
   const int grid = tiles < ctx->num_sms ? tiles : ctx->num_sms;
 
+  const bool fused = epi && (epi->addend || epi->w_bf16);
+  args.addend = fused ? epi->addend : nullptr;
+  args.slot_of_row = fused && epi->addend ? epi->slot_of_row : nullptr;
+  args.w = fused ? static_cast<const uint4*>(epi->w_bf16) : nullptr;
+  args.w_amax = fused ? epi->w_amax : nullptr;
+  args.inv_k = fused && epi->w_bf16 ? 1.0f / epi->dge_k : 1.0f;
+  args.expo = args.inv_k - 1.0f;
+  args.clip = fused ? epi->dge_clip : 0.0f;
   KernelScope scope(ctx, stream, KC_GEMM, 1);
-  if (gemm_kind == FP4_GEMM_F8F6F4) {
-    constexpr size_t kSmem = smem_bytes(FP4_GEMM_F8F6F4);
-    FP4_CUDA_TRY(cudaFuncSetAttribute(gemm_fp4_kernel<FP4_GEMM_F8F6F4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      int(kSmem)));
-    gemm_fp4_kernel<FP4_GEMM_F8F6F4><<<grid, NUM_THREADS, kSmem, stream>>>(map_a, map_b, args);
-  } else {
-    constexpr size_t kSmem = smem_bytes(FP4_GEMM_MXF4);
-    FP4_CUDA_TRY(cudaFuncSetAttribute(gemm_fp4_kernel<FP4_GEMM_MXF4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      int(kSmem)));
-    gemm_fp4_kernel<FP4_GEMM_MXF4><<<grid, NUM_THREADS, kSmem, stream>>>(map_a, map_b, args);
-  }
+  int rc2;
+  if (gemm_kind == FP4_GEMM_F8F6F4)
+    rc2 = fused ? launch_kernel<FP4_GEMM_F8F6F4, EPI_WGRAD>(grid, stream, map_a, map_b, args)
+                : launch_kernel<FP4_GEMM_F8F6F4, EPI_PLAIN>(grid, stream, map_a, map_b, args);
+  else
+    rc2 = fused ? launch_kernel<FP4_GEMM_MXF4, EPI_WGRAD>(grid, stream, map_a, map_b, args)
+                : launch_kernel<FP4_GEMM_MXF4, EPI_PLAIN>(grid, stream, map_a, map_b, args);
+  if (rc2 != FP4_OK) return rc2;
   FP4_CUDA_TRY(cudaGetLastError());
   return FP4_OK;
 }
