@@ -169,6 +169,8 @@ def main():
     ap.add_argument("--config", type=int, default=1)
     ap.add_argument("--gemm-kind", type=int, default=0, help="0 mxf4 (K=64), 1 f8f6f4 (K=32)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-share-activations", action="store_true",
+                    help="quantise the activation of every linear, also where q/k/v or gate/up read the same tensor")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -197,13 +199,19 @@ def main():
     layers = []
     ws_bytes = 0
     lib = fp4.load_library()
+    share = not args.no_share_activations
+    owner = {}                                   # id of the host activation array -> first layer that reads it
     for name, K, N, a_bits, w_bits, dy_bits in layer_inputs(cfg, WL, seed=rank):
         hA, hW, hG = pinned(a_bits), pinned(w_bits), pinned(dy_bits)
-        L = dict(name=name, K=K, N=N, hA=hA, hW=hW, hG=hG, A=hA.to(dev), W=hW.to(dev), G=hG.to(dev),
+        first = owner.setdefault(id(a_bits), len(layers)) if share else len(layers)
+        shared = first != len(layers)
+        L = dict(name=name, K=K, N=N, hA=hA, hW=hW, hG=hG, W=hW.to(dev), G=hG.to(dev),
+                 A=layers[first]["A"] if shared else hA.to(dev), reuse_a=shared,
                  Y=torch.empty((M, N), dtype=torch.bfloat16, device=dev),
                  dA=torch.empty((M, K), dtype=torch.bfloat16, device=dev),
                  dW=torch.empty((K, N), dtype=torch.bfloat16, device=dev),
-                 sa=fp4.QTensor(M, K, 0, dev, fp4.tail_capacity(M, K, alpha)), sw=fp4.QTensor(K, N, 1, dev),
+                 sa=layers[first]["sa"] if shared else fp4.QTensor(M, K, 0, dev, fp4.tail_capacity(M, K, alpha)),
+                 sw=fp4.QTensor(K, N, 1, dev),
                  hY=torch.empty((M, N), dtype=torch.bfloat16).pin_memory(),
                  hdA=torch.empty((M, K), dtype=torch.bfloat16).pin_memory(),
                  hdW=torch.empty((K, N), dtype=torch.bfloat16).pin_memory())
@@ -215,7 +223,8 @@ def main():
 
     def step():
         for L in layers:
-            fp4.fp4_linear_fwd(ctx, L["A"], L["W"], alpha, L["sa"], L["sw"], gemm_kind=kind, out=L["Y"])
+            fp4.fp4_linear_fwd(ctx, L["A"], L["W"], alpha, L["sa"], L["sw"], gemm_kind=kind, out=L["Y"],
+                               reuse_a=L["reuse_a"])
             fp4.fp4_linear_bwd(ctx, L["G"], L["W"], L["sa"], L["sw"], gemm_kind=kind, dA=L["dA"], dW=L["dW"])
 
     def step_host():
@@ -297,17 +306,18 @@ def main():
     fp4_peak = FP4_OVER_BF16 * peaks["bf16_tflops"]
     alu_peak = SM_COUNT * FMA_LANES * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
     steps = args.steps
-    elems_a = sum(M * L["K"] for L in layers)
+    elems_a = sum(M * L["K"] for L in layers if not L["reuse_a"])      # activations actually quantised
     elems_w = sum(L["K"] * L["N"] for L in layers)
     elems_g = sum(M * L["N"] for L in layers)
     nnz_total = sum(nnz)
+    nnz_quantised = sum(z for z, L in zip(nnz, layers) if not L["reuse_a"])
     work = {
         # class: (bound, algorithmic work per step, unit of the rate)
         "gemm": ("tensor", flop_step, "TFLOP/s"),
         "select": ("hbm", 2.0 * elems_a, "GB/s"),                                   # one read of A
         "encode": ("hbm", 3.125 * elems_a + 3.0 * elems_w + 2 * 2.5 * elems_g, "GB/s"),
         "absmax": ("hbm", 2.0 * elems_w + 2 * 2.0 * elems_g, "GB/s"),                # one read each
-        "sparse": ("hbm", 2 * 8.0 * nnz_total + 3 * elems_a / 8.0, "GB/s"),           # entries + 3 mask sweeps
+        "sparse": ("hbm", 2 * 8.0 * nnz_quantised + 3 * elems_a / 8.0, "GB/s"),       # entries + 3 mask sweeps
         "comp_fwd": ("alu", sum(2.0 * z * L["N"] for z, L in zip(nnz, layers)), "TFLOP/s"),
         "comp_wgrad_dge": ("alu", sum(2.0 * z * L["N"] + 8.0 * L["K"] * L["N"] for z, L in zip(nnz, layers)),
                            "TFLOP/s"),
@@ -348,6 +358,8 @@ def main():
                        "alpha": alpha, "dge": True, "gemm_kind": "mxf4" if kind == 0 else "f8f6f4",
                        "l2": f"inputs exceed L2: {resident_bytes / 1e6:.0f} MB touched per step",
                        "launch": "one CUDA graph per step, replayed",
+                       "shared_activations": ("q/k/v and gate/up read one activation tensor: quantised once, re-used"
+                                              if share else "every linear quantises its activation"),
                        "kernel_timing": f"CUDA events per kernel class over {args.steps} plainly launched steps "
                                         f"({ms_profiled / args.steps:.3f} ms/step with the events)",
                        "replicas": world},

@@ -139,11 +139,16 @@ int fp4_gemm(fp4_ctx* ctx, void* stream, const uint8_t* a_codes, const uint8_t* 
  *   A_bf16 [M x K], W_bf16 [K x N], Y [M x N] (BF16, or float if out_f32 != 0).
  *   savedA, savedW: caller-allocated fp4_qtensor buffers that receive the quantised operands
  *   and are handed to fp4_linear_bwd.  savedA needs codes, codes_t, amax, thresholds, nnz,
- *   csr_*, csc_*; savedW needs codes, codes_t, amax.  If reuse_w != 0, savedW already holds
- *   this weight's codes (weights change once per optimizer step) and is not recomputed.
+ *   csr_*, csc_*; savedW needs codes, codes_t, amax.
+ *   `reuse` is a bit mask: FP4_REUSE_W -- savedW already holds this weight's codes (weights
+ *   change once per optimizer step) and is not recomputed; FP4_REUSE_A -- savedA already holds
+ *   this activation quantised with the same alpha (the q/k/v projections of a layer, or its
+ *   gate/up projections, read the same activation) and is not recomputed.
  */
+#define FP4_REUSE_W 1
+#define FP4_REUSE_A 2
 int fp4_linear_fwd(fp4_ctx* ctx, void* stream, const void* A_bf16, const void* W_bf16,
-                   int64_t M, int64_t K, int64_t N, double alpha, int reuse_w, int gemm_kind,
+                   int64_t M, int64_t K, int64_t N, double alpha, int reuse, int gemm_kind,
                    void* Y, int out_f32, fp4_qtensor* savedA, fp4_qtensor* savedW,
                    int32_t* status);
 

@@ -223,6 +223,7 @@ def fp4_gemm(ctx: Context, a_codes: torch.Tensor, b_codes: torch.Tensor, row_ama
 
 def fp4_linear_fwd(ctx: Context, A: torch.Tensor, W: torch.Tensor, alpha: float, saved_a: QTensor | None = None,
                    saved_w: QTensor | None = None, reuse_w: bool = False, gemm_kind: int = FP4_GEMM_MXF4,
+                   reuse_a: bool = False,
                    out_f32: bool = False, out: torch.Tensor | None = None):
     M, K = A.shape
     K2, N = W.shape
@@ -233,7 +234,7 @@ def fp4_linear_fwd(ctx: Context, A: torch.Tensor, W: torch.Tensor, alpha: float,
         saved_w = QTensor(K, N, 1, A.device)
     if out is None:
         out = torch.empty((M, N), dtype=torch.float32 if out_f32 else torch.bfloat16, device=A.device)
-    _check(ctx.lib.fp4_linear_fwd(ctx.handle, _stream(), _ptr(A), _ptr(W), M, K, N, float(alpha), int(reuse_w),
+    _check(ctx.lib.fp4_linear_fwd(ctx.handle, _stream(), _ptr(A), _ptr(W), M, K, N, float(alpha), int(reuse_w) | (2 if reuse_a else 0),
                                   gemm_kind, _ptr(out), int(out_f32), C.byref(saved_a.struct),
                                   C.byref(saved_w.struct), _ptr(ctx.status)))
     return out, saved_a, saved_w

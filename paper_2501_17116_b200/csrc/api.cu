@@ -34,7 +34,7 @@ int check_qtensor_dense(const fp4_qtensor* q) {
 }
 
 int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf16, const void* W_bf16, int64_t M,
-                    int64_t K, int64_t N, double alpha, int reuse_w, int gemm_kind, void* Y, int out_f32,
+                    int64_t K, int64_t N, double alpha, int reuse, int gemm_kind, void* Y, int out_f32,
                     fp4_qtensor* savedA, fp4_qtensor* savedW, int32_t* status);
 int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_bf16, const void* W_bf16,
                     const fp4_qtensor* savedA, const fp4_qtensor* savedW, int64_t M, int64_t K, int64_t N, int dge_on,
@@ -180,7 +180,7 @@ int fp4_gemm(fp4_ctx* ctx, void* stream, const uint8_t* a_codes, const uint8_t* 
 }
 
 int fp4_linear_fwd(fp4_ctx* ctx, void* stream, const void* A_bf16, const void* W_bf16, int64_t M, int64_t K,
-                   int64_t N, double alpha, int reuse_w, int gemm_kind, void* Y, int out_f32, fp4_qtensor* savedA,
+                   int64_t N, double alpha, int reuse, int gemm_kind, void* Y, int out_f32, fp4_qtensor* savedA,
                    fp4_qtensor* savedW, int32_t* status) {
   if (!ctx || !A_bf16 || !W_bf16 || !Y || !savedA || !savedW || !status) return FP4_ERR_NULL;
   if (!mult128(M) || !mult128(K) || !mult128(N)) return FP4_ERR_SHAPE;
@@ -199,7 +199,7 @@ int fp4_linear_fwd(fp4_ctx* ctx, void* stream, const void* A_bf16, const void* W
   }
   if (fp4_workspace_bytes(M, K, N) > ctx->workspace_bytes) return FP4_ERR_WORKSPACE;
   return linear_fwd_impl(ctx, static_cast<cudaStream_t>(stream), Arena(ctx->workspace, ctx->workspace_bytes), A_bf16,
-                         W_bf16, M, K, N, alpha, reuse_w, gemm_kind, Y, out_f32, savedA, savedW, status);
+                         W_bf16, M, K, N, alpha, reuse, gemm_kind, Y, out_f32, savedA, savedW, status);
 }
 
 }  // extern "C"
@@ -207,11 +207,12 @@ int fp4_linear_fwd(fp4_ctx* ctx, void* stream, const void* A_bf16, const void* W
 namespace {
 
 int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf16, const void* W_bf16, int64_t M,
-                    int64_t K, int64_t N, double alpha, int reuse_w, int gemm_kind, void* Y, int out_f32,
+                    int64_t K, int64_t N, double alpha, int reuse, int gemm_kind, void* Y, int out_f32,
                     fp4_qtensor* savedA, fp4_qtensor* savedW, int32_t* status) {
   const bool occ = alpha < 1.0;
+  const bool reuse_w = (reuse & FP4_REUSE_W) != 0, reuse_a = (reuse & FP4_REUSE_A) != 0;
   float* y1 = occ ? arena.take<float>(size_t(M) * size_t(N)) : nullptr;
-  char* scratch_a = arena.take<char>(quantize_scratch_bytes(M, K));
+  char* scratch_a = reuse_a ? nullptr : arena.take<char>(quantize_scratch_bytes(M, K));
   char* scratch_w = reuse_w ? nullptr : arena.take<char>(quantize_scratch_bytes(K, N));
   if (!arena.ok) return FP4_ERR_WORKSPACE;
   int rc;
@@ -228,7 +229,7 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
     if (rc != FP4_OK) return rc;
     FP4_CUDA_TRY(cudaEventRecord(ctx->ev[1], ctx->side[0]));
   }
-  {
+  if (!reuse_a) {
     Arena a(scratch_a, quantize_scratch_bytes(M, K));
     savedA->rows = M;
     savedA->cols = K;
@@ -248,10 +249,10 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
                        status);
   if (rc != FP4_OK) return rc;
   // Y = store(Y1 + (A - A_c) W): one rounding of the fp32 sum.  Needs the CSR.
-  FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[3], 0));
+  if (!reuse_a) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[3], 0));
   rc = launch_comp_fwd(ctx, st, y1, savedA->csr_rowptr, savedA->csr_col, savedA->csr_val, W_bf16, M, K, N, Y, out_f32);
   if (rc != FP4_OK) return rc;
-  FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[4], 0));                      // savedA is complete on return
+  if (!reuse_a) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[4], 0));        // savedA is complete on return
   return FP4_OK;
 }
 

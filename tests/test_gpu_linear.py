@@ -112,6 +112,20 @@ def test_reuse_quantised_weight(lib, ctx):
     assert torch.equal(y2, y2_fresh)
 
 
+def test_reuse_quantised_activation(lib, ctx):
+    """q/k/v-style sharing: a second weight applied to an activation that is already quantised."""
+    a_bits, w_bits, dy_bits = WL.small_case(256, 384, 256, seed=9)
+    _, w2_bits, _ = WL.small_case(256, 384, 256, seed=10)
+    A, W1, W2, dY = _dev(a_bits), _dev(w_bits), _dev(w2_bits), _dev(dy_bits)
+    _, sa, _ = lib.fp4_linear_fwd(ctx, A, W1, 0.99)
+    y_shared, _, sw2 = lib.fp4_linear_fwd(ctx, A, W2, 0.99, saved_a=sa, reuse_a=True)
+    da_s, dw_s = lib.fp4_linear_bwd(ctx, dY, W2, sa, sw2)
+    y_fresh, sa2, sw2b = lib.fp4_linear_fwd(ctx, A, W2, 0.99)
+    da_f, dw_f = lib.fp4_linear_bwd(ctx, dY, W2, sa2, sw2b)
+    torch.cuda.synchronize()
+    assert torch.equal(y_shared, y_fresh) and torch.equal(da_s, da_f) and torch.equal(dw_s, dw_f)
+
+
 def test_config0_full_layer(lib, ctx):
     """The small configuration in full: X[256 x 1024] with 8 outlier channels, alpha = 0.99, DGE on."""
     cfg = WL.CONFIGS[0]
