@@ -266,6 +266,7 @@ def main():
     # pair around every kernel class on its launching stream (events cannot sit inside a graph).
     ctx.profile_reset()
     ctx.profile_enable(True)
+    ctx.set_overlap(False)              # one kernel at a time: durations are not inflated by SM sharing
     torch.cuda.synchronize()
     p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     p0.record()
@@ -276,6 +277,7 @@ def main():
     ms_profiled = p0.elapsed_time(p1)
     prof = ctx.profile_read()
     ctx.profile_enable(False)
+    ctx.set_overlap(True)
     ctx.profile_reset()
     nnz = [int(L["sa"].nnz.item()) if L["sa"].nnz is not None else 0 for L in layers]
 
@@ -360,8 +362,8 @@ def main():
                        "launch": "one CUDA graph per step, replayed",
                        "shared_activations": ("q/k/v and gate/up read one activation tensor: quantised once, re-used"
                                               if share else "every linear quantises its activation"),
-                       "kernel_timing": f"CUDA events per kernel class over {args.steps} plainly launched steps "
-                                        f"({ms_profiled / args.steps:.3f} ms/step with the events)",
+                       "kernel_timing": f"CUDA events per kernel class over {args.steps} plainly launched steps, side "
+                                        f"streams off ({ms_profiled / args.steps:.3f} ms/step that way)",
                        "replicas": world},
             "e2e": {"value": value_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": 1e3 * sec_e2e / args.steps},

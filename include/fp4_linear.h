@@ -201,6 +201,11 @@ int fp4_linear_step_host(fp4_ctx* ctx, void* stream, const void* A_host, const v
 #define FP4_KC_COMP_WGRAD  6   /* residual^T x dY + DGE factor + final store of dW            */
 #define FP4_KC_COUNT       7
 int fp4_profile_enable(fp4_ctx* ctx, int on);
+/* Inside one call, independent kernel chains (weight quantisation, sparse extraction, the
+ * weight-gradient branch) run on side streams owned by the context and rejoin `stream` before
+ * the call's work ends.  fp4_set_overlap(ctx, 0) puts every kernel on `stream` in program order
+ * (used to time kernels one at a time); the results are identical either way.  Default: on.  */
+int fp4_set_overlap(fp4_ctx* ctx, int on);
 int fp4_profile_reset(fp4_ctx* ctx);
 int fp4_profile_read(fp4_ctx* ctx, int kernel_class, double* total_ms, int64_t* launches);
 int64_t fp4_launch_count(fp4_ctx* ctx);

@@ -88,6 +88,7 @@ int fp4_create(fp4_ctx** out, int device, size_t workspace_bytes) {
   ctx->workspace_bytes = 0;
   ctx->encode_tiled = nullptr;
   ctx->profile = 0;
+  ctx->overlap = 1;
   ctx->launch_count = 0;
   ctx->records = new (std::nothrow) std::vector<ProfRecord>();
   for (auto& s : ctx->side) s = nullptr;
@@ -219,15 +220,19 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
 
   // Three independent chains: W (side stream 0), A up to its codes (caller's stream), and the
   // mask -> CSR / CSC stage of A (side stream 1), which only the compensation and the backward need.
+  const bool ov = ctx->overlap != 0;
   if (!reuse_w) {
-    FP4_CUDA_TRY(cudaEventRecord(ctx->ev[0], st));
-    FP4_CUDA_TRY(cudaStreamWaitEvent(ctx->side[0], ctx->ev[0], 0));
+    cudaStream_t s0 = ov ? ctx->side[0] : st;
+    if (ov) {
+      FP4_CUDA_TRY(cudaEventRecord(ctx->ev[0], st));
+      FP4_CUDA_TRY(cudaStreamWaitEvent(s0, ctx->ev[0], 0));
+    }
     Arena a(scratch_w, quantize_scratch_bytes(K, N));
     savedW->rows = K;
     savedW->cols = N;
-    rc = launch_quantize(ctx, ctx->side[0], a, W_bf16, K, N, /*scale_axis=*/1, 1.0, nullptr, 0, savedW, status);
+    rc = launch_quantize(ctx, s0, a, W_bf16, K, N, /*scale_axis=*/1, 1.0, nullptr, 0, savedW, status);
     if (rc != FP4_OK) return rc;
-    FP4_CUDA_TRY(cudaEventRecord(ctx->ev[1], ctx->side[0]));
+    if (ov) FP4_CUDA_TRY(cudaEventRecord(ctx->ev[1], s0));
   }
   if (!reuse_a) {
     Arena a(scratch_a, quantize_scratch_bytes(M, K));
@@ -235,11 +240,11 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
     savedA->cols = K;
     const SparseOverlap so = {ctx->side[1], ctx->ev[2], ctx->ev[3]};
     rc = launch_quantize(ctx, st, a, A_bf16, M, K, /*scale_axis=*/0, alpha, nullptr, 0, savedA, status,
-                         occ ? &so : nullptr);
+                         occ && ov ? &so : nullptr);
     if (rc != FP4_OK) return rc;
-    if (occ) FP4_CUDA_TRY(cudaEventRecord(ctx->ev[4], ctx->side[1]));       // CSR and CSC complete
+    if (occ && ov) FP4_CUDA_TRY(cudaEventRecord(ctx->ev[4], ctx->side[1]));  // CSR and CSC complete
   }
-  if (!reuse_w) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[1], 0));
+  if (!reuse_w && ov) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[1], 0));
   // Y1 = (Q(A_c) Q(W)) * d_A[m] * d_W[n]: A codes [M x K/2], W codes transposed [N x K/2].
   if (!occ) {
     return launch_gemm_fp4(ctx, st, savedA->codes, savedW->codes_t, M, N, K, savedA->amax, savedW->amax, Y, out_f32,
@@ -249,10 +254,10 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
                        status);
   if (rc != FP4_OK) return rc;
   // Y = store(Y1 + (A - A_c) W): one rounding of the fp32 sum.  Needs the CSR.
-  if (!reuse_a) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[3], 0));
+  if (!reuse_a && ov) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[3], 0));
   rc = launch_comp_fwd(ctx, st, y1, savedA->csr_rowptr, savedA->csr_col, savedA->csr_val, W_bf16, M, K, N, Y, out_f32);
   if (rc != FP4_OK) return rc;
-  if (!reuse_a) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[4], 0));        // savedA is complete on return
+  if (!reuse_a && ov) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[4], 0));  // savedA is complete on return
   return FP4_OK;
 }
 
@@ -298,7 +303,7 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
   // The weight-gradient chain runs on a side stream when both gradients are wanted.  Its first
   // part, the compensation dA^T dY of the non-empty residual columns, needs neither GEMM operand.
   cudaStream_t sw = st;
-  if (dA && dW) {
+  if (dA && dW && ctx->overlap) {
     sw = ctx->side[0];
     FP4_CUDA_TRY(cudaEventRecord(ctx->ev[5], st));
     FP4_CUDA_TRY(cudaStreamWaitEvent(sw, ctx->ev[5], 0));
@@ -316,8 +321,10 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
     rc = launch_quantize_dual(ctx, st, a, dY_bf16, M, N, savedW->amax, savedA->amax, g1_codes, g1_amax, g2_codes,
                               g2_amax);
     if (rc != FP4_OK) return rc;
-    FP4_CUDA_TRY(cudaEventRecord(ctx->ev[6], st));
-    FP4_CUDA_TRY(cudaStreamWaitEvent(sw, ctx->ev[6], 0));
+    if (sw != st) {
+      FP4_CUDA_TRY(cudaEventRecord(ctx->ev[6], st));
+      FP4_CUDA_TRY(cudaStreamWaitEvent(sw, ctx->ev[6], 0));
+    }
   } else if (dA) {
     fp4_qtensor g = {};
     g.rows = M; g.cols = N; g.codes = g1_codes; g.amax = g1_amax;
@@ -442,6 +449,12 @@ int fp4_linear_step_host(fp4_ctx* ctx, void* stream, const void* A_host, const v
     FP4_CUDA_TRY(cudaMemcpyAsync(status_host, status, 4, cudaMemcpyDeviceToHost, st));
     FP4_CUDA_TRY(cudaStreamSynchronize(st));
   }
+  return FP4_OK;
+}
+
+int fp4_set_overlap(fp4_ctx* ctx, int on) {
+  if (!ctx) return FP4_ERR_NULL;
+  ctx->overlap = on ? 1 : 0;
   return FP4_OK;
 }
 
