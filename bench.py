@@ -39,7 +39,15 @@ SM_COUNT, FMA_LANES = 148, 128      # plain fp32 pipe: 148 SMs x 128 FMA lanes x
 
 # DRAM bytes per launch of the dominant kernel from the committed ncu summaries
 # (profiles/*.md); None where no capture exists for the class.
-NCU_TRAFFIC_PER_UNIT = {}
+NCU_TRAFFIC_PER_UNIT = {
+    # profiles/gemm_fp4_llama1p3b.md: dram read + write of three consecutive launches, averaged (bytes per launch)
+    "gemm": 11.4e6,
+    "encode": 11.2e6,      # profiles/quantizer_encode_llama1p3b.md (writes still in L2 at kernel end)
+    "select": 16.8e6,      # profiles/quantizer_select_absmax_llama1p3b.md, hist_rowminmax_kernel
+    "absmax": 12.6e6,
+    "comp_fwd": 36.1e6,    # profiles/compensation_llama1p3b.md
+    "comp_wgrad_dge": 16.8e6,
+}
 
 
 def load_peaks():
