@@ -206,6 +206,9 @@ int fp4_profile_enable(fp4_ctx* ctx, int on);
  * the call's work ends.  fp4_set_overlap(ctx, 0) puts every kernel on `stream` in program order
  * (used to time kernels one at a time); the results are identical either way.  Default: on.  */
 int fp4_set_overlap(fp4_ctx* ctx, int on);
+/* MXF4 GEMMs on pairs of CTAs (tcgen05.mma.cta_group::2, 256 x 240 tile per pair: a third less
+ * operand traffic from L2 per flop).  Same results bit for bit.  Default: off.               */
+int fp4_set_gemm_pairs(fp4_ctx* ctx, int on);
 int fp4_profile_reset(fp4_ctx* ctx);
 int fp4_profile_read(fp4_ctx* ctx, int kernel_class, double* total_ms, int64_t* launches);
 int64_t fp4_launch_count(fp4_ctx* ctx);

@@ -89,6 +89,7 @@ int fp4_create(fp4_ctx** out, int device, size_t workspace_bytes) {
   ctx->encode_tiled = nullptr;
   ctx->profile = 0;
   ctx->overlap = 1;
+  ctx->gemm_pairs = 0;
   ctx->launch_count = 0;
   ctx->records = new (std::nothrow) std::vector<ProfRecord>();
   for (auto& s : ctx->side) s = nullptr;
@@ -455,6 +456,12 @@ int fp4_linear_step_host(fp4_ctx* ctx, void* stream, const void* A_host, const v
 int fp4_set_overlap(fp4_ctx* ctx, int on) {
   if (!ctx) return FP4_ERR_NULL;
   ctx->overlap = on ? 1 : 0;
+  return FP4_OK;
+}
+
+int fp4_set_gemm_pairs(fp4_ctx* ctx, int on) {
+  if (!ctx) return FP4_ERR_NULL;
+  ctx->gemm_pairs = on ? 1 : 0;
   return FP4_OK;
 }
 

@@ -37,6 +37,7 @@ struct fp4_ctx {
   cudaStream_t side[2];        // side streams for independent kernel chains inside one call
   cudaEvent_t  ev[8];          // fork / join events of those chains
   int      overlap;            // run independent kernel chains on the side streams (default on)
+  int      gemm_pairs;         // MXF4 GEMM on pairs of CTAs (tcgen05 cta_group::2)
   int      profile;            // record CUDA events around every kernel class
   long long launch_count;      // kernels enqueued since the last reset
   std::vector<ProfRecord>* records;
