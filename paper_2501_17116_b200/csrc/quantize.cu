@@ -21,7 +21,6 @@
 namespace {
 
 constexpr int HIST_THREADS = 1024;
-constexpr int HIST_WORDS = 32768;                 // two 16-bit counters per word
 constexpr int ENC_TM = 64;                        // tile rows of the encoder (= one strip)
 constexpr int ENC_TK = 256;                       // tile columns
 constexpr int ENC_THREADS = 256;
@@ -64,67 +63,95 @@ __global__ void init_occ_kernel(uint32_t* hist, int* row_max, int* row_min, int*
   if (t == 0) *ticket = 0;
 }
 
-// Shared-memory counters are 16-bit pairs.  A counter that reaches 0x8000 is moved to the global
-// histogram by the thread that made it so.  Between two block barriers the block adds at most
-// 8192 elements, so a counter stays below 0xC000 and never carries into its neighbour.
-__device__ __forceinline__ void bump(uint32_t* h, uint32_t* ghist, uint32_t bits) {
-  const uint32_t sh = (bits & 1u) << 4;
-  const uint32_t old = atomicAdd(&h[bits >> 1], 1u << sh);
-  if (((old >> sh) & 0xFFFFu) == 0x7FFFu) {
-    atomicSub(&h[bits >> 1], 0x8000u << sh);
-    atomicAdd(&ghist[bits], 0x8000u);
-  }
-}
+// Exact histogram with 32-bit shared-memory counters over a window of HIST_EXPS binary exponents
+// (both signs, all 128 mantissas): real tensors spread over far fewer exponents than BF16 offers.
+// Each block places its window just above the largest magnitude of its first 8192 elements.
+// Patterns outside the window (tiny values, later giants) go straight to the global histogram and
+// exact zeros are counted in registers, so every element is counted exactly once.  The window is
+// replicated HIST_COPIES times (one copy per group of warps) to thin out same-address conflicts;
+// the increments return no value and need no overflow handling.
+constexpr int HIST_EXPS = 24;
+constexpr int HIST_BINS = HIST_EXPS * 128 * 2;     // 6144 counters per copy
+constexpr int HIST_COPIES = 8;
+constexpr int HIST_SMEM_BYTES = HIST_BINS * HIST_COPIES * 4;
 
 __global__ void __launch_bounds__(HIST_THREADS, 1)
 hist_rowminmax_kernel(const uint4* __restrict__ x, long long n_vec_ll, int vec_per_row, uint32_t* __restrict__ ghist,
                       int* __restrict__ row_max, int* __restrict__ row_min) {
   extern __shared__ uint32_t h[];
-  for (int i = threadIdx.x; i < HIST_WORDS; i += HIST_THREADS) h[i] = 0;
+  __shared__ uint32_t s_top;
+  for (int i = threadIdx.x; i < HIST_BINS * HIST_COPIES; i += HIST_THREADS) h[i] = 0;
+  if (threadIdx.x == 0) s_top = 0;
   __syncthreads();
   const int n_vec = int(n_vec_ll);                 // rows * cols < 2^31
   const int stride = gridDim.x * HIST_THREADS;
   int i = blockIdx.x * HIST_THREADS + threadIdx.x;
+  uint4 nxt = make_uint4(0, 0, 0, 0);
+  if (i < n_vec) nxt = __ldg(&x[i]);
+  {
+    // window top: largest exponent-and-mantissa field among this block's first vectors
+    const uint32_t w[4] = {nxt.x, nxt.y, nxt.z, nxt.w};
+    uint32_t m = 0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) m = max(m, max(w[q] & 0x7FFFu, (w[q] >> 16) & 0x7FFFu));
+    m = __reduce_max_sync(0xFFFFFFFFu, m);
+    if ((threadIdx.x & 31) == 0) atomicMax(&s_top, m);
+  }
+  __syncthreads();
+  // window = exponents [e_top - HIST_EXPS + 1, e_top] with e_top four binades above the sample's maximum
+  const int e_top = min(254, int(s_top >> 7) + 4);
+  const uint32_t base = uint32_t(max(0, e_top - HIST_EXPS + 1)) << 7;
+  uint32_t* my_h = h + ((threadIdx.x >> 5) & (HIST_COPIES - 1)) * HIST_BINS;
+  uint32_t zeros_pos = 0, zeros_neg = 0;
   // row of vector i, advanced incrementally (one division per thread)
   int row = i / vec_per_row, rem = i - row * vec_per_row;
   const int row_step = stride / vec_per_row, rem_step = stride - row_step * vec_per_row;
-  uint4 nxt = make_uint4(0, 0, 0, 0);
-  if (i < n_vec) nxt = __ldg(&x[i]);
-  for (int base = blockIdx.x * HIST_THREADS; base < n_vec; base += stride) {
+  for (; i < n_vec; i += stride) {
     const uint4 v = nxt;
-    const bool valid = i < n_vec;
     if (i + stride < n_vec) nxt = __ldg(&x[i + stride]);
-    if (valid) {
-      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        bump(h, ghist, w[q] & 0xFFFFu);
-        bump(h, ghist, w[q] >> 16);
-      }
-      const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(w);
-      const __nv_bfloat162 mx = __hmax2(__hmax2(p[0], p[1]), __hmax2(p[2], p[3]));
-      const __nv_bfloat162 mn = __hmin2(__hmin2(p[0], p[1]), __hmin2(p[2], p[3]));
-      int kmax = float_to_ordered(fmaxf(__low2float(mx), __high2float(mx)));
-      int kmin = float_to_ordered(fminf(__low2float(mn), __high2float(mn)));
-      // 16 consecutive vectors (128 elements) never straddle a row: cols is a multiple of 128
-      const unsigned group = (threadIdx.x & 16) ? 0xFFFF0000u : 0x0000FFFFu;
-      kmax = __reduce_max_sync(group, kmax);
-      kmin = __reduce_min_sync(group, kmin);
-      if ((threadIdx.x & 15) == 0) {
-        atomicMax(&row_max[row], kmax);
-        atomicMin(&row_min[row], kmin);
+    for (int q = 0; q < 8; ++q) {
+      const uint32_t bits = (q & 1) ? (w[q >> 1] >> 16) : (w[q >> 1] & 0xFFFFu);
+      const uint32_t m15 = bits & 0x7FFFu;
+      const uint32_t off = m15 - base;
+      if (off < uint32_t(HIST_EXPS * 128)) {
+        atomicAdd(&my_h[2 * off + (bits >> 15)], 1u);
+      } else if (m15 == 0) {
+        if (bits) ++zeros_neg; else ++zeros_pos;
+      } else {
+        atomicAdd(&ghist[bits], 1u);
       }
     }
-    i += stride;
+    const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(w);
+    const __nv_bfloat162 mx = __hmax2(__hmax2(p[0], p[1]), __hmax2(p[2], p[3]));
+    const __nv_bfloat162 mn = __hmin2(__hmin2(p[0], p[1]), __hmin2(p[2], p[3]));
+    int kmax = float_to_ordered(fmaxf(__low2float(mx), __high2float(mx)));
+    int kmin = float_to_ordered(fminf(__low2float(mn), __high2float(mn)));
+    // 16 consecutive vectors (128 elements) never straddle a row: cols is a multiple of 128
+    const unsigned group = (threadIdx.x & 16) ? 0xFFFF0000u : 0x0000FFFFu;
+    kmax = __reduce_max_sync(group, kmax);
+    kmin = __reduce_min_sync(group, kmin);
+    if ((threadIdx.x & 15) == 0) {
+      atomicMax(&row_max[row], kmax);
+      atomicMin(&row_min[row], kmin);
+    }
     row += row_step;
     rem += rem_step;
     if (rem >= vec_per_row) { rem -= vec_per_row; ++row; }
-    __syncthreads();
   }
-  for (int idx = threadIdx.x; idx < HIST_WORDS; idx += HIST_THREADS) {
-    const uint32_t w = h[idx];
-    if (w & 0xFFFFu) atomicAdd(&ghist[2 * idx], w & 0xFFFFu);
-    if (w >> 16) atomicAdd(&ghist[2 * idx + 1], w >> 16);
+  zeros_pos = __reduce_add_sync(0xFFFFFFFFu, zeros_pos);
+  zeros_neg = __reduce_add_sync(0xFFFFFFFFu, zeros_neg);
+  if ((threadIdx.x & 31) == 0) {
+    if (zeros_pos) atomicAdd(&ghist[0x0000], zeros_pos);
+    if (zeros_neg) atomicAdd(&ghist[0x8000], zeros_neg);
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < HIST_BINS; idx += HIST_THREADS) {
+    uint32_t c = 0;
+#pragma unroll
+    for (int r = 0; r < HIST_COPIES; ++r) c += h[r * HIST_BINS + idx];
+    if (c) atomicAdd(&ghist[(uint32_t(idx & 1) << 15) | (base + uint32_t(idx >> 1))], c);
   }
 }
 
@@ -732,10 +759,10 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
       KernelScope scope(ctx, stream, KC_SELECT, 3);
       init_occ_kernel<<<64, 1024, 0, stream>>>(sc.hist, sc.row_max, sc.row_min, sc.row_cnt, rows, sc.ticket);
       FP4_CUDA_TRY(cudaFuncSetAttribute(hist_rowminmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        HIST_WORDS * 4));
+                                        HIST_SMEM_BYTES));
       long long blocks = (n_vec + HIST_THREADS - 1) / HIST_THREADS;
       if (blocks > ctx->num_sms) blocks = ctx->num_sms;
-      hist_rowminmax_kernel<<<int(blocks), HIST_THREADS, HIST_WORDS * 4, stream>>>(x, n_vec, cols / 8, sc.hist,
+      hist_rowminmax_kernel<<<int(blocks), HIST_THREADS, HIST_SMEM_BYTES, stream>>>(x, n_vec, cols / 8, sc.hist,
                                                                                   sc.row_max, sc.row_min);
       select_thresholds_kernel<<<SELECT_BLOCKS, 1024, 0, stream>>>(sc.hist, n, n_tail, out->thresholds, sc.seg_sum,
                                                                    sc.ticket);
@@ -893,7 +920,7 @@ extern "C" int fp4_quantile_thresholds_static(void* stream, const void* x_bf16, 
     int sms = 0;
     FP4_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
     FP4_CUDA_TRY(cudaFuncSetAttribute(hist_rowminmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      HIST_WORDS * 4));
+                                      HIST_SMEM_BYTES));
     sms_of_device[device] = sms;
     scratch_of_device[device] = ptr;
   }
@@ -912,7 +939,7 @@ extern "C" int fp4_quantile_thresholds_static(void* stream, const void* x_bf16, 
   const long long n_vec = n / 8;
   long long blocks = (n_vec + HIST_THREADS - 1) / HIST_THREADS;
   if (blocks > sms_of_device[device]) blocks = sms_of_device[device];
-  hist_rowminmax_kernel<<<int(blocks), HIST_THREADS, HIST_WORDS * 4, st>>>(static_cast<const uint4*>(x_bf16), n_vec,
+  hist_rowminmax_kernel<<<int(blocks), HIST_THREADS, HIST_SMEM_BYTES, st>>>(static_cast<const uint4*>(x_bf16), n_vec,
                                                                           int(cols / 8), hist, row_max, row_min);
   select_thresholds_kernel<<<SELECT_BLOCKS, 1024, 0, st>>>(hist, n, n_tail, thresholds, seg_sum, ticket);
   FP4_CUDA_TRY(cudaGetLastError());

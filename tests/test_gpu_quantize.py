@@ -144,6 +144,29 @@ def test_occ_with_heavy_ties_and_zeros(lib, ctx):
         _check_dense(q, ref)
 
 
+def test_occ_values_outside_the_histogram_window(lib, ctx):
+    """The histogram kernel keeps shared counters for a window of exponents chosen from the first
+    elements each block sees; everything else must still be counted exactly.  Here the head of the
+    tensor is small, the rest is a million times larger, and tiny / subnormal values are sprinkled in."""
+    rng = np.random.default_rng(12)
+    a = rng.standard_normal((1024, 2048)).astype(np.float32)
+    a[:640] *= np.float32(1e-3)
+    a[640:] *= np.float32(1e3)
+    a[700:, 17] *= np.float32(1e4)
+    tiny = rng.random(a.shape) < 0.01
+    a[tiny] = (rng.standard_normal(int(tiny.sum())) * 1e-30).astype(np.float32)
+    a[rng.random(a.shape) < 0.001] = np.float32(1e-39)          # below the smallest normal BF16
+    bits = WL.to_bf16_bits(a)
+    for alpha in (0.999, 0.9):
+        ctx.status.zero_()
+        q = lib.fp4_quantize(ctx, _dev(bits), 0, alpha=alpha)
+        torch.cuda.synchronize()
+        assert ctx.read_status() == 0
+        ref = O.occ_quantize(O.bf16_bits_to_f64(bits), alpha)
+        _check_sparse(q, ref)
+        _check_dense(q, ref)
+
+
 def test_config0_activation_and_weight(lib, ctx):
     cfg = WL.CONFIGS[0]
     a_bits = WL.activations(cfg, 1024)
