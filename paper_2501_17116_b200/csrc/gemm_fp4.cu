@@ -29,14 +29,15 @@
 namespace {
 
 constexpr int BM = 128;
-constexpr int STAGES = 4;
+constexpr int EPI_WARPS = 8;               // two epilogue warps per lane quarter of tensor memory
+__host__ __device__ constexpr int stages_of(int kind) { return kind == FP4_GEMM_F8F6F4 ? 3 : 4; }
 constexpr int A_STAGE_BYTES = BM * 128;
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_STRIDE = 256;          // tensor-memory columns between the two accumulator stages
 constexpr int SF_COL_B = 240;            // MXF4 only: unit block scales in the gap behind stage 0
 constexpr int SF_COL_A = 248;
-constexpr int STAGE_OUT_BYTES = 4 * 4096; // epilogue: 32 rows x 128 bytes of output per warp
+constexpr int STAGE_OUT_BYTES = EPI_WARPS * 4096;   // epilogue: 32 rows x 128 bytes of output per warp
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
 
 __host__ __device__ constexpr int tile_n(int kind) { return kind == FP4_GEMM_F8F6F4 ? 256 : 240; }
@@ -44,7 +45,8 @@ __host__ __device__ constexpr int b_stage_bytes(int kind) { return tile_n(kind) 
 __host__ __device__ constexpr int stage_bytes(int kind) { return A_STAGE_BYTES + b_stage_bytes(kind); }
 // operand ring, barriers, column de-scales [2][256], staging [4][4096], DGE column scales [2][256], slots [2][128]
 constexpr size_t smem_bytes(int kind) {
-  return 1024 + size_t(STAGES) * stage_bytes(kind) + 256 + 2 * 256 * 4 + STAGE_OUT_BYTES + 2 * 256 * 4 + 2 * 128 * 4;
+  return 1024 + size_t(stages_of(kind)) * stage_bytes(kind) + 256 + 2 * 256 * 4 + STAGE_OUT_BYTES + 2 * 256 * 4 +
+         2 * 128 * 4;
 }
 
 struct GemmArgs {
@@ -167,13 +169,13 @@ __device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&v)[32])
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-// Barrier over the 128 epilogue threads that also ORs a flag, so that all four warps take the
+// Barrier over the 256 epilogue threads that also ORs a flag, so that all four warps take the
 // same decision to give up (a warp must never be left alone at this barrier).
 __device__ __forceinline__ bool epilogue_bar_any(bool flag) {
   uint32_t r;
   asm volatile(
       "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\t"
-      "bar.red.or.pred p, 1, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      "bar.red.or.pred p, 1, 256, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(r)
       : "r"(uint32_t(flag))
       : "memory");
@@ -205,33 +207,23 @@ __host__ __device__ constexpr uint32_t idesc_mxf4() {
          (uint32_t(BM >> 4) << 24);
 }
 
-// Global operands of the fused weight-gradient epilogue for one 32 x 32 chunk, in the layout of
-// the store phase (iteration i, lane -> row i * RPI + lane / LPR, 8 columns from 8 * (lane % LPR)).
-// They are fetched one chunk ahead so that their latency hides under the previous chunk.
+// Weights of the fused weight-gradient epilogue for one 32 x 32 chunk, in the layout of the store
+// phase (iteration i, lane -> row i * RPI + lane / LPR, 8 columns from 8 * (lane % LPR)).  They
+// are fetched one chunk ahead so that their latency hides under the previous chunk.
 struct EpiPrefetch {
-  uint4 w[4];            // 8 BF16 weights
-  float4 add[4][2];      // 8 compensation values (zeros for rows without a compensation row)
+  uint4 w[4];            // 8 BF16 weights per store iteration
 };
 template <int EPI>
-__device__ __forceinline__ void epi_prefetch(EpiPrefetch& pf, const GemmArgs& args, size_t elem_off, int col0,
-                                             int width, int lane, const int* slot_rows) {
-  if (EPI != EPI_WGRAD) return;
+__device__ __forceinline__ void epi_prefetch(EpiPrefetch& pf, const GemmArgs& args, size_t elem_off, int width,
+                                             int lane) {
+  if (EPI != EPI_WGRAD || !args.w) return;
   const int lpr = width / 8, rpi = 32 / lpr;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     pf.w[i] = make_uint4(0, 0, 0, 0);
-    pf.add[i][0] = pf.add[i][1] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (i < lpr) {
-      const int row = i * rpi + lane / lpr;
-      const int p = lane % lpr;
-      const size_t o = elem_off + size_t(row) * size_t(args.J) + size_t(8 * p);
-      if (args.w) pf.w[i] = __ldg(&args.w[o >> 3]);
-      const int slot = slot_rows[row];
-      if (slot >= 0) {
-        const float* src = args.addend + size_t(slot) * size_t(args.J) + size_t(col0 + 8 * p);
-        pf.add[i][0] = __ldg(reinterpret_cast<const float4*>(src));
-        pf.add[i][1] = __ldg(reinterpret_cast<const float4*>(src + 4));
-      }
+      const size_t o = elem_off + size_t(i * rpi + lane / lpr) * size_t(args.J) + size_t(8 * (lane % lpr));
+      pf.w[i] = __ldg(&args.w[o >> 3]);
     }
   }
 }
@@ -247,9 +239,25 @@ template <int W, int EPI>
 __device__ __forceinline__ void scale_stage_store(uint32_t (&v)[32], float d_row, const float* dcol, uint8_t* stage,
                                                   const GemmArgs& args, size_t elem_off, int lane,
                                                   uint32_t next_taddr, int next_width, const EpiPrefetch& pf,
-                                                  const float* gcol) {
+                                                  const float* gcol, const int* slot_rows, int col0) {
   constexpr int SPR = W / 4;                        // 16-byte slots per staged row: 8 or 4
   constexpr int SH = SPR == 8 ? 0 : 1;
+  constexpr int LPR = W / 8;                        // lanes per row in the store phase: 4 or 2
+  constexpr int RPI = 32 / LPR;                     // rows per store instruction: 8 or 16
+  // compensation rows of the store phase: requested first, consumed after the staging
+  float4 add[EPI == EPI_WGRAD ? LPR : 1][2];
+  if (EPI == EPI_WGRAD) {
+#pragma unroll
+    for (int i = 0; i < LPR; ++i) {
+      add[i][0] = add[i][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+      const int slot = slot_rows[i * RPI + lane / LPR];
+      if (slot >= 0) {
+        const float* src = args.addend + size_t(slot) * size_t(args.J) + size_t(col0 + 8 * (lane % LPR));
+        add[i][0] = __ldg(reinterpret_cast<const float4*>(src));
+        add[i][1] = __ldg(reinterpret_cast<const float4*>(src + 4));
+      }
+    }
+  }
   float y[W];
 #pragma unroll
   for (int q = 0; q < W / 4; ++q) {
@@ -268,8 +276,6 @@ __device__ __forceinline__ void scale_stage_store(uint32_t (&v)[32], float d_row
   for (int j = 0; j < SPR; ++j)
     *reinterpret_cast<float4*>(my_row + ((j ^ fx) * 16)) = make_float4(y[4 * j], y[4 * j + 1], y[4 * j + 2], y[4 * j + 3]);
   __syncwarp();
-  constexpr int LPR = W / 8;                        // lanes per row in the store phase: 4 or 2
-  constexpr int RPI = 32 / LPR;                     // rows per store instruction: 8 or 16
 #pragma unroll
   for (int i = 0; i < LPR; ++i) {
     const int row = i * RPI + lane / LPR;
@@ -281,8 +287,8 @@ __device__ __forceinline__ void scale_stage_store(uint32_t (&v)[32], float d_row
     float f[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
     const size_t o = elem_off + size_t(row) * size_t(args.J) + size_t(8 * p);
     if (EPI == EPI_WGRAD) {
-      f[0] += pf.add[i][0].x; f[1] += pf.add[i][0].y; f[2] += pf.add[i][0].z; f[3] += pf.add[i][0].w;
-      f[4] += pf.add[i][1].x; f[5] += pf.add[i][1].y; f[6] += pf.add[i][1].z; f[7] += pf.add[i][1].w;
+      f[0] += add[i][0].x; f[1] += add[i][0].y; f[2] += add[i][0].z; f[3] += add[i][0].w;
+      f[4] += add[i][1].x; f[5] += add[i][1].y; f[6] += add[i][1].z; f[7] += add[i][1].w;
       if (args.w) {
         const uint32_t ww[4] = {pf.w[i].x, pf.w[i].y, pf.w[i].z, pf.w[i].w};
         const float4 g0 = *reinterpret_cast<const float4*>(gcol + 8 * p);
@@ -312,33 +318,37 @@ __device__ __forceinline__ void scale_stage_store(uint32_t (&v)[32], float d_row
   __syncwarp();
 }
 
-// Epilogue of one 128 x BN block of accumulators for one warp (32 rows): 32-column chunks are read
-// from tensor memory, de-scaled, staged and stored; `row_blk` is the index of the 128-row block.
+// Epilogue of one 128 x BN block of accumulators for one warp (32 rows of it): the two warps that
+// share a lane quarter take the 32-column chunks alternately (`group` 0: chunks 0, 2, ...; 1: the
+// odd ones).  Chunks are read from tensor memory, de-scaled, staged and stored; `row_blk` is the
+// index of the 128-row block.
 template <int EPI, int BN>
 __device__ __forceinline__ void epilogue_tile(const GemmArgs& args, int row_blk, int n_blk, uint32_t t_base, float d_row,
                                               const float* dcol, const float* gcol, const int* slot_rows,
-                                              uint8_t* stage, int quarter, int lane) {
+                                              uint8_t* stage, int quarter, int group, int lane) {
   // first element of this warp's 32 rows in this tile
   const size_t warp_off = size_t(row_blk * BM + quarter * 32) * size_t(args.J) + size_t(n_blk) * BN;
   const int n_valid = min(BN, args.J - n_blk * BN);           // ragged last tile in N (multiple of 16)
+  int c0 = 32 * group;
+  if (c0 >= n_valid) return;
   EpiPrefetch pf;
-  epi_prefetch<EPI>(pf, args, warp_off, n_blk * BN, min(32, n_valid), lane, slot_rows);
+  epi_prefetch<EPI>(pf, args, warp_off + c0, min(32, n_valid - c0), lane);
   uint32_t v[32];
-  if (n_valid >= 32) tmem_ld_32x32(t_base, v); else tmem_ld_32x16(t_base, v);
+  if (n_valid - c0 >= 32) tmem_ld_32x32(t_base + uint32_t(c0), v); else tmem_ld_32x16(t_base + uint32_t(c0), v);
 #pragma unroll 1
-  for (int c0 = 0; c0 < n_valid; c0 += 32) {
+  for (; c0 < n_valid; c0 += 64) {
     const int width = min(32, n_valid - c0);
-    const int next_width = n_valid - (c0 + 32);                // <= 0: this is the last chunk
-    const uint32_t next_taddr = t_base + uint32_t(c0 + 32);
+    const int next_width = n_valid - (c0 + 64);                // <= 0: this is the warp's last chunk
+    const uint32_t next_taddr = t_base + uint32_t(c0 + 64);
     const EpiPrefetch cur = pf;
-    if (next_width > 0)
-      epi_prefetch<EPI>(pf, args, warp_off + c0 + 32, n_blk * BN + c0 + 32, min(32, next_width), lane, slot_rows);
+    if (next_width > 0) epi_prefetch<EPI>(pf, args, warp_off + c0 + 64, min(32, next_width), lane);
     tmem_ld_wait();
     if (width == 32)
       scale_stage_store<32, EPI>(v, d_row, dcol + c0, stage, args, warp_off + c0, lane, next_taddr, next_width, cur,
-                                 gcol + c0);
+                                 gcol + c0, slot_rows, n_blk * BN + c0);
     else
-      scale_stage_store<16, EPI>(v, d_row, dcol + c0, stage, args, warp_off + c0, lane, next_taddr, 0, cur, gcol + c0);
+      scale_stage_store<16, EPI>(v, d_row, dcol + c0, stage, args, warp_off + c0, lane, next_taddr, 0, cur, gcol + c0,
+                                 slot_rows, n_blk * BN + c0);
   }
 }
 
@@ -347,6 +357,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                 const GemmArgs args) {
   constexpr int NACC = 2;
+  constexpr int STAGES = stages_of(KIND);
   constexpr int BN = tile_n(KIND);
   constexpr int B_STAGE_BYTES = b_stage_bytes(KIND);
   constexpr int STAGE_BYTES = stage_bytes(KIND);
@@ -377,7 +388,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(&acc_full[a], 1);
-      mbar_init(&acc_empty[a], 4);
+      mbar_init(&acc_empty[a], EPI_WARPS);
     }
     mbar_init(final_bar, 1);
     *abort_flag = 0;
@@ -400,7 +411,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   if (KIND == FP4_GEMM_MXF4) {
     // Unit block scales: every byte of the scale columns is 0x7F (UE8M0 2^0), so the layout the
     // instruction expects inside these columns does not matter.
-    if (warp >= 2) {
+    if (warp >= 2 && warp < 6) {
       const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
       for (int c = 0; c < 16; c += 8) tmem_st_32x8(tmem_base + lane_base + SF_COL_B + c, 0x7F7F7F7Fu);
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
@@ -493,7 +504,8 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   } else {
     // ------------------------------------------------------------------ epilogue -----------
     const int quarter = warp & 3;               // the lane quarter of tensor memory this warp may read
-    const int et = threadIdx.x - 64;            // 0..127 among the epilogue threads
+    const int group = (warp - 2) >> 2;          // which of the two warps of this quarter
+    const int et = threadIdx.x - 64;            // 0..255 among the epilogue threads
     int acc = 0;
     uint32_t acc_phase = 0;
     uint32_t tile_parity = 0;
@@ -506,7 +518,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       float* dcol = s_dcol + tile_parity * 256;
       float* gcol = s_gcol + tile_parity * 256;
       int* slot_rows = s_slot + tile_parity * 128;
-      for (int c = et; c < BN; c += 128) {
+      for (int c = et; c < BN; c += 32 * EPI_WARPS) {
         const int col = n_blk * BN + c;
         dcol[c] = (args.col_amax && col < args.J) ? __fdiv_rn(__ldg(&args.col_amax[col]), 6.0f) : 1.0f;
         if (EPI == EPI_WGRAD && args.w) {
@@ -514,12 +526,12 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           gcol[c] = am > 0.0f ? __fdiv_rn(6.0f, am) : 0.0f;
         }
       }
-      if (EPI == EPI_WGRAD) slot_rows[et] = args.slot_of_row ? __ldg(&args.slot_of_row[m_blk * BM + et]) : -1;
+      if (EPI == EPI_WGRAD && et < BM) slot_rows[et] = args.slot_of_row ? __ldg(&args.slot_of_row[m_blk * BM + et]) : -1;
       const bool ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, args.status);
       if (epilogue_bar_any(!ok)) break;            // also publishes dcol to the other warps
       tc_fence_after();
       epilogue_tile<EPI, BN>(args, m_blk, n_blk, tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * ACC_STRIDE),
-                             d_row, dcol, gcol, slot_rows + quarter * 32, s_out + quarter * 4096, quarter, lane);
+                             d_row, dcol, gcol, slot_rows + quarter * 32, s_out + (warp - 2) * 4096, quarter, group, lane);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[acc]);
@@ -628,7 +640,7 @@ gemm_fp4_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(&acc_full[a], 1);
-      mbar_init(&acc_empty[a], 8);                  // four epilogue warps in each CTA
+      mbar_init(&acc_empty[a], 2 * EPI_WARPS);      // the epilogue warps of both CTAs
     }
     mbar_init(final_bar, 1);
     *abort_flag = 0;
@@ -649,7 +661,7 @@ gemm_fp4_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp >= 2) {                                  // unit block scales in this CTA's tensor memory
+  if (warp >= 2 && warp < 6) {                      // unit block scales in this CTA's tensor memory
     const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
     for (int c = 0; c < 16; c += 8) tmem_st_32x8(tmem_base + lane_base + SF_COL_B + c, 0x7F7F7F7Fu);
     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
@@ -729,6 +741,7 @@ gemm_fp4_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   } else {
     // ------------------------------------------------------------------ epilogue (both CTAs)
     const int quarter = warp & 3;
+    const int group = (warp - 2) >> 2;
     const int et = threadIdx.x - 64;
     int acc = 0;
     uint32_t acc_phase = 0;
@@ -743,7 +756,7 @@ gemm_fp4_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       float* dcol = s_dcol + tile_parity * 256;
       float* gcol = s_gcol + tile_parity * 256;
       int* slot_rows = s_slot + tile_parity * 128;
-      for (int c = et; c < BN; c += 128) {
+      for (int c = et; c < BN; c += 32 * EPI_WARPS) {
         const int col = n_blk * BN + c;
         dcol[c] = (args.col_amax && col < args.J) ? __fdiv_rn(__ldg(&args.col_amax[col]), 6.0f) : 1.0f;
         if (EPI == EPI_WGRAD && args.w) {
@@ -751,14 +764,14 @@ gemm_fp4_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
           gcol[c] = am > 0.0f ? __fdiv_rn(6.0f, am) : 0.0f;
         }
       }
-      if (EPI == EPI_WGRAD)
+      if (EPI == EPI_WGRAD && et < BM)
         slot_rows[et] = (args.slot_of_row && rows_valid) ? __ldg(&args.slot_of_row[row_blk * BM + et]) : -1;
       const bool ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, args.status);
       if (epilogue_bar_any(!ok)) break;
       tc_fence_after();
       if (rows_valid)
         epilogue_tile<EPI, BN>(args, row_blk, n_blk, tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * ACC_STRIDE),
-                               d_row, dcol, gcol, slot_rows + quarter * 32, s_out + quarter * 4096, quarter, lane);
+                               d_row, dcol, gcol, slot_rows + quarter * 32, s_out + (warp - 2) * 4096, quarter, group, lane);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_even_cta(&acc_empty[acc]);
