@@ -43,7 +43,7 @@ constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
 __host__ __device__ constexpr int tile_n(int kind) { return kind == FP4_GEMM_F8F6F4 ? 256 : 240; }
 __host__ __device__ constexpr int b_stage_bytes(int kind) { return tile_n(kind) * 128; }
 __host__ __device__ constexpr int stage_bytes(int kind) { return A_STAGE_BYTES + b_stage_bytes(kind); }
-// operand ring, barriers, column de-scales [2][256], staging [4][4096], DGE column scales [2][256], slots [2][128]
+// operand ring, staging [8][4096], barriers, column de-scales [2][256], DGE column scales [2][256], slots [2][128]
 constexpr size_t smem_bytes(int kind) {
   return 1024 + size_t(stages_of(kind)) * stage_bytes(kind) + 256 + 2 * 256 * 4 + STAGE_OUT_BYTES + 2 * 256 * 4 +
          2 * 128 * 4;
@@ -123,6 +123,21 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, u
       ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
       : "memory");
 }
+// Bulk tensor store of one box from shared memory (issued by one thread; completion is tracked by
+// that thread's bulk groups).  x counts elements of the innermost dimension and must be a multiple
+// of 16 bytes' worth of them.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map), "r"(c0),
+               "r"(c1), "r"(smem_u32(src))
+               : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// All but the newest of this thread's bulk stores have finished reading shared memory.
+__device__ __forceinline__ void tma_store_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+// All of this thread's bulk stores are complete.
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
@@ -228,6 +243,82 @@ __device__ __forceinline__ void epi_prefetch(EpiPrefetch& pf, const GemmArgs& ar
   }
 }
 
+// Where the bulk stores of the plain epilogue take their boxes from and how they are described.
+struct OutMaps {
+  const CUtensorMap* unit;      // box of 32 rows x 64 bytes (16 floats or 32 BF16), 64-byte swizzle
+  const CUtensorMap* half;      // BF16 only: box of 32 rows x 16 columns, no swizzle
+};
+
+// Plain epilogue of one 32 x W chunk: de-scale this thread's row, write it into one of the warp's
+// two 2 KB staging buffers in the 64-byte-swizzled layout of the tensor map (16-byte slot s of row
+// r sits at s ^ ((r >> 1) & 3): row-wise writes touch every bank once), and let one lane hand the
+// box to the copy engine.  The warp never waits for global memory: before a buffer is written
+// again only the shared-memory read of the store that used it two stores ago must have finished.
+// `seq` counts the warp's stores and picks the buffer.
+template <int W>
+__device__ __forceinline__ void scale_bulk_store(uint32_t (&v)[32], float d_row, const float* dcol, uint8_t* stage,
+                                                 const GemmArgs& args, const OutMaps& maps, int row0, int col0,
+                                                 int lane, uint32_t next_taddr, int next_width, uint32_t& seq) {
+  float y[W];
+#pragma unroll
+  for (int q = 0; q < W / 4; ++q) {
+    const float4 dc = *reinterpret_cast<const float4*>(dcol + 4 * q);     // same address in every lane
+    y[4 * q + 0] = __fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 0]), d_row), dc.x);
+    y[4 * q + 1] = __fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 1]), d_row), dc.y);
+    y[4 * q + 2] = __fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 2]), d_row), dc.z);
+    y[4 * q + 3] = __fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 3]), d_row), dc.w);
+  }
+  // v is dead now: fetch the next chunk of accumulators under the staging and the stores
+  if (next_width >= 32) tmem_ld_32x32(next_taddr, v);
+  else if (next_width > 0) tmem_ld_32x16(next_taddr, v);
+  const int fx = (lane >> 1) & 3;
+  if (args.out_f32) {
+#pragma unroll
+    for (int u = 0; u < W / 16; ++u) {              // one box per 16 columns
+      uint8_t* buf = stage + (seq & 1u) * 2048;
+      ++seq;
+      if (lane == 0) tma_store_wait_read_1();
+      __syncwarp();
+      uint8_t* my_row = buf + lane * 64;
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        *reinterpret_cast<float4*>(my_row + ((j ^ fx) * 16)) =
+            make_float4(y[16 * u + 4 * j], y[16 * u + 4 * j + 1], y[16 * u + 4 * j + 2], y[16 * u + 4 * j + 3]);
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0) tma_store_2d(maps.unit, buf, col0 + 16 * u, row0);
+    }
+  } else {
+    uint4 packed[W / 8];
+#pragma unroll
+    for (int j = 0; j < W / 8; ++j) {
+      uint32_t w4[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(y[8 * j + 2 * q], y[8 * j + 2 * q + 1]);
+        w4[q] = *reinterpret_cast<uint32_t*>(&h);
+      }
+      packed[j] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+    }
+    uint8_t* buf = stage + (seq & 1u) * 2048;
+    ++seq;
+    if (lane == 0) tma_store_wait_read_1();
+    __syncwarp();
+    if (W == 32) {
+      uint8_t* my_row = buf + lane * 64;
+#pragma unroll
+      for (int j = 0; j < W / 8; ++j) *reinterpret_cast<uint4*>(my_row + ((j ^ fx) * 16)) = packed[j];
+    } else {
+      uint8_t* my_row = buf + lane * 32;
+#pragma unroll
+      for (int j = 0; j < W / 8; ++j) *reinterpret_cast<uint4*>(my_row + j * 16) = packed[j];
+    }
+    fence_async_smem();
+    __syncwarp();
+    if (lane == 0) tma_store_2d(W == 32 ? maps.unit : maps.half, buf, col0, row0);
+  }
+}
+
 // De-scale W accumulators of this thread's row, then store the warp's 32 x W block through a
 // shared staging tile so that every store instruction writes whole row segments: the thread-per-
 // row layout of tensor memory would otherwise touch 32 different lines per instruction.
@@ -325,7 +416,8 @@ __device__ __forceinline__ void scale_stage_store(uint32_t (&v)[32], float d_row
 template <int EPI, int BN>
 __device__ __forceinline__ void epilogue_tile(const GemmArgs& args, int row_blk, int n_blk, uint32_t t_base, float d_row,
                                               const float* dcol, const float* gcol, const int* slot_rows,
-                                              uint8_t* stage, int quarter, int group, int lane) {
+                                              uint8_t* stage, int quarter, int group, int lane, const OutMaps& maps,
+                                              uint32_t& store_seq) {
   // first element of this warp's 32 rows in this tile
   const size_t warp_off = size_t(row_blk * BM + quarter * 32) * size_t(args.J) + size_t(n_blk) * BN;
   const int n_valid = min(BN, args.J - n_blk * BN);           // ragged last tile in N (multiple of 16)
@@ -343,7 +435,13 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs& args, int row_blk,
     const EpiPrefetch cur = pf;
     if (next_width > 0) epi_prefetch<EPI>(pf, args, warp_off + c0 + 64, min(32, next_width), lane);
     tmem_ld_wait();
-    if (width == 32)
+    if (EPI == EPI_PLAIN) {
+      const int row0 = row_blk * BM + quarter * 32, col0 = n_blk * BN + c0;
+      if (width == 32)
+        scale_bulk_store<32>(v, d_row, dcol + c0, stage, args, maps, row0, col0, lane, next_taddr, next_width, store_seq);
+      else
+        scale_bulk_store<16>(v, d_row, dcol + c0, stage, args, maps, row0, col0, lane, next_taddr, 0, store_seq);
+    } else if (width == 32)
       scale_stage_store<32, EPI>(v, d_row, dcol + c0, stage, args, warp_off + c0, lane, next_taddr, next_width, cur,
                                  gcol + c0, slot_rows, n_blk * BN + c0);
     else
@@ -355,6 +453,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs& args, int row_blk,
 template <int KIND, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                 const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_out_half,
                 const GemmArgs args) {
   constexpr int NACC = 2;
   constexpr int STAGES = stages_of(KIND);
@@ -365,16 +464,17 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* smem_a = smem;
   uint8_t* smem_b = smem + STAGES * A_STAGE_BYTES;
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+  uint8_t* s_out = smem + STAGES * STAGE_BYTES;        // [8 warps][4096] staging, 1024-byte aligned
+  uint8_t* smem_misc = s_out + STAGE_OUT_BYTES;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_misc);
   uint64_t* empty_bar = full_bar + STAGES;
   uint64_t* acc_full = empty_bar + STAGES;
   uint64_t* acc_empty = acc_full + 2;
   uint64_t* final_bar = acc_empty + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(final_bar + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* s_dcol = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES + 256);   // [2][256] column de-scales
-  uint8_t* s_out = smem + STAGES * STAGE_BYTES + 256 + 2 * 256 * 4;              // [4 warps][4096] staging
-  float* s_gcol = reinterpret_cast<float*>(s_out + STAGE_OUT_BYTES);             // [2][256] 6 / w_amax (DGE)
+  float* s_dcol = reinterpret_cast<float*>(smem_misc + 256);                     // [2][256] column de-scales
+  float* s_gcol = s_dcol + 2 * 256;                                              // [2][256] 6 / w_amax (DGE)
   int* s_slot = reinterpret_cast<int*>(s_gcol + 2 * 256);                        // [2][128] compensation rows
 
   const int warp = threadIdx.x >> 5;
@@ -396,6 +496,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+    if (EPI == EPI_PLAIN) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out) : "memory");
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
@@ -509,6 +610,8 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     int acc = 0;
     uint32_t acc_phase = 0;
     uint32_t tile_parity = 0;
+    uint32_t store_seq = 0;
+    const OutMaps out_maps = {&map_out, &map_out_half};
     for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
       const int m_blk = t % args.num_m_blocks;
       const int n_blk = t / args.num_m_blocks;
@@ -531,13 +634,15 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       if (epilogue_bar_any(!ok)) break;            // also publishes dcol to the other warps
       tc_fence_after();
       epilogue_tile<EPI, BN>(args, m_blk, n_blk, tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * ACC_STRIDE),
-                             d_row, dcol, gcol, slot_rows + quarter * 32, s_out + (warp - 2) * 4096, quarter, group, lane);
+                             d_row, dcol, gcol, slot_rows + quarter * 32, s_out + (warp - 2) * 4096, quarter, group, lane,
+                             out_maps, store_seq);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[acc]);
       if (++acc == NACC) { acc = 0; acc_phase ^= 1u; }
       tile_parity ^= 1u;
     }
+    if (EPI == EPI_PLAIN && lane == 0) tma_store_wait_all();    // this warp's bulk stores have landed
   }
 
   tc_fence_before();
@@ -607,6 +712,7 @@ __device__ __forceinline__ void mbar_arrive_even_cta(uint64_t* bar) {
 template <int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_fp4_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                      const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_out_half,
                      const GemmArgs args) {
   constexpr int NACC = 2;
   constexpr int BN = PAIR_BN;
@@ -614,16 +720,17 @@ gemm_fp4_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* smem_a = smem;
   uint8_t* smem_b = smem + PAIR_STAGES * A_STAGE_BYTES;
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + PAIR_STAGES * PAIR_STAGE_BYTES);
+  uint8_t* s_out = smem + PAIR_STAGES * PAIR_STAGE_BYTES;
+  uint8_t* smem_misc = s_out + STAGE_OUT_BYTES;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_misc);
   uint64_t* empty_bar = full_bar + PAIR_STAGES;
   uint64_t* acc_full = empty_bar + PAIR_STAGES;
   uint64_t* acc_empty = acc_full + 2;
   uint64_t* final_bar = acc_empty + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(final_bar + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* s_dcol = reinterpret_cast<float*>(smem + PAIR_STAGES * PAIR_STAGE_BYTES + 256);
-  uint8_t* s_out = smem + PAIR_STAGES * PAIR_STAGE_BYTES + 256 + 2 * 256 * 4;
-  float* s_gcol = reinterpret_cast<float*>(s_out + STAGE_OUT_BYTES);
+  float* s_dcol = reinterpret_cast<float*>(smem_misc + 256);
+  float* s_gcol = s_dcol + 2 * 256;
   int* s_slot = reinterpret_cast<int*>(s_gcol + 2 * 256);
 
   const int warp = threadIdx.x >> 5;
@@ -648,6 +755,7 @@ gemm_fp4_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+    if (EPI == EPI_PLAIN) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out) : "memory");
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
@@ -746,6 +854,8 @@ gemm_fp4_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     int acc = 0;
     uint32_t acc_phase = 0;
     uint32_t tile_parity = 0;
+    uint32_t store_seq = 0;
+    const OutMaps out_maps = {&map_out, &map_out_half};
     for (int t = pair; t < num_tiles; t += num_pairs) {
       const int m_blk = t % args.num_m_blocks;
       const int n_blk = t / args.num_m_blocks;
@@ -771,13 +881,15 @@ gemm_fp4_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       tc_fence_after();
       if (rows_valid)
         epilogue_tile<EPI, BN>(args, row_blk, n_blk, tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * ACC_STRIDE),
-                               d_row, dcol, gcol, slot_rows + quarter * 32, s_out + (warp - 2) * 4096, quarter, group, lane);
+                               d_row, dcol, gcol, slot_rows + quarter * 32, s_out + (warp - 2) * 4096, quarter, group, lane,
+                               out_maps, store_seq);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_even_cta(&acc_empty[acc]);
       if (++acc == NACC) { acc = 0; acc_phase ^= 1u; }
       tile_parity ^= 1u;
     }
+    if (EPI == EPI_PLAIN && lane == 0) tma_store_wait_all();
   }
 
   tc_fence_before();
@@ -817,23 +929,45 @@ int make_codes_map(fp4_ctx* ctx, CUtensorMap* map, const uint8_t* codes, int64_t
   return r == CUDA_SUCCESS ? FP4_OK : FP4_ERR_CUDA;
 }
 
+// Tensor maps of the output [I x J] for the bulk stores of the plain epilogue: `unit` is a box of
+// 32 rows x 64 bytes with the 64-byte swizzle, `half` (BF16 output only) a box of 32 rows x 16
+// columns without swizzle for the 16-column remainder of a tile.
+int make_out_maps(fp4_ctx* ctx, CUtensorMap* unit, CUtensorMap* half, void* out, int64_t I, int64_t J, int out_f32) {
+  EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
+  if (!encode) return FP4_ERR_CUDA;
+  const size_t elt = out_f32 ? 4 : 2;
+  const cuuint64_t dims[2] = {cuuint64_t(J), cuuint64_t(I)};
+  const cuuint64_t strides[1] = {cuuint64_t(J) * elt};
+  const cuuint32_t elem_strides[2] = {1, 1};
+  const CUtensorMapDataType dt = out_f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+  const cuuint32_t box_unit[2] = {cuuint32_t(64 / elt), 32};
+  CUresult r = encode(unit, dt, 2, out, dims, strides, box_unit, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                      CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return FP4_ERR_CUDA;
+  const cuuint32_t box_half[2] = {16, 32};
+  r = encode(half, dt, 2, out, dims, strides, box_half, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             out_f32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? FP4_OK : FP4_ERR_CUDA;
+}
+
 template <int EPI>
 int launch_pair_kernel(int pairs, cudaStream_t stream, const CUtensorMap& map_a, const CUtensorMap& map_b,
-                       const GemmArgs& args) {
+                       const CUtensorMap& map_out, const CUtensorMap& map_out_half, const GemmArgs& args) {
   constexpr size_t kSmem = pair_smem_bytes();
   FP4_CUDA_TRY(cudaFuncSetAttribute(gemm_fp4_pair_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     int(kSmem)));
-  gemm_fp4_pair_kernel<EPI><<<2 * pairs, NUM_THREADS, kSmem, stream>>>(map_a, map_b, args);
+  gemm_fp4_pair_kernel<EPI><<<2 * pairs, NUM_THREADS, kSmem, stream>>>(map_a, map_b, map_out, map_out_half, args);
   return FP4_OK;
 }
 
 template <int KIND, int EPI>
 int launch_kernel(int grid, cudaStream_t stream, const CUtensorMap& map_a, const CUtensorMap& map_b,
-                  const GemmArgs& args) {
+                  const CUtensorMap& map_out, const CUtensorMap& map_out_half, const GemmArgs& args) {
   constexpr size_t kSmem = smem_bytes(KIND);
   FP4_CUDA_TRY(cudaFuncSetAttribute(gemm_fp4_kernel<KIND, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     int(kSmem)));
-  gemm_fp4_kernel<KIND, EPI><<<grid, NUM_THREADS, kSmem, stream>>>(map_a, map_b, args);
+  gemm_fp4_kernel<KIND, EPI><<<grid, NUM_THREADS, kSmem, stream>>>(map_a, map_b, map_out, map_out_half, args);
   return FP4_OK;
 }
 
@@ -854,6 +988,10 @@ int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, c
   if (rc != FP4_OK) return rc;
   const int BN = tile_n(gemm_kind);
   rc = make_codes_map(ctx, &map_b, b_codes, J, C, pair_mode ? PAIR_BN / 2 : BN, gemm_kind);
+  if (rc != FP4_OK) return rc;
+  if (reinterpret_cast<uintptr_t>(out) & 15) return FP4_ERR_ALIGN;
+  CUtensorMap map_out, map_out_half;
+  rc = make_out_maps(ctx, &map_out, &map_out_half, out, I, J, out_f32);
   if (rc != FP4_OK) return rc;
 
   GemmArgs args;
@@ -887,14 +1025,14 @@ int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, c
   if (pair_mode) {
     const int max_pairs = ctx->num_sms / 2;
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
-    rc2 = fused ? launch_pair_kernel<EPI_WGRAD>(pairs, stream, map_a, map_b, args)
-                : launch_pair_kernel<EPI_PLAIN>(pairs, stream, map_a, map_b, args);
+    rc2 = fused ? launch_pair_kernel<EPI_WGRAD>(pairs, stream, map_a, map_b, map_out, map_out_half, args)
+                : launch_pair_kernel<EPI_PLAIN>(pairs, stream, map_a, map_b, map_out, map_out_half, args);
   } else if (gemm_kind == FP4_GEMM_F8F6F4)
-    rc2 = fused ? launch_kernel<FP4_GEMM_F8F6F4, EPI_WGRAD>(grid, stream, map_a, map_b, args)
-                : launch_kernel<FP4_GEMM_F8F6F4, EPI_PLAIN>(grid, stream, map_a, map_b, args);
+    rc2 = fused ? launch_kernel<FP4_GEMM_F8F6F4, EPI_WGRAD>(grid, stream, map_a, map_b, map_out, map_out_half, args)
+                : launch_kernel<FP4_GEMM_F8F6F4, EPI_PLAIN>(grid, stream, map_a, map_b, map_out, map_out_half, args);
   else
-    rc2 = fused ? launch_kernel<FP4_GEMM_MXF4, EPI_WGRAD>(grid, stream, map_a, map_b, args)
-                : launch_kernel<FP4_GEMM_MXF4, EPI_PLAIN>(grid, stream, map_a, map_b, args);
+    rc2 = fused ? launch_kernel<FP4_GEMM_MXF4, EPI_WGRAD>(grid, stream, map_a, map_b, map_out, map_out_half, args)
+                : launch_kernel<FP4_GEMM_MXF4, EPI_PLAIN>(grid, stream, map_a, map_b, map_out, map_out_half, args);
   if (rc2 != FP4_OK) return rc2;
   FP4_CUDA_TRY(cudaGetLastError());
   return FP4_OK;
