@@ -6,12 +6,14 @@
 // form of all three GEMMs of the layer (Fig. 2; Eq. 3; Appendix C.2).  The two de-scales are
 // applied to the accumulators in the epilogue, after the GEMM, as Appendix C.2 prescribes.
 //
-// Structure: persistent CTAs (one per SM), 128 x BN output tile per CTA, six warps:
+// Structure: persistent CTAs (one per SM), 128 x BN output tile per CTA:
 //   warp 0      TMA producer: cp.async.bulk.tensor loads into 128-byte-swizzled shared memory,
 //               a ring of STAGES stages guarded by full/empty mbarriers;
 //   warp 1      allocates tensor memory and issues tcgen05.mma from one thread, fp32
 //               accumulators in tensor memory; tcgen05.commit releases stages and publishes tiles;
-//   warps 2..5  epilogue: tcgen05.ld the accumulators (one row per thread), de-scale, store.
+//   warps 2..   epilogue (8 warps; 16 with the fused weight-gradient epilogue): tcgen05.ld the
+//               accumulators (one row per thread), de-scale, write boxes into shared memory and
+//               hand them to the copy engine (cp.async.bulk.tensor stores).
 // Tensor memory holds two accumulator stages, so the epilogue of one tile runs under the MMAs of
 // the next.  512 columns are 2 x 256; the MXF4 flavour also needs a few columns for its block
 // scales, so its tile is 128 x 240 (2 x 240 accumulator columns + 16 scale columns).
@@ -29,24 +31,26 @@
 namespace {
 
 constexpr int BM = 128;
-constexpr int EPI_WARPS = 8;               // two epilogue warps per lane quarter of tensor memory
+// Epilogue warps: two per lane quarter of tensor memory for the plain epilogue, four for the
+// fused weight-gradient epilogue, whose DGE arithmetic needs the extra warps to hide its latency.
+enum { EPI_PLAIN = 0, EPI_WGRAD = 1 };
+__host__ __device__ constexpr int epi_warps(int epi) { return epi == EPI_WGRAD ? 16 : 8; }
+__host__ __device__ constexpr int num_threads(int epi) { return 64 + 32 * epi_warps(epi); }
 __host__ __device__ constexpr int stages_of(int kind) { return kind == FP4_GEMM_F8F6F4 ? 3 : 4; }
 constexpr int A_STAGE_BYTES = BM * 128;
-constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_STRIDE = 256;          // tensor-memory columns between the two accumulator stages
 constexpr int SF_COL_B = 240;            // MXF4 only: unit block scales in the gap behind stage 0
 constexpr int SF_COL_A = 248;
-constexpr int STAGE_OUT_BYTES = EPI_WARPS * 4096;   // epilogue: 32 rows x 128 bytes of output per warp
+constexpr int STAGE_OUT_BYTES = 32768;    // epilogue staging: 4 KB per warp (plain) or 2 KB (fused)
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
 
 __host__ __device__ constexpr int tile_n(int kind) { return kind == FP4_GEMM_F8F6F4 ? 256 : 240; }
 __host__ __device__ constexpr int b_stage_bytes(int kind) { return tile_n(kind) * 128; }
 __host__ __device__ constexpr int stage_bytes(int kind) { return A_STAGE_BYTES + b_stage_bytes(kind); }
-// operand ring, staging [8][4096], barriers, column de-scales [2][256], DGE column scales [2][256], slots [2][128]
+// operand ring, epilogue staging, barriers, column de-scales [2][256], DGE column scales [2][256]
 constexpr size_t smem_bytes(int kind) {
-  return 1024 + size_t(stages_of(kind)) * stage_bytes(kind) + 256 + 2 * 256 * 4 + STAGE_OUT_BYTES + 2 * 256 * 4 +
-         2 * 128 * 4;
+  return 1024 + size_t(stages_of(kind)) * stage_bytes(kind) + 256 + 2 * 256 * 4 + STAGE_OUT_BYTES + 2 * 256 * 4;
 }
 
 struct GemmArgs {
@@ -66,8 +70,6 @@ struct GemmArgs {
   const float* w_amax;
   float inv_k, expo, clip;
 };
-
-enum { EPI_PLAIN = 0, EPI_WGRAD = 1 };
 
 // ------------------------------------------------------------------ PTX wrappers ------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -133,6 +135,7 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void*
   asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 // All but the newest of this thread's bulk stores have finished reading shared memory.
+__device__ __forceinline__ void tma_store_wait_read_0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 // All of this thread's bulk stores are complete.
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
@@ -184,15 +187,15 @@ __device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&v)[32])
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-// Barrier over the 256 epilogue threads that also ORs a flag, so that all four warps take the
-// same decision to give up (a warp must never be left alone at this barrier).
-__device__ __forceinline__ bool epilogue_bar_any(bool flag) {
+// Barrier over the `count` epilogue threads that also ORs a flag, so that all warps take the same
+// decision to give up (a warp must never be left alone at this barrier).
+__device__ __forceinline__ bool epilogue_bar_any(bool flag, int count) {
   uint32_t r;
   asm volatile(
       "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\t"
-      "bar.red.or.pred p, 1, 256, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      "bar.red.or.pred p, 1, %2, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(r)
-      : "r"(uint32_t(flag))
+      : "r"(uint32_t(flag)), "r"(count)
       : "memory");
   return r != 0;
 }
@@ -222,62 +225,29 @@ __host__ __device__ constexpr uint32_t idesc_mxf4() {
          (uint32_t(BM >> 4) << 24);
 }
 
-// Weights of the fused weight-gradient epilogue for one 32 x 32 chunk, in the layout of the store
-// phase (iteration i, lane -> row i * RPI + lane / LPR, 8 columns from 8 * (lane % LPR)).  They
-// are fetched one chunk ahead so that their latency hides under the previous chunk.
-struct EpiPrefetch {
-  uint4 w[4];            // 8 BF16 weights per store iteration
-};
-template <int EPI>
-__device__ __forceinline__ void epi_prefetch(EpiPrefetch& pf, const GemmArgs& args, size_t elem_off, int width,
-                                             int lane) {
-  if (EPI != EPI_WGRAD || !args.w) return;
-  const int lpr = width / 8, rpi = 32 / lpr;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    pf.w[i] = make_uint4(0, 0, 0, 0);
-    if (i < lpr) {
-      const size_t o = elem_off + size_t(i * rpi + lane / lpr) * size_t(args.J) + size_t(8 * (lane % lpr));
-      pf.w[i] = __ldg(&args.w[o >> 3]);
-    }
-  }
-}
-
-// Where the bulk stores of the plain epilogue take their boxes from and how they are described.
+// Where the bulk stores of the epilogue take their boxes from and how they are described.
 struct OutMaps {
   const CUtensorMap* unit;      // box of 32 rows x 64 bytes (16 floats or 32 BF16), 64-byte swizzle
-  const CUtensorMap* half;      // BF16 only: box of 32 rows x 16 columns, no swizzle
+  const CUtensorMap* half;      // BF16 output: box of 32 rows x 16 columns, no swizzle
 };
 
-// Plain epilogue of one 32 x W chunk: de-scale this thread's row, write it into one of the warp's
-// two 2 KB staging buffers in the 64-byte-swizzled layout of the tensor map (16-byte slot s of row
-// r sits at s ^ ((r >> 1) & 3): row-wise writes touch every bank once), and let one lane hand the
-// box to the copy engine.  The warp never waits for global memory: before a buffer is written
-// again only the shared-memory read of the store that used it two stores ago must have finished.
-// `seq` counts the warp's stores and picks the buffer.
-template <int W>
-__device__ __forceinline__ void scale_bulk_store(uint32_t (&v)[32], float d_row, const float* dcol, uint8_t* stage,
-                                                 const GemmArgs& args, const OutMaps& maps, int row0, int col0,
-                                                 int lane, uint32_t next_taddr, int next_width, uint32_t& seq) {
-  float y[W];
-#pragma unroll
-  for (int q = 0; q < W / 4; ++q) {
-    const float4 dc = *reinterpret_cast<const float4*>(dcol + 4 * q);     // same address in every lane
-    y[4 * q + 0] = __fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 0]), d_row), dc.x);
-    y[4 * q + 1] = __fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 1]), d_row), dc.y);
-    y[4 * q + 2] = __fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 2]), d_row), dc.z);
-    y[4 * q + 3] = __fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 3]), d_row), dc.w);
-  }
-  // v is dead now: fetch the next chunk of accumulators under the staging and the stores
-  if (next_width >= 32) tmem_ld_32x32(next_taddr, v);
-  else if (next_width > 0) tmem_ld_32x16(next_taddr, v);
+// One 32 x W chunk of de-scaled (and, in the fused epilogue, compensated and DGE-weighted) values,
+// row `lane` in y[]: write it into a staging buffer in the layout of the tensor map and let one
+// lane hand the box to the copy engine.  With the 64-byte swizzle, 16-byte slot s of row r sits
+// at s ^ ((r >> 1) & 3), so the row-wise writes touch every bank once.  The warp never waits for
+// global memory: before a buffer is written again only the shared-memory read of the store that
+// used it last must have finished.  `seq` counts the warp's stores; with NBUF = 2 they alternate
+// between two 2 KB buffers.
+template <int W, int NBUF>
+__device__ __forceinline__ void bulk_store_chunk(const float (&y)[W], uint8_t* stage, int out_f32, const OutMaps& maps,
+                                                 int row0, int col0, int lane, uint32_t& seq) {
   const int fx = (lane >> 1) & 3;
-  if (args.out_f32) {
+  if (out_f32) {
 #pragma unroll
     for (int u = 0; u < W / 16; ++u) {              // one box per 16 columns
-      uint8_t* buf = stage + (seq & 1u) * 2048;
+      uint8_t* buf = stage + (NBUF == 2 ? (seq & 1u) * 2048 : 0);
       ++seq;
-      if (lane == 0) tma_store_wait_read_1();
+      if (lane == 0) { if (NBUF == 2) tma_store_wait_read_1(); else tma_store_wait_read_0(); }
       __syncwarp();
       uint8_t* my_row = buf + lane * 64;
 #pragma unroll
@@ -300,9 +270,11 @@ __device__ __forceinline__ void scale_bulk_store(uint32_t (&v)[32], float d_row,
       }
       packed[j] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
     }
-    uint8_t* buf = stage + (seq & 1u) * 2048;
+    // a 16-column BF16 box is 1 KB: two of them always fit the 2 KB every warp has
+    constexpr bool two = NBUF == 2 || W == 16;
+    uint8_t* buf = stage + (two ? (seq & 1u) * (W == 16 && NBUF == 1 ? 1024 : 2048) : 0);
     ++seq;
-    if (lane == 0) tma_store_wait_read_1();
+    if (lane == 0) { if (two) tma_store_wait_read_1(); else tma_store_wait_read_0(); }
     __syncwarp();
     if (W == 32) {
       uint8_t* my_row = buf + lane * 64;
@@ -319,37 +291,8 @@ __device__ __forceinline__ void scale_bulk_store(uint32_t (&v)[32], float d_row,
   }
 }
 
-// De-scale W accumulators of this thread's row, then store the warp's 32 x W block through a
-// shared staging tile so that every store instruction writes whole row segments: the thread-per-
-// row layout of tensor memory would otherwise touch 32 different lines per instruction.
-// The staging tile holds 32 rows of W floats in 16-byte slots; slot s of row r sits at s ^ f(r),
-// which keeps both the row-wise writes and the segment-wise reads free of bank conflicts.  In the
-// store phase a lane owns 8 consecutive columns of one row; the fused weight-gradient epilogue
-// adds the compensation row and applies the DGE factor there, with coalesced reads of W.
-template <int W, int EPI>
-__device__ __forceinline__ void scale_stage_store(uint32_t (&v)[32], float d_row, const float* dcol, uint8_t* stage,
-                                                  const GemmArgs& args, size_t elem_off, int lane,
-                                                  uint32_t next_taddr, int next_width, const EpiPrefetch& pf,
-                                                  const float* gcol, const int* slot_rows, int col0) {
-  constexpr int SPR = W / 4;                        // 16-byte slots per staged row: 8 or 4
-  constexpr int SH = SPR == 8 ? 0 : 1;
-  constexpr int LPR = W / 8;                        // lanes per row in the store phase: 4 or 2
-  constexpr int RPI = 32 / LPR;                     // rows per store instruction: 8 or 16
-  // compensation rows of the store phase: requested first, consumed after the staging
-  float4 add[EPI == EPI_WGRAD ? LPR : 1][2];
-  if (EPI == EPI_WGRAD) {
-#pragma unroll
-    for (int i = 0; i < LPR; ++i) {
-      add[i][0] = add[i][1] = make_float4(0.f, 0.f, 0.f, 0.f);
-      const int slot = slot_rows[i * RPI + lane / LPR];
-      if (slot >= 0) {
-        const float* src = args.addend + size_t(slot) * size_t(args.J) + size_t(col0 + 8 * (lane % LPR));
-        add[i][0] = __ldg(reinterpret_cast<const float4*>(src));
-        add[i][1] = __ldg(reinterpret_cast<const float4*>(src + 4));
-      }
-    }
-  }
-  float y[W];
+template <int W>
+__device__ __forceinline__ void descale_chunk(const uint32_t (&v)[32], float d_row, const float* dcol, float (&y)[W]) {
 #pragma unroll
   for (int q = 0; q < W / 4; ++q) {
     const float4 dc = *reinterpret_cast<const float4*>(dcol + 4 * q);     // same address in every lane
@@ -358,102 +301,115 @@ __device__ __forceinline__ void scale_stage_store(uint32_t (&v)[32], float d_row
     y[4 * q + 2] = __fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 2]), d_row), dc.z);
     y[4 * q + 3] = __fmul_rn(__fmul_rn(__uint_as_float(v[4 * q + 3]), d_row), dc.w);
   }
-  // v is dead now: fetch the next chunk of accumulators under the staging and the stores
-  if (next_width >= 32) tmem_ld_32x32(next_taddr, v);
-  else if (next_width > 0) tmem_ld_32x16(next_taddr, v);
-  uint8_t* my_row = stage + lane * (SPR * 16);
-  const int fx = (lane >> SH) & (SPR - 1);
-#pragma unroll
-  for (int j = 0; j < SPR; ++j)
-    *reinterpret_cast<float4*>(my_row + ((j ^ fx) * 16)) = make_float4(y[4 * j], y[4 * j + 1], y[4 * j + 2], y[4 * j + 3]);
-  __syncwarp();
-#pragma unroll
-  for (int i = 0; i < LPR; ++i) {
-    const int row = i * RPI + lane / LPR;
-    const int p = lane % LPR;
-    const int fr = (row >> SH) & (SPR - 1);
-    const uint8_t* srow = stage + row * (SPR * 16);
-    const float4 a = *reinterpret_cast<const float4*>(srow + (((2 * p) ^ fr) * 16));
-    const float4 b = *reinterpret_cast<const float4*>(srow + (((2 * p + 1) ^ fr) * 16));
-    float f[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-    const size_t o = elem_off + size_t(row) * size_t(args.J) + size_t(8 * p);
-    if (EPI == EPI_WGRAD) {
-      f[0] += add[i][0].x; f[1] += add[i][0].y; f[2] += add[i][0].z; f[3] += add[i][0].w;
-      f[4] += add[i][1].x; f[5] += add[i][1].y; f[6] += add[i][1].z; f[7] += add[i][1].w;
-      if (args.w) {
-        const uint32_t ww[4] = {pf.w[i].x, pf.w[i].y, pf.w[i].z, pf.w[i].w};
-        const float4 g0 = *reinterpret_cast<const float4*>(gcol + 8 * p);
-        const float4 g1 = *reinterpret_cast<const float4*>(gcol + 8 * p + 4);
-        const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const float wf = __uint_as_float((c & 1) ? (ww[c >> 1] & 0xFFFF0000u) : (ww[c >> 1] << 16));
-          f[c] *= dge_factor(__fmul_rn(wf, g[c]), args.expo, args.inv_k, args.clip);
-        }
-      }
-    }
-    if (args.out_f32) {
-      float4* dst = reinterpret_cast<float4*>(static_cast<float*>(args.out) + o);
-      dst[0] = make_float4(f[0], f[1], f[2], f[3]);
-      dst[1] = make_float4(f[4], f[5], f[6], f[7]);
-    } else {
-      uint32_t w4[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * q], f[2 * q + 1]);
-        w4[q] = *reinterpret_cast<uint32_t*>(&h);
-      }
-      *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(args.out) + o) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
-    }
-  }
-  __syncwarp();
 }
 
-// Epilogue of one 128 x BN block of accumulators for one warp (32 rows of it): the two warps that
-// share a lane quarter take the 32-column chunks alternately (`group` 0: chunks 0, 2, ...; 1: the
-// odd ones).  Chunks are read from tensor memory, de-scaled, staged and stored; `row_blk` is the
-// index of the 128-row block.
-template <int EPI, int BN>
-__device__ __forceinline__ void epilogue_tile(const GemmArgs& args, int row_blk, int n_blk, uint32_t t_base, float d_row,
-                                              const float* dcol, const float* gcol, const int* slot_rows,
-                                              uint8_t* stage, int quarter, int group, int lane, const OutMaps& maps,
-                                              uint32_t& store_seq) {
-  // first element of this warp's 32 rows in this tile
-  const size_t warp_off = size_t(row_blk * BM + quarter * 32) * size_t(args.J) + size_t(n_blk) * BN;
+// Plain epilogue of one 128 x BN block of accumulators for one warp (32 rows of it).  The warps
+// that share a lane quarter take the 32-column chunks in turn (`group` g of G: chunks g, g + G,
+// ...).  Chunks are read from tensor memory (the next one under the stores of the current one),
+// de-scaled and stored; `row_blk` is the index of the 128-row block.
+template <int BN, int G>
+__device__ __forceinline__ void epilogue_tile_plain(const GemmArgs& args, int row_blk, int n_blk, uint32_t t_base,
+                                                    float d_row, const float* dcol, uint8_t* stage, int quarter,
+                                                    int group, int lane, const OutMaps& maps, uint32_t& seq) {
   const int n_valid = min(BN, args.J - n_blk * BN);           // ragged last tile in N (multiple of 16)
+  const int row0 = row_blk * BM + quarter * 32;
   int c0 = 32 * group;
   if (c0 >= n_valid) return;
-  EpiPrefetch pf;
-  epi_prefetch<EPI>(pf, args, warp_off + c0, min(32, n_valid - c0), lane);
   uint32_t v[32];
   if (n_valid - c0 >= 32) tmem_ld_32x32(t_base + uint32_t(c0), v); else tmem_ld_32x16(t_base + uint32_t(c0), v);
 #pragma unroll 1
-  for (; c0 < n_valid; c0 += 64) {
+  for (; c0 < n_valid; c0 += 32 * G) {
     const int width = min(32, n_valid - c0);
-    const int next_width = n_valid - (c0 + 64);                // <= 0: this is the warp's last chunk
-    const uint32_t next_taddr = t_base + uint32_t(c0 + 64);
-    const EpiPrefetch cur = pf;
-    if (next_width > 0) epi_prefetch<EPI>(pf, args, warp_off + c0 + 64, min(32, next_width), lane);
+    const int next_width = n_valid - (c0 + 32 * G);            // <= 0: this is the warp's last chunk
+    const uint32_t next_taddr = t_base + uint32_t(c0 + 32 * G);
     tmem_ld_wait();
-    if (EPI == EPI_PLAIN) {
-      const int row0 = row_blk * BM + quarter * 32, col0 = n_blk * BN + c0;
-      if (width == 32)
-        scale_bulk_store<32>(v, d_row, dcol + c0, stage, args, maps, row0, col0, lane, next_taddr, next_width, store_seq);
-      else
-        scale_bulk_store<16>(v, d_row, dcol + c0, stage, args, maps, row0, col0, lane, next_taddr, 0, store_seq);
-    } else if (width == 32)
-      scale_stage_store<32, EPI>(v, d_row, dcol + c0, stage, args, warp_off + c0, lane, next_taddr, next_width, cur,
-                                 gcol + c0, slot_rows, n_blk * BN + c0);
-    else
-      scale_stage_store<16, EPI>(v, d_row, dcol + c0, stage, args, warp_off + c0, lane, next_taddr, 0, cur, gcol + c0,
-                                 slot_rows, n_blk * BN + c0);
+    if (width == 32) {
+      float y[32];
+      descale_chunk<32>(v, d_row, dcol + c0, y);
+      if (next_width >= 32) tmem_ld_32x32(next_taddr, v);      // v is dead: fetch under the stores
+      else if (next_width > 0) tmem_ld_32x16(next_taddr, v);
+      bulk_store_chunk<32, 2>(y, stage, args.out_f32, maps, row0, n_blk * BN + c0, lane, seq);
+    } else {
+      float y[16];
+      descale_chunk<16>(v, d_row, dcol + c0, y);
+      bulk_store_chunk<16, 2>(y, stage, args.out_f32, maps, row0, n_blk * BN + c0, lane, seq);
+    }
+  }
+}
+
+// Operands of the fused weight-gradient epilogue for 16 columns of this thread's row: the BF16
+// weights that drive the DGE factor and the compensation row.  They are requested one chunk
+// ahead, right after the previous chunk's have been consumed.
+struct WgradOperands {
+  uint4 w[2];            // 16 BF16 weights
+  float4 add[4];         // 16 floats of the compensation row (zeros without one)
+};
+__device__ __forceinline__ void wgrad_fetch(WgradOperands& op, const GemmArgs& args, int row, int slot, int col) {
+  if (args.w) {
+    const uint4* src = args.w + ((size_t(row) * size_t(args.J) + size_t(col)) >> 3);
+    op.w[0] = __ldg(src);
+    op.w[1] = __ldg(src + 1);
+  }
+#pragma unroll
+  for (int j = 0; j < 4; ++j) op.add[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (slot >= 0) {
+    const float4* src = reinterpret_cast<const float4*>(args.addend + size_t(slot) * size_t(args.J) + size_t(col));
+#pragma unroll
+    for (int j = 0; j < 4; ++j) op.add[j] = __ldg(src + j);
+  }
+}
+
+// Fused weight-gradient epilogue for one warp: 16-column chunks, every thread keeps its own row
+//   out[k, n] = store( (acc * d_col[n] + addend[slot[k], n]) * Q'(w[k, n] * 6 / w_amax[n]) ).
+// The thread-per-row layout of tensor memory is kept throughout: the weights and the
+// compensation row are read as whole 32-byte sectors per thread, the results leave through a
+// bulk store.  `first` holds the operands of the warp's first chunk, requested by the caller
+// before the accumulators were awaited.
+template <int BN, int G>
+__device__ __forceinline__ void epilogue_tile_wgrad(const GemmArgs& args, int row_blk, int n_blk, uint32_t t_base,
+                                                    float d_row, const float* dcol, const float* gcol, int slot,
+                                                    uint8_t* stage, int quarter, int group, int lane,
+                                                    const OutMaps& maps, uint32_t& seq, WgradOperands& op) {
+  const int n_valid = min(BN, args.J - n_blk * BN);
+  const int row0 = row_blk * BM + quarter * 32;
+  int c0 = 16 * group;
+  if (c0 >= n_valid) return;
+  uint32_t v[32];
+  tmem_ld_32x16(t_base + uint32_t(c0), v);
+#pragma unroll 1
+  for (; c0 < n_valid; c0 += 16 * G) {
+    const bool more = c0 + 16 * G < n_valid;
+    tmem_ld_wait();
+    float y[16];
+    descale_chunk<16>(v, d_row, dcol + c0, y);
+    if (more) tmem_ld_32x16(t_base + uint32_t(c0 + 16 * G), v);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      y[4 * j + 0] += op.add[j].x; y[4 * j + 1] += op.add[j].y; y[4 * j + 2] += op.add[j].z; y[4 * j + 3] += op.add[j].w;
+    }
+    if (args.w) {
+      const uint32_t ww[8] = {op.w[0].x, op.w[0].y, op.w[0].z, op.w[0].w, op.w[1].x, op.w[1].y, op.w[1].z, op.w[1].w};
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float4 g4 = *reinterpret_cast<const float4*>(gcol + c0 + 4 * q);   // same address in every lane
+        const float g[4] = {g4.x, g4.y, g4.z, g4.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int c = 4 * q + e;
+          const float wf = __uint_as_float((c & 1) ? (ww[c >> 1] & 0xFFFF0000u) : (ww[c >> 1] << 16));
+          y[c] *= dge_factor(__fmul_rn(wf, g[e]), args.expo, args.inv_k, args.clip);
+        }
+      }
+    }
+    if (more) wgrad_fetch(op, args, row0 + lane, slot, n_blk * BN + c0 + 16 * G);
+    bulk_store_chunk<16, 1>(y, stage, args.out_f32, maps, row0, n_blk * BN + c0, lane, seq);
   }
 }
 
 template <int KIND, int EPI>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(num_threads(EPI), 1)
 gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                 const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_out_half,
+                 const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_out_aux,
                 const GemmArgs args) {
   constexpr int NACC = 2;
   constexpr int STAGES = stages_of(KIND);
@@ -475,7 +431,6 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* s_dcol = reinterpret_cast<float*>(smem_misc + 256);                     // [2][256] column de-scales
   float* s_gcol = s_dcol + 2 * 256;                                              // [2][256] 6 / w_amax (DGE)
-  int* s_slot = reinterpret_cast<int*>(s_gcol + 2 * 256);                        // [2][128] compensation rows
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -488,7 +443,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(&acc_full[a], 1);
-      mbar_init(&acc_empty[a], EPI_WARPS);
+      mbar_init(&acc_empty[a], epi_warps(EPI));
     }
     mbar_init(final_bar, 1);
     *abort_flag = 0;
@@ -496,7 +451,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
-    if (EPI == EPI_PLAIN) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out) : "memory");
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
@@ -604,14 +559,17 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     }
   } else {
     // ------------------------------------------------------------------ epilogue -----------
+    constexpr int EW = epi_warps(EPI);
+    constexpr int G = EW / 4;                   // warps per lane quarter
     const int quarter = warp & 3;               // the lane quarter of tensor memory this warp may read
-    const int group = (warp - 2) >> 2;          // which of the two warps of this quarter
-    const int et = threadIdx.x - 64;            // 0..255 among the epilogue threads
+    const int group = (warp - 2) >> 2;          // which of the G warps of this quarter
+    const int et = threadIdx.x - 64;            // index among the epilogue threads
+    uint8_t* stage = s_out + (warp - 2) * (STAGE_OUT_BYTES / EW);
     int acc = 0;
     uint32_t acc_phase = 0;
     uint32_t tile_parity = 0;
     uint32_t store_seq = 0;
-    const OutMaps out_maps = {&map_out, &map_out_half};
+    const OutMaps out_maps = {&map_out, &map_out_aux};
     for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
       const int m_blk = t % args.num_m_blocks;
       const int n_blk = t / args.num_m_blocks;
@@ -620,8 +578,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const float d_row = args.row_amax ? __fdiv_rn(__ldg(&args.row_amax[row]), 6.0f) : 1.0f;
       float* dcol = s_dcol + tile_parity * 256;
       float* gcol = s_gcol + tile_parity * 256;
-      int* slot_rows = s_slot + tile_parity * 128;
-      for (int c = et; c < BN; c += 32 * EPI_WARPS) {
+      for (int c = et; c < BN; c += 32 * EW) {
         const int col = n_blk * BN + c;
         dcol[c] = (args.col_amax && col < args.J) ? __fdiv_rn(__ldg(&args.col_amax[col]), 6.0f) : 1.0f;
         if (EPI == EPI_WGRAD && args.w) {
@@ -629,20 +586,29 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           gcol[c] = am > 0.0f ? __fdiv_rn(6.0f, am) : 0.0f;
         }
       }
-      if (EPI == EPI_WGRAD && et < BM) slot_rows[et] = args.slot_of_row ? __ldg(&args.slot_of_row[m_blk * BM + et]) : -1;
+      int slot = -1;
+      WgradOperands op;
+      if (EPI == EPI_WGRAD) {
+        if (args.slot_of_row) slot = __ldg(&args.slot_of_row[row]);
+        if (n_blk * BN + 16 * group < args.J) wgrad_fetch(op, args, row, slot, n_blk * BN + 16 * group);
+      }
       const bool ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, args.status);
-      if (epilogue_bar_any(!ok)) break;            // also publishes dcol to the other warps
+      if (epilogue_bar_any(!ok, 32 * EW)) break;   // also publishes dcol to the other warps
       tc_fence_after();
-      epilogue_tile<EPI, BN>(args, m_blk, n_blk, tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * ACC_STRIDE),
-                             d_row, dcol, gcol, slot_rows + quarter * 32, s_out + (warp - 2) * 4096, quarter, group, lane,
-                             out_maps, store_seq);
+      const uint32_t t_base = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * ACC_STRIDE);
+      if (EPI == EPI_WGRAD)
+        epilogue_tile_wgrad<BN, G>(args, m_blk, n_blk, t_base, d_row, dcol, gcol, slot, stage, quarter, group, lane,
+                                   out_maps, store_seq, op);
+      else
+        epilogue_tile_plain<BN, G>(args, m_blk, n_blk, t_base, d_row, dcol, stage, quarter, group, lane, out_maps,
+                                   store_seq);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[acc]);
       if (++acc == NACC) { acc = 0; acc_phase ^= 1u; }
       tile_parity ^= 1u;
     }
-    if (EPI == EPI_PLAIN && lane == 0) tma_store_wait_all();    // this warp's bulk stores have landed
+    if (lane == 0) tma_store_wait_all();    // this warp's bulk stores have landed
   }
 
   tc_fence_before();
@@ -665,7 +631,7 @@ constexpr int PAIR_B_STAGE_BYTES = (PAIR_BN / 2) * 128;
 constexpr int PAIR_STAGE_BYTES = A_STAGE_BYTES + PAIR_B_STAGE_BYTES;
 constexpr uint32_t PEER_BIT_MASK = 0xFEFFFFFFu;     // clears the CTA-rank bit of a shared::cluster address
 constexpr size_t pair_smem_bytes() {
-  return 1024 + size_t(PAIR_STAGES) * PAIR_STAGE_BYTES + 256 + 2 * 256 * 4 + STAGE_OUT_BYTES + 2 * 256 * 4 + 2 * 128 * 4;
+  return 1024 + size_t(PAIR_STAGES) * PAIR_STAGE_BYTES + 256 + 2 * 256 * 4 + STAGE_OUT_BYTES + 2 * 256 * 4;
 }
 __host__ __device__ constexpr uint32_t idesc_mxf4_pair() {
   return (1u << 7) | (1u << 10) | (uint32_t(PAIR_BN >> 3) << 17) | (1u << 23) | (uint32_t(256 >> 4) << 24);
@@ -710,9 +676,9 @@ __device__ __forceinline__ void mbar_arrive_even_cta(uint64_t* bar) {
 }
 
 template <int EPI>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(num_threads(EPI), 1)
 gemm_fp4_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                      const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_out_half,
+                      const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_out_aux,
                      const GemmArgs args) {
   constexpr int NACC = 2;
   constexpr int BN = PAIR_BN;
@@ -731,7 +697,6 @@ gemm_fp4_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* s_dcol = reinterpret_cast<float*>(smem_misc + 256);
   float* s_gcol = s_dcol + 2 * 256;
-  int* s_slot = reinterpret_cast<int*>(s_gcol + 2 * 256);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -747,7 +712,7 @@ gemm_fp4_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(&acc_full[a], 1);
-      mbar_init(&acc_empty[a], 2 * EPI_WARPS);      // the epilogue warps of both CTAs
+      mbar_init(&acc_empty[a], 2 * epi_warps(EPI));      // the epilogue warps of both CTAs
     }
     mbar_init(final_bar, 1);
     *abort_flag = 0;
@@ -755,7 +720,7 @@ gemm_fp4_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
-    if (EPI == EPI_PLAIN) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out) : "memory");
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
@@ -848,14 +813,17 @@ gemm_fp4_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
     }
   } else {
     // ------------------------------------------------------------------ epilogue (both CTAs)
+    constexpr int EW = epi_warps(EPI);
+    constexpr int G = EW / 4;
     const int quarter = warp & 3;
     const int group = (warp - 2) >> 2;
     const int et = threadIdx.x - 64;
+    uint8_t* stage = s_out + (warp - 2) * (STAGE_OUT_BYTES / EW);
     int acc = 0;
     uint32_t acc_phase = 0;
     uint32_t tile_parity = 0;
     uint32_t store_seq = 0;
-    const OutMaps out_maps = {&map_out, &map_out_half};
+    const OutMaps out_maps = {&map_out, &map_out_aux};
     for (int t = pair; t < num_tiles; t += num_pairs) {
       const int m_blk = t % args.num_m_blocks;
       const int n_blk = t / args.num_m_blocks;
@@ -865,8 +833,7 @@ gemm_fp4_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
       const float d_row = (args.row_amax && rows_valid) ? __fdiv_rn(__ldg(&args.row_amax[row]), 6.0f) : 1.0f;
       float* dcol = s_dcol + tile_parity * 256;
       float* gcol = s_gcol + tile_parity * 256;
-      int* slot_rows = s_slot + tile_parity * 128;
-      for (int c = et; c < BN; c += 32 * EPI_WARPS) {
+      for (int c = et; c < BN; c += 32 * EW) {
         const int col = n_blk * BN + c;
         dcol[c] = (args.col_amax && col < args.J) ? __fdiv_rn(__ldg(&args.col_amax[col]), 6.0f) : 1.0f;
         if (EPI == EPI_WGRAD && args.w) {
@@ -874,22 +841,31 @@ gemm_fp4_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
           gcol[c] = am > 0.0f ? __fdiv_rn(6.0f, am) : 0.0f;
         }
       }
-      if (EPI == EPI_WGRAD && et < BM)
-        slot_rows[et] = (args.slot_of_row && rows_valid) ? __ldg(&args.slot_of_row[row_blk * BM + et]) : -1;
+      int slot = -1;
+      WgradOperands op;
+      if (EPI == EPI_WGRAD && rows_valid) {
+        if (args.slot_of_row) slot = __ldg(&args.slot_of_row[row]);
+        if (n_blk * BN + 16 * group < args.J) wgrad_fetch(op, args, row, slot, n_blk * BN + 16 * group);
+      }
       const bool ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, args.status);
-      if (epilogue_bar_any(!ok)) break;
+      if (epilogue_bar_any(!ok, 32 * EW)) break;
       tc_fence_after();
-      if (rows_valid)
-        epilogue_tile<EPI, BN>(args, row_blk, n_blk, tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * ACC_STRIDE),
-                               d_row, dcol, gcol, slot_rows + quarter * 32, s_out + (warp - 2) * 4096, quarter, group, lane,
-                               out_maps, store_seq);
+      const uint32_t t_base = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * ACC_STRIDE);
+      if (rows_valid) {
+        if (EPI == EPI_WGRAD)
+          epilogue_tile_wgrad<BN, G>(args, row_blk, n_blk, t_base, d_row, dcol, gcol, slot, stage, quarter, group, lane,
+                                     out_maps, store_seq, op);
+        else
+          epilogue_tile_plain<BN, G>(args, row_blk, n_blk, t_base, d_row, dcol, stage, quarter, group, lane, out_maps,
+                                     store_seq);
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_even_cta(&acc_empty[acc]);
       if (++acc == NACC) { acc = 0; acc_phase ^= 1u; }
       tile_parity ^= 1u;
     }
-    if (EPI == EPI_PLAIN && lane == 0) tma_store_wait_all();
+    if (lane == 0) tma_store_wait_all();
   }
 
   tc_fence_before();
@@ -929,10 +905,10 @@ int make_codes_map(fp4_ctx* ctx, CUtensorMap* map, const uint8_t* codes, int64_t
   return r == CUDA_SUCCESS ? FP4_OK : FP4_ERR_CUDA;
 }
 
-// Tensor maps of the output [I x J] for the bulk stores of the plain epilogue: `unit` is a box of
-// 32 rows x 64 bytes with the 64-byte swizzle, `half` (BF16 output only) a box of 32 rows x 16
-// columns without swizzle for the 16-column remainder of a tile.
-int make_out_maps(fp4_ctx* ctx, CUtensorMap* unit, CUtensorMap* half, void* out, int64_t I, int64_t J, int out_f32) {
+// Tensor maps of the output [I x J] for the bulk stores of the epilogue.  `unit` is a box of 32 rows
+// x 64 bytes with the 64-byte swizzle; `aux` is, for BF16 output, a box of 32 rows x 16 columns
+// without swizzle (16-column chunks) and unused for fp32 output (a copy of `unit`).
+int make_out_maps(fp4_ctx* ctx, CUtensorMap* unit, CUtensorMap* aux, void* out, int64_t I, int64_t J, int out_f32) {
   EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
   if (!encode) return FP4_ERR_CUDA;
   const size_t elt = out_f32 ? 4 : 2;
@@ -944,8 +920,8 @@ int make_out_maps(fp4_ctx* ctx, CUtensorMap* unit, CUtensorMap* half, void* out,
   CUresult r = encode(unit, dt, 2, out, dims, strides, box_unit, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
                       CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return FP4_ERR_CUDA;
-  const cuuint32_t box_half[2] = {16, 32};
-  r = encode(half, dt, 2, out, dims, strides, box_half, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
+  const cuuint32_t box_aux[2] = {16, 32};
+  r = encode(aux, dt, 2, out, dims, strides, box_aux, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
              out_f32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? FP4_OK : FP4_ERR_CUDA;
@@ -953,21 +929,21 @@ int make_out_maps(fp4_ctx* ctx, CUtensorMap* unit, CUtensorMap* half, void* out,
 
 template <int EPI>
 int launch_pair_kernel(int pairs, cudaStream_t stream, const CUtensorMap& map_a, const CUtensorMap& map_b,
-                       const CUtensorMap& map_out, const CUtensorMap& map_out_half, const GemmArgs& args) {
+                       const CUtensorMap& map_out, const CUtensorMap& map_out_aux, const GemmArgs& args) {
   constexpr size_t kSmem = pair_smem_bytes();
   FP4_CUDA_TRY(cudaFuncSetAttribute(gemm_fp4_pair_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     int(kSmem)));
-  gemm_fp4_pair_kernel<EPI><<<2 * pairs, NUM_THREADS, kSmem, stream>>>(map_a, map_b, map_out, map_out_half, args);
+  gemm_fp4_pair_kernel<EPI><<<2 * pairs, num_threads(EPI), kSmem, stream>>>(map_a, map_b, map_out, map_out_aux, args);
   return FP4_OK;
 }
 
 template <int KIND, int EPI>
 int launch_kernel(int grid, cudaStream_t stream, const CUtensorMap& map_a, const CUtensorMap& map_b,
-                  const CUtensorMap& map_out, const CUtensorMap& map_out_half, const GemmArgs& args) {
+                  const CUtensorMap& map_out, const CUtensorMap& map_out_aux, const GemmArgs& args) {
   constexpr size_t kSmem = smem_bytes(KIND);
   FP4_CUDA_TRY(cudaFuncSetAttribute(gemm_fp4_kernel<KIND, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     int(kSmem)));
-  gemm_fp4_kernel<KIND, EPI><<<grid, NUM_THREADS, kSmem, stream>>>(map_a, map_b, map_out, map_out_half, args);
+  gemm_fp4_kernel<KIND, EPI><<<grid, num_threads(EPI), kSmem, stream>>>(map_a, map_b, map_out, map_out_aux, args);
   return FP4_OK;
 }
 
@@ -990,8 +966,8 @@ int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, c
   rc = make_codes_map(ctx, &map_b, b_codes, J, C, pair_mode ? PAIR_BN / 2 : BN, gemm_kind);
   if (rc != FP4_OK) return rc;
   if (reinterpret_cast<uintptr_t>(out) & 15) return FP4_ERR_ALIGN;
-  CUtensorMap map_out, map_out_half;
-  rc = make_out_maps(ctx, &map_out, &map_out_half, out, I, J, out_f32);
+  CUtensorMap map_out, map_out_aux;
+  rc = make_out_maps(ctx, &map_out, &map_out_aux, out, I, J, out_f32);
   if (rc != FP4_OK) return rc;
 
   GemmArgs args;
@@ -1025,14 +1001,14 @@ int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, c
   if (pair_mode) {
     const int max_pairs = ctx->num_sms / 2;
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
-    rc2 = fused ? launch_pair_kernel<EPI_WGRAD>(pairs, stream, map_a, map_b, map_out, map_out_half, args)
-                : launch_pair_kernel<EPI_PLAIN>(pairs, stream, map_a, map_b, map_out, map_out_half, args);
+    rc2 = fused ? launch_pair_kernel<EPI_WGRAD>(pairs, stream, map_a, map_b, map_out, map_out_aux, args)
+                : launch_pair_kernel<EPI_PLAIN>(pairs, stream, map_a, map_b, map_out, map_out_aux, args);
   } else if (gemm_kind == FP4_GEMM_F8F6F4)
-    rc2 = fused ? launch_kernel<FP4_GEMM_F8F6F4, EPI_WGRAD>(grid, stream, map_a, map_b, map_out, map_out_half, args)
-                : launch_kernel<FP4_GEMM_F8F6F4, EPI_PLAIN>(grid, stream, map_a, map_b, map_out, map_out_half, args);
+    rc2 = fused ? launch_kernel<FP4_GEMM_F8F6F4, EPI_WGRAD>(grid, stream, map_a, map_b, map_out, map_out_aux, args)
+                : launch_kernel<FP4_GEMM_F8F6F4, EPI_PLAIN>(grid, stream, map_a, map_b, map_out, map_out_aux, args);
   else
-    rc2 = fused ? launch_kernel<FP4_GEMM_MXF4, EPI_WGRAD>(grid, stream, map_a, map_b, map_out, map_out_half, args)
-                : launch_kernel<FP4_GEMM_MXF4, EPI_PLAIN>(grid, stream, map_a, map_b, map_out, map_out_half, args);
+    rc2 = fused ? launch_kernel<FP4_GEMM_MXF4, EPI_WGRAD>(grid, stream, map_a, map_b, map_out, map_out_aux, args)
+                : launch_kernel<FP4_GEMM_MXF4, EPI_PLAIN>(grid, stream, map_a, map_b, map_out, map_out_aux, args);
   if (rc2 != FP4_OK) return rc2;
   FP4_CUDA_TRY(cudaGetLastError());
   return FP4_OK;
