@@ -173,11 +173,21 @@ int fp4_linear_bwd(fp4_ctx* ctx, void* stream, const void* dY_bf16, const void* 
 /*
  * fp4_linear_step_host -- one forward + backward of the layer with HOST buffers (pinned memory
  * recommended): copies A, W, dY to the device, runs fp4_linear_fwd and fp4_linear_bwd with
- * BF16 outputs, and copies Y, dA, dW back, all on `stream`.  It is the same path as the two
- * calls above (Fig. 2, Eq. 3, Eq. 6); only the staging is added.  Device staging and the saved
- * quantised operands live in the context's workspace: fp4_step_host_workspace_bytes() gives
- * the size needed.  `status_host` (host int32, may be NULL) receives the device status word;
- * reading it makes the call wait for the stream.  All six tensor pointers are HOST pointers.
+ * BF16 outputs, and copies Y, dA, dW back.  It is the same path as the two calls above (Fig. 2,
+ * Eq. 3, Eq. 6); only the staging is added.  Device staging and the saved quantised operands
+ * live in the context's workspace: fp4_step_host_workspace_bytes() gives the size needed.
+ * Ordering: the outputs are complete once the work this call enqueues on `stream` is.  The host
+ * inputs must be ready when the call is made (the copies to the device need not wait for work
+ * enqueued on `stream` earlier).  With a workspace of at least
+ * fp4_step_host_workspace_bytes() for the call's shape the three phases run on streams of the
+ * context (copies in, kernels, copies back) over two sets of device buffers, so that the inputs
+ * of call i + 1 travel and its kernels run while call i copies back; the host buffers of a
+ * call must stay untouched until its work on `stream` is complete, as with any asynchronous
+ * copy.  A smaller workspace that still holds one set of everything is accepted and runs the
+ * call on `stream` alone; fp4_set_overlap(ctx, 0) does the same.  Calls on one context must be
+ * issued from one thread and on one stream (or streams ordered by the caller).
+ * `status_host` (host int32, may be NULL) receives the device status word; reading it makes the
+ * call wait for the stream.  All six tensor pointers are HOST pointers.
  */
 size_t fp4_step_host_workspace_bytes(int64_t M, int64_t K, int64_t N, double alpha);
 int fp4_linear_step_host(fp4_ctx* ctx, void* stream, const void* A_host, const void* W_host,

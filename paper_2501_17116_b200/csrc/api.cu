@@ -94,6 +94,11 @@ int fp4_create(fp4_ctx** out, int device, size_t workspace_bytes) {
   ctx->records = new (std::nothrow) std::vector<ProfRecord>();
   for (auto& s : ctx->side) s = nullptr;
   for (auto& e : ctx->ev) e = nullptr;
+  ctx->copy_stream = ctx->compute_stream = ctx->return_stream = nullptr;
+  for (auto& e : ctx->host_step_done) e = nullptr;
+  for (auto& e : ctx->host_step_copied) e = nullptr;
+  for (auto& e : ctx->host_step_computed) e = nullptr;
+  ctx->host_step_parity = 0;
   cudaDeviceProp prop;
   if (!ctx->records || cudaGetDeviceProperties(&prop, device) != cudaSuccess) {
     delete ctx->records;
@@ -121,6 +126,12 @@ int fp4_create(fp4_ctx** out, int device, size_t workspace_bytes) {
   bool ok = true;
   for (auto& s : ctx->side) ok = ok && cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) == cudaSuccess;
   for (auto& e : ctx->ev) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&ctx->compute_stream, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&ctx->return_stream, cudaStreamNonBlocking) == cudaSuccess;
+  for (auto& e : ctx->host_step_computed) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
+  for (auto& e : ctx->host_step_done) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
+  for (auto& e : ctx->host_step_copied) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
   if (!ok) {
     fp4_destroy(ctx);
     return FP4_ERR_CUDA;
@@ -135,6 +146,15 @@ int fp4_destroy(fp4_ctx* ctx) {
   for (auto& s : ctx->side)
     if (s) cudaStreamDestroy(s);
   for (auto& e : ctx->ev)
+    if (e) cudaEventDestroy(e);
+  if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+  if (ctx->compute_stream) cudaStreamDestroy(ctx->compute_stream);
+  if (ctx->return_stream) cudaStreamDestroy(ctx->return_stream);
+  for (auto& e : ctx->host_step_computed)
+    if (e) cudaEventDestroy(e);
+  for (auto& e : ctx->host_step_done)
+    if (e) cudaEventDestroy(e);
+  for (auto& e : ctx->host_step_copied)
     if (e) cudaEventDestroy(e);
   if (ctx->workspace) cudaFree(ctx->workspace);
   if (ctx->records) {
@@ -390,20 +410,30 @@ int64_t step_capacity(int64_t M, int64_t K, double alpha) {
   return alpha < 1.0 ? 2 * llround((1.0 - alpha) * double(M * K)) : 0;
 }
 
+// fp4_linear_step_host: bytes of one set of device inputs (the outputs have the same three sizes),
+// and of everything else it carves.
+size_t step_host_io_bytes(int64_t M, int64_t K, int64_t N) {
+  return round256(size_t(M) * K * 2) + round256(size_t(K) * N * 2) + round256(size_t(M) * N * 2);
+}
+size_t step_host_shared_bytes(int64_t M, int64_t K, int64_t N, double alpha) {
+  const size_t cap = size_t(step_capacity(M, K, alpha));
+  size_t b = 2 * round256(size_t(M) * K / 2) + 2 * round256(size_t(K) * N / 2);                          // codes
+  b += round256(size_t(M) * 4) + round256(size_t(N) * 4);                                                // amax
+  b += 4 * round256(cap * 4) + round256((size_t(M) + 1) * 4) + round256((size_t(K) + 1) * 4) + 3 * 256;   // sparse
+  b += 256;                                                                                              // status
+  return b + fp4_workspace_bytes(M, K, N);
+}
+
 }  // namespace
 
 extern "C" {
 
 size_t fp4_step_host_workspace_bytes(int64_t M, int64_t K, int64_t N, double alpha) {
   if (M <= 0 || K <= 0 || N <= 0) return 0;
-  const size_t cap = size_t(step_capacity(M, K, alpha));
-  size_t b = 0;
-  b += 2 * (round256(size_t(M) * K * 2) + round256(size_t(K) * N * 2) + round256(size_t(M) * N * 2));  // in + out
-  b += 2 * round256(size_t(M) * K / 2) + 2 * round256(size_t(K) * N / 2);                                // codes
-  b += round256(size_t(M) * 4) + round256(size_t(N) * 4);                                                // amax
-  b += 4 * round256(cap * 4) + round256((size_t(M) + 1) * 4) + round256((size_t(K) + 1) * 4) + 3 * 256;   // sparse
-  b += 256;                                                                                              // status
-  return b + fp4_workspace_bytes(M, K, N);
+  // Sized so that the pipelined layout fits: four slots (two input sets, two output sets) of an
+  // eighth each, everything else in the second half.
+  const size_t io = step_host_io_bytes(M, K, N), shared = step_host_shared_bytes(M, K, N, alpha);
+  return (8 * io > 2 * shared ? 8 * io : 2 * shared) + 1024;
 }
 
 int fp4_linear_step_host(fp4_ctx* ctx, void* stream, const void* A_host, const void* W_host, const void* dY_host,
@@ -416,40 +446,83 @@ int fp4_linear_step_host(fp4_ctx* ctx, void* stream, const void* A_host, const v
   if (gemm_kind != FP4_GEMM_MXF4 && gemm_kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;
   if (dge_on && !(dge_k > 1.0f && dge_clip > 0.0f)) return FP4_ERR_ARG;
   if (alpha < 1.0 && step_capacity(M, K, alpha) >= M * K) return FP4_ERR_ALPHA;
-  if (fp4_step_host_workspace_bytes(M, K, N, alpha) > ctx->workspace_bytes) return FP4_ERR_WORKSPACE;
+  const size_t io_bytes = step_host_io_bytes(M, K, N), shared_bytes = step_host_shared_bytes(M, K, N, alpha);
+  if (2 * io_bytes + shared_bytes > ctx->workspace_bytes) return FP4_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-  Arena arena(ctx->workspace, ctx->workspace_bytes);
+  // Workspace layout.  Pipelined: four slots of an eighth of the workspace each -- input sets 0, 1
+  // and output sets 0, 1 -- and everything else (saved operands, scratch) in the second half.
+  // Call i uses set i % 2: its inputs travel on the context's copy stream while call i - 1 still
+  // computes, its kernels run on the context's compute stream while call i - 1 copies back on the
+  // context's return stream, and `stream` waits for the copies back.  A call whose tensors do not
+  // fit that layout carves the whole workspace from its start, runs on `stream` alone and is
+  // ordered after everything earlier calls left in flight.
+  const size_t slot = (ctx->workspace_bytes / 8) & ~size_t(255);
+  const bool pipelined = ctx->overlap && io_bytes <= slot && shared_bytes <= ctx->workspace_bytes - 4 * slot;
+  const int set = ctx->host_step_parity;
+  Arena in_arena = pipelined ? Arena(ctx->workspace + size_t(set) * slot, slot) : Arena(ctx->workspace, io_bytes);
+  Arena out_arena = pipelined ? Arena(ctx->workspace + size_t(2 + set) * slot, slot)
+                              : Arena(ctx->workspace + io_bytes, io_bytes);
+  Arena arena = pipelined ? Arena(ctx->workspace + 4 * slot, ctx->workspace_bytes - 4 * slot)
+                          : Arena(ctx->workspace + 2 * io_bytes, ctx->workspace_bytes - 2 * io_bytes);
   const size_t a_bytes = size_t(M) * K * 2, w_bytes = size_t(K) * N * 2, y_bytes = size_t(M) * N * 2;
-  char* dA_in = arena.take<char>(a_bytes);
-  char* dW_in = arena.take<char>(w_bytes);
-  char* dG_in = arena.take<char>(y_bytes);
-  char* dY_out = arena.take<char>(y_bytes);
-  char* dA_out = arena.take<char>(a_bytes);
-  char* dW_out = arena.take<char>(w_bytes);
+  char* dA_in = in_arena.take<char>(a_bytes);
+  char* dW_in = in_arena.take<char>(w_bytes);
+  char* dG_in = in_arena.take<char>(y_bytes);
+  char* dY_out = out_arena.take<char>(y_bytes);
+  char* dA_out = out_arena.take<char>(a_bytes);
+  char* dW_out = out_arena.take<char>(w_bytes);
   int32_t* status = arena.take<int32_t>(1);
   fp4_qtensor qa, qw;
   carve_qtensor(arena, &qa, M, K, 0, step_capacity(M, K, alpha));
   carve_qtensor(arena, &qw, K, N, 1, 0);
-  if (!arena.ok) return FP4_ERR_WORKSPACE;
+  if (!arena.ok || !in_arena.ok || !out_arena.ok) return FP4_ERR_WORKSPACE;
   Arena rest(arena.base + arena.off, arena.size - arena.off);
 
-  FP4_CUDA_TRY(cudaMemsetAsync(status, 0, 4, st));
-  FP4_CUDA_TRY(cudaMemcpyAsync(dA_in, A_host, a_bytes, cudaMemcpyHostToDevice, st));
-  FP4_CUDA_TRY(cudaMemcpyAsync(dW_in, W_host, w_bytes, cudaMemcpyHostToDevice, st));
-  FP4_CUDA_TRY(cudaMemcpyAsync(dG_in, dY_host, y_bytes, cudaMemcpyHostToDevice, st));
-  int rc = linear_fwd_impl(ctx, st, rest, dA_in, dW_in, M, K, N, alpha, 0, gemm_kind, dY_out, 0, &qa, &qw, status);
+  cudaStream_t s_in = st, s_cmp = st, s_out = st;      // copies in, kernels, copies back
+  if (pipelined) {
+    s_in = ctx->copy_stream;
+    s_cmp = ctx->compute_stream;
+    s_out = ctx->return_stream;
+    // The copies in do not wait for `stream`: it carries the previous call's copies back, which
+    // they are meant to overlap.  The host inputs must therefore be ready when the call is made.
+    // both slots of this set were last used by the call before the previous one
+    FP4_CUDA_TRY(cudaStreamWaitEvent(s_in, ctx->host_step_done[set], 0));
+  } else {
+    FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->host_step_done[0], 0));
+    FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->host_step_done[1], 0));
+  }
+  FP4_CUDA_TRY(cudaMemcpyAsync(dA_in, A_host, a_bytes, cudaMemcpyHostToDevice, s_in));
+  FP4_CUDA_TRY(cudaMemcpyAsync(dW_in, W_host, w_bytes, cudaMemcpyHostToDevice, s_in));
+  FP4_CUDA_TRY(cudaMemcpyAsync(dG_in, dY_host, y_bytes, cudaMemcpyHostToDevice, s_in));
+  if (pipelined) {
+    FP4_CUDA_TRY(cudaEventRecord(ctx->host_step_copied[set], s_in));
+    FP4_CUDA_TRY(cudaStreamWaitEvent(s_cmp, ctx->host_step_copied[set], 0));
+  }
+  FP4_CUDA_TRY(cudaMemsetAsync(status, 0, 4, s_cmp));
+  int rc = linear_fwd_impl(ctx, s_cmp, rest, dA_in, dW_in, M, K, N, alpha, 0, gemm_kind, dY_out, 0, &qa, &qw, status);
   if (rc != FP4_OK) return rc;
-  rc = linear_bwd_impl(ctx, st, rest, dG_in, dW_in, &qa, &qw, M, K, N, dge_on, dge_k, dge_clip, gemm_kind, dA_out,
+  rc = linear_bwd_impl(ctx, s_cmp, rest, dG_in, dW_in, &qa, &qw, M, K, N, dge_on, dge_k, dge_clip, gemm_kind, dA_out,
                        dW_out, 0, status);
   if (rc != FP4_OK) return rc;
-  FP4_CUDA_TRY(cudaMemcpyAsync(Y_host, dY_out, y_bytes, cudaMemcpyDeviceToHost, st));
-  FP4_CUDA_TRY(cudaMemcpyAsync(dA_host, dA_out, a_bytes, cudaMemcpyDeviceToHost, st));
-  FP4_CUDA_TRY(cudaMemcpyAsync(dW_host, dW_out, w_bytes, cudaMemcpyDeviceToHost, st));
-  if (status_host) {
-    FP4_CUDA_TRY(cudaMemcpyAsync(status_host, status, 4, cudaMemcpyDeviceToHost, st));
-    FP4_CUDA_TRY(cudaStreamSynchronize(st));
+  if (pipelined) {
+    FP4_CUDA_TRY(cudaEventRecord(ctx->host_step_computed[set], s_cmp));
+    FP4_CUDA_TRY(cudaStreamWaitEvent(s_out, ctx->host_step_computed[set], 0));
   }
+  FP4_CUDA_TRY(cudaMemcpyAsync(Y_host, dY_out, y_bytes, cudaMemcpyDeviceToHost, s_out));
+  FP4_CUDA_TRY(cudaMemcpyAsync(dA_host, dA_out, a_bytes, cudaMemcpyDeviceToHost, s_out));
+  FP4_CUDA_TRY(cudaMemcpyAsync(dW_host, dW_out, w_bytes, cudaMemcpyDeviceToHost, s_out));
+  if (status_host) FP4_CUDA_TRY(cudaMemcpyAsync(status_host, status, 4, cudaMemcpyDeviceToHost, s_out));
+  if (pipelined) {
+    FP4_CUDA_TRY(cudaEventRecord(ctx->host_step_done[set], s_out));
+    FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->host_step_done[set], 0));
+    ctx->host_step_parity ^= 1;
+  } else {
+    // later pipelined calls may use either set only after this call has left the workspace
+    FP4_CUDA_TRY(cudaEventRecord(ctx->host_step_done[0], st));
+    FP4_CUDA_TRY(cudaEventRecord(ctx->host_step_done[1], st));
+  }
+  if (status_host) FP4_CUDA_TRY(cudaStreamSynchronize(st));
   return FP4_OK;
 }
 

@@ -36,6 +36,14 @@ struct fp4_ctx {
   void*    encode_tiled;       // cuTensorMapEncodeTiled, fetched through the runtime
   cudaStream_t side[2];        // side streams for independent kernel chains inside one call
   cudaEvent_t  ev[8];          // fork / join events of those chains
+  // fp4_linear_step_host, pipelined over consecutive calls:
+  cudaStream_t copy_stream;          // host-to-device copies of a call's inputs
+  cudaStream_t compute_stream;       // its kernels
+  cudaStream_t return_stream;        // device-to-host copies of its outputs
+  cudaEvent_t  host_step_copied[2];  // the inputs of set i have arrived
+  cudaEvent_t  host_step_computed[2];// the outputs of set i are complete on the device
+  cudaEvent_t  host_step_done[2];    // the call that used set i has left the workspace
+  int      host_step_parity;         // set of the next pipelined call
   int      overlap;            // run independent kernel chains on the side streams (default on)
   int      gemm_pairs;         // MXF4 GEMM on pairs of CTAs (tcgen05 cta_group::2)
   int      profile;            // record CUDA events around every kernel class

@@ -1,0 +1,93 @@
+"""GPU tests of fp4_linear_step_host: the host-buffer entry point gives the results of the
+device-resident calls, also when consecutive calls of different shapes are pipelined."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import fp4_oracle as O
+from paper_2501_17116_b200 import workloads as WL
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = [(256, 256, 384), (128, 512, 128), (384, 128, 640), (256, 256, 384), (128, 128, 128)]
+ALPHA = 0.99
+
+
+def _host(bits):
+    return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+
+
+def _inputs(i, M, K, N):
+    a, w, g = WL.small_case(M, K, N, seed=100 + i)
+    return _host(a), _host(w), _host(g)
+
+
+def _device_reference(lib, M, K, N, hA, hW, hG):
+    ctx = lib.Context.for_shape(M, K, N)
+    Y, sa, sw = lib.fp4_linear_fwd(ctx, hA.cuda(), hW.cuda(), ALPHA, out_f32=False)
+    dA, dW = lib.fp4_linear_bwd(ctx, hG.cuda(), hW.cuda(), sa, sw, out_f32=False)
+    torch.cuda.synchronize()
+    assert ctx.read_status() == 0
+    out = (Y.cpu(), dA.cpu(), dW.cpu())
+    ctx.close()
+    return out
+
+
+@pytest.mark.parametrize("workspace", ["pipelined", "minimal"])
+def test_sequence_of_calls_matches_device_path(lib, workspace):
+    """Five calls back to back without waiting in between: every call's outputs are bit-identical to
+    the device-resident forward + backward of the same inputs (both paths run the same kernels)."""
+    cases = [(s, _inputs(i, *s)) for i, s in enumerate(SHAPES)]
+    need = max(int(lib.load_library().fp4_step_host_workspace_bytes(M, K, N, ALPHA)) for (M, K, N), _ in cases)
+    if workspace == "minimal":
+        need = need * 3 // 4 + 4096       # holds one set of everything for every shape, not always the four slots
+    ctx = lib.Context(0, need)
+    outs = []
+    for (M, K, N), (hA, hW, hG) in cases:
+        hY = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+        hdA = torch.empty((M, K), dtype=torch.bfloat16).pin_memory()
+        hdW = torch.empty((K, N), dtype=torch.bfloat16).pin_memory()
+        lib.fp4_linear_step_host(ctx, hA, hW, hG, ALPHA, hY, hdA, hdW, read_status=False)
+        outs.append((hY, hdA, hdW))
+    torch.cuda.synchronize()
+    for ((M, K, N), (hA, hW, hG)), got in zip(cases, outs):
+        want = _device_reference(lib, M, K, N, hA, hW, hG)
+        for g, w, name in zip(got, want, ("Y", "dA", "dW")):
+            assert torch.equal(g.view(torch.int16), w.view(torch.int16)), (M, K, N, name)
+    ctx.close()
+
+
+def test_status_word_and_oracle(lib):
+    """One call with the status read back, against the oracle's forward output."""
+    M, K, N = 256, 256, 384
+    a, w, g = WL.small_case(M, K, N, seed=7)
+    hA, hW, hG = _host(a), _host(w), _host(g)
+    ctx = lib.Context(0, int(lib.load_library().fp4_step_host_workspace_bytes(M, K, N, ALPHA)))
+    hY = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+    hdA = torch.empty((M, K), dtype=torch.bfloat16).pin_memory()
+    hdW = torch.empty((K, N), dtype=torch.bfloat16).pin_memory()
+    assert lib.fp4_linear_step_host(ctx, hA, hW, hG, ALPHA, hY, hdA, hdW) == 0
+    fwd = O.linear_fwd(a, w, ALPHA)
+    bwd = O.linear_bwd(g, w, fwd)
+    got = hY.float().numpy().astype(np.float64)
+    want = O.f64_to_bf16_f64(fwd.y)
+    # the stored value is the BF16 rounding of the oracle value, or a neighbour near a rounding boundary
+    assert (np.abs(got - fwd.y) <= np.abs(want - fwd.y) + 1e-3 * (np.abs(fwd.y_fp4) + np.abs(fwd.y_comp))).all()
+    assert (got == want).mean() > 0.99
+    assert (hdA.float().numpy().astype(np.float64) == O.f64_to_bf16_f64(bwd.da)).mean() > 0.99
+    assert (hdW.float().numpy().astype(np.float64) == O.f64_to_bf16_f64(bwd.dw)).mean() > 0.99
+    ctx.close()
+
+
+def test_workspace_too_small_is_refused(lib):
+    M, K, N = 256, 256, 384
+    a, w, g = WL.small_case(M, K, N, seed=7)
+    hA, hW, hG = _host(a), _host(w), _host(g)
+    ctx = lib.Context(0, 1 << 16)
+    hY = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+    hdA = torch.empty((M, K), dtype=torch.bfloat16).pin_memory()
+    hdW = torch.empty((K, N), dtype=torch.bfloat16).pin_memory()
+    with pytest.raises(lib.Fp4Error) as e:
+        lib.fp4_linear_step_host(ctx, hA, hW, hG, ALPHA, hY, hdA, hdW)
+    assert e.value.code == -5
+    ctx.close()
