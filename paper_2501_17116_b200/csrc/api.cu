@@ -87,6 +87,7 @@ int fp4_create(fp4_ctx** out, int device, size_t workspace_bytes) {
   ctx->workspace = nullptr;
   ctx->workspace_bytes = 0;
   ctx->encode_tiled = nullptr;
+  ctx->occ_hist = nullptr;
   ctx->profile = 0;
   ctx->overlap = 1;
   ctx->gemm_pairs = 0;
@@ -124,6 +125,9 @@ int fp4_create(fp4_ctx** out, int device, size_t workspace_bytes) {
     ctx->workspace_bytes = workspace_bytes;
   }
   bool ok = true;
+  // counters of the quantile selection (quantisation with clamping): cleared here, once
+  ok = ok && cudaMalloc(reinterpret_cast<void**>(&ctx->occ_hist), quantize_persistent_bytes()) == cudaSuccess;
+  ok = ok && cudaMemset(ctx->occ_hist, 0, quantize_persistent_bytes()) == cudaSuccess;
   for (auto& s : ctx->side) ok = ok && cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) == cudaSuccess;
   for (auto& e : ctx->ev) ok = ok && cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
@@ -157,6 +161,7 @@ int fp4_destroy(fp4_ctx* ctx) {
   for (auto& e : ctx->host_step_copied)
     if (e) cudaEventDestroy(e);
   if (ctx->workspace) cudaFree(ctx->workspace);
+  if (ctx->occ_hist) cudaFree(ctx->occ_hist);
   if (ctx->records) {
     fp4_profile_reset(ctx);
     delete ctx->records;
@@ -239,8 +244,9 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
   if (!arena.ok) return FP4_ERR_WORKSPACE;
   int rc;
 
-  // Three independent chains: W (side stream 0), A up to its codes (caller's stream), and the
-  // mask -> CSR / CSC stage of A (side stream 1), which only the compensation and the backward need.
+  // Independent chains: W (side stream 0), A up to its codes (caller's stream), and the
+  // mask -> CSR and mask -> CSC stages of A (side streams 1 and 0), which only the compensation
+  // and the backward need.
   const bool ov = ctx->overlap != 0;
   if (!reuse_w) {
     cudaStream_t s0 = ov ? ctx->side[0] : st;
@@ -259,11 +265,11 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
     Arena a(scratch_a, quantize_scratch_bytes(M, K));
     savedA->rows = M;
     savedA->cols = K;
-    const SparseOverlap so = {ctx->side[1], ctx->ev[2], ctx->ev[3]};
+    // CSR on side stream 1, CSC on side stream 0 (behind W's short chain, which has ended by then)
+    const SparseOverlap so = {ctx->side[1], ctx->ev[2], ctx->ev[3], ctx->side[0], ctx->ev[7]};
     rc = launch_quantize(ctx, st, a, A_bf16, M, K, /*scale_axis=*/0, alpha, nullptr, 0, savedA, status,
                          occ && ov ? &so : nullptr);
     if (rc != FP4_OK) return rc;
-    if (occ && ov) FP4_CUDA_TRY(cudaEventRecord(ctx->ev[4], ctx->side[1]));  // CSR and CSC complete
   }
   if (!reuse_w && ov) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[1], 0));
   // Y1 = (Q(A_c) Q(W)) * d_A[m] * d_W[n]: A codes [M x K/2], W codes transposed [N x K/2].
@@ -278,7 +284,7 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
   if (!reuse_a && ov) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[3], 0));
   rc = launch_comp_fwd(ctx, st, y1, savedA->csr_rowptr, savedA->csr_col, savedA->csr_val, W_bf16, M, K, N, Y, out_f32);
   if (rc != FP4_OK) return rc;
-  if (!reuse_a && ov) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[4], 0));  // savedA is complete on return
+  if (!reuse_a && ov) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[7], 0));  // the CSC too: savedA is complete on return
   return FP4_OK;
 }
 

@@ -34,6 +34,7 @@ struct fp4_ctx {
   char*    workspace;
   size_t   workspace_bytes;
   void*    encode_tiled;       // cuTensorMapEncodeTiled, fetched through the runtime
+  uint32_t* occ_hist;          // quantile selection: two sets of global counters, parity, ticket
   cudaStream_t side[2];        // side streams for independent kernel chains inside one call
   cudaEvent_t  ev[8];          // fork / join events of those chains
   // fp4_linear_step_host, pipelined over consecutive calls:
@@ -134,18 +135,22 @@ int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, c
                     void* out, int out_f32, int gemm_kind, int32_t* status,
                     const GemmEpilogue* epilogue = nullptr);
 
-// Lets the mask -> CSR / CSC stage of a clamping quantisation run on a side stream: it starts
-// after `encoded` (recorded on the main stream), `csr_done` is recorded on the side stream once
-// the CSR is complete.  The caller joins the side stream (the CSC follows the CSR on it).
+// Lets the mask -> CSR / CSC stage of a clamping quantisation run beside the caller's stream: both
+// chains start after `encoded` (recorded on the main stream); the CSR chain runs on `stream` and
+// records `csr_done` there; the CSC chain runs on `stream_csc` and records `csc_done` there (null:
+// it follows the CSR on `stream`).  The caller joins the streams.
 struct SparseOverlap {
   cudaStream_t stream;
   cudaEvent_t encoded;
   cudaEvent_t csr_done;
+  cudaStream_t stream_csc;
+  cudaEvent_t csc_done;
 };
 
 // Quantiser pieces (quantize.cu)
 // `prescale_is_amax`: the prescale vector holds amax values and stands for amax / 6.
 size_t quantize_scratch_bytes(int64_t rows, int64_t cols);
+size_t quantize_persistent_bytes();
 int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void* x_bf16, int64_t rows,
                     int64_t cols, int scale_axis, double alpha, const float* prescale,
                     int prescale_is_amax, fp4_qtensor* out, int32_t* status,

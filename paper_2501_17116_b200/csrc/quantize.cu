@@ -3,9 +3,9 @@
 //
 // Passes over a [rows x cols] BF16 tensor:
 //   with outlier clamping (activations)
-//     1. hist_rowminmax   one read: 65536-bin histogram of the BF16 bit patterns (exact, in shared
-//                         memory) + signed max / min of every row
-//     2. select           cumulative counts -> the two order statistics lo, hi (bit exact)
+//     1. hist_select      one read: 65536-bin histogram of the BF16 bit patterns (exact, in shared
+//                         memory) + signed max / min of every row; the block that finishes last
+//     2.                  turns the cumulative counts into the two order statistics lo, hi
 //     3. encode           one read: clamp, per-row scale from the clamped row extremes, Q, both
 //                         nibble layouts, a 1-bit-per-element mask of the clamped entries, and
 //                         the number of clamped entries per row and per (64-row strip, column)
@@ -24,7 +24,6 @@ constexpr int HIST_THREADS = 1024;
 constexpr int ENC_TM = 64;                        // tile rows of the encoder (= one strip)
 constexpr int ENC_TK = 256;                       // tile columns
 constexpr int ENC_THREADS = 256;
-constexpr int SELECT_BLOCKS = 64;                 // 64 x 1024 histogram positions
 
 enum Mode { MODE_ROWS = 0, MODE_COLS = 1, MODE_DUAL = 2 };
 
@@ -39,30 +38,8 @@ __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w 
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
 // ------------------------------------------------------------------------------------------
-// 1. histogram of bit patterns + row extremes
+// 1. + 2. histogram of bit patterns, row extremes, order statistics -- one kernel
 // ------------------------------------------------------------------------------------------
-__global__ void init_row_extremes_kernel(int* row_max, int* row_min, int rows) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < rows) {
-    row_max[i] = INT_MIN;
-    row_min[i] = INT_MAX;
-  }
-}
-
-// Everything the clamping path accumulates into starts from its identity.
-__global__ void init_occ_kernel(uint32_t* hist, int* row_max, int* row_min, int* row_cnt, int rows,
-                                unsigned* ticket) {
-  const int stride = gridDim.x * blockDim.x;
-  const int t = blockIdx.x * blockDim.x + threadIdx.x;
-  for (int i = t; i < 65536; i += stride) hist[i] = 0;
-  for (int i = t; i < rows; i += stride) {
-    row_max[i] = INT_MIN;
-    row_min[i] = INT_MAX;
-    row_cnt[i] = 0;
-  }
-  if (t == 0) *ticket = 0;
-}
-
 // Exact histogram with 32-bit shared-memory counters over a window of HIST_EXPS binary exponents
 // (both signs, all 128 mantissas): real tensors spread over far fewer exponents than BF16 offers.
 // Each block places its window just above the largest magnitude of its first 8192 elements.
@@ -70,97 +47,25 @@ __global__ void init_occ_kernel(uint32_t* hist, int* row_max, int* row_min, int*
 // exact zeros are counted in registers, so every element is counted exactly once.  The window is
 // replicated HIST_COPIES times (one copy per group of warps) to thin out same-address conflicts;
 // the increments return no value and need no overflow handling.
+//
+// A block owns whole rows (a contiguous range of them), so the signed max / min of a row are
+// reduced in shared memory and written with plain stores, as is the zero that starts the row's
+// count of clamped entries: nothing the kernel writes per row needs initialising.
+//
+// Every count also goes into one of 32 coarse counters (2048 consecutive positions of the
+// ascending real order each).  The block that finishes last (a ticket, no waiting) finds the
+// coarse range of each of the two ranks and reads only those 2048 fine counters: lo and hi.
+// The context keeps two sets of counters and a device-side parity: a call counts into set p,
+// clears set 1 - p at its start (every block a slice, plain stores) and flips the parity at its
+// end, so the set a call counts into is always zero and no separate clearing pass exists.  With
+// `parity` null (the allocation-free entry point, which clears its one set itself) set 0 is used.
 constexpr int HIST_EXPS = 24;
 constexpr int HIST_BINS = HIST_EXPS * 128 * 2;     // 6144 counters per copy
 constexpr int HIST_COPIES = 8;
 constexpr int HIST_SMEM_BYTES = HIST_BINS * HIST_COPIES * 4;
-
-__global__ void __launch_bounds__(HIST_THREADS, 1)
-hist_rowminmax_kernel(const uint4* __restrict__ x, long long n_vec_ll, int vec_per_row, uint32_t* __restrict__ ghist,
-                      int* __restrict__ row_max, int* __restrict__ row_min) {
-  extern __shared__ uint32_t h[];
-  __shared__ uint32_t s_top;
-  for (int i = threadIdx.x; i < HIST_BINS * HIST_COPIES; i += HIST_THREADS) h[i] = 0;
-  if (threadIdx.x == 0) s_top = 0;
-  __syncthreads();
-  const int n_vec = int(n_vec_ll);                 // rows * cols < 2^31
-  const int stride = gridDim.x * HIST_THREADS;
-  int i = blockIdx.x * HIST_THREADS + threadIdx.x;
-  uint4 nxt = make_uint4(0, 0, 0, 0);
-  if (i < n_vec) nxt = __ldg(&x[i]);
-  {
-    // window top: largest exponent-and-mantissa field among this block's first vectors
-    const uint32_t w[4] = {nxt.x, nxt.y, nxt.z, nxt.w};
-    uint32_t m = 0;
-#pragma unroll
-    for (int q = 0; q < 4; ++q) m = max(m, max(w[q] & 0x7FFFu, (w[q] >> 16) & 0x7FFFu));
-    m = __reduce_max_sync(0xFFFFFFFFu, m);
-    if ((threadIdx.x & 31) == 0) atomicMax(&s_top, m);
-  }
-  __syncthreads();
-  // window = exponents [e_top - HIST_EXPS + 1, e_top] with e_top four binades above the sample's maximum
-  const int e_top = min(254, int(s_top >> 7) + 4);
-  const uint32_t base = uint32_t(max(0, e_top - HIST_EXPS + 1)) << 7;
-  uint32_t* my_h = h + ((threadIdx.x >> 5) & (HIST_COPIES - 1)) * HIST_BINS;
-  uint32_t zeros_pos = 0, zeros_neg = 0;
-  // row of vector i, advanced incrementally (one division per thread)
-  int row = i / vec_per_row, rem = i - row * vec_per_row;
-  const int row_step = stride / vec_per_row, rem_step = stride - row_step * vec_per_row;
-  for (; i < n_vec; i += stride) {
-    const uint4 v = nxt;
-    if (i + stride < n_vec) nxt = __ldg(&x[i + stride]);
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int q = 0; q < 8; ++q) {
-      const uint32_t bits = (q & 1) ? (w[q >> 1] >> 16) : (w[q >> 1] & 0xFFFFu);
-      const uint32_t m15 = bits & 0x7FFFu;
-      const uint32_t off = m15 - base;
-      if (off < uint32_t(HIST_EXPS * 128)) {
-        atomicAdd(&my_h[2 * off + (bits >> 15)], 1u);
-      } else if (m15 == 0) {
-        if (bits) ++zeros_neg; else ++zeros_pos;
-      } else {
-        atomicAdd(&ghist[bits], 1u);
-      }
-    }
-    const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(w);
-    const __nv_bfloat162 mx = __hmax2(__hmax2(p[0], p[1]), __hmax2(p[2], p[3]));
-    const __nv_bfloat162 mn = __hmin2(__hmin2(p[0], p[1]), __hmin2(p[2], p[3]));
-    int kmax = float_to_ordered(fmaxf(__low2float(mx), __high2float(mx)));
-    int kmin = float_to_ordered(fminf(__low2float(mn), __high2float(mn)));
-    // 16 consecutive vectors (128 elements) never straddle a row: cols is a multiple of 128
-    const unsigned group = (threadIdx.x & 16) ? 0xFFFF0000u : 0x0000FFFFu;
-    kmax = __reduce_max_sync(group, kmax);
-    kmin = __reduce_min_sync(group, kmin);
-    if ((threadIdx.x & 15) == 0) {
-      atomicMax(&row_max[row], kmax);
-      atomicMin(&row_min[row], kmin);
-    }
-    row += row_step;
-    rem += rem_step;
-    if (rem >= vec_per_row) { rem -= vec_per_row; ++row; }
-  }
-  zeros_pos = __reduce_add_sync(0xFFFFFFFFu, zeros_pos);
-  zeros_neg = __reduce_add_sync(0xFFFFFFFFu, zeros_neg);
-  if ((threadIdx.x & 31) == 0) {
-    if (zeros_pos) atomicAdd(&ghist[0x0000], zeros_pos);
-    if (zeros_neg) atomicAdd(&ghist[0x8000], zeros_neg);
-  }
-  __syncthreads();
-  for (int idx = threadIdx.x; idx < HIST_BINS; idx += HIST_THREADS) {
-    uint32_t c = 0;
-#pragma unroll
-    for (int r = 0; r < HIST_COPIES; ++r) c += h[r * HIST_BINS + idx];
-    if (c) atomicAdd(&ghist[(uint32_t(idx & 1) << 15) | (base + uint32_t(idx >> 1))], c);
-  }
-}
-
-// ------------------------------------------------------------------------------------------
-// 2. order statistics from the histogram
-// ------------------------------------------------------------------------------------------
-// Position p in ascending real order: p < 32768 are the negative patterns from 0xFFFF down to
-// 0x8000 (-0), p >= 32768 the non-negative patterns from 0x0000 up.
-__device__ __forceinline__ uint32_t pos_to_bits(int p) { return p < 32768 ? uint32_t(0xFFFF - p) : uint32_t(p - 32768); }
+constexpr int HIST_ROW_SLOTS = 512;                // rows whose extremes a block reduces at a time
+constexpr int HIST_COARSE = 32;                    // coarse counters: 2048 positions each
+constexpr int HIST_SET_WORDS = 65536 + HIST_COARSE; // one set: fine counters, then coarse counters
 
 // Inclusive scan of one value per thread over a block of 1024 threads.
 __device__ __forceinline__ long long block_scan_1024(long long v, long long* warp_tot /*[32] shared*/) {
@@ -186,54 +91,201 @@ __device__ __forceinline__ long long block_scan_1024(long long v, long long* war
   return v;
 }
 
-// 64 blocks sum 1024 positions each; the block that finishes last (a ticket, no waiting) locates
-// the two ranks among the segment sums and then inside their segments.
-__global__ void __launch_bounds__(1024, 1)
-select_thresholds_kernel(const uint32_t* __restrict__ ghist, long long n, long long n_tail, float* thresholds,
-                         unsigned long long* seg_sum, unsigned* ticket) {
-  __shared__ long long warp_tot[32];
-  __shared__ long long s_before[2];
-  __shared__ int s_seg[2];
+// Position p in ascending real order: p < 32768 are the negative patterns from 0xFFFF down to
+// 0x8000 (-0), p >= 32768 the non-negative patterns from 0x0000 up.
+__device__ __forceinline__ uint32_t pos_to_bits(int p) { return p < 32768 ? uint32_t(0xFFFF - p) : uint32_t(p - 32768); }
+__device__ __forceinline__ int bits_to_pos(uint32_t bits) { return (bits & 0x8000u) ? int(0xFFFFu - bits) : int(bits) + 32768; }
+
+__global__ void __launch_bounds__(HIST_THREADS, 1)
+hist_select_kernel(const uint4* __restrict__ x, int rows, int vec_per_row, uint32_t* sets, unsigned* parity,
+                   int* __restrict__ row_max, int* __restrict__ row_min, int* __restrict__ row_cnt, long long n,
+                   long long n_tail, float* __restrict__ thresholds, unsigned* ticket) {
+  extern __shared__ uint32_t h[];
+  __shared__ uint32_t s_top;
+  __shared__ int s_rmax[HIST_ROW_SLOTS], s_rmin[HIST_ROW_SLOTS];
+  __shared__ uint32_t s_coarse[HIST_COARSE];
   __shared__ int s_last;
-  const int t = threadIdx.x;
-  const long long c = ghist[pos_to_bits(blockIdx.x * 1024 + t)];
-  const long long incl = block_scan_1024(c, warp_tot);
-  if (t == 1023) {
-    seg_sum[blockIdx.x] = (unsigned long long)incl;
-    __threadfence();
-    s_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
+  const int tid = threadIdx.x;
+  const unsigned par = parity ? (*reinterpret_cast<volatile unsigned*>(parity) & 1u) : 0u;
+  uint32_t* ghist = sets + size_t(par) * HIST_SET_WORDS;
+  uint32_t* gcoarse = ghist + 65536;
+  if (parity) {
+    // this block's slice of the other set, for the next call
+    uint32_t* other = sets + size_t(par ^ 1u) * HIST_SET_WORDS;
+    const int per = (HIST_SET_WORDS + gridDim.x - 1) / gridDim.x;
+    const int w0 = blockIdx.x * per, w1 = min(HIST_SET_WORDS, w0 + per);
+    for (int i = w0 + tid; i < w1; i += HIST_THREADS) other[i] = 0;
   }
+  {
+    uint4* h4 = reinterpret_cast<uint4*>(h);
+    for (int i = tid; i < HIST_BINS * HIST_COPIES / 4; i += HIST_THREADS) h4[i] = make_uint4(0, 0, 0, 0);
+  }
+  if (tid < HIST_COARSE) s_coarse[tid] = 0;
+  if (tid == 0) s_top = 0;
+  __syncthreads();
+  const int r_begin = int((long long)rows * blockIdx.x / gridDim.x);
+  const int r_end = int((long long)rows * (blockIdx.x + 1) / gridDim.x);
+  const long long v_end_all = (long long)r_end * vec_per_row;
+  {
+    // window top: largest exponent-and-mantissa field among this block's first vectors
+    const long long i0 = (long long)r_begin * vec_per_row + tid;
+    uint32_t m = 0;
+    if (i0 < v_end_all) {
+      const uint4 v = __ldg(&x[i0]);
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int q = 0; q < 4; ++q) m = max(m, max(w[q] & 0x7FFFu, (w[q] >> 16) & 0x7FFFu));
+    }
+    m = __reduce_max_sync(0xFFFFFFFFu, m);
+    if ((tid & 31) == 0) atomicMax(&s_top, m);
+  }
+  __syncthreads();
+  // window = exponents [e_top - HIST_EXPS + 1, e_top] with e_top four binades above the sample's maximum
+  const int e_top = min(254, int(s_top >> 7) + 4);
+  const uint32_t base = uint32_t(max(0, e_top - HIST_EXPS + 1)) << 7;
+  uint32_t* my_h = h + ((tid >> 5) & (HIST_COPIES - 1)) * HIST_BINS;
+  uint32_t zeros_pos = 0, zeros_neg = 0;
+  for (int r0 = r_begin; r0 < r_end; r0 += HIST_ROW_SLOTS) {
+    const int r1 = min(r_end, r0 + HIST_ROW_SLOTS);
+    for (int r = tid; r < r1 - r0; r += HIST_THREADS) {
+      s_rmax[r] = INT_MIN;
+      s_rmin[r] = INT_MAX;
+    }
+    __syncthreads();
+    const long long v_end = (long long)r1 * vec_per_row;
+    long long i = (long long)r0 * vec_per_row + tid;
+    // row of vector i relative to r0, advanced incrementally (one division per thread and batch)
+    int row = tid / vec_per_row, rem = tid - row * vec_per_row;
+    const int row_step = HIST_THREADS / vec_per_row, rem_step = HIST_THREADS - row_step * vec_per_row;
+    uint4 nxt = make_uint4(0, 0, 0, 0);
+    if (i < v_end) nxt = __ldg(&x[i]);
+    for (; i < v_end; i += HIST_THREADS) {
+      const uint4 v = nxt;
+      if (i + HIST_THREADS < v_end) nxt = __ldg(&x[i + HIST_THREADS]);
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        const uint32_t bits = (q & 1) ? (w[q >> 1] >> 16) : (w[q >> 1] & 0xFFFFu);
+        const uint32_t m15 = bits & 0x7FFFu;
+        const uint32_t off = m15 - base;
+        if (off < uint32_t(HIST_EXPS * 128)) {
+          atomicAdd(&my_h[2 * off + (bits >> 15)], 1u);
+        } else if (m15 == 0) {
+          if (bits) ++zeros_neg; else ++zeros_pos;
+        } else {
+          atomicAdd(&ghist[bits], 1u);
+          atomicAdd(&s_coarse[bits_to_pos(bits) >> 11], 1u);
+        }
+      }
+      const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(w);
+      const __nv_bfloat162 mx = __hmax2(__hmax2(p[0], p[1]), __hmax2(p[2], p[3]));
+      const __nv_bfloat162 mn = __hmin2(__hmin2(p[0], p[1]), __hmin2(p[2], p[3]));
+      int kmax = float_to_ordered(fmaxf(__low2float(mx), __high2float(mx)));
+      int kmin = float_to_ordered(fminf(__low2float(mn), __high2float(mn)));
+      // 16 consecutive vectors (128 elements) never straddle a row: cols is a multiple of 128
+      const unsigned group = (tid & 16) ? 0xFFFF0000u : 0x0000FFFFu;
+      kmax = __reduce_max_sync(group, kmax);
+      kmin = __reduce_min_sync(group, kmin);
+      if ((tid & 15) == 0) {
+        atomicMax(&s_rmax[row], kmax);
+        atomicMin(&s_rmin[row], kmin);
+      }
+      row += row_step;
+      rem += rem_step;
+      if (rem >= vec_per_row) { rem -= vec_per_row; ++row; }
+    }
+    __syncthreads();
+    for (int r = tid; r < r1 - r0; r += HIST_THREADS) {
+      row_max[r0 + r] = s_rmax[r];
+      row_min[r0 + r] = s_rmin[r];
+      if (row_cnt) row_cnt[r0 + r] = 0;
+    }
+    __syncthreads();
+  }
+  zeros_pos = __reduce_add_sync(0xFFFFFFFFu, zeros_pos);
+  zeros_neg = __reduce_add_sync(0xFFFFFFFFu, zeros_neg);
+  if ((tid & 31) == 0) {
+    if (zeros_pos) { atomicAdd(&ghist[0x0000], zeros_pos); atomicAdd(&s_coarse[bits_to_pos(0x0000u) >> 11], zeros_pos); }
+    if (zeros_neg) { atomicAdd(&ghist[0x8000], zeros_neg); atomicAdd(&s_coarse[bits_to_pos(0x8000u) >> 11], zeros_neg); }
+  }
+  for (int idx = tid; idx < HIST_BINS; idx += HIST_THREADS) {
+    uint32_t c = 0;
+#pragma unroll
+    for (int r = 0; r < HIST_COPIES; ++r) c += h[r * HIST_BINS + idx];
+    if (c) {
+      const uint32_t bits = (uint32_t(idx & 1) << 15) | (base + uint32_t(idx >> 1));
+      atomicAdd(&ghist[bits], c);
+      atomicAdd(&s_coarse[bits_to_pos(bits) >> 11], c);
+    }
+  }
+  __syncthreads();
+  if (tid < HIST_COARSE && s_coarse[tid]) atomicAdd(&gcoarse[tid], s_coarse[tid]);
+  // ---- the last block to get here selects -------------------------------------------------
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  const long long rank[2] = {n_tail, n - 1 - n_tail};
-  __shared__ long long s_sum[SELECT_BLOCKS];
-  if (t < int(gridDim.x)) s_sum[t] = (long long)reinterpret_cast<volatile unsigned long long*>(seg_sum)[t];
-  __syncthreads();
-  if (t == 0) {
-    long long run = 0;
-    int q = 0;
-    for (int sgm = 0; sgm < int(gridDim.x) && q < 2; ++sgm) {
-      const long long sz = s_sum[sgm];
-      while (q < 2 && rank[q] < run + sz) {
-        s_seg[q] = sgm;
-        s_before[q] = run;
-        ++q;
+  if (tid < 64) {
+    // warp q finds rank q: the coarse range first (one counter per lane), then the range's 2048
+    // fine counters in 16 steps of 128 consecutive positions (4 per lane, all loads issued at once)
+    const int q = tid >> 5, lane = tid & 31;
+    const long long rank = q == 0 ? n_tail : n - 1 - n_tail;
+    const long long cc = __ldcg(&gcoarse[lane]);
+    long long sc = cc;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const long long up = __shfl_up_sync(0xFFFFFFFFu, sc, off);
+      if (lane >= off) sc += up;
+    }
+    const unsigned holds = __ballot_sync(0xFFFFFFFFu, rank >= sc - cc && rank < sc);   // exactly one lane
+    const int region = __ffs(holds) - 1;
+    long long run = __shfl_sync(0xFFFFFFFFu, sc - cc, region);                          // counts before the range
+    // positions of the range in ascending order; in memory they ascend (region >= 16) or descend
+    const bool desc = region < 16;
+    const uint32_t* first = ghist + (desc ? (0xFFFF - 2048 * region - 2047) : 2048 * (region - 16));
+    bool done = false;
+#pragma unroll 1
+    for (int half = 0; half < 2; ++half) {              // eight steps' loads in flight at a time
+      uint4 c[8];
+#pragma unroll
+      for (int s8 = 0; s8 < 8; ++s8) {
+        // step st covers positions 128 st .. 128 st + 127 of the range; lane l its positions 4 l .. 4 l + 3
+        const int st = 8 * half + s8;
+        const int word = desc ? (2048 - 128 * st - 4 * lane - 4) : (128 * st + 4 * lane);
+        c[s8] = __ldcg(reinterpret_cast<const uint4*>(first + word));
       }
-      run += sz;
+#pragma unroll
+      for (int s8 = 0; s8 < 8; ++s8) {
+        const int st = 8 * half + s8;
+        // in ascending position order
+        const long long v0 = desc ? c[s8].w : c[s8].x, v1 = desc ? c[s8].z : c[s8].y;
+        const long long v2 = desc ? c[s8].y : c[s8].z, v3 = desc ? c[s8].x : c[s8].w;
+        const long long mine = v0 + v1 + v2 + v3;
+        long long incl = mine;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const long long up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+          if (lane >= off) incl += up;
+        }
+        const long long before = run + incl - mine;
+        if (!done && rank >= before && rank < before + mine) {
+          const int p0 = 2048 * region + 128 * st + 4 * lane;
+          const int k = rank < before + v0 ? 0 : (rank < before + v0 + v1 ? 1 : (rank < before + v0 + v1 + v2 ? 2 : 3));
+          const uint32_t bits = pos_to_bits(p0 + k);
+          thresholds[q] = __uint_as_float((bits == 0x8000u ? 0u : bits) << 16);   // thresholds are real numbers: -0 is +0
+        }
+        const long long total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+        done = done || rank < run + total;
+        run += total;
+      }
     }
   }
   __syncthreads();
-  for (int q = 0; q < 2; ++q) {
-    const int p = s_seg[q] * 1024 + t;
-    const long long cq = ghist[pos_to_bits(p)];
-    __syncthreads();                                  // warp_tot is reused
-    const long long iq = s_before[q] + block_scan_1024(cq, warp_tot);
-    if (rank[q] >= iq - cq && rank[q] < iq) {         // exactly one thread
-      uint32_t bits = pos_to_bits(p);
-      if (bits == 0x8000u) bits = 0;                  // thresholds are real numbers: -0 is +0
-      thresholds[q] = __uint_as_float(bits << 16);
-    }
+  if (tid == 0) {
+    if (parity) *parity = par ^ 1u;
+    *ticket = 0;
   }
 }
 
@@ -672,7 +724,6 @@ csc_fill_kernel(const uint32_t* __restrict__ mask, const __nv_bfloat16* __restri
 size_t r256(size_t b) { return (b + 255) & ~size_t(255); }
 
 struct Scratch {
-  uint32_t* hist;
   int* row_max;
   int* row_min;
   uint32_t* amax_rows;
@@ -684,14 +735,11 @@ struct Scratch {
   int* strip_off;
   float* pre_rows;
   float* pre_cols;
-  unsigned long long* seg_sum;
-  unsigned* ticket;
   bool ok;
 };
 
 Scratch carve(Arena& arena, int rows, int cols, bool occ) {
   Scratch s = {};
-  s.hist = arena.take<uint32_t>(65536);
   s.row_max = arena.take<int>(rows);
   s.row_min = arena.take<int>(rows);
   s.amax_rows = arena.take<uint32_t>(rows);
@@ -700,8 +748,6 @@ Scratch carve(Arena& arena, int rows, int cols, bool occ) {
   s.col_cnt = arena.take<int>(cols);
   s.pre_rows = arena.take<float>(rows);
   s.pre_cols = arena.take<float>(cols);
-  s.seg_sum = arena.take<unsigned long long>(SELECT_BLOCKS);
-  s.ticket = arena.take<unsigned>(1);
   if (occ) {
     s.mask = arena.take<uint8_t>(size_t(rows) * cols / 8);
     s.strip_cnt = arena.take<uint8_t>(size_t(rows / ENC_TM) * cols);
@@ -713,11 +759,12 @@ Scratch carve(Arena& arena, int rows, int cols, bool occ) {
 
 }  // namespace
 
+// Counters of the quantile selection that live as long as the context: two sets, parity, ticket.
+size_t quantize_persistent_bytes() { return (2 * size_t(HIST_SET_WORDS) + 64) * 4; }
+
 size_t quantize_scratch_bytes(int64_t rows, int64_t cols) {
   size_t b = 0;
-  b += r256(65536 * 4);                                          // histogram
   b += 5 * r256(size_t(rows) * 4) + 4 * r256(size_t(cols) * 4);   // per-row / per-column vectors
-  b += r256(SELECT_BLOCKS * 8) + 256;                            // segment sums, ticket
   b += r256(size_t(rows) * size_t(cols) / 8);                    // outlier mask
   b += r256(size_t(rows / ENC_TM) * size_t(cols));               // per-strip column counts (bytes)
   b += r256(size_t(rows / ENC_TM) * size_t(cols) * 4);           // per-strip column offsets
@@ -756,16 +803,17 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
     const long long n_tail = llround((1.0 - alpha) * double(n));
     const long long n_vec = n / 8;
     {
-      KernelScope scope(ctx, stream, KC_SELECT, 3);
-      init_occ_kernel<<<64, 1024, 0, stream>>>(sc.hist, sc.row_max, sc.row_min, sc.row_cnt, rows, sc.ticket);
-      FP4_CUDA_TRY(cudaFuncSetAttribute(hist_rowminmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+      // The two sets of global counters, their parity and the ticket belong to the context: the
+      // kernel keeps the set it is about to use zero (see there), so nothing is cleared here.
+      KernelScope scope(ctx, stream, KC_SELECT, 1);
+      FP4_CUDA_TRY(cudaFuncSetAttribute(hist_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         HIST_SMEM_BYTES));
       long long blocks = (n_vec + HIST_THREADS - 1) / HIST_THREADS;
       if (blocks > ctx->num_sms) blocks = ctx->num_sms;
-      hist_rowminmax_kernel<<<int(blocks), HIST_THREADS, HIST_SMEM_BYTES, stream>>>(x, n_vec, cols / 8, sc.hist,
-                                                                                  sc.row_max, sc.row_min);
-      select_thresholds_kernel<<<SELECT_BLOCKS, 1024, 0, stream>>>(sc.hist, n, n_tail, out->thresholds, sc.seg_sum,
-                                                                   sc.ticket);
+      unsigned* parity = reinterpret_cast<unsigned*>(ctx->occ_hist + 2 * HIST_SET_WORDS);
+      hist_select_kernel<<<int(blocks), HIST_THREADS, HIST_SMEM_BYTES, stream>>>(
+          x, rows, cols / 8, ctx->occ_hist, parity, sc.row_max, sc.row_min, sc.row_cnt, n, n_tail, out->thresholds,
+          parity + 1);
     }
     {
       KernelScope scope(ctx, stream, KC_ENCODE, 1);
@@ -777,19 +825,32 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
       FP4_CUDA_TRY(cudaEventRecord(overlap->encoded, stream));
       FP4_CUDA_TRY(cudaStreamWaitEvent(sp, overlap->encoded, 0));
     }
-    KernelScope scope(ctx, sp, KC_SPARSE, 5);
+    // The CSC chain takes a stream of its own where the caller offers one: it shares only the
+    // mask and the counts with the CSR chain.
+    cudaStream_t sc2 = sp;
+    if (sp != stream && overlap->stream_csc) {
+      sc2 = overlap->stream_csc;
+      FP4_CUDA_TRY(cudaStreamWaitEvent(sc2, overlap->encoded, 0));
+    }
     const uint32_t* mask32 = reinterpret_cast<const uint32_t*>(sc.mask);
     const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x_bf16);
     const int strips = rows / ENC_TM;
-    scan_counts_kernel<<<1, 1024, 0, sp>>>(sc.row_cnt, rows, out->csr_rowptr, out->nnz, out->sparse_cap, status);
-    csr_fill_kernel<<<(rows + 7) / 8, 256, 0, sp>>>(mask32, xb, rows, cols, out->thresholds, out->csr_rowptr,
-                                                    out->sparse_cap, out->csr_col, out->csr_val);
+    {
+      KernelScope scope(ctx, sp, KC_SPARSE, 2);
+      scan_counts_kernel<<<1, 1024, 0, sp>>>(sc.row_cnt, rows, out->csr_rowptr, out->nnz, out->sparse_cap, status);
+      csr_fill_kernel<<<(rows + 7) / 8, 256, 0, sp>>>(mask32, xb, rows, cols, out->thresholds, out->csr_rowptr,
+                                                      out->sparse_cap, out->csr_col, out->csr_val);
+    }
     if (sp != stream) FP4_CUDA_TRY(cudaEventRecord(overlap->csr_done, sp));
-    csc_strip_prefix_kernel<<<(cols + 255) / 256, 256, 0, sp>>>(sc.strip_cnt, cols, strips, sc.strip_off, sc.col_cnt);
-    scan_counts_kernel<<<1, 1024, 0, sp>>>(sc.col_cnt, cols, out->csc_colptr, nullptr, out->sparse_cap, nullptr);
-    const dim3 cgrid((cols / 32 + 7) / 8, strips);
-    csc_fill_kernel<<<cgrid, 256, 0, sp>>>(mask32, xb, rows, cols, out->thresholds, out->csc_colptr, sc.strip_off,
-                                           out->sparse_cap, out->csc_row, out->csc_val);
+    {
+      KernelScope scope(ctx, sc2, KC_SPARSE, 3);
+      csc_strip_prefix_kernel<<<(cols + 255) / 256, 256, 0, sc2>>>(sc.strip_cnt, cols, strips, sc.strip_off, sc.col_cnt);
+      scan_counts_kernel<<<1, 1024, 0, sc2>>>(sc.col_cnt, cols, out->csc_colptr, nullptr, out->sparse_cap, nullptr);
+      const dim3 cgrid((cols / 32 + 7) / 8, strips);
+      csc_fill_kernel<<<cgrid, 256, 0, sc2>>>(mask32, xb, rows, cols, out->thresholds, out->csc_colptr, sc.strip_off,
+                                              out->sparse_cap, out->csc_row, out->csc_val);
+    }
+    if (sc2 != sp) FP4_CUDA_TRY(cudaEventRecord(overlap->csc_done, sc2));
   } else {
     if (prescale && prescale_is_amax) {
       float* d = scale_axis == 0 ? sc.pre_cols : sc.pre_rows;
@@ -888,7 +949,7 @@ int launch_quantize_dual(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const 
 // library image: every GPU that loads the library holds these 769 KB until the process exits.
 namespace {
 constexpr size_t STATIC_HIST_BYTES = 65536 * sizeof(uint32_t);
-constexpr size_t STATIC_SELECT_BYTES = 1024;      // 64 segment sums (512 B) + ticket, padded
+constexpr size_t STATIC_SELECT_BYTES = 1024;      // 32 coarse counters, then (at 512) the ticket
 constexpr size_t STATIC_SCRATCH_BYTES =
     STATIC_HIST_BYTES + STATIC_SELECT_BYTES + 2 * size_t(FP4_STATIC_MAX_ROWS) * sizeof(int);
 constexpr int STATIC_MAX_DEVICES = 64;
@@ -919,29 +980,27 @@ extern "C" int fp4_quantile_thresholds_static(void* stream, const void* x_bf16, 
     FP4_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
     int sms = 0;
     FP4_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
-    FP4_CUDA_TRY(cudaFuncSetAttribute(hist_rowminmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    FP4_CUDA_TRY(cudaFuncSetAttribute(hist_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       HIST_SMEM_BYTES));
     sms_of_device[device] = sms;
     scratch_of_device[device] = ptr;
   }
   unsigned char* base = static_cast<unsigned char*>(scratch_of_device[device]);
   uint32_t* hist = reinterpret_cast<uint32_t*>(base);
-  unsigned long long* seg_sum = reinterpret_cast<unsigned long long*>(base + STATIC_HIST_BYTES);
-  unsigned* ticket = reinterpret_cast<unsigned*>(base + STATIC_HIST_BYTES + 512);
+  unsigned* ticket = reinterpret_cast<unsigned*>(base + STATIC_HIST_BYTES + 512);   // behind the coarse counters
   int* row_max = reinterpret_cast<int*>(base + STATIC_HIST_BYTES + STATIC_SELECT_BYTES);
   int* row_min = row_max + FP4_STATIC_MAX_ROWS;
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // The array keeps what the previous call left: the histogram and the ticket must start from
-  // zero and the row extremes from their identities.
+  // The array keeps what the previous call left (a call that was cut short may have left counts
+  // behind): the histogram and the ticket are cleared; the row extremes are written before read.
   FP4_CUDA_TRY(cudaMemsetAsync(base, 0, STATIC_HIST_BYTES + STATIC_SELECT_BYTES, st));
-  init_row_extremes_kernel<<<int((rows + 255) / 256), 256, 0, st>>>(row_max, row_min, int(rows));
   const long long n_vec = n / 8;
   long long blocks = (n_vec + HIST_THREADS - 1) / HIST_THREADS;
   if (blocks > sms_of_device[device]) blocks = sms_of_device[device];
-  hist_rowminmax_kernel<<<int(blocks), HIST_THREADS, HIST_SMEM_BYTES, st>>>(static_cast<const uint4*>(x_bf16), n_vec,
-                                                                          int(cols / 8), hist, row_max, row_min);
-  select_thresholds_kernel<<<SELECT_BLOCKS, 1024, 0, st>>>(hist, n, n_tail, thresholds, seg_sum, ticket);
+  hist_select_kernel<<<int(blocks), HIST_THREADS, HIST_SMEM_BYTES, st>>>(
+      static_cast<const uint4*>(x_bf16), int(rows), int(cols / 8), hist, nullptr, row_max, row_min, nullptr, n, n_tail,
+      thresholds, ticket);
   FP4_CUDA_TRY(cudaGetLastError());
   return FP4_OK;
 }

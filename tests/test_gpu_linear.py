@@ -101,6 +101,32 @@ def test_ste_switch_and_dge_parameters(lib, ctx):
         assert_close_f32(dw.cpu().numpy(), b.dw, b.s_fp4 * b.dge, b.s_comp * b.dge, f"dW dge={dge_on} k={k}")
 
 
+@pytest.mark.parametrize("M,K,N,hot,alpha", [
+    (128, 256, 128, 40, 0.92),     # 40 nearly full columns
+    (512, 256, 384, 20, 0.98),     # 20 nearly full columns of 512 entries: long columns, many rounds per warp
+    (256, 384, 128, 3, 0.999),     # few entries: short columns only
+])
+def test_weight_gradient_compensation_column_classes(lib, ctx, M, K, N, hot, alpha):
+    """The compensation of the weight gradient treats long and short residual columns differently;
+    both must give the oracle's sums, run to run identically."""
+    a_bits, w_bits, dy_bits = WL.small_case(M, K, N, seed=hot, alpha_outliers=hot)
+    f = O.linear_fwd(a_bits, w_bits, alpha)
+    b = O.linear_bwd(dy_bits, w_bits, f)
+    A, W, dY = _dev(a_bits), _dev(w_bits), _dev(dy_bits)
+    ctx.status.zero_()
+    _, sa, sw = lib.fp4_linear_fwd(ctx, A, W, alpha)
+    _, dw = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, out_f32=True, want_da=False)
+    _, dw_again = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, out_f32=True, want_da=False)
+    torch.cuda.synchronize()
+    assert ctx.read_status() == 0
+    counts = np.diff(sa.csc_colptr.cpu().numpy())
+    if hot >= 20:
+        assert (counts >= 64).sum() >= hot // 2                       # the case does reach the long-column kernel
+    assert np.abs(b.s_comp).max() > 0
+    assert_close_f32(dw.cpu().numpy(), b.dw, b.s_fp4 * b.dge, b.s_comp * b.dge, "dW")
+    assert torch.equal(dw, dw_again)                                   # fixed summation order
+
+
 def test_reuse_quantised_weight(lib, ctx):
     a_bits, w_bits, _ = WL.small_case(128, 256, 256, seed=5)
     a2_bits, _, _ = WL.small_case(128, 256, 256, seed=6)
