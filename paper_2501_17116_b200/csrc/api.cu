@@ -365,22 +365,34 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
     rc = launch_quantize(ctx, st, a, dY_bf16, M, N, /*scale_axis=*/1, 1.0, savedA->amax, 1, &g, status);
     if (rc != FP4_OK) return rc;
   }
+  // dW[k,n] = store( (d_G''[n] * sum_m Aq[m,k] G''[m,n] + comp[k,n]) * Q'(W[k,n] * 6 / amax_W[n]) ):
+  // the compensation rows and the DGE factor are applied in the GEMM's epilogue.
+  GemmEpilogue epi = {};
+  epi.addend = comp;
+  epi.slot_of_row = slot_of_col;
+  epi.w_bf16 = dge_on ? W_bf16 : nullptr;
+  epi.w_amax = savedW->amax;
+  epi.dge_k = dge_k;
+  epi.dge_clip = dge_clip;
+  // dA = d_G'[m] * sum_n G'[m,n] Wq[k,n]
+  const Fp4GemmDesc wgrad = {savedA->codes_t, g2_codes, K, N, M, nullptr, g2_amax, dW, out_f32, &epi};
+  const Fp4GemmDesc dgrad = {g1_codes, savedW->codes, M, K, N, g1_amax, nullptr, dA, out_f32, nullptr};
+  const bool pairs = gemm_kind == FP4_GEMM_MXF4 && ctx->gemm_pairs;
+  if (dA && dW && !pairs) {
+    // Both GEMMs in one launch on the caller's stream, the weight gradient's tiles first (their
+    // epilogue is the longer one and then runs under the other GEMM's MMAs).
+    if (sw != st) {
+      FP4_CUDA_TRY(cudaEventRecord(ctx->ev[7], sw));
+      FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[7], 0));
+    }
+    return launch_gemm_fp4_two(ctx, st, wgrad, dgrad, gemm_kind, status);
+  }
   if (dW) {
-    // dW[k,n] = store( (d_G''[n] * sum_m Aq[m,k] G''[m,n] + comp[k,n]) * Q'(W[k,n] * 6 / amax_W[n]) ):
-    // the compensation rows and the DGE factor are applied in the GEMM's epilogue.
-    GemmEpilogue epi = {};
-    epi.addend = comp;
-    epi.slot_of_row = slot_of_col;
-    epi.w_bf16 = dge_on ? W_bf16 : nullptr;
-    epi.w_amax = savedW->amax;
-    epi.dge_k = dge_k;
-    epi.dge_clip = dge_clip;
-    rc = launch_gemm_fp4(ctx, sw, savedA->codes_t, g2_codes, K, N, M, nullptr, g2_amax, dW, out_f32, gemm_kind, status,
-                         &epi);
+    rc = launch_gemm_fp4(ctx, sw, wgrad.a_codes, wgrad.b_codes, K, N, M, nullptr, g2_amax, dW, out_f32, gemm_kind,
+                         status, &epi);
     if (rc != FP4_OK) return rc;
   }
   if (dA) {
-    // dA = d_G'[m] * sum_n G'[m,n] Wq[k,n]
     rc = launch_gemm_fp4(ctx, st, g1_codes, savedW->codes, M, K, N, g1_amax, nullptr, dA, out_f32, gemm_kind, status);
     if (rc != FP4_OK) return rc;
   }

@@ -135,6 +135,21 @@ int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, c
                     void* out, int out_f32, int gemm_kind, int32_t* status,
                     const GemmEpilogue* epilogue = nullptr);
 
+// One GEMM, for launches that take two of them.
+struct Fp4GemmDesc {
+  const uint8_t* a_codes;
+  const uint8_t* b_codes;
+  int64_t I, J, C;
+  const float* row_amax;
+  const float* col_amax;
+  void* out;
+  int out_f32;
+  const GemmEpilogue* epilogue;
+};
+// Both GEMMs in one launch; the tiles of `first` are computed first.  Not available on CTA pairs.
+int launch_gemm_fp4_two(fp4_ctx* ctx, cudaStream_t stream, const Fp4GemmDesc& first, const Fp4GemmDesc& second,
+                        int gemm_kind, int32_t* status);
+
 // Lets the mask -> CSR / CSC stage of a clamping quantisation run beside the caller's stream: both
 // chains start after `encoded` (recorded on the main stream); the CSR chain runs on `stream` and
 // records `csr_done` there; the CSC chain runs on `stream_csc` and records `csc_done` there (null:

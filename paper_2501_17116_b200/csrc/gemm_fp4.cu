@@ -409,8 +409,10 @@ __device__ __forceinline__ void epilogue_tile_wgrad(const GemmArgs& args, int ro
 template <int KIND, int EPI>
 __global__ void __launch_bounds__(num_threads(EPI), 1)
 gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                 const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_out_aux,
-                const GemmArgs args) {
+                const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_out_aux,
+                const __grid_constant__ GemmArgs args, const __grid_constant__ CUtensorMap map_a2,
+                const __grid_constant__ CUtensorMap map_b2, const __grid_constant__ CUtensorMap map_out2,
+                const __grid_constant__ CUtensorMap map_out_aux2, const __grid_constant__ GemmArgs args2) {
   constexpr int NACC = 2;
   constexpr int STAGES = stages_of(KIND);
   constexpr int BN = tile_n(KIND);
@@ -434,7 +436,11 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int num_tiles = args.num_m_blocks * args.num_n_blocks;
+  // Two problems may share one launch (args2 with no tiles: one problem): the tiles of the first
+  // come first, then those of the second, so that the epilogue of one problem's last tiles runs
+  // under the MMAs of the other's first.
+  const int tiles_first = args.num_m_blocks * args.num_n_blocks;
+  const int num_tiles = tiles_first + args2.num_m_blocks * args2.num_n_blocks;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -452,6 +458,11 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out) : "memory");
+    if (args2.num_m_blocks) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a2) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b2) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out2) : "memory");
+    }
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
@@ -485,14 +496,19 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       uint32_t fills = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-        const int m_blk = t % args.num_m_blocks;
-        const int n_blk = t / args.num_m_blocks;
-        for (int kb = 0; kb < args.num_k_blocks; ++kb) {
+        const bool second = t >= tiles_first;
+        const GemmArgs& pa = second ? args2 : args;
+        const CUtensorMap* ma = second ? &map_a2 : &map_a;
+        const CUtensorMap* mb = second ? &map_b2 : &map_b;
+        const int tt = second ? t - tiles_first : t;
+        const int m_blk = tt % pa.num_m_blocks;
+        const int n_blk = tt / pa.num_m_blocks;
+        for (int kb = 0; kb < pa.num_k_blocks; ++kb) {
           ok = mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, args.status);
           if (!ok) break;
           mbar_arrive_expect_tx(&full_bar[stage], args.tx_bytes);
-          tma_load_2d(smem_a + stage * A_STAGE_BYTES, &map_a, &full_bar[stage], kb * 128, m_blk * BM);
-          tma_load_2d(smem_b + stage * B_STAGE_BYTES, &map_b, &full_bar[stage], kb * 128, n_blk * BN);
+          tma_load_2d(smem_a + stage * A_STAGE_BYTES, ma, &full_bar[stage], kb * 128, m_blk * BM);
+          tma_load_2d(smem_b + stage * B_STAGE_BYTES, mb, &full_bar[stage], kb * 128, n_blk * BN);
           ++fills;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -523,7 +539,8 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + uint32_t(acc * ACC_STRIDE);
-        for (int kb = 0; kb < args.num_k_blocks; ++kb) {
+        const int num_k_blocks = t >= tiles_first ? args2.num_k_blocks : args.num_k_blocks;
+        for (int kb = 0; kb < num_k_blocks; ++kb) {
           ok = mbar_wait(&full_bar[stage], phase, abort_flag, args.status);
           if (!ok) break;
           tc_fence_after();
@@ -569,38 +586,41 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     uint32_t acc_phase = 0;
     uint32_t tile_parity = 0;
     uint32_t store_seq = 0;
-    const OutMaps out_maps = {&map_out, &map_out_aux};
     for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
-      const int m_blk = t % args.num_m_blocks;
-      const int n_blk = t / args.num_m_blocks;
+      const bool second = t >= tiles_first;
+      const GemmArgs& pa = second ? args2 : args;
+      const OutMaps out_maps = {second ? &map_out2 : &map_out, second ? &map_out_aux2 : &map_out_aux};
+      const int tt = second ? t - tiles_first : t;
+      const int m_blk = tt % pa.num_m_blocks;
+      const int n_blk = tt / pa.num_m_blocks;
       // De-scales of this tile are fetched before the accumulators are awaited, under the MMAs.
       const int row = m_blk * BM + quarter * 32 + lane;
-      const float d_row = args.row_amax ? __fdiv_rn(__ldg(&args.row_amax[row]), 6.0f) : 1.0f;
+      const float d_row = pa.row_amax ? __fdiv_rn(__ldg(&pa.row_amax[row]), 6.0f) : 1.0f;
       float* dcol = s_dcol + tile_parity * 256;
       float* gcol = s_gcol + tile_parity * 256;
       for (int c = et; c < BN; c += 32 * EW) {
         const int col = n_blk * BN + c;
-        dcol[c] = (args.col_amax && col < args.J) ? __fdiv_rn(__ldg(&args.col_amax[col]), 6.0f) : 1.0f;
-        if (EPI == EPI_WGRAD && args.w) {
-          const float am = col < args.J ? __ldg(&args.w_amax[col]) : 0.0f;
+        dcol[c] = (pa.col_amax && col < pa.J) ? __fdiv_rn(__ldg(&pa.col_amax[col]), 6.0f) : 1.0f;
+        if (EPI == EPI_WGRAD && pa.w) {
+          const float am = col < pa.J ? __ldg(&pa.w_amax[col]) : 0.0f;
           gcol[c] = am > 0.0f ? __fdiv_rn(6.0f, am) : 0.0f;
         }
       }
       int slot = -1;
       WgradOperands op;
       if (EPI == EPI_WGRAD) {
-        if (args.slot_of_row) slot = __ldg(&args.slot_of_row[row]);
-        if (n_blk * BN + 16 * group < args.J) wgrad_fetch(op, args, row, slot, n_blk * BN + 16 * group);
+        if (pa.slot_of_row) slot = __ldg(&pa.slot_of_row[row]);
+        if (n_blk * BN + 16 * group < pa.J) wgrad_fetch(op, pa, row, slot, n_blk * BN + 16 * group);
       }
       const bool ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, args.status);
       if (epilogue_bar_any(!ok, 32 * EW)) break;   // also publishes dcol to the other warps
       tc_fence_after();
       const uint32_t t_base = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * ACC_STRIDE);
       if (EPI == EPI_WGRAD)
-        epilogue_tile_wgrad<BN, G>(args, m_blk, n_blk, t_base, d_row, dcol, gcol, slot, stage, quarter, group, lane,
+        epilogue_tile_wgrad<BN, G>(pa, m_blk, n_blk, t_base, d_row, dcol, gcol, slot, stage, quarter, group, lane,
                                    out_maps, store_seq, op);
       else
-        epilogue_tile_plain<BN, G>(args, m_blk, n_blk, t_base, d_row, dcol, stage, quarter, group, lane, out_maps,
+        epilogue_tile_plain<BN, G>(pa, m_blk, n_blk, t_base, d_row, dcol, stage, quarter, group, lane, out_maps,
                                    store_seq);
       tc_fence_before();
       __syncwarp();
@@ -937,13 +957,68 @@ int launch_pair_kernel(int pairs, cudaStream_t stream, const CUtensorMap& map_a,
   return FP4_OK;
 }
 
+struct Problem {
+  CUtensorMap map_a, map_b, map_out, map_out_aux;
+  GemmArgs args;
+  bool fused;
+};
+
 template <int KIND, int EPI>
-int launch_kernel(int grid, cudaStream_t stream, const CUtensorMap& map_a, const CUtensorMap& map_b,
-                  const CUtensorMap& map_out, const CUtensorMap& map_out_aux, const GemmArgs& args) {
+int launch_kernel(int grid, cudaStream_t stream, const Problem& p, const Problem* second = nullptr) {
   constexpr size_t kSmem = smem_bytes(KIND);
   FP4_CUDA_TRY(cudaFuncSetAttribute(gemm_fp4_kernel<KIND, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     int(kSmem)));
-  gemm_fp4_kernel<KIND, EPI><<<grid, num_threads(EPI), kSmem, stream>>>(map_a, map_b, map_out, map_out_aux, args);
+  Problem none = p;
+  none.args.num_m_blocks = none.args.num_n_blocks = 0;          // a second problem without tiles
+  const Problem& q = second ? *second : none;
+  gemm_fp4_kernel<KIND, EPI><<<grid, num_threads(EPI), kSmem, stream>>>(p.map_a, p.map_b, p.map_out, p.map_out_aux,
+                                                                        p.args, q.map_a, q.map_b, q.map_out,
+                                                                        q.map_out_aux, q.args);
+  return FP4_OK;
+}
+
+// Tensor maps and arguments of one GEMM.
+int make_problem(fp4_ctx* ctx, Problem* p, const Fp4GemmDesc& d, int gemm_kind, bool pair_mode, int32_t* status) {
+  if (gemm_kind != FP4_GEMM_MXF4 && gemm_kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;
+  // The byte-container form expands 32 bytes of a packed row into 64, so its rows must start on
+  // 32-byte boundaries (C/2 a multiple of 32 holds for every multiple of 128).
+  const uintptr_t need = gemm_kind == FP4_GEMM_F8F6F4 ? 31 : 15;
+  if ((reinterpret_cast<uintptr_t>(d.a_codes) & need) || (reinterpret_cast<uintptr_t>(d.b_codes) & need))
+    return FP4_ERR_ALIGN;
+  int rc = make_codes_map(ctx, &p->map_a, d.a_codes, d.I, d.C, BM, gemm_kind);
+  if (rc != FP4_OK) return rc;
+  const int BN = tile_n(gemm_kind);
+  rc = make_codes_map(ctx, &p->map_b, d.b_codes, d.J, d.C, pair_mode ? PAIR_BN / 2 : BN, gemm_kind);
+  if (rc != FP4_OK) return rc;
+  if (reinterpret_cast<uintptr_t>(d.out) & 15) return FP4_ERR_ALIGN;
+  rc = make_out_maps(ctx, &p->map_out, &p->map_out_aux, d.out, d.I, d.J, d.out_f32);
+  if (rc != FP4_OK) return rc;
+
+  GemmArgs& args = p->args;
+  args.I = int(d.I);
+  args.J = int(d.J);
+  const int k_per_stage = gemm_kind == FP4_GEMM_F8F6F4 ? 128 : 256;   // elements per 128-byte row
+  args.num_k_blocks = int((d.C + k_per_stage - 1) / k_per_stage);
+  args.num_m_blocks = pair_mode ? int((d.I + 255) / 256) : int(d.I / BM);
+  args.num_n_blocks = int((d.J + BN - 1) / BN);
+  // The transaction count of a copy is in bytes read from global memory: the byte-container form
+  // fills a 48 KB stage from 24 KB of packed nibbles.
+  args.tx_bytes = gemm_kind == FP4_GEMM_F8F6F4 ? stage_bytes(gemm_kind) / 2 : stage_bytes(gemm_kind);
+  args.row_amax = d.row_amax;
+  args.col_amax = d.col_amax;
+  args.out = d.out;
+  args.out_f32 = d.out_f32;
+  args.status = status;
+  const GemmEpilogue* epi = d.epilogue;
+  const bool fused = epi && (epi->addend || epi->w_bf16);
+  p->fused = fused;
+  args.addend = fused ? epi->addend : nullptr;
+  args.slot_of_row = fused && epi->addend ? epi->slot_of_row : nullptr;
+  args.w = fused ? static_cast<const uint4*>(epi->w_bf16) : nullptr;
+  args.w_amax = fused ? epi->w_amax : nullptr;
+  args.inv_k = fused && epi->w_bf16 ? 1.0f / epi->dge_k : 1.0f;
+  args.expo = args.inv_k - 1.0f;
+  args.clip = fused ? epi->dge_clip : 0.0f;
   return FP4_OK;
 }
 
@@ -952,63 +1027,47 @@ int launch_kernel(int grid, cudaStream_t stream, const CUtensorMap& map_a, const
 int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, const uint8_t* b_codes, int64_t I,
                     int64_t J, int64_t C, const float* row_amax, const float* col_amax, void* out, int out_f32,
                     int gemm_kind, int32_t* status, const GemmEpilogue* epi) {
-  if (gemm_kind != FP4_GEMM_MXF4 && gemm_kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;
-  // The byte-container form expands 32 bytes of a packed row into 64, so its rows must start on
-  // 32-byte boundaries (C/2 a multiple of 32 holds for every multiple of 128).
-  const uintptr_t need = gemm_kind == FP4_GEMM_F8F6F4 ? 31 : 15;
-  if ((reinterpret_cast<uintptr_t>(a_codes) & need) || (reinterpret_cast<uintptr_t>(b_codes) & need))
-    return FP4_ERR_ALIGN;
+  const Fp4GemmDesc d = {a_codes, b_codes, I, J, C, row_amax, col_amax, out, out_f32, epi};
   const bool pair_mode = gemm_kind == FP4_GEMM_MXF4 && ctx->gemm_pairs;
-  CUtensorMap map_a, map_b;
-  int rc = make_codes_map(ctx, &map_a, a_codes, I, C, BM, gemm_kind);
+  Problem p;
+  int rc = make_problem(ctx, &p, d, gemm_kind, pair_mode, status);
   if (rc != FP4_OK) return rc;
-  const int BN = tile_n(gemm_kind);
-  rc = make_codes_map(ctx, &map_b, b_codes, J, C, pair_mode ? PAIR_BN / 2 : BN, gemm_kind);
-  if (rc != FP4_OK) return rc;
-  if (reinterpret_cast<uintptr_t>(out) & 15) return FP4_ERR_ALIGN;
-  CUtensorMap map_out, map_out_aux;
-  rc = make_out_maps(ctx, &map_out, &map_out_aux, out, I, J, out_f32);
-  if (rc != FP4_OK) return rc;
-
-  GemmArgs args;
-  args.I = int(I);
-  args.J = int(J);
-  const int k_per_stage = gemm_kind == FP4_GEMM_F8F6F4 ? 128 : 256;   // elements per 128-byte row
-  args.num_k_blocks = int((C + k_per_stage - 1) / k_per_stage);
-  args.num_m_blocks = pair_mode ? int((I + 255) / 256) : int(I / BM);
-  args.num_n_blocks = int((J + BN - 1) / BN);
-  // The transaction count of a copy is in bytes read from global memory: the byte-container form
-  // fills a 48 KB stage from 24 KB of packed nibbles.
-  args.tx_bytes = gemm_kind == FP4_GEMM_F8F6F4 ? stage_bytes(gemm_kind) / 2 : stage_bytes(gemm_kind);
-  args.row_amax = row_amax;
-  args.col_amax = col_amax;
-  args.out = out;
-  args.out_f32 = out_f32;
-  args.status = status;
+  const GemmArgs& args = p.args;
   const int tiles = args.num_m_blocks * args.num_n_blocks;
   const int grid = tiles < ctx->num_sms ? tiles : ctx->num_sms;
-
-  const bool fused = epi && (epi->addend || epi->w_bf16);
-  args.addend = fused ? epi->addend : nullptr;
-  args.slot_of_row = fused && epi->addend ? epi->slot_of_row : nullptr;
-  args.w = fused ? static_cast<const uint4*>(epi->w_bf16) : nullptr;
-  args.w_amax = fused ? epi->w_amax : nullptr;
-  args.inv_k = fused && epi->w_bf16 ? 1.0f / epi->dge_k : 1.0f;
-  args.expo = args.inv_k - 1.0f;
-  args.clip = fused ? epi->dge_clip : 0.0f;
   KernelScope scope(ctx, stream, KC_GEMM, 1);
   int rc2;
   if (pair_mode) {
     const int max_pairs = ctx->num_sms / 2;
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
-    rc2 = fused ? launch_pair_kernel<EPI_WGRAD>(pairs, stream, map_a, map_b, map_out, map_out_aux, args)
-                : launch_pair_kernel<EPI_PLAIN>(pairs, stream, map_a, map_b, map_out, map_out_aux, args);
+    rc2 = p.fused ? launch_pair_kernel<EPI_WGRAD>(pairs, stream, p.map_a, p.map_b, p.map_out, p.map_out_aux, args)
+                  : launch_pair_kernel<EPI_PLAIN>(pairs, stream, p.map_a, p.map_b, p.map_out, p.map_out_aux, args);
   } else if (gemm_kind == FP4_GEMM_F8F6F4)
-    rc2 = fused ? launch_kernel<FP4_GEMM_F8F6F4, EPI_WGRAD>(grid, stream, map_a, map_b, map_out, map_out_aux, args)
-                : launch_kernel<FP4_GEMM_F8F6F4, EPI_PLAIN>(grid, stream, map_a, map_b, map_out, map_out_aux, args);
+    rc2 = p.fused ? launch_kernel<FP4_GEMM_F8F6F4, EPI_WGRAD>(grid, stream, p)
+                  : launch_kernel<FP4_GEMM_F8F6F4, EPI_PLAIN>(grid, stream, p);
   else
-    rc2 = fused ? launch_kernel<FP4_GEMM_MXF4, EPI_WGRAD>(grid, stream, map_a, map_b, map_out, map_out_aux, args)
-                : launch_kernel<FP4_GEMM_MXF4, EPI_PLAIN>(grid, stream, map_a, map_b, map_out, map_out_aux, args);
+    rc2 = p.fused ? launch_kernel<FP4_GEMM_MXF4, EPI_WGRAD>(grid, stream, p)
+                  : launch_kernel<FP4_GEMM_MXF4, EPI_PLAIN>(grid, stream, p);
+  if (rc2 != FP4_OK) return rc2;
+  FP4_CUDA_TRY(cudaGetLastError());
+  return FP4_OK;
+}
+
+// Two GEMMs in one launch (single-CTA kernels only): the tiles of `first` are computed first.  Both
+// run through the 16-warp epilogue; a problem without fused work simply has nothing to add.
+int launch_gemm_fp4_two(fp4_ctx* ctx, cudaStream_t stream, const Fp4GemmDesc& first, const Fp4GemmDesc& second,
+                        int gemm_kind, int32_t* status) {
+  if (gemm_kind == FP4_GEMM_MXF4 && ctx->gemm_pairs) return FP4_ERR_ARG;
+  Problem p, q;
+  int rc = make_problem(ctx, &p, first, gemm_kind, false, status);
+  if (rc != FP4_OK) return rc;
+  rc = make_problem(ctx, &q, second, gemm_kind, false, status);
+  if (rc != FP4_OK) return rc;
+  const int tiles = p.args.num_m_blocks * p.args.num_n_blocks + q.args.num_m_blocks * q.args.num_n_blocks;
+  const int grid = tiles < ctx->num_sms ? tiles : ctx->num_sms;
+  KernelScope scope(ctx, stream, KC_GEMM, 1);
+  const int rc2 = gemm_kind == FP4_GEMM_F8F6F4 ? launch_kernel<FP4_GEMM_F8F6F4, EPI_WGRAD>(grid, stream, p, &q)
+                                                : launch_kernel<FP4_GEMM_MXF4, EPI_WGRAD>(grid, stream, p, &q);
   if (rc2 != FP4_OK) return rc2;
   FP4_CUDA_TRY(cudaGetLastError());
   return FP4_OK;
