@@ -917,8 +917,10 @@ int launch_quantize_dual(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const 
   aa.d_row_out = sc.pre_rows;
   aa.amax_rows = sc.amax_rows;
   aa.amax_cols = sc.amax_cols;
-  FP4_CUDA_TRY(cudaMemsetAsync(sc.amax_rows, 0, size_t(rows) * 4, stream));
-  FP4_CUDA_TRY(cudaMemsetAsync(sc.amax_cols, 0, size_t(cols) * 4, stream));
+  // amax_rows and amax_cols are carved one behind the other: one clearing covers both
+  FP4_CUDA_TRY(cudaMemsetAsync(sc.amax_rows, 0,
+                               size_t(reinterpret_cast<char*>(sc.amax_cols + cols) - reinterpret_cast<char*>(sc.amax_rows)),
+                               stream));
   {
     KernelScope scope(ctx, stream, KC_ABSMAX, 1);
     absmax_tile_kernel<MODE_DUAL><<<tile_grid, ENC_THREADS, 0, stream>>>(aa);
