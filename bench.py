@@ -40,13 +40,13 @@ SM_COUNT, FMA_LANES = 148, 128      # plain fp32 pipe: 148 SMs x 128 FMA lanes x
 # DRAM bytes per launch of the dominant kernel from the committed ncu summaries
 # (profiles/*.md); None where no capture exists for the class.
 NCU_TRAFFIC_PER_UNIT = {
-    # profiles/gemm_fp4_llama1p3b.md: dram read + write of three consecutive launches, averaged (bytes per launch)
-    "gemm": 11.4e6,
-    "encode": 11.2e6,      # profiles/quantizer_encode_llama1p3b.md (writes still in L2 at kernel end)
-    "select": 16.8e6,      # profiles/quantizer_select_absmax_llama1p3b.md, hist_rowminmax_kernel
+    # mean DRAM read + write per launch of the class, from the captures summarised under profiles/
+    "gemm": 17.4e6,        # gemm_fp4_llama1p3b.md: forward 6.4 MB, backward (two GEMMs per launch) 28.3 MB
+    "encode": 14.0e6,      # quantizer_encode_llama1p3b.md (writes still in L2 at kernel end)
+    "select": 16.9e6,      # quantizer_select_absmax_llama1p3b.md, hist_select_kernel
     "absmax": 12.6e6,
-    "comp_fwd": 36.1e6,    # profiles/compensation_llama1p3b.md
-    "comp_wgrad_dge": 16.8e6,
+    "comp_fwd": 36.1e6,    # compensation_llama1p3b.md
+    "comp_wgrad_dge": 6.5e6,
 }
 
 
@@ -353,10 +353,10 @@ def main():
     # ------------------------------------------------------------------ CPU baseline -------
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        tf, times = oracle_sample_tflops(cfg, WL, 2, M)
+        tf, times = oracle_sample_tflops(cfg, WL, 5, M)
         lin = cfg.linears[0]
         cpu_baseline = {"value": tf / min(times), "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
-                        "sample": f"fwd+bwd of linear '{lin.name}' ({lin.K}x{lin.N}) at {M} tokens, best of 2",
+                        "sample": f"fwd+bwd of linear '{lin.name}' ({lin.K}x{lin.N}) at {M} tokens, best of 5",
                         "seconds": round(min(times), 3)}
 
     if rank == 0:
