@@ -48,7 +48,7 @@ extern "C" {
 
 /* bits of the device status word */
 #define FP4_DEV_SPARSE_OVERFLOW  1   /* more residual entries than sparse_cap                */
-#define FP4_DEV_NONFINITE        2   /* reserved: a non-finite input was seen                */
+#define FP4_DEV_NONFINITE        2   /* an input holds an infinity or a NaN: outputs unspecified */
 #define FP4_DEV_TIMEOUT          4   /* a bounded wait inside a kernel ran out               */
 
 /* gemm_kind: which tcgen05.mma flavour multiplies the E2M1 codes */

@@ -346,7 +346,7 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
   if (dA && dW) {
     Arena a = q_arena;
     rc = launch_quantize_dual(ctx, st, a, dY_bf16, M, N, savedW->amax, savedA->amax, g1_codes, g1_amax, g2_codes,
-                              g2_amax);
+                              g2_amax, status);
     if (rc != FP4_OK) return rc;
     if (sw != st) {
       FP4_CUDA_TRY(cudaEventRecord(ctx->ev[6], st));

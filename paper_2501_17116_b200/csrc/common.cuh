@@ -176,7 +176,7 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
 int launch_quantize_dual(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void* x_bf16, int64_t rows,
                          int64_t cols, const float* amax_col_pre, const float* amax_row_pre,
                          uint8_t* codes_rows, float* amax_rows_out, uint8_t* codes_t_cols,
-                         float* amax_cols_out);
+                         float* amax_cols_out, int32_t* status);
 
 // Sparse compensation and epilogues (compensate.cu)
 // y[m,:] = store( y1[m,:] + sum_{entries of row m} val * dense[col,:] )

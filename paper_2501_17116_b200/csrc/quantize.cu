@@ -99,7 +99,7 @@ __device__ __forceinline__ int bits_to_pos(uint32_t bits) { return (bits & 0x800
 __global__ void __launch_bounds__(HIST_THREADS, 1)
 hist_select_kernel(const uint4* __restrict__ x, int rows, int vec_per_row, uint32_t* sets, unsigned* parity,
                    int* __restrict__ row_max, int* __restrict__ row_min, int* __restrict__ row_cnt, long long n,
-                   long long n_tail, float* __restrict__ thresholds, unsigned* ticket) {
+                   long long n_tail, float* __restrict__ thresholds, unsigned* ticket, int32_t* status) {
   extern __shared__ uint32_t h[];
   __shared__ uint32_t s_top;
   __shared__ int s_rmax[HIST_ROW_SLOTS], s_rmin[HIST_ROW_SLOTS];
@@ -145,6 +145,7 @@ hist_select_kernel(const uint4* __restrict__ x, int rows, int vec_per_row, uint3
   const uint32_t base = uint32_t(max(0, e_top - HIST_EXPS + 1)) << 7;
   uint32_t* my_h = h + ((tid >> 5) & (HIST_COPIES - 1)) * HIST_BINS;
   uint32_t zeros_pos = 0, zeros_neg = 0;
+  bool nonfinite = false;
   for (int r0 = r_begin; r0 < r_end; r0 += HIST_ROW_SLOTS) {
     const int r1 = min(r_end, r0 + HIST_ROW_SLOTS);
     for (int r = tid; r < r1 - r0; r += HIST_THREADS) {
@@ -175,6 +176,7 @@ hist_select_kernel(const uint4* __restrict__ x, int rows, int vec_per_row, uint3
         } else {
           atomicAdd(&ghist[bits], 1u);
           atomicAdd(&s_coarse[bits_to_pos(bits) >> 11], 1u);
+          if (m15 >= 0x7F80u) nonfinite = true;         // infinity or NaN: always outside the window
         }
       }
       const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(w);
@@ -202,6 +204,7 @@ hist_select_kernel(const uint4* __restrict__ x, int rows, int vec_per_row, uint3
     }
     __syncthreads();
   }
+  if (__any_sync(0xFFFFFFFFu, nonfinite) && (tid & 31) == 0 && status) atomicOr(status, FP4_DEV_NONFINITE);
   zeros_pos = __reduce_add_sync(0xFFFFFFFFu, zeros_pos);
   zeros_neg = __reduce_add_sync(0xFFFFFFFFu, zeros_neg);
   if ((tid & 31) == 0) {
@@ -308,6 +311,7 @@ struct AbsmaxArgs {
   float* d_row_out;
   uint32_t* amax_rows;          // float bits, zero-initialised (non-negative floats order as integers)
   uint32_t* amax_cols;
+  int32_t* status;              // FP4_DEV_NONFINITE is raised when a maximum is infinite or NaN
 };
 
 // Tile of 64 rows x 256 columns per block, same thread mapping as the encoder: warp w owns rows
@@ -347,31 +351,39 @@ absmax_tile_kernel(const AbsmaxArgs a) {
   float pc[8];
 #pragma unroll
   for (int c = 0; c < 8; ++c) pc[c] = (want_rows && a.pre_col && in_cols) ? s_pcol[8 * lane + c] : 1.0f;
-  float cm[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  // maxima as unsigned bit patterns of |x|: they order like the numbers, and a NaN (which fmaxf
+  // would drop) ends up above infinity and is seen
+  uint32_t cm[8] = {0, 0, 0, 0, 0, 0, 0, 0};
 #pragma unroll
   for (int r = 0; r < 8; ++r) {
     const uint32_t w[4] = {v[r].x, v[r].y, v[r].z, v[r].w};
     const float pr = (want_cols && a.pre_row) ? s_prow[8 * warp + r] : 1.0f;
-    float rm = 0.0f;
+    uint32_t rm = 0;
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
       const float f = (c & 1) ? bf16_hi(w[c >> 1]) : bf16_lo(w[c >> 1]);
-      if (want_rows) rm = fmaxf(rm, fabsf(a.pre_col ? __fmul_rn(f, pc[c]) : f));
-      if (want_cols) cm[c] = fmaxf(cm[c], fabsf(a.pre_row ? __fmul_rn(f, pr) : f));
+      if (want_rows) rm = max(rm, __float_as_uint(fabsf(a.pre_col ? __fmul_rn(f, pc[c]) : f)));
+      if (want_cols) cm[c] = max(cm[c], __float_as_uint(fabsf(a.pre_row ? __fmul_rn(f, pr) : f)));
     }
     if (want_rows) {
-      const uint32_t g = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(rm));
-      if (lane == 0) atomicMax(&a.amax_rows[row0 + 8 * warp + r], g);
+      const uint32_t g = __reduce_max_sync(0xFFFFFFFFu, rm);
+      if (lane == 0) {
+        atomicMax(&a.amax_rows[row0 + 8 * warp + r], g);
+        if (g >= 0x7F800000u && a.status) atomicOr(a.status, FP4_DEV_NONFINITE);
+      }
     }
   }
   if (want_cols) {
 #pragma unroll
-    for (int c = 0; c < 8; ++c) s_cmax[warp][8 * lane + c] = __float_as_uint(cm[c]);
+    for (int c = 0; c < 8; ++c) s_cmax[warp][8 * lane + c] = cm[c];
     __syncthreads();
     uint32_t m = 0;
 #pragma unroll
     for (int w8 = 0; w8 < 8; ++w8) m = max(m, s_cmax[w8][tid]);
-    if (col0 + tid < a.cols) atomicMax(&a.amax_cols[col0 + tid], m);
+    if (col0 + tid < a.cols) {
+      atomicMax(&a.amax_cols[col0 + tid], m);
+      if (m >= 0x7F800000u && a.status) atomicOr(a.status, FP4_DEV_NONFINITE);
+    }
   }
 }
 
@@ -813,7 +825,7 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
       unsigned* parity = reinterpret_cast<unsigned*>(ctx->occ_hist + 2 * HIST_SET_WORDS);
       hist_select_kernel<<<int(blocks), HIST_THREADS, HIST_SMEM_BYTES, stream>>>(
           x, rows, cols / 8, ctx->occ_hist, parity, sc.row_max, sc.row_min, sc.row_cnt, n, n_tail, out->thresholds,
-          parity + 1);
+          parity + 1, status);
     }
     {
       KernelScope scope(ctx, stream, KC_ENCODE, 1);
@@ -865,6 +877,7 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
     aa.cols = cols;
     aa.amax_rows = sc.amax_rows;
     aa.amax_cols = sc.amax_cols;
+    aa.status = status;
     if (scale_axis == 0) {
       aa.pre_col = prescale;
       ea.pre_col = prescale;
@@ -901,7 +914,7 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
 // column-scaled transposed codes of dY (.) (amax_row_pre / 6).
 int launch_quantize_dual(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void* x_bf16, int64_t rows64,
                          int64_t cols64, const float* amax_col_pre, const float* amax_row_pre, uint8_t* codes_rows,
-                         float* amax_rows_out, uint8_t* codes_t_cols, float* amax_cols_out) {
+                         float* amax_rows_out, uint8_t* codes_t_cols, float* amax_cols_out, int32_t* status) {
   const int rows = int(rows64), cols = int(cols64);
   Scratch sc = carve(arena, rows, cols, false);
   if (!sc.ok) return FP4_ERR_WORKSPACE;
@@ -917,6 +930,7 @@ int launch_quantize_dual(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const 
   aa.d_row_out = sc.pre_rows;
   aa.amax_rows = sc.amax_rows;
   aa.amax_cols = sc.amax_cols;
+  aa.status = status;
   // amax_rows and amax_cols are carved one behind the other: one clearing covers both
   FP4_CUDA_TRY(cudaMemsetAsync(sc.amax_rows, 0,
                                size_t(reinterpret_cast<char*>(sc.amax_cols + cols) - reinterpret_cast<char*>(sc.amax_rows)),
@@ -1002,7 +1016,7 @@ extern "C" int fp4_quantile_thresholds_static(void* stream, const void* x_bf16, 
   if (blocks > sms_of_device[device]) blocks = sms_of_device[device];
   hist_select_kernel<<<int(blocks), HIST_THREADS, HIST_SMEM_BYTES, st>>>(
       static_cast<const uint4*>(x_bf16), int(rows), int(cols / 8), hist, nullptr, row_max, row_min, nullptr, n, n_tail,
-      thresholds, ticket);
+      thresholds, ticket, nullptr);
   FP4_CUDA_TRY(cudaGetLastError());
   return FP4_OK;
 }

@@ -194,6 +194,33 @@ def test_run_to_run_determinism(lib, ctx):
         assert torch.equal(getattr(a, name), getattr(b, name)), name
 
 
+@pytest.mark.parametrize("bad", [0x7F80, 0xFF80, 0x7FC0])          # +inf, -inf, NaN
+def test_non_finite_inputs_raise_the_status_bit(lib, ctx, bad):
+    """An infinity or a NaN anywhere in the input sets FP4_DEV_NONFINITE (outputs are then unspecified
+    but every write stays in bounds); finite inputs leave the word at zero."""
+    rng = np.random.default_rng(bad)
+    bits = WL.to_bf16_bits(rng.standard_normal((256, 384)).astype(np.float32))
+    dirty = bits.copy()
+    dirty[200, 301] = bad
+    for x, want in ((bits, 0), (dirty, lib.FP4_DEV_NONFINITE)):
+        for axis, alpha in ((0, 1.0), (1, 1.0), (0, 0.99)):
+            ctx.status.zero_()
+            lib.fp4_quantize(ctx, _dev(x), axis, alpha=alpha)
+            torch.cuda.synchronize()
+            assert ctx.read_status() & lib.FP4_DEV_NONFINITE == want, (axis, alpha)
+    # through the layer: a bad output gradient is seen by the backward's quantiser
+    a_bits, w_bits, dy_bits = WL.small_case(256, 384, 256, seed=3)
+    ctx.status.zero_()
+    _, sa, sw = lib.fp4_linear_fwd(ctx, _dev(a_bits), _dev(w_bits), 0.99)
+    torch.cuda.synchronize()
+    assert ctx.read_status() == 0
+    dy_bits = dy_bits.copy()
+    dy_bits[17, 5] = bad
+    lib.fp4_linear_bwd(ctx, _dev(dy_bits), _dev(w_bits), sa, sw)
+    torch.cuda.synchronize()
+    assert ctx.read_status() & lib.FP4_DEV_NONFINITE
+
+
 def test_host_side_argument_errors(lib, ctx):
     x = torch.zeros((128, 128), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(lib.Fp4Error) as e:
