@@ -14,12 +14,13 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 
 
 size_t round256(size_t b) { return (b + 255) & ~size_t(255); }
 
-// Bytes the backward needs on top of the quantiser scratch: both quantised copies of dY and
-// the fp32 GEMM result that the compensation / DGE epilogue kernel consumes.
+// Bytes a call needs on top of the quantiser scratch: the fp32 GEMM result the forward compensation
+// kernel consumes (the backward keeps its compact compensation rows there), both quantised copies
+// of dY, and the lists of the residual's non-empty columns.
 size_t linear_scratch_bytes(int64_t M, int64_t K, int64_t N) {
   size_t b = 0;
   const size_t big = size_t(M > K ? M : K) * size_t(N);
-  b += round256(big * sizeof(float));                 // fp32 GEMM result (fwd: M x N, wgrad: K x N)
+  b += round256(big * sizeof(float));                 // fwd: M x N result; bwd: up to K compensation rows of N
   b += 2 * round256(size_t(M) * size_t(N) / 2);       // dY codes, both scalings
   b += round256(size_t(M) * 4) + round256(size_t(N) * 4);   // their amax vectors
   b += 2 * round256(size_t(M > N ? M : N) * 4);       // de-scale vectors used as prescale

@@ -1,5 +1,5 @@
-// Outlier compensation (Section 3.2: the sparse residual times a dense high-precision matrix)
-// fused with the final store, and the DGE factor of the weight gradient (Eq. 6, Eq. 8).
+// Outlier compensation (Section 3.2: the sparse residual times a dense high-precision matrix):
+// forward fused with the final store, weight gradient (Eq. 6) as compact rows for the GEMM's epilogue.
 //
 //   forward   Y[m, :]  = store( Y1[m, :] + sum_{(m,k) in dA} dA[m,k] * W[k, :] )
 //   wgrad     C[slot(k), :] = sum_{(m,k) in dA} dA[m,k] * dY[m, :]   for the columns k that hold entries;
