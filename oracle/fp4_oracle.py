@@ -37,6 +37,14 @@ Readings of points the paper leaves open (each also listed in the design notes):
   lies along the contraction is folded into dY before dY is quantised.
   PARITY UNPINNED by the paper for this choice: it is pinned only by brute
   force and by an algebraic identity (see tests).
+* FP8 operands (the W4A8 and W8A4 settings of the ablation in Section 4.3, and the
+  reading of the backward that keeps dY in FP8): the paper names the settings, not
+  the format's details.  Reading taken: OCP E4M3 (4 exponent bits, bias 7, 3 mantissa
+  bits, no infinity, largest finite value 448), round to nearest even with saturation,
+  the sign of the input kept, vector-wise absmax scaling along the same axes as for
+  E2M1 with MAX = 448.  OCC belongs to 4-bit activations and DGE to 4-bit weights, so
+  an E4M3 activation is not clamped and an E4M3 weight gets the straight-through
+  estimator.  PARITY UNPINNED by the paper for all of this as well.
 """
 from __future__ import annotations
 
@@ -127,14 +135,51 @@ def rn32(x) -> np.ndarray:
     return np.asarray(x, dtype=np.float64).astype(np.float32).astype(np.float64)
 
 
-def absmax_scales(amax):
-    """gamma = RN32(MAX_fp4 / amax) (Eq. 1) and the de-scale d = RN32(amax / MAX_fp4)."""
+def absmax_scales(amax, fmax: float = FP4_MAX):
+    """gamma = RN32(MAX / amax) (Eq. 1) and the de-scale d = RN32(amax / MAX)."""
     a32 = np.asarray(amax, dtype=np.float32)
-    six = np.float32(FP4_MAX)
+    top = np.float32(fmax)
     with np.errstate(divide="ignore", invalid="ignore"):
-        gamma = np.where(a32 > 0, six / a32, np.float32(0)).astype(np.float32)
-        d = (a32 / six).astype(np.float32)
+        gamma = np.where(a32 > 0, top / a32, np.float32(0)).astype(np.float32)
+        d = (a32 / top).astype(np.float32)
     return gamma, d
+
+
+# --------------------------------------------------------------------------- #
+# FP8 E4M3 (Section 2 names the format; Section 4.3 the W4A8 / W8A4 settings)
+# --------------------------------------------------------------------------- #
+E4M3_MAX = 448.0
+
+
+def e4m3_decode(codes) -> np.ndarray:
+    """Value of every E4M3 byte: S.EEEE.MMM, bias 7, subnormals at E = 0, S.1111.111 is NaN."""
+    c = np.asarray(codes, dtype=np.uint8).astype(np.int64)
+    e = (c >> 3) & 0xF
+    m = (c & 7).astype(np.float64)
+    mag = np.where(e == 0, m / 8.0 * 2.0 ** -6, (1.0 + m / 8.0) * np.exp2((e - 7).astype(np.float64)))
+    mag = np.where((c & 0x7F) == 0x7F, np.nan, mag)
+    return np.where(c & 0x80, -mag, mag)
+
+
+def e4m3_quantize(v32) -> np.ndarray:
+    """Nearest E4M3 value of float32 numbers (ties to the even mantissa), saturating at 448.
+
+    Returns the codes; the sign bit is the sign of the input, also when the result is zero.
+    """
+    v = np.asarray(v32, dtype=np.float32).astype(np.float64)
+    a = np.minimum(np.abs(v), E4M3_MAX)
+    _, ex = np.frexp(a)                                  # a = m * 2**ex with m in [0.5, 1)
+    e = np.clip(ex - 1, -6, 8)                           # binade of a (subnormals share e = -6)
+    step = np.exp2((e - 3).astype(np.float64))           # spacing of the grid inside that binade
+    q = np.minimum(np.rint(a / step) * step, E4M3_MAX)   # np.rint rounds halves to even
+    _, exq = np.frexp(q)
+    eq = np.clip(exq - 1, -6, 8)
+    normal = q >= 2.0 ** -6
+    field_e = np.where(normal, eq + 7, 0).astype(np.int64)
+    field_m = np.where(normal, np.rint((q / np.exp2(eq.astype(np.float64)) - 1.0) * 8.0),
+                       np.rint(q / 2.0 ** -9)).astype(np.int64)
+    sign = np.signbit(v).astype(np.int64)
+    return ((sign << 7) | (field_e << 3) | field_m).astype(np.uint8)
 
 
 @dataclass
@@ -152,14 +197,23 @@ class Quantized:
     csr: tuple = field(default=None)   # (rowptr int32[rows+1], col int32[nnz], val float32[nnz])
     csc: tuple = field(default=None)   # (colptr int32[cols+1], row int32[nnz], val float32[nnz])
     residual: np.ndarray = None  # dense float64 [rows, cols] (zeros outside the tails)
+    fmt: str = "e2m1"            # "e2m1": one nibble code per element; "e4m3": one byte per element
+
+    @property
+    def fmax(self):
+        return FP4_MAX if self.fmt == "e2m1" else E4M3_MAX
 
     @property
     def gamma(self):
-        return absmax_scales(self.amax)[0]
+        return absmax_scales(self.amax, self.fmax)[0]
 
     @property
     def descale(self):
-        return absmax_scales(self.amax)[1]
+        return absmax_scales(self.amax, self.fmax)[1]
+
+    def values(self):
+        """The numbers the codes stand for, float64 [rows, cols]."""
+        return e2m1_decode(self.codes) if self.fmt == "e2m1" else e4m3_decode(self.codes)
 
     def packed(self):
         """[rows, cols/2] bytes, column pairs packed."""
@@ -170,7 +224,7 @@ class Quantized:
         return pack_nibbles(np.ascontiguousarray(self.codes.T))
 
 
-def absmax_quantize(x, scale_axis: int, prescale=None) -> Quantized:
+def absmax_quantize(x, scale_axis: int, prescale=None, fmt: str = "e2m1") -> Quantized:
     """Vector-wise absmax quantisation of a 2-D float64 array of BF16-exact numbers.
 
     ``scale_axis`` 0: one scale per row (token-wise, activations, Section 4.1);
@@ -178,6 +232,8 @@ def absmax_quantize(x, scale_axis: int, prescale=None) -> Quantized:
     Appendix C.2 where sf is 1 x c_o).
     ``prescale``: optional float32 vector laid along the *other* axis that
     multiplies x first, x <- RN32(x * prescale) (used for dY in the backward).
+    ``fmt``: "e2m1" (Eq. 1 with MAX = 6 and the quantiser of Appendix A) or "e4m3"
+    (MAX = 448, nearest-even rounding: the FP8 operand of the W4A8 / W8A4 settings).
     """
     x = np.asarray(x, dtype=np.float64)
     rows, cols = x.shape
@@ -186,12 +242,12 @@ def absmax_quantize(x, scale_axis: int, prescale=None) -> Quantized:
         p = p[None, :] if scale_axis == 0 else p[:, None]
         x = rn32(x * p)                     # exact double product, one rounding
     amax = np.max(np.abs(x), axis=1 - scale_axis).astype(np.float32)
-    gamma, _ = absmax_scales(amax)
+    gamma, _ = absmax_scales(amax, FP4_MAX if fmt == "e2m1" else E4M3_MAX)
     g = gamma.astype(np.float64)
     g = g[:, None] if scale_axis == 0 else g[None, :]
     scaled = (x * g).astype(np.float32)     # RN32(x * gamma): the product is exact in double
-    codes = lut_quantize(scaled)
-    return Quantized(rows, cols, scale_axis, codes, amax, scaled)
+    codes = lut_quantize(scaled) if fmt == "e2m1" else e4m3_quantize(scaled)
+    return Quantized(rows, cols, scale_axis, codes, amax, scaled, fmt=fmt)
 
 
 # --------------------------------------------------------------------------- #
@@ -273,6 +329,18 @@ def gemm_codes(codes_a, codes_b) -> np.ndarray:
     return (a2 @ b2.T) / 4.0
 
 
+def gemm_values(qa: Quantized, qb: Quantized, transpose_a: bool = False, transpose_b: bool = False) -> np.ndarray:
+    """acc[i, j] = sum_c val_a[i, c] * val_b[j, c] for operands of either format, exact.
+
+    E2M1 values are multiples of 2^-1 up to 6 and E4M3 values multiples of 2^-9 up to 448, so
+    every product is a multiple of 2^-18 below 2^18 and sums of up to 2^17 of them are exact in
+    float64.  ``transpose_*`` takes the operand's codes transposed first.
+    """
+    va = qa.values().T if transpose_a else qa.values()
+    vb = qb.values().T if transpose_b else qb.values()
+    return va @ vb.T
+
+
 # --------------------------------------------------------------------------- #
 # Differentiable gradient estimator: Eq. 7, Eq. 8
 # --------------------------------------------------------------------------- #
@@ -322,16 +390,27 @@ class Forward:
     qw: Quantized
 
 
-def linear_fwd(a_bits, w_bits, alpha: float) -> Forward:
+def linear_fwd(a_bits, w_bits, alpha: float, fmt_a: str = "e2m1", fmt_w: str = "e2m1") -> Forward:
     """Y = (Q(A_c) Q(W)) (.) scales + dA W  (Fig. 2, Section 3.2).
 
     ``a_bits`` uint16 [M, K] and ``w_bits`` uint16 [K, N] are BF16 bit patterns.
+    ``fmt_a`` / ``fmt_w`` = "e4m3" give the W4A8 / W8A4 settings of Section 4.3: an E4M3
+    activation is quantised token-wise without clamping (alpha must then be 1).
     """
     a = bf16_bits_to_f64(a_bits)
     w = bf16_bits_to_f64(w_bits)
-    qa = occ_quantize(a, alpha)                 # token-wise, with OCC
-    qw = absmax_quantize(w, 1)                  # channel-wise (per output channel)
-    acc = gemm_codes(qa.codes, qw.codes.T)      # contraction over k
+    if fmt_a == "e2m1":
+        qa = occ_quantize(a, alpha)             # token-wise, with OCC
+    else:
+        if alpha != 1.0:
+            raise ValueError("outlier clamping belongs to 4-bit activations")
+        qa = absmax_quantize(a, 0, fmt=fmt_a)
+        qa.residual = np.zeros_like(a)
+    qw = absmax_quantize(w, 1, fmt=fmt_w)       # channel-wise (per output channel)
+    if fmt_a == "e2m1" and fmt_w == "e2m1":
+        acc = gemm_codes(qa.codes, qw.codes.T)  # contraction over k
+    else:
+        acc = gemm_values(qa, qw, transpose_b=True)
     d_a = qa.descale.astype(np.float64)
     d_w = qw.descale.astype(np.float64)
     y_fp4 = (acc * d_a[:, None]) * d_w[None, :]
@@ -352,20 +431,28 @@ class Backward:
 
 
 def linear_bwd(dy_bits, w_bits, fwd: Forward, dge_on: bool = True,
-               k: float = 5.0, clip: float = 3.0) -> Backward:
-    """dL/dA = dL/dY W_q^T and dL/dW = (A^T dL/dY) (.) Q'(W_scaled) (Eq. 3, Eq. 6, App. C.2)."""
+               k: float = 5.0, clip: float = 3.0, fmt_dy: str = "e2m1") -> Backward:
+    """dL/dA = dL/dY W_q^T and dL/dW = (A^T dL/dY) (.) Q'(W_scaled) (Eq. 3, Eq. 6, App. C.2).
+
+    ``fmt_dy`` = "e4m3" keeps both quantised copies of dY in FP8.  The operands saved by the
+    forward keep the format the forward gave them.  The DGE factor belongs to 4-bit weights:
+    with an E4M3 weight the straight-through estimator is used whatever ``dge_on`` says.
+    """
     dy = bf16_bits_to_f64(dy_bits)
     qa, qw = fwd.qa, fwd.qw
     d_a, d_w = qa.descale, qw.descale
+    all_fp4 = qa.fmt == "e2m1" and qw.fmt == "e2m1" and fmt_dy == "e2m1"
     # dgrad: sum_n dY[m,n] d_W[n] val(codeW[k,n]); the W de-scale is folded into dY.
-    qg1 = absmax_quantize(dy, 0, prescale=d_w)
-    da = gemm_codes(qg1.codes, qw.codes) * qg1.descale.astype(np.float64)[:, None]
+    qg1 = absmax_quantize(dy, 0, prescale=d_w, fmt=fmt_dy)
+    acc1 = gemm_codes(qg1.codes, qw.codes) if all_fp4 else gemm_values(qg1, qw)
+    da = acc1 * qg1.descale.astype(np.float64)[:, None]
     # wgrad: sum_m d_A[m] val(codeA[m,k]) dY[m,n]; the A de-scale is folded into dY.
-    qg2 = absmax_quantize(dy, 1, prescale=d_a)
-    s_fp4 = gemm_codes(qa.codes.T, qg2.codes.T) * qg2.descale.astype(np.float64)[None, :]
+    qg2 = absmax_quantize(dy, 1, prescale=d_a, fmt=fmt_dy)
+    acc2 = gemm_codes(qa.codes.T, qg2.codes.T) if all_fp4 else gemm_values(qa, qg2, transpose_a=True, transpose_b=True)
+    s_fp4 = acc2 * qg2.descale.astype(np.float64)[None, :]
     s_comp = qa.residual.T @ dy
     s = s_fp4 + s_comp
-    if dge_on:
+    if dge_on and qw.fmt == "e2m1":
         factor = dge_fprime(qw.scaled.astype(np.float64), k, clip)
     else:
         factor = np.ones_like(s)            # straight-through estimator, f' = 1
