@@ -54,6 +54,10 @@ extern "C" {
 /* gemm_kind: which tcgen05.mma flavour multiplies the E2M1 codes */
 #define FP4_GEMM_MXF4    0   /* packed nibbles, K = 64 per instruction, unit block scales    */
 #define FP4_GEMM_F8F6F4  1   /* nibbles in byte containers, K = 32 per instruction           */
+/* fp4_gemm only: the byte-container kind with E4M3 bytes as one or both operands */
+#define FP4_GEMM_F8F6F4_A8    2   /* a_codes are E4M3 bytes [I x C], b_codes E2M1 nibbles  */
+#define FP4_GEMM_F8F6F4_B8    3   /* a_codes E2M1 nibbles, b_codes E4M3 bytes [J x C]      */
+#define FP4_GEMM_F8F6F4_A8B8  4   /* both operands E4M3 bytes                              */
 
 typedef struct fp4_ctx fp4_ctx;   /* opaque: device id, SM count, workspace */
 
@@ -126,6 +130,9 @@ int fp4_quantize(fp4_ctx* ctx, void* stream, const void* x_bf16, int64_t rows, i
  *   a_codes [I x C/2], b_codes [J x C/2]: both operands have the contraction contiguous.
  *   out     [I x J], float if out_f32 != 0 else BF16.
  *   I, J, C multiples of 128.  gemm_kind: FP4_GEMM_MXF4 or FP4_GEMM_F8F6F4.
+ * With FP4_GEMM_F8F6F4_A8 / _B8 / _A8B8 the named operands are OCP E4M3 bytes, one per element
+ * ([rows x C]), with d = amax / 448 (the mixed-precision settings W4A8 / W8A4 of Section 4.3);
+ * the accumulation is then fp32 without the exactness E2M1 products have.
  */
 int fp4_gemm(fp4_ctx* ctx, void* stream, const uint8_t* a_codes, const uint8_t* b_codes,
              int64_t I, int64_t J, int64_t C, const float* row_amax, const float* col_amax,

@@ -15,6 +15,9 @@ from .build import LIB_PATH
 
 FP4_GEMM_MXF4 = 0
 FP4_GEMM_F8F6F4 = 1
+FP4_GEMM_F8F6F4_A8 = 2
+FP4_GEMM_F8F6F4_B8 = 3
+FP4_GEMM_F8F6F4_A8B8 = 4
 FP4_DEV_SPARSE_OVERFLOW = 1
 FP4_DEV_NONFINITE = 2
 FP4_DEV_TIMEOUT = 4
@@ -221,12 +224,16 @@ def fp4_quantize(ctx: Context, x: torch.Tensor, scale_axis: int, alpha: float = 
 
 def fp4_gemm(ctx: Context, a_codes: torch.Tensor, b_codes: torch.Tensor, row_amax=None, col_amax=None,
              out_f32: bool = True, gemm_kind: int = FP4_GEMM_MXF4, out: torch.Tensor | None = None):
-    I, c2 = a_codes.shape
-    J = b_codes.shape[0]
-    assert b_codes.shape[1] == c2
+    """out = (a b^T) with the two de-scales; E2M1 operands are packed two per byte, E4M3 operands
+    (FP4_GEMM_F8F6F4_A8 / _B8 / _A8B8) one per byte."""
+    a8 = gemm_kind in (FP4_GEMM_F8F6F4_A8, FP4_GEMM_F8F6F4_A8B8)
+    b8 = gemm_kind in (FP4_GEMM_F8F6F4_B8, FP4_GEMM_F8F6F4_A8B8)
+    I, J = a_codes.shape[0], b_codes.shape[0]
+    Cc = a_codes.shape[1] * (1 if a8 else 2)
+    assert b_codes.shape[1] * (1 if b8 else 2) == Cc
     if out is None:
         out = torch.empty((I, J), dtype=torch.float32 if out_f32 else torch.bfloat16, device=a_codes.device)
-    _check(ctx.lib.fp4_gemm(ctx.handle, _stream(), _ptr(a_codes), _ptr(b_codes), I, J, 2 * c2, _ptr(row_amax),
+    _check(ctx.lib.fp4_gemm(ctx.handle, _stream(), _ptr(a_codes), _ptr(b_codes), I, J, Cc, _ptr(row_amax),
                             _ptr(col_amax), _ptr(out), int(out_f32), gemm_kind, _ptr(ctx.status)))
     return out
 

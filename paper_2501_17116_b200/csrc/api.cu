@@ -203,8 +203,12 @@ int fp4_gemm(fp4_ctx* ctx, void* stream, const uint8_t* a_codes, const uint8_t* 
   if (!ctx || !a_codes || !b_codes || !out || !status) return FP4_ERR_NULL;
   if (!mult128(I) || !mult128(J) || !mult128(C)) return FP4_ERR_SHAPE;
   if (!aligned16(out)) return FP4_ERR_ALIGN;
+  if (gemm_kind < FP4_GEMM_MXF4 || gemm_kind > FP4_GEMM_F8F6F4_A8B8) return FP4_ERR_ARG;
+  const bool a8 = gemm_kind == FP4_GEMM_F8F6F4_A8 || gemm_kind == FP4_GEMM_F8F6F4_A8B8;
+  const bool b8 = gemm_kind == FP4_GEMM_F8F6F4_B8 || gemm_kind == FP4_GEMM_F8F6F4_A8B8;
+  const int kind = gemm_kind >= FP4_GEMM_F8F6F4 ? FP4_GEMM_F8F6F4 : FP4_GEMM_MXF4;
   return launch_gemm_fp4(ctx, static_cast<cudaStream_t>(stream), a_codes, b_codes, I, J, C, row_amax, col_amax, out,
-                         out_f32, gemm_kind, status);
+                         out_f32, kind, status, nullptr, a8, b8);
 }
 
 int fp4_linear_fwd(fp4_ctx* ctx, void* stream, const void* A_bf16, const void* W_bf16, int64_t M, int64_t K,

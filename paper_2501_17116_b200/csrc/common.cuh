@@ -133,7 +133,7 @@ struct GemmEpilogue {
 int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, const uint8_t* b_codes,
                     int64_t I, int64_t J, int64_t C, const float* row_amax, const float* col_amax,
                     void* out, int out_f32, int gemm_kind, int32_t* status,
-                    const GemmEpilogue* epilogue = nullptr);
+                    const GemmEpilogue* epilogue = nullptr, bool a_e4m3 = false, bool b_e4m3 = false);
 
 // One GEMM, for launches that take two of them.
 struct Fp4GemmDesc {
@@ -145,6 +145,8 @@ struct Fp4GemmDesc {
   void* out;
   int out_f32;
   const GemmEpilogue* epilogue;
+  bool a_e4m3 = false;          // operand formats: E2M1 nibbles unless E4M3 bytes (byte-container kind only)
+  bool b_e4m3 = false;
 };
 // Both GEMMs in one launch; the tiles of `first` are computed first.  Not available on CTA pairs.
 int launch_gemm_fp4_two(fp4_ctx* ctx, cudaStream_t stream, const Fp4GemmDesc& first, const Fp4GemmDesc& second,

@@ -58,6 +58,8 @@ struct GemmArgs {
   int num_k_blocks;
   int num_m_blocks, num_n_blocks;
   uint32_t tx_bytes;
+  uint32_t idesc;              // instruction descriptor (operand formats differ per problem)
+  float row_div, col_div;      // largest value of the row / column operand's format: 6 (E2M1) or 448 (E4M3)
   const float* row_amax;
   const float* col_amax;
   void* out;
@@ -216,9 +218,10 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
   return d;
 }
 // Instruction descriptors: M = 128, N = tile_n, both operands K-major, E2M1 x E2M1 -> fp32.
-__host__ __device__ constexpr uint32_t idesc_f8f6f4() {
-  return (1u << 4) | (5u << 7) | (5u << 10) | (uint32_t(tile_n(FP4_GEMM_F8F6F4) >> 3) << 17) |
-         (uint32_t(BM >> 4) << 24);
+// kind::f8f6f4 format fields: E4M3 = 0, E2M1 = 5
+__host__ __device__ constexpr uint32_t idesc_f8f6f4(bool a_e4m3 = false, bool b_e4m3 = false) {
+  return (1u << 4) | ((a_e4m3 ? 0u : 5u) << 7) | ((b_e4m3 ? 0u : 5u) << 10) |
+         (uint32_t(tile_n(FP4_GEMM_F8F6F4) >> 3) << 17) | (uint32_t(BM >> 4) << 24);
 }
 __host__ __device__ constexpr uint32_t idesc_mxf4() {
   return (1u << 7) | (1u << 10) | (uint32_t(tile_n(FP4_GEMM_MXF4) >> 3) << 17) | (1u << 23) |
@@ -506,7 +509,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         for (int kb = 0; kb < pa.num_k_blocks; ++kb) {
           ok = mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, args.status);
           if (!ok) break;
-          mbar_arrive_expect_tx(&full_bar[stage], args.tx_bytes);
+          mbar_arrive_expect_tx(&full_bar[stage], pa.tx_bytes);
           tma_load_2d(smem_a + stage * A_STAGE_BYTES, ma, &full_bar[stage], kb * 128, m_blk * BM);
           tma_load_2d(smem_b + stage * B_STAGE_BYTES, mb, &full_bar[stage], kb * 128, n_blk * BN);
           ++fills;
@@ -533,13 +536,13 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      const uint32_t idesc = (KIND == FP4_GEMM_F8F6F4) ? idesc_f8f6f4() : idesc_mxf4();
       for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
         ok = mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, args.status);
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + uint32_t(acc * ACC_STRIDE);
         const int num_k_blocks = t >= tiles_first ? args2.num_k_blocks : args.num_k_blocks;
+        const uint32_t idesc = t >= tiles_first ? args2.idesc : args.idesc;
         for (int kb = 0; kb < num_k_blocks; ++kb) {
           ok = mbar_wait(&full_bar[stage], phase, abort_flag, args.status);
           if (!ok) break;
@@ -595,12 +598,12 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const int n_blk = tt / pa.num_m_blocks;
       // De-scales of this tile are fetched before the accumulators are awaited, under the MMAs.
       const int row = m_blk * BM + quarter * 32 + lane;
-      const float d_row = pa.row_amax ? __fdiv_rn(__ldg(&pa.row_amax[row]), 6.0f) : 1.0f;
+      const float d_row = pa.row_amax ? __fdiv_rn(__ldg(&pa.row_amax[row]), pa.row_div) : 1.0f;
       float* dcol = s_dcol + tile_parity * 256;
       float* gcol = s_gcol + tile_parity * 256;
       for (int c = et; c < BN; c += 32 * EW) {
         const int col = n_blk * BN + c;
-        dcol[c] = (pa.col_amax && col < pa.J) ? __fdiv_rn(__ldg(&pa.col_amax[col]), 6.0f) : 1.0f;
+        dcol[c] = (pa.col_amax && col < pa.J) ? __fdiv_rn(__ldg(&pa.col_amax[col]), pa.col_div) : 1.0f;
         if (EPI == EPI_WGRAD && pa.w) {
           const float am = col < pa.J ? __ldg(&pa.w_amax[col]) : 0.0f;
           gcol[c] = am > 0.0f ? __fdiv_rn(6.0f, am) : 0.0f;
@@ -900,24 +903,31 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// Tensor map over packed codes [rows x C/2 bytes] with a box of 128 bytes x box_rows.
+// Tensor map over the codes of one operand with a box of 128 bytes of shared memory x box_rows:
+// packed nibbles [rows x C/2 bytes] (E2M1) or bytes [rows x C] (E4M3, byte-container kind only).
 int make_codes_map(fp4_ctx* ctx, CUtensorMap* map, const uint8_t* codes, int64_t rows, int64_t C, int box_rows,
-                   int gemm_kind) {
+                   int gemm_kind, bool e4m3) {
   EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
   if (!encode) return FP4_ERR_CUDA;
-  const cuuint64_t strides[1] = {cuuint64_t(C / 2)};
   const cuuint32_t elem_strides[2] = {1, 1};
+  const cuuint32_t box[2] = {128, cuuint32_t(box_rows)};
   CUresult r;
-  if (gemm_kind == FP4_GEMM_F8F6F4) {
+  if (e4m3) {
+    const cuuint64_t dims[2] = {cuuint64_t(C), cuuint64_t(rows)};
+    const cuuint64_t strides[1] = {cuuint64_t(C)};
+    r = encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(codes), dims, strides, box, elem_strides,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else if (gemm_kind == FP4_GEMM_F8F6F4) {
     // global memory packed, shared memory 16 nibbles + 8 bytes of padding per 16 bytes
     const cuuint64_t dims[2] = {cuuint64_t(C), cuuint64_t(rows)};
-    const cuuint32_t box[2] = {128, cuuint32_t(box_rows)};
+    const cuuint64_t strides[1] = {cuuint64_t(C / 2)};
     r = encode(map, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, 2, const_cast<uint8_t*>(codes), dims, strides, box,
                elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   } else {
     const cuuint64_t dims[2] = {cuuint64_t(C / 2), cuuint64_t(rows)};
-    const cuuint32_t box[2] = {128, cuuint32_t(box_rows)};
+    const cuuint64_t strides[1] = {cuuint64_t(C / 2)};
     r = encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(codes), dims, strides, box, elem_strides,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -980,15 +990,16 @@ int launch_kernel(int grid, cudaStream_t stream, const Problem& p, const Problem
 // Tensor maps and arguments of one GEMM.
 int make_problem(fp4_ctx* ctx, Problem* p, const Fp4GemmDesc& d, int gemm_kind, bool pair_mode, int32_t* status) {
   if (gemm_kind != FP4_GEMM_MXF4 && gemm_kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;
+  if ((d.a_e4m3 || d.b_e4m3) && gemm_kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;   // E4M3 needs the byte-container kind
   // The byte-container form expands 32 bytes of a packed row into 64, so its rows must start on
   // 32-byte boundaries (C/2 a multiple of 32 holds for every multiple of 128).
   const uintptr_t need = gemm_kind == FP4_GEMM_F8F6F4 ? 31 : 15;
   if ((reinterpret_cast<uintptr_t>(d.a_codes) & need) || (reinterpret_cast<uintptr_t>(d.b_codes) & need))
     return FP4_ERR_ALIGN;
-  int rc = make_codes_map(ctx, &p->map_a, d.a_codes, d.I, d.C, BM, gemm_kind);
+  int rc = make_codes_map(ctx, &p->map_a, d.a_codes, d.I, d.C, BM, gemm_kind, d.a_e4m3);
   if (rc != FP4_OK) return rc;
   const int BN = tile_n(gemm_kind);
-  rc = make_codes_map(ctx, &p->map_b, d.b_codes, d.J, d.C, pair_mode ? PAIR_BN / 2 : BN, gemm_kind);
+  rc = make_codes_map(ctx, &p->map_b, d.b_codes, d.J, d.C, pair_mode ? PAIR_BN / 2 : BN, gemm_kind, d.b_e4m3);
   if (rc != FP4_OK) return rc;
   if (reinterpret_cast<uintptr_t>(d.out) & 15) return FP4_ERR_ALIGN;
   rc = make_out_maps(ctx, &p->map_out, &p->map_out_aux, d.out, d.I, d.J, d.out_f32);
@@ -1002,8 +1013,14 @@ int make_problem(fp4_ctx* ctx, Problem* p, const Fp4GemmDesc& d, int gemm_kind, 
   args.num_m_blocks = pair_mode ? int((d.I + 255) / 256) : int(d.I / BM);
   args.num_n_blocks = int((d.J + BN - 1) / BN);
   // The transaction count of a copy is in bytes read from global memory: the byte-container form
-  // fills a 48 KB stage from 24 KB of packed nibbles.
-  args.tx_bytes = gemm_kind == FP4_GEMM_F8F6F4 ? stage_bytes(gemm_kind) / 2 : stage_bytes(gemm_kind);
+  // fills a stage's 128-byte rows from 64 bytes of packed nibbles (E2M1) or from 128 bytes (E4M3).
+  if (gemm_kind == FP4_GEMM_F8F6F4)
+    args.tx_bytes = uint32_t(A_STAGE_BYTES / (d.a_e4m3 ? 1 : 2) + b_stage_bytes(gemm_kind) / (d.b_e4m3 ? 1 : 2));
+  else
+    args.tx_bytes = stage_bytes(gemm_kind);
+  args.idesc = gemm_kind == FP4_GEMM_F8F6F4 ? idesc_f8f6f4(d.a_e4m3, d.b_e4m3) : idesc_mxf4();
+  args.row_div = d.a_e4m3 ? 448.0f : 6.0f;
+  args.col_div = d.b_e4m3 ? 448.0f : 6.0f;
   args.row_amax = d.row_amax;
   args.col_amax = d.col_amax;
   args.out = d.out;
@@ -1026,8 +1043,10 @@ int make_problem(fp4_ctx* ctx, Problem* p, const Fp4GemmDesc& d, int gemm_kind, 
 
 int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, const uint8_t* b_codes, int64_t I,
                     int64_t J, int64_t C, const float* row_amax, const float* col_amax, void* out, int out_f32,
-                    int gemm_kind, int32_t* status, const GemmEpilogue* epi) {
-  const Fp4GemmDesc d = {a_codes, b_codes, I, J, C, row_amax, col_amax, out, out_f32, epi};
+                    int gemm_kind, int32_t* status, const GemmEpilogue* epi, bool a_e4m3, bool b_e4m3) {
+  Fp4GemmDesc d = {a_codes, b_codes, I, J, C, row_amax, col_amax, out, out_f32, epi};
+  d.a_e4m3 = a_e4m3;
+  d.b_e4m3 = b_e4m3;
   const bool pair_mode = gemm_kind == FP4_GEMM_MXF4 && ctx->gemm_pairs;
   Problem p;
   int rc = make_problem(ctx, &p, d, gemm_kind, pair_mode, status);

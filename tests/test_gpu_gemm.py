@@ -82,6 +82,47 @@ def test_descales_fp32_and_bf16(lib, ctx, kind):
     assert torch.equal(outb.cpu(), wantb)
 
 
+@pytest.mark.parametrize("kind_name", ["FP4_GEMM_F8F6F4_A8", "FP4_GEMM_F8F6F4_B8", "FP4_GEMM_F8F6F4_A8B8"])
+@pytest.mark.parametrize("shape", [(128, 256, 256), (384, 640, 1152), (256, 512, 4096)])
+def test_mixed_e4m3_operands(lib, ctx, kind_name, shape):
+    """E4M3 bytes as one or both operands of the byte-container kind (the W4A8 / W8A4 settings).
+    The products are not all on one binary scale, so the fp32 accumulation is compared at the
+    GEMM tolerance of 1e-3 of the summed magnitudes, and is in fact far closer."""
+    I, J, C = shape
+    kind = getattr(lib, kind_name)
+    a8 = kind_name in ("FP4_GEMM_F8F6F4_A8", "FP4_GEMM_F8F6F4_A8B8")
+    b8 = kind_name in ("FP4_GEMM_F8F6F4_B8", "FP4_GEMM_F8F6F4_A8B8")
+    rng = np.random.default_rng(I + J + C + len(kind_name))
+
+    def fp8(rows):
+        c = rng.integers(0, 256, (rows, C), dtype=np.uint8)
+        c[(c & 0x7F) == 0x7F] = 0x38                       # no NaN codes
+        return c
+
+    ca = fp8(I) if a8 else _codes(rng, I, C)
+    cb = fp8(J) if b8 else _codes(rng, J, C)
+    va = O.e4m3_decode(ca) if a8 else O.e2m1_decode(ca)
+    vb = O.e4m3_decode(cb) if b8 else O.e2m1_decode(cb)
+    a = torch.from_numpy(ca if a8 else O.pack_nibbles(ca)).cuda()
+    b = torch.from_numpy(cb if b8 else O.pack_nibbles(cb)).cuda()
+    ra = (rng.random(I) * 4 + 0.1).astype(np.float32)
+    cam = (rng.random(J) * 0.1 + 0.01).astype(np.float32)
+    ctx.status.zero_()
+    raw = lib.fp4_gemm(ctx, a, b, gemm_kind=kind)
+    out = lib.fp4_gemm(ctx, a, b, torch.from_numpy(ra).cuda(), torch.from_numpy(cam).cuda(), gemm_kind=kind)
+    torch.cuda.synchronize()
+    assert ctx.read_status() == 0
+    ref = va @ vb.T
+    mag = np.abs(va) @ np.abs(vb).T
+    err = np.abs(raw.cpu().numpy().astype(np.float64) - ref)
+    assert (err <= 1e-3 * mag).all()
+    assert (err <= 2.0 ** -18 * mag).all()                 # what fp32 accumulation of exact products gives
+    d_row = (ra / np.float32(448 if a8 else 6)).astype(np.float32)
+    d_col = (cam / np.float32(448 if b8 else 6)).astype(np.float32)
+    want = (raw.cpu().numpy() * d_row[:, None]).astype(np.float32) * d_col[None, :]
+    np.testing.assert_array_equal(out.cpu().numpy(), want.astype(np.float32))   # the two de-scales, in this order
+
+
 def test_argument_errors(lib, ctx):
     a = torch.zeros((128, 64), dtype=torch.uint8, device="cuda")
     with pytest.raises(lib.Fp4Error) as e:
