@@ -52,12 +52,17 @@ extern "C" {
 #define FP4_DEV_TIMEOUT          4   /* a bounded wait inside a kernel ran out               */
 
 /* gemm_kind: which tcgen05.mma flavour multiplies the E2M1 codes */
+#define FP4_FORMAT_E2M1  0
+#define FP4_FORMAT_E4M3  1
+
 #define FP4_GEMM_MXF4    0   /* packed nibbles, K = 64 per instruction, unit block scales    */
 #define FP4_GEMM_F8F6F4  1   /* nibbles in byte containers, K = 32 per instruction           */
 /* fp4_gemm only: the byte-container kind with E4M3 bytes as one or both operands */
 #define FP4_GEMM_F8F6F4_A8    2   /* a_codes are E4M3 bytes [I x C], b_codes E2M1 nibbles  */
 #define FP4_GEMM_F8F6F4_B8    3   /* a_codes E2M1 nibbles, b_codes E4M3 bytes [J x C]      */
 #define FP4_GEMM_F8F6F4_A8B8  4   /* both operands E4M3 bytes                              */
+/* fp4_linear_bwd only, OR-ed into gemm_kind (FP4_GEMM_F8F6F4): dY is quantised to E4M3 bytes */
+#define FP4_BWD_DY_E4M3       0x100
 
 typedef struct fp4_ctx fp4_ctx;   /* opaque: device id, SM count, workspace */
 
@@ -81,6 +86,12 @@ typedef struct fp4_qtensor {
   int64_t  sparse_cap;     /* capacity in entries; 2 * round((1-alpha) * rows * cols) always
                               suffices                                                        */
   int32_t* nnz;            /* [1] number of residual entries                                  */
+  int32_t  format;         /* set by the caller: FP4_FORMAT_E2M1 (0, as described above) or
+                              FP4_FORMAT_E4M3: OCP E4M3 bytes, one per element (codes
+                              [rows x cols], codes_t [cols x rows]), MAX = 448 in place of 6,
+                              nearest-even rounding with saturation, no clamping: the FP8
+                              operand of the W4A8 / W8A4 settings of Section 4.3            */
+  int32_t  reserved;       /* 0                                                               */
 } fp4_qtensor;
 
 /* Create a context on `device` with a workspace of `workspace_bytes` (cudaMalloc'ed here,

@@ -18,6 +18,9 @@ FP4_GEMM_F8F6F4 = 1
 FP4_GEMM_F8F6F4_A8 = 2
 FP4_GEMM_F8F6F4_B8 = 3
 FP4_GEMM_F8F6F4_A8B8 = 4
+FP4_BWD_DY_E4M3 = 0x100
+FP4_FORMAT_E2M1 = 0
+FP4_FORMAT_E4M3 = 1
 FP4_DEV_SPARSE_OVERFLOW = 1
 FP4_DEV_NONFINITE = 2
 FP4_DEV_TIMEOUT = 4
@@ -36,7 +39,7 @@ class fp4_qtensor(C.Structure):
         ("codes", C.c_void_p), ("codes_t", C.c_void_p), ("amax", C.c_void_p), ("thresholds", C.c_void_p),
         ("csr_rowptr", C.c_void_p), ("csr_col", C.c_void_p), ("csr_val", C.c_void_p),
         ("csc_colptr", C.c_void_p), ("csc_row", C.c_void_p), ("csc_val", C.c_void_p),
-        ("sparse_cap", C.c_int64), ("nnz", C.c_void_p),
+        ("sparse_cap", C.c_int64), ("nnz", C.c_void_p), ("format", C.c_int32), ("reserved", C.c_int32),
     ]
 
 
@@ -177,11 +180,12 @@ class QTensor:
     """Caller-owned buffers of one quantised operand (struct fp4_qtensor)."""
 
     def __init__(self, rows: int, cols: int, scale_axis: int, device, sparse_cap: int = 0,
-                 codes: bool = True, codes_t: bool = True):
+                 codes: bool = True, codes_t: bool = True, fmt: int = FP4_FORMAT_E2M1):
         dev = device
-        self.rows, self.cols, self.scale_axis = rows, cols, scale_axis
-        self.codes = torch.empty((rows, cols // 2), dtype=torch.uint8, device=dev) if codes else None
-        self.codes_t = torch.empty((cols, rows // 2), dtype=torch.uint8, device=dev) if codes_t else None
+        self.rows, self.cols, self.scale_axis, self.fmt = rows, cols, scale_axis, fmt
+        per_byte = 2 if fmt == FP4_FORMAT_E2M1 else 1          # E2M1 nibbles or E4M3 bytes
+        self.codes = torch.empty((rows, cols // per_byte), dtype=torch.uint8, device=dev) if codes else None
+        self.codes_t = torch.empty((cols, rows // per_byte), dtype=torch.uint8, device=dev) if codes_t else None
         self.amax = torch.empty(rows if scale_axis == 0 else cols, dtype=torch.float32, device=dev)
         self.sparse_cap = int(sparse_cap)
         if sparse_cap > 0:
@@ -200,7 +204,7 @@ class QTensor:
         self.struct = fp4_qtensor(
             rows, cols, _ptr(self.codes), _ptr(self.codes_t), _ptr(self.amax), _ptr(self.thresholds),
             _ptr(self.csr_rowptr), _ptr(self.csr_col), _ptr(self.csr_val),
-            _ptr(self.csc_colptr), _ptr(self.csc_row), _ptr(self.csc_val), self.sparse_cap, _ptr(self.nnz))
+            _ptr(self.csc_colptr), _ptr(self.csc_row), _ptr(self.csc_val), self.sparse_cap, _ptr(self.nnz), fmt, 0)
 
 
 def tail_capacity(rows: int, cols: int, alpha: float) -> int:
@@ -212,11 +216,12 @@ def tail_capacity(rows: int, cols: int, alpha: float) -> int:
 
 
 def fp4_quantize(ctx: Context, x: torch.Tensor, scale_axis: int, alpha: float = 1.0, prescale=None,
-                 codes: bool = True, codes_t: bool = True, out: QTensor | None = None) -> QTensor:
+                 codes: bool = True, codes_t: bool = True, out: QTensor | None = None,
+                 fmt: int = FP4_FORMAT_E2M1) -> QTensor:
     assert x.dtype == torch.bfloat16 and x.is_cuda and x.is_contiguous() and x.dim() == 2
     rows, cols = x.shape
     if out is None:
-        out = QTensor(rows, cols, scale_axis, x.device, tail_capacity(rows, cols, alpha), codes, codes_t)
+        out = QTensor(rows, cols, scale_axis, x.device, tail_capacity(rows, cols, alpha), codes, codes_t, fmt)
     _check(ctx.lib.fp4_quantize(ctx.handle, _stream(), _ptr(x), rows, cols, scale_axis, float(alpha),
                                 _ptr(prescale), C.byref(out.struct), _ptr(ctx.status)))
     return out
@@ -241,14 +246,17 @@ def fp4_gemm(ctx: Context, a_codes: torch.Tensor, b_codes: torch.Tensor, row_ama
 def fp4_linear_fwd(ctx: Context, A: torch.Tensor, W: torch.Tensor, alpha: float, saved_a: QTensor | None = None,
                    saved_w: QTensor | None = None, reuse_w: bool = False, gemm_kind: int = FP4_GEMM_MXF4,
                    reuse_a: bool = False,
-                   out_f32: bool = False, out: torch.Tensor | None = None):
+                   out_f32: bool = False, out: torch.Tensor | None = None,
+                   fmt_a: int = FP4_FORMAT_E2M1, fmt_w: int = FP4_FORMAT_E2M1):
+    """Forward of the layer.  `fmt_a` / `fmt_w` = FP4_FORMAT_E4M3 give the W4A8 / W8A4 settings (the
+    formats are those of the saved operands; they need gemm_kind = FP4_GEMM_F8F6F4)."""
     M, K = A.shape
     K2, N = W.shape
     assert K == K2 and A.dtype == torch.bfloat16 and W.dtype == torch.bfloat16
     if saved_a is None:
-        saved_a = QTensor(M, K, 0, A.device, tail_capacity(M, K, alpha))
+        saved_a = QTensor(M, K, 0, A.device, tail_capacity(M, K, alpha), fmt=fmt_a)
     if saved_w is None:
-        saved_w = QTensor(K, N, 1, A.device)
+        saved_w = QTensor(K, N, 1, A.device, fmt=fmt_w)
     if out is None:
         out = torch.empty((M, N), dtype=torch.float32 if out_f32 else torch.bfloat16, device=A.device)
     _check(ctx.lib.fp4_linear_fwd(ctx.handle, _stream(), _ptr(A), _ptr(W), M, K, N, float(alpha), int(reuse_w) | (2 if reuse_a else 0),
@@ -260,7 +268,10 @@ def fp4_linear_fwd(ctx: Context, A: torch.Tensor, W: torch.Tensor, alpha: float,
 def fp4_linear_bwd(ctx: Context, dY: torch.Tensor, W: torch.Tensor, saved_a: QTensor, saved_w: QTensor,
                    dge_on: bool = True, dge_k: float = 5.0, dge_clip: float = 3.0,
                    gemm_kind: int = FP4_GEMM_MXF4, out_f32: bool = False, dA=None, dW=None,
-                   want_da: bool = True, want_dw: bool = True):
+                   want_da: bool = True, want_dw: bool = True, dy_e4m3: bool = False):
+    """Backward of the layer.  `dy_e4m3` quantises dY to E4M3 bytes instead of E2M1 nibbles."""
+    if dy_e4m3:
+        gemm_kind |= FP4_BWD_DY_E4M3
     M, N = dY.shape
     K = W.shape[0]
     dt = torch.float32 if out_f32 else torch.bfloat16

@@ -21,7 +21,7 @@ size_t linear_scratch_bytes(int64_t M, int64_t K, int64_t N) {
   size_t b = 0;
   const size_t big = size_t(M > K ? M : K) * size_t(N);
   b += round256(big * sizeof(float));                 // fwd: M x N result; bwd: up to K compensation rows of N
-  b += 2 * round256(size_t(M) * size_t(N) / 2);       // dY codes, both scalings
+  b += 2 * round256(size_t(M) * size_t(N));           // dY codes, both scalings (E4M3 bytes at most)
   b += round256(size_t(M) * 4) + round256(size_t(N) * 4);   // their amax vectors
   b += 2 * round256(size_t(M > N ? M : N) * 4);       // de-scale vectors used as prescale
   b += round256((2 * size_t(K) + 2) * 4) + round256(size_t(K) * 4);   // non-empty residual columns, their slots
@@ -179,10 +179,11 @@ int fp4_quantize(fp4_ctx* ctx, void* stream, const void* x_bf16, int64_t rows, i
   if (!(alpha > 0.5 && alpha <= 1.0)) return FP4_ERR_ALPHA;
   int rc = check_qtensor_dense(out);
   if (rc != FP4_OK) return rc;
+  if (out->format != FP4_FORMAT_E2M1 && out->format != FP4_FORMAT_E4M3) return FP4_ERR_ARG;
   if (!aligned16(x_bf16) || !aligned16(out->codes) || !aligned16(out->codes_t) || !aligned16(out->amax))
     return FP4_ERR_ALIGN;
   if (alpha < 1.0) {
-    if (scale_axis != 0 || prescale) return FP4_ERR_ARG;
+    if (scale_axis != 0 || prescale || out->format != FP4_FORMAT_E2M1) return FP4_ERR_ARG;
     const int64_t n = rows * cols;
     const int64_t n_tail = llround((1.0 - alpha) * double(n));
     if (2 * n_tail >= n) return FP4_ERR_ALPHA;
@@ -194,7 +195,7 @@ int fp4_quantize(fp4_ctx* ctx, void* stream, const void* x_bf16, int64_t rows, i
   out->rows = rows;
   out->cols = cols;
   return launch_quantize(ctx, static_cast<cudaStream_t>(stream), arena, x_bf16, rows, cols, scale_axis, alpha,
-                         prescale, 0, out, status);
+                         prescale, 0.0f, out, status);
 }
 
 int fp4_gemm(fp4_ctx* ctx, void* stream, const uint8_t* a_codes, const uint8_t* b_codes, int64_t I, int64_t J,
@@ -223,6 +224,12 @@ int fp4_linear_fwd(fp4_ctx* ctx, void* stream, const void* A_bf16, const void* W
   if (!savedW->codes || !savedW->codes_t || !savedW->amax) return FP4_ERR_NULL;
   if (!aligned16(A_bf16) || !aligned16(W_bf16) || !aligned16(Y)) return FP4_ERR_ALIGN;
   const bool occ = alpha < 1.0;
+  {
+    const bool a8 = savedA->format == FP4_FORMAT_E4M3, w8 = savedW->format == FP4_FORMAT_E4M3;
+    if ((savedA->format != FP4_FORMAT_E2M1 && !a8) || (savedW->format != FP4_FORMAT_E2M1 && !w8)) return FP4_ERR_ARG;
+    if ((a8 || w8) && gemm_kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;   // E4M3 needs the byte-container kind
+    if (a8 && occ) return FP4_ERR_ARG;                                    // clamping belongs to 4-bit activations
+  }
   if (occ) {
     const int64_t n_tail = llround((1.0 - alpha) * double(M * K));
     if (2 * n_tail >= M * K) return FP4_ERR_ALPHA;
@@ -262,7 +269,7 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
     Arena a(scratch_w, quantize_scratch_bytes(K, N));
     savedW->rows = K;
     savedW->cols = N;
-    rc = launch_quantize(ctx, s0, a, W_bf16, K, N, /*scale_axis=*/1, 1.0, nullptr, 0, savedW, status);
+    rc = launch_quantize(ctx, s0, a, W_bf16, K, N, /*scale_axis=*/1, 1.0, nullptr, 0.0f, savedW, status);
     if (rc != FP4_OK) return rc;
     if (ov) FP4_CUDA_TRY(cudaEventRecord(ctx->ev[1], s0));
   }
@@ -272,18 +279,26 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
     savedA->cols = K;
     // CSR on side stream 1, CSC on side stream 0 (behind W's short chain, which has ended by then)
     const SparseOverlap so = {ctx->side[1], ctx->ev[2], ctx->ev[3], ctx->side[0], ctx->ev[7]};
-    rc = launch_quantize(ctx, st, a, A_bf16, M, K, /*scale_axis=*/0, alpha, nullptr, 0, savedA, status,
+    rc = launch_quantize(ctx, st, a, A_bf16, M, K, /*scale_axis=*/0, alpha, nullptr, 0.0f, savedA, status,
                          occ && ov ? &so : nullptr);
     if (rc != FP4_OK) return rc;
   }
   if (!reuse_w && ov) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[1], 0));
   // Y1 = (Q(A_c) Q(W)) * d_A[m] * d_W[n]: A codes [M x K/2], W codes transposed [N x K/2].
+  const bool a8 = savedA->format == FP4_FORMAT_E4M3, w8 = savedW->format == FP4_FORMAT_E4M3;
   if (!occ) {
+    // Without clamping there is no residual: a saved operand that still carries the sparse
+    // structure of an earlier clamped use is marked empty, so that the backward adds nothing.
+    if (!reuse_a && savedA->csc_colptr && savedA->csr_rowptr && savedA->nnz) {
+      FP4_CUDA_TRY(cudaMemsetAsync(savedA->csc_colptr, 0, (size_t(K) + 1) * 4, st));
+      FP4_CUDA_TRY(cudaMemsetAsync(savedA->csr_rowptr, 0, (size_t(M) + 1) * 4, st));
+      FP4_CUDA_TRY(cudaMemsetAsync(savedA->nnz, 0, 4, st));
+    }
     return launch_gemm_fp4(ctx, st, savedA->codes, savedW->codes_t, M, N, K, savedA->amax, savedW->amax, Y, out_f32,
-                           gemm_kind, status);
+                           gemm_kind, status, nullptr, a8, w8);
   }
   rc = launch_gemm_fp4(ctx, st, savedA->codes, savedW->codes_t, M, N, K, savedA->amax, savedW->amax, y1, 1, gemm_kind,
-                       status);
+                       status, nullptr, a8, w8);
   if (rc != FP4_OK) return rc;
   // Y = store(Y1 + (A - A_c) W): one rounding of the fp32 sum.  Needs the CSR.
   if (!reuse_a && ov) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[3], 0));
@@ -304,7 +319,13 @@ int fp4_linear_bwd(fp4_ctx* ctx, void* stream, const void* dY_bf16, const void* 
   if (!dA && !dW) return FP4_ERR_NULL;
   if (!mult128(M) || !mult128(K) || !mult128(N)) return FP4_ERR_SHAPE;
   if (M * K >= (int64_t(1) << 31) || K * N >= (int64_t(1) << 31) || M * N >= (int64_t(1) << 31)) return FP4_ERR_SHAPE;
-  if (gemm_kind != FP4_GEMM_MXF4 && gemm_kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;
+  {
+    const int kind = gemm_kind & ~FP4_BWD_DY_E4M3;
+    if (kind != FP4_GEMM_MXF4 && kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;
+    const bool any8 = (gemm_kind & FP4_BWD_DY_E4M3) || savedA->format == FP4_FORMAT_E4M3 ||
+                      savedW->format == FP4_FORMAT_E4M3;
+    if (any8 && kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;             // E4M3 needs the byte-container kind
+  }
   if (dge_on && !(dge_k > 1.0f && dge_clip > 0.0f)) return FP4_ERR_ARG;
   if (!savedA->codes_t || !savedA->amax || !savedW->codes || !savedW->amax) return FP4_ERR_NULL;
   if (!aligned16(dY_bf16) || !aligned16(W_bf16) || !aligned16(dA) || !aligned16(dW)) return FP4_ERR_ALIGN;
@@ -322,8 +343,13 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
                     float dge_k, float dge_clip, int gemm_kind, void* dA, void* dW, int out_f32, int32_t* status) {
   const bool has_comp = dW && savedA->csc_colptr != nullptr;
   float* comp = has_comp ? arena.take<float>(size_t(K) * size_t(N)) : nullptr;   // compact: one row per non-empty column
-  uint8_t* g1_codes = dA ? arena.take<uint8_t>(size_t(M) * size_t(N) / 2) : nullptr;   // dY (.) d_W, token-wise
-  uint8_t* g2_codes = dW ? arena.take<uint8_t>(size_t(M) * size_t(N) / 2) : nullptr;   // dY (.) d_A, channel-wise
+  const bool dy8 = (gemm_kind & FP4_BWD_DY_E4M3) != 0;                 // dY as E4M3 bytes instead of E2M1 nibbles
+  gemm_kind &= ~FP4_BWD_DY_E4M3;
+  const bool a8 = savedA->format == FP4_FORMAT_E4M3, w8 = savedW->format == FP4_FORMAT_E4M3;
+  const float a_div = a8 ? 448.0f : 6.0f, w_div = w8 ? 448.0f : 6.0f;  // de-scale = amax / MAX of the operand's format
+  const size_t g_bytes = size_t(M) * size_t(N) / (dy8 ? 1 : 2);
+  uint8_t* g1_codes = dA ? arena.take<uint8_t>(g_bytes) : nullptr;      // dY (.) d_W, token-wise
+  uint8_t* g2_codes = dW ? arena.take<uint8_t>(g_bytes) : nullptr;      // dY (.) d_A, channel-wise
   float* g1_amax = arena.take<float>(size_t(M));
   float* g2_amax = arena.take<float>(size_t(N));
   int* col_lists = arena.take<int>(2 * size_t(K) + 2);
@@ -351,7 +377,7 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
   if (dA && dW) {
     Arena a = q_arena;
     rc = launch_quantize_dual(ctx, st, a, dY_bf16, M, N, savedW->amax, savedA->amax, g1_codes, g1_amax, g2_codes,
-                              g2_amax, status);
+                              g2_amax, status, dy8, w_div, a_div);
     if (rc != FP4_OK) return rc;
     if (sw != st) {
       FP4_CUDA_TRY(cudaEventRecord(ctx->ev[6], st));
@@ -359,15 +385,15 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
     }
   } else if (dA) {
     fp4_qtensor g = {};
-    g.rows = M; g.cols = N; g.codes = g1_codes; g.amax = g1_amax;
+    g.rows = M; g.cols = N; g.codes = g1_codes; g.amax = g1_amax; g.format = dy8 ? FP4_FORMAT_E4M3 : FP4_FORMAT_E2M1;
     Arena a = q_arena;
-    rc = launch_quantize(ctx, st, a, dY_bf16, M, N, /*scale_axis=*/0, 1.0, savedW->amax, 1, &g, status);
+    rc = launch_quantize(ctx, st, a, dY_bf16, M, N, /*scale_axis=*/0, 1.0, savedW->amax, w_div, &g, status);
     if (rc != FP4_OK) return rc;
   } else {
     fp4_qtensor g = {};
-    g.rows = M; g.cols = N; g.codes_t = g2_codes; g.amax = g2_amax;
+    g.rows = M; g.cols = N; g.codes_t = g2_codes; g.amax = g2_amax; g.format = dy8 ? FP4_FORMAT_E4M3 : FP4_FORMAT_E2M1;
     Arena a = q_arena;
-    rc = launch_quantize(ctx, st, a, dY_bf16, M, N, /*scale_axis=*/1, 1.0, savedA->amax, 1, &g, status);
+    rc = launch_quantize(ctx, st, a, dY_bf16, M, N, /*scale_axis=*/1, 1.0, savedA->amax, a_div, &g, status);
     if (rc != FP4_OK) return rc;
   }
   // dW[k,n] = store( (d_G''[n] * sum_m Aq[m,k] G''[m,n] + comp[k,n]) * Q'(W[k,n] * 6 / amax_W[n]) ):
@@ -375,13 +401,17 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
   GemmEpilogue epi = {};
   epi.addend = comp;
   epi.slot_of_row = slot_of_col;
-  epi.w_bf16 = dge_on ? W_bf16 : nullptr;
+  epi.w_bf16 = (dge_on && !w8) ? W_bf16 : nullptr;      // the DGE factor belongs to 4-bit weights
   epi.w_amax = savedW->amax;
   epi.dge_k = dge_k;
   epi.dge_clip = dge_clip;
   // dA = d_G'[m] * sum_n G'[m,n] Wq[k,n]
-  const Fp4GemmDesc wgrad = {savedA->codes_t, g2_codes, K, N, M, nullptr, g2_amax, dW, out_f32, &epi};
-  const Fp4GemmDesc dgrad = {g1_codes, savedW->codes, M, K, N, g1_amax, nullptr, dA, out_f32, nullptr};
+  Fp4GemmDesc wgrad = {savedA->codes_t, g2_codes, K, N, M, nullptr, g2_amax, dW, out_f32, &epi};
+  wgrad.a_e4m3 = a8;
+  wgrad.b_e4m3 = dy8;
+  Fp4GemmDesc dgrad = {g1_codes, savedW->codes, M, K, N, g1_amax, nullptr, dA, out_f32, nullptr};
+  dgrad.a_e4m3 = dy8;
+  dgrad.b_e4m3 = w8;
   const bool pairs = gemm_kind == FP4_GEMM_MXF4 && ctx->gemm_pairs;
   if (dA && dW && !pairs) {
     // Both GEMMs in one launch on the caller's stream, the weight gradient's tiles first (their
@@ -394,11 +424,12 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
   }
   if (dW) {
     rc = launch_gemm_fp4(ctx, sw, wgrad.a_codes, wgrad.b_codes, K, N, M, nullptr, g2_amax, dW, out_f32, gemm_kind,
-                         status, &epi);
+                         status, &epi, a8, dy8);
     if (rc != FP4_OK) return rc;
   }
   if (dA) {
-    rc = launch_gemm_fp4(ctx, st, g1_codes, savedW->codes, M, K, N, g1_amax, nullptr, dA, out_f32, gemm_kind, status);
+    rc = launch_gemm_fp4(ctx, st, g1_codes, savedW->codes, M, K, N, g1_amax, nullptr, dA, out_f32, gemm_kind, status,
+                         nullptr, dy8, w8);
     if (rc != FP4_OK) return rc;
   }
   if (sw != st) {

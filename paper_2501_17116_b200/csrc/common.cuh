@@ -165,20 +165,23 @@ struct SparseOverlap {
 };
 
 // Quantiser pieces (quantize.cu)
-// `prescale_is_amax`: the prescale vector holds amax values and stands for amax / 6.
+// `prescale_div` > 0: the prescale vector holds amax values and stands for amax / prescale_div (6 for an
+// E2M1 operand, 448 for an E4M3 one); 0: the vector is used as it is.  out->format selects E2M1 or E4M3.
 size_t quantize_scratch_bytes(int64_t rows, int64_t cols);
 size_t quantize_persistent_bytes();
 int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void* x_bf16, int64_t rows,
                     int64_t cols, int scale_axis, double alpha, const float* prescale,
-                    int prescale_is_amax, fp4_qtensor* out, int32_t* status,
+                    float prescale_div, fp4_qtensor* out, int32_t* status,
                     const SparseOverlap* overlap = nullptr);
 
-// dY for both backward GEMMs in one read: row-scaled codes of x (.) (amax_col_pre / 6) with their
-// row amax, and column-scaled transposed codes of x (.) (amax_row_pre / 6) with their column amax.
+// dY for both backward GEMMs in one read: row-scaled codes of x (.) (amax_col_pre / col_pre_div) with
+// their row amax, and column-scaled transposed codes of x (.) (amax_row_pre / row_pre_div) with their
+// column amax; E2M1 nibbles or E4M3 bytes.
 int launch_quantize_dual(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void* x_bf16, int64_t rows,
                          int64_t cols, const float* amax_col_pre, const float* amax_row_pre,
                          uint8_t* codes_rows, float* amax_rows_out, uint8_t* codes_t_cols,
-                         float* amax_cols_out, int32_t* status);
+                         float* amax_cols_out, int32_t* status, bool e4m3 = false, float col_pre_div = 6.0f,
+                         float row_pre_div = 6.0f);
 
 // Sparse compensation and epilogues (compensate.cu)
 // y[m,:] = store( y1[m,:] + sum_{entries of row m} val * dense[col,:] )

@@ -295,10 +295,11 @@ hist_select_kernel(const uint4* __restrict__ x, int rows, int vec_per_row, uint3
 // ------------------------------------------------------------------------------------------
 // absmax without clamping
 // ------------------------------------------------------------------------------------------
-// d[i] = amax[i] / 6 rounded once: the de-scale vector of a quantised operand, used as a prescale
-__global__ void descale_kernel(const float* __restrict__ amax, int n, float* __restrict__ d) {
+// d[i] = amax[i] / MAX rounded once (MAX = 6 for E2M1, 448 for E4M3): the de-scale vector of a
+// quantised operand, used as a prescale
+__global__ void descale_kernel(const float* __restrict__ amax, int n, float div, float* __restrict__ d) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) d[i] = __fdiv_rn(amax[i], 6.0f);
+  if (i < n) d[i] = __fdiv_rn(amax[i], div);
 }
 
 struct AbsmaxArgs {
@@ -306,7 +307,7 @@ struct AbsmaxArgs {
   int rows, cols;
   const float* pre_col;         // multiplies along columns before the row-wise maximum (or null)
   const float* pre_row;         // multiplies along rows before the column-wise maximum (or null)
-  int pre_is_amax;              // the two vectors hold amax values: use amax / 6 and store it
+  float pre_col_div, pre_row_div;   // > 0: the vector holds amax values: use amax / div (6 or 448) and store it
   float* d_col_out;             // dual mode: the de-scale vectors actually used, for the encoder
   float* d_row_out;
   uint32_t* amax_rows;          // float bits, zero-initialised (non-negative floats order as integers)
@@ -330,13 +331,13 @@ absmax_tile_kernel(const AbsmaxArgs a) {
     const int c = col0 + tid;
     if (c < a.cols) {
       const float v = __ldg(&a.pre_col[c]);
-      s_pcol[tid] = a.pre_is_amax ? __fdiv_rn(v, 6.0f) : v;
+      s_pcol[tid] = a.pre_col_div > 0.0f ? __fdiv_rn(v, a.pre_col_div) : v;
       if (a.d_col_out && blockIdx.y == 0) a.d_col_out[c] = s_pcol[tid];
     }
   }
   if (want_cols && a.pre_row && tid < ENC_TM) {
     const float v = __ldg(&a.pre_row[row0 + tid]);
-    s_prow[tid] = a.pre_is_amax ? __fdiv_rn(v, 6.0f) : v;
+    s_prow[tid] = a.pre_row_div > 0.0f ? __fdiv_rn(v, a.pre_row_div) : v;
     if (a.d_row_out && blockIdx.x == 0) a.d_row_out[row0 + tid] = s_prow[tid];
   }
   __syncthreads();
@@ -604,6 +605,137 @@ encode_kernel(const EncodeArgs a) {
 }
 
 // ------------------------------------------------------------------------------------------
+// 3b. E4M3 encoder (FP8 operands of the W4A8 / W8A4 settings and of the FP8 reading of dY)
+// ------------------------------------------------------------------------------------------
+// Two floats -> two E4M3 bytes (first value in the low byte): nearest even, saturating at 448,
+// the sign kept also on zero.
+__device__ __forceinline__ uint32_t e4m3x2(float lo, float hi) {
+  uint16_t r;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+// 4 x 4 byte transpose: in[r] byte c -> out[c] byte r
+__device__ __forceinline__ void transpose4x4_bytes(uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t (&c)[4]) {
+  const uint32_t t0 = __byte_perm(a0, a1, 0x5140), t1 = __byte_perm(a2, a3, 0x5140);
+  const uint32_t t2 = __byte_perm(a0, a1, 0x7362), t3 = __byte_perm(a2, a3, 0x7362);
+  c[0] = __byte_perm(t0, t1, 0x5410);
+  c[1] = __byte_perm(t0, t1, 0x7632);
+  c[2] = __byte_perm(t2, t3, 0x5410);
+  c[3] = __byte_perm(t2, t3, 0x7632);
+}
+
+// Same tile and thread mapping as encode_kernel, one byte per element: `codes` [rows x cols] bytes
+// (row-scaled in dual mode), `codes_t` [cols x rows] bytes (column-scaled in dual mode).  No
+// clamping: outlier clamping belongs to 4-bit activations.
+template <int MODE, bool PRESCALE>
+__global__ void __launch_bounds__(ENC_THREADS)
+encode_e4m3_kernel(const EncodeArgs a) {
+  __shared__ float s_gcol[ENC_TK];
+  __shared__ float s_grow[ENC_TM];
+  __shared__ float s_prow[ENC_TM];
+  __shared__ uint2 tile_t[8 * 8 * 32];
+  const int tid = threadIdx.x;
+  const int warp = tid >> 5, lane = tid & 31;
+  const int row0 = blockIdx.y * ENC_TM;
+  const int col0 = blockIdx.x * ENC_TK;
+  const int vec_per_row = a.cols >> 3;
+  constexpr bool ROW_SCALED = MODE != MODE_COLS;
+  constexpr bool COL_SCALED = MODE != MODE_ROWS;
+  if (ROW_SCALED && tid < ENC_TM) {
+    const int r = row0 + tid;
+    const float amax = __uint_as_float(a.amax_rows[r]);
+    s_grow[tid] = amax > 0.0f ? __fdiv_rn(448.0f, amax) : 0.0f;
+    if (blockIdx.x == 0) a.amax_out_rows[r] = amax;
+  }
+  if (COL_SCALED) {
+    const int c = col0 + tid;
+    if (c < a.cols) {
+      const float amax = __uint_as_float(a.amax_cols[c]);
+      s_gcol[tid] = amax > 0.0f ? __fdiv_rn(448.0f, amax) : 0.0f;
+      if (blockIdx.y == 0) a.amax_out_cols[c] = amax;
+    }
+    if (PRESCALE && tid < ENC_TM) s_prow[tid] = __ldg(&a.pre_row[row0 + tid]);
+  }
+  __syncthreads();
+
+  const int col = col0 + 8 * lane;
+  const bool in_cols = col < a.cols;
+  uint4 v[8];
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+    v[r] = make_uint4(0, 0, 0, 0);
+    if (in_cols) v[r] = __ldg(&a.x[(long long)(row0 + 8 * warp + r) * vec_per_row + (col >> 3)]);
+  }
+  float gc[8], pc[8];
+  if (COL_SCALED) {
+#pragma unroll
+    for (int c = 0; c < 8; ++c) gc[c] = in_cols ? s_gcol[8 * lane + c] : 0.0f;
+  }
+  if (ROW_SCALED && PRESCALE) {
+#pragma unroll
+    for (int c = 0; c < 8; ++c) pc[c] = in_cols ? __ldg(&a.pre_col[col + c]) : 0.0f;
+  }
+  uint32_t lo4[8], hi4[8];                            // bytes of columns 0..3 / 4..7 of each row (output for codes_t)
+  uint8_t* codes8 = reinterpret_cast<uint8_t*>(a.codes);
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+    const uint32_t w[4] = {v[r].x, v[r].y, v[r].z, v[r].w};
+    float f[8], f2[8];
+    const float grow = ROW_SCALED ? s_grow[8 * warp + r] : 0.0f;
+    const float prow = (COL_SCALED && PRESCALE) ? s_prow[8 * warp + r] : 1.0f;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      const float xv = (c & 1) ? bf16_hi(w[c >> 1]) : bf16_lo(w[c >> 1]);
+      if constexpr (MODE == MODE_ROWS) {
+        f[c] = __fmul_rn(PRESCALE ? __fmul_rn(xv, pc[c]) : xv, grow);
+      } else if constexpr (MODE == MODE_COLS) {
+        f[c] = __fmul_rn(PRESCALE ? __fmul_rn(xv, prow) : xv, gc[c]);
+      } else {
+        f[c] = __fmul_rn(__fmul_rn(xv, pc[c]), grow);
+        f2[c] = __fmul_rn(__fmul_rn(xv, prow), gc[c]);
+      }
+    }
+    const uint32_t b_lo = e4m3x2(f[0], f[1]) | (e4m3x2(f[2], f[3]) << 16);
+    const uint32_t b_hi = e4m3x2(f[4], f[5]) | (e4m3x2(f[6], f[7]) << 16);
+    if (in_cols && codes8)
+      *reinterpret_cast<uint2*>(codes8 + (long long)(row0 + 8 * warp + r) * a.cols + col) = make_uint2(b_lo, b_hi);
+    if constexpr (MODE == MODE_DUAL) {
+      lo4[r] = e4m3x2(f2[0], f2[1]) | (e4m3x2(f2[2], f2[3]) << 16);
+      hi4[r] = e4m3x2(f2[4], f2[5]) | (e4m3x2(f2[6], f2[7]) << 16);
+    } else {
+      lo4[r] = b_lo;
+      hi4[r] = b_hi;
+    }
+  }
+  if (a.codes_t) {
+    // 8 x 8 byte transpose in registers: column c of this thread's block as the bytes of rows 0..7
+    uint32_t q00[4], q01[4], q10[4], q11[4];
+    transpose4x4_bytes(lo4[0], lo4[1], lo4[2], lo4[3], q00);     // columns 0..3, rows 0..3
+    transpose4x4_bytes(lo4[4], lo4[5], lo4[6], lo4[7], q01);     // columns 0..3, rows 4..7
+    transpose4x4_bytes(hi4[0], hi4[1], hi4[2], hi4[3], q10);     // columns 4..7, rows 0..3
+    transpose4x4_bytes(hi4[4], hi4[5], hi4[6], hi4[7], q11);     // columns 4..7, rows 4..7
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      tile_t[(c * 8 + warp) * 32 + lane] = make_uint2(q00[c], q01[c]);
+      tile_t[((c + 4) * 8 + warp) * 32 + lane] = make_uint2(q10[c], q11[c]);
+    }
+  }
+  __syncthreads();
+  if (a.codes_t) {
+    // thread (c = warp, j = lane) owns column col0 + 8 j + c: 64 rows = 64 bytes
+    const int k = col0 + 8 * lane + warp;
+    if (k < a.cols) {
+      uint2 o[8];
+#pragma unroll
+      for (int w8 = 0; w8 < 8; ++w8) o[w8] = tile_t[(warp * 8 + w8) * 32 + lane];
+      uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(a.codes_t) + (long long)k * a.rows + row0);
+#pragma unroll
+      for (int h = 0; h < 4; ++h) dst[h] = make_uint4(o[2 * h].x, o[2 * h].y, o[2 * h + 1].x, o[2 * h + 1].y);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // 4. mask -> CSR / CSC
 // ------------------------------------------------------------------------------------------
 // Exclusive prefix sum of n counts by one block; ptr[n] = total.  Also publishes nnz and raises
@@ -784,11 +916,14 @@ size_t quantize_scratch_bytes(int64_t rows, int64_t cols) {
 }
 
 int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void* x_bf16, int64_t rows64,
-                    int64_t cols64, int scale_axis, double alpha, const float* prescale, int prescale_is_amax,
+                    int64_t cols64, int scale_axis, double alpha, const float* prescale, float prescale_div,
                     fp4_qtensor* out, int32_t* status, const SparseOverlap* overlap) {
   const int rows = int(rows64), cols = int(cols64);
   const long long n = (long long)rows * cols;
   const bool occ = alpha < 1.0;
+  const bool e4m3 = out->format == FP4_FORMAT_E4M3;
+  if (out->format != FP4_FORMAT_E2M1 && !e4m3) return FP4_ERR_ARG;
+  if (e4m3 && occ) return FP4_ERR_ARG;               // outlier clamping belongs to 4-bit activations
   const uint4* x = static_cast<const uint4*>(x_bf16);
   Scratch sc = carve(arena, rows, cols, occ);
   if (!sc.ok) return FP4_ERR_WORKSPACE;
@@ -864,11 +999,11 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
     }
     if (sc2 != sp) FP4_CUDA_TRY(cudaEventRecord(overlap->csc_done, sc2));
   } else {
-    if (prescale && prescale_is_amax) {
+    if (prescale && prescale_div > 0.0f) {
       float* d = scale_axis == 0 ? sc.pre_cols : sc.pre_rows;
       const int np = scale_axis == 0 ? cols : rows;
       KernelScope scope(ctx, stream, KC_ABSMAX, 1);
-      descale_kernel<<<(np + 255) / 256, 256, 0, stream>>>(prescale, np, d);
+      descale_kernel<<<(np + 255) / 256, 256, 0, stream>>>(prescale, np, prescale_div, d);
       prescale = d;
     }
     AbsmaxArgs aa = {};
@@ -887,7 +1022,11 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
         absmax_tile_kernel<MODE_ROWS><<<tile_grid, ENC_THREADS, 0, stream>>>(aa);
       }
       KernelScope scope(ctx, stream, KC_ENCODE, 1);
-      if (prescale)
+      if (e4m3 && prescale)
+        encode_e4m3_kernel<MODE_ROWS, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
+      else if (e4m3)
+        encode_e4m3_kernel<MODE_ROWS, false><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
+      else if (prescale)
         encode_kernel<MODE_ROWS, false, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
       else
         encode_kernel<MODE_ROWS, false, false><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
@@ -900,7 +1039,11 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
         absmax_tile_kernel<MODE_COLS><<<tile_grid, ENC_THREADS, 0, stream>>>(aa);
       }
       KernelScope scope(ctx, stream, KC_ENCODE, 1);
-      if (prescale)
+      if (e4m3 && prescale)
+        encode_e4m3_kernel<MODE_COLS, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
+      else if (e4m3)
+        encode_e4m3_kernel<MODE_COLS, false><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
+      else if (prescale)
         encode_kernel<MODE_COLS, false, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
       else
         encode_kernel<MODE_COLS, false, false><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
@@ -914,7 +1057,8 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
 // column-scaled transposed codes of dY (.) (amax_row_pre / 6).
 int launch_quantize_dual(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void* x_bf16, int64_t rows64,
                          int64_t cols64, const float* amax_col_pre, const float* amax_row_pre, uint8_t* codes_rows,
-                         float* amax_rows_out, uint8_t* codes_t_cols, float* amax_cols_out, int32_t* status) {
+                         float* amax_rows_out, uint8_t* codes_t_cols, float* amax_cols_out, int32_t* status,
+                         bool e4m3, float col_pre_div, float row_pre_div) {
   const int rows = int(rows64), cols = int(cols64);
   Scratch sc = carve(arena, rows, cols, false);
   if (!sc.ok) return FP4_ERR_WORKSPACE;
@@ -925,7 +1069,8 @@ int launch_quantize_dual(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const 
   aa.cols = cols;
   aa.pre_col = amax_col_pre;
   aa.pre_row = amax_row_pre;
-  aa.pre_is_amax = 1;
+  aa.pre_col_div = col_pre_div;
+  aa.pre_row_div = row_pre_div;
   aa.d_col_out = sc.pre_cols;
   aa.d_row_out = sc.pre_rows;
   aa.amax_rows = sc.amax_rows;
@@ -952,7 +1097,10 @@ int launch_quantize_dual(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const 
   ea.amax_out_rows = amax_rows_out;
   ea.amax_out_cols = amax_cols_out;
   KernelScope scope(ctx, stream, KC_ENCODE, 1);
-  encode_kernel<MODE_DUAL, false, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
+  if (e4m3)
+    encode_e4m3_kernel<MODE_DUAL, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
+  else
+    encode_kernel<MODE_DUAL, false, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
   FP4_CUDA_TRY(cudaGetLastError());
   return FP4_OK;
 }
