@@ -176,6 +176,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=1)
     ap.add_argument("--gemm-kind", type=int, default=0, help="0 mxf4 (K=64), 1 f8f6f4 (K=32)")
+    ap.add_argument("--precision", default="w4a4", choices=["w4a4", "w4a8", "w8a4", "w4a4-dy8"],
+                    help="operand formats: w4a4 (the method, default); w4a8 / w8a4: E4M3 activations / weights "
+                         "(the ablation settings); w4a4-dy8: dY quantised to E4M3.  All but w4a4 need --gemm-kind 1")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-share-activations", action="store_true",
                     help="quantise the activation of every linear, also where q/k/v or gate/up read the same tensor")
@@ -199,6 +202,13 @@ def main():
     alpha = cfg.alphas[0]
     M = cfg.M
     kind = args.gemm_kind
+    fmt_a = fp4.FP4_FORMAT_E4M3 if args.precision == "w4a8" else fp4.FP4_FORMAT_E2M1
+    fmt_w = fp4.FP4_FORMAT_E4M3 if args.precision == "w8a4" else fp4.FP4_FORMAT_E2M1
+    dy8 = args.precision == "w4a4-dy8"
+    if args.precision != "w4a4":
+        assert kind == 1, "E4M3 operands need the byte-container GEMM: pass --gemm-kind 1"
+    if fmt_a == fp4.FP4_FORMAT_E4M3:
+        alpha = 1.0                              # outlier clamping belongs to 4-bit activations
 
     # ------------------------------------------------------------------ inputs ------------
     def pinned(bits):
@@ -218,8 +228,8 @@ def main():
                  Y=torch.empty((M, N), dtype=torch.bfloat16, device=dev),
                  dA=torch.empty((M, K), dtype=torch.bfloat16, device=dev),
                  dW=torch.empty((K, N), dtype=torch.bfloat16, device=dev),
-                 sa=layers[first]["sa"] if shared else fp4.QTensor(M, K, 0, dev, fp4.tail_capacity(M, K, alpha)),
-                 sw=fp4.QTensor(K, N, 1, dev),
+                 sa=layers[first]["sa"] if shared else fp4.QTensor(M, K, 0, dev, fp4.tail_capacity(M, K, alpha), fmt=fmt_a),
+                 sw=fp4.QTensor(K, N, 1, dev, fmt=fmt_w),
                  hY=torch.empty((M, N), dtype=torch.bfloat16).pin_memory(),
                  hdA=torch.empty((M, K), dtype=torch.bfloat16).pin_memory(),
                  hdW=torch.empty((K, N), dtype=torch.bfloat16).pin_memory())
@@ -233,7 +243,8 @@ def main():
         for L in layers:
             fp4.fp4_linear_fwd(ctx, L["A"], L["W"], alpha, L["sa"], L["sw"], gemm_kind=kind, out=L["Y"],
                                reuse_a=L["reuse_a"])
-            fp4.fp4_linear_bwd(ctx, L["G"], L["W"], L["sa"], L["sw"], gemm_kind=kind, dA=L["dA"], dW=L["dW"])
+            fp4.fp4_linear_bwd(ctx, L["G"], L["W"], L["sa"], L["sw"], gemm_kind=kind, dA=L["dA"], dW=L["dW"],
+                               dy_e4m3=dy8)
 
     def step_host():
         for L in layers:
@@ -290,30 +301,34 @@ def main():
     nnz = [int(L["sa"].nnz.item()) if L["sa"].nnz is not None else 0 for L in layers]
 
     # ------------------------------------------------------------------ end to end ---------
-    for _ in range(3):
-        step_host()
-    torch.cuda.synchronize()
-    harness.barrier()
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0.record()
-    for _ in range(args.steps):
-        step_host()
-    t1.record()
-    torch.cuda.synchronize()
-    harness.barrier()
-    ms_e2e = t0.elapsed_time(t1)
+    # (the host-buffer entry point takes the method's own formats only)
+    ms_e2e = None
+    if args.precision == "w4a4":
+        for _ in range(3):
+            step_host()
+        torch.cuda.synchronize()
+        harness.barrier()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(args.steps):
+            step_host()
+        t1.record()
+        torch.cuda.synchronize()
+        harness.barrier()
+        ms_e2e = t0.elapsed_time(t1)
     clocks = sampler.stop()
 
     sec = harness.max_over_ranks(ms / 1e3, dev)
-    sec_e2e = harness.max_over_ranks(ms_e2e / 1e3, dev)
+    sec_e2e = harness.max_over_ranks(ms_e2e / 1e3, dev) if ms_e2e is not None else None
     total_flop = harness.sum_over_ranks(flop_step * args.steps, dev)
     value = total_flop / sec / 1e12
-    value_e2e = total_flop / sec_e2e / 1e12
+    value_e2e = total_flop / sec_e2e / 1e12 if sec_e2e else None
     h2d = sum((M * L["K"] + L["K"] * L["N"] + M * L["N"]) * 2 for L in layers)
     d2h = h2d
 
     # ------------------------------------------------------------------ rooflines ----------
-    fp4_peak = FP4_OVER_BF16 * peaks["bf16_tflops"]
+    # the byte-container kind runs at the FP8 rate (K = 32 per instruction), the MXF4 kind at twice that
+    fp4_peak = (FP4_OVER_BF16 if kind == 0 else FP4_OVER_BF16 / 2) * peaks["bf16_tflops"]
     alu_peak = SM_COUNT * FMA_LANES * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
     steps = args.steps
     elems_a = sum(M * L["K"] for L in layers if not L["reuse_a"])      # activations actually quantised
@@ -347,7 +362,8 @@ def main():
     roofline = {"kernel": dominant, "bound": dk["bound"], "achieved": dk["achieved"], "peak": dk["peak"],
                 "unit": dk["unit"], "frac": dk["frac"], "traffic": NCU_TRAFFIC_PER_UNIT.get(dominant),
                 "peak_source": ("of measured" if peaks["source"] == "measured" else "of fallback")
-                + (": 4 x sustained bf16 cuBLAS" if dk["bound"] == "tensor" else
+                + ((": 4 x sustained bf16 cuBLAS" if kind == 0 else ": 2 x sustained bf16 cuBLAS (FP8-rate kind)")
+                   if dk["bound"] == "tensor" else
                    ": copy bandwidth" if dk["bound"] == "hbm" else ": 148 SMs x 128 FMA x 2 x max clock")}
 
     # ------------------------------------------------------------------ CPU baseline -------
@@ -363,9 +379,11 @@ def main():
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * sec / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "fp4_e2m1", "data": "synthetic",
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": "fp4_e2m1" if args.precision == "w4a4" else "fp4_e2m1+fp8_e4m3", "data": "synthetic",
             "config": {"workload": cfg.name, "tokens": M, "linears": [f"{L['name']}:{L['K']}x{L['N']}" for L in layers],
                        "alpha": alpha, "dge": True, "gemm_kind": "mxf4" if kind == 0 else "f8f6f4",
+                       "precision": args.precision,
                        "l2": f"inputs exceed L2: {resident_bytes / 1e6:.0f} MB touched per step",
                        "launch": "one CUDA graph per step, replayed",
                        "shared_activations": ("q/k/v and gate/up read one activation tensor: quantised once, re-used"
@@ -373,8 +391,8 @@ def main():
                        "kernel_timing": f"CUDA events per kernel class over {args.steps} plainly launched steps, side "
                                         f"streams off ({ms_profiled / args.steps:.3f} ms/step that way)",
                        "replicas": world},
-            "e2e": {"value": value_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "ms_per_step": 1e3 * sec_e2e / args.steps},
+            "e2e": ({"value": value_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                     "ms_per_step": 1e3 * sec_e2e / args.steps} if sec_e2e else None),
             "gpu_launches": launches,
             "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu_baseline, "clocks": clocks,
             "residual_nnz": nnz_total,

@@ -155,6 +155,8 @@ int fp4_gemm(fp4_ctx* ctx, void* stream, const uint8_t* a_codes, const uint8_t* 
  * A is clamped at the alpha-quantiles and quantised token-wise, W channel-wise; the residual
  * A - A_c multiplies the BF16 weight in fp32; both branches meet in fp32 and are rounded once.
  *   A_bf16 [M x K], W_bf16 [K x N], Y [M x N] (BF16, or float if out_f32 != 0).
+ *   savedA->format / savedW->format = FP4_FORMAT_E4M3 give the W4A8 / W8A4 settings of Section 4.3
+ *   (gemm_kind must then be FP4_GEMM_F8F6F4; an E4M3 activation is not clamped: alpha must be 1).
  *   savedA, savedW: caller-allocated fp4_qtensor buffers that receive the quantised operands
  *   and are handed to fp4_linear_bwd.  savedA needs codes, codes_t, amax, thresholds, nnz,
  *   csr_*, csc_*; savedW needs codes, codes_t, amax.
@@ -181,6 +183,8 @@ int fp4_linear_fwd(fp4_ctx* ctx, void* stream, const void* A_bf16, const void* W
  * multiplication by d_A[m] (wgrad), so that the forward's codes of W and A are re-used.
  *   dY_bf16 [M x N], W_bf16 [K x N], dA [M x K], dW [K x N] (BF16, or float if out_f32).
  *   dA or dW may be NULL to skip that gradient.
+ *   gemm_kind | FP4_BWD_DY_E4M3 quantises both copies of dY to E4M3 bytes; the saved operands keep
+ *   the formats the forward gave them; with an E4M3 weight Q' = 1 whatever dge_on says.
  */
 int fp4_linear_bwd(fp4_ctx* ctx, void* stream, const void* dY_bf16, const void* W_bf16,
                    const fp4_qtensor* savedA, const fp4_qtensor* savedW,
