@@ -24,7 +24,7 @@ size_t linear_scratch_bytes(int64_t M, int64_t K, int64_t N) {
   b += 2 * round256(size_t(M) * size_t(N));           // dY codes, both scalings (E4M3 bytes at most)
   b += round256(size_t(M) * 4) + round256(size_t(N) * 4);   // their amax vectors
   b += 2 * round256(size_t(M > N ? M : N) * 4);       // de-scale vectors used as prescale
-  b += round256((2 * size_t(K) + 2) * 4) + round256(size_t(K) * 4);   // non-empty residual columns, their slots
+  b += comp_wgrad_scratch_bytes(M, K, N);             // non-empty residual columns, dense-column buffers
   return b;
 }
 
@@ -352,8 +352,9 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
   uint8_t* g2_codes = dW ? arena.take<uint8_t>(g_bytes) : nullptr;      // dY (.) d_A, channel-wise
   float* g1_amax = arena.take<float>(size_t(M));
   float* g2_amax = arena.take<float>(size_t(N));
-  int* col_lists = arena.take<int>(2 * size_t(K) + 2);
-  int* slot_of_col = arena.take<int>(size_t(K));
+  Arena comp_arena(arena.base + arena.off, comp_wgrad_scratch_bytes(M, K, N));
+  arena.take<char>(comp_wgrad_scratch_bytes(M, K, N));
+  int* slot_of_col = nullptr;
   if (!arena.ok) return FP4_ERR_WORKSPACE;
   Arena q_arena(arena.base + arena.off, arena.size - arena.off);
   int rc;
@@ -367,8 +368,7 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
     FP4_CUDA_TRY(cudaStreamWaitEvent(sw, ctx->ev[5], 0));
   }
   if (has_comp) {
-    rc = launch_comp_wgrad(ctx, sw, savedA->csc_colptr, savedA->csc_row, savedA->csc_val, dY_bf16, col_lists,
-                           slot_of_col, comp, K, N);
+    rc = launch_comp_wgrad(ctx, sw, savedA, dY_bf16, comp_arena, &slot_of_col, comp, M, K, N);
     if (rc != FP4_OK) return rc;
   }
 

@@ -190,8 +190,9 @@ int launch_comp_fwd(fp4_ctx* ctx, cudaStream_t stream, const float* y1, const in
                     int64_t N, void* y, int out_f32);
 // Weight-gradient compensation into a compact buffer: for every column k of the residual that
 // holds entries, comp[slot_of_col[k], :] = sum_{entries of column k} val * dy[row, :].
-// `lists`: scratch of 2 K + 2 ints; `slot_of_col`: [K] ints (-1 where the column is empty).
-int launch_comp_wgrad(fp4_ctx* ctx, cudaStream_t stream, const int32_t* colptr, const int32_t* row,
-                      const float* val, const void* dy_bf16, int* lists, int* slot_of_col, float* comp,
-                      int64_t K, int64_t N);
+// Lists, slots and the dense path's buffers are carved from `scratch` (comp_wgrad_scratch_bytes); the slot
+// vector is handed back for the GEMM's epilogue.  `a` is the saved activation (CSC; CSR for the dense path).
+int launch_comp_wgrad(fp4_ctx* ctx, cudaStream_t stream, const fp4_qtensor* a, const void* dy_bf16, Arena& scratch,
+                      int** slot_of_col_out, float* comp, int64_t M, int64_t K, int64_t N);
+size_t comp_wgrad_scratch_bytes(int64_t M, int64_t K, int64_t N);
 

@@ -83,56 +83,200 @@ comp_fwd_kernel(const float* __restrict__ y1, const int* __restrict__ rowptr, co
   store8(y, out_f32, off, y8);
 }
 
-constexpr int LONG_COLUMN = 64;            // entries from which a column gets a whole 1024-thread block
+constexpr int LONG_COLUMN = 512;           // entries from which a column gets a whole 1024-thread block
 constexpr int LONG_THREADS = 1024;
+constexpr int DENSE_SLOTS = 8;             // dense columns handled per pass (accumulators per lane: 8 x 8)
+constexpr int DENSE_MAX = 160;             // dense columns at most; further ones are treated as long
+constexpr int DENSE_MAX_CHUNKS = 40;       // chunks of tokens whose partial sums are added afterwards
 
-// Two ascending lists of the columns that hold residual entries: "long" columns (at least
-// LONG_COLUMN entries: the outlier channels) and "short" ones; counts[0], counts[1] their sizes.
-__global__ void __launch_bounds__(1024, 1)
-nonempty_columns_kernel(const int* __restrict__ colptr, int K, int* __restrict__ list_long,
-                        int* __restrict__ list_short, int* __restrict__ counts, int* __restrict__ slot_of_col) {
-  __shared__ unsigned long long warp_tot[32];
-  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-  const int per = (K + 1023) / 1024;
-  const int b = min(K, t * per), e = min(K, b + per);
-  unsigned long long c = 0;                          // low word: long columns, high word: short columns
-  for (int k = b; k < e; ++k) {
-    const int n = colptr[k + 1] - colptr[k];
-    if (n >= LONG_COLUMN) c += 1ull;
-    else if (n > 0) c += 1ull << 32;
-  }
-  unsigned long long incl = c;
+// Exclusive scan of one int per thread over a 1024-thread block; the block's total goes to *total.
+__device__ __forceinline__ int block_exclusive_scan_1024(int c, int* warp_tot, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = c;
 #pragma unroll
   for (int off = 1; off < 32; off <<= 1) {
-    const unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+    const int up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
     if (lane >= off) incl += up;
   }
+  __syncthreads();                                   // warp_tot may still be read from the previous scan
   if (lane == 31) warp_tot[warp] = incl;
   __syncthreads();
   if (warp == 0) {
-    unsigned long long v = warp_tot[lane];
+    int v = warp_tot[lane];
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
-      const unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, v, off);
+      const int up = __shfl_up_sync(0xFFFFFFFFu, v, off);
       if (lane >= off) v += up;
     }
     warp_tot[lane] = v;
   }
   __syncthreads();
-  const unsigned long long before = incl - c + (warp ? warp_tot[warp - 1] : 0ull);
-  // rows of the compact buffer: long columns first (in list order), then the short ones
-  const int n_long = int(warp_tot[31] & 0xFFFFFFFFull);
-  int pos_long = int(before & 0xFFFFFFFFull), pos_short = int(before >> 32);
+  *total = warp_tot[31];
+  return incl - c + (warp ? warp_tot[warp - 1] : 0);
+}
+
+// The columns of the residual that hold entries, by how full they are: "dense" (at least
+// `dense_from` entries, the first DENSE_MAX of them: outlier channels that most tokens hit,
+// Appendix D), "long" (at least LONG_COLUMN entries) and "short".  The long and the short ones
+// are listed in ascending order; counts[0..2] are the three sizes.  Rows of the compact buffer:
+// dense columns first, then the long, then the short ones, each in ascending column order;
+// slot_of_col[k] is column k's row or -1.  dense_from = INT_MAX switches the dense class off.
+__global__ void __launch_bounds__(1024, 1)
+nonempty_columns_kernel(const int* __restrict__ colptr, int K, int dense_from, int* __restrict__ list_long,
+                        int* __restrict__ list_short, int* __restrict__ counts, int* __restrict__ slot_of_col) {
+  __shared__ int warp_tot[32];
+  const int t = threadIdx.x;
+  const int per = (K + 1023) / 1024;
+  const int b = min(K, t * per), e = min(K, b + per);
+  int c_cand = 0;
+  for (int k = b; k < e; ++k) c_cand += (colptr[k + 1] - colptr[k] >= dense_from) ? 1 : 0;
+  int n_cand;
+  int rank = block_exclusive_scan_1024(c_cand, warp_tot, &n_cand);     // dense candidates before this thread
+  const int n_dense = min(n_cand, DENSE_MAX);
+  int c_long = 0, c_short = 0;
+  {
+    int r = rank;
+    for (int k = b; k < e; ++k) {
+      const int n = colptr[k + 1] - colptr[k];
+      if (n >= dense_from && r++ < DENSE_MAX) continue;
+      if (n >= LONG_COLUMN) ++c_long;
+      else if (n > 0) ++c_short;
+    }
+  }
+  int n_long, n_short;
+  int pos_long = block_exclusive_scan_1024(c_long, warp_tot, &n_long);
+  int pos_short = block_exclusive_scan_1024(c_short, warp_tot, &n_short);
   for (int k = b; k < e; ++k) {
     const int n = colptr[k + 1] - colptr[k];
     int slot = -1;
-    if (n >= LONG_COLUMN) { slot = pos_long; list_long[pos_long++] = k; }
-    else if (n > 0) { slot = n_long + pos_short; list_short[pos_short++] = k; }
+    if (n >= dense_from && rank < DENSE_MAX) slot = rank;
+    else if (n >= LONG_COLUMN) { slot = n_dense + pos_long; list_long[pos_long++] = k; }
+    else if (n > 0) { slot = n_dense + n_long + pos_short; list_short[pos_short++] = k; }
+    if (n >= dense_from) ++rank;
     slot_of_col[k] = slot;
   }
-  if (t == 1023) {
-    counts[0] = int(warp_tot[31] & 0xFFFFFFFFull);
-    counts[1] = int(warp_tot[31] >> 32);
+  if (t == 0) {
+    counts[0] = n_dense;
+    counts[1] = n_long;
+    counts[2] = n_short;
+  }
+}
+
+// Dense columns, step 1: their residual values as a dense matrix V[g][m][8] (group g holds the
+// compact rows 8 g .. 8 g + 7), zero where a token has no entry.  One warp per token walks the
+// token's CSR row.
+__global__ void __launch_bounds__(COMP_THREADS)
+dense_values_kernel(const int* __restrict__ rowptr, const int* __restrict__ col, const float* __restrict__ val,
+                    const int* __restrict__ slot_of_col, const int* __restrict__ counts, float* __restrict__ V, int M) {
+  const int n_dense = counts[0];
+  if (n_dense == 0) return;
+  const int groups = (n_dense + DENSE_SLOTS - 1) / DENSE_SLOTS;
+  const int lane = threadIdx.x & 31;
+  const int m = blockIdx.x * (COMP_THREADS / 32) + (threadIdx.x >> 5);
+  if (m >= M) return;
+  for (int i = lane; i < groups * DENSE_SLOTS; i += 32)
+    V[(size_t(i / DENSE_SLOTS) * M + m) * DENSE_SLOTS + (i % DENSE_SLOTS)] = 0.0f;
+  __syncwarp();
+  for (int e = rowptr[m] + lane; e < rowptr[m + 1]; e += 32) {
+    const int slot = slot_of_col[col[e]];
+    if (slot >= 0 && slot < n_dense) V[(size_t(slot / DENSE_SLOTS) * M + m) * DENSE_SLOTS + (slot % DENSE_SLOTS)] = val[e];
+  }
+}
+
+// Dense columns, step 2: C[slot, n] = sum_m V[m, slot] * dY[m, n] as a skinny dense product on the
+// plain ALUs: a block owns 256 output columns (8 per lane) and one chunk of the tokens, its 8
+// warps take the chunk's tokens in turn (four tokens' loads in flight), every lane keeps 8 x 8
+// accumulators, and dY is read once per group of 8 columns instead of once per entry.  The warps'
+// sums are added in warp order and, with more than one chunk, written as partial sums that
+// dense_reduce_kernel adds in chunk order: the result does not depend on scheduling.
+__global__ void __launch_bounds__(COMP_THREADS, 2)
+comp_wgrad_dense_kernel(float* __restrict__ out, const float* __restrict__ V, const uint4* __restrict__ dy,
+                        const int* __restrict__ counts, int M, int N, int rows_per_chunk, long long chunk_stride) {
+  constexpr int WARPS = COMP_THREADS / 32;
+  constexpr int FLY = 4;
+  __shared__ float red[WARPS][4][COMP_COLS];                    // 32 KB: four compact rows at a time
+  const int n_dense = counts[0];
+  if (n_dense == 0) return;
+  const int groups = (n_dense + DENSE_SLOTS - 1) / DENSE_SLOTS;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n0 = blockIdx.x * COMP_COLS + 8 * lane;
+  const bool in_cols = n0 < N;
+  const int r0 = blockIdx.y * rows_per_chunk, r1 = min(M, r0 + rows_per_chunk);
+  const int vec_per_row = N >> 3, vcol = n0 >> 3;
+  float* dst = out + (long long)blockIdx.y * chunk_stride;
+  for (int g = 0; g < groups; ++g) {
+    float acc[DENSE_SLOTS][8];
+#pragma unroll
+    for (int s = 0; s < DENSE_SLOTS; ++s)
+#pragma unroll
+      for (int c = 0; c < 8; ++c) acc[s][c] = 0.0f;
+    if (in_cols) {
+      const float4* vg = reinterpret_cast<const float4*>(V + size_t(g) * M * DENSE_SLOTS);
+      for (int r = r0 + warp; r < r1; r += WARPS * FLY) {
+        uint4 d[FLY];
+        float4 v[FLY][DENSE_SLOTS / 4];
+#pragma unroll
+        for (int u = 0; u < FLY; ++u) {
+          const int ru = r + u * WARPS;
+          const bool live = ru < r1;                            // past the end: zeros times token r
+          d[u] = __ldg(&dy[(long long)(live ? ru : r) * vec_per_row + vcol]);
+#pragma unroll
+          for (int q = 0; q < DENSE_SLOTS / 4; ++q)             // same address in every lane
+            v[u][q] = live ? __ldg(&vg[size_t(ru) * (DENSE_SLOTS / 4) + q]) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < FLY; ++u) {
+#pragma unroll
+          for (int q = 0; q < DENSE_SLOTS / 4; ++q) {
+            fma8(acc[4 * q + 0], v[u][q].x, d[u]);
+            fma8(acc[4 * q + 1], v[u][q].y, d[u]);
+            fma8(acc[4 * q + 2], v[u][q].z, d[u]);
+            fma8(acc[4 * q + 3], v[u][q].w, d[u]);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int b = 0; b < DENSE_SLOTS / 4; ++b) {
+      __syncthreads();                                  // the previous batch has been read
+#pragma unroll
+      for (int sl = 0; sl < 4; ++sl) {
+        *reinterpret_cast<float4*>(&red[warp][sl][8 * lane]) =
+            make_float4(acc[4 * b + sl][0], acc[4 * b + sl][1], acc[4 * b + sl][2], acc[4 * b + sl][3]);
+        *reinterpret_cast<float4*>(&red[warp][sl][8 * lane + 4]) =
+            make_float4(acc[4 * b + sl][4], acc[4 * b + sl][5], acc[4 * b + sl][6], acc[4 * b + sl][7]);
+      }
+      __syncthreads();
+      const int n = blockIdx.x * COMP_COLS + threadIdx.x;
+#pragma unroll
+      for (int sl = 0; sl < 4; ++sl) {
+        const int slot = g * DENSE_SLOTS + 4 * b + sl;
+        if (slot < n_dense && n < N) {
+          float t = 0.0f;
+#pragma unroll
+          for (int w = 0; w < WARPS; ++w) t += red[w][sl][threadIdx.x];
+          dst[(long long)slot * N + n] = t;
+        }
+      }
+    }
+  }
+}
+
+// Dense columns, step 3 (only with more than one chunk): C[slot, n] = sum over the chunks, in order.
+__global__ void __launch_bounds__(256)
+dense_reduce_kernel(float* __restrict__ comp, const float* __restrict__ partial, const int* __restrict__ counts, int N,
+                    int chunks, long long chunk_stride) {
+  const long long total = (long long)counts[0] * N;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    float t = 0.0f;
+    for (int c0 = 0; c0 < chunks; c0 += 8) {            // eight loads in flight, added in chunk order
+      float p[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) p[u] = c0 + u < chunks ? __ldg(&partial[(long long)(c0 + u) * chunk_stride + i]) : 0.0f;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) t += p[u];
+    }
+    comp[i] = t;
   }
 }
 
@@ -188,7 +332,7 @@ comp_wgrad_long_kernel(float* __restrict__ comp, const int* __restrict__ colptr,
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n0 = blockIdx.x * COMP_COLS + 8 * lane;
   const bool in_cols = n0 < N;
-  const int n_cols = *count;
+  const int n_dense = count[0], n_cols = count[1];
   for (int slot = blockIdx.y; slot < n_cols; slot += gridDim.y) {
     const int k = list[slot];
     float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
@@ -204,7 +348,7 @@ comp_wgrad_long_kernel(float* __restrict__ comp, const int* __restrict__ colptr,
 #pragma unroll
         for (int c = 0; c < 8; ++c) t[c] += part[w][lane][c];
       }
-      store8_f32(comp + (long long)slot * N + n0, t);
+      store8_f32(comp + (long long)(n_dense + slot) * N + n0, t);
     }
   }
 }
@@ -217,12 +361,12 @@ comp_wgrad_short_kernel(float* __restrict__ comp, const int* __restrict__ colptr
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n0 = blockIdx.x * COMP_COLS + 8 * lane;
   if (n0 >= N) return;
-  const int n_long = counts[0], n_cols = counts[1];
+  const int n_before = counts[0] + counts[1], n_cols = counts[2];
   for (int slot = blockIdx.y * 8 + warp; slot < n_cols; slot += gridDim.y * 8) {
     const int k = list[slot];
     float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     strided_entries_times_dense(acc, row, val, colptr[k], colptr[k + 1], 1, dy, N >> 3, n0 >> 3);
-    store8_f32(comp + (long long)(n_long + slot) * N + n0, acc);
+    store8_f32(comp + (long long)(n_before + slot) * N + n0, acc);
   }
 }
 
@@ -238,24 +382,65 @@ int launch_comp_fwd(fp4_ctx* ctx, cudaStream_t stream, const float* y1, const in
   return FP4_OK;
 }
 
-int launch_comp_wgrad(fp4_ctx* ctx, cudaStream_t stream, const int32_t* colptr, const int32_t* row, const float* val,
-                      const void* dy_bf16, int* lists, int* slot_of_col, float* comp, int64_t K, int64_t N) {
-  KernelScope scope(ctx, stream, KC_COMP_WGRAD, 3);
-  // lists: [K] long columns, [K] short columns, two counters
+// Chunks of tokens of the dense path: about 2 x 148 blocks in all, at least 64 tokens per chunk.
+static int dense_chunks(int64_t M, int64_t N) {
+  const int n_blocks = int((N + COMP_COLS - 1) / COMP_COLS);
+  int chunks = 296 / n_blocks;
+  chunks = chunks < 1 ? 1 : (chunks > DENSE_MAX_CHUNKS ? DENSE_MAX_CHUNKS : chunks);
+  if (int64_t(chunks) * 64 > M) chunks = int(M / 64) > 0 ? int(M / 64) : 1;
+  return chunks;
+}
+
+size_t comp_wgrad_scratch_bytes(int64_t M, int64_t K, int64_t N) {
+  auto r256 = [](size_t b) { return (b + 255) & ~size_t(255); };
+  size_t b = r256((2 * size_t(K) + 4) * 4) + r256(size_t(K) * 4);                     // lists + counters, slots
+  b += r256(size_t(DENSE_MAX) * size_t(M) * 4);                                       // V
+  b += r256(size_t(dense_chunks(M, N)) * size_t(DENSE_MAX) * size_t(N) * 4);          // partial sums
+  return b;
+}
+
+int launch_comp_wgrad(fp4_ctx* ctx, cudaStream_t stream, const fp4_qtensor* a, const void* dy_bf16, Arena& scratch,
+                      int** slot_of_col_out, float* comp, int64_t M, int64_t K, int64_t N) {
+  // lists: [K] long columns, [K] short columns, three counters
+  int* lists = scratch.take<int>(2 * size_t(K) + 4);
+  int* slot_of_col = scratch.take<int>(size_t(K));
+  float* V = scratch.take<float>(size_t(DENSE_MAX) * size_t(M));
+  const int chunks = dense_chunks(M, N);
+  float* partial = scratch.take<float>(size_t(chunks) * size_t(DENSE_MAX) * size_t(N));
+  if (!scratch.ok) return FP4_ERR_WORKSPACE;
+  *slot_of_col_out = slot_of_col;
   int* list_long = lists;
   int* list_short = lists + K;
   int* counts = lists + 2 * K;
-  nonempty_columns_kernel<<<1, 1024, 0, stream>>>(colptr, int(K), list_long, list_short, counts, slot_of_col);
+  // The dense path pays when the residual is heavy (two launches more, far less traffic): it is
+  // taken when the residual may hold at least 1 % of the activation (alpha <= 0.995), for the
+  // columns that at least a quarter of the tokens hit.
+  const bool dense = a->csr_rowptr && a->sparse_cap * 100 >= M * K;
+  const int dense_from = dense ? int(M / 4 > LONG_COLUMN ? M / 4 : LONG_COLUMN) : INT_MAX;
   const unsigned n_blocks = unsigned((N + COMP_COLS - 1) / COMP_COLS);
+  const int rows_per_chunk = int((M + chunks - 1) / chunks);
+  KernelScope scope(ctx, stream, KC_COMP_WGRAD, 3 + (dense ? (chunks > 1 ? 3 : 2) : 0));
+  nonempty_columns_kernel<<<1, 1024, 0, stream>>>(a->csc_colptr, int(K), dense_from, list_long, list_short, counts,
+                                                  slot_of_col);
   const uint4* dy = static_cast<const uint4*>(dy_bf16);
+  if (dense) {
+    dense_values_kernel<<<unsigned((M + 7) / 8), COMP_THREADS, 0, stream>>>(a->csr_rowptr, a->csr_col, a->csr_val,
+                                                                           slot_of_col, counts, V, int(M));
+    const long long chunk_stride = (long long)DENSE_MAX * N;
+    comp_wgrad_dense_kernel<<<dim3(n_blocks, unsigned(chunks)), COMP_THREADS, 0, stream>>>(
+        chunks > 1 ? partial : comp, V, dy, counts, int(M), int(N), rows_per_chunk, chunk_stride);
+    if (chunks > 1)
+      dense_reduce_kernel<<<unsigned(2 * ctx->num_sms), 256, 0, stream>>>(comp, partial, counts, int(N), chunks,
+                                                                         chunk_stride);
+  }
   unsigned gy = unsigned(4 * ctx->num_sms) / n_blocks;          // long columns: 2 resident blocks per SM
   gy = gy < 1 ? 1 : (gy > unsigned(K) ? unsigned(K) : gy);
-  comp_wgrad_long_kernel<<<dim3(n_blocks, gy), LONG_THREADS, 0, stream>>>(comp, colptr, row, val, dy, list_long,
-                                                                         counts, int(N));
+  comp_wgrad_long_kernel<<<dim3(n_blocks, gy), LONG_THREADS, 0, stream>>>(comp, a->csc_colptr, a->csc_row, a->csc_val,
+                                                                         dy, list_long, counts, int(N));
   gy = unsigned(32 * ctx->num_sms) / n_blocks;                   // short columns: 8 per block
   gy = gy < 1 ? 1 : (gy > unsigned((K + 7) / 8) ? unsigned((K + 7) / 8) : gy);
-  comp_wgrad_short_kernel<<<dim3(n_blocks, gy), COMP_THREADS, 0, stream>>>(comp, colptr, row, val, dy, list_short,
-                                                                           counts, int(N));
+  comp_wgrad_short_kernel<<<dim3(n_blocks, gy), COMP_THREADS, 0, stream>>>(comp, a->csc_colptr, a->csc_row,
+                                                                           a->csc_val, dy, list_short, counts, int(N));
   FP4_CUDA_TRY(cudaGetLastError());
   return FP4_OK;
 }
