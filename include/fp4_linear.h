@@ -19,6 +19,9 @@
  *    two per byte with the even element in bits 3:0.  A negative zero code is never written.
  *  - Calls are asynchronous on `stream` (a cudaStream_t passed as void*).  They return 0 or
  *    a negative FP4_ERR_* code for errors found on the host before anything is enqueued.
+ *  - A context holds one workspace and a few counters that its calls share: the work of two calls
+ *    on the same context must not overlap on the GPU (issue them on one stream, or order the
+ *    streams); use one context per concurrent stream.
  *  - Conditions found on the device are OR-ed into the caller's device word `*status`
  *    (FP4_DEV_* bits).  When a bit is set the outputs are unspecified but every write stayed
  *    inside the caller's buffers.  Every device-side wait is bounded: a stalled pipeline
