@@ -105,10 +105,12 @@ def test_ste_switch_and_dge_parameters(lib, ctx):
     (128, 256, 128, 40, 0.92),     # 40 nearly full columns
     (512, 256, 384, 20, 0.98),     # 20 nearly full columns of 512 entries: long columns, many rounds per warp
     (256, 384, 128, 3, 0.999),     # few entries: short columns only
+    (1024, 512, 256, 200, 0.78),   # 200 full columns of 1024 entries: more than the dense class takes (160); the rest are long
+    (1024, 256, 384, 12, 0.97),    # 12 full columns: dense class (two passes of 8), several chunks of tokens
 ])
 def test_weight_gradient_compensation_column_classes(lib, ctx, M, K, N, hot, alpha):
-    """The compensation of the weight gradient treats long and short residual columns differently;
-    both must give the oracle's sums, run to run identically."""
+    """The compensation of the weight gradient treats dense, long and short residual columns
+    differently; all must give the oracle's sums, run to run identically."""
     a_bits, w_bits, dy_bits = WL.small_case(M, K, N, seed=hot, alpha_outliers=hot)
     f = O.linear_fwd(a_bits, w_bits, alpha)
     b = O.linear_bwd(dy_bits, w_bits, f)
@@ -120,8 +122,8 @@ def test_weight_gradient_compensation_column_classes(lib, ctx, M, K, N, hot, alp
     torch.cuda.synchronize()
     assert ctx.read_status() == 0
     counts = np.diff(sa.csc_colptr.cpu().numpy())
-    if hot >= 20:
-        assert (counts >= 64).sum() >= hot // 2                       # the case does reach the long-column kernel
+    if M >= 1024:
+        assert (counts >= 512).sum() >= hot // 2                      # the case does reach the dense / long classes
     assert np.abs(b.s_comp).max() > 0
     assert_close_f32(dw.cpu().numpy(), b.dw, b.s_fp4 * b.dge, b.s_comp * b.dge, "dW")
     assert torch.equal(dw, dw_again)                                   # fixed summation order

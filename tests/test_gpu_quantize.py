@@ -128,6 +128,23 @@ def test_occ_quantize_matches_oracle(lib, ctx, shape, alpha, dist):
     _check_dense(q, ref)
 
 
+def test_occ_tall_tensor_many_rows_per_block(lib, ctx):
+    """81 920 rows of 128: more rows per histogram block than its shared row slots hold at once, so
+    the row extremes are reduced in several batches."""
+    rows, cols, alpha = 81920, 128, 0.999
+    cfg = WL.Config(51, "tall", rows, (), "normal", 2, 40.0, "channels_count", (alpha,))
+    bits = WL.activations(cfg, cols, seed=2, layer=7)
+    big = lib.Context(0, int(lib.load_library().fp4_workspace_bytes(rows, cols, 128)))
+    big.status.zero_()
+    q = lib.fp4_quantize(big, _dev(bits), 0, alpha=alpha)
+    torch.cuda.synchronize()
+    assert big.read_status() == 0
+    ref = O.occ_quantize(O.bf16_bits_to_f64(bits), alpha)
+    _check_sparse(q, ref)
+    _check_dense(q, ref)
+    big.close()
+
+
 def test_occ_with_heavy_ties_and_zeros(lib, ctx):
     """Few distinct values: thresholds sit on big ties (entries equal to a threshold carry no
     residual), one bin holds far more than 2^16 entries, and lo is a zero."""
