@@ -42,11 +42,14 @@ __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w 
 // ------------------------------------------------------------------------------------------
 // Exact histogram with 32-bit shared-memory counters over a window of HIST_EXPS binary exponents
 // (both signs, all 128 mantissas): real tensors spread over far fewer exponents than BF16 offers.
-// Each block places its window just above the largest magnitude of its first 8192 elements.
+// Each block places its window HIST_HEADROOM binades above the largest magnitude of its first 8192
+// elements.  A vector of eight elements is tested against the window as a whole (four packed BF16
+// comparisons); if all eight are inside, each costs one extraction, one address and one increment.
 // Patterns outside the window (tiny values, later giants) go straight to the global histogram and
 // exact zeros are counted in registers, so every element is counted exactly once.  The window is
 // replicated HIST_COPIES times (one copy per group of warps) to thin out same-address conflicts;
-// the increments return no value and need no overflow handling.
+// the increments return no value and need no overflow handling.  What bounds the loop is the
+// shared-memory pipe: the increments of a warp fall into random banks.
 //
 // A block owns whole rows (a contiguous range of them), so the signed max / min of a row are
 // reduced in shared memory and written with plain stores, as is the zero that starts the row's
@@ -60,9 +63,16 @@ __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w 
 // end, so the set a call counts into is always zero and no separate clearing pass exists.  With
 // `parity` null (the allocation-free entry point, which clears its one set itself) set 0 is used.
 constexpr int HIST_EXPS = 24;
-constexpr int HIST_BINS = HIST_EXPS * 128 * 2;     // 6144 counters per copy
-constexpr int HIST_COPIES = 8;
-constexpr int HIST_SMEM_BYTES = HIST_BINS * HIST_COPIES * 4;
+constexpr int HIST_WINDOW = HIST_EXPS * 128;       // 3072 magnitudes in the window, per sign
+constexpr int HIST_COPIES = 4;
+constexpr int HIST_HEADROOM = 1;                   // binades between the sample's maximum and the window's top
+constexpr int HIST_FLY = 4;                        // vectors a lane loads per unit
+constexpr int HIST_CHUNK = 32 * HIST_FLY;          // vectors of one row a warp takes at a time
+// Counter of pattern b in copy c: word c * HIST_WINDOW + (b - base).  The sign bit of b is left in
+// place, so the negative half of every copy lies 0x8000 words (128 KB) above its positive half and
+// the index of an element is its pattern minus a constant; the words between the halves are unused.
+constexpr int HIST_NEG_WORD = 0x8000;
+constexpr int HIST_SMEM_BYTES = (HIST_NEG_WORD + HIST_COPIES * HIST_WINDOW) * 4;
 constexpr int HIST_ROW_SLOTS = 512;                // rows whose extremes a block reduces at a time
 constexpr int HIST_COARSE = 32;                    // coarse counters: 2048 positions each
 constexpr int HIST_SET_WORDS = 65536 + HIST_COARSE; // one set: fine counters, then coarse counters
@@ -106,6 +116,15 @@ hist_select_kernel(const uint4* __restrict__ x, int rows, int vec_per_row, uint3
   __shared__ uint32_t s_coarse[HIST_COARSE];
   __shared__ int s_last;
   const int tid = threadIdx.x;
+  const int r_begin = int((long long)rows * blockIdx.x / gridDim.x);
+  const int r_end = int((long long)rows * (blockIdx.x + 1) / gridDim.x);
+  const int lane = tid & 31;
+  // sample for the window's top, issued first: its latency hides behind the clearing below
+  uint4 sample = make_uint4(0, 0, 0, 0);
+  {
+    const long long i0 = (long long)r_begin * vec_per_row + tid;
+    if (i0 < (long long)r_end * vec_per_row) sample = __ldg(&x[i0]);
+  }
   const unsigned par = parity ? (*reinterpret_cast<volatile unsigned*>(parity) & 1u) : 0u;
   uint32_t* ghist = sets + size_t(par) * HIST_SET_WORDS;
   uint32_t* gcoarse = ghist + 65536;
@@ -117,33 +136,36 @@ hist_select_kernel(const uint4* __restrict__ x, int rows, int vec_per_row, uint3
     for (int i = w0 + tid; i < w1; i += HIST_THREADS) other[i] = 0;
   }
   {
-    uint4* h4 = reinterpret_cast<uint4*>(h);
-    for (int i = tid; i < HIST_BINS * HIST_COPIES / 4; i += HIST_THREADS) h4[i] = make_uint4(0, 0, 0, 0);
+    uint4* pos4 = reinterpret_cast<uint4*>(h);
+    uint4* neg4 = reinterpret_cast<uint4*>(h + HIST_NEG_WORD);
+    for (int i = tid; i < HIST_WINDOW * HIST_COPIES / 4; i += HIST_THREADS)
+      pos4[i] = neg4[i] = make_uint4(0, 0, 0, 0);
   }
   if (tid < HIST_COARSE) s_coarse[tid] = 0;
   if (tid == 0) s_top = 0;
   __syncthreads();
-  const int r_begin = int((long long)rows * blockIdx.x / gridDim.x);
-  const int r_end = int((long long)rows * (blockIdx.x + 1) / gridDim.x);
-  const long long v_end_all = (long long)r_end * vec_per_row;
   {
     // window top: largest exponent-and-mantissa field among this block's first vectors
-    const long long i0 = (long long)r_begin * vec_per_row + tid;
+    const uint32_t w[4] = {sample.x, sample.y, sample.z, sample.w};
     uint32_t m = 0;
-    if (i0 < v_end_all) {
-      const uint4 v = __ldg(&x[i0]);
-      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-      for (int q = 0; q < 4; ++q) m = max(m, max(w[q] & 0x7FFFu, (w[q] >> 16) & 0x7FFFu));
-    }
+    for (int q = 0; q < 4; ++q) m = max(m, max(w[q] & 0x7FFFu, (w[q] >> 16) & 0x7FFFu));
     m = __reduce_max_sync(0xFFFFFFFFu, m);
-    if ((tid & 31) == 0) atomicMax(&s_top, m);
+    if ((tid & 31) == 0 && m) atomicMax(&s_top, m);
   }
   __syncthreads();
-  // window = exponents [e_top - HIST_EXPS + 1, e_top] with e_top four binades above the sample's maximum
-  const int e_top = min(254, int(s_top >> 7) + 4);
+  // window = exponents [e_top - HIST_EXPS + 1, e_top] with e_top HIST_HEADROOM binades above the sample's
+  // maximum (what lies above the window is counted in global memory like what lies below it)
+  const int e_top = min(254, int(s_top >> 7) + HIST_HEADROOM);
   const uint32_t base = uint32_t(max(0, e_top - HIST_EXPS + 1)) << 7;
-  uint32_t* my_h = h + ((tid >> 5) & (HIST_COPIES - 1)) * HIST_BINS;
+  // The window's bounds as BF16 numbers (magnitudes order like their patterns; the upper bound is at
+  // most the pattern of infinity, and a NaN fails every comparison)
+  const __nv_bfloat162 lo_bf = __halves2bfloat162(__ushort_as_bfloat16((unsigned short)base),
+                                                  __ushort_as_bfloat16((unsigned short)base));
+  const __nv_bfloat162 hi_bf = __halves2bfloat162(__ushort_as_bfloat16((unsigned short)(base + HIST_WINDOW)),
+                                                  __ushort_as_bfloat16((unsigned short)(base + HIST_WINDOW)));
+  // this warp's copy: counter of pattern b at word b + my_off
+  const int my_off = ((tid >> 5) & (HIST_COPIES - 1)) * HIST_WINDOW - int(base);
   uint32_t zeros_pos = 0, zeros_neg = 0;
   bool nonfinite = false;
   for (int r0 = r_begin; r0 < r_end; r0 += HIST_ROW_SLOTS) {
@@ -153,48 +175,69 @@ hist_select_kernel(const uint4* __restrict__ x, int rows, int vec_per_row, uint3
       s_rmin[r] = INT_MAX;
     }
     __syncthreads();
-    const long long v_end = (long long)r1 * vec_per_row;
-    long long i = (long long)r0 * vec_per_row + tid;
-    // row of vector i relative to r0, advanced incrementally (one division per thread and batch)
-    int row = tid / vec_per_row, rem = tid - row * vec_per_row;
-    const int row_step = HIST_THREADS / vec_per_row, rem_step = HIST_THREADS - row_step * vec_per_row;
-    uint4 nxt = make_uint4(0, 0, 0, 0);
-    if (i < v_end) nxt = __ldg(&x[i]);
-    for (; i < v_end; i += HIST_THREADS) {
-      const uint4 v = nxt;
-      if (i + HIST_THREADS < v_end) nxt = __ldg(&x[i + HIST_THREADS]);
-      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    // A unit is a stretch of up to HIST_CHUNK consecutive vectors of one row; warp w takes units
+    // w, w + 32, ...  A lane loads its HIST_FLY vectors of the unit (vectors lane, lane + 32, ... of
+    // the stretch) before it counts any of them, keeps the unit's extremes packed in two registers,
+    // and the warp reduces them once per unit.
+    const int chunks_per_row = (vec_per_row + HIST_CHUNK - 1) / HIST_CHUNK;
+    const int units = (r1 - r0) * chunks_per_row;
+    for (int u = tid >> 5; u < units; u += HIST_THREADS / 32) {
+      const int row = u / chunks_per_row;
+      const int v0 = (u - row * chunks_per_row) * HIST_CHUNK;
+      const int mine = min(HIST_CHUNK, vec_per_row - v0) - lane;       // vectors lane, lane + 32, ... below this
+      const uint4* px = x + ((long long)(r0 + row) * vec_per_row + v0 + lane);
+      uint4 vv[HIST_FLY];
 #pragma unroll
-      for (int q = 0; q < 8; ++q) {
-        const uint32_t bits = (q & 1) ? (w[q >> 1] >> 16) : (w[q >> 1] & 0xFFFFu);
-        const uint32_t m15 = bits & 0x7FFFu;
-        const uint32_t off = m15 - base;
-        if (off < uint32_t(HIST_EXPS * 128)) {
-          atomicAdd(&my_h[2 * off + (bits >> 15)], 1u);
-        } else if (m15 == 0) {
-          if (bits) ++zeros_neg; else ++zeros_pos;
-        } else {
-          atomicAdd(&ghist[bits], 1u);
-          atomicAdd(&s_coarse[bits_to_pos(bits) >> 11], 1u);
-          if (m15 >= 0x7F80u) nonfinite = true;         // infinity or NaN: always outside the window
+      for (int k = 0; k < HIST_FLY; ++k)
+        if (32 * k < mine) vv[k] = __ldg(px + 32 * k);
+      __nv_bfloat162 umax = __float2bfloat162_rn(-INFINITY), umin = __float2bfloat162_rn(INFINITY);
+#pragma unroll
+      for (int k = 0; k < HIST_FLY; ++k) {
+        if (32 * k >= mine) break;
+        const uint32_t w[4] = {vv[k].x, vv[k].y, vv[k].z, vv[k].w};
+        const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(w);
+        // all eight magnitudes inside the window?  (half-precision comparisons: they leave the
+        // integer pipe to the index arithmetic)
+        bool inside = true;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const __nv_bfloat162 mag = __habs2(p[q]);
+          inside = inside && __hbge2(mag, lo_bf) && __hblt2(mag, hi_bf);
         }
+        if (inside) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            atomicAdd(&h[int(w[q] & 0xFFFFu) + my_off], 1u);
+            atomicAdd(&h[int(w[q] >> 16) + my_off], 1u);
+          }
+        } else {
+#pragma unroll 1
+          for (int e = 0; e < 8; ++e) {
+            const uint32_t word = (e & 4) ? ((e & 2) ? w[3] : w[2]) : ((e & 2) ? w[1] : w[0]);
+            const uint32_t bits = (e & 1) ? (word >> 16) : (word & 0xFFFFu);
+            const uint32_t m15 = bits & 0x7FFFu;
+            if (m15 - base < uint32_t(HIST_WINDOW)) {
+              atomicAdd(&h[int(bits) + my_off], 1u);
+            } else if (m15 == 0) {
+              if (bits) ++zeros_neg; else ++zeros_pos;
+            } else {
+              atomicAdd(&ghist[bits], 1u);
+              atomicAdd(&s_coarse[bits_to_pos(bits) >> 11], 1u);
+              if (m15 >= 0x7F80u) nonfinite = true;       // infinity or NaN: always outside the window
+            }
+          }
+        }
+        umax = __hmax2(umax, __hmax2(__hmax2(p[0], p[1]), __hmax2(p[2], p[3])));
+        umin = __hmin2(umin, __hmin2(__hmin2(p[0], p[1]), __hmin2(p[2], p[3])));
       }
-      const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(w);
-      const __nv_bfloat162 mx = __hmax2(__hmax2(p[0], p[1]), __hmax2(p[2], p[3]));
-      const __nv_bfloat162 mn = __hmin2(__hmin2(p[0], p[1]), __hmin2(p[2], p[3]));
-      int kmax = float_to_ordered(fmaxf(__low2float(mx), __high2float(mx)));
-      int kmin = float_to_ordered(fminf(__low2float(mn), __high2float(mn)));
-      // 16 consecutive vectors (128 elements) never straddle a row: cols is a multiple of 128
-      const unsigned group = (tid & 16) ? 0xFFFF0000u : 0x0000FFFFu;
-      kmax = __reduce_max_sync(group, kmax);
-      kmin = __reduce_min_sync(group, kmin);
-      if ((tid & 15) == 0) {
+      int kmax = float_to_ordered(fmaxf(__low2float(umax), __high2float(umax)));
+      int kmin = float_to_ordered(fminf(__low2float(umin), __high2float(umin)));
+      kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+      kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+      if (lane == 0) {
         atomicMax(&s_rmax[row], kmax);
         atomicMin(&s_rmin[row], kmin);
       }
-      row += row_step;
-      rem += rem_step;
-      if (rem >= vec_per_row) { rem -= vec_per_row; ++row; }
     }
     __syncthreads();
     for (int r = tid; r < r1 - r0; r += HIST_THREADS) {
@@ -211,12 +254,13 @@ hist_select_kernel(const uint4* __restrict__ x, int rows, int vec_per_row, uint3
     if (zeros_pos) { atomicAdd(&ghist[0x0000], zeros_pos); atomicAdd(&s_coarse[bits_to_pos(0x0000u) >> 11], zeros_pos); }
     if (zeros_neg) { atomicAdd(&ghist[0x8000], zeros_neg); atomicAdd(&s_coarse[bits_to_pos(0x8000u) >> 11], zeros_neg); }
   }
-  for (int idx = tid; idx < HIST_BINS; idx += HIST_THREADS) {
+  for (int idx = tid; idx < 2 * HIST_WINDOW; idx += HIST_THREADS) {
+    const int neg = idx >= HIST_WINDOW, off = idx - neg * HIST_WINDOW;
     uint32_t c = 0;
 #pragma unroll
-    for (int r = 0; r < HIST_COPIES; ++r) c += h[r * HIST_BINS + idx];
+    for (int r = 0; r < HIST_COPIES; ++r) c += h[neg * HIST_NEG_WORD + r * HIST_WINDOW + off];
     if (c) {
-      const uint32_t bits = (uint32_t(idx & 1) << 15) | (base + uint32_t(idx >> 1));
+      const uint32_t bits = (uint32_t(neg) << 15) | (base + uint32_t(off));
       atomicAdd(&ghist[bits], c);
       atomicAdd(&s_coarse[bits_to_pos(bits) >> 11], c);
     }
@@ -230,10 +274,14 @@ hist_select_kernel(const uint4* __restrict__ x, int rows, int vec_per_row, uint3
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  if (tid < 64) {
-    // warp q finds rank q: the coarse range first (one counter per lane), then the range's 2048
-    // fine counters in 16 steps of 128 consecutive positions (4 per lane, all loads issued at once)
-    const int q = tid >> 5, lane = tid & 31;
+  {
+    // Rank q (0: lower, 1: upper) is served by warps 16 q .. 16 q + 15.  Every warp finds the rank's
+    // coarse range (one coarse counter per lane), then warp st of the 16 reads step st of the range's
+    // 2048 fine counters: 128 consecutive positions, 4 per lane.  The step totals meet in shared
+    // memory; the warp whose step holds the rank writes the threshold.
+    static_assert(HIST_THREADS == 1024, "two ranks x sixteen steps, one warp each");
+    __shared__ long long s_step[2][16];
+    const int warp = tid >> 5, lane = tid & 31, q = warp >> 4, st = warp & 15;
     const long long rank = q == 0 ? n_tail : n - 1 - n_tail;
     const long long cc = __ldcg(&gcoarse[lane]);
     long long sc = cc;
@@ -243,46 +291,32 @@ hist_select_kernel(const uint4* __restrict__ x, int rows, int vec_per_row, uint3
       if (lane >= off) sc += up;
     }
     const unsigned holds = __ballot_sync(0xFFFFFFFFu, rank >= sc - cc && rank < sc);   // exactly one lane
-    const int region = __ffs(holds) - 1;
+    const int region = holds ? __ffs(holds) - 1 : 0;
     long long run = __shfl_sync(0xFFFFFFFFu, sc - cc, region);                          // counts before the range
     // positions of the range in ascending order; in memory they ascend (region >= 16) or descend
     const bool desc = region < 16;
     const uint32_t* first = ghist + (desc ? (0xFFFF - 2048 * region - 2047) : 2048 * (region - 16));
-    bool done = false;
-#pragma unroll 1
-    for (int half = 0; half < 2; ++half) {              // eight steps' loads in flight at a time
-      uint4 c[8];
+    const int word = desc ? (2048 - 128 * st - 4 * lane - 4) : (128 * st + 4 * lane);
+    const uint4 c = __ldcg(reinterpret_cast<const uint4*>(first + word));
+    // in ascending position order
+    const long long v0 = desc ? c.w : c.x, v1 = desc ? c.z : c.y;
+    const long long v2 = desc ? c.y : c.z, v3 = desc ? c.x : c.w;
+    const long long mine = v0 + v1 + v2 + v3;
+    long long incl = mine;
 #pragma unroll
-      for (int s8 = 0; s8 < 8; ++s8) {
-        // step st covers positions 128 st .. 128 st + 127 of the range; lane l its positions 4 l .. 4 l + 3
-        const int st = 8 * half + s8;
-        const int word = desc ? (2048 - 128 * st - 4 * lane - 4) : (128 * st + 4 * lane);
-        c[s8] = __ldcg(reinterpret_cast<const uint4*>(first + word));
-      }
-#pragma unroll
-      for (int s8 = 0; s8 < 8; ++s8) {
-        const int st = 8 * half + s8;
-        // in ascending position order
-        const long long v0 = desc ? c[s8].w : c[s8].x, v1 = desc ? c[s8].z : c[s8].y;
-        const long long v2 = desc ? c[s8].y : c[s8].z, v3 = desc ? c[s8].x : c[s8].w;
-        const long long mine = v0 + v1 + v2 + v3;
-        long long incl = mine;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-          const long long up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-          if (lane >= off) incl += up;
-        }
-        const long long before = run + incl - mine;
-        if (!done && rank >= before && rank < before + mine) {
-          const int p0 = 2048 * region + 128 * st + 4 * lane;
-          const int k = rank < before + v0 ? 0 : (rank < before + v0 + v1 ? 1 : (rank < before + v0 + v1 + v2 ? 2 : 3));
-          const uint32_t bits = pos_to_bits(p0 + k);
-          thresholds[q] = __uint_as_float((bits == 0x8000u ? 0u : bits) << 16);   // thresholds are real numbers: -0 is +0
-        }
-        const long long total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-        done = done || rank < run + total;
-        run += total;
-      }
+    for (int off = 1; off < 32; off <<= 1) {
+      const long long up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+      if (lane >= off) incl += up;
+    }
+    if (lane == 31) s_step[q][st] = incl;
+    __syncthreads();
+    for (int j = 0; j < st; ++j) run += s_step[q][j];
+    const long long before = run + incl - mine;
+    if (holds && rank >= before && rank < before + mine) {
+      const int p0 = 2048 * region + 128 * st + 4 * lane;
+      const int k = rank < before + v0 ? 0 : (rank < before + v0 + v1 ? 1 : (rank < before + v0 + v1 + v2 ? 2 : 3));
+      const uint32_t bits = pos_to_bits(p0 + k);
+      thresholds[q] = __uint_as_float((bits == 0x8000u ? 0u : bits) << 16);   // thresholds are real numbers: -0 is +0
     }
   }
   __syncthreads();
