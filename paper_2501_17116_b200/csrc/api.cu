@@ -484,10 +484,11 @@ extern "C" {
 
 size_t fp4_step_host_workspace_bytes(int64_t M, int64_t K, int64_t N, double alpha) {
   if (M <= 0 || K <= 0 || N <= 0) return 0;
-  // Sized so that the pipelined layout fits: four slots (two input sets, two output sets) of an
-  // eighth each, everything else in the second half.
+  // Sized so that the pipelined layout fits: 2 HOST_STEP_SETS slots (input sets, then output sets)
+  // in the first half, everything else in the second half.
   const size_t io = step_host_io_bytes(M, K, N), shared = step_host_shared_bytes(M, K, N, alpha);
-  return (8 * io > 2 * shared ? 8 * io : 2 * shared) + 1024;
+  const size_t slots = 4 * HOST_STEP_SETS * io;
+  return (slots > 2 * shared ? slots : 2 * shared) + 1024;
 }
 
 int fp4_linear_step_host(fp4_ctx* ctx, void* stream, const void* A_host, const void* W_host, const void* dY_host,
@@ -504,20 +505,21 @@ int fp4_linear_step_host(fp4_ctx* ctx, void* stream, const void* A_host, const v
   if (2 * io_bytes + shared_bytes > ctx->workspace_bytes) return FP4_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-  // Workspace layout.  Pipelined: four slots of an eighth of the workspace each -- input sets 0, 1
-  // and output sets 0, 1 -- and everything else (saved operands, scratch) in the second half.
-  // Call i uses set i % 2: its inputs travel on the context's copy stream while call i - 1 still
+  // Workspace layout.  Pipelined: 2 HOST_STEP_SETS slots in the first half of the workspace -- the
+  // input sets, then the output sets -- and everything else (saved operands, scratch) in the second
+  // half.  Call i uses set i % HOST_STEP_SETS: its inputs travel on the context's copy stream while call i - 1 still
   // computes, its kernels run on the context's compute stream while call i - 1 copies back on the
   // context's return stream, and `stream` waits for the copies back.  A call whose tensors do not
   // fit that layout carves the whole workspace from its start, runs on `stream` alone and is
   // ordered after everything earlier calls left in flight.
-  const size_t slot = (ctx->workspace_bytes / 8) & ~size_t(255);
-  const bool pipelined = ctx->overlap && io_bytes <= slot && shared_bytes <= ctx->workspace_bytes - 4 * slot;
+  constexpr int SETS = HOST_STEP_SETS;
+  const size_t slot = (ctx->workspace_bytes / (4 * SETS)) & ~size_t(255);
+  const bool pipelined = ctx->overlap && io_bytes <= slot && shared_bytes <= ctx->workspace_bytes - 2 * SETS * slot;
   const int set = ctx->host_step_parity;
   Arena in_arena = pipelined ? Arena(ctx->workspace + size_t(set) * slot, slot) : Arena(ctx->workspace, io_bytes);
-  Arena out_arena = pipelined ? Arena(ctx->workspace + size_t(2 + set) * slot, slot)
+  Arena out_arena = pipelined ? Arena(ctx->workspace + size_t(SETS + set) * slot, slot)
                               : Arena(ctx->workspace + io_bytes, io_bytes);
-  Arena arena = pipelined ? Arena(ctx->workspace + 4 * slot, ctx->workspace_bytes - 4 * slot)
+  Arena arena = pipelined ? Arena(ctx->workspace + 2 * SETS * slot, ctx->workspace_bytes - 2 * SETS * slot)
                           : Arena(ctx->workspace + 2 * io_bytes, ctx->workspace_bytes - 2 * io_bytes);
   const size_t a_bytes = size_t(M) * K * 2, w_bytes = size_t(K) * N * 2, y_bytes = size_t(M) * N * 2;
   char* dA_in = in_arena.take<char>(a_bytes);
@@ -540,11 +542,14 @@ int fp4_linear_step_host(fp4_ctx* ctx, void* stream, const void* A_host, const v
     s_out = ctx->return_stream;
     // The copies in do not wait for `stream`: it carries the previous call's copies back, which
     // they are meant to overlap.  The host inputs must therefore be ready when the call is made.
-    // both slots of this set were last used by the call before the previous one
-    FP4_CUDA_TRY(cudaStreamWaitEvent(s_in, ctx->host_step_done[set], 0));
+    // Both slots of this set were last used HOST_STEP_SETS calls ago: that call's kernels have
+    // to be done with the input slot before the copies in start, its copies back with the output
+    // slot before this call's kernels start -- the copies in do not wait for those copies back, so
+    // the two copy directions both stay busy.
+    FP4_CUDA_TRY(cudaStreamWaitEvent(s_in, ctx->host_step_computed[set], 0));
+    FP4_CUDA_TRY(cudaStreamWaitEvent(s_cmp, ctx->host_step_done[set], 0));
   } else {
-    FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->host_step_done[0], 0));
-    FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->host_step_done[1], 0));
+    for (int i = 0; i < SETS; ++i) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->host_step_done[i], 0));
   }
   FP4_CUDA_TRY(cudaMemcpyAsync(dA_in, A_host, a_bytes, cudaMemcpyHostToDevice, s_in));
   FP4_CUDA_TRY(cudaMemcpyAsync(dW_in, W_host, w_bytes, cudaMemcpyHostToDevice, s_in));
@@ -570,11 +575,13 @@ int fp4_linear_step_host(fp4_ctx* ctx, void* stream, const void* A_host, const v
   if (pipelined) {
     FP4_CUDA_TRY(cudaEventRecord(ctx->host_step_done[set], s_out));
     FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->host_step_done[set], 0));
-    ctx->host_step_parity ^= 1;
+    ctx->host_step_parity = (set + 1) % SETS;
   } else {
     // later pipelined calls may use either set only after this call has left the workspace
-    FP4_CUDA_TRY(cudaEventRecord(ctx->host_step_done[0], st));
-    FP4_CUDA_TRY(cudaEventRecord(ctx->host_step_done[1], st));
+    for (int i = 0; i < SETS; ++i) {
+      FP4_CUDA_TRY(cudaEventRecord(ctx->host_step_done[i], st));
+      FP4_CUDA_TRY(cudaEventRecord(ctx->host_step_computed[i], st));
+    }
   }
   if (status_host) FP4_CUDA_TRY(cudaStreamSynchronize(st));
   return FP4_OK;

@@ -28,6 +28,11 @@ struct ProfRecord {
   cudaEvent_t start, stop;
 };
 
+// fp4_linear_step_host keeps this many sets of device input and output buffers in flight.  Two keep
+// both copy directions busy (measured: a third set changes nothing, the copies back are never short
+// of finished outputs for long).
+constexpr int HOST_STEP_SETS = 2;
+
 struct fp4_ctx {
   int      device;
   int      num_sms;
@@ -41,9 +46,9 @@ struct fp4_ctx {
   cudaStream_t copy_stream;          // host-to-device copies of a call's inputs
   cudaStream_t compute_stream;       // its kernels
   cudaStream_t return_stream;        // device-to-host copies of its outputs
-  cudaEvent_t  host_step_copied[2];  // the inputs of set i have arrived
-  cudaEvent_t  host_step_computed[2];// the outputs of set i are complete on the device
-  cudaEvent_t  host_step_done[2];    // the call that used set i has left the workspace
+  cudaEvent_t  host_step_copied[HOST_STEP_SETS];  // the inputs of set i have arrived
+  cudaEvent_t  host_step_computed[HOST_STEP_SETS];// the outputs of set i are complete on the device
+  cudaEvent_t  host_step_done[HOST_STEP_SETS];    // the call that used set i has left the workspace
   int      host_step_parity;         // set of the next pipelined call
   int      overlap;            // run independent kernel chains on the side streams (default on)
   int      gemm_pairs;         // MXF4 GEMM on pairs of CTAs (tcgen05 cta_group::2)
