@@ -25,6 +25,7 @@ size_t linear_scratch_bytes(int64_t M, int64_t K, int64_t N) {
   b += round256(size_t(M) * 4) + round256(size_t(N) * 4);   // their amax vectors
   b += 2 * round256(size_t(M > N ? M : N) * 4);       // de-scale vectors used as prescale
   b += comp_wgrad_scratch_bytes(M, K, N);             // non-empty residual columns, dense-column buffers
+  b += fwd_tail_scratch_bytes(M, K, N);               // operands of the forward GEMM's dense tail
   return b;
 }
 
@@ -253,6 +254,11 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
   float* y1 = occ ? arena.take<float>(size_t(M) * size_t(N)) : nullptr;
   char* scratch_a = reuse_a ? nullptr : arena.take<char>(quantize_scratch_bytes(M, K));
   char* scratch_w = reuse_w ? nullptr : arena.take<char>(quantize_scratch_bytes(K, N));
+  // A heavy residual (the caller's capacity says it may hold at least 1 % of the activation, alpha <=
+  // 0.995) sends its hot columns through the GEMM as a dense tail instead of per-entry gathers.
+  const bool tail_on = occ && !ctx->gemm_pairs && savedA->csr_rowptr && savedA->csc_colptr &&
+                       savedA->sparse_cap * 100 >= M * K;
+  char* scratch_tail = tail_on ? arena.take<char>(fwd_tail_scratch_bytes(M, K, N)) : nullptr;
   if (!arena.ok) return FP4_ERR_WORKSPACE;
   int rc;
 
@@ -297,12 +303,26 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
     return launch_gemm_fp4(ctx, st, savedA->codes, savedW->codes_t, M, N, K, savedA->amax, savedW->amax, Y, out_f32,
                            gemm_kind, status, nullptr, a8, w8);
   }
+  GemmTail tail = {nullptr, nullptr, nullptr};
+  const int* hot_slot_of_col = nullptr;
+  if (tail_on) {
+    // The tail's operands need the CSR, the CSC's column pointers and W's amax: both sparse chains
+    // are joined before the GEMM here (without a tail they run beside it).
+    if (!reuse_a && ov) {
+      FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[3], 0));
+      FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[7], 0));
+    }
+    Arena ta(scratch_tail, fwd_tail_scratch_bytes(M, K, N));
+    rc = launch_fwd_tail(ctx, st, savedA, W_bf16, savedW->amax, w8 ? 448.0f : 6.0f, ta, M, K, N, &tail, &hot_slot_of_col);
+    if (rc != FP4_OK) return rc;
+  }
   rc = launch_gemm_fp4(ctx, st, savedA->codes, savedW->codes_t, M, N, K, savedA->amax, savedW->amax, y1, 1, gemm_kind,
-                       status, nullptr, a8, w8);
+                       status, nullptr, a8, w8, tail_on ? &tail : nullptr);
   if (rc != FP4_OK) return rc;
   // Y = store(Y1 + (A - A_c) W): one rounding of the fp32 sum.  Needs the CSR.
   if (!reuse_a && ov) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[3], 0));
-  rc = launch_comp_fwd(ctx, st, y1, savedA->csr_rowptr, savedA->csr_col, savedA->csr_val, W_bf16, M, K, N, Y, out_f32);
+  rc = launch_comp_fwd(ctx, st, y1, savedA->csr_rowptr, savedA->csr_col, savedA->csr_val, W_bf16, M, K, N, Y, out_f32,
+                       hot_slot_of_col, tail.count);
   if (rc != FP4_OK) return rc;
   if (!reuse_a && ov) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[7], 0));  // the CSC too: savedA is complete on return
   return FP4_OK;

@@ -132,13 +132,31 @@ struct GemmEpilogue {
   float dge_k, dge_clip;
 };
 
+// Dense tail of the forward GEMM: the residual's hot columns (outlier channels, Appendix D) as extra
+// contraction columns on the tensor cores instead of per-entry gathers.  With h <= TAIL_MAX_COLS hot
+// columns, `a` is [I x TAIL_WIDTH] and `b` [J x TAIL_WIDTH] FP16, row-major, made of blocks of 64
+// columns: for every 64 hot columns the blocks (A_hi, A_hi, A_lo) and (B_hi, B_lo, B_hi), where
+// x_hi + x_lo is the two-term FP16 split of the fp32 value x, so that the three products sum to
+// A B up to 2^-21.  A = residual / (row de-scale * 256), B = 256 * weight / column de-scale: the
+// epilogue's de-scales then turn the tail's sum into residual x weight.  *count (device) is h; 0
+// switches the tail off.
+constexpr int TAIL_MAX_COLS = 128;
+constexpr int TAIL_WIDTH = 3 * TAIL_MAX_COLS;
+constexpr float TAIL_SCALE = 256.0f;
+struct GemmTail {
+  const void* a;
+  const void* b;
+  const int* count;
+};
+
 // ---- internal launchers (each enqueues on `stream`, returns an FP4_* host code) -------------
 
 // out[i,j] = (sum_c a[i,c] b[j,c]) * (row_amax[i]/6) * (col_amax[j]/6)
 int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, const uint8_t* b_codes,
                     int64_t I, int64_t J, int64_t C, const float* row_amax, const float* col_amax,
                     void* out, int out_f32, int gemm_kind, int32_t* status,
-                    const GemmEpilogue* epilogue = nullptr, bool a_e4m3 = false, bool b_e4m3 = false);
+                    const GemmEpilogue* epilogue = nullptr, bool a_e4m3 = false, bool b_e4m3 = false,
+                    const GemmTail* tail = nullptr);
 
 // One GEMM, for launches that take two of them.
 struct Fp4GemmDesc {
@@ -192,7 +210,13 @@ int launch_quantize_dual(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const 
 // y[m,:] = store( y1[m,:] + sum_{entries of row m} val * dense[col,:] )
 int launch_comp_fwd(fp4_ctx* ctx, cudaStream_t stream, const float* y1, const int32_t* rowptr,
                     const int32_t* col, const float* val, const void* w_bf16, int64_t M, int64_t K,
-                    int64_t N, void* y, int out_f32);
+                    int64_t N, void* y, int out_f32, const int* slot_of_col = nullptr,
+                    const int* tail_count = nullptr);
+// The forward GEMM's dense tail (see GemmTail): operands built from the saved activation and the weights.
+size_t fwd_tail_scratch_bytes(int64_t M, int64_t K, int64_t N);
+int launch_fwd_tail(fp4_ctx* ctx, cudaStream_t stream, const fp4_qtensor* a, const void* w_bf16, const float* w_amax,
+                    float w_div, Arena& scratch, int64_t M, int64_t K, int64_t N, GemmTail* tail,
+                    const int** slot_of_col_out);
 // Weight-gradient compensation into a compact buffer: for every column k of the residual that
 // holds entries, comp[slot_of_col[k], :] = sum_{entries of column k} val * dy[row, :].
 // Lists, slots and the dense path's buffers are carved from `scratch` (comp_wgrad_scratch_bytes); the slot

@@ -9,6 +9,8 @@
 // owns one output row and 256 of its columns (8 per lane); the sparse entries of that row (CSR
 // for the forward, CSC for the weight gradient) are walked in order, so the result is
 // deterministic.  The FP4 branch and the compensation meet in fp32 and are rounded once.
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 
 namespace {
@@ -69,8 +71,10 @@ __device__ __forceinline__ void sparse_row_times_dense(float (&acc)[8], const in
 __global__ void __launch_bounds__(COMP_THREADS)
 comp_fwd_kernel(const float* __restrict__ y1, const int* __restrict__ rowptr, const int* __restrict__ col,
                 const float* __restrict__ val, const uint4* __restrict__ w, int M, int N, void* y, int out_f32) {
-  const int m = blockIdx.y * 8 + (threadIdx.x >> 5);
-  const int n0 = blockIdx.x * COMP_COLS + 8 * (threadIdx.x & 31);
+  // blocks that follow one another share the 256 output columns, i.e. the same slab of the weight
+  // rows (K x 512 bytes): it stays in L2 while the tokens stream past
+  const int m = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int n0 = blockIdx.y * COMP_COLS + 8 * (threadIdx.x & 31);
   if (m >= M || n0 >= N) return;
   // Y1 is requested first: its latency runs under the dependent chain row pointer -> entry -> weight row
   const long long off = (long long)m * N + n0;
@@ -78,6 +82,66 @@ comp_fwd_kernel(const float* __restrict__ y1, const int* __restrict__ rowptr, co
   const float4 b = __ldg(reinterpret_cast<const float4*>(y1 + off + 4));
   float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
   sparse_row_times_dense(acc, col, val, __ldg(&rowptr[m]), __ldg(&rowptr[m + 1]), w, N >> 3, n0 >> 3);
+  const float y8[8] = {a.x + acc[0], a.y + acc[1], a.z + acc[2], a.w + acc[3],
+                       b.x + acc[4], b.y + acc[5], b.z + acc[6], b.w + acc[7]};
+  store8(y, out_f32, off, y8);
+}
+
+// The same with the entries of the hot columns left out (the GEMM's dense tail has added them):
+// slot_of_col[k] in [0, *tail_count) marks a hot column.  The lanes of a warp share the token, so
+// they read 32 entries at a time, drop the hot ones and hand the others round by shuffle, four
+// weight-row loads in flight as above; the order of the additions stays ascending.
+__global__ void __launch_bounds__(COMP_THREADS)
+comp_fwd_skip_kernel(const float* __restrict__ y1, const int* __restrict__ rowptr, const int* __restrict__ col,
+                     const float* __restrict__ val, const uint4* __restrict__ w, int M, int N, void* y, int out_f32,
+                     const int* __restrict__ slot_of_col, const int* __restrict__ tail_count) {
+  const int m = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  const int n0 = blockIdx.y * COMP_COLS + 8 * lane;
+  if (m >= M) return;                                   // whole warps only: the shuffles below need every lane
+  const bool live = n0 < N;
+  const long long off = (long long)m * N + (live ? n0 : 0);
+  float4 a = make_float4(0, 0, 0, 0), b = a;
+  if (live) {
+    a = __ldg(reinterpret_cast<const float4*>(y1 + off));
+    b = __ldg(reinterpret_cast<const float4*>(y1 + off + 4));
+  }
+  const unsigned hot = unsigned(__ldg(tail_count));
+  const int vec_per_row = N >> 3, vcol = (live ? n0 : 0) >> 3;
+  float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  const int e1 = __ldg(&rowptr[m + 1]);
+  for (int base = __ldg(&rowptr[m]); base < e1; base += 32) {
+    const int e = base + lane;
+    int k = 0;
+    float v = 0.0f;
+    bool keep = false;
+    if (e < e1) {
+      k = __ldg(&col[e]);
+      v = __ldg(&val[e]);
+      keep = unsigned(__ldg(&slot_of_col[k])) >= hot;   // -1 (no slot) compares as a large number
+    }
+    unsigned mask = __ballot_sync(0xFFFFFFFFu, keep);
+    while (mask) {
+      int r[4];
+      float vv[4];
+      uint4 d[4];
+      int cnt = 0;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int src = mask ? __ffs(mask) - 1 : 0;
+        r[u] = __shfl_sync(0xFFFFFFFFu, k, src);
+        vv[u] = __shfl_sync(0xFFFFFFFFu, v, src);
+        if (mask) { ++cnt; mask &= mask - 1; } else vv[u] = 0.0f;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (u < cnt) d[u] = __ldg(&w[(long long)r[u] * vec_per_row + vcol]);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (u < cnt) fma8(acc, vv[u], d[u]);
+    }
+  }
+  if (!live) return;
   const float y8[8] = {a.x + acc[0], a.y + acc[1], a.z + acc[2], a.w + acc[3],
                        b.x + acc[4], b.y + acc[5], b.z + acc[6], b.w + acc[7]};
   store8(y, out_f32, off, y8);
@@ -113,6 +177,97 @@ __device__ __forceinline__ int block_exclusive_scan_1024(int c, int* warp_tot, i
   __syncthreads();
   *total = warp_tot[31];
   return incl - c + (warp ? warp_tot[warp - 1] : 0);
+}
+
+// Hot columns of the residual for the forward GEMM's dense tail: the first TAIL_MAX_COLS columns, in
+// ascending order, that hold at least `hot_from` entries.  slot_of_col[k] is column k's position
+// among them or -1, list_hot the inverse, *count their number.
+__global__ void __launch_bounds__(1024, 1)
+hot_columns_kernel(const int* __restrict__ colptr, int K, int hot_from, int* __restrict__ list_hot,
+                   int* __restrict__ slot_of_col, int* __restrict__ count) {
+  __shared__ int warp_tot[32];
+  const int t = threadIdx.x;
+  const int per = (K + 1023) / 1024;
+  const int b = min(K, t * per), e = min(K, b + per);
+  int c = 0;
+  for (int k = b; k < e; ++k) c += (colptr[k + 1] - colptr[k] >= hot_from) ? 1 : 0;
+  int total;
+  int rank = block_exclusive_scan_1024(c, warp_tot, &total);
+  for (int k = b; k < e; ++k) {
+    int slot = -1;
+    if (colptr[k + 1] - colptr[k] >= hot_from) {
+      if (rank < TAIL_MAX_COLS) { slot = rank; list_hot[rank] = k; }
+      ++rank;
+    }
+    slot_of_col[k] = slot;
+  }
+  if (t == 0) *count = min(total, TAIL_MAX_COLS);
+}
+
+// Two-term FP16 split of x: hi = RN16(x), lo = RN16(x - hi).
+__device__ __forceinline__ void split_half(float x, __half& hi, __half& lo) {
+  hi = __float2half_rn(x);
+  lo = __float2half_rn(x - __half2float(hi));
+}
+
+// A operand of the dense tail: row m holds, for hot column s = 64 j + c, the value
+// x = residual[m, k_s] / (d_A[m] * TAIL_SCALE) as x_hi at columns 192 j + c and 192 j + 64 + c and
+// x_lo at 192 j + 128 + c; zero elsewhere.  One warp per token walks the token's CSR row.  A value
+// that FP16 cannot hold (or a token whose de-scale is zero) switches the tail off for this call:
+// *count becomes 0 and the per-entry kernel keeps every entry.
+__global__ void __launch_bounds__(COMP_THREADS)
+tail_a_kernel(const int* __restrict__ rowptr, const int* __restrict__ col, const float* __restrict__ val,
+              const int* __restrict__ slot_of_col, int* __restrict__ count, const float* __restrict__ amax_row,
+              float row_div, __half* __restrict__ ta, int M) {
+  const int hot = *count;
+  if (hot == 0) return;
+  const int lane = threadIdx.x & 31;
+  const int m = blockIdx.x * (COMP_THREADS / 32) + (threadIdx.x >> 5);
+  if (m >= M) return;
+  uint32_t* row32 = reinterpret_cast<uint32_t*>(ta + size_t(m) * TAIL_WIDTH);
+  for (int i = lane; i < TAIL_WIDTH / 2; i += 32) row32[i] = 0u;
+  __syncwarp();
+  const float scale = __fdiv_rn(__ldg(&amax_row[m]), row_div) * TAIL_SCALE;
+  __half* row = ta + size_t(m) * TAIL_WIDTH;
+  bool bad = false;
+  for (int e = rowptr[m] + lane; e < rowptr[m + 1]; e += 32) {
+    const int slot = slot_of_col[col[e]];
+    if (unsigned(slot) >= unsigned(hot)) continue;
+    const float x = __fdiv_rn(val[e], scale);
+    if (!(fabsf(x) <= 65504.0f)) { bad = true; continue; }         // also catches NaN (0 / 0)
+    __half hi, lo;
+    split_half(x, hi, lo);
+    const int at = 192 * (slot >> 6) + (slot & 63);
+    row[at] = hi;
+    row[at + 64] = hi;
+    row[at + 128] = lo;
+  }
+  if (bad) atomicExch(count, 0);
+}
+
+// B operand of the dense tail: row n holds, for hot column s = 64 j + c, the value
+// x = TAIL_SCALE * W[k_s, n] / d_W[n] as x_hi at 192 j + c and 192 j + 128 + c and x_lo at
+// 192 j + 64 + c (|x| <= 6 * 256 for an E2M1 operand: the weight is at most amax in magnitude).  The buffer
+// was cleared before.  One thread per (n, group of hot columns).
+__global__ void __launch_bounds__(256)
+tail_b_kernel(const __nv_bfloat16* __restrict__ w, const int* __restrict__ list_hot, const int* __restrict__ count,
+              const float* __restrict__ amax_col, float col_div, __half* __restrict__ tb, int N) {
+  const int hot = *count;
+  const int n = blockIdx.x * 256 + threadIdx.x;
+  if (n >= N) return;
+  const float d = __fdiv_rn(__ldg(&amax_col[n]), col_div);
+  const float inv_ok = d > 0.0f ? 1.0f : 0.0f;
+  __half* row = tb + size_t(n) * TAIL_WIDTH;
+  for (int s = blockIdx.y; s < hot; s += gridDim.y) {
+    const float wv = __bfloat162float(w[size_t(list_hot[s]) * N + n]);
+    const float x = inv_ok != 0.0f ? __fdiv_rn(wv * TAIL_SCALE, d) : 0.0f;
+    __half hi, lo;
+    split_half(x, hi, lo);
+    const int at = 192 * (s >> 6) + (s & 63);
+    row[at] = hi;
+    row[at + 64] = lo;
+    row[at + 128] = hi;
+  }
 }
 
 // The columns of the residual that hold entries, by how full they are: "dense" (at least
@@ -373,11 +528,16 @@ comp_wgrad_short_kernel(float* __restrict__ comp, const int* __restrict__ colptr
 }  // namespace
 
 int launch_comp_fwd(fp4_ctx* ctx, cudaStream_t stream, const float* y1, const int32_t* rowptr, const int32_t* col,
-                    const float* val, const void* w_bf16, int64_t M, int64_t, int64_t N, void* y, int out_f32) {
-  const dim3 grid(unsigned((N + COMP_COLS - 1) / COMP_COLS), unsigned((M + 7) / 8));
+                    const float* val, const void* w_bf16, int64_t M, int64_t, int64_t N, void* y, int out_f32,
+                    const int* slot_of_col, const int* tail_count) {
+  const dim3 grid(unsigned((M + 7) / 8), unsigned((N + COMP_COLS - 1) / COMP_COLS));
   KernelScope scope(ctx, stream, KC_COMP_FWD, 1);
-  comp_fwd_kernel<<<grid, COMP_THREADS, 0, stream>>>(y1, rowptr, col, val, static_cast<const uint4*>(w_bf16), int(M),
-                                                     int(N), y, out_f32);
+  if (slot_of_col && tail_count)
+    comp_fwd_skip_kernel<<<grid, COMP_THREADS, 0, stream>>>(y1, rowptr, col, val, static_cast<const uint4*>(w_bf16),
+                                                            int(M), int(N), y, out_f32, slot_of_col, tail_count);
+  else
+    comp_fwd_kernel<<<grid, COMP_THREADS, 0, stream>>>(y1, rowptr, col, val, static_cast<const uint4*>(w_bf16), int(M),
+                                                       int(N), y, out_f32);
   FP4_CUDA_TRY(cudaGetLastError());
   return FP4_OK;
 }
@@ -397,6 +557,40 @@ size_t comp_wgrad_scratch_bytes(int64_t M, int64_t K, int64_t N) {
   b += r256(size_t(DENSE_MAX) * size_t(M) * 4);                                       // V
   b += r256(size_t(dense_chunks(M, N)) * size_t(DENSE_MAX) * size_t(N) * 4);          // partial sums
   return b;
+}
+
+size_t fwd_tail_scratch_bytes(int64_t M, int64_t K, int64_t N) {
+  auto r256 = [](size_t b) { return (b + 255) & ~size_t(255); };
+  return r256(size_t(M) * TAIL_WIDTH * 2) + r256(size_t(N) * TAIL_WIDTH * 2) + r256(size_t(K) * 4) +
+         r256(TAIL_MAX_COLS * 4) + 256;
+}
+
+// Prepares the dense tail of the forward GEMM from the saved activation `a` (CSR, CSC column
+// pointers, row amax) and the weights; fills `tail` and hands back the slot vector and the count
+// for the per-entry kernel.  Buffers come from `scratch` (fwd_tail_scratch_bytes).
+int launch_fwd_tail(fp4_ctx* ctx, cudaStream_t stream, const fp4_qtensor* a, const void* w_bf16, const float* w_amax,
+                    float w_div, Arena& scratch, int64_t M, int64_t K, int64_t N, GemmTail* tail,
+                    const int** slot_of_col_out) {
+  __half* ta = scratch.take<__half>(size_t(M) * TAIL_WIDTH);
+  __half* tb = scratch.take<__half>(size_t(N) * TAIL_WIDTH);
+  int* slot_of_col = scratch.take<int>(size_t(K));
+  int* list_hot = scratch.take<int>(TAIL_MAX_COLS);
+  int* count = scratch.take<int>(1);
+  if (!scratch.ok) return FP4_ERR_WORKSPACE;
+  const int hot_from = int(M / 4 > LONG_COLUMN ? M / 4 : LONG_COLUMN);
+  KernelScope scope(ctx, stream, KC_COMP_FWD, 3);
+  hot_columns_kernel<<<1, 1024, 0, stream>>>(a->csc_colptr, int(K), hot_from, list_hot, slot_of_col, count);
+  FP4_CUDA_TRY(cudaMemsetAsync(tb, 0, size_t(N) * TAIL_WIDTH * 2, stream));
+  tail_a_kernel<<<unsigned((M + 7) / 8), COMP_THREADS, 0, stream>>>(a->csr_rowptr, a->csr_col, a->csr_val, slot_of_col,
+                                                                   count, a->amax, 6.0f, ta, int(M));
+  tail_b_kernel<<<dim3(unsigned((N + 255) / 256), 16), 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(w_bf16),
+                                                                        list_hot, count, w_amax, w_div, tb, int(N));
+  FP4_CUDA_TRY(cudaGetLastError());
+  tail->a = ta;
+  tail->b = tb;
+  tail->count = count;
+  *slot_of_col_out = slot_of_col;
+  return FP4_OK;
 }
 
 int launch_comp_wgrad(fp4_ctx* ctx, cudaStream_t stream, const fp4_qtensor* a, const void* dy_bf16, Arena& scratch,

@@ -71,6 +71,12 @@ struct GemmArgs {
   const uint4* w;
   const float* w_amax;
   float inv_k, expo, clip;
+  // dense tail (single-problem launches only): after the FP4 k-blocks of a tile, 3 * ceil(*tail_count / 64)
+  // k-blocks of 64 FP16 columns each from the maps that otherwise describe a second problem are
+  // accumulated into the same tile with kind::f16 (null: no tail)
+  const int* tail_count;
+  uint32_t tail_tx_bytes;
+  uint32_t tail_idesc;
 };
 
 // ------------------------------------------------------------------ PTX wrappers ------------
@@ -157,6 +163,14 @@ __device__ __forceinline__ void mma_f8f6f4(uint32_t d_tmem, uint64_t a_desc, uin
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+__device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 __device__ __forceinline__ void mma_mxf4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                          uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
   asm volatile(
@@ -222,6 +236,10 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
 __host__ __device__ constexpr uint32_t idesc_f8f6f4(bool a_e4m3 = false, bool b_e4m3 = false) {
   return (1u << 4) | ((a_e4m3 ? 0u : 5u) << 7) | ((b_e4m3 ? 0u : 5u) << 10) |
          (uint32_t(tile_n(FP4_GEMM_F8F6F4) >> 3) << 17) | (uint32_t(BM >> 4) << 24);
+}
+// kind::f16 with FP16 operands (format 0) and fp32 accumulators, M = 128, N = the kind's tile width
+__host__ __device__ constexpr uint32_t idesc_f16(int gemm_kind) {
+  return (1u << 4) | (uint32_t(tile_n(gemm_kind) >> 3) << 17) | (uint32_t(BM >> 4) << 24);
 }
 __host__ __device__ constexpr uint32_t idesc_mxf4() {
   return (1u << 7) | (1u << 10) | (uint32_t(tile_n(FP4_GEMM_MXF4) >> 3) << 17) | (1u << 23) |
@@ -461,11 +479,11 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out) : "memory");
-    if (args2.num_m_blocks) {
+    if (args2.num_m_blocks || args.tail_count) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a2) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b2) : "memory");
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out2) : "memory");
     }
+    if (args2.num_m_blocks) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out2) : "memory");
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
@@ -498,6 +516,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       uint32_t phase = 0;
       uint32_t fills = 0;
       bool ok = true;
+      const int tail_kb = args.tail_count ? 3 * ((min(*args.tail_count, TAIL_MAX_COLS) + 63) / 64) : 0;
       for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
         const bool second = t >= tiles_first;
         const GemmArgs& pa = second ? args2 : args;
@@ -512,6 +531,15 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           mbar_arrive_expect_tx(&full_bar[stage], pa.tx_bytes);
           tma_load_2d(smem_a + stage * A_STAGE_BYTES, ma, &full_bar[stage], kb * 128, m_blk * BM);
           tma_load_2d(smem_b + stage * B_STAGE_BYTES, mb, &full_bar[stage], kb * 128, n_blk * BN);
+          ++fills;
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        for (int kb = 0; kb < tail_kb && ok; ++kb) {      // dense tail: FP16 columns 64 kb .. 64 kb + 63
+          ok = mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, args.status);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&full_bar[stage], args.tail_tx_bytes);
+          tma_load_2d(smem_a + stage * A_STAGE_BYTES, &map_a2, &full_bar[stage], kb * 64, m_blk * BM);
+          tma_load_2d(smem_b + stage * B_STAGE_BYTES, &map_b2, &full_bar[stage], kb * 64, n_blk * BN);
           ++fills;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -536,6 +564,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
+      const int tail_kb = args.tail_count ? 3 * ((min(*args.tail_count, TAIL_MAX_COLS) + 63) / 64) : 0;
       for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
         ok = mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, args.status);
         if (!ok) break;
@@ -561,6 +590,18 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             }
           }
           tc_commit(&empty_bar[stage]);       // frees the stage once these MMAs have read it
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        for (int kb = 0; kb < tail_kb && ok; ++kb) {
+          ok = mbar_wait(&full_bar[stage], phase, abort_flag, args.status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t a_desc = make_smem_desc(smem_u32(smem_a + stage * A_STAGE_BYTES));
+          const uint64_t b_desc = make_smem_desc(smem_u32(smem_b + stage * B_STAGE_BYTES));
+#pragma unroll
+          for (int k = 0; k < 4; ++k)          // 16 FP16 columns = 32 bytes of the 128-byte row per instruction
+            mma_f16(d_tmem, a_desc + uint64_t(2 * k), b_desc + uint64_t(2 * k), args.tail_idesc, 1u);
+          tc_commit(&empty_bar[stage]);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
@@ -935,6 +976,22 @@ int make_codes_map(fp4_ctx* ctx, CUtensorMap* map, const uint8_t* codes, int64_t
   return r == CUDA_SUCCESS ? FP4_OK : FP4_ERR_CUDA;
 }
 
+// Tensor map over one operand of the dense tail: FP16 [rows x TAIL_WIDTH], a box of 64 columns (128
+// bytes) x box_rows, laid out in shared memory like a stage of codes.
+int make_tail_map(fp4_ctx* ctx, CUtensorMap* map, const void* base, int64_t rows, int box_rows) {
+  EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
+  if (!encode) return FP4_ERR_CUDA;
+  if (reinterpret_cast<uintptr_t>(base) & 15) return FP4_ERR_ALIGN;
+  const cuuint64_t dims[2] = {cuuint64_t(TAIL_WIDTH), cuuint64_t(rows)};
+  const cuuint64_t strides[1] = {cuuint64_t(TAIL_WIDTH) * 2};
+  const cuuint32_t box[2] = {64, cuuint32_t(box_rows)};
+  const cuuint32_t elem_strides[2] = {1, 1};
+  const CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+                            elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? FP4_OK : FP4_ERR_CUDA;
+}
+
 // Tensor maps of the output [I x J] for the bulk stores of the epilogue.  `unit` is a box of 32 rows
 // x 64 bytes with the 64-byte swizzle; `aux` is, for BF16 output, a box of 32 rows x 16 columns
 // without swizzle (16-column chunks) and unused for fp32 output (a copy of `unit`).
@@ -1036,6 +1093,9 @@ int make_problem(fp4_ctx* ctx, Problem* p, const Fp4GemmDesc& d, int gemm_kind, 
   args.inv_k = fused && epi->w_bf16 ? 1.0f / epi->dge_k : 1.0f;
   args.expo = args.inv_k - 1.0f;
   args.clip = fused ? epi->dge_clip : 0.0f;
+  args.tail_count = nullptr;
+  args.tail_tx_bytes = uint32_t(A_STAGE_BYTES + b_stage_bytes(gemm_kind));
+  args.tail_idesc = idesc_f16(gemm_kind);
   return FP4_OK;
 }
 
@@ -1043,7 +1103,8 @@ int make_problem(fp4_ctx* ctx, Problem* p, const Fp4GemmDesc& d, int gemm_kind, 
 
 int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, const uint8_t* b_codes, int64_t I,
                     int64_t J, int64_t C, const float* row_amax, const float* col_amax, void* out, int out_f32,
-                    int gemm_kind, int32_t* status, const GemmEpilogue* epi, bool a_e4m3, bool b_e4m3) {
+                    int gemm_kind, int32_t* status, const GemmEpilogue* epi, bool a_e4m3, bool b_e4m3,
+                    const GemmTail* tail) {
   Fp4GemmDesc d = {a_codes, b_codes, I, J, C, row_amax, col_amax, out, out_f32, epi};
   d.a_e4m3 = a_e4m3;
   d.b_e4m3 = b_e4m3;
@@ -1051,6 +1112,19 @@ int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, c
   Problem p;
   int rc = make_problem(ctx, &p, d, gemm_kind, pair_mode, status);
   if (rc != FP4_OK) return rc;
+  // The dense tail's operands travel in the slots of a second problem that has no tiles.
+  Problem with_tail;
+  if (tail) {
+    if (pair_mode) return FP4_ERR_ARG;
+    with_tail = p;
+    with_tail.args.num_m_blocks = with_tail.args.num_n_blocks = 0;
+    rc = make_tail_map(ctx, &with_tail.map_a, tail->a, I, BM);
+    if (rc != FP4_OK) return rc;
+    rc = make_tail_map(ctx, &with_tail.map_b, tail->b, J, tile_n(gemm_kind));
+    if (rc != FP4_OK) return rc;
+    p.args.tail_count = tail->count;
+  }
+  const Problem* second = tail ? &with_tail : nullptr;
   const GemmArgs& args = p.args;
   const int tiles = args.num_m_blocks * args.num_n_blocks;
   const int grid = tiles < ctx->num_sms ? tiles : ctx->num_sms;
@@ -1062,11 +1136,11 @@ int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, c
     rc2 = p.fused ? launch_pair_kernel<EPI_WGRAD>(pairs, stream, p.map_a, p.map_b, p.map_out, p.map_out_aux, args)
                   : launch_pair_kernel<EPI_PLAIN>(pairs, stream, p.map_a, p.map_b, p.map_out, p.map_out_aux, args);
   } else if (gemm_kind == FP4_GEMM_F8F6F4)
-    rc2 = p.fused ? launch_kernel<FP4_GEMM_F8F6F4, EPI_WGRAD>(grid, stream, p)
-                  : launch_kernel<FP4_GEMM_F8F6F4, EPI_PLAIN>(grid, stream, p);
+    rc2 = p.fused ? launch_kernel<FP4_GEMM_F8F6F4, EPI_WGRAD>(grid, stream, p, second)
+                  : launch_kernel<FP4_GEMM_F8F6F4, EPI_PLAIN>(grid, stream, p, second);
   else
-    rc2 = p.fused ? launch_kernel<FP4_GEMM_MXF4, EPI_WGRAD>(grid, stream, p)
-                  : launch_kernel<FP4_GEMM_MXF4, EPI_PLAIN>(grid, stream, p);
+    rc2 = p.fused ? launch_kernel<FP4_GEMM_MXF4, EPI_WGRAD>(grid, stream, p, second)
+                  : launch_kernel<FP4_GEMM_MXF4, EPI_PLAIN>(grid, stream, p, second);
   if (rc2 != FP4_OK) return rc2;
   FP4_CUDA_TRY(cudaGetLastError());
   return FP4_OK;
