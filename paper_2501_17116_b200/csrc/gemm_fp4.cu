@@ -463,6 +463,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   const int tiles_first = args.num_m_blocks * args.num_n_blocks;
   const int num_tiles = tiles_first + args2.num_m_blocks * args2.num_n_blocks;
 
+  int pre = 0;          // thread 0: k-blocks of its first tile already requested (see below)
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(&full_bar[s], 1);
@@ -476,14 +477,33 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+    // This thread is the producer.  The stages are empty and the barriers are its own work, so it
+    // requests the first k-blocks of its first tile now: they travel while tensor memory is
+    // allocated and the block synchronises.
+    if (int(blockIdx.x) < num_tiles) {
+      const bool second = int(blockIdx.x) >= tiles_first;
+      const GemmArgs& pa = second ? args2 : args;
+      const CUtensorMap* ma = second ? &map_a2 : &map_a;
+      const CUtensorMap* mb = second ? &map_b2 : &map_b;
+      const int tt = second ? int(blockIdx.x) - tiles_first : int(blockIdx.x);
+      const int m_blk = tt % pa.num_m_blocks, n_blk = tt / pa.num_m_blocks;
+      pre = pa.num_k_blocks < STAGES ? pa.num_k_blocks : STAGES;
+      for (int kb = 0; kb < pre; ++kb) {
+        mbar_arrive_expect_tx(&full_bar[kb], pa.tx_bytes);
+        tma_load_2d(smem_a + kb * A_STAGE_BYTES, ma, &full_bar[kb], kb * 128, m_blk * BM);
+        tma_load_2d(smem_b + kb * B_STAGE_BYTES, mb, &full_bar[kb], kb * 128, n_blk * BN);
+      }
+    }
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out) : "memory");
-    if (args2.num_m_blocks || args.tail_count) {
+    if (args.tail_count) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a2) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b2) : "memory");
     }
-    if (args2.num_m_blocks) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out2) : "memory");
+    if (args2.num_m_blocks) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a2) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b2) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out2) : "memory");
+    }
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
@@ -512,9 +532,9 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer -------
     if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      uint32_t fills = 0;
+      int stage = pre == STAGES ? 0 : pre;
+      uint32_t phase = pre == STAGES ? 1u : 0u;
+      uint32_t fills = uint32_t(pre);
       bool ok = true;
       const int tail_kb = args.tail_count ? 3 * ((min(*args.tail_count, TAIL_MAX_COLS) + 63) / 64) : 0;
       for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
@@ -525,7 +545,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const int tt = second ? t - tiles_first : t;
         const int m_blk = tt % pa.num_m_blocks;
         const int n_blk = tt / pa.num_m_blocks;
-        for (int kb = 0; kb < pa.num_k_blocks; ++kb) {
+        for (int kb = (t == int(blockIdx.x) ? pre : 0); kb < pa.num_k_blocks; ++kb) {
           ok = mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, args.status);
           if (!ok) break;
           mbar_arrive_expect_tx(&full_bar[stage], pa.tx_bytes);
