@@ -161,6 +161,20 @@ def test_forward_dense_tail(lib, ctx, M, K, N, hot, alpha, kind):
     assert torch.equal(y16, y16_again)
 
 
+def test_forward_dense_tail_with_e4m3_weights(lib, ctx):
+    """W8A4 with a heavy residual: the tail's weight operand is divided by the E4M3 de-scale (amax / 448)."""
+    M, K, N, hot, alpha = 1024, 256, 384, 20, 0.92
+    a_bits, w_bits, _ = WL.small_case(M, K, N, seed=31, alpha_outliers=hot)
+    f = O.linear_fwd(a_bits, w_bits, alpha, fmt_w="e4m3")
+    ctx.status.zero_()
+    y32, sa, _ = lib.fp4_linear_fwd(ctx, _dev(a_bits), _dev(w_bits), alpha, gemm_kind=lib.FP4_GEMM_F8F6F4, out_f32=True,
+                                    fmt_w=lib.FP4_FORMAT_E4M3)
+    torch.cuda.synchronize()
+    assert ctx.read_status() == 0
+    assert int((np.diff(sa.csc_colptr.cpu().numpy()) >= 512).sum()) > 0
+    assert_close_f32(y32.cpu().numpy(), f.y, f.y_fp4, f.y_comp, "Y")
+
+
 def test_forward_dense_tail_falls_back_on_huge_outliers(lib, ctx):
     """A residual too large for the tail's FP16 operands (relative to its token's scale) switches the
     tail off on the device for that call; the per-entry kernel then adds every entry."""
