@@ -9,6 +9,13 @@ of a rounding boundary; at least 99 % of the values must be the rounding itself.
 branches nearly cancel, "relative" is taken against |fp4 branch| + |compensation branch| as in
 float mode (callers that pass the branches), since that is what the fp32 sum before the rounding
 is held to.
+
+Accumulation floor of the dense tail.  With a heavy residual the hot columns' products are added
+inside the tensor cores, whose fp32 accumulation rounds toward zero: up to 24 additions (6 blocks
+of 64 FP16 columns, 4 instructions each), each off by at most 2^-23 of the running sum, plus 2^-21
+from the two-term FP16 splits, i.e. at most 4e-6 of sum_k |dA[m,k]| |W[k,n]|.  Where both branches
+cancel to a thousandth of their terms that floor can exceed 1e-3 of the branches, so the cases that
+can take the tail add TAIL_FLOOR * (|dA| |W|)[m,n] to the allowance.
 """
 import numpy as np
 import pytest
@@ -19,6 +26,12 @@ from paper_2501_17116_b200 import workloads as WL
 
 pytestmark = pytest.mark.gpu
 RTOL = 1e-3
+TAIL_FLOOR = 4e-6
+
+
+def tail_floor(f: "O.Forward", w_bits):
+    """Allowance for the tensor cores' accumulation of the dense tail: TAIL_FLOOR * (|dA| |W|)."""
+    return TAIL_FLOOR * (np.abs(f.qa.residual) @ np.abs(O.bf16_bits_to_f64(w_bits)))
 
 
 @pytest.fixture(scope="module")
@@ -32,20 +45,20 @@ def _dev(bits):
     return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
 
 
-def assert_close_f32(got, want, branch_a, branch_b=None, what=""):
+def assert_close_f32(got, want, branch_a, branch_b=None, what="", floor=0.0):
     scale = np.abs(branch_a) + (0 if branch_b is None else np.abs(branch_b))
     err = np.abs(got.astype(np.float64) - want)
-    bad = err > RTOL * scale + 1e-300
+    bad = err > RTOL * scale + floor + 1e-300
     assert not bad.any(), f"{what}: {bad.sum()} of {bad.size} outside tolerance, worst {np.max(err / (scale + 1e-300))}"
 
 
-def assert_bf16_rounding(got_bf16: torch.Tensor, want, what="", branch_a=None, branch_b=None):
+def assert_bf16_rounding(got_bf16: torch.Tensor, want, what="", branch_a=None, branch_b=None, floor=0.0):
     got = got_bf16.float().cpu().numpy().astype(np.float64)
     r = O.f64_to_bf16_f64(want)
     exact = got == r
     scale = np.abs(want) if branch_a is None else np.abs(branch_a) + (0 if branch_b is None else np.abs(branch_b))
     # a neighbouring BF16 value is accepted only if the oracle value is within RTOL of the midpoint
-    near = np.abs(got - want) <= np.abs(r - want) + RTOL * scale
+    near = np.abs(got - want) <= np.abs(r - want) + RTOL * scale + floor
     ok = exact | near
     assert ok.all(), f"{what}: {np.sum(~ok)} of {ok.size} values are not the BF16 rounding of the oracle"
     assert exact.mean() > 0.99, f"{what}: only {exact.mean():.4f} match the rounding exactly"
@@ -156,8 +169,8 @@ def test_forward_dense_tail(lib, ctx, M, K, N, hot, alpha, kind):
     counts = np.diff(sa.csc_colptr.cpu().numpy())
     n_hot = int((counts >= max(M // 4, 512)).sum())
     assert (n_hot > 0) == (hot >= 12)                                   # the case is in the regime it names
-    assert_close_f32(y32.cpu().numpy(), f.y, f.y_fp4, f.y_comp, "Y")
-    assert_bf16_rounding(y16, f.y, "Y bf16", f.y_fp4, f.y_comp)
+    assert_close_f32(y32.cpu().numpy(), f.y, f.y_fp4, f.y_comp, "Y", tail_floor(f, w_bits))
+    assert_bf16_rounding(y16, f.y, "Y bf16", f.y_fp4, f.y_comp, tail_floor(f, w_bits))
     assert torch.equal(y16, y16_again)
 
 
@@ -172,7 +185,7 @@ def test_forward_dense_tail_with_e4m3_weights(lib, ctx):
     torch.cuda.synchronize()
     assert ctx.read_status() == 0
     assert int((np.diff(sa.csc_colptr.cpu().numpy()) >= 512).sum()) > 0
-    assert_close_f32(y32.cpu().numpy(), f.y, f.y_fp4, f.y_comp, "Y")
+    assert_close_f32(y32.cpu().numpy(), f.y, f.y_fp4, f.y_comp, "Y", tail_floor(f, w_bits))
 
 
 def test_forward_dense_tail_falls_back_on_huge_outliers(lib, ctx):
