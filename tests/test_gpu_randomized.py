@@ -26,6 +26,14 @@ def ctx(lib):
     c.close()
 
 
+def _fp8_floor(terms, contraction):
+    """Allowance for a GEMM with an E4M3 operand: its products are not on one binary scale, so the
+    tensor cores' fp32 accumulation (rounding toward zero, one addition per 32 contraction columns)
+    is no longer exact: at most 2 * 2^-23 of the running sum per instruction, bounded here against
+    the sum of the magnitudes of the products.  GEMMs of E2M1 operands alone are exact: no floor."""
+    return 2.0 * -(-contraction // 32) * 2.0 ** -23 * terms
+
+
 def _draws(n, seed):
     rng = np.random.default_rng(seed)
     out = []
@@ -38,29 +46,95 @@ def _draws(n, seed):
         hot = int(rng.choice([0, 2, 9, 40]))
         kind = int(rng.integers(0, 2))
         dge = bool(rng.integers(0, 2))
-        out.append((i, M, K, N, alpha, dist, hot, kind, dge))
+        # FP8 settings need the byte-container kind; an E4M3 activation is not clamped
+        fp8 = str(rng.choice(["none", "none", "w8", "a8", "dy8", "w8+dy8"])) if kind == 1 else "none"
+        if fp8 == "a8":
+            alpha = 1.0
+        out.append((i, M, K, N, alpha, dist, hot, kind, dge, fp8))
     return out
 
 
-@pytest.mark.parametrize("i,M,K,N,alpha,dist,hot,kind,dge",
+@pytest.mark.parametrize("i,M,K,N,alpha,dist,hot,kind,dge,fp8",
                          _draws(int(os.environ.get("FP4_RANDOM_DRAWS", "16")), seed=2501))
-def test_random_layer_matches_oracle(lib, ctx, i, M, K, N, alpha, dist, hot, kind, dge):
+def test_random_layer_matches_oracle(lib, ctx, i, M, K, N, alpha, dist, hot, kind, dge, fp8):
     a_bits, w_bits, dy_bits = WL.small_case(M, K, N, seed=1000 + i, alpha_outliers=hot, dist=dist)
-    f = O.linear_fwd(a_bits, w_bits, alpha)
-    b = O.linear_bwd(dy_bits, w_bits, f, dge_on=dge)
+    fmt_a = "e4m3" if fp8 == "a8" else "e2m1"
+    fmt_w = "e4m3" if "w8" in fp8 else "e2m1"
+    fmt_dy = "e4m3" if "dy8" in fp8 else "e2m1"
+    code = {"e2m1": lib.FP4_FORMAT_E2M1, "e4m3": lib.FP4_FORMAT_E4M3}
+    f = O.linear_fwd(a_bits, w_bits, alpha, fmt_a=fmt_a, fmt_w=fmt_w)
+    b = O.linear_bwd(dy_bits, w_bits, f, dge_on=dge, fmt_dy=fmt_dy)
     A, W, dY = _dev(a_bits), _dev(w_bits), _dev(dy_bits)
     ctx.status.zero_()
-    y32, sa, sw = lib.fp4_linear_fwd(ctx, A, W, alpha, gemm_kind=kind, out_f32=True)
-    da32, dw32 = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, gemm_kind=kind, out_f32=True, dge_on=dge)
+    y32, sa, sw = lib.fp4_linear_fwd(ctx, A, W, alpha, gemm_kind=kind, out_f32=True, fmt_a=code[fmt_a],
+                                     fmt_w=code[fmt_w])
+    da32, dw32 = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, gemm_kind=kind, out_f32=True, dge_on=dge,
+                                    dy_e4m3=fmt_dy == "e4m3")
     torch.cuda.synchronize()
     assert ctx.read_status() == 0
-    _saved_matches(sa, sw, f)
+    if fp8 in ("none", "dy8"):
+        _saved_matches(sa, sw, f)
+    else:
+        np.testing.assert_array_equal(sa.amax.cpu().numpy(), f.qa.amax)
+        np.testing.assert_array_equal(sw.amax.cpu().numpy(), f.qw.amax)
+        np.testing.assert_array_equal(sa.codes.cpu().numpy(), f.qa.packed() if fmt_a == "e2m1" else f.qa.codes)
+        np.testing.assert_array_equal(sw.codes_t.cpu().numpy(),
+                                      f.qw.packed_t() if fmt_w == "e2m1" else np.ascontiguousarray(f.qw.codes.T))
     if alpha < 1.0:
         th = sa.thresholds.cpu().numpy()
         assert (float(th[0]), float(th[1])) == (f.qa.lo, f.qa.hi)
         assert int(sa.nnz.item()) == int(np.count_nonzero(f.qa.residual))
     # heavy residuals with enough tokens may send hot columns through the GEMM's dense tail
-    floor = tail_floor(f, w_bits) if (alpha <= 0.995 and M >= 512) else 0.0
-    assert_close_f32(y32.cpu().numpy(), f.y, f.y_fp4, f.y_comp, "Y", floor)
-    assert_close_f32(da32.cpu().numpy(), b.da, b.da, None, "dA")
-    assert_close_f32(dw32.cpu().numpy(), b.dw, b.s_fp4 * b.dge, b.s_comp * b.dge, "dW")
+    floor_y = tail_floor(f, w_bits) if (alpha <= 0.995 and M >= 512) else 0.0
+    floor_da = floor_dw = 0.0
+    va, vw = np.abs(f.qa.values()), np.abs(f.qw.values())
+    vg1, vg2 = np.abs(b.qg_dgrad.values()), np.abs(b.qg_wgrad.values())
+    d64 = lambda q: q.descale.astype(np.float64)
+    if fmt_a == "e4m3" or fmt_w == "e4m3":
+        floor_y = floor_y + _fp8_floor((va @ vw) * d64(f.qa)[:, None] * d64(f.qw)[None, :], K)
+    if fmt_dy == "e4m3" or fmt_w == "e4m3":
+        floor_da = _fp8_floor((vg1 @ vw.T) * d64(b.qg_dgrad)[:, None], N)
+    if fmt_a == "e4m3" or fmt_dy == "e4m3":
+        floor_dw = _fp8_floor((va.T @ vg2) * d64(b.qg_wgrad)[None, :] * b.dge, M)
+    assert_close_f32(y32.cpu().numpy(), f.y, f.y_fp4, f.y_comp, "Y", floor_y)
+    assert_close_f32(da32.cpu().numpy(), b.da, b.da, None, "dA", floor_da)
+    assert_close_f32(dw32.cpu().numpy(), b.dw, b.s_fp4 * b.dge, b.s_comp * b.dge, "dW", floor_dw)
+
+
+def _quantizer_draws(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        rows = int(rng.choice([128, 256, 512, 1024]))
+        cols = int(rng.choice([128, 384, 640, 1152, 2048]))
+        alpha = float(rng.choice([0.9999, 0.999, 0.99, 0.97, 0.9]))
+        spread = int(rng.choice([0, 4, 20, 60]))           # binades over which the rows' scales are spread
+        zeros = float(rng.choice([0.0, 0.01, 0.5]))        # fraction of exact zeros
+        out.append((i, rows, cols, alpha, spread, zeros))
+    return out
+
+
+@pytest.mark.parametrize("i,rows,cols,alpha,spread,zeros",
+                         _quantizer_draws(int(os.environ.get("FP4_RANDOM_DRAWS", "16")), seed=1711))
+def test_random_clamping_quantizer_is_bit_exact(lib, ctx, i, rows, cols, alpha, spread, zeros):
+    """Thresholds, codes in both layouts, amax and the sparse residual on tensors whose rows live on
+    scales spread over many binades (values outside the histogram kernel's window, subnormals),
+    with ties and exact zeros of both signs."""
+    from test_gpu_quantize import _check_dense, _check_sparse
+    rng = np.random.default_rng(5000 + i)
+    a = rng.standard_normal((rows, cols)).astype(np.float32)
+    if spread:
+        a *= np.exp2(rng.integers(-spread, spread + 1, size=(rows, 1))).astype(np.float32)
+    if i % 3 == 0:
+        a = np.round(a * 4) / 4                            # many ties
+    if zeros:
+        mask = rng.random(a.shape) < zeros
+        a[mask] = np.where(rng.random(int(mask.sum())) < 0.5, 0.0, -0.0).astype(np.float32)
+    bits = WL.to_bf16_bits(a)
+    ctx.status.zero_()
+    q = lib.fp4_quantize(ctx, _dev(bits), 0, alpha=alpha)
+    torch.cuda.synchronize()
+    assert ctx.read_status() == 0
+    ref = O.occ_quantize(O.bf16_bits_to_f64(bits), alpha)
+    _check_sparse(q, ref)
+    _check_dense(q, ref)
