@@ -138,3 +138,35 @@ def test_random_clamping_quantizer_is_bit_exact(lib, ctx, i, rows, cols, alpha, 
     ref = O.occ_quantize(O.bf16_bits_to_f64(bits), alpha)
     _check_sparse(q, ref)
     _check_dense(q, ref)
+
+
+@pytest.mark.parametrize("seed", [7, 8])
+def test_random_sequence_of_host_steps(lib, seed):
+    """Twenty host-buffer steps of random shapes issued back to back on a workspace that fits the
+    pipelined layout for some of them only: every output equals the device-resident path's, bit for
+    bit, whatever mix of pipelined and single-stream calls the sequence produces."""
+    from test_gpu_step_host import ALPHA, _device_reference, _inputs
+    rng = np.random.default_rng(seed)
+    shapes = [(128, 128, 128), (256, 256, 384), (128, 512, 128), (384, 128, 640), (512, 384, 256)]
+    seq = [shapes[int(rng.integers(0, len(shapes)))] for _ in range(20)]
+    needs = sorted(int(lib.load_library().fp4_step_host_workspace_bytes(M, K, N, ALPHA)) for M, K, N in shapes)
+    ctx = lib.Context(0, needs[len(needs) // 2] if seed % 2 else needs[-1])
+    cases, outs = [], []
+    for i, (M, K, N) in enumerate(seq):
+        hA, hW, hG = _inputs(200 + i, M, K, N)
+        hY = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+        hdA = torch.empty((M, K), dtype=torch.bfloat16).pin_memory()
+        hdW = torch.empty((K, N), dtype=torch.bfloat16).pin_memory()
+        try:
+            lib.fp4_linear_step_host(ctx, hA, hW, hG, ALPHA, hY, hdA, hdW, read_status=False)
+        except Exception:
+            continue                                   # a shape the smaller workspace cannot hold at all
+        cases.append(((M, K, N), (hA, hW, hG)))
+        outs.append((hY, hdA, hdW))
+    torch.cuda.synchronize()
+    assert len(cases) >= 10
+    for ((M, K, N), (hA, hW, hG)), got in zip(cases, outs):
+        want = _device_reference(lib, M, K, N, hA, hW, hG)
+        for g, w, name in zip(got, want, ("Y", "dA", "dW")):
+            assert torch.equal(g.view(torch.int16), w.view(torch.int16)), (M, K, N, name)
+    ctx.close()
