@@ -37,9 +37,9 @@ def _nibbles_of_rows(packed_t_dev, rows):
     return np.where(odd, b >> 4, b & 0xF).T.astype(np.uint8)
 
 
-def _close(got, want, scale, what):
+def _close(got, want, scale, what, floor=0.0):
     err = np.abs(np.asarray(got, dtype=np.float64) - want)
-    bad = err > RTOL * scale + 1e-300
+    bad = err > RTOL * scale + floor + 1e-300
     assert not bad.any(), f"{what}: {bad.sum()} of {bad.size} outside tolerance"
 
 
@@ -122,7 +122,10 @@ def test_full_size_layer_matches_sampled_oracle(lib, ci, lname, alpha):
         * d_w[cols_w].astype(np.float64)[None, :]
     y_comp = resid @ w_cols
     got = y32[torch.as_tensor(rows, device="cuda")][:, torch.as_tensor(cols_w, device="cuda")].cpu().numpy()
-    _close(got, y_fp4 + y_comp, np.abs(y_fp4) + np.abs(y_comp), "Y")
+    # heavy residuals send their hot columns through the GEMM's dense tail: accumulation floor of
+    # the tensor cores as in test_gpu_linear.py (4e-6 of the summed magnitudes of the residual's products)
+    floor = 4e-6 * (np.abs(resid) @ np.abs(w_cols)) if alpha <= 0.995 else 0.0
+    _close(got, y_fp4 + y_comp, np.abs(y_fp4) + np.abs(y_comp), "Y", floor)
 
     # ---- dgrad: dA on rows x cols_a ----------------------------------------------------------------
     qg1 = O.absmax_quantize(O.bf16_bits_to_f64(dy_bits[rows]), 0, prescale=d_w)
