@@ -44,7 +44,10 @@ Readings of points the paper leaves open (each also listed in the design notes):
   the sign of the input kept, vector-wise absmax scaling along the same axes as for
   E2M1 with MAX = 448.  OCC belongs to 4-bit activations and DGE to 4-bit weights, so
   an E4M3 activation is not clamped and an E4M3 weight gets the straight-through
-  estimator.  PARITY UNPINNED by the paper for all of this as well.
+  estimator.  PARITY UNPINNED by the paper for all of this as well.  The other FP8
+  variant the paper names (Section 2), E5M2 (5 exponent bits, bias 15, 2 mantissa
+  bits, infinities and NaNs at exponent field 31, largest finite value 57344), is
+  offered the same way, with MAX = 57344 and saturation to the largest finite value.
 """
 from __future__ import annotations
 
@@ -182,6 +185,46 @@ def e4m3_quantize(v32) -> np.ndarray:
     return ((sign << 7) | (field_e << 3) | field_m).astype(np.uint8)
 
 
+# --------------------------------------------------------------------------- #
+# FP8 E5M2 (the other variant Section 2 names)
+# --------------------------------------------------------------------------- #
+E5M2_MAX = 57344.0
+
+
+def e5m2_decode(codes) -> np.ndarray:
+    """Value of every E5M2 byte: S.EEEEE.MM, bias 15, subnormals at E = 0, E = 31 is infinity (M = 0) or NaN."""
+    c = np.asarray(codes, dtype=np.uint8).astype(np.int64)
+    e = (c >> 2) & 0x1F
+    m = (c & 3).astype(np.float64)
+    mag = np.where(e == 0, m / 4.0 * 2.0 ** -14, (1.0 + m / 4.0) * np.exp2((e - 15).astype(np.float64)))
+    mag = np.where(e == 31, np.where(m == 0, np.inf, np.nan), mag)
+    return np.where(c & 0x80, -mag, mag)
+
+
+def e5m2_quantize(v32) -> np.ndarray:
+    """Nearest E5M2 value of float32 numbers (ties to the even mantissa), saturating at 57344.
+
+    Returns the codes; the sign bit is the sign of the input, also when the result is zero.
+    """
+    v = np.asarray(v32, dtype=np.float32).astype(np.float64)
+    a = np.minimum(np.abs(v), E5M2_MAX)
+    _, ex = np.frexp(a)
+    e = np.clip(ex - 1, -14, 15)                         # binade of a (subnormals share e = -14)
+    step = np.exp2((e - 2).astype(np.float64))           # spacing of the grid inside that binade
+    q = np.minimum(np.rint(a / step) * step, E5M2_MAX)   # np.rint rounds halves to even
+    _, exq = np.frexp(q)
+    eq = np.clip(exq - 1, -14, 15)
+    normal = q >= 2.0 ** -14
+    field_e = np.where(normal, eq + 15, 0).astype(np.int64)
+    field_m = np.where(normal, np.rint((q / np.exp2(eq.astype(np.float64)) - 1.0) * 4.0),
+                       np.rint(q / 2.0 ** -16)).astype(np.int64)
+    sign = np.signbit(v).astype(np.int64)
+    return ((sign << 7) | (field_e << 2) | field_m).astype(np.uint8)
+
+
+FORMAT_MAX = {"e2m1": 6.0, "e4m3": E4M3_MAX, "e5m2": E5M2_MAX}
+
+
 @dataclass
 class Quantized:
     """Everything one call of the quantiser produces (all host arrays)."""
@@ -197,11 +240,11 @@ class Quantized:
     csr: tuple = field(default=None)   # (rowptr int32[rows+1], col int32[nnz], val float32[nnz])
     csc: tuple = field(default=None)   # (colptr int32[cols+1], row int32[nnz], val float32[nnz])
     residual: np.ndarray = None  # dense float64 [rows, cols] (zeros outside the tails)
-    fmt: str = "e2m1"            # "e2m1": one nibble code per element; "e4m3": one byte per element
+    fmt: str = "e2m1"            # "e2m1": one nibble code per element; "e4m3" / "e5m2": one byte per element
 
     @property
     def fmax(self):
-        return FP4_MAX if self.fmt == "e2m1" else E4M3_MAX
+        return FORMAT_MAX[self.fmt]
 
     @property
     def gamma(self):
@@ -213,7 +256,7 @@ class Quantized:
 
     def values(self):
         """The numbers the codes stand for, float64 [rows, cols]."""
-        return e2m1_decode(self.codes) if self.fmt == "e2m1" else e4m3_decode(self.codes)
+        return {"e2m1": e2m1_decode, "e4m3": e4m3_decode, "e5m2": e5m2_decode}[self.fmt](self.codes)
 
     def packed(self):
         """[rows, cols/2] bytes, column pairs packed."""
@@ -232,8 +275,9 @@ def absmax_quantize(x, scale_axis: int, prescale=None, fmt: str = "e2m1") -> Qua
     Appendix C.2 where sf is 1 x c_o).
     ``prescale``: optional float32 vector laid along the *other* axis that
     multiplies x first, x <- RN32(x * prescale) (used for dY in the backward).
-    ``fmt``: "e2m1" (Eq. 1 with MAX = 6 and the quantiser of Appendix A) or "e4m3"
-    (MAX = 448, nearest-even rounding: the FP8 operand of the W4A8 / W8A4 settings).
+    ``fmt``: "e2m1" (Eq. 1 with MAX = 6 and the quantiser of Appendix A), "e4m3"
+    (MAX = 448, nearest-even rounding: the FP8 operand of the W4A8 / W8A4 settings) or "e5m2"
+    (MAX = 57344, the same rounding).
     """
     x = np.asarray(x, dtype=np.float64)
     rows, cols = x.shape
@@ -242,11 +286,11 @@ def absmax_quantize(x, scale_axis: int, prescale=None, fmt: str = "e2m1") -> Qua
         p = p[None, :] if scale_axis == 0 else p[:, None]
         x = rn32(x * p)                     # exact double product, one rounding
     amax = np.max(np.abs(x), axis=1 - scale_axis).astype(np.float32)
-    gamma, _ = absmax_scales(amax, FP4_MAX if fmt == "e2m1" else E4M3_MAX)
+    gamma, _ = absmax_scales(amax, FORMAT_MAX[fmt])
     g = gamma.astype(np.float64)
     g = g[:, None] if scale_axis == 0 else g[None, :]
     scaled = (x * g).astype(np.float32)     # RN32(x * gamma): the product is exact in double
-    codes = lut_quantize(scaled) if fmt == "e2m1" else e4m3_quantize(scaled)
+    codes = {"e2m1": lut_quantize, "e4m3": e4m3_quantize, "e5m2": e5m2_quantize}[fmt](scaled)
     return Quantized(rows, cols, scale_axis, codes, amax, scaled, fmt=fmt)
 
 
@@ -334,7 +378,9 @@ def gemm_values(qa: Quantized, qb: Quantized, transpose_a: bool = False, transpo
 
     E2M1 values are multiples of 2^-1 up to 6 and E4M3 values multiples of 2^-9 up to 448, so
     every product is a multiple of 2^-18 below 2^18 and sums of up to 2^17 of them are exact in
-    float64.  ``transpose_*`` takes the operand's codes transposed first.
+    float64.  E5M2 values are multiples of 2^-16 up to 57344: with an E2M1 partner the sums are
+    still exact (multiples of 2^-17 below 2^19), with an 8-bit partner they are float64 sums
+    (2^-53 of the summed magnitudes).  ``transpose_*`` takes the operand's codes transposed first.
     """
     va = qa.values().T if transpose_a else qa.values()
     vb = qb.values().T if transpose_b else qb.values()

@@ -105,7 +105,7 @@ def test_mixed_layer_against_exact_rationals(fmt_a, fmt_w, fmt_dy):
         for n in range(N):
             want = sum(va[m][k] * g2[m][n] for m in range(M)) * d2[n] + sum(res[m][k] * dy[m][n] for m in range(M))
             assert abs(Fraction(float(b.s[k, n])) - want) <= abs(want) * Fraction(1, 10 ** 12) + Fraction(1, 10 ** 300)
-    if fmt_w == "e4m3":
+    if fmt_w != "e2m1":
         assert (b.dge == 1.0).all()                         # straight-through for an 8-bit weight
     else:
         np.testing.assert_array_equal(b.dge, O.dge_fprime(f.qw.scaled.astype(np.float64)))
@@ -133,3 +133,73 @@ def test_activation_clamping_is_refused_for_fp8_activations():
     a_bits, w_bits, _ = WL.small_case(4, 8, 4, seed=1)
     with pytest.raises(ValueError):
         O.linear_fwd(a_bits, w_bits, 0.99, fmt_a="e4m3")
+
+
+# ---------------------------------------------------------------------------------------------
+# E5M2, the other FP8 variant Section 2 names
+# ---------------------------------------------------------------------------------------------
+FINITE_E5M2 = np.array([c for c in range(256) if ((c >> 2) & 0x1F) != 0x1F], dtype=np.uint8)
+
+
+def test_e5m2_decode_matches_the_format_definition():
+    for ln in golden_lines("e5m2_spot_values.txt"):
+        code, val = ln.split()
+        assert O.e5m2_decode(np.array([int(code, 16)], dtype=np.uint8))[0] == float(val)
+    v = O.e5m2_decode(np.arange(256, dtype=np.uint8))
+    assert v[0x7C] == np.inf and v[0xFC] == -np.inf and np.isnan(v[[0x7D, 0x7E, 0x7F, 0xFD, 0xFE, 0xFF]]).all()
+    pos = v[:0x7C]
+    assert (np.diff(pos) > 0).all()                        # codes order like their values
+    np.testing.assert_array_equal(v[0x80:0xFC], -pos)       # sign-magnitude
+    assert pos.max() == 57344.0 and pos[1] == 2.0 ** -16
+    assert (pos * 65536 == np.rint(pos * 65536)).all()     # every value is an integer multiple of 2^-16
+
+
+def test_e5m2_quantize_is_nearest_with_ties_to_even_and_saturates():
+    grid = O.e5m2_decode(FINITE_E5M2[FINITE_E5M2 < 0x80])  # non-negative values, ascending
+    rng = np.random.default_rng(1)
+    mids = (grid[:-1] + grid[1:]) / 2                       # every tie of the format
+    probes = np.concatenate([grid, mids, np.nextafter(mids.astype(np.float32), np.float32(np.inf)).astype(np.float64),
+                             np.nextafter(mids.astype(np.float32), np.float32(0)).astype(np.float64),
+                             rng.uniform(0, 57344, 20000), rng.uniform(0, 0.001, 5000)])
+    probes = probes.astype(np.float32)
+    for sign in (1.0, -1.0):
+        v = (sign * probes).astype(np.float32)
+        codes = O.e5m2_quantize(v)
+        got = np.abs(O.e5m2_decode(codes))
+        a = np.abs(v.astype(np.float64))
+        dist = np.abs(a[:, None] - grid[None, :])
+        best = dist.min(axis=1)
+        assert (np.abs(got - a) == best).all()              # a nearest value
+        tie = (dist == best[:, None]).sum(axis=1) == 2
+        assert ((codes[tie] & 1) == 0).all()                # of two nearest, the even mantissa
+        assert ((codes >> 7) == (1 if sign < 0 else 0)).all()   # the input's sign, zero included
+    big = np.array([57345, 61440, 65535, 65536, 1e6, 3e38], dtype=np.float32)
+    np.testing.assert_array_equal(O.e5m2_quantize(big), np.full(6, 0x7B, dtype=np.uint8))    # never infinity
+    np.testing.assert_array_equal(O.e5m2_quantize(-big), np.full(6, 0xFB, dtype=np.uint8))
+
+
+def test_e5m2_quantize_is_the_identity_on_the_grid():
+    v = O.e5m2_decode(FINITE_E5M2).astype(np.float32)
+    np.testing.assert_array_equal(O.e5m2_quantize(v), FINITE_E5M2)
+
+
+@pytest.mark.parametrize("axis", [0, 1])
+def test_absmax_scaling_to_57344(axis):
+    rng = np.random.default_rng(13 + axis)
+    x = O.bf16_bits_to_f64(WL.to_bf16_bits(rng.standard_normal((24, 40)).astype(np.float32)))
+    q = O.absmax_quantize(x, axis, fmt="e5m2")
+    vals = q.values()
+    where = np.abs(x) == np.abs(x).max(axis=1 - axis, keepdims=True)
+    assert (np.abs(vals[where]) == 57344.0).all()           # the absmax element sits on MAX
+    assert np.isfinite(vals).all()
+    step = np.where(np.abs(vals) >= 2.0 ** -14, 2.0 ** (np.floor(np.log2(np.maximum(np.abs(vals), 1e-30))) - 2), 2.0 ** -16)
+    assert (np.abs(vals - q.scaled.astype(np.float64)) <= step / 2 * (1 + 1e-12)).all()
+    g, d = O.absmax_scales(q.amax, 57344.0)
+    np.testing.assert_array_equal(g, (np.float32(57344) / q.amax).astype(np.float32))
+    np.testing.assert_array_equal(d, (q.amax / np.float32(57344)).astype(np.float32))
+
+
+@pytest.mark.parametrize("fmt_a,fmt_w,fmt_dy", [("e2m1", "e2m1", "e5m2"), ("e2m1", "e4m3", "e5m2"),
+                                                ("e5m2", "e2m1", "e2m1"), ("e4m3", "e5m2", "e5m2")])
+def test_mixed_layer_with_e5m2_against_exact_rationals(fmt_a, fmt_w, fmt_dy):
+    test_mixed_layer_against_exact_rationals(fmt_a, fmt_w, fmt_dy)
