@@ -176,9 +176,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=1)
     ap.add_argument("--gemm-kind", type=int, default=0, help="0 mxf4 (K=64), 1 f8f6f4 (K=32)")
-    ap.add_argument("--precision", default="w4a4", choices=["w4a4", "w4a8", "w8a4", "w4a4-dy8"],
+    ap.add_argument("--precision", default="w4a4", choices=["w4a4", "w4a8", "w8a4", "w4a4-dy8", "w4a4-dy8e5m2"],
                     help="operand formats: w4a4 (the method, default); w4a8 / w8a4: E4M3 activations / weights "
-                         "(the ablation settings); w4a4-dy8: dY quantised to E4M3.  All but w4a4 need --gemm-kind 1")
+                         "(the ablation settings); w4a4-dy8 / w4a4-dy8e5m2: dY quantised to E4M3 / E5M2.  All but w4a4 need --gemm-kind 1")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-share-activations", action="store_true",
                     help="quantise the activation of every linear, also where q/k/v or gate/up read the same tensor")
@@ -204,7 +204,7 @@ def main():
     kind = args.gemm_kind
     fmt_a = fp4.FP4_FORMAT_E4M3 if args.precision == "w4a8" else fp4.FP4_FORMAT_E2M1
     fmt_w = fp4.FP4_FORMAT_E4M3 if args.precision == "w8a4" else fp4.FP4_FORMAT_E2M1
-    dy8 = args.precision == "w4a4-dy8"
+    dy8 = {"w4a4-dy8": fp4.FP4_FORMAT_E4M3, "w4a4-dy8e5m2": fp4.FP4_FORMAT_E5M2}.get(args.precision, fp4.FP4_FORMAT_E2M1)
     if args.precision != "w4a4":
         assert kind == 1, "E4M3 operands need the byte-container GEMM: pass --gemm-kind 1"
     if fmt_a == fp4.FP4_FORMAT_E4M3:
@@ -244,7 +244,7 @@ def main():
             fp4.fp4_linear_fwd(ctx, L["A"], L["W"], alpha, L["sa"], L["sw"], gemm_kind=kind, out=L["Y"],
                                reuse_a=L["reuse_a"])
             fp4.fp4_linear_bwd(ctx, L["G"], L["W"], L["sa"], L["sw"], gemm_kind=kind, dA=L["dA"], dW=L["dW"],
-                               dy_e4m3=dy8)
+                               dy_fmt=dy8)
 
     def step_host():
         for L in layers:
@@ -380,7 +380,7 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * sec / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None,
-            "dtype": "fp4_e2m1" if args.precision == "w4a4" else "fp4_e2m1+fp8_e4m3", "data": "synthetic",
+            "dtype": "fp4_e2m1" if args.precision == "w4a4" else ("fp4_e2m1+fp8_e5m2" if args.precision.endswith("e5m2") else "fp4_e2m1+fp8_e4m3"), "data": "synthetic",
             "config": {"workload": cfg.name, "tokens": M, "linears": [f"{L['name']}:{L['K']}x{L['N']}" for L in layers],
                        "alpha": alpha, "dge": True, "gemm_kind": "mxf4" if kind == 0 else "f8f6f4",
                        "precision": args.precision,

@@ -57,6 +57,7 @@ extern "C" {
 /* gemm_kind: which tcgen05.mma flavour multiplies the E2M1 codes */
 #define FP4_FORMAT_E2M1  0
 #define FP4_FORMAT_E4M3  1
+#define FP4_FORMAT_E5M2  2
 
 #define FP4_GEMM_MXF4    0   /* packed nibbles, K = 64 per instruction, unit block scales    */
 #define FP4_GEMM_F8F6F4  1   /* nibbles in byte containers, K = 32 per instruction           */
@@ -64,8 +65,13 @@ extern "C" {
 #define FP4_GEMM_F8F6F4_A8    2   /* a_codes are E4M3 bytes [I x C], b_codes E2M1 nibbles  */
 #define FP4_GEMM_F8F6F4_B8    3   /* a_codes E2M1 nibbles, b_codes E4M3 bytes [J x C]      */
 #define FP4_GEMM_F8F6F4_A8B8  4   /* both operands E4M3 bytes                              */
-/* fp4_linear_bwd only, OR-ed into gemm_kind (FP4_GEMM_F8F6F4): dY is quantised to E4M3 bytes */
+/* OR-ed into one of the three kinds above: that operand's bytes are E5M2 instead of E4M3 */
+#define FP4_GEMM_A_E5M2       0x10
+#define FP4_GEMM_B_E5M2       0x20
+/* fp4_linear_bwd only, OR-ed into gemm_kind (FP4_GEMM_F8F6F4): dY is quantised to E4M3 or to
+ * E5M2 bytes (one of the two) */
 #define FP4_BWD_DY_E4M3       0x100
+#define FP4_BWD_DY_E5M2       0x200
 
 typedef struct fp4_ctx fp4_ctx;   /* opaque: device id, SM count, workspace */
 
@@ -93,7 +99,9 @@ typedef struct fp4_qtensor {
                               FP4_FORMAT_E4M3: OCP E4M3 bytes, one per element (codes
                               [rows x cols], codes_t [cols x rows]), MAX = 448 in place of 6,
                               nearest-even rounding with saturation, no clamping: the FP8
-                              operand of the W4A8 / W8A4 settings of Section 4.3            */
+                              operand of the W4A8 / W8A4 settings of Section 4.3; or
+                              FP4_FORMAT_E5M2: OCP E5M2 bytes in the same layouts, MAX = 57344,
+                              saturation to the largest finite value (never an infinity)    */
   int32_t  reserved;       /* 0                                                               */
 } fp4_qtensor;
 
@@ -146,7 +154,8 @@ int fp4_quantize(fp4_ctx* ctx, void* stream, const void* x_bf16, int64_t rows, i
  *   I, J, C multiples of 128.  gemm_kind: FP4_GEMM_MXF4 or FP4_GEMM_F8F6F4.
  * With FP4_GEMM_F8F6F4_A8 / _B8 / _A8B8 the named operands are OCP E4M3 bytes, one per element
  * ([rows x C]), with d = amax / 448 (the mixed-precision settings W4A8 / W8A4 of Section 4.3);
- * the accumulation is then fp32 without the exactness E2M1 products have.
+ * the accumulation is then fp32 without the exactness E2M1 products have.  FP4_GEMM_A_E5M2 /
+ * FP4_GEMM_B_E5M2 OR-ed in make the named 8-bit operand OCP E5M2 (d = amax / 57344).
  */
 int fp4_gemm(fp4_ctx* ctx, void* stream, const uint8_t* a_codes, const uint8_t* b_codes,
              int64_t I, int64_t J, int64_t C, const float* row_amax, const float* col_amax,
@@ -158,8 +167,9 @@ int fp4_gemm(fp4_ctx* ctx, void* stream, const uint8_t* a_codes, const uint8_t* 
  * A is clamped at the alpha-quantiles and quantised token-wise, W channel-wise; the residual
  * A - A_c multiplies the BF16 weight in fp32; both branches meet in fp32 and are rounded once.
  *   A_bf16 [M x K], W_bf16 [K x N], Y [M x N] (BF16, or float if out_f32 != 0).
- *   savedA->format / savedW->format = FP4_FORMAT_E4M3 give the W4A8 / W8A4 settings of Section 4.3
- *   (gemm_kind must then be FP4_GEMM_F8F6F4; an E4M3 activation is not clamped: alpha must be 1).
+ *   savedA->format / savedW->format = FP4_FORMAT_E4M3 (or FP4_FORMAT_E5M2) give the W4A8 / W8A4
+ *   settings of Section 4.3 (gemm_kind must then be FP4_GEMM_F8F6F4; an 8-bit activation is not
+ *   clamped: alpha must be 1).
  *   savedA, savedW: caller-allocated fp4_qtensor buffers that receive the quantised operands
  *   and are handed to fp4_linear_bwd.  savedA needs codes, codes_t, amax, thresholds, nnz,
  *   csr_*, csc_*; savedW needs codes, codes_t, amax.
@@ -186,8 +196,9 @@ int fp4_linear_fwd(fp4_ctx* ctx, void* stream, const void* A_bf16, const void* W
  * multiplication by d_A[m] (wgrad), so that the forward's codes of W and A are re-used.
  *   dY_bf16 [M x N], W_bf16 [K x N], dA [M x K], dW [K x N] (BF16, or float if out_f32).
  *   dA or dW may be NULL to skip that gradient.
- *   gemm_kind | FP4_BWD_DY_E4M3 quantises both copies of dY to E4M3 bytes; the saved operands keep
- *   the formats the forward gave them; with an E4M3 weight Q' = 1 whatever dge_on says.
+ *   gemm_kind | FP4_BWD_DY_E4M3 (or FP4_BWD_DY_E5M2) quantises both copies of dY to E4M3 (E5M2)
+ *   bytes; the saved operands keep the formats the forward gave them; with an 8-bit weight Q' = 1
+ *   whatever dge_on says.
  */
 int fp4_linear_bwd(fp4_ctx* ctx, void* stream, const void* dY_bf16, const void* W_bf16,
                    const fp4_qtensor* savedA, const fp4_qtensor* savedW,

@@ -18,9 +18,13 @@ FP4_GEMM_F8F6F4 = 1
 FP4_GEMM_F8F6F4_A8 = 2
 FP4_GEMM_F8F6F4_B8 = 3
 FP4_GEMM_F8F6F4_A8B8 = 4
+FP4_GEMM_A_E5M2 = 0x10
+FP4_GEMM_B_E5M2 = 0x20
 FP4_BWD_DY_E4M3 = 0x100
+FP4_BWD_DY_E5M2 = 0x200
 FP4_FORMAT_E2M1 = 0
 FP4_FORMAT_E4M3 = 1
+FP4_FORMAT_E5M2 = 2
 FP4_DEV_SPARSE_OVERFLOW = 1
 FP4_DEV_NONFINITE = 2
 FP4_DEV_TIMEOUT = 4
@@ -183,7 +187,7 @@ class QTensor:
                  codes: bool = True, codes_t: bool = True, fmt: int = FP4_FORMAT_E2M1):
         dev = device
         self.rows, self.cols, self.scale_axis, self.fmt = rows, cols, scale_axis, fmt
-        per_byte = 2 if fmt == FP4_FORMAT_E2M1 else 1          # E2M1 nibbles or E4M3 bytes
+        per_byte = 2 if fmt == FP4_FORMAT_E2M1 else 1          # E2M1 nibbles or FP8 bytes
         self.codes = torch.empty((rows, cols // per_byte), dtype=torch.uint8, device=dev) if codes else None
         self.codes_t = torch.empty((cols, rows // per_byte), dtype=torch.uint8, device=dev) if codes_t else None
         self.amax = torch.empty(rows if scale_axis == 0 else cols, dtype=torch.float32, device=dev)
@@ -229,10 +233,11 @@ def fp4_quantize(ctx: Context, x: torch.Tensor, scale_axis: int, alpha: float = 
 
 def fp4_gemm(ctx: Context, a_codes: torch.Tensor, b_codes: torch.Tensor, row_amax=None, col_amax=None,
              out_f32: bool = True, gemm_kind: int = FP4_GEMM_MXF4, out: torch.Tensor | None = None):
-    """out = (a b^T) with the two de-scales; E2M1 operands are packed two per byte, E4M3 operands
-    (FP4_GEMM_F8F6F4_A8 / _B8 / _A8B8) one per byte."""
-    a8 = gemm_kind in (FP4_GEMM_F8F6F4_A8, FP4_GEMM_F8F6F4_A8B8)
-    b8 = gemm_kind in (FP4_GEMM_F8F6F4_B8, FP4_GEMM_F8F6F4_A8B8)
+    """out = (a b^T) with the two de-scales; E2M1 operands are packed two per byte, FP8 operands
+    (FP4_GEMM_F8F6F4_A8 / _B8 / _A8B8: E4M3, or E5M2 with FP4_GEMM_A_E5M2 / _B_E5M2 OR-ed in) one per byte."""
+    base_kind = gemm_kind & ~(FP4_GEMM_A_E5M2 | FP4_GEMM_B_E5M2)
+    a8 = base_kind in (FP4_GEMM_F8F6F4_A8, FP4_GEMM_F8F6F4_A8B8)
+    b8 = base_kind in (FP4_GEMM_F8F6F4_B8, FP4_GEMM_F8F6F4_A8B8)
     I, J = a_codes.shape[0], b_codes.shape[0]
     Cc = a_codes.shape[1] * (1 if a8 else 2)
     assert b_codes.shape[1] * (1 if b8 else 2) == Cc
@@ -268,10 +273,14 @@ def fp4_linear_fwd(ctx: Context, A: torch.Tensor, W: torch.Tensor, alpha: float,
 def fp4_linear_bwd(ctx: Context, dY: torch.Tensor, W: torch.Tensor, saved_a: QTensor, saved_w: QTensor,
                    dge_on: bool = True, dge_k: float = 5.0, dge_clip: float = 3.0,
                    gemm_kind: int = FP4_GEMM_MXF4, out_f32: bool = False, dA=None, dW=None,
-                   want_da: bool = True, want_dw: bool = True, dy_e4m3: bool = False):
-    """Backward of the layer.  `dy_e4m3` quantises dY to E4M3 bytes instead of E2M1 nibbles."""
-    if dy_e4m3:
+                   want_da: bool = True, want_dw: bool = True, dy_e4m3: bool = False,
+                   dy_fmt: int = FP4_FORMAT_E2M1):
+    """Backward of the layer.  `dy_fmt` = FP4_FORMAT_E4M3 / FP4_FORMAT_E5M2 (or `dy_e4m3`) quantises dY
+    to FP8 bytes instead of E2M1 nibbles."""
+    if dy_e4m3 or dy_fmt == FP4_FORMAT_E4M3:
         gemm_kind |= FP4_BWD_DY_E4M3
+    elif dy_fmt == FP4_FORMAT_E5M2:
+        gemm_kind |= FP4_BWD_DY_E5M2
     M, N = dY.shape
     K = W.shape[0]
     dt = torch.float32 if out_f32 else torch.bfloat16

@@ -11,6 +11,8 @@ namespace {
 
 bool mult128(int64_t v) { return v > 0 && (v % 128) == 0; }
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+bool known_format(int f) { return f == FP4_FORMAT_E2M1 || f == FP4_FORMAT_E4M3 || f == FP4_FORMAT_E5M2; }
+bool is_fp8(int f) { return f == FP4_FORMAT_E4M3 || f == FP4_FORMAT_E5M2; }
 
 size_t round256(size_t b) { return (b + 255) & ~size_t(255); }
 
@@ -180,7 +182,7 @@ int fp4_quantize(fp4_ctx* ctx, void* stream, const void* x_bf16, int64_t rows, i
   if (!(alpha > 0.5 && alpha <= 1.0)) return FP4_ERR_ALPHA;
   int rc = check_qtensor_dense(out);
   if (rc != FP4_OK) return rc;
-  if (out->format != FP4_FORMAT_E2M1 && out->format != FP4_FORMAT_E4M3) return FP4_ERR_ARG;
+  if (!known_format(out->format)) return FP4_ERR_ARG;
   if (!aligned16(x_bf16) || !aligned16(out->codes) || !aligned16(out->codes_t) || !aligned16(out->amax))
     return FP4_ERR_ALIGN;
   if (alpha < 1.0) {
@@ -205,12 +207,18 @@ int fp4_gemm(fp4_ctx* ctx, void* stream, const uint8_t* a_codes, const uint8_t* 
   if (!ctx || !a_codes || !b_codes || !out || !status) return FP4_ERR_NULL;
   if (!mult128(I) || !mult128(J) || !mult128(C)) return FP4_ERR_SHAPE;
   if (!aligned16(out)) return FP4_ERR_ALIGN;
+  const int e5m2_flags = gemm_kind & (FP4_GEMM_A_E5M2 | FP4_GEMM_B_E5M2);
+  gemm_kind &= ~(FP4_GEMM_A_E5M2 | FP4_GEMM_B_E5M2);
   if (gemm_kind < FP4_GEMM_MXF4 || gemm_kind > FP4_GEMM_F8F6F4_A8B8) return FP4_ERR_ARG;
   const bool a8 = gemm_kind == FP4_GEMM_F8F6F4_A8 || gemm_kind == FP4_GEMM_F8F6F4_A8B8;
   const bool b8 = gemm_kind == FP4_GEMM_F8F6F4_B8 || gemm_kind == FP4_GEMM_F8F6F4_A8B8;
+  // the E5M2 flags qualify an 8-bit operand
+  if (((e5m2_flags & FP4_GEMM_A_E5M2) && !a8) || ((e5m2_flags & FP4_GEMM_B_E5M2) && !b8)) return FP4_ERR_ARG;
+  const int a_format = a8 ? ((e5m2_flags & FP4_GEMM_A_E5M2) ? FP4_FORMAT_E5M2 : FP4_FORMAT_E4M3) : FP4_FORMAT_E2M1;
+  const int b_format = b8 ? ((e5m2_flags & FP4_GEMM_B_E5M2) ? FP4_FORMAT_E5M2 : FP4_FORMAT_E4M3) : FP4_FORMAT_E2M1;
   const int kind = gemm_kind >= FP4_GEMM_F8F6F4 ? FP4_GEMM_F8F6F4 : FP4_GEMM_MXF4;
   return launch_gemm_fp4(ctx, static_cast<cudaStream_t>(stream), a_codes, b_codes, I, J, C, row_amax, col_amax, out,
-                         out_f32, kind, status, nullptr, a8, b8);
+                         out_f32, kind, status, nullptr, a_format, b_format);
 }
 
 int fp4_linear_fwd(fp4_ctx* ctx, void* stream, const void* A_bf16, const void* W_bf16, int64_t M, int64_t K,
@@ -226,9 +234,9 @@ int fp4_linear_fwd(fp4_ctx* ctx, void* stream, const void* A_bf16, const void* W
   if (!aligned16(A_bf16) || !aligned16(W_bf16) || !aligned16(Y)) return FP4_ERR_ALIGN;
   const bool occ = alpha < 1.0;
   {
-    const bool a8 = savedA->format == FP4_FORMAT_E4M3, w8 = savedW->format == FP4_FORMAT_E4M3;
-    if ((savedA->format != FP4_FORMAT_E2M1 && !a8) || (savedW->format != FP4_FORMAT_E2M1 && !w8)) return FP4_ERR_ARG;
-    if ((a8 || w8) && gemm_kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;   // E4M3 needs the byte-container kind
+    const bool a8 = is_fp8(savedA->format), w8 = is_fp8(savedW->format);
+    if (!known_format(savedA->format) || !known_format(savedW->format)) return FP4_ERR_ARG;
+    if ((a8 || w8) && gemm_kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;   // FP8 operands need the byte-container kind
     if (a8 && occ) return FP4_ERR_ARG;                                    // clamping belongs to 4-bit activations
   }
   if (occ) {
@@ -291,7 +299,7 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
   }
   if (!reuse_w && ov) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[1], 0));
   // Y1 = (Q(A_c) Q(W)) * d_A[m] * d_W[n]: A codes [M x K/2], W codes transposed [N x K/2].
-  const bool a8 = savedA->format == FP4_FORMAT_E4M3, w8 = savedW->format == FP4_FORMAT_E4M3;
+  const int a8 = savedA->format, w8 = savedW->format;      // operand formats (0: E2M1)
   if (!occ) {
     // Without clamping there is no residual: a saved operand that still carries the sparse
     // structure of an earlier clamped use is marked empty, so that the backward adds nothing.
@@ -313,7 +321,7 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
       FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[7], 0));
     }
     Arena ta(scratch_tail, fwd_tail_scratch_bytes(M, K, N));
-    rc = launch_fwd_tail(ctx, st, savedA, W_bf16, savedW->amax, w8 ? 448.0f : 6.0f, ta, M, K, N, &tail, &hot_slot_of_col);
+    rc = launch_fwd_tail(ctx, st, savedA, W_bf16, savedW->amax, fp8_max(w8), ta, M, K, N, &tail, &hot_slot_of_col);
     if (rc != FP4_OK) return rc;
   }
   rc = launch_gemm_fp4(ctx, st, savedA->codes, savedW->codes_t, M, N, K, savedA->amax, savedW->amax, y1, 1, gemm_kind,
@@ -340,11 +348,13 @@ int fp4_linear_bwd(fp4_ctx* ctx, void* stream, const void* dY_bf16, const void* 
   if (!mult128(M) || !mult128(K) || !mult128(N)) return FP4_ERR_SHAPE;
   if (M * K >= (int64_t(1) << 31) || K * N >= (int64_t(1) << 31) || M * N >= (int64_t(1) << 31)) return FP4_ERR_SHAPE;
   {
-    const int kind = gemm_kind & ~FP4_BWD_DY_E4M3;
+    const int dy_flags = gemm_kind & (FP4_BWD_DY_E4M3 | FP4_BWD_DY_E5M2);
+    const int kind = gemm_kind & ~(FP4_BWD_DY_E4M3 | FP4_BWD_DY_E5M2);
     if (kind != FP4_GEMM_MXF4 && kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;
-    const bool any8 = (gemm_kind & FP4_BWD_DY_E4M3) || savedA->format == FP4_FORMAT_E4M3 ||
-                      savedW->format == FP4_FORMAT_E4M3;
-    if (any8 && kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;             // E4M3 needs the byte-container kind
+    if (dy_flags == (FP4_BWD_DY_E4M3 | FP4_BWD_DY_E5M2)) return FP4_ERR_ARG;   // one format for dY
+    if (!known_format(savedA->format) || !known_format(savedW->format)) return FP4_ERR_ARG;
+    const bool any8 = dy_flags || is_fp8(savedA->format) || is_fp8(savedW->format);
+    if (any8 && kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;             // FP8 operands need the byte-container kind
   }
   if (dge_on && !(dge_k > 1.0f && dge_clip > 0.0f)) return FP4_ERR_ARG;
   if (!savedA->codes_t || !savedA->amax || !savedW->codes || !savedW->amax) return FP4_ERR_NULL;
@@ -363,10 +373,11 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
                     float dge_k, float dge_clip, int gemm_kind, void* dA, void* dW, int out_f32, int32_t* status) {
   const bool has_comp = dW && savedA->csc_colptr != nullptr;
   float* comp = has_comp ? arena.take<float>(size_t(K) * size_t(N)) : nullptr;   // compact: one row per non-empty column
-  const bool dy8 = (gemm_kind & FP4_BWD_DY_E4M3) != 0;                 // dY as E4M3 bytes instead of E2M1 nibbles
-  gemm_kind &= ~FP4_BWD_DY_E4M3;
-  const bool a8 = savedA->format == FP4_FORMAT_E4M3, w8 = savedW->format == FP4_FORMAT_E4M3;
-  const float a_div = a8 ? 448.0f : 6.0f, w_div = w8 ? 448.0f : 6.0f;  // de-scale = amax / MAX of the operand's format
+  // dY as FP8 bytes instead of E2M1 nibbles: its format (0: E2M1)
+  const int dy8 = (gemm_kind & FP4_BWD_DY_E5M2) ? FP4_FORMAT_E5M2 : ((gemm_kind & FP4_BWD_DY_E4M3) ? FP4_FORMAT_E4M3 : 0);
+  gemm_kind &= ~(FP4_BWD_DY_E4M3 | FP4_BWD_DY_E5M2);
+  const int a8 = savedA->format, w8 = savedW->format;                  // operand formats (0: E2M1)
+  const float a_div = fp8_max(a8), w_div = fp8_max(w8);                // de-scale = amax / MAX of the operand's format
   const size_t g_bytes = size_t(M) * size_t(N) / (dy8 ? 1 : 2);
   uint8_t* g1_codes = dA ? arena.take<uint8_t>(g_bytes) : nullptr;      // dY (.) d_W, token-wise
   uint8_t* g2_codes = dW ? arena.take<uint8_t>(g_bytes) : nullptr;      // dY (.) d_A, channel-wise
@@ -405,13 +416,13 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
     }
   } else if (dA) {
     fp4_qtensor g = {};
-    g.rows = M; g.cols = N; g.codes = g1_codes; g.amax = g1_amax; g.format = dy8 ? FP4_FORMAT_E4M3 : FP4_FORMAT_E2M1;
+    g.rows = M; g.cols = N; g.codes = g1_codes; g.amax = g1_amax; g.format = dy8;
     Arena a = q_arena;
     rc = launch_quantize(ctx, st, a, dY_bf16, M, N, /*scale_axis=*/0, 1.0, savedW->amax, w_div, &g, status);
     if (rc != FP4_OK) return rc;
   } else {
     fp4_qtensor g = {};
-    g.rows = M; g.cols = N; g.codes_t = g2_codes; g.amax = g2_amax; g.format = dy8 ? FP4_FORMAT_E4M3 : FP4_FORMAT_E2M1;
+    g.rows = M; g.cols = N; g.codes_t = g2_codes; g.amax = g2_amax; g.format = dy8;
     Arena a = q_arena;
     rc = launch_quantize(ctx, st, a, dY_bf16, M, N, /*scale_axis=*/1, 1.0, savedA->amax, a_div, &g, status);
     if (rc != FP4_OK) return rc;
@@ -427,11 +438,11 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
   epi.dge_clip = dge_clip;
   // dA = d_G'[m] * sum_n G'[m,n] Wq[k,n]
   Fp4GemmDesc wgrad = {savedA->codes_t, g2_codes, K, N, M, nullptr, g2_amax, dW, out_f32, &epi};
-  wgrad.a_e4m3 = a8;
-  wgrad.b_e4m3 = dy8;
+  wgrad.a_format = a8;
+  wgrad.b_format = dy8;
   Fp4GemmDesc dgrad = {g1_codes, savedW->codes, M, K, N, g1_amax, nullptr, dA, out_f32, nullptr};
-  dgrad.a_e4m3 = dy8;
-  dgrad.b_e4m3 = w8;
+  dgrad.a_format = dy8;
+  dgrad.b_format = w8;
   const bool pairs = gemm_kind == FP4_GEMM_MXF4 && ctx->gemm_pairs;
   if (dA && dW && !pairs) {
     // Both GEMMs in one launch on the caller's stream, the weight gradient's tiles first (their

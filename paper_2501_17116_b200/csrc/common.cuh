@@ -132,6 +132,11 @@ struct GemmEpilogue {
   float dge_k, dge_clip;
 };
 
+// Largest value of an operand format: what an absmax scale maps the vector's maximum to.
+inline float fp8_max(int format) {
+  return format == FP4_FORMAT_E5M2 ? 57344.0f : (format == FP4_FORMAT_E4M3 ? 448.0f : 6.0f);
+}
+
 // Dense tail of the forward GEMM: the residual's hot columns (outlier channels, Appendix D) as extra
 // contraction columns on the tensor cores instead of per-entry gathers.  With h <= TAIL_MAX_COLS hot
 // columns, `a` is [I x TAIL_WIDTH] and `b` [J x TAIL_WIDTH] FP16, row-major, made of blocks of 64
@@ -155,8 +160,8 @@ struct GemmTail {
 int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, const uint8_t* b_codes,
                     int64_t I, int64_t J, int64_t C, const float* row_amax, const float* col_amax,
                     void* out, int out_f32, int gemm_kind, int32_t* status,
-                    const GemmEpilogue* epilogue = nullptr, bool a_e4m3 = false, bool b_e4m3 = false,
-                    const GemmTail* tail = nullptr);
+                    const GemmEpilogue* epilogue = nullptr, int a_format = FP4_FORMAT_E2M1,
+                    int b_format = FP4_FORMAT_E2M1, const GemmTail* tail = nullptr);
 
 // One GEMM, for launches that take two of them.
 struct Fp4GemmDesc {
@@ -168,8 +173,8 @@ struct Fp4GemmDesc {
   void* out;
   int out_f32;
   const GemmEpilogue* epilogue;
-  bool a_e4m3 = false;          // operand formats: E2M1 nibbles unless E4M3 bytes (byte-container kind only)
-  bool b_e4m3 = false;
+  int a_format = FP4_FORMAT_E2M1;   // operand formats: E2M1 nibbles, or E4M3 / E5M2 bytes (byte-container kind only)
+  int b_format = FP4_FORMAT_E2M1;
 };
 // Both GEMMs in one launch; the tiles of `first` are computed first.  Not available on CTA pairs.
 int launch_gemm_fp4_two(fp4_ctx* ctx, cudaStream_t stream, const Fp4GemmDesc& first, const Fp4GemmDesc& second,
@@ -203,7 +208,7 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
 int launch_quantize_dual(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void* x_bf16, int64_t rows,
                          int64_t cols, const float* amax_col_pre, const float* amax_row_pre,
                          uint8_t* codes_rows, float* amax_rows_out, uint8_t* codes_t_cols,
-                         float* amax_cols_out, int32_t* status, bool e4m3 = false, float col_pre_div = 6.0f,
+                         float* amax_cols_out, int32_t* status, int format = FP4_FORMAT_E2M1, float col_pre_div = 6.0f,
                          float row_pre_div = 6.0f);
 
 // Sparse compensation and epilogues (compensate.cu)

@@ -233,8 +233,12 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
 }
 // Instruction descriptors: M = 128, N = tile_n, both operands K-major, E2M1 x E2M1 -> fp32.
 // kind::f8f6f4 format fields: E4M3 = 0, E2M1 = 5
-__host__ __device__ constexpr uint32_t idesc_f8f6f4(bool a_e4m3 = false, bool b_e4m3 = false) {
-  return (1u << 4) | ((a_e4m3 ? 0u : 5u) << 7) | ((b_e4m3 ? 0u : 5u) << 10) |
+// format field of the byte-container kind for an operand format of the C interface
+__host__ __device__ constexpr uint32_t f8f6f4_code(int format) {
+  return format == FP4_FORMAT_E4M3 ? 0u : (format == FP4_FORMAT_E5M2 ? 1u : 5u);
+}
+__host__ __device__ constexpr uint32_t idesc_f8f6f4(int a_format = FP4_FORMAT_E2M1, int b_format = FP4_FORMAT_E2M1) {
+  return (1u << 4) | (f8f6f4_code(a_format) << 7) | (f8f6f4_code(b_format) << 10) |
          (uint32_t(tile_n(FP4_GEMM_F8F6F4) >> 3) << 17) | (uint32_t(BM >> 4) << 24);
 }
 // kind::f16 with FP16 operands (format 0) and fp32 accumulators, M = 128, N = the kind's tile width
@@ -967,7 +971,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 // Tensor map over the codes of one operand with a box of 128 bytes of shared memory x box_rows:
 // packed nibbles [rows x C/2 bytes] (E2M1) or bytes [rows x C] (E4M3, byte-container kind only).
 int make_codes_map(fp4_ctx* ctx, CUtensorMap* map, const uint8_t* codes, int64_t rows, int64_t C, int box_rows,
-                   int gemm_kind, bool e4m3) {
+                   int gemm_kind, bool e4m3 /* an FP8 format: one byte per element */) {
   EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
   if (!encode) return FP4_ERR_CUDA;
   const cuuint32_t elem_strides[2] = {1, 1};
@@ -1067,16 +1071,17 @@ int launch_kernel(int grid, cudaStream_t stream, const Problem& p, const Problem
 // Tensor maps and arguments of one GEMM.
 int make_problem(fp4_ctx* ctx, Problem* p, const Fp4GemmDesc& d, int gemm_kind, bool pair_mode, int32_t* status) {
   if (gemm_kind != FP4_GEMM_MXF4 && gemm_kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;
-  if ((d.a_e4m3 || d.b_e4m3) && gemm_kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;   // E4M3 needs the byte-container kind
+  const bool a8 = d.a_format != FP4_FORMAT_E2M1, b8 = d.b_format != FP4_FORMAT_E2M1;   // FP8 bytes
+  if ((a8 || b8) && gemm_kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;   // FP8 operands need the byte-container kind
   // The byte-container form expands 32 bytes of a packed row into 64, so its rows must start on
   // 32-byte boundaries (C/2 a multiple of 32 holds for every multiple of 128).
   const uintptr_t need = gemm_kind == FP4_GEMM_F8F6F4 ? 31 : 15;
   if ((reinterpret_cast<uintptr_t>(d.a_codes) & need) || (reinterpret_cast<uintptr_t>(d.b_codes) & need))
     return FP4_ERR_ALIGN;
-  int rc = make_codes_map(ctx, &p->map_a, d.a_codes, d.I, d.C, BM, gemm_kind, d.a_e4m3);
+  int rc = make_codes_map(ctx, &p->map_a, d.a_codes, d.I, d.C, BM, gemm_kind, a8);
   if (rc != FP4_OK) return rc;
   const int BN = tile_n(gemm_kind);
-  rc = make_codes_map(ctx, &p->map_b, d.b_codes, d.J, d.C, pair_mode ? PAIR_BN / 2 : BN, gemm_kind, d.b_e4m3);
+  rc = make_codes_map(ctx, &p->map_b, d.b_codes, d.J, d.C, pair_mode ? PAIR_BN / 2 : BN, gemm_kind, b8);
   if (rc != FP4_OK) return rc;
   if (reinterpret_cast<uintptr_t>(d.out) & 15) return FP4_ERR_ALIGN;
   rc = make_out_maps(ctx, &p->map_out, &p->map_out_aux, d.out, d.I, d.J, d.out_f32);
@@ -1092,12 +1097,12 @@ int make_problem(fp4_ctx* ctx, Problem* p, const Fp4GemmDesc& d, int gemm_kind, 
   // The transaction count of a copy is in bytes read from global memory: the byte-container form
   // fills a stage's 128-byte rows from 64 bytes of packed nibbles (E2M1) or from 128 bytes (E4M3).
   if (gemm_kind == FP4_GEMM_F8F6F4)
-    args.tx_bytes = uint32_t(A_STAGE_BYTES / (d.a_e4m3 ? 1 : 2) + b_stage_bytes(gemm_kind) / (d.b_e4m3 ? 1 : 2));
+    args.tx_bytes = uint32_t(A_STAGE_BYTES / (a8 ? 1 : 2) + b_stage_bytes(gemm_kind) / (b8 ? 1 : 2));
   else
     args.tx_bytes = stage_bytes(gemm_kind);
-  args.idesc = gemm_kind == FP4_GEMM_F8F6F4 ? idesc_f8f6f4(d.a_e4m3, d.b_e4m3) : idesc_mxf4();
-  args.row_div = d.a_e4m3 ? 448.0f : 6.0f;
-  args.col_div = d.b_e4m3 ? 448.0f : 6.0f;
+  args.idesc = gemm_kind == FP4_GEMM_F8F6F4 ? idesc_f8f6f4(d.a_format, d.b_format) : idesc_mxf4();
+  args.row_div = fp8_max(d.a_format);
+  args.col_div = fp8_max(d.b_format);
   args.row_amax = d.row_amax;
   args.col_amax = d.col_amax;
   args.out = d.out;
@@ -1123,11 +1128,11 @@ int make_problem(fp4_ctx* ctx, Problem* p, const Fp4GemmDesc& d, int gemm_kind, 
 
 int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, const uint8_t* b_codes, int64_t I,
                     int64_t J, int64_t C, const float* row_amax, const float* col_amax, void* out, int out_f32,
-                    int gemm_kind, int32_t* status, const GemmEpilogue* epi, bool a_e4m3, bool b_e4m3,
+                    int gemm_kind, int32_t* status, const GemmEpilogue* epi, int a_format, int b_format,
                     const GemmTail* tail) {
   Fp4GemmDesc d = {a_codes, b_codes, I, J, C, row_amax, col_amax, out, out_f32, epi};
-  d.a_e4m3 = a_e4m3;
-  d.b_e4m3 = b_e4m3;
+  d.a_format = a_format;
+  d.b_format = b_format;
   const bool pair_mode = gemm_kind == FP4_GEMM_MXF4 && ctx->gemm_pairs;
   Problem p;
   int rc = make_problem(ctx, &p, d, gemm_kind, pair_mode, status);

@@ -491,6 +491,8 @@ struct EncodeArgs {
   uint8_t* mask;                // clamp: [rows x cols/8] bytes
   int* row_cnt;                 // clamp: clamped entries per row (zero-initialised)
   uint8_t* strip_cnt;           // clamp: [rows/64 x cols] clamped entries per (strip, column)
+  float fmax;                   // FP8 encoder: the format's largest value (448 or 57344)
+  int e5m2;                     // FP8 encoder: E5M2 bytes instead of E4M3 bytes
 };
 
 // MODE_ROWS: one scale per row -> codes and / or codes_t.  MODE_COLS: one scale per column.
@@ -639,13 +641,16 @@ encode_kernel(const EncodeArgs a) {
 }
 
 // ------------------------------------------------------------------------------------------
-// 3b. E4M3 encoder (FP8 operands of the W4A8 / W8A4 settings and of the FP8 reading of dY)
+// 3b. FP8 encoder (FP8 operands of the W4A8 / W8A4 settings and of the FP8 reading of dY)
 // ------------------------------------------------------------------------------------------
-// Two floats -> two E4M3 bytes (first value in the low byte): nearest even, saturating at 448,
-// the sign kept also on zero.
-__device__ __forceinline__ uint32_t e4m3x2(float lo, float hi) {
+// Two floats -> two FP8 bytes (first value in the low byte), E4M3 or E5M2: nearest even, saturating
+// at the format's largest finite value (448 / 57344), the sign kept also on zero.
+__device__ __forceinline__ uint32_t fp8x2(float lo, float hi, int e5m2) {
   uint16_t r;
-  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+  if (e5m2)
+    asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+  else
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
   return r;
 }
 // 4 x 4 byte transpose: in[r] byte c -> out[c] byte r
@@ -663,7 +668,7 @@ __device__ __forceinline__ void transpose4x4_bytes(uint32_t a0, uint32_t a1, uin
 // clamping: outlier clamping belongs to 4-bit activations.
 template <int MODE, bool PRESCALE>
 __global__ void __launch_bounds__(ENC_THREADS)
-encode_e4m3_kernel(const EncodeArgs a) {
+encode_fp8_kernel(const EncodeArgs a) {
   __shared__ float s_gcol[ENC_TK];
   __shared__ float s_grow[ENC_TM];
   __shared__ float s_prow[ENC_TM];
@@ -678,14 +683,14 @@ encode_e4m3_kernel(const EncodeArgs a) {
   if (ROW_SCALED && tid < ENC_TM) {
     const int r = row0 + tid;
     const float amax = __uint_as_float(a.amax_rows[r]);
-    s_grow[tid] = amax > 0.0f ? __fdiv_rn(448.0f, amax) : 0.0f;
+    s_grow[tid] = amax > 0.0f ? __fdiv_rn(a.fmax, amax) : 0.0f;
     if (blockIdx.x == 0) a.amax_out_rows[r] = amax;
   }
   if (COL_SCALED) {
     const int c = col0 + tid;
     if (c < a.cols) {
       const float amax = __uint_as_float(a.amax_cols[c]);
-      s_gcol[tid] = amax > 0.0f ? __fdiv_rn(448.0f, amax) : 0.0f;
+      s_gcol[tid] = amax > 0.0f ? __fdiv_rn(a.fmax, amax) : 0.0f;
       if (blockIdx.y == 0) a.amax_out_cols[c] = amax;
     }
     if (PRESCALE && tid < ENC_TM) s_prow[tid] = __ldg(&a.pre_row[row0 + tid]);
@@ -729,13 +734,13 @@ encode_e4m3_kernel(const EncodeArgs a) {
         f2[c] = __fmul_rn(__fmul_rn(xv, prow), gc[c]);
       }
     }
-    const uint32_t b_lo = e4m3x2(f[0], f[1]) | (e4m3x2(f[2], f[3]) << 16);
-    const uint32_t b_hi = e4m3x2(f[4], f[5]) | (e4m3x2(f[6], f[7]) << 16);
+    const uint32_t b_lo = fp8x2(f[0], f[1], a.e5m2) | (fp8x2(f[2], f[3], a.e5m2) << 16);
+    const uint32_t b_hi = fp8x2(f[4], f[5], a.e5m2) | (fp8x2(f[6], f[7], a.e5m2) << 16);
     if (in_cols && codes8)
       *reinterpret_cast<uint2*>(codes8 + (long long)(row0 + 8 * warp + r) * a.cols + col) = make_uint2(b_lo, b_hi);
     if constexpr (MODE == MODE_DUAL) {
-      lo4[r] = e4m3x2(f2[0], f2[1]) | (e4m3x2(f2[2], f2[3]) << 16);
-      hi4[r] = e4m3x2(f2[4], f2[5]) | (e4m3x2(f2[6], f2[7]) << 16);
+      lo4[r] = fp8x2(f2[0], f2[1], a.e5m2) | (fp8x2(f2[2], f2[3], a.e5m2) << 16);
+      hi4[r] = fp8x2(f2[4], f2[5], a.e5m2) | (fp8x2(f2[6], f2[7], a.e5m2) << 16);
     } else {
       lo4[r] = b_lo;
       hi4[r] = b_hi;
@@ -955,7 +960,7 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
   const int rows = int(rows64), cols = int(cols64);
   const long long n = (long long)rows * cols;
   const bool occ = alpha < 1.0;
-  const bool e4m3 = out->format == FP4_FORMAT_E4M3;
+  const bool e4m3 = out->format == FP4_FORMAT_E4M3 || out->format == FP4_FORMAT_E5M2;   // an FP8 format
   if (out->format != FP4_FORMAT_E2M1 && !e4m3) return FP4_ERR_ARG;
   if (e4m3 && occ) return FP4_ERR_ARG;               // outlier clamping belongs to 4-bit activations
   const uint4* x = static_cast<const uint4*>(x_bf16);
@@ -978,6 +983,8 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
   ea.mask = sc.mask;
   ea.row_cnt = sc.row_cnt;
   ea.strip_cnt = sc.strip_cnt;
+  ea.e5m2 = out->format == FP4_FORMAT_E5M2;
+  ea.fmax = fp8_max(out->format);
   const dim3 tile_grid((cols + ENC_TK - 1) / ENC_TK, rows / ENC_TM);
 
   if (occ) {
@@ -1057,9 +1064,9 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
       }
       KernelScope scope(ctx, stream, KC_ENCODE, 1);
       if (e4m3 && prescale)
-        encode_e4m3_kernel<MODE_ROWS, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
+        encode_fp8_kernel<MODE_ROWS, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
       else if (e4m3)
-        encode_e4m3_kernel<MODE_ROWS, false><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
+        encode_fp8_kernel<MODE_ROWS, false><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
       else if (prescale)
         encode_kernel<MODE_ROWS, false, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
       else
@@ -1074,9 +1081,9 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
       }
       KernelScope scope(ctx, stream, KC_ENCODE, 1);
       if (e4m3 && prescale)
-        encode_e4m3_kernel<MODE_COLS, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
+        encode_fp8_kernel<MODE_COLS, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
       else if (e4m3)
-        encode_e4m3_kernel<MODE_COLS, false><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
+        encode_fp8_kernel<MODE_COLS, false><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
       else if (prescale)
         encode_kernel<MODE_COLS, false, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
       else
@@ -1092,7 +1099,8 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
 int launch_quantize_dual(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void* x_bf16, int64_t rows64,
                          int64_t cols64, const float* amax_col_pre, const float* amax_row_pre, uint8_t* codes_rows,
                          float* amax_rows_out, uint8_t* codes_t_cols, float* amax_cols_out, int32_t* status,
-                         bool e4m3, float col_pre_div, float row_pre_div) {
+                         int format, float col_pre_div, float row_pre_div) {
+  const bool e4m3 = format != FP4_FORMAT_E2M1;       // an FP8 format
   const int rows = int(rows64), cols = int(cols64);
   Scratch sc = carve(arena, rows, cols, false);
   if (!sc.ok) return FP4_ERR_WORKSPACE;
@@ -1130,9 +1138,11 @@ int launch_quantize_dual(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const 
   ea.codes_t = reinterpret_cast<uint32_t*>(codes_t_cols);
   ea.amax_out_rows = amax_rows_out;
   ea.amax_out_cols = amax_cols_out;
+  ea.e5m2 = format == FP4_FORMAT_E5M2;
+  ea.fmax = fp8_max(format);
   KernelScope scope(ctx, stream, KC_ENCODE, 1);
   if (e4m3)
-    encode_e4m3_kernel<MODE_DUAL, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
+    encode_fp8_kernel<MODE_DUAL, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
   else
     encode_kernel<MODE_DUAL, false, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
   FP4_CUDA_TRY(cudaGetLastError());

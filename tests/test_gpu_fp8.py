@@ -85,12 +85,15 @@ CASES = [
     (384, 640, 384, "e2m1", "e2m1", "e4m3", 0.99),    # dY in FP8
     (128, 256, 128, "e4m3", "e2m1", "e4m3", 1.0),
     (256, 1152, 256, "e2m1", "e4m3", "e4m3", 0.99),
+    (384, 640, 384, "e2m1", "e2m1", "e5m2", 0.99),    # dY in E5M2, the usual FP8 format of gradients
+    (256, 384, 640, "e2m1", "e4m3", "e5m2", 0.98),    # W8A4 with E5M2 gradients
+    (128, 256, 128, "e5m2", "e2m1", "e5m2", 1.0),
 ]
 
 
 @pytest.mark.parametrize("M,K,N,fmt_a,fmt_w,fmt_dy,alpha", CASES)
 def test_mixed_precision_layer_matches_oracle(lib, ctx, M, K, N, fmt_a, fmt_w, fmt_dy, alpha):
-    code = {"e2m1": lib.FP4_FORMAT_E2M1, "e4m3": lib.FP4_FORMAT_E4M3}
+    code = {"e2m1": lib.FP4_FORMAT_E2M1, "e4m3": lib.FP4_FORMAT_E4M3, "e5m2": lib.FP4_FORMAT_E5M2}
     a_bits, w_bits, dy_bits = WL.small_case(M, K, N, seed=M + K + N)
     f = O.linear_fwd(a_bits, w_bits, alpha, fmt_a=fmt_a, fmt_w=fmt_w)
     b = O.linear_bwd(dy_bits, w_bits, f, fmt_dy=fmt_dy)
@@ -98,10 +101,10 @@ def test_mixed_precision_layer_matches_oracle(lib, ctx, M, K, N, fmt_a, fmt_w, f
     kind = lib.FP4_GEMM_F8F6F4
     ctx.status.zero_()
     y32, sa, sw = lib.fp4_linear_fwd(ctx, A, W, alpha, gemm_kind=kind, out_f32=True, fmt_a=code[fmt_a], fmt_w=code[fmt_w])
-    da32, dw32 = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, gemm_kind=kind, out_f32=True, dy_e4m3=fmt_dy == "e4m3")
-    da_only, _ = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, gemm_kind=kind, out_f32=True, dy_e4m3=fmt_dy == "e4m3",
+    da32, dw32 = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, gemm_kind=kind, out_f32=True, dy_fmt=code[fmt_dy])
+    da_only, _ = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, gemm_kind=kind, out_f32=True, dy_fmt=code[fmt_dy],
                                     want_dw=False)
-    _, dw_only = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, gemm_kind=kind, out_f32=True, dy_e4m3=fmt_dy == "e4m3",
+    _, dw_only = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, gemm_kind=kind, out_f32=True, dy_fmt=code[fmt_dy],
                                     want_da=False)
     torch.cuda.synchronize()
     assert ctx.read_status() == 0
@@ -115,5 +118,68 @@ def test_mixed_precision_layer_matches_oracle(lib, ctx, M, K, N, fmt_a, fmt_w, f
     _close(da32.cpu().numpy(), b.da, b.da, None, "dA")
     _close(dw32.cpu().numpy(), b.dw, b.s_fp4 * b.dge, b.s_comp * b.dge, "dW")
     assert torch.equal(da_only, da32) and torch.equal(dw_only, dw32)     # one-gradient calls take the same path
-    if fmt_w == "e4m3":
+    if fmt_w != "e2m1":
         assert (b.dge == 1.0).all()
+
+
+@pytest.mark.parametrize("axis", [0, 1])
+@pytest.mark.parametrize("shape", [(128, 128), (256, 384)])
+def test_e5m2_quantize_matches_oracle(lib, ctx, axis, shape):
+    rng = np.random.default_rng(shape[0] + shape[1] + axis + 50)
+    x = rng.standard_normal(shape).astype(np.float32) * np.exp2(rng.integers(-12, 4, size=shape)).astype(np.float32)
+    bits = WL.to_bf16_bits(x)                          # wide range: E5M2 subnormals are reached
+    bits[3, :] = 0
+    bits[7, 9] = 0x8000                               # negative zero input keeps its sign
+    ctx.status.zero_()
+    q = lib.fp4_quantize(ctx, _dev(bits), axis, fmt=lib.FP4_FORMAT_E5M2)
+    torch.cuda.synchronize()
+    assert ctx.read_status() == 0
+    ref = O.absmax_quantize(O.bf16_bits_to_f64(bits), axis, fmt="e5m2")
+    np.testing.assert_array_equal(q.amax.cpu().numpy(), ref.amax)
+    np.testing.assert_array_equal(q.codes.cpu().numpy(), ref.codes)
+    np.testing.assert_array_equal(q.codes_t.cpu().numpy(), np.ascontiguousarray(ref.codes.T))
+
+
+def test_e5m2_conversion_on_every_bf16_value_in_range(lib, ctx):
+    """Rows whose amax is 57344 (gamma = 1) carry every BF16 value up to 57344: every E5M2 value,
+    every midpoint between two of them (BF16 has five more mantissa bits) and their neighbours."""
+    bits = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    v = O.bf16_bits_to_f64(bits)
+    keep = bits[np.isfinite(v) & (np.abs(v) <= 57344.0)]
+    cols = 256
+    rows = -(-keep.size // (cols - 1))
+    rows = -(-rows // 128) * 128
+    x = np.zeros((rows, cols), dtype=np.uint16)
+    x[:, 0] = 0x4760                                   # 57344.0 in every row -> gamma = 1
+    body = np.zeros(rows * (cols - 1), dtype=np.uint16)
+    body[:keep.size] = keep
+    x[:, 1:] = body.reshape(rows, cols - 1)
+    q = lib.fp4_quantize(ctx, _dev(x), 0, fmt=lib.FP4_FORMAT_E5M2)
+    torch.cuda.synchronize()
+    ref = O.absmax_quantize(O.bf16_bits_to_f64(x), 0, fmt="e5m2")
+    assert (ref.amax == 57344.0).all()
+    np.testing.assert_array_equal(q.codes.cpu().numpy(), ref.codes)
+
+
+def test_gemm_with_e5m2_operands(lib, ctx):
+    """fp4_gemm on the byte-container kind with an E5M2 operand on either side."""
+    rng = np.random.default_rng(9)
+    I, J, C = 128, 256, 384
+    xa = O.bf16_bits_to_f64(WL.to_bf16_bits(rng.standard_normal((I, C)).astype(np.float32)))
+    xb = O.bf16_bits_to_f64(WL.to_bf16_bits(rng.standard_normal((J, C)).astype(np.float32)))
+    for fa, fb, kind in (("e5m2", "e2m1", lib.FP4_GEMM_F8F6F4_A8 | lib.FP4_GEMM_A_E5M2),
+                         ("e2m1", "e5m2", lib.FP4_GEMM_F8F6F4_B8 | lib.FP4_GEMM_B_E5M2),
+                         ("e5m2", "e4m3", lib.FP4_GEMM_F8F6F4_A8B8 | lib.FP4_GEMM_A_E5M2)):
+        qa, qb = O.absmax_quantize(xa, 0, fmt=fa), O.absmax_quantize(xb, 0, fmt=fb)
+        ca = torch.from_numpy(qa.packed() if fa == "e2m1" else qa.codes).cuda()
+        cb = torch.from_numpy(qb.packed() if fb == "e2m1" else qb.codes).cuda()
+        got = lib.fp4_gemm(ctx, ca, cb, torch.from_numpy(qa.amax).cuda(), torch.from_numpy(qb.amax).cuda(),
+                           gemm_kind=kind)
+        torch.cuda.synchronize()
+        want = (O.gemm_values(qa, qb) * qa.descale.astype(np.float64)[:, None]) * qb.descale.astype(np.float64)[None, :]
+        terms = (np.abs(qa.values()) @ np.abs(qb.values()).T) * qa.descale.astype(np.float64)[:, None] \
+            * qb.descale.astype(np.float64)[None, :]
+        err = np.abs(got.cpu().numpy().astype(np.float64) - want)
+        assert (err <= RTOL * np.abs(want) + 2 * (C // 32) * 2.0 ** -23 * terms).all(), (fa, fb)
+    with pytest.raises(lib.Fp4Error):                  # the E5M2 flag qualifies an 8-bit operand
+        lib.fp4_gemm(ctx, ca, cb, None, None, gemm_kind=lib.FP4_GEMM_F8F6F4 | lib.FP4_GEMM_A_E5M2)

@@ -47,8 +47,8 @@ def _draws(n, seed):
         kind = int(rng.integers(0, 2))
         dge = bool(rng.integers(0, 2))
         # FP8 settings need the byte-container kind; an E4M3 activation is not clamped
-        fp8 = str(rng.choice(["none", "none", "w8", "a8", "dy8", "w8+dy8"])) if kind == 1 else "none"
-        if fp8 == "a8":
+        fp8 = str(rng.choice(["none", "none", "w8", "a8", "dy8", "w8+dy8", "dy5", "w8+dy5", "a5"])) if kind == 1 else "none"
+        if fp8 in ("a8", "a5"):
             alpha = 1.0
         out.append((i, M, K, N, alpha, dist, hot, kind, dge, fp8))
     return out
@@ -58,10 +58,10 @@ def _draws(n, seed):
                          _draws(int(os.environ.get("FP4_RANDOM_DRAWS", "16")), seed=2501))
 def test_random_layer_matches_oracle(lib, ctx, i, M, K, N, alpha, dist, hot, kind, dge, fp8):
     a_bits, w_bits, dy_bits = WL.small_case(M, K, N, seed=1000 + i, alpha_outliers=hot, dist=dist)
-    fmt_a = "e4m3" if fp8 == "a8" else "e2m1"
+    fmt_a = {"a8": "e4m3", "a5": "e5m2"}.get(fp8, "e2m1")
     fmt_w = "e4m3" if "w8" in fp8 else "e2m1"
-    fmt_dy = "e4m3" if "dy8" in fp8 else "e2m1"
-    code = {"e2m1": lib.FP4_FORMAT_E2M1, "e4m3": lib.FP4_FORMAT_E4M3}
+    fmt_dy = "e4m3" if "dy8" in fp8 else ("e5m2" if "dy5" in fp8 else "e2m1")
+    code = {"e2m1": lib.FP4_FORMAT_E2M1, "e4m3": lib.FP4_FORMAT_E4M3, "e5m2": lib.FP4_FORMAT_E5M2}
     f = O.linear_fwd(a_bits, w_bits, alpha, fmt_a=fmt_a, fmt_w=fmt_w)
     b = O.linear_bwd(dy_bits, w_bits, f, dge_on=dge, fmt_dy=fmt_dy)
     A, W, dY = _dev(a_bits), _dev(w_bits), _dev(dy_bits)
@@ -69,10 +69,10 @@ def test_random_layer_matches_oracle(lib, ctx, i, M, K, N, alpha, dist, hot, kin
     y32, sa, sw = lib.fp4_linear_fwd(ctx, A, W, alpha, gemm_kind=kind, out_f32=True, fmt_a=code[fmt_a],
                                      fmt_w=code[fmt_w])
     da32, dw32 = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, gemm_kind=kind, out_f32=True, dge_on=dge,
-                                    dy_e4m3=fmt_dy == "e4m3")
+                                    dy_fmt=code[fmt_dy])
     torch.cuda.synchronize()
     assert ctx.read_status() == 0
-    if fp8 in ("none", "dy8"):
+    if fp8 in ("none", "dy8", "dy5"):
         _saved_matches(sa, sw, f)
     else:
         np.testing.assert_array_equal(sa.amax.cpu().numpy(), f.qa.amax)
@@ -90,11 +90,11 @@ def test_random_layer_matches_oracle(lib, ctx, i, M, K, N, alpha, dist, hot, kin
     va, vw = np.abs(f.qa.values()), np.abs(f.qw.values())
     vg1, vg2 = np.abs(b.qg_dgrad.values()), np.abs(b.qg_wgrad.values())
     d64 = lambda q: q.descale.astype(np.float64)
-    if fmt_a == "e4m3" or fmt_w == "e4m3":
+    if fmt_a != "e2m1" or fmt_w != "e2m1":
         floor_y = floor_y + _fp8_floor((va @ vw) * d64(f.qa)[:, None] * d64(f.qw)[None, :], K)
-    if fmt_dy == "e4m3" or fmt_w == "e4m3":
+    if fmt_dy != "e2m1" or fmt_w != "e2m1":
         floor_da = _fp8_floor((vg1 @ vw.T) * d64(b.qg_dgrad)[:, None], N)
-    if fmt_a == "e4m3" or fmt_dy == "e4m3":
+    if fmt_a != "e2m1" or fmt_dy != "e2m1":
         floor_dw = _fp8_floor((va.T @ vg2) * d64(b.qg_wgrad)[None, :] * b.dge, M)
     assert_close_f32(y32.cpu().numpy(), f.y, f.y_fp4, f.y_comp, "Y", floor_y)
     assert_close_f32(da32.cpu().numpy(), b.da, b.da, None, "dA", floor_da)
