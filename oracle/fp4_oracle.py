@@ -302,13 +302,24 @@ def tail_count(n: int, alpha: float) -> int:
     return int(math.floor((1.0 - float(alpha)) * float(n) + 0.5))
 
 
-def quantile_thresholds(a, alpha: float):
-    """(lo, hi, n_tail): the (1-alpha)- and alpha-quantiles as order statistics."""
+def quantile_thresholds(a, alpha: float, quantile: str = "signed"):
+    """(lo, hi, n_tail): the (1-alpha)- and alpha-quantiles as order statistics.
+
+    ``quantile`` = "signed" is the paper's form (Section 3.2: clamp between the alpha-quantile and
+    the (1-alpha)-quantile of the values).  "abs" is a variant outside the paper: one threshold t
+    on the magnitudes, the order statistic of |x| that at most 2 n_tail entries exceed, with
+    lo = -t and hi = +t (the same number of entries may leave the clamp as in the signed form).
+    """
     a = np.asarray(a, dtype=np.float64)
     n = a.size
     n_tail = tail_count(n, alpha)
     if not (2 * n_tail < n):
         raise ValueError("alpha leaves nothing between the two tails")
+    if quantile == "abs":
+        t = float(np.sort(np.abs(a).ravel())[n - 1 - 2 * n_tail])
+        return -t + 0.0, t, n_tail            # "+ 0.0" turns -0.0 into +0.0
+    if quantile != "signed":
+        raise ValueError(quantile)
     s = np.sort(a.ravel())
     lo = float(s[n_tail]) + 0.0             # "+ 0.0" turns -0.0 into +0.0
     hi = float(s[n - 1 - n_tail]) + 0.0
@@ -337,7 +348,7 @@ def sparse_from_dense(r):
     return csr, csc
 
 
-def occ_quantize(a, alpha: float) -> Quantized:
+def occ_quantize(a, alpha: float, quantile: str = "signed") -> Quantized:
     """Clamp at the quantiles, keep the sparse residual, then token-wise absmax + Q.
 
     The clamp comes first: its purpose is to shrink the range the absmax scale
@@ -350,7 +361,7 @@ def occ_quantize(a, alpha: float) -> Quantized:
         q.csr, q.csc = sparse_from_dense(q.residual)
         q.lo, q.hi = float("-inf"), float("inf")
         return q
-    lo, hi, n_tail = quantile_thresholds(a, alpha)
+    lo, hi, n_tail = quantile_thresholds(a, alpha, quantile)
     a_c, r = occ_split(a, lo, hi)
     q = absmax_quantize(a_c, 0)
     q.lo, q.hi, q.n_tail = lo, hi, n_tail
@@ -436,7 +447,8 @@ class Forward:
     qw: Quantized
 
 
-def linear_fwd(a_bits, w_bits, alpha: float, fmt_a: str = "e2m1", fmt_w: str = "e2m1") -> Forward:
+def linear_fwd(a_bits, w_bits, alpha: float, fmt_a: str = "e2m1", fmt_w: str = "e2m1",
+               quantile: str = "signed") -> Forward:
     """Y = (Q(A_c) Q(W)) (.) scales + dA W  (Fig. 2, Section 3.2).
 
     ``a_bits`` uint16 [M, K] and ``w_bits`` uint16 [K, N] are BF16 bit patterns.
@@ -446,7 +458,7 @@ def linear_fwd(a_bits, w_bits, alpha: float, fmt_a: str = "e2m1", fmt_w: str = "
     a = bf16_bits_to_f64(a_bits)
     w = bf16_bits_to_f64(w_bits)
     if fmt_a == "e2m1":
-        qa = occ_quantize(a, alpha)             # token-wise, with OCC
+        qa = occ_quantize(a, alpha, quantile)   # token-wise, with OCC
     else:
         if alpha != 1.0:
             raise ValueError("outlier clamping belongs to 4-bit activations")

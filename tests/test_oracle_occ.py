@@ -158,3 +158,40 @@ def test_compensation_trend_of_table1():
         snr.append(_snr_db(a, rec))
     assert snr[1] > snr[0]
     assert snr[1] < snr[2] < snr[3]
+
+
+# ---------------------------------------------------------------------------------------------
+# The variant outside the paper: one threshold on the magnitudes
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("n,alpha", [(50, 0.9), (1000, 0.99), (4096, 0.97), (777, 0.999)])
+def test_abs_threshold_by_counting(n, alpha):
+    """t is characterised without sorting: at most 2 n_tail magnitudes lie above it and more than
+    2 n_tail lie at or above it; the clamp is symmetric."""
+    rng = np.random.default_rng(n)
+    a = np.round(rng.standard_normal(n) * 8) / 8 * rng.choice([1.0, 30.0], n, p=[0.95, 0.05])   # with ties
+    lo, hi, n_tail = O.quantile_thresholds(a, alpha, quantile="abs")
+    assert lo == -hi and hi >= 0 and n_tail == O.tail_count(n, alpha)
+    assert np.sum(np.abs(a) > hi) <= 2 * n_tail < np.sum(np.abs(a) >= hi)
+    assert hi in np.abs(a)                                  # an order statistic, not an interpolation
+
+
+def test_abs_threshold_on_a_hand_worked_case():
+    a = np.array([0.5, -7.0, 2.0, -1.0, 3.0, 0.0, -0.25, 6.0, 1.5, -2.5])      # magnitudes sorted: 0 .25 .5 1 1.5 2 2.5 3 6 7
+    lo, hi, n_tail = O.quantile_thresholds(a, 0.9, quantile="abs")              # n_tail = 1: two entries may leave
+    assert (lo, hi, n_tail) == (-3.0, 3.0, 1)
+    q = O.occ_quantize(a.reshape(1, -1), 0.9, quantile="abs")
+    np.testing.assert_array_equal(q.residual, np.array([[0, -4.0, 0, 0, 0, 0, 0, 3.0, 0, 0]]))
+    z = np.zeros(10)
+    z[3] = -5.0
+    assert O.quantile_thresholds(z, 0.8, quantile="abs")[:2] == (0.0, 0.0)      # t = 0: lo is +0, not -0
+    assert not np.signbit(O.quantile_thresholds(z, 0.8, quantile="abs")[0])
+
+
+def test_abs_and_signed_forms_agree_on_mirrored_data():
+    """A tensor that holds -x for every x has symmetric order statistics: both forms clamp alike."""
+    rng = np.random.default_rng(4)
+    h = rng.standard_normal(500)
+    a = np.concatenate([h, -h])
+    s = O.quantile_thresholds(a, 0.99)
+    b = O.quantile_thresholds(a, 0.99, quantile="abs")
+    assert s[1] == b[1] and s[0] == b[0] == -s[1]
