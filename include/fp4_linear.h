@@ -255,6 +255,14 @@ int fp4_set_overlap(fp4_ctx* ctx, int on);
 /* MXF4 GEMMs on pairs of CTAs (tcgen05.mma.cta_group::2, 256 x 240 tile per pair: a third less
  * operand traffic from L2 per flop).  Same results bit for bit.  Default: off.               */
 int fp4_set_gemm_pairs(fp4_ctx* ctx, int on);
+/* Which order statistics the clamp of an activation uses (fp4_quantize with alpha < 1 and the
+ * calls built on it; not fp4_quantile_thresholds_static).  FP4_QUANTILE_SIGNED (default): the
+ * paper's form (Section 3.2), lo and hi the (1-alpha)- and alpha-quantiles of the values.
+ * FP4_QUANTILE_ABS, a variant outside the paper: one threshold t on the magnitudes, the order
+ * statistic of |x| that at most 2 n_tail entries exceed; lo = -t, hi = t.                     */
+#define FP4_QUANTILE_SIGNED 0
+#define FP4_QUANTILE_ABS    1
+int fp4_set_quantile_mode(fp4_ctx* ctx, int mode);
 int fp4_profile_reset(fp4_ctx* ctx);
 int fp4_profile_read(fp4_ctx* ctx, int kernel_class, double* total_ms, int64_t* launches);
 int64_t fp4_launch_count(fp4_ctx* ctx);

@@ -104,6 +104,7 @@ int fp4_create(fp4_ctx** out, int device, size_t workspace_bytes) {
   for (auto& e : ctx->host_step_copied) e = nullptr;
   for (auto& e : ctx->host_step_computed) e = nullptr;
   ctx->host_step_parity = 0;
+  ctx->quantile_mode = FP4_QUANTILE_SIGNED;
   cudaDeviceProp prop;
   if (!ctx->records || cudaGetDeviceProperties(&prop, device) != cudaSuccess) {
     delete ctx->records;
@@ -621,6 +622,13 @@ int fp4_linear_step_host(fp4_ctx* ctx, void* stream, const void* A_host, const v
 int fp4_set_overlap(fp4_ctx* ctx, int on) {
   if (!ctx) return FP4_ERR_NULL;
   ctx->overlap = on ? 1 : 0;
+  return FP4_OK;
+}
+
+int fp4_set_quantile_mode(fp4_ctx* ctx, int mode) {
+  if (!ctx) return FP4_ERR_NULL;
+  if (mode != FP4_QUANTILE_SIGNED && mode != FP4_QUANTILE_ABS) return FP4_ERR_ARG;
+  ctx->quantile_mode = mode;
   return FP4_OK;
 }
 

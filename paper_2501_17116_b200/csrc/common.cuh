@@ -50,6 +50,7 @@ struct fp4_ctx {
   cudaEvent_t  host_step_computed[HOST_STEP_SETS];// the outputs of set i are complete on the device
   cudaEvent_t  host_step_done[HOST_STEP_SETS];    // the call that used set i has left the workspace
   int      host_step_parity;         // set of the next pipelined call
+  int      quantile_mode;            // FP4_QUANTILE_SIGNED (the paper's clamp) or FP4_QUANTILE_ABS
   int      overlap;            // run independent kernel chains on the side streams (default on)
   int      gemm_pairs;         // MXF4 GEMM on pairs of CTAs (tcgen05 cta_group::2)
   int      profile;            // record CUDA events around every kernel class

@@ -109,7 +109,7 @@ __device__ __forceinline__ int bits_to_pos(uint32_t bits) { return (bits & 0x800
 __global__ void __launch_bounds__(HIST_THREADS, 1)
 hist_select_kernel(const uint4* __restrict__ x, int rows, int vec_per_row, uint32_t* sets, unsigned* parity,
                    int* __restrict__ row_max, int* __restrict__ row_min, int* __restrict__ row_cnt, long long n,
-                   long long n_tail, float* __restrict__ thresholds, unsigned* ticket, int32_t* status) {
+                   long long n_tail, float* __restrict__ thresholds, unsigned* ticket, int32_t* status, int abs_mode) {
   extern __shared__ uint32_t h[];
   __shared__ uint32_t s_top;
   __shared__ int s_rmax[HIST_ROW_SLOTS], s_rmin[HIST_ROW_SLOTS];
@@ -282,8 +282,11 @@ hist_select_kernel(const uint4* __restrict__ x, int rows, int vec_per_row, uint3
     static_assert(HIST_THREADS == 1024, "two ranks x sixteen steps, one warp each");
     __shared__ long long s_step[2][16];
     const int warp = tid >> 5, lane = tid & 31, q = warp >> 4, st = warp & 15;
-    const long long rank = q == 0 ? n_tail : n - 1 - n_tail;
-    const long long cc = __ldcg(&gcoarse[lane]);
+    // abs_mode: one rank in the order of the magnitudes (both warp groups find it, the first writes
+    // -t and t): magnitude range c holds the positive range 16 + c and the negative range 15 - c.
+    const long long rank = abs_mode ? n - 1 - 2 * n_tail : (q == 0 ? n_tail : n - 1 - n_tail);
+    const long long cc = !abs_mode ? (long long)__ldcg(&gcoarse[lane])
+                         : (lane < 16 ? (long long)__ldcg(&gcoarse[16 + lane]) + __ldcg(&gcoarse[15 - lane]) : 0ll);
     long long sc = cc;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -294,10 +297,15 @@ hist_select_kernel(const uint4* __restrict__ x, int rows, int vec_per_row, uint3
     const int region = holds ? __ffs(holds) - 1 : 0;
     long long run = __shfl_sync(0xFFFFFFFFu, sc - cc, region);                          // counts before the range
     // positions of the range in ascending order; in memory they ascend (region >= 16) or descend
-    const bool desc = region < 16;
-    const uint32_t* first = ghist + (desc ? (0xFFFF - 2048 * region - 2047) : 2048 * (region - 16));
+    const bool desc = !abs_mode && region < 16;
+    const uint32_t* first = abs_mode ? ghist + 2048 * region
+                                     : ghist + (desc ? (0xFFFF - 2048 * region - 2047) : 2048 * (region - 16));
     const int word = desc ? (2048 - 128 * st - 4 * lane - 4) : (128 * st + 4 * lane);
-    const uint4 c = __ldcg(reinterpret_cast<const uint4*>(first + word));
+    uint4 c = __ldcg(reinterpret_cast<const uint4*>(first + word));
+    if (abs_mode) {                                   // the same magnitudes with the sign bit set
+      const uint4 cn = __ldcg(reinterpret_cast<const uint4*>(first + 0x8000 + word));
+      c = make_uint4(c.x + cn.x, c.y + cn.y, c.z + cn.z, c.w + cn.w);
+    }
     // in ascending position order
     const long long v0 = desc ? c.w : c.x, v1 = desc ? c.z : c.y;
     const long long v2 = desc ? c.y : c.z, v3 = desc ? c.x : c.w;
@@ -315,8 +323,16 @@ hist_select_kernel(const uint4* __restrict__ x, int rows, int vec_per_row, uint3
     if (holds && rank >= before && rank < before + mine) {
       const int p0 = 2048 * region + 128 * st + 4 * lane;
       const int k = rank < before + v0 ? 0 : (rank < before + v0 + v1 ? 1 : (rank < before + v0 + v1 + v2 ? 2 : 3));
-      const uint32_t bits = pos_to_bits(p0 + k);
-      thresholds[q] = __uint_as_float((bits == 0x8000u ? 0u : bits) << 16);   // thresholds are real numbers: -0 is +0
+      if (abs_mode) {
+        const uint32_t m15 = uint32_t(p0 + k);          // p0 counts magnitudes here
+        if (q == 0) {
+          thresholds[1] = __uint_as_float(m15 << 16);
+          thresholds[0] = __uint_as_float(m15 ? (m15 | 0x8000u) << 16 : 0u);
+        }
+      } else {
+        const uint32_t bits = pos_to_bits(p0 + k);
+        thresholds[q] = __uint_as_float((bits == 0x8000u ? 0u : bits) << 16);   // thresholds are real numbers: -0 is +0
+      }
     }
   }
   __syncthreads();
@@ -1001,7 +1017,7 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
       unsigned* parity = reinterpret_cast<unsigned*>(ctx->occ_hist + 2 * HIST_SET_WORDS);
       hist_select_kernel<<<int(blocks), HIST_THREADS, HIST_SMEM_BYTES, stream>>>(
           x, rows, cols / 8, ctx->occ_hist, parity, sc.row_max, sc.row_min, sc.row_cnt, n, n_tail, out->thresholds,
-          parity + 1, status);
+          parity + 1, status, ctx->quantile_mode);
     }
     {
       KernelScope scope(ctx, stream, KC_ENCODE, 1);
@@ -1208,7 +1224,7 @@ extern "C" int fp4_quantile_thresholds_static(void* stream, const void* x_bf16, 
   if (blocks > sms_of_device[device]) blocks = sms_of_device[device];
   hist_select_kernel<<<int(blocks), HIST_THREADS, HIST_SMEM_BYTES, st>>>(
       static_cast<const uint4*>(x_bf16), int(rows), int(cols / 8), hist, nullptr, row_max, row_min, nullptr, n, n_tail,
-      thresholds, ticket, nullptr);
+      thresholds, ticket, nullptr, 0);
   FP4_CUDA_TRY(cudaGetLastError());
   return FP4_OK;
 }

@@ -257,3 +257,45 @@ def test_host_side_argument_errors(lib, ctx):
         lib.fp4_quantize(small, x, 0)
     assert e.value.code == -5                                   # workspace
     small.close()
+
+
+@pytest.mark.parametrize("shape,alpha,dist", [((128, 128), 0.99, "normal"), ((256, 384), 0.97, "student_t3"),
+                                              ((1024, 640), 0.999, "laplace")])
+def test_magnitude_quantile_variant_matches_oracle(lib, shape, alpha, dist):
+    """FP4_QUANTILE_ABS: one threshold on |x| (a variant outside the paper) -- thresholds, codes, amax
+    and the sparse residual bit for bit; the default mode of another context is untouched."""
+    cfg = WL.Config(52, "t", shape[0], (), dist, 3, 40.0, "channels_count", (alpha,))
+    bits = WL.activations(cfg, shape[1], seed=3, layer=shape[0])
+    c = lib.Context(0, 256 << 20)
+    c.set_quantile_mode(lib.FP4_QUANTILE_ABS)
+    q = lib.fp4_quantize(c, _dev(bits), 0, alpha=alpha)
+    torch.cuda.synchronize()
+    assert c.read_status() == 0
+    ref = O.occ_quantize(O.bf16_bits_to_f64(bits), alpha, quantile="abs")
+    assert ref.lo == -ref.hi
+    _check_sparse(q, ref)
+    _check_dense(q, ref)
+    c.set_quantile_mode(lib.FP4_QUANTILE_SIGNED)
+    q = lib.fp4_quantize(c, _dev(bits), 0, alpha=alpha)
+    torch.cuda.synchronize()
+    _check_sparse(q, O.occ_quantize(O.bf16_bits_to_f64(bits), alpha))
+    with pytest.raises(lib.Fp4Error):
+        c.set_quantile_mode(7)
+    c.close()
+
+
+def test_magnitude_quantile_with_ties_and_a_zero_threshold(lib):
+    rng = np.random.default_rng(21)
+    vals = np.array([0.0, -0.0, 0.5, -0.5, 1.0, -3.0, 64.0], dtype=np.float32)
+    for prob, alpha in (([0.5, 0.3, 0.05, 0.05, 0.05, 0.03, 0.02], 0.9),        # t = 0.5 sits on a big tie
+                        ([0.6, 0.37, 0.01, 0.01, 0.005, 0.003, 0.002], 0.99)):   # t = 0: lo must be +0
+        a = rng.choice(vals, size=(256, 512), p=prob)
+        bits = WL.to_bf16_bits(a)
+        c = lib.Context(0, 256 << 20)
+        c.set_quantile_mode(lib.FP4_QUANTILE_ABS)
+        q = lib.fp4_quantize(c, _dev(bits), 0, alpha=alpha)
+        torch.cuda.synchronize()
+        ref = O.occ_quantize(O.bf16_bits_to_f64(bits), alpha, quantile="abs")
+        _check_sparse(q, ref)
+        _check_dense(q, ref)
+        c.close()

@@ -131,11 +131,16 @@ def test_random_clamping_quantizer_is_bit_exact(lib, ctx, i, rows, cols, alpha, 
         mask = rng.random(a.shape) < zeros
         a[mask] = np.where(rng.random(int(mask.sum())) < 0.5, 0.0, -0.0).astype(np.float32)
     bits = WL.to_bf16_bits(a)
+    quantile = "abs" if i % 4 == 1 else "signed"           # every fourth draw: the one-threshold variant
     ctx.status.zero_()
-    q = lib.fp4_quantize(ctx, _dev(bits), 0, alpha=alpha)
-    torch.cuda.synchronize()
+    ctx.set_quantile_mode(lib.FP4_QUANTILE_ABS if quantile == "abs" else lib.FP4_QUANTILE_SIGNED)
+    try:
+        q = lib.fp4_quantize(ctx, _dev(bits), 0, alpha=alpha)
+        torch.cuda.synchronize()
+    finally:
+        ctx.set_quantile_mode(lib.FP4_QUANTILE_SIGNED)
     assert ctx.read_status() == 0
-    ref = O.occ_quantize(O.bf16_bits_to_f64(bits), alpha)
+    ref = O.occ_quantize(O.bf16_bits_to_f64(bits), alpha, quantile=quantile)
     _check_sparse(q, ref)
     _check_dense(q, ref)
 
