@@ -182,6 +182,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-share-activations", action="store_true",
                     help="quantise the activation of every linear, also where q/k/v or gate/up read the same tensor")
+    ap.add_argument("--cache-weights", action="store_true",
+                    help="micro-batch steps of gradient accumulation: the weights' codes are those of the step's "
+                         "first micro-batch (quantised before the timed region), re-used by every timed step")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -242,9 +245,11 @@ def main():
     def step():
         for L in layers:
             fp4.fp4_linear_fwd(ctx, L["A"], L["W"], alpha, L["sa"], L["sw"], gemm_kind=kind, out=L["Y"],
-                               reuse_a=L["reuse_a"])
+                               reuse_a=L["reuse_a"], reuse_w=cached_w[0])
             fp4.fp4_linear_bwd(ctx, L["G"], L["W"], L["sa"], L["sw"], gemm_kind=kind, dA=L["dA"], dW=L["dW"],
                                dy_fmt=dy8)
+
+    cached_w = [False]                           # --cache-weights: set after the first (untimed) step
 
     def step_host():
         for L in layers:
@@ -256,6 +261,7 @@ def main():
     # rejoin the capturing stream) and replayed: the timed region is K replays back to back.
     for _ in range(args.warmup):
         step()
+        cached_w[0] = args.cache_weights
     torch.cuda.synchronize()
     assert ctx.read_status() == 0, "device status word is set"
     ctx.profile_reset()
@@ -388,6 +394,8 @@ def main():
                        "launch": "one CUDA graph per step, replayed",
                        "shared_activations": ("q/k/v and gate/up read one activation tensor: quantised once, re-used"
                                               if share else "every linear quantises its activation"),
+                       "weights": ("codes of the weights cached across the timed steps (micro-batches of one "
+                                   "optimizer step)" if args.cache_weights else "quantised in every step"),
                        "kernel_timing": f"CUDA events per kernel class over {args.steps} plainly launched steps, side "
                                         f"streams off ({ms_profiled / args.steps:.3f} ms/step that way)",
                        "replicas": world},
