@@ -4,7 +4,8 @@ Seeded draws over shapes (multiples of 128, ragged against every tile size), cla
 activation distributions, number of outlier channels, GEMM kind and DGE setting.  Every draw checks
 what the fixed cases check: saved operands bit for bit, the three outputs within the bar stated in
 test_gpu_linear.py.  The draws are fixed by the seed, so a failure reproduces; FP4_RANDOM_DRAWS in
-the environment sets how many are made (default 16).
+the environment sets how many are made (default 16); FP4_TEST_NO_OVERLAP=1 runs them with the
+library's side streams switched off.
 """
 import os
 
@@ -22,6 +23,8 @@ pytestmark = pytest.mark.gpu
 @pytest.fixture(scope="module")
 def ctx(lib):
     c = lib.Context(0, 1 << 30)
+    if os.environ.get("FP4_TEST_NO_OVERLAP"):          # the same draws with every kernel on one stream
+        c.set_overlap(False)
     yield c
     c.close()
 
