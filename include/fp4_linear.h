@@ -177,6 +177,11 @@ int fp4_gemm(fp4_ctx* ctx, void* stream, const uint8_t* a_codes, const uint8_t* 
  *   change once per optimizer step) and is not recomputed; FP4_REUSE_A -- savedA already holds
  *   this activation quantised with the same alpha (the q/k/v projections of a layer, or its
  *   gate/up projections, read the same activation) and is not recomputed.
+ *   With a heavy residual (savedA->sparse_cap at least 1 % of M * K, i.e. alpha <= 0.995) the
+ *   residual's columns that at least max(M / 4, 512) tokens hit -- the outlier channels of
+ *   Appendix D, up to 128 of them -- are multiplied on the tensor cores inside the GEMM (two-term
+ *   FP16 splits of residual and weight); the other entries are added per entry in fp32.  The
+ *   result differs from the per-entry sum by at most 4e-6 * sum_k |A - A_c|[m,k] |W|[k,n].
  */
 #define FP4_REUSE_W 1
 #define FP4_REUSE_A 2
