@@ -254,15 +254,21 @@ hist_select_kernel(const uint4* __restrict__ x, int rows, int vec_per_row, uint3
     if (zeros_pos) { atomicAdd(&ghist[0x0000], zeros_pos); atomicAdd(&s_coarse[bits_to_pos(0x0000u) >> 11], zeros_pos); }
     if (zeros_neg) { atomicAdd(&ghist[0x8000], zeros_neg); atomicAdd(&s_coarse[bits_to_pos(0x8000u) >> 11], zeros_neg); }
   }
-  for (int idx = tid; idx < 2 * HIST_WINDOW; idx += HIST_THREADS) {
-    const int neg = idx >= HIST_WINDOW, off = idx - neg * HIST_WINDOW;
-    uint32_t c = 0;
+  // Two neighbouring counters (an even pattern and the next one: same sign, same coarse range) leave
+  // with one 64-bit add; no 32-bit half can overflow into the other (n < 2^31).
+  for (int idx = tid; idx < HIST_WINDOW; idx += HIST_THREADS) {
+    const int neg = idx >= HIST_WINDOW / 2, off = 2 * (idx - neg * (HIST_WINDOW / 2));
+    uint32_t c0 = 0, c1 = 0;
 #pragma unroll
-    for (int r = 0; r < HIST_COPIES; ++r) c += h[neg * HIST_NEG_WORD + r * HIST_WINDOW + off];
-    if (c) {
+    for (int r = 0; r < HIST_COPIES; ++r) {
+      const uint2 c = *reinterpret_cast<const uint2*>(&h[neg * HIST_NEG_WORD + r * HIST_WINDOW + off]);
+      c0 += c.x;
+      c1 += c.y;
+    }
+    if (c0 | c1) {
       const uint32_t bits = (uint32_t(neg) << 15) | (base + uint32_t(off));
-      atomicAdd(&ghist[bits], c);
-      atomicAdd(&s_coarse[bits_to_pos(bits) >> 11], c);
+      atomicAdd(reinterpret_cast<unsigned long long*>(&ghist[bits]), (unsigned long long)c0 | ((unsigned long long)c1 << 32));
+      atomicAdd(&s_coarse[bits_to_pos(bits) >> 11], c0 + c1);
     }
   }
   __syncthreads();
