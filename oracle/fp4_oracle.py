@@ -241,6 +241,8 @@ class Quantized:
     csc: tuple = field(default=None)   # (colptr int32[cols+1], row int32[nnz], val float32[nnz])
     residual: np.ndarray = None  # dense float64 [rows, cols] (zeros outside the tails)
     fmt: str = "e2m1"            # "e2m1": one nibble code per element; "e4m3" / "e5m2": one byte per element
+    lo_rows: np.ndarray = None   # per-token variant of the clamp: thresholds of every row
+    hi_rows: np.ndarray = None
 
     @property
     def fmax(self):
@@ -348,13 +350,39 @@ def sparse_from_dense(r):
     return csr, csc
 
 
+def token_thresholds(a, alpha: float):
+    """(lo[rows], hi[rows], n_tail): the signed order statistics of every token (row) on its own.
+
+    A variant outside the paper (which takes the quantiles of the whole tensor): n_tail =
+    round((1 - alpha) * cols) entries of every row may leave the clamp on either side.
+    """
+    a = np.asarray(a, dtype=np.float64)
+    cols = a.shape[1]
+    n_tail = tail_count(cols, alpha)
+    if not (2 * n_tail < cols):
+        raise ValueError("alpha leaves nothing between the two tails of a row")
+    s = np.sort(a, axis=1)
+    return s[:, n_tail] + 0.0, s[:, cols - 1 - n_tail] + 0.0, n_tail      # "+ 0.0" turns -0.0 into +0.0
+
+
 def occ_quantize(a, alpha: float, quantile: str = "signed") -> Quantized:
     """Clamp at the quantiles, keep the sparse residual, then token-wise absmax + Q.
 
     The clamp comes first: its purpose is to shrink the range the absmax scale
-    has to cover (Section 3.2, first paragraph).
+    has to cover (Section 3.2, first paragraph).  ``quantile`` = "token" takes the thresholds of
+    every row from that row alone (``lo_rows`` / ``hi_rows`` of the result; ``lo`` / ``hi`` are NaN).
     """
     a = np.asarray(a, dtype=np.float64)
+    if alpha < 1.0 and quantile == "token":
+        lo_r, hi_r, n_tail = token_thresholds(a, alpha)
+        a_c = np.minimum(np.maximum(a, lo_r[:, None]), hi_r[:, None])
+        r = a - a_c
+        q = absmax_quantize(a_c, 0)
+        q.lo, q.hi, q.n_tail = float("nan"), float("nan"), n_tail
+        q.lo_rows, q.hi_rows = lo_r, hi_r
+        q.residual = r
+        q.csr, q.csc = sparse_from_dense(r)
+        return q
     if alpha >= 1.0:
         q = absmax_quantize(a, 0)
         q.residual = np.zeros_like(a)

@@ -195,3 +195,39 @@ def test_abs_and_signed_forms_agree_on_mirrored_data():
     s = O.quantile_thresholds(a, 0.99)
     b = O.quantile_thresholds(a, 0.99, quantile="abs")
     assert s[1] == b[1] and s[0] == b[0] == -s[1]
+
+
+# ---------------------------------------------------------------------------------------------
+# The variant outside the paper: thresholds per token
+# ---------------------------------------------------------------------------------------------
+def test_token_thresholds_are_the_rows_own_order_statistics():
+    rng = np.random.default_rng(9)
+    a = _bf16_normal(rng, (6, 200)) * np.array([[1], [10], [0.1], [1], [100], [1]])
+    a[3, :50] = a[3, 50:100]                               # ties
+    lo, hi, n_tail = O.token_thresholds(a, 0.97)
+    assert n_tail == 6
+    for m in range(6):
+        row = a[m]
+        assert (row < lo[m]).sum() <= n_tail < (row <= lo[m]).sum()     # by counting, not by sorting
+        assert (row > hi[m]).sum() <= n_tail < (row >= hi[m]).sum()
+        assert lo[m] in row and hi[m] in row
+        # a row on its own is what the tensor-wide form makes of a one-row tensor
+        assert (lo[m], hi[m]) == O.quantile_thresholds(row[None, :], 0.97)[:2]
+
+
+def test_token_variant_identity_bounds_and_counts():
+    rng = np.random.default_rng(10)
+    a = _bf16_normal(rng, (16, 256))
+    a[:, 7] *= 30.0
+    q = O.occ_quantize(a, 0.99, quantile="token")
+    assert q.n_tail == 3 and q.lo_rows.shape == (16,)
+    a_c = np.minimum(np.maximum(a, q.lo_rows[:, None]), q.hi_rows[:, None])
+    np.testing.assert_array_equal(a_c + q.residual, a)      # clamped + residual == original, exactly
+    per_row = (q.residual != 0).sum(axis=1)
+    assert (per_row <= 2 * q.n_tail).all() and per_row.max() > 0
+    np.testing.assert_array_equal(q.amax, np.abs(a_c).max(axis=1).astype(np.float32))
+    rowptr, col, val = q.csr
+    np.testing.assert_array_equal(np.diff(rowptr), per_row)
+    whole = O.occ_quantize(a, 0.99)                          # the paper's form clamps the outlier column only
+    assert (whole.residual != 0).sum() <= 2 * whole.n_tail
+    assert not np.array_equal(whole.codes, q.codes)
