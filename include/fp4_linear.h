@@ -264,9 +264,14 @@ int fp4_set_gemm_pairs(fp4_ctx* ctx, int on);
  * calls built on it; not fp4_quantile_thresholds_static).  FP4_QUANTILE_SIGNED (default): the
  * paper's form (Section 3.2), lo and hi the (1-alpha)- and alpha-quantiles of the values.
  * FP4_QUANTILE_ABS, a variant outside the paper: one threshold t on the magnitudes, the order
- * statistic of |x| that at most 2 n_tail entries exceed; lo = -t, hi = t.                     */
+ * statistic of |x| that at most 2 n_tail entries exceed; lo = -t, hi = t.
+ * FP4_QUANTILE_TOKEN, another variant outside the paper: the signed form per token -- row m is
+ * clamped between its own order statistics, round((1 - alpha) * cols) entries on either side; the
+ * operand's `thresholds` then holds 2 * rows floats (lo, hi of every row) and its `sparse_cap`
+ * must be at least 2 * rows * round((1 - alpha) * cols).                                       */
 #define FP4_QUANTILE_SIGNED 0
 #define FP4_QUANTILE_ABS    1
+#define FP4_QUANTILE_TOKEN  2
 int fp4_set_quantile_mode(fp4_ctx* ctx, int mode);
 int fp4_profile_reset(fp4_ctx* ctx);
 int fp4_profile_read(fp4_ctx* ctx, int kernel_class, double* total_ms, int64_t* launches);

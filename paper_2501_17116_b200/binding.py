@@ -37,6 +37,7 @@ EXPORTS = ("fp4_create", "fp4_destroy", "fp4_workspace_bytes", "fp4_status_strin
 FP4_STATIC_MAX_ROWS = 65536
 FP4_QUANTILE_SIGNED = 0
 FP4_QUANTILE_ABS = 1
+FP4_QUANTILE_TOKEN = 2
 KERNEL_CLASSES = ("gemm", "select", "encode", "absmax", "sparse", "comp_fwd", "comp_wgrad_dge")
 
 
@@ -182,7 +183,8 @@ class Context:
         _check(self.lib.fp4_set_gemm_pairs(self.handle, int(on)))
 
     def set_quantile_mode(self, mode: int):
-        """FP4_QUANTILE_SIGNED (the paper's clamp, default) or FP4_QUANTILE_ABS (one threshold on |x|)."""
+        """FP4_QUANTILE_SIGNED (the paper's clamp, default), FP4_QUANTILE_ABS (one threshold on |x|) or
+        FP4_QUANTILE_TOKEN (signed thresholds per token)."""
         _check(self.lib.fp4_set_quantile_mode(self.handle, int(mode)))
 
     def launch_count(self) -> int:
@@ -203,7 +205,9 @@ class QTensor:
         self.sparse_cap = int(sparse_cap)
         if sparse_cap > 0:
             cap = max(int(sparse_cap), 1)
-            self.thresholds = torch.zeros(2, dtype=torch.float32, device=dev)
+            # lo, hi of the tensor; with thresholds per token the library fills all 2 * rows (lo, hi of every row)
+            self.thresholds_rows = torch.zeros(2 * rows, dtype=torch.float32, device=dev)
+            self.thresholds = self.thresholds_rows[:2]
             self.csr_rowptr = torch.zeros(rows + 1, dtype=torch.int32, device=dev)
             self.csr_col = torch.zeros(cap, dtype=torch.int32, device=dev)
             self.csr_val = torch.zeros(cap, dtype=torch.float32, device=dev)
@@ -212,7 +216,7 @@ class QTensor:
             self.csc_val = torch.zeros(cap, dtype=torch.float32, device=dev)
             self.nnz = torch.zeros(1, dtype=torch.int32, device=dev)
         else:
-            self.thresholds = self.csr_rowptr = self.csr_col = self.csr_val = None
+            self.thresholds = self.thresholds_rows = self.csr_rowptr = self.csr_col = self.csr_val = None
             self.csc_colptr = self.csc_row = self.csc_val = self.nnz = None
         self.struct = fp4_qtensor(
             rows, cols, _ptr(self.codes), _ptr(self.codes_t), _ptr(self.amax), _ptr(self.thresholds),
@@ -221,11 +225,13 @@ class QTensor:
 
 
 def tail_capacity(rows: int, cols: int, alpha: float) -> int:
-    """2 * n_tail: the guaranteed bound on the number of residual entries."""
+    """The guaranteed bound on the number of residual entries, whichever form of the clamp is set:
+    2 * n_tail of the tensor, or rows * 2 * n_tail of a row for thresholds per token."""
     if alpha >= 1.0:
         return 0
     import math
-    return 2 * int(math.floor((1.0 - alpha) * rows * cols + 0.5))
+    return max(2 * int(math.floor((1.0 - alpha) * rows * cols + 0.5)),
+               2 * rows * int(math.floor((1.0 - alpha) * cols + 0.5)))
 
 
 def fp4_quantize(ctx: Context, x: torch.Tensor, scale_axis: int, alpha: float = 1.0, prescale=None,

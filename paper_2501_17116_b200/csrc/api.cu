@@ -189,8 +189,13 @@ int fp4_quantize(fp4_ctx* ctx, void* stream, const void* x_bf16, int64_t rows, i
   if (alpha < 1.0) {
     if (scale_axis != 0 || prescale || out->format != FP4_FORMAT_E2M1) return FP4_ERR_ARG;
     const int64_t n = rows * cols;
-    const int64_t n_tail = llround((1.0 - alpha) * double(n));
+    int64_t n_tail = llround((1.0 - alpha) * double(n));
     if (2 * n_tail >= n) return FP4_ERR_ALPHA;
+    if (ctx->quantile_mode == FP4_QUANTILE_TOKEN) {       // per token: every row has its own two tails
+      const int64_t per_row = llround((1.0 - alpha) * double(cols));
+      if (2 * per_row >= cols) return FP4_ERR_ALPHA;
+      n_tail = rows * per_row;
+    }
     rc = check_qtensor_sparse(out, n_tail);
     if (rc != FP4_OK) return rc;
   }
@@ -241,8 +246,13 @@ int fp4_linear_fwd(fp4_ctx* ctx, void* stream, const void* A_bf16, const void* W
     if (a8 && occ) return FP4_ERR_ARG;                                    // clamping belongs to 4-bit activations
   }
   if (occ) {
-    const int64_t n_tail = llround((1.0 - alpha) * double(M * K));
+    int64_t n_tail = llround((1.0 - alpha) * double(M * K));
     if (2 * n_tail >= M * K) return FP4_ERR_ALPHA;
+    if (ctx->quantile_mode == FP4_QUANTILE_TOKEN) {       // per token: every row has its own two tails
+      const int64_t per_row = llround((1.0 - alpha) * double(K));
+      if (2 * per_row >= K) return FP4_ERR_ALPHA;
+      n_tail = M * per_row;
+    }
     int rc = check_qtensor_sparse(savedA, n_tail);
     if (rc != FP4_OK) return rc;
   }
@@ -481,7 +491,7 @@ void carve_qtensor(Arena& a, fp4_qtensor* q, int64_t rows, int64_t cols, int sca
   q->amax = a.take<float>(size_t(scale_axis == 0 ? rows : cols));
   q->sparse_cap = cap;
   if (cap > 0) {
-    q->thresholds = a.take<float>(2);
+    q->thresholds = a.take<float>(2 * size_t(rows));      // room for thresholds per token (fp4_set_quantile_mode)
     q->nnz = a.take<int32_t>(1);
     q->csr_rowptr = a.take<int32_t>(size_t(rows) + 1);
     q->csr_col = a.take<int32_t>(size_t(cap));
@@ -492,8 +502,13 @@ void carve_qtensor(Arena& a, fp4_qtensor* q, int64_t rows, int64_t cols, int sca
   }
 }
 
+// Residual entries a step may produce under either form of the clamp: 2 n_tail of the tensor, or
+// two tails of round((1 - alpha) K) entries in every row (thresholds per token).
 int64_t step_capacity(int64_t M, int64_t K, double alpha) {
-  return alpha < 1.0 ? 2 * llround((1.0 - alpha) * double(M * K)) : 0;
+  if (!(alpha < 1.0)) return 0;
+  const int64_t whole = 2 * llround((1.0 - alpha) * double(M * K));
+  const int64_t per_token = 2 * M * llround((1.0 - alpha) * double(K));
+  return whole > per_token ? whole : per_token;
 }
 
 // fp4_linear_step_host: bytes of one set of device inputs (the outputs have the same three sizes),
@@ -506,6 +521,7 @@ size_t step_host_shared_bytes(int64_t M, int64_t K, int64_t N, double alpha) {
   size_t b = 2 * round256(size_t(M) * K / 2) + 2 * round256(size_t(K) * N / 2);                          // codes
   b += round256(size_t(M) * 4) + round256(size_t(N) * 4);                                                // amax
   b += 4 * round256(cap * 4) + round256((size_t(M) + 1) * 4) + round256((size_t(K) + 1) * 4) + 3 * 256;   // sparse
+  b += round256(2 * size_t(M) * 4);                                                                      // thresholds
   b += 256;                                                                                              // status
   return b + fp4_workspace_bytes(M, K, N);
 }
@@ -627,7 +643,7 @@ int fp4_set_overlap(fp4_ctx* ctx, int on) {
 
 int fp4_set_quantile_mode(fp4_ctx* ctx, int mode) {
   if (!ctx) return FP4_ERR_NULL;
-  if (mode != FP4_QUANTILE_SIGNED && mode != FP4_QUANTILE_ABS) return FP4_ERR_ARG;
+  if (mode != FP4_QUANTILE_SIGNED && mode != FP4_QUANTILE_ABS && mode != FP4_QUANTILE_TOKEN) return FP4_ERR_ARG;
   ctx->quantile_mode = mode;
   return FP4_OK;
 }

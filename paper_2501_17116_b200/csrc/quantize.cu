@@ -349,6 +349,113 @@ hist_select_kernel(const uint4* __restrict__ x, int rows, int vec_per_row, uint3
 }
 
 // ------------------------------------------------------------------------------------------
+// 1c. thresholds per token (a variant outside the paper, which clamps at tensor-wide quantiles)
+// ------------------------------------------------------------------------------------------
+// One block per row: exact order statistics of the row's 16-bit patterns by a two-pass radix
+// select in shared memory (high byte of the position in ascending real order, then the low byte
+// inside the bin that holds the rank), both ranks at once; also the row's extremes, the zero that
+// starts its count of clamped entries, and the non-finite flag, like the tensor-wide kernel.
+// thresholds[2 m] = lo of row m, thresholds[2 m + 1] = hi (a -0 threshold is written as +0).
+__global__ void __launch_bounds__(256)
+row_select_kernel(const uint4* __restrict__ x, int vec_per_row, int n_tail, int* __restrict__ row_max,
+                  int* __restrict__ row_min, int* __restrict__ row_cnt, float* __restrict__ thresholds,
+                  int32_t* status) {
+  __shared__ uint32_t hist[3][256];          // pass 1; pass 2 for the lower rank; pass 2 for the upper rank
+  __shared__ int s_bin[2], s_rank[2], s_max[8], s_min[8];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int m = blockIdx.x;
+  const uint4* row = x + (long long)m * vec_per_row;
+  const int cols = 8 * vec_per_row;
+  for (int i = tid; i < 3 * 256; i += 256) (&hist[0][0])[i] = 0;
+  __syncthreads();
+  int kmax = INT_MIN, kmin = INT_MAX;
+  bool nonfinite = false;
+  for (int v = tid; v < vec_per_row; v += 256) {
+    const uint4 q = __ldg(&row[v]);
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const uint32_t bits = (e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xFFFFu);
+      atomicAdd(&hist[0][bits_to_pos(bits) >> 8], 1u);
+      if ((bits & 0x7FFFu) >= 0x7F80u) nonfinite = true;
+      const int key = float_to_ordered(__uint_as_float(bits << 16));
+      kmax = max(kmax, key);
+      kmin = min(kmin, key);
+    }
+  }
+  kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+  kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+  if (lane == 0) { s_max[warp] = kmax; s_min[warp] = kmin; }
+  if (__any_sync(0xFFFFFFFFu, nonfinite) && lane == 0 && status) atomicOr(status, FP4_DEV_NONFINITE);
+  __syncthreads();
+  if (tid == 0) {
+    int a = s_max[0], b = s_min[0];
+    for (int i = 1; i < 8; ++i) { a = max(a, s_max[i]); b = min(b, s_min[i]); }
+    row_max[m] = a;
+    row_min[m] = b;
+    if (row_cnt) row_cnt[m] = 0;
+  }
+  // the bin of each rank: warp q scans the 256 counts for rank q (8 per lane)
+  if (warp < 2) {
+    const int rank = warp == 0 ? n_tail : cols - 1 - n_tail;
+    int c[8], mine = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { c[i] = int(hist[0][8 * lane + i]); mine += c[i]; }
+    int incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+      if (lane >= off) incl += up;
+    }
+    int before = incl - mine;
+    if (rank >= before && rank < incl) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        if (rank >= before && rank < before + c[i]) { s_bin[warp] = 8 * lane + i; s_rank[warp] = rank - before; }
+        before += c[i];
+      }
+    }
+  }
+  __syncthreads();
+  const int bin_lo = s_bin[0], bin_hi = s_bin[1];
+  for (int v = tid; v < vec_per_row; v += 256) {      // second pass: the row is in L1 / L2 now
+    const uint4 q = __ldg(&row[v]);
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const uint32_t bits = (e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xFFFFu);
+      const int pos = bits_to_pos(bits);
+      if ((pos >> 8) == bin_lo) atomicAdd(&hist[1][pos & 255], 1u);
+      if ((pos >> 8) == bin_hi) atomicAdd(&hist[2][pos & 255], 1u);
+    }
+  }
+  __syncthreads();
+  if (warp < 2) {
+    const int rank = s_rank[warp];
+    int c[8], mine = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { c[i] = int(hist[1 + warp][8 * lane + i]); mine += c[i]; }
+    int incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+      if (lane >= off) incl += up;
+    }
+    int before = incl - mine;
+    if (rank >= before && rank < incl) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        if (rank >= before && rank < before + c[i]) {
+          const uint32_t bits = pos_to_bits(256 * s_bin[warp] + 8 * lane + i);
+          thresholds[2 * m + warp] = __uint_as_float((bits == 0x8000u ? 0u : bits) << 16);
+        }
+        before += c[i];
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // absmax without clamping
 // ------------------------------------------------------------------------------------------
 // d[i] = amax[i] / MAX rounded once (MAX = 6 for E2M1, 448 for E4M3): the de-scale vector of a
@@ -520,7 +627,7 @@ struct EncodeArgs {
 // MODE_ROWS: one scale per row -> codes and / or codes_t.  MODE_COLS: one scale per column.
 // MODE_DUAL: codes hold the row-scaled tensor x (.) pre_col, codes_t the column-scaled tensor
 // x (.) pre_row.  OCC (clamping) implies MODE_ROWS without prescale.
-template <int MODE, bool OCC, bool PRESCALE>
+template <int MODE, bool OCC, bool PRESCALE, bool PER_TOKEN = false>
 __global__ void __launch_bounds__(ENC_THREADS)
 encode_kernel(const EncodeArgs a) {
   __shared__ float s_gcol[ENC_TK];
@@ -528,6 +635,7 @@ encode_kernel(const EncodeArgs a) {
   __shared__ float s_prow[ENC_TM];
   __shared__ uint32_t tile_t[8 * 8 * 32];
   __shared__ int s_colcnt[OCC ? ENC_TK : 1];
+  __shared__ float s_thr[PER_TOKEN ? 2 * ENC_TM : 1];      // per-token clamp: lo, hi of the tile's rows
   const int tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31;
   const int row0 = blockIdx.y * ENC_TM;
@@ -537,8 +645,10 @@ encode_kernel(const EncodeArgs a) {
   constexpr bool COL_SCALED = MODE != MODE_ROWS;
   float lo = 0.f, hi = 0.f;
   if (OCC) {
-    lo = a.thresholds[0];
-    hi = a.thresholds[1];
+    if constexpr (!PER_TOKEN) {
+      lo = a.thresholds[0];
+      hi = a.thresholds[1];
+    }
     s_colcnt[tid] = 0;
   }
 
@@ -546,6 +656,10 @@ encode_kernel(const EncodeArgs a) {
     const int r = row0 + tid;
     float amax;
     if (OCC) {
+      if constexpr (PER_TOKEN) {
+        lo = s_thr[2 * tid] = a.thresholds[2 * r];
+        hi = s_thr[2 * tid + 1] = a.thresholds[2 * r + 1];
+      }
       const float mx = fminf(fmaxf(ordered_to_float(a.row_max[r]), lo), hi);
       const float mn = fminf(fmaxf(ordered_to_float(a.row_min[r]), lo), hi);
       amax = fmaxf(fabsf(mx), fabsf(mn));
@@ -594,6 +708,10 @@ encode_kernel(const EncodeArgs a) {
     uint32_t obits = 0;
     const float grow = ROW_SCALED ? s_grow[8 * warp + r] : 0.0f;
     const float prow = (COL_SCALED && PRESCALE) ? s_prow[8 * warp + r] : 1.0f;
+    if constexpr (PER_TOKEN) {
+      lo = s_thr[2 * (8 * warp + r)];
+      hi = s_thr[2 * (8 * warp + r) + 1];
+    }
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
       float xv = (c & 1) ? bf16_hi(w[c >> 1]) : bf16_lo(w[c >> 1]);
@@ -830,7 +948,7 @@ __device__ __forceinline__ float residual_of(const __nv_bfloat16* x, long long i
 
 __global__ void __launch_bounds__(256)
 csr_fill_kernel(const uint32_t* __restrict__ mask, const __nv_bfloat16* __restrict__ x, int rows, int cols,
-                const float* __restrict__ thresholds, const int* __restrict__ rowptr, long long cap,
+                const float* __restrict__ thresholds, int thr_per_row, const int* __restrict__ rowptr, long long cap,
                 int* __restrict__ csr_col, float* __restrict__ csr_val) {
   const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
@@ -838,7 +956,7 @@ csr_fill_kernel(const uint32_t* __restrict__ mask, const __nv_bfloat16* __restri
   int base = rowptr[row];
   if (rowptr[row + 1] == base) return;                // nothing clamped in this row
   const int words_per_row = cols >> 5;
-  const float lo = thresholds[0], hi = thresholds[1];
+  const float lo = thresholds[thr_per_row ? 2 * row : 0], hi = thresholds[thr_per_row ? 2 * row + 1 : 1];
   for (int w0 = 0; w0 < words_per_row; w0 += 32) {
     const int w = w0 + lane;
     uint32_t m = w < words_per_row ? mask[(long long)row * words_per_row + w] : 0u;
@@ -886,7 +1004,7 @@ csc_strip_prefix_kernel(const uint8_t* __restrict__ strip_cnt, int cols, int str
 // column, so all gathers of a column are issued at once and the order is by row by construction.
 __global__ void __launch_bounds__(256)
 csc_fill_kernel(const uint32_t* __restrict__ mask, const __nv_bfloat16* __restrict__ x, int rows, int cols,
-                const float* __restrict__ thresholds, const int* __restrict__ colptr,
+                const float* __restrict__ thresholds, int thr_per_row, const int* __restrict__ colptr,
                 const int* __restrict__ strip_off, long long cap, int* __restrict__ csc_row,
                 float* __restrict__ csc_val) {
   const int q = blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -899,7 +1017,6 @@ csc_fill_kernel(const uint32_t* __restrict__ mask, const __nv_bfloat16* __restri
   const uint32_t any0 = __reduce_or_sync(0xFFFFFFFFu, w0);
   const uint32_t any1 = __reduce_or_sync(0xFFFFFFFFu, w1);
   if (!(any0 | any1)) return;
-  const float lo = thresholds[0], hi = thresholds[1];
   // lane c holds the next free position of column 32 q + c
   int next = colptr[32 * q + lane] + strip_off[(long long)blockIdx.y * cols + 32 * q + lane];
   const uint32_t lt_mask = (1u << lane) - 1u;
@@ -908,6 +1025,7 @@ csc_fill_kernel(const uint32_t* __restrict__ mask, const __nv_bfloat16* __restri
     const uint32_t w = half ? w1 : w0;
     uint32_t any = half ? any1 : any0;
     const int r = r0 + 32 * half + lane;
+    const float lo = thresholds[thr_per_row ? 2 * r : 0], hi = thresholds[thr_per_row ? 2 * r + 1 : 1];
     while (any) {
       const int c = __ffs(any) - 1;
       any &= any - 1;
@@ -1009,10 +1127,16 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
   ea.fmax = fp8_max(out->format);
   const dim3 tile_grid((cols + ENC_TK - 1) / ENC_TK, rows / ENC_TM);
 
+  const int per_token = occ && ctx->quantile_mode == FP4_QUANTILE_TOKEN;
   if (occ) {
     const long long n_tail = llround((1.0 - alpha) * double(n));
     const long long n_vec = n / 8;
-    {
+    if (per_token) {
+      KernelScope scope(ctx, stream, KC_SELECT, 1);
+      const int n_tail_row = int(llround((1.0 - alpha) * double(cols)));
+      row_select_kernel<<<rows, 256, 0, stream>>>(x, cols / 8, n_tail_row, sc.row_max, sc.row_min, sc.row_cnt,
+                                                  out->thresholds, status);
+    } else {
       // The two sets of global counters, their parity and the ticket belong to the context: the
       // kernel keeps the set it is about to use zero (see there), so nothing is cleared here.
       KernelScope scope(ctx, stream, KC_SELECT, 1);
@@ -1023,11 +1147,14 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
       unsigned* parity = reinterpret_cast<unsigned*>(ctx->occ_hist + 2 * HIST_SET_WORDS);
       hist_select_kernel<<<int(blocks), HIST_THREADS, HIST_SMEM_BYTES, stream>>>(
           x, rows, cols / 8, ctx->occ_hist, parity, sc.row_max, sc.row_min, sc.row_cnt, n, n_tail, out->thresholds,
-          parity + 1, status, ctx->quantile_mode);
+          parity + 1, status, ctx->quantile_mode == FP4_QUANTILE_ABS);
     }
     {
       KernelScope scope(ctx, stream, KC_ENCODE, 1);
-      encode_kernel<MODE_ROWS, true, false><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
+      if (per_token)
+        encode_kernel<MODE_ROWS, true, false, true><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
+      else
+        encode_kernel<MODE_ROWS, true, false><<<tile_grid, ENC_THREADS, 0, stream>>>(ea);
     }
     cudaStream_t sp = stream;
     if (overlap && overlap->stream) {
@@ -1048,7 +1175,7 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
     {
       KernelScope scope(ctx, sp, KC_SPARSE, 2);
       scan_counts_kernel<<<1, 1024, 0, sp>>>(sc.row_cnt, rows, out->csr_rowptr, out->nnz, out->sparse_cap, status);
-      csr_fill_kernel<<<(rows + 7) / 8, 256, 0, sp>>>(mask32, xb, rows, cols, out->thresholds, out->csr_rowptr,
+      csr_fill_kernel<<<(rows + 7) / 8, 256, 0, sp>>>(mask32, xb, rows, cols, out->thresholds, per_token, out->csr_rowptr,
                                                       out->sparse_cap, out->csr_col, out->csr_val);
     }
     if (sp != stream) FP4_CUDA_TRY(cudaEventRecord(overlap->csr_done, sp));
@@ -1057,7 +1184,7 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
       csc_strip_prefix_kernel<<<(cols + 255) / 256, 256, 0, sc2>>>(sc.strip_cnt, cols, strips, sc.strip_off, sc.col_cnt);
       scan_counts_kernel<<<1, 1024, 0, sc2>>>(sc.col_cnt, cols, out->csc_colptr, nullptr, out->sparse_cap, nullptr);
       const dim3 cgrid((cols / 32 + 7) / 8, strips);
-      csc_fill_kernel<<<cgrid, 256, 0, sc2>>>(mask32, xb, rows, cols, out->thresholds, out->csc_colptr, sc.strip_off,
+      csc_fill_kernel<<<cgrid, 256, 0, sc2>>>(mask32, xb, rows, cols, out->thresholds, per_token, out->csc_colptr, sc.strip_off,
                                               out->sparse_cap, out->csc_row, out->csc_val);
     }
     if (sc2 != sp) FP4_CUDA_TRY(cudaEventRecord(overlap->csc_done, sc2));

@@ -299,3 +299,61 @@ def test_magnitude_quantile_with_ties_and_a_zero_threshold(lib):
         _check_sparse(q, ref)
         _check_dense(q, ref)
         c.close()
+
+
+def _check_token_mode(q, ref):
+    th = q.thresholds_rows.cpu().numpy()
+    rows = ref.rows
+    np.testing.assert_array_equal(th[0:2 * rows:2], ref.lo_rows.astype(np.float32))
+    np.testing.assert_array_equal(th[1:2 * rows:2], ref.hi_rows.astype(np.float32))
+    assert not (np.signbit(th) & (th == 0)).any()        # a zero threshold is +0
+    nnz = int(q.nnz.item())
+    rowptr, col, val = ref.csr
+    colptr, row, cval = ref.csc
+    assert nnz == rowptr[-1]
+    np.testing.assert_array_equal(q.csr_rowptr.cpu().numpy(), rowptr)
+    np.testing.assert_array_equal(q.csr_col.cpu().numpy()[:nnz], col)
+    np.testing.assert_array_equal(q.csr_val.cpu().numpy()[:nnz], val)
+    np.testing.assert_array_equal(q.csc_colptr.cpu().numpy(), colptr)
+    np.testing.assert_array_equal(q.csc_row.cpu().numpy()[:nnz], row)
+    np.testing.assert_array_equal(q.csc_val.cpu().numpy()[:nnz], cval)
+    _check_dense(q, ref)
+
+
+@pytest.mark.parametrize("shape,alpha,dist", [((128, 128), 0.97, "normal"), ((256, 384), 0.99, "student_t3"),
+                                              ((384, 1152), 0.999, "laplace"), ((128, 2048), 0.9, "normal")])
+def test_per_token_thresholds_variant_matches_oracle(lib, shape, alpha, dist):
+    """FP4_QUANTILE_TOKEN: every row clamped at its own order statistics (a variant outside the paper):
+    2 * rows thresholds, codes, amax and the sparse residual bit for bit."""
+    cfg = WL.Config(53, "t", shape[0], (), dist, 3, 40.0, "channels_count", (alpha,))
+    bits = WL.activations(cfg, shape[1], seed=4, layer=shape[0])
+    bits[5, :] = 0                                       # a zero row: thresholds +0, nothing clamped
+    bits[6, ::2] = bits[6, 1::2]                         # a row of pairs: ties
+    c = lib.Context(0, 256 << 20)
+    c.set_quantile_mode(lib.FP4_QUANTILE_TOKEN)
+    q = lib.fp4_quantize(c, _dev(bits), 0, alpha=alpha)
+    torch.cuda.synchronize()
+    assert c.read_status() == 0
+    _check_token_mode(q, O.occ_quantize(O.bf16_bits_to_f64(bits), alpha, quantile="token"))
+    c.close()
+
+
+def test_per_token_thresholds_through_the_layer(lib):
+    """Forward and backward with thresholds per token: the residual, its compensation in both passes
+    and the saved operands follow the oracle's variant."""
+    from test_gpu_linear import assert_close_f32
+    M, K, N, alpha = 256, 384, 256, 0.98
+    a_bits, w_bits, dy_bits = WL.small_case(M, K, N, seed=17)
+    f = O.linear_fwd(a_bits, w_bits, alpha, quantile="token")
+    b = O.linear_bwd(dy_bits, w_bits, f)
+    c = lib.Context(0, 512 << 20)
+    c.set_quantile_mode(lib.FP4_QUANTILE_TOKEN)
+    y32, sa, sw = lib.fp4_linear_fwd(c, _dev(a_bits), _dev(w_bits), alpha, out_f32=True)
+    da32, dw32 = lib.fp4_linear_bwd(c, _dev(dy_bits), _dev(w_bits), sa, sw, out_f32=True)
+    torch.cuda.synchronize()
+    assert c.read_status() == 0
+    _check_token_mode(sa, f.qa)
+    assert_close_f32(y32.cpu().numpy(), f.y, f.y_fp4, f.y_comp, "Y")
+    assert_close_f32(da32.cpu().numpy(), b.da, b.da, None, "dA")
+    assert_close_f32(dw32.cpu().numpy(), b.dw, b.s_fp4 * b.dge, b.s_comp * b.dge, "dW")
+    c.close()

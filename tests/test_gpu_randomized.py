@@ -125,7 +125,7 @@ def test_random_clamping_quantizer_is_bit_exact(lib, ctx, i, rows, cols, alpha, 
     """Thresholds, codes in both layouts, amax and the sparse residual on tensors whose rows live on
     scales spread over many binades (values outside the histogram kernel's window, subnormals),
     with ties and exact zeros of both signs."""
-    from test_gpu_quantize import _check_dense, _check_sparse
+    from test_gpu_quantize import _check_dense, _check_sparse, _check_token_mode
     rng = np.random.default_rng(5000 + i)
     a = rng.standard_normal((rows, cols)).astype(np.float32)
     if spread:
@@ -136,9 +136,11 @@ def test_random_clamping_quantizer_is_bit_exact(lib, ctx, i, rows, cols, alpha, 
         mask = rng.random(a.shape) < zeros
         a[mask] = np.where(rng.random(int(mask.sum())) < 0.5, 0.0, -0.0).astype(np.float32)
     bits = WL.to_bf16_bits(a)
-    quantile = "abs" if i % 4 == 1 else "signed"           # every fourth draw: the one-threshold variant
+    # every fourth draw each: the one-threshold variant, thresholds per token
+    quantile = {1: "abs", 2: "token"}.get(i % 4, "signed")
     ctx.status.zero_()
-    ctx.set_quantile_mode(lib.FP4_QUANTILE_ABS if quantile == "abs" else lib.FP4_QUANTILE_SIGNED)
+    ctx.set_quantile_mode({"abs": lib.FP4_QUANTILE_ABS, "token": lib.FP4_QUANTILE_TOKEN,
+                           "signed": lib.FP4_QUANTILE_SIGNED}[quantile])
     try:
         q = lib.fp4_quantize(ctx, _dev(bits), 0, alpha=alpha)
         torch.cuda.synchronize()
@@ -146,6 +148,9 @@ def test_random_clamping_quantizer_is_bit_exact(lib, ctx, i, rows, cols, alpha, 
         ctx.set_quantile_mode(lib.FP4_QUANTILE_SIGNED)
     assert ctx.read_status() == 0
     ref = O.occ_quantize(O.bf16_bits_to_f64(bits), alpha, quantile=quantile)
+    if quantile == "token":
+        _check_token_mode(q, ref)
+        return
     _check_sparse(q, ref)
     _check_dense(q, ref)
 

@@ -91,3 +91,32 @@ def test_workspace_too_small_is_refused(lib):
         lib.fp4_linear_step_host(ctx, hA, hW, hG, ALPHA, hY, hdA, hdW)
     assert e.value.code == -5
     ctx.close()
+
+
+def test_host_step_with_thresholds_per_token(lib):
+    """The host-buffer entry point under FP4_QUANTILE_TOKEN: its carved operand holds 2 * rows thresholds
+    and room for two tails per row; the outputs equal the device-resident calls in the same mode."""
+    M, K, N = 256, 384, 256
+    hA, hW, hG = _inputs(50, M, K, N)
+    ref = lib.Context.for_shape(M, K, N)
+    ref.set_quantile_mode(lib.FP4_QUANTILE_TOKEN)
+    Y, sa, sw = lib.fp4_linear_fwd(ref, hA.cuda(), hW.cuda(), ALPHA)
+    dA, dW = lib.fp4_linear_bwd(ref, hG.cuda(), hW.cuda(), sa, sw)
+    torch.cuda.synchronize()
+    ctx = lib.Context(0, int(lib.load_library().fp4_step_host_workspace_bytes(M, K, N, ALPHA)))
+    ctx.set_quantile_mode(lib.FP4_QUANTILE_TOKEN)
+    hY = torch.empty((M, N), dtype=torch.bfloat16).pin_memory()
+    hdA = torch.empty((M, K), dtype=torch.bfloat16).pin_memory()
+    hdW = torch.empty((K, N), dtype=torch.bfloat16).pin_memory()
+    for _ in range(2):
+        lib.fp4_linear_step_host(ctx, hA, hW, hG, ALPHA, hY, hdA, hdW, read_status=True)
+    assert ctx.read_status() == 0 and ref.read_status() == 0
+    for got, want in ((hY, Y), (hdA, dA), (hdW, dW)):
+        assert torch.equal(got.view(torch.int16), want.cpu().view(torch.int16))
+    # and the default mode gives something else on this input (the modes are really distinct)
+    dflt = lib.Context.for_shape(M, K, N)
+    Y0, _, _ = lib.fp4_linear_fwd(dflt, hA.cuda(), hW.cuda(), ALPHA)
+    torch.cuda.synchronize()
+    assert not torch.equal(Y0, Y)
+    for c in (ref, ctx, dflt):
+        c.close()
