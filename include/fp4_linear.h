@@ -85,7 +85,8 @@ typedef struct fp4_qtensor {
                               vector (after the clamp and the optional prescale); the scale
                               of Eq. 1 is gamma = 6 / amax and the de-scale amax / 6, each
                               rounded once to float                                           */
-  float*   thresholds;     /* [2] = {lo, hi}: the (1-alpha)- and alpha-quantile (OCC only)    */
+  float*   thresholds;     /* [2] = {lo, hi}: the (1-alpha)- and alpha-quantile (OCC only);
+                              [2 * rows] under FP4_QUANTILE_TOKEN (fp4_set_quantile_mode)     */
   int32_t* csr_rowptr;     /* [rows + 1]                                                      */
   int32_t* csr_col;        /* [sparse_cap] column index, ascending within a row               */
   float*   csr_val;        /* [sparse_cap] x - clamp(x)                                       */
