@@ -3,8 +3,9 @@
 
 One step = one pass of the whole hot path (quantile select, clamp, quantise, FP4 GEMM,
 compensation; dY quantisation, dgrad, wgrad, compensation, DGE) over every linear of the
-workload.  The workload is the LLaMA-1.3B-shaped layer set at 4096 tokens (the second entry of
-the configuration list); inputs are seeded and synthetic.
+workload.  The default workload is the largest single-GPU configuration: the seven linears of a
+LLaMA-13B-shaped decoder layer at 16384 tokens, alpha = 0.99, DGE on (the last entry of the
+configuration list); `--config I` selects another.  Inputs are seeded and synthetic.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config I]
 
@@ -12,7 +13,9 @@ Prints ONE JSON line.  `value` = sum over linears of 6 M K N flop / device time 
 inputs resident in HBM.  `e2e` = the same through fp4_linear_step_host with pinned host buffers,
 host<->device copies inside the timed region.  `roofline` describes the kernel class that takes
 the largest share of the step, timed live with CUDA events on the launching stream; `kernels`
-lists every class.  With `--impl reference` the CPU oracle is timed on the host cores instead.
+lists every class; `kernels_isolated` times single kernels alone (the GEMM at 8192^3 and at the
+workload's largest GEMM, the quantiser kernels on the workload's largest tensor), each with its
+own clock samples.  With `--impl reference` the CPU oracle is timed on the host cores instead.
 """
 from __future__ import annotations
 
@@ -33,20 +36,23 @@ METRIC = "fp4_linear_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
 # fallback peaks (an earlier measurement on this machine), used only if MEASURED_PEAKS.json is absent
 FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
 FALLBACK_BF16_TFLOPS_SUSTAINED = 1400.0
 FP4_OVER_BF16 = 4.0                 # nominal dense ratio 9 : 2.25 PFLOP/s
 SM_COUNT, FMA_LANES = 148, 128      # plain fp32 pipe: 148 SMs x 128 FMA lanes x 2 flop
+BURST_SECONDS = 1.0                 # a class timed inside a region shorter than this is held to the burst peak
 
-# DRAM bytes per launch of the dominant kernel from the committed ncu summaries
-# (profiles/*.md); None where no capture exists for the class.
-NCU_TRAFFIC_PER_UNIT = {
-    # mean DRAM read + write per launch of the class, from the captures summarised under profiles/
-    "gemm": 17.4e6,        # gemm_fp4_llama1p3b.md: forward 6.4 MB, backward (two GEMMs per launch) 28.3 MB
-    "encode": 14.0e6,      # quantizer_encode_llama1p3b.md (writes still in L2 at kernel end)
-    "select": 16.9e6,      # quantizer_select_absmax_llama1p3b.md, hist_select_kernel
-    "absmax": 12.6e6,
-    "comp_fwd": 36.1e6,    # compensation_llama1p3b.md
-    "comp_wgrad_dge": 6.5e6,
+# DRAM bytes (read + write) per launch of a kernel class, from the ncu captures summarised under
+# profiles/, keyed by workload; a class without a capture on that workload reports null.
+NCU_TRAFFIC_PER_LAUNCH = {
+    "llama-1.3b-layer": {
+        "gemm": 17.4e6,        # profiles/gemm_fp4_llama1p3b.md: forward 6.4 MB, backward (two GEMMs per launch) 28.3 MB
+        "encode": 14.0e6,      # profiles/quantizer_encode_llama1p3b.md (writes still in L2 at kernel end)
+        "select": 16.9e6,      # profiles/quantizer_select_absmax_llama1p3b.md
+        "absmax": 12.6e6,
+        "comp_fwd": 36.1e6,    # profiles/compensation_llama1p3b.md
+        "comp_wgrad_dge": 6.5e6,
+    },
 }
 
 
@@ -54,10 +60,11 @@ def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         p = json.load(open(path))
-        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops_sustained"]),
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_burst=float(p["bf16_tflops"]),
+                    bf16_sustained=float(p["bf16_tflops_sustained"]),
                     sm_max_mhz=float(p.get("sm_max_mhz", 1965.0)), source="measured")
-    return dict(hbm_gbs=FALLBACK_HBM_GBS, bf16_tflops=FALLBACK_BF16_TFLOPS_SUSTAINED, sm_max_mhz=1965.0,
-                source="fallback")
+    return dict(hbm_gbs=FALLBACK_HBM_GBS, bf16_burst=FALLBACK_BF16_TFLOPS,
+                bf16_sustained=FALLBACK_BF16_TFLOPS_SUSTAINED, sm_max_mhz=1965.0, source="fallback")
 
 
 class ClockSampler:
@@ -125,6 +132,9 @@ def layer_inputs(cfg, WL, seed=0):
     return out
 
 
+ORACLE_SAMPLE_TOKENS = 1024         # tokens of the first linear the oracle is timed on (a bounded sample)
+
+
 def oracle_sample_tflops(cfg, WL, reps: int, m_rows: int):
     """The oracle as it stands on the first linear of the workload, `m_rows` tokens; TFLOP/s."""
     from oracle import fp4_oracle as O
@@ -143,20 +153,25 @@ def oracle_sample_tflops(cfg, WL, reps: int, m_rows: int):
     return flop / 1e12, times
 
 
+def oracle_sample_text(cfg, m_rows: int) -> str:
+    lin = cfg.linears[0]
+    return (f"oracle fwd+bwd (select, clamp, quantise, GEMMs, compensation, DGE) of linear '{lin.name}' "
+            f"({lin.K}x{lin.N}) on the first {m_rows} of {cfg.M} tokens")
+
+
 def run_reference(args):
     """CPU oracle on the host cores; rank 0 alone works and prints."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
     from paper_2501_17116_b200 import workloads as WL
     cfg = WL.CONFIGS[args.config]
-    m_rows = 1024
+    m_rows = min(ORACLE_SAMPLE_TOKENS, cfg.M)
     tf, times = oracle_sample_tflops(cfg, WL, args.warmup + args.steps, m_rows)
     timed = times[args.warmup:]
     sec = float(np.sum(timed))
     value = tf * len(timed) / sec
     cores = os.cpu_count()
-    lin = cfg.linears[0]
-    sample = f"oracle fwd+bwd of linear '{lin.name}' ({lin.K}x{lin.N}) on the first {m_rows} tokens per step"
+    sample = oracle_sample_text(cfg, m_rows) + " per step"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sec / len(timed),
@@ -168,18 +183,126 @@ def run_reference(args):
     }))
 
 
+def timed_with_clocks(gpu_index: int, fn, min_seconds: float = 0.4):
+    """Runs fn() repeatedly for at least `min_seconds` of device time with the clocks sampled
+    beside it; returns (reps, elapsed ms by CUDA events on the current stream, clock record)."""
+    import torch
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    fn()
+    e1.record()
+    torch.cuda.synchronize()
+    reps = max(5, int(min_seconds * 1e3 / max(e0.elapsed_time(e1), 1e-3)))
+    sampler = ClockSampler(gpu_index)
+    sampler.start()
+    time.sleep(0.12)
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    return reps, ms, sampler.stop()
+
+
+def isolated_kernels(fp4, WL, cfg, dev, gpu_index: int, kind: int, peaks) -> dict:
+    """Single kernels timed alone, each with its own clock samples: the GEMM at 8192^3 and at the
+    workload's largest GEMM, the quantiser kernels on the workload's largest activation-sized
+    tensor (larger than L2, so every repetition reads it from HBM)."""
+    import torch
+    out = {}
+    burst = (FP4_OVER_BF16 if kind == 0 else FP4_OVER_BF16 / 2) * peaks["bf16_burst"]
+    ctx = fp4.Context(gpu_index, 1 << 20)
+    big = max(cfg.linears, key=lambda l: l.K * l.N)
+    for label, (I, J, Cc) in (("gemm_8192x8192x8192", (8192, 8192, 8192)),
+                              (f"gemm_fwd_{big.name}_{cfg.M}x{big.N}x{big.K}", (cfg.M, big.N, big.K))):
+        a = torch.randint(0, 255, (I, Cc // 2), dtype=torch.uint8, device=dev)
+        b = torch.randint(0, 255, (J, Cc // 2), dtype=torch.uint8, device=dev)
+        ra, ca = torch.rand(I, device=dev), torch.rand(J, device=dev)
+        o = torch.empty((I, J), dtype=torch.bfloat16, device=dev)
+        reps, ms, clk = timed_with_clocks(
+            gpu_index, lambda: fp4.fp4_gemm(ctx, a, b, ra, ca, out_f32=False, gemm_kind=kind, out=o))
+        tf = 2.0 * I * J * Cc * reps / (ms / 1e3) / 1e12
+        out[label] = {"bound": "tensor", "us": round(1e3 * ms / reps, 2), "achieved": round(tf, 1), "unit": "TFLOP/s",
+                      "peak": round(burst, 1), "frac": round(tf / burst, 4),
+                      "peak_source": "4 x burst bf16 cuBLAS (kernel timed alone)", "reps": reps, "clocks": clk}
+        del a, b, o
+    assert ctx.read_status() == 0
+    ctx.close()
+
+    # quantiser kernels on the largest activation-sized tensor of the workload
+    M = cfg.M
+    Kq = max(max(l.K for l in cfg.linears), max(l.N for l in cfg.linears))
+    alpha = cfg.alphas[0]
+    x = torch.from_numpy(WL.activations(cfg, Kq, M=M).view(np.int16)).to(dev).view(torch.bfloat16)
+    ctx = fp4.Context(gpu_index, int(fp4.load_library().fp4_workspace_bytes(M, Kq, 128)))
+    q = fp4.QTensor(M, Kq, 0, dev, fp4.tail_capacity(M, Kq, alpha))
+    qw = fp4.QTensor(M, Kq, 1, dev)
+    ctx.set_overlap(False)
+    elems = float(M) * Kq
+
+    def both():
+        fp4.fp4_quantize(ctx, x, 0, alpha=alpha, out=q)      # token-wise with clamping: select, encode, sparse
+        fp4.fp4_quantize(ctx, x, 1, out=qw)                  # channel-wise, no clamp: absmax, encode
+
+    for _ in range(2):
+        both()
+    torch.cuda.synchronize()
+    ctx.profile_reset()
+    ctx.profile_enable(True)
+    sampler = ClockSampler(gpu_index)
+    sampler.start()
+    time.sleep(0.12)
+    reps = 0
+    t0 = time.perf_counter()
+    while reps < 5 or time.perf_counter() - t0 < 0.4:
+        fp4.fp4_quantize(ctx, x, 0, alpha=alpha, out=q)
+        reps += 1
+        torch.cuda.synchronize()
+    occ = ctx.profile_read()
+    ctx.profile_reset()
+    reps_w = 0
+    t0 = time.perf_counter()
+    while reps_w < 5 or time.perf_counter() - t0 < 0.4:
+        fp4.fp4_quantize(ctx, x, 1, out=qw)
+        reps_w += 1
+        torch.cuda.synchronize()
+    plain = ctx.profile_read()
+    clk = sampler.stop()
+    ctx.profile_enable(False)
+    shape = f"{M}x{Kq}"
+    for label, rec, n, bytes_per_elem in (
+            (f"select_{shape}", occ["select"], reps, 2.0),
+            (f"encode_clamped_{shape}", occ["encode"], reps, 3.125),
+            (f"absmax_{shape}", plain["absmax"], reps_w, 2.0),
+            (f"encode_{shape}", plain["encode"], reps_w, 3.0)):
+        ms = rec[0] / n
+        gbs = bytes_per_elem * elems / (ms / 1e3) / 1e9 if ms > 0 else 0.0
+        out[label] = {"bound": "hbm", "us": round(1e3 * ms, 2), "achieved": round(gbs, 1), "unit": "GB/s",
+                      "peak": peaks["hbm_gbs"], "frac": round(gbs / peaks["hbm_gbs"], 4),
+                      "bytes_per_element": bytes_per_elem, "reps": n, "clocks": clk}
+    assert ctx.read_status() == 0
+    ctx.close()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=1)
+    ap.add_argument("--config", type=int, default=4)
     ap.add_argument("--gemm-kind", type=int, default=0, help="0 mxf4 (K=64), 1 f8f6f4 (K=32)")
     ap.add_argument("--precision", default="w4a4", choices=["w4a4", "w4a8", "w8a4", "w4a4-dy8", "w4a4-dy8e5m2"],
                     help="operand formats: w4a4 (the method, default); w4a8 / w8a4: E4M3 activations / weights "
                          "(the ablation settings); w4a4-dy8 / w4a4-dy8e5m2: dY quantised to E4M3 / E5M2.  All but w4a4 need --gemm-kind 1")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer measurement (profiling runs)")
+    ap.add_argument("--no-isolated", action="store_true", help="skip the single-kernel measurements")
     ap.add_argument("--no-share-activations", action="store_true",
                     help="quantise the activation of every linear, also where q/k/v or gate/up read the same tensor")
     ap.add_argument("--cache-weights", action="store_true",
@@ -309,7 +432,7 @@ def main():
     # ------------------------------------------------------------------ end to end ---------
     # (the host-buffer entry point takes the method's own formats only)
     ms_e2e = None
-    if args.precision == "w4a4":
+    if args.precision == "w4a4" and not args.no_e2e:
         for _ in range(3):
             step_host()
         torch.cuda.synchronize()
@@ -333,8 +456,13 @@ def main():
     d2h = h2d
 
     # ------------------------------------------------------------------ rooflines ----------
-    # the byte-container kind runs at the FP8 rate (K = 32 per instruction), the MXF4 kind at twice that
-    fp4_peak = (FP4_OVER_BF16 if kind == 0 else FP4_OVER_BF16 / 2) * peaks["bf16_tflops"]
+    # Tensor peak: 4 x the measured BF16 cuBLAS rate (nominal dense FP4 : BF16 = 9 : 2.25); the
+    # byte-container kind runs at the FP8 rate (K = 32 per instruction), half of that.  The burst
+    # figure applies to a class whose timed region is short, the sustained one to a seconds-long one.
+    ratio = FP4_OVER_BF16 if kind == 0 else FP4_OVER_BF16 / 2
+    region_seconds = ms_profiled / 1e3
+    use_burst = region_seconds < BURST_SECONDS
+    fp4_peak = ratio * (peaks["bf16_burst"] if use_burst else peaks["bf16_sustained"])
     alu_peak = SM_COUNT * FMA_LANES * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
     steps = args.steps
     elems_a = sum(M * L["K"] for L in layers if not L["reuse_a"])      # activations actually quantised
@@ -343,15 +471,25 @@ def main():
     nnz_total = sum(nnz)
     nnz_quantised = sum(z for z, L in zip(nnz, layers) if not L["reuse_a"])
     work = {
-        # class: (bound, algorithmic work per step, unit of the rate)
+        # class: (bound, algorithmic work per step, unit of the rate).  Bytes are what the method
+        # itself has to move: every tensor read once per kernel class that needs it, codes written
+        # once per layout (A: 2 + 0.5 + 0.5 + 1/8 mask; W: 2 + 1; dY: 2 + 0.5 + 0.5, both backward
+        # copies from one read).
         "gemm": ("tensor", flop_step, "TFLOP/s"),
-        "select": ("hbm", 2.0 * elems_a, "GB/s"),                                   # one read of A
-        "encode": ("hbm", 3.125 * elems_a + 3.0 * elems_w + 2 * 2.5 * elems_g, "GB/s"),
-        "absmax": ("hbm", 2.0 * elems_w + 2 * 2.0 * elems_g, "GB/s"),                # one read each
+        "select": ("hbm", 2.0 * elems_a, "GB/s"),
+        "encode": ("hbm", 3.125 * elems_a + 3.0 * elems_w + 3.0 * elems_g, "GB/s"),
+        "absmax": ("hbm", 2.0 * elems_w + 2.0 * elems_g, "GB/s"),
         "sparse": ("hbm", 2 * 8.0 * nnz_quantised + 3 * elems_a / 8.0, "GB/s"),       # entries + 3 mask sweeps
         "comp_fwd": ("alu", sum(2.0 * z * L["N"] for z, L in zip(nnz, layers)), "TFLOP/s"),
         "comp_wgrad_dge": ("alu", sum(2.0 * z * L["N"] + 8.0 * L["K"] * L["N"] for z, L in zip(nnz, layers)),
                            "TFLOP/s"),
+    }
+    src = "of measured" if peaks["source"] == "measured" else "of fallback"
+    peak_text = {
+        "tensor": f"{src}: {ratio:g} x {'burst' if use_burst else 'sustained'} bf16 cuBLAS "
+                  f"(classes timed inside a {region_seconds:.2f} s region)",
+        "hbm": f"{src}: copy bandwidth",
+        "alu": "148 SMs x 128 FMA x 2 x max clock",
     }
     kernels = {}
     total_ms = sum(v[0] for v in prof.values()) or 1.0
@@ -363,22 +501,27 @@ def main():
         kernels[name] = {"bound": bound, "achieved": round(achieved, 2), "peak": round(peak, 1), "unit": unit,
                          "frac": round(achieved / peak, 4), "ms_per_step": round(t_ms / steps, 4),
                          "share": round(t_ms / total_ms, 4), "launches_per_step": n // steps}
+        if bound == "tensor":
+            kernels[name]["frac_of_burst"] = round(achieved / (ratio * peaks["bf16_burst"]), 4)
+            kernels[name]["frac_of_sustained"] = round(achieved / (ratio * peaks["bf16_sustained"]), 4)
     dominant = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
     dk = kernels[dominant]
+    traffic = NCU_TRAFFIC_PER_LAUNCH.get(cfg.name, {}).get(dominant) if args.precision == "w4a4" and kind == 0 else None
     roofline = {"kernel": dominant, "bound": dk["bound"], "achieved": dk["achieved"], "peak": dk["peak"],
-                "unit": dk["unit"], "frac": dk["frac"], "traffic": NCU_TRAFFIC_PER_UNIT.get(dominant),
-                "peak_source": ("of measured" if peaks["source"] == "measured" else "of fallback")
-                + ((": 4 x sustained bf16 cuBLAS" if kind == 0 else ": 2 x sustained bf16 cuBLAS (FP8-rate kind)")
-                   if dk["bound"] == "tensor" else
-                   ": copy bandwidth" if dk["bound"] == "hbm" else ": 148 SMs x 128 FMA x 2 x max clock")}
+                "unit": dk["unit"], "frac": dk["frac"], "traffic": traffic, "peak_source": peak_text[dk["bound"]]}
+
+    # ------------------------------------------------------------------ single kernels -----
+    kernels_isolated = None
+    if not args.no_isolated and args.precision == "w4a4":
+        kernels_isolated = isolated_kernels(fp4, WL, cfg, dev, local_rank, kind, peaks)
 
     # ------------------------------------------------------------------ CPU baseline -------
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        tf, times = oracle_sample_tflops(cfg, WL, 5, M)
-        lin = cfg.linears[0]
+        m_rows = min(ORACLE_SAMPLE_TOKENS, M)
+        tf, times = oracle_sample_tflops(cfg, WL, 3, m_rows)
         cpu_baseline = {"value": tf / min(times), "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
-                        "sample": f"fwd+bwd of linear '{lin.name}' ({lin.K}x{lin.N}) at {M} tokens, best of 5",
+                        "sample": oracle_sample_text(cfg, m_rows) + ", best of 3",
                         "seconds": round(min(times), 3)}
 
     if rank == 0:
@@ -402,7 +545,8 @@ def main():
             "e2e": ({"value": value_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                      "ms_per_step": 1e3 * sec_e2e / args.steps} if sec_e2e else None),
             "gpu_launches": launches,
-            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu_baseline, "clocks": clocks,
+            "roofline": roofline, "kernels": kernels, "kernels_isolated": kernels_isolated,
+            "cpu_baseline": cpu_baseline, "clocks": clocks,
             "residual_nnz": nnz_total,
         }))
     ctx.close()
