@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB_PATH = os.path.join(HERE, "libfp4linear.so")
-SOURCES = ("api.cu", "gemm_fp4.cu", "quantize.cu", "compensate.cu")
+SOURCES = ("api.cu", "gemm_fp4.cu", "quantize.cu", "compensate.cu", "wgrad_dense_tc.cu")
 
 
 def _nvcc() -> str:

@@ -410,7 +410,7 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
     FP4_CUDA_TRY(cudaStreamWaitEvent(sw, ctx->ev[5], 0));
   }
   if (has_comp) {
-    rc = launch_comp_wgrad(ctx, sw, savedA, dY_bf16, comp_arena, &slot_of_col, comp, M, K, N);
+    rc = launch_comp_wgrad(ctx, sw, savedA, dY_bf16, comp_arena, &slot_of_col, comp, M, K, N, status);
     if (rc != FP4_OK) return rc;
   }
 

@@ -232,6 +232,17 @@ int launch_fwd_tail(fp4_ctx* ctx, cudaStream_t stream, const fp4_qtensor* a, con
 // Lists, slots and the dense path's buffers are carved from `scratch` (comp_wgrad_scratch_bytes); the slot
 // vector is handed back for the GEMM's epilogue.  `a` is the saved activation (CSC; CSR for the dense path).
 int launch_comp_wgrad(fp4_ctx* ctx, cudaStream_t stream, const fp4_qtensor* a, const void* dy_bf16, Arena& scratch,
-                      int** slot_of_col_out, float* comp, int64_t M, int64_t K, int64_t N);
+                      int** slot_of_col_out, float* comp, int64_t M, int64_t K, int64_t N, int32_t* status);
 size_t comp_wgrad_scratch_bytes(int64_t M, int64_t K, int64_t N);
+
+// Dense columns of the residual in the weight gradient, on the tensor cores (wgrad_dense_tc.cu):
+// C[s, :] = sum_m V[m, s] dY[m, :] for the s < counts[0] <= DENSE_TC_MAX dense columns, as `splits`
+// sets of partial sums ([splits][DENSE_TC_MAX][N], one per range of tokens) that the caller adds in
+// order.  `vt` holds 3 * DENSE_TC_MAX * M BF16 values of scratch.
+constexpr int DENSE_TC_MAX = 128;
+int dense_tc_splits(const fp4_ctx* ctx, int64_t M, int64_t N);
+size_t dense_tc_scratch_bytes(int64_t M, int64_t N);
+int launch_comp_wgrad_dense_tc(fp4_ctx* ctx, cudaStream_t stream, const fp4_qtensor* a, const int* slot_of_col,
+                               const int* counts, const void* dy_bf16, void* vt, float* partial, int splits,
+                               int64_t M, int64_t N, int32_t* status);
 

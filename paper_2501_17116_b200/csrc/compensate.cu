@@ -149,9 +149,6 @@ comp_fwd_skip_kernel(const float* __restrict__ y1, const int* __restrict__ rowpt
 
 constexpr int LONG_COLUMN = 512;           // entries from which a column gets a whole 1024-thread block
 constexpr int LONG_THREADS = 1024;
-constexpr int DENSE_SLOTS = 8;             // dense columns handled per pass (accumulators per lane: 8 x 8)
-constexpr int DENSE_MAX = 160;             // dense columns at most; further ones are treated as long
-constexpr int DENSE_MAX_CHUNKS = 40;       // chunks of tokens whose partial sums are added afterwards
 
 // Exclusive scan of one int per thread over a 1024-thread block; the block's total goes to *total.
 __device__ __forceinline__ int block_exclusive_scan_1024(int c, int* warp_tot, int* total) {
@@ -271,7 +268,7 @@ tail_b_kernel(const __nv_bfloat16* __restrict__ w, const int* __restrict__ list_
 }
 
 // The columns of the residual that hold entries, by how full they are: "dense" (at least
-// `dense_from` entries, the first DENSE_MAX of them: outlier channels that most tokens hit,
+// `dense_from` entries, the first DENSE_TC_MAX of them: outlier channels that most tokens hit,
 // Appendix D), "long" (at least LONG_COLUMN entries) and "short".  The long and the short ones
 // are listed in ascending order; counts[0..2] are the three sizes.  Rows of the compact buffer:
 // dense columns first, then the long, then the short ones, each in ascending column order;
@@ -287,13 +284,13 @@ nonempty_columns_kernel(const int* __restrict__ colptr, int K, int dense_from, i
   for (int k = b; k < e; ++k) c_cand += (colptr[k + 1] - colptr[k] >= dense_from) ? 1 : 0;
   int n_cand;
   int rank = block_exclusive_scan_1024(c_cand, warp_tot, &n_cand);     // dense candidates before this thread
-  const int n_dense = min(n_cand, DENSE_MAX);
+  const int n_dense = min(n_cand, DENSE_TC_MAX);
   int c_long = 0, c_short = 0;
   {
     int r = rank;
     for (int k = b; k < e; ++k) {
       const int n = colptr[k + 1] - colptr[k];
-      if (n >= dense_from && r++ < DENSE_MAX) continue;
+      if (n >= dense_from && r++ < DENSE_TC_MAX) continue;
       if (n >= LONG_COLUMN) ++c_long;
       else if (n > 0) ++c_short;
     }
@@ -304,7 +301,7 @@ nonempty_columns_kernel(const int* __restrict__ colptr, int K, int dense_from, i
   for (int k = b; k < e; ++k) {
     const int n = colptr[k + 1] - colptr[k];
     int slot = -1;
-    if (n >= dense_from && rank < DENSE_MAX) slot = rank;
+    if (n >= dense_from && rank < DENSE_TC_MAX) slot = rank;
     else if (n >= LONG_COLUMN) { slot = n_dense + pos_long; list_long[pos_long++] = k; }
     else if (n > 0) { slot = n_dense + n_long + pos_short; list_short[pos_short++] = k; }
     if (n >= dense_from) ++rank;
@@ -317,107 +314,8 @@ nonempty_columns_kernel(const int* __restrict__ colptr, int K, int dense_from, i
   }
 }
 
-// Dense columns, step 1: their residual values as a dense matrix V[g][m][8] (group g holds the
-// compact rows 8 g .. 8 g + 7), zero where a token has no entry.  One warp per token walks the
-// token's CSR row.
-__global__ void __launch_bounds__(COMP_THREADS)
-dense_values_kernel(const int* __restrict__ rowptr, const int* __restrict__ col, const float* __restrict__ val,
-                    const int* __restrict__ slot_of_col, const int* __restrict__ counts, float* __restrict__ V, int M) {
-  const int n_dense = counts[0];
-  if (n_dense == 0) return;
-  const int groups = (n_dense + DENSE_SLOTS - 1) / DENSE_SLOTS;
-  const int lane = threadIdx.x & 31;
-  const int m = blockIdx.x * (COMP_THREADS / 32) + (threadIdx.x >> 5);
-  if (m >= M) return;
-  for (int i = lane; i < groups * DENSE_SLOTS; i += 32)
-    V[(size_t(i / DENSE_SLOTS) * M + m) * DENSE_SLOTS + (i % DENSE_SLOTS)] = 0.0f;
-  __syncwarp();
-  for (int e = rowptr[m] + lane; e < rowptr[m + 1]; e += 32) {
-    const int slot = slot_of_col[col[e]];
-    if (slot >= 0 && slot < n_dense) V[(size_t(slot / DENSE_SLOTS) * M + m) * DENSE_SLOTS + (slot % DENSE_SLOTS)] = val[e];
-  }
-}
-
-// Dense columns, step 2: C[slot, n] = sum_m V[m, slot] * dY[m, n] as a skinny dense product on the
-// plain ALUs: a block owns 256 output columns (8 per lane) and one chunk of the tokens, its 8
-// warps take the chunk's tokens in turn (four tokens' loads in flight), every lane keeps 8 x 8
-// accumulators, and dY is read once per group of 8 columns instead of once per entry.  The warps'
-// sums are added in warp order and, with more than one chunk, written as partial sums that
-// dense_reduce_kernel adds in chunk order: the result does not depend on scheduling.
-__global__ void __launch_bounds__(COMP_THREADS, 2)
-comp_wgrad_dense_kernel(float* __restrict__ out, const float* __restrict__ V, const uint4* __restrict__ dy,
-                        const int* __restrict__ counts, int M, int N, int rows_per_chunk, long long chunk_stride) {
-  constexpr int WARPS = COMP_THREADS / 32;
-  constexpr int FLY = 4;
-  __shared__ float red[WARPS][4][COMP_COLS];                    // 32 KB: four compact rows at a time
-  const int n_dense = counts[0];
-  if (n_dense == 0) return;
-  const int groups = (n_dense + DENSE_SLOTS - 1) / DENSE_SLOTS;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * COMP_COLS + 8 * lane;
-  const bool in_cols = n0 < N;
-  const int r0 = blockIdx.y * rows_per_chunk, r1 = min(M, r0 + rows_per_chunk);
-  const int vec_per_row = N >> 3, vcol = n0 >> 3;
-  float* dst = out + (long long)blockIdx.y * chunk_stride;
-  for (int g = 0; g < groups; ++g) {
-    float acc[DENSE_SLOTS][8];
-#pragma unroll
-    for (int s = 0; s < DENSE_SLOTS; ++s)
-#pragma unroll
-      for (int c = 0; c < 8; ++c) acc[s][c] = 0.0f;
-    if (in_cols) {
-      const float4* vg = reinterpret_cast<const float4*>(V + size_t(g) * M * DENSE_SLOTS);
-      for (int r = r0 + warp; r < r1; r += WARPS * FLY) {
-        uint4 d[FLY];
-        float4 v[FLY][DENSE_SLOTS / 4];
-#pragma unroll
-        for (int u = 0; u < FLY; ++u) {
-          const int ru = r + u * WARPS;
-          const bool live = ru < r1;                            // past the end: zeros times token r
-          d[u] = __ldg(&dy[(long long)(live ? ru : r) * vec_per_row + vcol]);
-#pragma unroll
-          for (int q = 0; q < DENSE_SLOTS / 4; ++q)             // same address in every lane
-            v[u][q] = live ? __ldg(&vg[size_t(ru) * (DENSE_SLOTS / 4) + q]) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-#pragma unroll
-        for (int u = 0; u < FLY; ++u) {
-#pragma unroll
-          for (int q = 0; q < DENSE_SLOTS / 4; ++q) {
-            fma8(acc[4 * q + 0], v[u][q].x, d[u]);
-            fma8(acc[4 * q + 1], v[u][q].y, d[u]);
-            fma8(acc[4 * q + 2], v[u][q].z, d[u]);
-            fma8(acc[4 * q + 3], v[u][q].w, d[u]);
-          }
-        }
-      }
-    }
-#pragma unroll
-    for (int b = 0; b < DENSE_SLOTS / 4; ++b) {
-      __syncthreads();                                  // the previous batch has been read
-#pragma unroll
-      for (int sl = 0; sl < 4; ++sl) {
-        *reinterpret_cast<float4*>(&red[warp][sl][8 * lane]) =
-            make_float4(acc[4 * b + sl][0], acc[4 * b + sl][1], acc[4 * b + sl][2], acc[4 * b + sl][3]);
-        *reinterpret_cast<float4*>(&red[warp][sl][8 * lane + 4]) =
-            make_float4(acc[4 * b + sl][4], acc[4 * b + sl][5], acc[4 * b + sl][6], acc[4 * b + sl][7]);
-      }
-      __syncthreads();
-      const int n = blockIdx.x * COMP_COLS + threadIdx.x;
-#pragma unroll
-      for (int sl = 0; sl < 4; ++sl) {
-        const int slot = g * DENSE_SLOTS + 4 * b + sl;
-        if (slot < n_dense && n < N) {
-          float t = 0.0f;
-#pragma unroll
-          for (int w = 0; w < WARPS; ++w) t += red[w][sl][threadIdx.x];
-          dst[(long long)slot * N + n] = t;
-        }
-      }
-    }
-  }
-}
-
-// Dense columns, step 3 (only with more than one chunk): C[slot, n] = sum over the chunks, in order.
+// Dense columns (their partial sums come from the tensor-core kernel, one set per range of tokens):
+// C[slot, n] = sum over the ranges, in order.
 __global__ void __launch_bounds__(256)
 dense_reduce_kernel(float* __restrict__ comp, const float* __restrict__ partial, const int* __restrict__ counts, int N,
                     int chunks, long long chunk_stride) {
@@ -542,20 +440,10 @@ int launch_comp_fwd(fp4_ctx* ctx, cudaStream_t stream, const float* y1, const in
   return FP4_OK;
 }
 
-// Chunks of tokens of the dense path: about 2 x 148 blocks in all, at least 64 tokens per chunk.
-static int dense_chunks(int64_t M, int64_t N) {
-  const int n_blocks = int((N + COMP_COLS - 1) / COMP_COLS);
-  int chunks = 296 / n_blocks;
-  chunks = chunks < 1 ? 1 : (chunks > DENSE_MAX_CHUNKS ? DENSE_MAX_CHUNKS : chunks);
-  if (int64_t(chunks) * 64 > M) chunks = int(M / 64) > 0 ? int(M / 64) : 1;
-  return chunks;
-}
-
 size_t comp_wgrad_scratch_bytes(int64_t M, int64_t K, int64_t N) {
   auto r256 = [](size_t b) { return (b + 255) & ~size_t(255); };
   size_t b = r256((2 * size_t(K) + 4) * 4) + r256(size_t(K) * 4);                     // lists + counters, slots
-  b += r256(size_t(DENSE_MAX) * size_t(M) * 4);                                       // V
-  b += r256(size_t(dense_chunks(M, N)) * size_t(DENSE_MAX) * size_t(N) * 4);          // partial sums
+  b += dense_tc_scratch_bytes(M, N);                                                  // BF16 terms, partial sums
   return b;
 }
 
@@ -594,38 +482,34 @@ int launch_fwd_tail(fp4_ctx* ctx, cudaStream_t stream, const fp4_qtensor* a, con
 }
 
 int launch_comp_wgrad(fp4_ctx* ctx, cudaStream_t stream, const fp4_qtensor* a, const void* dy_bf16, Arena& scratch,
-                      int** slot_of_col_out, float* comp, int64_t M, int64_t K, int64_t N) {
+                      int** slot_of_col_out, float* comp, int64_t M, int64_t K, int64_t N, int32_t* status) {
   // lists: [K] long columns, [K] short columns, three counters
   int* lists = scratch.take<int>(2 * size_t(K) + 4);
   int* slot_of_col = scratch.take<int>(size_t(K));
-  float* V = scratch.take<float>(size_t(DENSE_MAX) * size_t(M));
-  const int chunks = dense_chunks(M, N);
-  float* partial = scratch.take<float>(size_t(chunks) * size_t(DENSE_MAX) * size_t(N));
+  const int splits = dense_tc_splits(ctx, M, N);
+  void* vt = scratch.take<uint16_t>(size_t(3) * DENSE_TC_MAX * size_t(M));
+  float* partial = scratch.take<float>(size_t(splits) * DENSE_TC_MAX * size_t(N));
   if (!scratch.ok) return FP4_ERR_WORKSPACE;
   *slot_of_col_out = slot_of_col;
   int* list_long = lists;
   int* list_short = lists + K;
   int* counts = lists + 2 * K;
-  // The dense path pays when the residual is heavy (two launches more, far less traffic): it is
-  // taken when the residual may hold at least 1 % of the activation (alpha <= 0.995), for the
-  // columns that at least a quarter of the tokens hit.
-  const bool dense = a->csr_rowptr && a->sparse_cap * 100 >= M * K;
+  // Columns that at least a quarter of the tokens hit (the outlier channels) form the dense class,
+  // whose product runs on the tensor cores; it needs the CSR.
+  const bool dense = a->csr_rowptr != nullptr;
   const int dense_from = dense ? int(M / 4 > LONG_COLUMN ? M / 4 : LONG_COLUMN) : INT_MAX;
   const unsigned n_blocks = unsigned((N + COMP_COLS - 1) / COMP_COLS);
-  const int rows_per_chunk = int((M + chunks - 1) / chunks);
-  KernelScope scope(ctx, stream, KC_COMP_WGRAD, 3 + (dense ? (chunks > 1 ? 3 : 2) : 0));
+  KernelScope scope(ctx, stream, KC_COMP_WGRAD, 3 + (dense ? (splits > 1 ? 3 : 2) : 0));
   nonempty_columns_kernel<<<1, 1024, 0, stream>>>(a->csc_colptr, int(K), dense_from, list_long, list_short, counts,
                                                   slot_of_col);
   const uint4* dy = static_cast<const uint4*>(dy_bf16);
   if (dense) {
-    dense_values_kernel<<<unsigned((M + 7) / 8), COMP_THREADS, 0, stream>>>(a->csr_rowptr, a->csr_col, a->csr_val,
-                                                                           slot_of_col, counts, V, int(M));
-    const long long chunk_stride = (long long)DENSE_MAX * N;
-    comp_wgrad_dense_kernel<<<dim3(n_blocks, unsigned(chunks)), COMP_THREADS, 0, stream>>>(
-        chunks > 1 ? partial : comp, V, dy, counts, int(M), int(N), rows_per_chunk, chunk_stride);
-    if (chunks > 1)
-      dense_reduce_kernel<<<unsigned(2 * ctx->num_sms), 256, 0, stream>>>(comp, partial, counts, int(N), chunks,
-                                                                         chunk_stride);
+    const int rc = launch_comp_wgrad_dense_tc(ctx, stream, a, slot_of_col, counts, dy_bf16, vt,
+                                              splits > 1 ? partial : comp, splits, M, N, status);
+    if (rc != FP4_OK) return rc;
+    if (splits > 1)
+      dense_reduce_kernel<<<unsigned(2 * ctx->num_sms), 256, 0, stream>>>(comp, partial, counts, int(N), splits,
+                                                                         (long long)DENSE_TC_MAX * N);
   }
   unsigned gy = unsigned(4 * ctx->num_sms) / n_blocks;          // long columns: 2 resident blocks per SM
   gy = gy < 1 ? 1 : (gy > unsigned(K) ? unsigned(K) : gy);
