@@ -258,9 +258,6 @@ int fp4_profile_enable(fp4_ctx* ctx, int on);
  * the call's work ends.  fp4_set_overlap(ctx, 0) puts every kernel on `stream` in program order
  * (used to time kernels one at a time); the results are identical either way.  Default: on.  */
 int fp4_set_overlap(fp4_ctx* ctx, int on);
-/* MXF4 GEMMs on pairs of CTAs (tcgen05.mma.cta_group::2, 256 x 240 tile per pair: a third less
- * operand traffic from L2 per flop).  Same results bit for bit.  Default: off.               */
-int fp4_set_gemm_pairs(fp4_ctx* ctx, int on);
 /* Which order statistics the clamp of an activation uses (fp4_quantize with alpha < 1 and the
  * calls built on it; not fp4_quantile_thresholds_static).  FP4_QUANTILE_SIGNED (default): the
  * paper's form (Section 3.2), lo and hi the (1-alpha)- and alpha-quantiles of the values.

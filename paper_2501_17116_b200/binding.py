@@ -32,7 +32,7 @@ FP4_DEV_TIMEOUT = 4
 EXPORTS = ("fp4_create", "fp4_destroy", "fp4_workspace_bytes", "fp4_status_string", "fp4_quantize",
            "fp4_gemm", "fp4_linear_fwd", "fp4_linear_bwd", "fp4_step_host_workspace_bytes",
            "fp4_linear_step_host", "fp4_profile_enable", "fp4_profile_reset", "fp4_profile_read",
-           "fp4_launch_count", "fp4_quantile_thresholds_static", "fp4_set_overlap", "fp4_set_gemm_pairs",
+           "fp4_launch_count", "fp4_quantile_thresholds_static", "fp4_set_overlap",
            "fp4_set_quantile_mode")
 FP4_STATIC_MAX_ROWS = 65536
 FP4_QUANTILE_SIGNED = 0
@@ -95,8 +95,6 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.fp4_profile_reset.restype = C.c_int
     lib.fp4_profile_read.argtypes = [vp, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     lib.fp4_profile_read.restype = C.c_int
-    lib.fp4_set_gemm_pairs.argtypes = [vp, C.c_int]
-    lib.fp4_set_gemm_pairs.restype = C.c_int
     lib.fp4_set_overlap.argtypes = [vp, C.c_int]
     lib.fp4_set_quantile_mode.argtypes = [vp, C.c_int]
     lib.fp4_set_quantile_mode.restype = C.c_int
@@ -178,9 +176,6 @@ class Context:
 
     def set_overlap(self, on: bool = True):
         _check(self.lib.fp4_set_overlap(self.handle, int(on)))
-
-    def set_gemm_pairs(self, on: bool = True):
-        _check(self.lib.fp4_set_gemm_pairs(self.handle, int(on)))
 
     def set_quantile_mode(self, mode: int):
         """FP4_QUANTILE_SIGNED (the paper's clamp, default), FP4_QUANTILE_ABS (one threshold on |x|) or

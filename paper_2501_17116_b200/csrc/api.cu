@@ -94,7 +94,6 @@ int fp4_create(fp4_ctx** out, int device, size_t workspace_bytes) {
   ctx->occ_hist = nullptr;
   ctx->profile = 0;
   ctx->overlap = 1;
-  ctx->gemm_pairs = 0;
   ctx->launch_count = 0;
   ctx->records = new (std::nothrow) std::vector<ProfRecord>();
   for (auto& s : ctx->side) s = nullptr;
@@ -275,7 +274,7 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
   char* scratch_w = reuse_w ? nullptr : arena.take<char>(quantize_scratch_bytes(K, N));
   // A heavy residual (the caller's capacity says it may hold at least 1 % of the activation, alpha <=
   // 0.995) sends its hot columns through the GEMM as a dense tail instead of per-entry gathers.
-  const bool tail_on = occ && !ctx->gemm_pairs && savedA->csr_rowptr && savedA->csc_colptr &&
+  const bool tail_on = occ && savedA->csr_rowptr && savedA->csc_colptr &&
                        savedA->sparse_cap * 100 >= M * K;
   char* scratch_tail = tail_on ? arena.take<char>(fwd_tail_scratch_bytes(M, K, N)) : nullptr;
   if (!arena.ok) return FP4_ERR_WORKSPACE;
@@ -454,8 +453,7 @@ int linear_bwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* dY_b
   Fp4GemmDesc dgrad = {g1_codes, savedW->codes, M, K, N, g1_amax, nullptr, dA, out_f32, nullptr};
   dgrad.a_format = dy8;
   dgrad.b_format = w8;
-  const bool pairs = gemm_kind == FP4_GEMM_MXF4 && ctx->gemm_pairs;
-  if (dA && dW && !pairs) {
+  if (dA && dW) {
     // Both GEMMs in one launch on the caller's stream, the weight gradient's tiles first (their
     // epilogue is the longer one and then runs under the other GEMM's MMAs).
     if (sw != st) {
@@ -645,12 +643,6 @@ int fp4_set_quantile_mode(fp4_ctx* ctx, int mode) {
   if (!ctx) return FP4_ERR_NULL;
   if (mode != FP4_QUANTILE_SIGNED && mode != FP4_QUANTILE_ABS && mode != FP4_QUANTILE_TOKEN) return FP4_ERR_ARG;
   ctx->quantile_mode = mode;
-  return FP4_OK;
-}
-
-int fp4_set_gemm_pairs(fp4_ctx* ctx, int on) {
-  if (!ctx) return FP4_ERR_NULL;
-  ctx->gemm_pairs = on ? 1 : 0;
   return FP4_OK;
 }
 

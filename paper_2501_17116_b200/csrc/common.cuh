@@ -52,7 +52,6 @@ struct fp4_ctx {
   int      host_step_parity;         // set of the next pipelined call
   int      quantile_mode;            // FP4_QUANTILE_SIGNED (the paper's clamp) or FP4_QUANTILE_ABS
   int      overlap;            // run independent kernel chains on the side streams (default on)
-  int      gemm_pairs;         // MXF4 GEMM on pairs of CTAs (tcgen05 cta_group::2)
   int      profile;            // record CUDA events around every kernel class
   long long launch_count;      // kernels enqueued since the last reset
   std::vector<ProfRecord>* records;
@@ -181,7 +180,7 @@ struct Fp4GemmDesc {
   int a_format = FP4_FORMAT_E2M1;   // operand formats: E2M1 nibbles, or E4M3 / E5M2 bytes (byte-container kind only)
   int b_format = FP4_FORMAT_E2M1;
 };
-// Both GEMMs in one launch; the tiles of `first` are computed first.  Not available on CTA pairs.
+// Both GEMMs in one launch; the tiles of `first` are computed first.
 int launch_gemm_fp4_two(fp4_ctx* ctx, cudaStream_t stream, const Fp4GemmDesc& first, const Fp4GemmDesc& second,
                         int gemm_kind, int32_t* status);
 

@@ -554,264 +554,6 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   }
 }
 
-// ----------------------------------------------------------------------------------------------
-// Two-CTA flavour (MXF4 only): a cluster of two CTAs computes a 256 x 240 tile with
-// tcgen05.mma.cta_group::2.  Each CTA loads its own 128 rows of A and one half (120 rows) of the B
-// tile, so the operand traffic from L2 per flop drops by a third; each CTA holds the accumulators
-// of its own 128 rows.  The even CTA of the pair issues the MMAs; both CTAs' copies complete on
-// its `full` barrier, its commits release the stages and publish the tiles in both CTAs, and both
-// epilogues report back to its `acc_empty` barrier.  No copy is multicast.
-constexpr int PAIR_STAGES = 6;
-constexpr int PAIR_BN = 240;
-constexpr int PAIR_B_STAGE_BYTES = (PAIR_BN / 2) * 128;
-constexpr int PAIR_STAGE_BYTES = A_STAGE_BYTES + PAIR_B_STAGE_BYTES;
-constexpr uint32_t PEER_BIT_MASK = 0xFEFFFFFFu;     // clears the CTA-rank bit of a shared::cluster address
-constexpr size_t pair_smem_bytes() {
-  return 1024 + size_t(PAIR_STAGES) * PAIR_STAGE_BYTES + 256 + 2 * 256 * 4 + STAGE_OUT_BYTES + 2 * 256 * 4;
-}
-__host__ __device__ constexpr uint32_t idesc_mxf4_pair() {
-  return (1u << 7) | (1u << 10) | (uint32_t(PAIR_BN >> 3) << 17) | (1u << 23) | (uint32_t(256 >> 4) << 24);
-}
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// Both CTAs issue their copies; the transaction bytes land on the even CTA's barrier.
-__device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar) & PEER_BIT_MASK), "r"(c0), "r"(c1)
-      : "memory");
-}
-__device__ __forceinline__ void mma_mxf4_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                              uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %6, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%4], [%5], p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate)
-      : "memory");
-}
-// Arrive on the barrier at this shared-memory offset in both CTAs of the pair once the MMAs retire.
-__device__ __forceinline__ void tc_commit_pair_both(uint64_t* bar) {
-  asm volatile(
-      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-      ::"r"(smem_u32(bar)), "h"(uint16_t(3))
-      : "memory");
-}
-__device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-               : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_even_cta(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(smem_u32(bar) & PEER_BIT_MASK) : "memory");
-}
-
-template <int EPI>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(num_threads(EPI), 1)
-gemm_fp4_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                      const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_out_aux,
-                     const GemmArgs args) {
-  constexpr int NACC = 2;
-  constexpr int BN = PAIR_BN;
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* smem_a = smem;
-  uint8_t* smem_b = smem + PAIR_STAGES * A_STAGE_BYTES;
-  uint8_t* s_out = smem + PAIR_STAGES * PAIR_STAGE_BYTES;
-  uint8_t* smem_misc = s_out + STAGE_OUT_BYTES;
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_misc);
-  uint64_t* empty_bar = full_bar + PAIR_STAGES;
-  uint64_t* acc_full = empty_bar + PAIR_STAGES;
-  uint64_t* acc_empty = acc_full + 2;
-  uint64_t* final_bar = acc_empty + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(final_bar + 1);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* s_dcol = reinterpret_cast<float*>(smem_misc + 256);
-  float* s_gcol = s_dcol + 2 * 256;
-
-  const int warp = threadIdx.x >> 5;
-  const int lane = threadIdx.x & 31;
-  const uint32_t rank = cluster_ctarank();          // 0: issues the MMAs
-  const int pair = blockIdx.x >> 1;
-  const int num_pairs = gridDim.x >> 1;
-  const int num_tiles = args.num_m_blocks * args.num_n_blocks;     // num_m_blocks counts 256-row blocks here
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < PAIR_STAGES; ++s) {
-      mbar_init(&full_bar[s], 1);
-      mbar_init(&empty_bar[s], 1);
-    }
-    for (int a = 0; a < 2; ++a) {
-      mbar_init(&acc_full[a], 1);
-      mbar_init(&acc_empty[a], 2 * epi_warps(EPI));      // the epilogue warps of both CTAs
-    }
-    mbar_init(final_bar, 1);
-    *abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_out) : "memory");
-  }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"(TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-  }
-  tc_fence_before();
-  __syncthreads();
-  cluster_sync_all();                               // the peer's barriers exist before anything targets them
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-
-  if (warp >= 2 && warp < 6) {                      // unit block scales in this CTA's tensor memory
-    const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
-    for (int c = 0; c < 16; c += 8) tmem_st_32x8(tmem_base + lane_base + SF_COL_B + c, 0x7F7F7F7Fu);
-    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-  }
-  tc_fence_before();
-  __syncthreads();
-  cluster_sync_all();                               // both CTAs' scales are in place before the first MMA
-  tc_fence_after();
-
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer (both CTAs)
-    if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      bool ok = true;
-      for (int t = pair; t < num_tiles && ok; t += num_pairs) {
-        const int m_blk = t % args.num_m_blocks;
-        const int n_blk = t / args.num_m_blocks;
-        for (int kb = 0; kb < args.num_k_blocks; ++kb) {
-          ok = mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, args.status);
-          if (!ok) break;
-          if (rank == 0) mbar_arrive_expect_tx(&full_bar[stage], 2u * PAIR_STAGE_BYTES);
-          tma_load_2d_pair(smem_a + stage * A_STAGE_BYTES, &map_a, &full_bar[stage], kb * 128,
-                           m_blk * 256 + int(rank) * BM);
-          tma_load_2d_pair(smem_b + stage * PAIR_B_STAGE_BYTES, &map_b, &full_bar[stage], kb * 128,
-                           n_blk * BN + int(rank) * (BN / 2));
-          if (++stage == PAIR_STAGES) { stage = 0; phase ^= 1u; }
-        }
-      }
-      if (!ok) {
-        // Gave up: give the copies already in flight (they signal the even CTA) time to land.
-        const uint64_t t0 = global_timer_ns();
-        while (global_timer_ns() - t0 < 200000ull) {}
-      }
-    }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer (even CTA)
-    if (lane == 0 && rank == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      int acc = 0;
-      uint32_t acc_phase = 0;
-      bool ok = true;
-      const uint32_t idesc = idesc_mxf4_pair();
-      for (int t = pair; t < num_tiles && ok; t += num_pairs) {
-        ok = mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, args.status);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t d_tmem = tmem_base + uint32_t(acc * ACC_STRIDE);
-        for (int kb = 0; kb < args.num_k_blocks; ++kb) {
-          ok = mbar_wait(&full_bar[stage], phase, abort_flag, args.status);
-          if (!ok) break;
-          tc_fence_after();
-          const uint64_t a_desc = make_smem_desc(smem_u32(smem_a + stage * A_STAGE_BYTES));
-          const uint64_t b_desc = make_smem_desc(smem_u32(smem_b + stage * PAIR_B_STAGE_BYTES));
-#pragma unroll
-          for (int k = 0; k < 4; ++k)
-            mma_mxf4_pair(d_tmem, a_desc + uint64_t(2 * k), b_desc + uint64_t(2 * k), idesc, tmem_base + SF_COL_A,
-                          tmem_base + SF_COL_B, (kb | k) != 0 ? 1u : 0u);
-          tc_commit_pair_both(&empty_bar[stage]);   // frees the stage in both CTAs
-          if (++stage == PAIR_STAGES) { stage = 0; phase ^= 1u; }
-        }
-        if (!ok) break;
-        tc_commit_pair_both(&acc_full[acc]);        // the tile is complete in both CTAs
-        if (++acc == NACC) { acc = 0; acc_phase ^= 1u; }
-      }
-      // All MMAs must have retired before either CTA frees tensor memory or leaves.
-      tc_commit_pair(final_bar);
-      const uint64_t t0 = global_timer_ns();
-      while (!mbar_try_wait(final_bar, 0)) {
-        if (global_timer_ns() - t0 > WAIT_LIMIT_NS) {
-          atomicOr(args.status, FP4_DEV_TIMEOUT);
-          break;
-        }
-      }
-    }
-  } else {
-    // ------------------------------------------------------------------ epilogue (both CTAs)
-    constexpr int EW = epi_warps(EPI);
-    constexpr int G = EW / 4;
-    const int quarter = warp & 3;
-    const int group = (warp - 2) >> 2;
-    const int et = threadIdx.x - 64;
-    uint8_t* stage = s_out + (warp - 2) * (STAGE_OUT_BYTES / EW);
-    int acc = 0;
-    uint32_t acc_phase = 0;
-    uint32_t tile_parity = 0;
-    uint32_t store_seq = 0;
-    const OutMaps out_maps = {&map_out, &map_out_aux};
-    for (int t = pair; t < num_tiles; t += num_pairs) {
-      const int m_blk = t % args.num_m_blocks;
-      const int n_blk = t / args.num_m_blocks;
-      const int row_blk = 2 * m_blk + int(rank);                   // this CTA's 128-row block
-      const bool rows_valid = row_blk * BM < args.I;               // odd number of 128-row blocks: last one is empty
-      const int row = row_blk * BM + quarter * 32 + lane;
-      const float d_row = (args.row_amax && rows_valid) ? __fdiv_rn(__ldg(&args.row_amax[row]), 6.0f) : 1.0f;
-      float* dcol = s_dcol + tile_parity * 256;
-      float* gcol = s_gcol + tile_parity * 256;
-      for (int c = et; c < BN; c += 32 * EW) {
-        const int col = n_blk * BN + c;
-        dcol[c] = (args.col_amax && col < args.J) ? __fdiv_rn(__ldg(&args.col_amax[col]), 6.0f) : 1.0f;
-        if (EPI == EPI_WGRAD && args.w) {
-          const float am = col < args.J ? __ldg(&args.w_amax[col]) : 0.0f;
-          gcol[c] = am > 0.0f ? __fdiv_rn(6.0f, am) : 0.0f;
-        }
-      }
-      int slot = -1;
-      WgradOperands op;
-      if (EPI == EPI_WGRAD && rows_valid) {
-        if (args.slot_of_row) slot = __ldg(&args.slot_of_row[row]);
-        if (n_blk * BN + 16 * group < args.J) wgrad_fetch(op, args, row, slot, n_blk * BN + 16 * group);
-      }
-      const bool ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, args.status);
-      if (epilogue_bar_any(!ok, 32 * EW)) break;
-      tc_fence_after();
-      const uint32_t t_base = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * ACC_STRIDE);
-      if (rows_valid) {
-        if (EPI == EPI_WGRAD)
-          epilogue_tile_wgrad<BN, G>(args, row_blk, n_blk, t_base, d_row, dcol, gcol, slot, stage, quarter, group, lane,
-                                     out_maps, store_seq, op);
-        else
-          epilogue_tile_plain<BN, G>(args, row_blk, n_blk, t_base, d_row, dcol, stage, quarter, group, lane, out_maps,
-                                     store_seq);
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_even_cta(&acc_empty[acc]);
-      if (++acc == NACC) { acc = 0; acc_phase ^= 1u; }
-      tile_parity ^= 1u;
-    }
-    if (lane == 0) tma_store_wait_all();
-  }
-
-  tc_fence_before();
-  __syncthreads();
-  cluster_sync_all();                               // neither CTA leaves while the other may still touch it
-  if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
-  }
-}
-
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -886,16 +628,6 @@ int make_out_maps(fp4_ctx* ctx, CUtensorMap* unit, CUtensorMap* aux, void* out, 
   return r == CUDA_SUCCESS ? FP4_OK : FP4_ERR_CUDA;
 }
 
-template <int EPI>
-int launch_pair_kernel(int pairs, cudaStream_t stream, const CUtensorMap& map_a, const CUtensorMap& map_b,
-                       const CUtensorMap& map_out, const CUtensorMap& map_out_aux, const GemmArgs& args) {
-  constexpr size_t kSmem = pair_smem_bytes();
-  FP4_CUDA_TRY(cudaFuncSetAttribute(gemm_fp4_pair_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    int(kSmem)));
-  gemm_fp4_pair_kernel<EPI><<<2 * pairs, num_threads(EPI), kSmem, stream>>>(map_a, map_b, map_out, map_out_aux, args);
-  return FP4_OK;
-}
-
 struct Problem {
   CUtensorMap map_a, map_b, map_out, map_out_aux;
   GemmArgs args;
@@ -917,7 +649,7 @@ int launch_kernel(int grid, cudaStream_t stream, const Problem& p, const Problem
 }
 
 // Tensor maps and arguments of one GEMM.
-int make_problem(fp4_ctx* ctx, Problem* p, const Fp4GemmDesc& d, int gemm_kind, bool pair_mode, int32_t* status) {
+int make_problem(fp4_ctx* ctx, Problem* p, const Fp4GemmDesc& d, int gemm_kind, int32_t* status) {
   if (gemm_kind != FP4_GEMM_MXF4 && gemm_kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;
   const bool a8 = d.a_format != FP4_FORMAT_E2M1, b8 = d.b_format != FP4_FORMAT_E2M1;   // FP8 bytes
   if ((a8 || b8) && gemm_kind != FP4_GEMM_F8F6F4) return FP4_ERR_ARG;   // FP8 operands need the byte-container kind
@@ -929,7 +661,7 @@ int make_problem(fp4_ctx* ctx, Problem* p, const Fp4GemmDesc& d, int gemm_kind, 
   int rc = make_codes_map(ctx, &p->map_a, d.a_codes, d.I, d.C, BM, gemm_kind, a8);
   if (rc != FP4_OK) return rc;
   const int BN = tile_n(gemm_kind);
-  rc = make_codes_map(ctx, &p->map_b, d.b_codes, d.J, d.C, pair_mode ? PAIR_BN / 2 : BN, gemm_kind, b8);
+  rc = make_codes_map(ctx, &p->map_b, d.b_codes, d.J, d.C, BN, gemm_kind, b8);
   if (rc != FP4_OK) return rc;
   if (reinterpret_cast<uintptr_t>(d.out) & 15) return FP4_ERR_ALIGN;
   rc = make_out_maps(ctx, &p->map_out, &p->map_out_aux, d.out, d.I, d.J, d.out_f32);
@@ -940,7 +672,7 @@ int make_problem(fp4_ctx* ctx, Problem* p, const Fp4GemmDesc& d, int gemm_kind, 
   args.J = int(d.J);
   const int k_per_stage = gemm_kind == FP4_GEMM_F8F6F4 ? 128 : 256;   // elements per 128-byte row
   args.num_k_blocks = int((d.C + k_per_stage - 1) / k_per_stage);
-  args.num_m_blocks = pair_mode ? int((d.I + 255) / 256) : int(d.I / BM);
+  args.num_m_blocks = int(d.I / BM);
   args.num_n_blocks = int((d.J + BN - 1) / BN);
   // The transaction count of a copy is in bytes read from global memory: the byte-container form
   // fills a stage's 128-byte rows from 64 bytes of packed nibbles (E2M1) or from 128 bytes (E4M3).
@@ -981,14 +713,12 @@ int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, c
   Fp4GemmDesc d = {a_codes, b_codes, I, J, C, row_amax, col_amax, out, out_f32, epi};
   d.a_format = a_format;
   d.b_format = b_format;
-  const bool pair_mode = gemm_kind == FP4_GEMM_MXF4 && ctx->gemm_pairs;
   Problem p;
-  int rc = make_problem(ctx, &p, d, gemm_kind, pair_mode, status);
+  int rc = make_problem(ctx, &p, d, gemm_kind, status);
   if (rc != FP4_OK) return rc;
   // The dense tail's operands travel in the slots of a second problem that has no tiles.
   Problem with_tail;
   if (tail) {
-    if (pair_mode) return FP4_ERR_ARG;
     with_tail = p;
     with_tail.args.num_m_blocks = with_tail.args.num_n_blocks = 0;
     rc = make_tail_map(ctx, &with_tail.map_a, tail->a, I, BM);
@@ -1003,12 +733,7 @@ int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, c
   const int grid = tiles < ctx->num_sms ? tiles : ctx->num_sms;
   KernelScope scope(ctx, stream, KC_GEMM, 1);
   int rc2;
-  if (pair_mode) {
-    const int max_pairs = ctx->num_sms / 2;
-    const int pairs = tiles < max_pairs ? tiles : max_pairs;
-    rc2 = p.fused ? launch_pair_kernel<EPI_WGRAD>(pairs, stream, p.map_a, p.map_b, p.map_out, p.map_out_aux, args)
-                  : launch_pair_kernel<EPI_PLAIN>(pairs, stream, p.map_a, p.map_b, p.map_out, p.map_out_aux, args);
-  } else if (gemm_kind == FP4_GEMM_F8F6F4)
+  if (gemm_kind == FP4_GEMM_F8F6F4)
     rc2 = p.fused ? launch_kernel<FP4_GEMM_F8F6F4, EPI_WGRAD>(grid, stream, p, second)
                   : launch_kernel<FP4_GEMM_F8F6F4, EPI_PLAIN>(grid, stream, p, second);
   else
@@ -1019,15 +744,14 @@ int launch_gemm_fp4(fp4_ctx* ctx, cudaStream_t stream, const uint8_t* a_codes, c
   return FP4_OK;
 }
 
-// Two GEMMs in one launch (single-CTA kernels only): the tiles of `first` are computed first.  Both
+// Two GEMMs in one launch: the tiles of `first` are computed first.  Both
 // run through the 16-warp epilogue; a problem without fused work simply has nothing to add.
 int launch_gemm_fp4_two(fp4_ctx* ctx, cudaStream_t stream, const Fp4GemmDesc& first, const Fp4GemmDesc& second,
                         int gemm_kind, int32_t* status) {
-  if (gemm_kind == FP4_GEMM_MXF4 && ctx->gemm_pairs) return FP4_ERR_ARG;
   Problem p, q;
-  int rc = make_problem(ctx, &p, first, gemm_kind, false, status);
+  int rc = make_problem(ctx, &p, first, gemm_kind, status);
   if (rc != FP4_OK) return rc;
-  rc = make_problem(ctx, &q, second, gemm_kind, false, status);
+  rc = make_problem(ctx, &q, second, gemm_kind, status);
   if (rc != FP4_OK) return rc;
   const int tiles = p.args.num_m_blocks * p.args.num_n_blocks + q.args.num_m_blocks * q.args.num_n_blocks;
   const int grid = tiles < ctx->num_sms ? tiles : ctx->num_sms;

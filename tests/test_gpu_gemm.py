@@ -8,11 +8,9 @@ from oracle import fp4_oracle as O
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(scope="module", params=["one_cta", "cta_pairs"])
-def ctx(lib, request):
-    """Every GEMM test runs on single CTAs and on CTA pairs (the MXF4 flavour has both forms)."""
+@pytest.fixture(scope="module")
+def ctx(lib):
     c = lib.Context(0, 64 << 20)
-    c.set_gemm_pairs(request.param == "cta_pairs")
     yield c
     c.close()
 

@@ -5,7 +5,7 @@ activation distributions, number of outlier channels, GEMM kind and DGE setting.
 what the fixed cases check: saved operands bit for bit, the three outputs within the bar stated in
 test_gpu_linear.py.  The draws are fixed by the seed, so a failure reproduces; FP4_RANDOM_DRAWS in
 the environment sets how many are made (default 16); FP4_TEST_NO_OVERLAP=1 runs them with the
-library's side streams switched off, FP4_TEST_GEMM_PAIRS=1 with the two-CTA GEMM flavour.
+library's side streams switched off.
 """
 import os
 
@@ -25,8 +25,6 @@ def ctx(lib):
     c = lib.Context(0, 1 << 30)
     if os.environ.get("FP4_TEST_NO_OVERLAP"):          # the same draws with every kernel on one stream
         c.set_overlap(False)
-    if os.environ.get("FP4_TEST_GEMM_PAIRS"):          # ... with the MXF4 GEMMs on CTA pairs
-        c.set_gemm_pairs(True)
     yield c
     c.close()
 
