@@ -12,7 +12,8 @@
  * ---------------------------------------
  *  - Every tensor pointer is a DEVICE pointer unless the parameter is documented as host.
  *    Tensors are dense, row-major and 16-byte aligned.  The caller owns every tensor; the
- *    context owns only its workspace.  Nothing is allocated after fp4_create().
+ *    context owns only its workspace.  Nothing is allocated after fp4_create() (outside profiling
+ *    mode, fp4_profile_enable, which creates a pair of CUDA events per kernel class and call).
  *  - Notation: A[M x K] activations, W[K x N] weights (input channels x output channels),
  *    Y[M x N] = A W.  M, K and N must be multiples of 128.
  *  - E2M1 codes are sign-magnitude nibbles (bit 3 sign; 0..7 -> 0, .5, 1, 1.5, 2, 3, 4, 6),
@@ -46,19 +47,20 @@ extern "C" {
 #define FP4_ERR_WORKSPACE  (-5)   /* the context's workspace is too small for this call      */
 #define FP4_ERR_CUDA       (-6)   /* a CUDA runtime / driver call failed                     */
 #define FP4_ERR_ARG        (-7)   /* an argument has an unsupported value                    */
-#define FP4_ERR_CAPACITY   (-8)   /* sparse_cap is below the guaranteed bound 2 * n_tail     */
+#define FP4_ERR_CAPACITY   (-8)   /* sparse_cap is below fp4_sparse_capacity()               */
 #define FP4_ERR_STATIC_LIMIT (-9) /* input larger than the fixed scratch of a *_static call  */
 
-/* bits of the device status word */
-#define FP4_DEV_SPARSE_OVERFLOW  1   /* more residual entries than sparse_cap                */
+/* bits of the device status word (bit 0 is not used: the residual cannot outgrow a capacity the
+ * host has accepted, see fp4_sparse_capacity) */
 #define FP4_DEV_NONFINITE        2   /* an input holds an infinity or a NaN: outputs unspecified */
 #define FP4_DEV_TIMEOUT          4   /* a bounded wait inside a kernel ran out               */
 
-/* gemm_kind: which tcgen05.mma flavour multiplies the E2M1 codes */
+/* fp4_qtensor.format: how a quantised operand is stored */
 #define FP4_FORMAT_E2M1  0
 #define FP4_FORMAT_E4M3  1
 #define FP4_FORMAT_E5M2  2
 
+/* gemm_kind: which tcgen05.mma flavour multiplies the codes */
 #define FP4_GEMM_MXF4    0   /* packed nibbles, K = 64 per instruction, unit block scales    */
 #define FP4_GEMM_F8F6F4  1   /* nibbles in byte containers, K = 32 per instruction           */
 /* fp4_gemm only: the byte-container kind with E4M3 bytes as one or both operands */
@@ -93,8 +95,8 @@ typedef struct fp4_qtensor {
   int32_t* csc_colptr;     /* [cols + 1]                                                      */
   int32_t* csc_row;        /* [sparse_cap] row index, ascending within a column               */
   float*   csc_val;        /* [sparse_cap]                                                    */
-  int64_t  sparse_cap;     /* capacity in entries; 2 * round((1-alpha) * rows * cols) always
-                              suffices                                                        */
+  int64_t  sparse_cap;     /* capacity in entries: at least fp4_sparse_capacity(rows, cols, alpha,
+                              mode), i.e. 2 * round((1-alpha) * rows * cols) for the paper's clamp */
   int32_t* nnz;            /* [1] number of residual entries                                  */
   int32_t  format;         /* set by the caller: FP4_FORMAT_E2M1 (0, as described above) or
                               FP4_FORMAT_E4M3: OCP E4M3 bytes, one per element (codes
@@ -113,6 +115,13 @@ int fp4_destroy(fp4_ctx* ctx);
 
 /* Workspace that fp4_quantize / fp4_linear_fwd / fp4_linear_bwd need for these sizes.      */
 size_t fp4_workspace_bytes(int64_t M, int64_t K, int64_t N);
+
+/* Residual entries that clamping at `alpha` can produce at most (Section 3.2: two tails of
+ * n_tail = llround((1 - alpha) * rows * cols) entries; with FP4_QUANTILE_TOKEN two tails of
+ * llround((1 - alpha) * cols) entries in every row): the least `sparse_cap` the calls accept.
+ * 0 for alpha == 1; -1 for arguments outside their range.  `quantile_mode` is one of the
+ * FP4_QUANTILE_* values below.                                                              */
+int64_t fp4_sparse_capacity(int64_t rows, int64_t cols, double alpha, int quantile_mode);
 
 /* Text of a host return code (static string).                                              */
 const char* fp4_status_string(int code);
@@ -271,6 +280,15 @@ int fp4_set_overlap(fp4_ctx* ctx, int on);
 #define FP4_QUANTILE_ABS    1
 #define FP4_QUANTILE_TOKEN  2
 int fp4_set_quantile_mode(fp4_ctx* ctx, int mode);
+/* Failure-path testing (no counterpart in the paper).  FP4_DEBUG_WAIT_LIMIT_US: the limit, in
+ * microseconds, of every device-side wait of the GEMM kernels this context launches from now on
+ * (0 restores the default of 2 s).  FP4_DEBUG_SKIP_FILL: the producer of the GEMM's first CTA leaves
+ * out its fill number `value` of the shared-memory ring (no copy, no arrival; -1: none), so that
+ * the consumer's wait runs out: the kernel raises FP4_DEV_TIMEOUT, frees its tensor memory and
+ * returns; the context stays usable.                                                        */
+#define FP4_DEBUG_WAIT_LIMIT_US 1
+#define FP4_DEBUG_SKIP_FILL     2
+int fp4_debug_set(fp4_ctx* ctx, int key, int64_t value);
 int fp4_profile_reset(fp4_ctx* ctx);
 int fp4_profile_read(fp4_ctx* ctx, int kernel_class, double* total_ms, int64_t* launches);
 int64_t fp4_launch_count(fp4_ctx* ctx);
@@ -293,9 +311,11 @@ int64_t fp4_launch_count(fp4_ctx* ctx);
  *               is enqueued
  *   alpha       0.5 < alpha < 1
  *   thresholds  device float[2]: receives {lo, hi}, bit-identical to what fp4_quantize writes
+ * A NaN or an infinity in the input is not reported (the call has no status word): the thresholds
+ * are then unspecified.
  * The work is enqueued on `stream` for the current device.  The first call on each device also
- * looks up the device address of the scratch array and sets a kernel attribute; make that first
- * call before any stream capture begins.  All calls on a device share the one scratch array
+ * looks up the device address of the scratch array and sets a kernel attribute (once per device,
+ * safe to race between host threads); make that first call before any stream capture begins.  All calls on a device share the one scratch array
  * (it is cleared at the start of each call): two calls whose work overlaps on the GPU -- issued
  * to different streams without ordering between them -- race and give wrong thresholds.
  */

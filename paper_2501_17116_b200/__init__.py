@@ -6,7 +6,7 @@ seeded workload generators stay usable on a machine without CUDA; every compute
 entry point loads it on first use and raises if it has not been built.
 """
 from .binding import (  # noqa: F401
-    FP4_DEV_NONFINITE, FP4_DEV_SPARSE_OVERFLOW, FP4_DEV_TIMEOUT, FP4_GEMM_F8F6F4, FP4_GEMM_F8F6F4_A8, FP4_GEMM_F8F6F4_A8B8, FP4_GEMM_F8F6F4_B8, FP4_GEMM_MXF4,
+    FP4_DEV_NONFINITE, FP4_DEV_TIMEOUT, FP4_GEMM_F8F6F4, FP4_GEMM_F8F6F4_A8, FP4_GEMM_F8F6F4_A8B8, FP4_GEMM_F8F6F4_B8, FP4_GEMM_MXF4,
     FP4_BWD_DY_E4M3, FP4_BWD_DY_E5M2, FP4_FORMAT_E2M1, FP4_FORMAT_E4M3, FP4_FORMAT_E5M2, FP4_GEMM_A_E5M2, FP4_GEMM_B_E5M2, FP4_QUANTILE_ABS, FP4_QUANTILE_SIGNED, FP4_QUANTILE_TOKEN, EXPORTS,
     Context, Fp4Error, QTensor, fp4_gemm, fp4_linear_bwd, fp4_linear_fwd, fp4_linear_step_host, fp4_quantile_thresholds_static, fp4_quantize, load_library,
     tail_capacity, KERNEL_CLASSES,

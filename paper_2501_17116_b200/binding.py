@@ -25,19 +25,20 @@ FP4_BWD_DY_E5M2 = 0x200
 FP4_FORMAT_E2M1 = 0
 FP4_FORMAT_E4M3 = 1
 FP4_FORMAT_E5M2 = 2
-FP4_DEV_SPARSE_OVERFLOW = 1
 FP4_DEV_NONFINITE = 2
 FP4_DEV_TIMEOUT = 4
 
 EXPORTS = ("fp4_create", "fp4_destroy", "fp4_workspace_bytes", "fp4_status_string", "fp4_quantize",
            "fp4_gemm", "fp4_linear_fwd", "fp4_linear_bwd", "fp4_step_host_workspace_bytes",
            "fp4_linear_step_host", "fp4_profile_enable", "fp4_profile_reset", "fp4_profile_read",
-           "fp4_launch_count", "fp4_quantile_thresholds_static", "fp4_set_overlap",
+           "fp4_launch_count", "fp4_quantile_thresholds_static", "fp4_set_overlap", "fp4_debug_set", "fp4_sparse_capacity",
            "fp4_set_quantile_mode")
 FP4_STATIC_MAX_ROWS = 65536
 FP4_QUANTILE_SIGNED = 0
 FP4_QUANTILE_ABS = 1
 FP4_QUANTILE_TOKEN = 2
+FP4_DEBUG_WAIT_LIMIT_US = 1
+FP4_DEBUG_SKIP_FILL = 2
 KERNEL_CLASSES = ("gemm", "select", "encode", "absmax", "sparse", "comp_fwd", "comp_wgrad_dge")
 
 
@@ -95,6 +96,10 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.fp4_profile_reset.restype = C.c_int
     lib.fp4_profile_read.argtypes = [vp, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     lib.fp4_profile_read.restype = C.c_int
+    lib.fp4_debug_set.argtypes = [vp, C.c_int, i64]
+    lib.fp4_debug_set.restype = C.c_int
+    lib.fp4_sparse_capacity.argtypes = [i64, i64, C.c_double, C.c_int]
+    lib.fp4_sparse_capacity.restype = C.c_int64
     lib.fp4_set_overlap.argtypes = [vp, C.c_int]
     lib.fp4_set_quantile_mode.argtypes = [vp, C.c_int]
     lib.fp4_set_quantile_mode.restype = C.c_int
@@ -182,6 +187,10 @@ class Context:
         FP4_QUANTILE_TOKEN (signed thresholds per token)."""
         _check(self.lib.fp4_set_quantile_mode(self.handle, int(mode)))
 
+    def debug_set(self, key: int, value: int):
+        """Failure-path testing: FP4_DEBUG_WAIT_LIMIT_US / FP4_DEBUG_SKIP_FILL (fp4_debug_set)."""
+        _check(self.lib.fp4_debug_set(self.handle, int(key), int(value)))
+
     def launch_count(self) -> int:
         return int(self.lib.fp4_launch_count(self.handle))
 
@@ -220,13 +229,12 @@ class QTensor:
 
 
 def tail_capacity(rows: int, cols: int, alpha: float) -> int:
-    """The guaranteed bound on the number of residual entries, whichever form of the clamp is set:
-    2 * n_tail of the tensor, or rows * 2 * n_tail of a row for thresholds per token."""
-    if alpha >= 1.0:
-        return 0
-    import math
-    return max(2 * int(math.floor((1.0 - alpha) * rows * cols + 0.5)),
-               2 * rows * int(math.floor((1.0 - alpha) * cols + 0.5)))
+    """A `sparse_cap` that suffices whichever form of the clamp is set on the context: the larger of
+    fp4_sparse_capacity for the tensor-wide clamp and for thresholds per token."""
+    lib = load_library()
+    caps = [int(lib.fp4_sparse_capacity(rows, cols, float(alpha), m)) for m in (FP4_QUANTILE_SIGNED, FP4_QUANTILE_TOKEN)]
+    assert min(caps) >= 0, "rows, cols or alpha outside their range"
+    return max(caps)
 
 
 def fp4_quantize(ctx: Context, x: torch.Tensor, scale_axis: int, alpha: float = 1.0, prescale=None,

@@ -66,7 +66,7 @@ const char* fp4_status_string(int code) {
     case FP4_ERR_WORKSPACE: return "the context's workspace is too small";
     case FP4_ERR_CUDA: return "a CUDA call failed";
     case FP4_ERR_ARG: return "an argument has an unsupported value";
-    case FP4_ERR_CAPACITY: return "sparse_cap is below 2 * n_tail";
+    case FP4_ERR_CAPACITY: return "sparse_cap is below fp4_sparse_capacity()";
     case FP4_ERR_STATIC_LIMIT: return "input exceeds the fixed scratch of the allocation-free entry point";
     default: return "unknown status";
   }
@@ -93,6 +93,8 @@ int fp4_create(fp4_ctx** out, int device, size_t workspace_bytes) {
   ctx->encode_tiled = nullptr;
   ctx->occ_hist = nullptr;
   ctx->profile = 0;
+  ctx->debug_wait_limit_ns = 0;
+  ctx->debug_skip_fill = -1;
   ctx->overlap = 1;
   ctx->launch_count = 0;
   ctx->records = new (std::nothrow) std::vector<ProfRecord>();
@@ -644,6 +646,29 @@ int fp4_set_quantile_mode(fp4_ctx* ctx, int mode) {
   if (mode != FP4_QUANTILE_SIGNED && mode != FP4_QUANTILE_ABS && mode != FP4_QUANTILE_TOKEN) return FP4_ERR_ARG;
   ctx->quantile_mode = mode;
   return FP4_OK;
+}
+
+int fp4_debug_set(fp4_ctx* ctx, int key, int64_t value) {
+  if (!ctx) return FP4_ERR_NULL;
+  if (key == FP4_DEBUG_WAIT_LIMIT_US) {
+    if (value < 0 || value > 10000000) return FP4_ERR_ARG;
+    ctx->debug_wait_limit_ns = uint64_t(value) * 1000u;
+  } else if (key == FP4_DEBUG_SKIP_FILL) {
+    if (value < -1 || value > (1 << 30)) return FP4_ERR_ARG;
+    ctx->debug_skip_fill = int(value);
+  } else {
+    return FP4_ERR_ARG;
+  }
+  return FP4_OK;
+}
+
+int64_t fp4_sparse_capacity(int64_t rows, int64_t cols, double alpha, int quantile_mode) {
+  if (rows <= 0 || cols <= 0 || !(alpha > 0.5 && alpha <= 1.0)) return -1;
+  if (quantile_mode != FP4_QUANTILE_SIGNED && quantile_mode != FP4_QUANTILE_ABS && quantile_mode != FP4_QUANTILE_TOKEN)
+    return -1;
+  if (!(alpha < 1.0)) return 0;
+  if (quantile_mode == FP4_QUANTILE_TOKEN) return 2 * rows * llround((1.0 - alpha) * double(cols));
+  return 2 * llround((1.0 - alpha) * double(rows * cols));
 }
 
 int fp4_profile_enable(fp4_ctx* ctx, int on) {

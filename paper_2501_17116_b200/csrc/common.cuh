@@ -52,6 +52,8 @@ struct fp4_ctx {
   int      host_step_parity;         // set of the next pipelined call
   int      quantile_mode;            // FP4_QUANTILE_SIGNED (the paper's clamp) or FP4_QUANTILE_ABS
   int      overlap;            // run independent kernel chains on the side streams (default on)
+  uint64_t debug_wait_limit_ns;  // fp4_debug_set: limit of the GEMM's device-side waits (0: the default, 2 s)
+  int      debug_skip_fill;    // fp4_debug_set: fill of shared memory that CTA 0's producer leaves out (-1: none)
   int      profile;            // record CUDA events around every kernel class
   long long launch_count;      // kernels enqueued since the last reset
   std::vector<ProfRecord>* records;

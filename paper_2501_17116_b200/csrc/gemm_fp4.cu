@@ -77,6 +77,10 @@ struct GemmArgs {
   const int* tail_count;
   uint32_t tail_tx_bytes;
   uint32_t tail_idesc;
+  // failure-path testing (fp4_debug_set): limit of every wait of this launch, and the index of one
+  // fill of shared memory that the producer of CTA 0 leaves out (-1: none)
+  uint64_t wait_limit_ns;
+  int skip_fill;
 };
 
 // Instruction descriptors: M = 128, N = tile_n, both operands K-major, E2M1 x E2M1 -> fp32.
@@ -398,16 +402,18 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         const int m_blk = tt % pa.num_m_blocks;
         const int n_blk = tt / pa.num_m_blocks;
         for (int kb = (t == int(blockIdx.x) ? pre : 0); kb < pa.num_k_blocks; ++kb) {
-          ok = mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, args.status);
+          ok = mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, args.status, args.wait_limit_ns);
           if (!ok) break;
-          mbar_arrive_expect_tx(&full_bar[stage], pa.tx_bytes);
-          tma_load_2d(smem_a + stage * A_STAGE_BYTES, ma, &full_bar[stage], kb * 128, m_blk * BM);
-          tma_load_2d(smem_b + stage * B_STAGE_BYTES, mb, &full_bar[stage], kb * 128, n_blk * BN);
+          if (blockIdx.x != 0 || int(fills) != args.skip_fill) {      // a left-out fill: no copy, no arrival
+            mbar_arrive_expect_tx(&full_bar[stage], pa.tx_bytes);
+            tma_load_2d(smem_a + stage * A_STAGE_BYTES, ma, &full_bar[stage], kb * 128, m_blk * BM);
+            tma_load_2d(smem_b + stage * B_STAGE_BYTES, mb, &full_bar[stage], kb * 128, n_blk * BN);
+          }
           ++fills;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
         for (int kb = 0; kb < tail_kb && ok; ++kb) {      // dense tail: FP16 columns 64 kb .. 64 kb + 63
-          ok = mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, args.status);
+          ok = mbar_wait(&empty_bar[stage], phase ^ 1u, abort_flag, args.status, args.wait_limit_ns);
           if (!ok) break;
           mbar_arrive_expect_tx(&full_bar[stage], args.tail_tx_bytes);
           tma_load_2d(smem_a + stage * A_STAGE_BYTES, &map_a2, &full_bar[stage], kb * 64, m_blk * BM);
@@ -438,14 +444,14 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       bool ok = true;
       const int tail_kb = args.tail_count ? 3 * ((min(*args.tail_count, TAIL_MAX_COLS) + 63) / 64) : 0;
       for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-        ok = mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, args.status);
+        ok = mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, args.status, args.wait_limit_ns);
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + uint32_t(acc * ACC_STRIDE);
         const int num_k_blocks = t >= tiles_first ? args2.num_k_blocks : args.num_k_blocks;
         const uint32_t idesc = t >= tiles_first ? args2.idesc : args.idesc;
         for (int kb = 0; kb < num_k_blocks; ++kb) {
-          ok = mbar_wait(&full_bar[stage], phase, abort_flag, args.status);
+          ok = mbar_wait(&full_bar[stage], phase, abort_flag, args.status, args.wait_limit_ns);
           if (!ok) break;
           tc_fence_after();
           const uint64_t a_desc = make_smem_desc(smem_u32(smem_a + stage * A_STAGE_BYTES));
@@ -465,7 +471,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
         for (int kb = 0; kb < tail_kb && ok; ++kb) {
-          ok = mbar_wait(&full_bar[stage], phase, abort_flag, args.status);
+          ok = mbar_wait(&full_bar[stage], phase, abort_flag, args.status, args.wait_limit_ns);
           if (!ok) break;
           tc_fence_after();
           const uint64_t a_desc = make_smem_desc(smem_u32(smem_a + stage * A_STAGE_BYTES));
@@ -484,7 +490,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       tc_commit(final_bar);
       const uint64_t t0 = global_timer_ns();
       while (!mbar_try_wait(final_bar, 0)) {
-        if (global_timer_ns() - t0 > WAIT_LIMIT_NS) {
+        if (global_timer_ns() - t0 > args.wait_limit_ns) {
           atomicOr(args.status, FP4_DEV_TIMEOUT);
           break;
         }
@@ -528,7 +534,7 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (pa.slot_of_row) slot = __ldg(&pa.slot_of_row[row]);
         if (n_blk * BN + 16 * group < pa.J) wgrad_fetch(op, pa, row, slot, n_blk * BN + 16 * group);
       }
-      const bool ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, args.status);
+      const bool ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, args.status, args.wait_limit_ns);
       if (epilogue_bar_any(!ok, 32 * EW)) break;   // also publishes dcol to the other warps
       tc_fence_after();
       const uint32_t t_base = tmem_base + (uint32_t(quarter * 32) << 16) + uint32_t(acc * ACC_STRIDE);
@@ -698,6 +704,8 @@ int make_problem(fp4_ctx* ctx, Problem* p, const Fp4GemmDesc& d, int gemm_kind, 
   args.inv_k = fused && epi->w_bf16 ? 1.0f / epi->dge_k : 1.0f;
   args.expo = args.inv_k - 1.0f;
   args.clip = fused ? epi->dge_clip : 0.0f;
+  args.wait_limit_ns = ctx->debug_wait_limit_ns ? ctx->debug_wait_limit_ns : WAIT_LIMIT_NS;
+  args.skip_fill = ctx->debug_skip_fill;
   args.tail_count = nullptr;
   args.tail_tx_bytes = uint32_t(A_STAGE_BYTES + b_stage_bytes(gemm_kind));
   args.tail_idesc = idesc_f16(gemm_kind);

@@ -16,6 +16,8 @@
 //     2. encode           one read
 // The "dual" mode serves the backward pass: one read of dY yields the token-wise codes of
 // dY (.) d_W[n] and the channel-wise codes of dY (.) d_A[m].
+#include <mutex>
+
 #include "common.cuh"
 
 namespace {
@@ -917,11 +919,11 @@ encode_fp8_kernel(const EncodeArgs a) {
 // ------------------------------------------------------------------------------------------
 // 4. mask -> CSR / CSC
 // ------------------------------------------------------------------------------------------
-// Exclusive prefix sum of n counts by one block; ptr[n] = total.  Also publishes nnz and raises
-// the overflow flag when the total exceeds the caller's capacity.
+// Exclusive prefix sum of n counts by one block; ptr[n] = total.  Also publishes nnz.  (The total
+// cannot exceed the caller's capacity: the host refuses capacities below 2 n_tail, and at most
+// n_tail entries lie beyond either threshold.  The fill kernels still guard every write.)
 __global__ void __launch_bounds__(1024, 1)
-scan_counts_kernel(const int* __restrict__ cnt, int n, int* __restrict__ ptr, int* nnz_out, long long cap,
-                   int32_t* status) {
+scan_counts_kernel(const int* __restrict__ cnt, int n, int* __restrict__ ptr, int* nnz_out) {
   __shared__ long long warp_tot[32];
   const int t = threadIdx.x;
   const int per = (n + 1023) / 1024;
@@ -937,7 +939,6 @@ scan_counts_kernel(const int* __restrict__ cnt, int n, int* __restrict__ ptr, in
   if (t == 1023) {
     ptr[n] = int(incl);
     if (nnz_out) *nnz_out = int(incl);
-    if (status && incl > cap) atomicOr(status, FP4_DEV_SPARSE_OVERFLOW);
   }
 }
 
@@ -1174,7 +1175,7 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
     const int strips = rows / ENC_TM;
     {
       KernelScope scope(ctx, sp, KC_SPARSE, 2);
-      scan_counts_kernel<<<1, 1024, 0, sp>>>(sc.row_cnt, rows, out->csr_rowptr, out->nnz, out->sparse_cap, status);
+      scan_counts_kernel<<<1, 1024, 0, sp>>>(sc.row_cnt, rows, out->csr_rowptr, out->nnz);
       csr_fill_kernel<<<(rows + 7) / 8, 256, 0, sp>>>(mask32, xb, rows, cols, out->thresholds, per_token, out->csr_rowptr,
                                                       out->sparse_cap, out->csr_col, out->csr_val);
     }
@@ -1182,7 +1183,7 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
     {
       KernelScope scope(ctx, sc2, KC_SPARSE, 3);
       csc_strip_prefix_kernel<<<(cols + 255) / 256, 256, 0, sc2>>>(sc.strip_cnt, cols, strips, sc.strip_off, sc.col_cnt);
-      scan_counts_kernel<<<1, 1024, 0, sc2>>>(sc.col_cnt, cols, out->csc_colptr, nullptr, out->sparse_cap, nullptr);
+      scan_counts_kernel<<<1, 1024, 0, sc2>>>(sc.col_cnt, cols, out->csc_colptr, nullptr);
       const dim3 cgrid((cols / 32 + 7) / 8, strips);
       csc_fill_kernel<<<cgrid, 256, 0, sc2>>>(mask32, xb, rows, cols, out->thresholds, per_token, out->csc_colptr, sc.strip_off,
                                               out->sparse_cap, out->csc_row, out->csc_val);
@@ -1316,9 +1317,10 @@ static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_B
 extern "C" int fp4_quantile_thresholds_static(void* stream, const void* x_bf16, int64_t rows, int64_t cols,
                                               double alpha, float* thresholds) {
   // In host code `g_static_scratch` is only a handle; the device address of this device's copy
-  // is looked up once per device and cached.
+  // is looked up once per device and cached (under a lock: host threads may race to the first call).
   static void* scratch_of_device[STATIC_MAX_DEVICES] = {};
   static int sms_of_device[STATIC_MAX_DEVICES] = {};
+  static std::mutex setup_lock;
   if (!x_bf16 || !thresholds) return FP4_ERR_NULL;
   if (rows <= 0 || cols <= 0 || (rows % 128) || (cols % 128) || rows * cols >= (int64_t(1) << 31))
     return FP4_ERR_SHAPE;
@@ -1332,6 +1334,7 @@ extern "C" int fp4_quantile_thresholds_static(void* stream, const void* x_bf16, 
   int device = -1;
   FP4_CUDA_TRY(cudaGetDevice(&device));
   if (device < 0 || device >= STATIC_MAX_DEVICES) return FP4_ERR_ARG;
+  std::unique_lock<std::mutex> guard(setup_lock);
   if (!scratch_of_device[device]) {
     void* ptr = nullptr;
     FP4_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
@@ -1342,7 +1345,9 @@ extern "C" int fp4_quantile_thresholds_static(void* stream, const void* x_bf16, 
     sms_of_device[device] = sms;
     scratch_of_device[device] = ptr;
   }
+  const int num_sms = sms_of_device[device];
   unsigned char* base = static_cast<unsigned char*>(scratch_of_device[device]);
+  guard.unlock();
   uint32_t* hist = reinterpret_cast<uint32_t*>(base);
   unsigned* ticket = reinterpret_cast<unsigned*>(base + STATIC_HIST_BYTES + 512);   // behind the coarse counters
   int* row_max = reinterpret_cast<int*>(base + STATIC_HIST_BYTES + STATIC_SELECT_BYTES);
@@ -1354,7 +1359,7 @@ extern "C" int fp4_quantile_thresholds_static(void* stream, const void* x_bf16, 
   FP4_CUDA_TRY(cudaMemsetAsync(base, 0, STATIC_HIST_BYTES + STATIC_SELECT_BYTES, st));
   const long long n_vec = n / 8;
   long long blocks = (n_vec + HIST_THREADS - 1) / HIST_THREADS;
-  if (blocks > sms_of_device[device]) blocks = sms_of_device[device];
+  if (blocks > num_sms) blocks = num_sms;
   hist_select_kernel<<<int(blocks), HIST_THREADS, HIST_SMEM_BYTES, st>>>(
       static_cast<const uint4*>(x_bf16), int(rows), int(cols / 8), hist, nullptr, row_max, row_min, nullptr, n, n_tail,
       thresholds, ticket, nullptr, 0);

@@ -183,3 +183,30 @@ def test_gemm_with_e5m2_operands(lib, ctx):
         assert (err <= RTOL * np.abs(want) + 2 * (C // 32) * 2.0 ** -23 * terms).all(), (fa, fb)
     with pytest.raises(lib.Fp4Error):                  # the E5M2 flag qualifies an 8-bit operand
         lib.fp4_gemm(ctx, ca, cb, None, None, gemm_kind=lib.FP4_GEMM_F8F6F4 | lib.FP4_GEMM_A_E5M2)
+
+
+def test_fp8_accumulation_stays_inside_its_floor(lib, ctx):
+    """Measures what the accumulation floor of GEMMs with an 8-bit operand allows for (one tensor-core
+    addition per 32 contraction columns, each off by at most 2 * 2^-23 of the running sum).  Rows of
+    A against rows of B whose products alternate in sign cancel to a small fraction of their summed
+    magnitudes; the GPU's sum must stay within half of that floor (plus the rounding of the two
+    de-scales), at the longest contraction the workloads have."""
+    rng = np.random.default_rng(31)
+    I, J, C = 128, 128, 16384
+    xa = np.abs(rng.standard_normal((I, C))).astype(np.float32)
+    xb = np.abs(rng.standard_normal((J, C))).astype(np.float32)
+    xb[:, ::2] *= -1.0                                                # alternating signs along the contraction
+    xa = O.bf16_bits_to_f64(WL.to_bf16_bits(xa))
+    xb = O.bf16_bits_to_f64(WL.to_bf16_bits(xb))
+    qa, qb = O.absmax_quantize(xa, 0, fmt="e4m3"), O.absmax_quantize(xb, 0, fmt="e2m1")
+    ca, cb = torch.from_numpy(qa.codes).cuda(), torch.from_numpy(qb.packed()).cuda()
+    got = lib.fp4_gemm(ctx, ca, cb, torch.from_numpy(qa.amax).cuda(), torch.from_numpy(qb.amax).cuda(),
+                       gemm_kind=lib.FP4_GEMM_F8F6F4_A8)
+    torch.cuda.synchronize()
+    scale = qa.descale.astype(np.float64)[:, None] * qb.descale.astype(np.float64)[None, :]
+    want = O.gemm_values(qa, qb) * scale
+    terms = (np.abs(qa.values()) @ np.abs(qb.values()).T) * scale
+    assert np.median(np.abs(want) / terms) < 0.05                     # the sums do cancel
+    floor = 2.0 * (C // 32) * 2.0 ** -23 * terms
+    err = np.abs(got.cpu().numpy().astype(np.float64) - want)
+    assert (err <= 0.5 * floor + 4 * 2.0 ** -23 * np.abs(want)).all(), f"{np.max(err / floor):.3f} of the floor"

@@ -17,8 +17,12 @@ from paper_2501_17116_b200 import workloads as WL
 pytestmark = pytest.mark.gpu
 RTOL = 1e-3
 
-# (config index, linear name, alpha)
-CASES = [(1, "q", 0.999), (1, "down", 0.999), (2, "down", 0.99), (3, "q", 0.9999), (4, "gate", 0.99)]
+# (config index, linear name, alpha): an attention and an MLP linear of every layer set, both swept
+# alphas of the 7B MLP block
+CASES = [(1, "q", 0.999), (1, "gate", 0.999), (1, "down", 0.999),
+         (2, "gate", 0.99), (2, "down", 0.99), (2, "gate", 0.999), (2, "down", 0.999),
+         (3, "q", 0.9999),
+         (4, "q", 0.99), (4, "gate", 0.99), (4, "down", 0.99)]
 
 
 def _dev(bits):
@@ -43,6 +47,17 @@ def _close(got, want, scale, what, floor=0.0):
     assert not bad.any(), f"{what}: {bad.sum()} of {bad.size} outside tolerance"
 
 
+def _bf16(out16, rows, cols, want, scale, what, floor=0.0):
+    """The BF16 output on the sampled entries: the rounding of the oracle value, or a neighbouring
+    BF16 number where the oracle value lies within the tolerance of a rounding boundary."""
+    got = out16[torch.as_tensor(rows, device="cuda")][:, torch.as_tensor(cols, device="cuda")].float().cpu().numpy()
+    got = got.astype(np.float64)
+    r = O.f64_to_bf16_f64(want)
+    ok = (got == r) | (np.abs(got - want) <= np.abs(r - want) + RTOL * scale + floor)
+    assert ok.all(), f"{what}: {np.sum(~ok)} of {ok.size} values are not the BF16 rounding of the oracle"
+    assert (got == r).mean() > 0.99, f"{what}: only {(got == r).mean():.4f} match the rounding exactly"
+
+
 @pytest.mark.parametrize("ci,lname,alpha", CASES)
 def test_full_size_layer_matches_sampled_oracle(lib, ci, lname, alpha):
     cfg = WL.CONFIGS[ci]
@@ -57,6 +72,9 @@ def test_full_size_layer_matches_sampled_oracle(lib, ci, lname, alpha):
     ctx = lib.Context.for_shape(M, K, N)
     y32, sa, sw = lib.fp4_linear_fwd(ctx, A, W, alpha, out_f32=True)
     da32, dw32 = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, out_f32=True)
+    # the BF16 outputs the benchmark times, from the same saved operands
+    y16, _, _ = lib.fp4_linear_fwd(ctx, A, W, alpha, saved_a=sa, saved_w=sw, reuse_a=True, reuse_w=True)
+    da16, dw16 = lib.fp4_linear_bwd(ctx, dY, W, sa, sw)
     torch.cuda.synchronize()
     assert ctx.read_status() == 0
 
@@ -126,6 +144,7 @@ def test_full_size_layer_matches_sampled_oracle(lib, ci, lname, alpha):
     # the tensor cores as in test_gpu_linear.py (4e-6 of the summed magnitudes of the residual's products)
     floor = 4e-6 * (np.abs(resid) @ np.abs(w_cols)) if alpha <= 0.995 else 0.0
     _close(got, y_fp4 + y_comp, np.abs(y_fp4) + np.abs(y_comp), "Y", floor)
+    _bf16(y16, rows, cols_w, y_fp4 + y_comp, np.abs(y_fp4) + np.abs(y_comp), "Y (BF16)", floor)
 
     # ---- dgrad: dA on rows x cols_a ----------------------------------------------------------------
     qg1 = O.absmax_quantize(O.bf16_bits_to_f64(dy_bits[rows]), 0, prescale=d_w)
@@ -136,6 +155,7 @@ def test_full_size_layer_matches_sampled_oracle(lib, ci, lname, alpha):
     da_ref = O.gemm_codes(qg1.codes, w_sel_codes) * qg1.descale.astype(np.float64)[:, None]
     got = da32[torch.as_tensor(rows, device="cuda")][:, torch.as_tensor(cols_a, device="cuda")].cpu().numpy()
     _close(got, da_ref, np.abs(da_ref), "dA")
+    _bf16(da16, rows, cols_a, da_ref, np.abs(da_ref), "dA (BF16)")
 
     # ---- wgrad: dW on cols_a x cols_w ----------------------------------------------------------------
     gamma_a, _ = O.absmax_scales(amax_a)
@@ -146,5 +166,10 @@ def test_full_size_layer_matches_sampled_oracle(lib, ci, lname, alpha):
     w_scaled = (O.bf16_bits_to_f64(w_bits[np.ix_(cols_a, cols_w)]) * gamma_w[cols_w].astype(np.float64)[None, :]).astype(np.float32)
     factor = O.dge_fprime(w_scaled.astype(np.float64))
     got = dw32[torch.as_tensor(cols_a, device="cuda")][:, torch.as_tensor(cols_w, device="cuda")].cpu().numpy()
-    _close(got, (s_fp4 + s_comp) * factor, (np.abs(s_fp4) + np.abs(s_comp)) * factor, "dW")
+    # dense residual columns are summed on the tensor cores in chunks of 128 tokens: the same
+    # accumulation floor as the forward tail, against the summed magnitudes of the column's products
+    floor_w = 4e-6 * (np.abs(resid_cols).T @ np.abs(O.bf16_bits_to_f64(dy_bits[:, cols_w]))) * factor
+    _close(got, (s_fp4 + s_comp) * factor, (np.abs(s_fp4) + np.abs(s_comp)) * factor, "dW", floor_w)
+    _bf16(dw16, cols_a, cols_w, (s_fp4 + s_comp) * factor, (np.abs(s_fp4) + np.abs(s_comp)) * factor, "dW (BF16)",
+          floor_w)
     ctx.close()

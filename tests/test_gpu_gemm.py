@@ -129,3 +129,31 @@ def test_argument_errors(lib, ctx):
     with pytest.raises(lib.Fp4Error) as e:
         lib.fp4_gemm(ctx, a, a, gemm_kind=7)
     assert e.value.code == -7
+
+
+def test_a_wait_that_runs_out_raises_timeout_and_leaves_the_context_usable(lib):
+    """Every device-side wait of the GEMM is bounded.  With the debug switches of the library the
+    producer of the first CTA leaves out one fill of the shared-memory ring while the limit of the
+    waits is 1 ms: the consumer's wait runs out, the kernel raises FP4_DEV_TIMEOUT, frees its tensor
+    memory and returns; the next GEMM on the same context is exact again."""
+    rng = np.random.default_rng(77)
+    ca, cb = _codes(rng, 256, 4096), _codes(rng, 256, 4096)          # 16 fills per tile (MXF4), 32 (byte containers)
+    want = O.gemm_codes(ca, cb)
+    a = torch.from_numpy(O.pack_nibbles(ca)).cuda()
+    b = torch.from_numpy(O.pack_nibbles(cb)).cuda()
+    c = lib.Context(0, 64 << 20)
+    for kind in KINDS:
+        c.debug_set(lib.binding.FP4_DEBUG_WAIT_LIMIT_US, 1000)
+        c.debug_set(lib.binding.FP4_DEBUG_SKIP_FILL, 6)
+        c.status.zero_()
+        lib.fp4_gemm(c, a, b, gemm_kind=kind)
+        torch.cuda.synchronize()                                       # the kernel returned
+        assert c.read_status() & lib.FP4_DEV_TIMEOUT
+        c.debug_set(lib.binding.FP4_DEBUG_SKIP_FILL, -1)
+        c.debug_set(lib.binding.FP4_DEBUG_WAIT_LIMIT_US, 0)
+        c.status.zero_()
+        out = lib.fp4_gemm(c, a, b, gemm_kind=kind)
+        torch.cuda.synchronize()
+        assert c.read_status() == 0
+        np.testing.assert_array_equal(out.cpu().numpy().astype(np.float64), want)
+    c.close()

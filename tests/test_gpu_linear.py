@@ -251,3 +251,91 @@ def test_config0_full_layer(lib, ctx):
         assert_close_f32(da32.cpu().numpy(), b.da, b.da, None, "dA")
         assert_close_f32(dw32.cpu().numpy(), b.dw, b.s_fp4 * b.dge, b.s_comp * b.dge, "dW")
         assert_bf16_rounding(y16, f.y, "Y")
+
+
+def test_dge_factor_alone_on_every_scaled_weight(lib, ctx):
+    """Q' of Eq. 8 (k = 5, cap 3.0) read by itself.  One token of sixes (de-scale exactly 1)
+    against one row of dY of 0.75 (de-scale exactly 1/8) makes the weight-gradient sum S exactly
+    6 * 6 / 8 = 4.5 everywhere (no clamp, no residual), so dW in float mode is 4.5 times the factor:
+    it is held to 1e-5 relative of the oracle's closed form on every BF16 weight pattern of magnitude
+    <= 6, under column scales gamma = 1, 2 and 1/4 (the scaled weight is formed in fp32 on both sides)."""
+    M, K, N = 128, 256, 256
+    pats = np.arange(0x0000, 0x40C1, dtype=np.uint16)                 # +0 ... +6.0
+    pats = np.concatenate([pats, pats | np.uint16(0x8000)])           # and the negatives
+    assert pats.size <= (K - 1) * N
+    w = np.zeros((K, N), dtype=np.uint16)
+    body = np.resize(pats, (K - 1) * N).reshape(K - 1, N)
+    w[1:] = body
+    w[0] = 0x40C0                                                      # 6.0 in every column: amax = 6, gamma = 1
+    # other column scales: amax = 3 (gamma 2; patterns up to 3.0 only) and amax = 24 (gamma 1/4)
+    w[0, 64:128] = 0x4040                                              # 3.0
+    big = (w[1:, 64:128] & np.uint16(0x7FFF)) > 0x4040
+    w[1:, 64:128][big] = 0x3F80                                        # 1.0 where the pattern would exceed the column's amax
+    w[0, 128:192] = 0x41C0                                             # 24.0
+    a = np.zeros((M, K), dtype=np.uint16)
+    a[0] = 0x40C0                                                      # token 0: sixes
+    dy = np.zeros((M, N), dtype=np.uint16)
+    dy[0] = 0x3F40                                                     # 0.75
+    f = O.linear_fwd(a, w, 1.0)
+    b = O.linear_bwd(dy, w, f)
+    assert np.all(b.s_fp4 == 4.5) and not np.any(b.s_comp)             # the sum is exact: dW is 4.5 times the factor
+    A, W, dY = _dev(a), _dev(w), _dev(dy)
+    ctx.status.zero_()
+    _, sa, sw = lib.fp4_linear_fwd(ctx, A, W, 1.0)
+    _, dw = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, out_f32=True, want_da=False)
+    torch.cuda.synchronize()
+    assert ctx.read_status() == 0
+    got = dw.cpu().numpy().astype(np.float64) / 4.5
+    assert np.array_equal(b.dw, 4.5 * b.dge)
+    rel = np.abs(got - b.dge) / b.dge
+    assert rel.max() <= 1e-5, f"DGE factor off by {rel.max():.2e} relative"
+    assert (b.dge == 3.0).sum() > 50 and (b.dge < 0.21).sum() > 100    # the cap and the grid points are both in the sample
+    assert np.array_equal(got[b.dge == 3.0], b.dge[b.dge == 3.0])      # the cap is exact
+
+
+def test_tensor_core_accumulation_stays_inside_its_floor(lib, ctx):
+    """Measures what TAIL_FLOOR allows for.  120 hot columns whose residual entries alternate in
+    sign against weights of one sign make the compensation branch cancel (sums of ~120 terms far
+    below the sum of their magnitudes), which is where the tensor cores' truncating fp32 additions
+    show.  Derivation of the floor: 24 additions per accumulator, each off by at most 2^-23 of the
+    running sum, plus 2^-21 from the two-term FP16 splits: 3.4e-6 of sum |dA| |W|, rounded up to
+    4e-6.  The forward (dense tail of the GEMM) and the weight gradient (dense columns, chunks of
+    128 tokens) must both stay within half of TAIL_FLOOR beyond the fp32 rounding of the two
+    branches; a constant that is too tight or a kernel that loses precision fails here."""
+    assert 24 * 2.0 ** -23 + 2.0 ** -21 <= TAIL_FLOOR
+    M, K, N, hot, alpha = 1024, 512, 384, 120, 0.85
+    a_bits, w_bits, dy_bits = WL.small_case(M, K, N, seed=1234, alpha_outliers=hot)
+    a = O.bf16_bits_to_f64(a_bits)
+    # hot columns: magnitudes kept, signs alternating along the columns, so that a token's residual sums cancel
+    col_energy = np.abs(a).sum(axis=0)
+    hot_cols = np.argsort(col_energy)[-hot:]
+    sign = np.where(np.arange(hot) % 2 == 0, 1.0, -1.0)
+    a[:, hot_cols] = np.abs(a[:, hot_cols]) * sign[None, :]
+    a_bits = WL.to_bf16_bits(a.astype(np.float32))
+    w = np.abs(O.bf16_bits_to_f64(w_bits))                             # weights of one sign
+    w_bits = WL.to_bf16_bits(w.astype(np.float32))
+    dy = np.abs(O.bf16_bits_to_f64(dy_bits))
+    dy[::2] *= -1.0                                                    # tokens alternate in sign: the sums over tokens cancel
+    dy_bits = WL.to_bf16_bits(dy.astype(np.float32))
+    f = O.linear_fwd(a_bits, w_bits, alpha)
+    b = O.linear_bwd(dy_bits, w_bits, f)
+    mags_y = np.abs(f.qa.residual) @ np.abs(O.bf16_bits_to_f64(w_bits))
+    mags_w = np.abs(f.qa.residual).T @ np.abs(O.bf16_bits_to_f64(dy_bits))
+    assert np.median(np.abs(f.y_comp) / mags_y) < 0.2                  # the compensation sums do cancel
+    A, W, dY = _dev(a_bits), _dev(w_bits), _dev(dy_bits)
+    ctx.status.zero_()
+    y, sa, sw = lib.fp4_linear_fwd(ctx, A, W, alpha, out_f32=True)
+    _, dw = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, out_f32=True, want_da=False)
+    torch.cuda.synchronize()
+    assert ctx.read_status() == 0
+    counts = np.diff(sa.csc_colptr.cpu().numpy())
+    assert (counts >= 512).sum() >= 100                                # the dense paths are taken
+    ulp = 2.0 ** -23
+    err_y = np.abs(y.cpu().numpy().astype(np.float64) - f.y)
+    allow_y = 0.5 * TAIL_FLOOR * mags_y + 8 * ulp * (np.abs(f.y_fp4) + np.abs(f.y_comp))
+    assert (err_y <= allow_y).all(), f"forward tail: {np.max(err_y / (TAIL_FLOOR * mags_y + 1e-300)):.3f} of the floor"
+    err_w = np.abs(dw.cpu().numpy().astype(np.float64) - b.dw)
+    allow_w = (0.5 * TAIL_FLOOR * mags_w + 8 * ulp * (np.abs(b.s_fp4) + np.abs(b.s_comp))) * b.dge * (1 + 1e-5)
+    # entries added per entry in fp32 (the scattered ones) get the ordinary summation bound on top
+    allow_w += 64 * ulp * mags_w * b.dge
+    assert (err_w <= allow_w).all(), f"weight gradient: {np.max(err_w / (TAIL_FLOOR * mags_w * b.dge + 1e-300)):.3f} of the floor"

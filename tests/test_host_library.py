@@ -81,3 +81,21 @@ def test_missing_library_fails_loudly(tmp_path):
 def test_tail_capacity_matches_the_header_rule():
     assert fp4.tail_capacity(256, 1024, 0.99) == 2 * 2621
     assert fp4.tail_capacity(128, 128, 1.0) == 0
+
+
+def test_sparse_capacity_is_the_librarys_rule(lib):
+    """Two tails of n_tail = round((1 - alpha) n) entries (Section 3.2 as read here); per token two
+    tails of round((1 - alpha) cols) entries in every row."""
+    cap = lib.fp4_sparse_capacity
+    assert cap(256, 1024, 0.99, fp4.FP4_QUANTILE_SIGNED) == 2 * 2621            # n_tail of the first configuration
+    assert cap(256, 1024, 0.99, fp4.FP4_QUANTILE_ABS) == 2 * 2621
+    assert cap(256, 1024, 0.99, fp4.FP4_QUANTILE_TOKEN) == 2 * 256 * 10
+    assert cap(16384, 13824, 0.99, fp4.FP4_QUANTILE_SIGNED) == 2 * 2264924       # the largest activation of the workloads
+    assert cap(128, 128, 1.0, fp4.FP4_QUANTILE_SIGNED) == 0
+    assert cap(128, 128, 0.4, fp4.FP4_QUANTILE_SIGNED) == -1
+    assert cap(128, 128, 0.99, 7) == -1
+    assert cap(0, 128, 0.99, fp4.FP4_QUANTILE_SIGNED) == -1
+
+
+def test_debug_switches_validate_their_arguments(lib):
+    assert lib.fp4_debug_set(None, 1, 1000) == -1

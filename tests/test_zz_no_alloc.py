@@ -11,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import fp4_oracle as O
 from paper_2501_17116_b200 import workloads as WL
 
 pytestmark = pytest.mark.gpu
@@ -36,6 +37,18 @@ def test_static_thresholds_equal_the_quantisers_on_two_calls_in_a_row(lib):
     assert torch.equal(got2, want2)
     assert got1[0] < 0 < got1[1]
     ctx.close()
+
+
+def test_static_thresholds_equal_the_oracles(lib):
+    """The same call against the CPU oracle's order statistics, on two calls in a row, the second
+    at the largest row count the fixed scratch takes."""
+    out = torch.empty(2, dtype=torch.float32, device="cuda")
+    a1 = WL.activations(WL.CONFIGS[0], 1024, seed=5)                               # 256 x 1024
+    a2 = WL.activations(WL.CONFIGS[1], 128, seed=6, M=lib.binding.FP4_STATIC_MAX_ROWS)   # 65536 x 128
+    for bits, alpha in ((a1, 0.99), (a2, 0.999), (a1, 0.97)):
+        got = lib.fp4_quantile_thresholds_static(_dev(bits), alpha, out=out).cpu().numpy()
+        lo, hi, _ = O.quantile_thresholds(O.bf16_bits_to_f64(bits), alpha)
+        assert (float(got[0]), float(got[1])) == (float(lo), float(hi))
 
 
 def test_static_entry_rejects_what_its_fixed_scratch_cannot_hold(lib):
