@@ -429,6 +429,41 @@ def main():
     ctx.profile_reset()
     nnz = [int(L["sa"].nnz.item()) if L["sa"].nnz is not None else 0 for L in layers]
 
+    # Residual entries that are gathered per entry (one row of the dense matrix each): all but those
+    # of the dense columns (at least max(M / 4, 512) entries, the first 128 of them), which go through
+    # the tensor cores -- in the weight gradient always, in the forward with a heavy residual.
+    def scattered_entries(L, forward):
+        sa = L["sa"]
+        if sa.nnz is None:
+            return 0
+        total = int(sa.nnz.item())
+        if forward and not (sa.sparse_cap * 100 >= M * L["K"]):
+            return total
+        counts = (sa.csc_colptr[1:] - sa.csc_colptr[:-1]).cpu().numpy()
+        dense = np.nonzero(counts >= max(M // 4, 512))[0][:128]
+        return total - int(counts[dense].sum())
+
+    gathered_fwd = sum(scattered_entries(L, True) * L["N"] * 2.0 for L in layers)
+    gathered_bwd = sum(scattered_entries(L, False) * L["N"] * 2.0 for L in layers)
+
+    # L2 read bandwidth, measured here: the bound of those gathers
+    l2_gbs = None
+    if alpha < 1.0:
+        probe = torch.empty(32 << 20, dtype=torch.uint8, device=dev)
+        sink = torch.zeros(1, dtype=torch.int32, device=dev)
+        blocks, reps = 4 * SM_COUNT, 1
+        best = None
+        for _ in range(4):
+            q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            q0.record()
+            fp4.fp4_l2_read_probe(probe, reps, blocks, sink)
+            q1.record()
+            torch.cuda.synchronize()
+            t = q0.elapsed_time(q1)
+            best = t if best is None else min(best, t)
+        l2_gbs = blocks * reps * probe.numel() / (best / 1e3) / 1e9
+        del probe
+
     # ------------------------------------------------------------------ end to end ---------
     # (the host-buffer entry point takes the method's own formats only)
     ms_e2e = None
@@ -480,27 +515,36 @@ def main():
         "encode": ("hbm", 3.125 * elems_a + 3.0 * elems_w + 3.0 * elems_g, "GB/s"),
         "absmax": ("hbm", 2.0 * elems_w + 2.0 * elems_g, "GB/s"),
         "sparse": ("hbm", 2 * 8.0 * nnz_quantised + 3 * elems_a / 8.0, "GB/s"),       # entries + 3 mask sweeps
-        "comp_fwd": ("alu", sum(2.0 * z * L["N"] for z, L in zip(nnz, layers)), "TFLOP/s"),
-        "comp_wgrad_dge": ("alu", sum(2.0 * z * L["N"] + 8.0 * L["K"] * L["N"] for z, L in zip(nnz, layers)),
-                           "TFLOP/s"),
+        # compensation: 2 nnz N flop on the plain ALUs by the method's own count; what bounds the
+        # kernels is the L2 traffic of the per-entry gathers (one BF16 row of the dense matrix per
+        # scattered entry), reported against the L2 read bandwidth measured above
+        "comp_fwd": ("l2", gathered_fwd, "GB/s"),
+        "comp_wgrad_dge": ("l2", gathered_bwd, "GB/s"),
     }
+    alu_flop = {"comp_fwd": sum(2.0 * z * L["N"] for z, L in zip(nnz, layers)),
+                "comp_wgrad_dge": sum(2.0 * z * L["N"] + 8.0 * L["K"] * L["N"] for z, L in zip(nnz, layers))}
     src = "of measured" if peaks["source"] == "measured" else "of fallback"
     peak_text = {
         "tensor": f"{src}: {ratio:g} x {'burst' if use_burst else 'sustained'} bf16 cuBLAS "
                   f"(classes timed inside a {region_seconds:.2f} s region)",
         "hbm": f"{src}: copy bandwidth",
-        "alu": "148 SMs x 128 FMA x 2 x max clock",
+        "l2": "of measured: L2 read bandwidth by fp4_l2_read_probe in this run (32 MB buffer, 16-byte loads)",
     }
     kernels = {}
     total_ms = sum(v[0] for v in prof.values()) or 1.0
     for name, (t_ms, n) in prof.items():
         bound, w_step, unit = work[name]
-        peak = {"tensor": fp4_peak, "hbm": peaks["hbm_gbs"], "alu": alu_peak}[bound]
+        peak = {"tensor": fp4_peak, "hbm": peaks["hbm_gbs"], "l2": l2_gbs or 1.0}[bound]
         scale = 1e12 if unit == "TFLOP/s" else 1e9
         achieved = (w_step * steps / (t_ms / 1e3) / scale) if t_ms > 0 else 0.0
         kernels[name] = {"bound": bound, "achieved": round(achieved, 2), "peak": round(peak, 1), "unit": unit,
                          "frac": round(achieved / peak, 4), "ms_per_step": round(t_ms / steps, 4),
                          "share": round(t_ms / total_ms, 4), "launches_per_step": n // steps}
+        if bound == "l2":
+            # the method's own flop count against the plain fp32 pipe (148 SMs x 128 FMA x 2 x max clock)
+            tf = alu_flop[name] * steps / (t_ms / 1e3) / 1e12 if t_ms > 0 else 0.0
+            kernels[name]["alu_tflops"] = round(tf, 2)
+            kernels[name]["alu_frac"] = round(tf / alu_peak, 4)
         if bound == "tensor":
             kernels[name]["frac_of_burst"] = round(achieved / (ratio * peaks["bf16_burst"]), 4)
             kernels[name]["frac_of_sustained"] = round(achieved / (ratio * peaks["bf16_sustained"]), 4)

@@ -262,6 +262,14 @@ int fp4_linear_step_host(fp4_ctx* ctx, void* stream, const void* A_host, const v
 #define FP4_KC_COMP_WGRAD  6   /* residual^T x dY + DGE factor + final store of dW            */
 #define FP4_KC_COUNT       7
 int fp4_profile_enable(fp4_ctx* ctx, int on);
+/* Measurement support (no counterpart in the paper): a read-only kernel for measuring the bandwidth
+ * of the L2 cache, the bound of the per-entry gathers of the sparse compensation (Section 3.2: one
+ * row of the dense matrix per residual entry).  `blocks` blocks of 256 threads each read all of
+ * `buf` (`bytes`, a multiple of 16384, at least 65536, 16-byte aligned; choose it smaller than L2)
+ * `repeats` times with 16-byte loads that bypass L1, every block from its own starting offset.
+ * Bytes read = blocks * repeats * bytes; the caller times the call.  `sink` is a device word the
+ * kernel may write.                                                                          */
+int fp4_l2_read_probe(void* stream, const void* buf, size_t bytes, int repeats, int blocks, unsigned* sink);
 /* Inside one call, independent kernel chains (weight quantisation, sparse extraction, the
  * weight-gradient branch) run on side streams owned by the context and rejoin `stream` before
  * the call's work ends.  fp4_set_overlap(ctx, 0) puts every kernel on `stream` in program order

@@ -8,7 +8,7 @@ entry point loads it on first use and raises if it has not been built.
 from .binding import (  # noqa: F401
     FP4_DEV_NONFINITE, FP4_DEV_TIMEOUT, FP4_GEMM_F8F6F4, FP4_GEMM_F8F6F4_A8, FP4_GEMM_F8F6F4_A8B8, FP4_GEMM_F8F6F4_B8, FP4_GEMM_MXF4,
     FP4_BWD_DY_E4M3, FP4_BWD_DY_E5M2, FP4_FORMAT_E2M1, FP4_FORMAT_E4M3, FP4_FORMAT_E5M2, FP4_GEMM_A_E5M2, FP4_GEMM_B_E5M2, FP4_QUANTILE_ABS, FP4_QUANTILE_SIGNED, FP4_QUANTILE_TOKEN, EXPORTS,
-    Context, Fp4Error, QTensor, fp4_gemm, fp4_linear_bwd, fp4_linear_fwd, fp4_linear_step_host, fp4_quantile_thresholds_static, fp4_quantize, load_library,
+    Context, Fp4Error, QTensor, fp4_gemm, fp4_linear_bwd, fp4_linear_fwd, fp4_linear_step_host, fp4_quantile_thresholds_static, fp4_quantize, fp4_l2_read_probe, load_library,
     tail_capacity, KERNEL_CLASSES,
 )
 from . import workloads  # noqa: F401

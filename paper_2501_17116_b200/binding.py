@@ -31,7 +31,7 @@ FP4_DEV_TIMEOUT = 4
 EXPORTS = ("fp4_create", "fp4_destroy", "fp4_workspace_bytes", "fp4_status_string", "fp4_quantize",
            "fp4_gemm", "fp4_linear_fwd", "fp4_linear_bwd", "fp4_step_host_workspace_bytes",
            "fp4_linear_step_host", "fp4_profile_enable", "fp4_profile_reset", "fp4_profile_read",
-           "fp4_launch_count", "fp4_quantile_thresholds_static", "fp4_set_overlap", "fp4_debug_set", "fp4_sparse_capacity",
+           "fp4_launch_count", "fp4_quantile_thresholds_static", "fp4_set_overlap", "fp4_l2_read_probe", "fp4_debug_set", "fp4_sparse_capacity",
            "fp4_set_quantile_mode")
 FP4_STATIC_MAX_ROWS = 65536
 FP4_QUANTILE_SIGNED = 0
@@ -96,6 +96,8 @@ def load_library(path: str | None = None) -> C.CDLL:
     lib.fp4_profile_reset.restype = C.c_int
     lib.fp4_profile_read.argtypes = [vp, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     lib.fp4_profile_read.restype = C.c_int
+    lib.fp4_l2_read_probe.argtypes = [vp, vp, C.c_size_t, C.c_int, C.c_int, vp]
+    lib.fp4_l2_read_probe.restype = C.c_int
     lib.fp4_debug_set.argtypes = [vp, C.c_int, i64]
     lib.fp4_debug_set.restype = C.c_int
     lib.fp4_sparse_capacity.argtypes = [i64, i64, C.c_double, C.c_int]
@@ -342,3 +344,9 @@ def fp4_quantile_thresholds_static(x: torch.Tensor, alpha: float, out: torch.Ten
     _check(load_library().fp4_quantile_thresholds_static(_stream(), _ptr(x), x.shape[0], x.shape[1], float(alpha),
                                                          _ptr(out)))
     return out
+
+
+def fp4_l2_read_probe(buf: torch.Tensor, repeats: int, blocks: int, sink: torch.Tensor):
+    """Measurement support: `blocks` blocks read all of `buf` `repeats` times through L2 (the caller times it)."""
+    _check(load_library().fp4_l2_read_probe(_stream(), _ptr(buf), buf.numel() * buf.element_size(), int(repeats),
+                                            int(blocks), _ptr(sink)))
