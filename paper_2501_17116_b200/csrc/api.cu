@@ -277,7 +277,7 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
   // A heavy residual (the caller's capacity says it may hold at least 1 % of the activation, alpha <=
   // 0.995) sends its hot columns through the GEMM as a dense tail instead of per-entry gathers.
   const bool tail_on = occ && savedA->csr_rowptr && savedA->csc_colptr &&
-                       savedA->sparse_cap * 100 >= M * K;
+                       savedA->sparse_cap * 100 >= M * K && M >= 512;   // a hot column holds at least 512 entries
   char* scratch_tail = tail_on ? arena.take<char>(fwd_tail_scratch_bytes(M, K, N)) : nullptr;
   if (!arena.ok) return FP4_ERR_WORKSPACE;
   int rc;

@@ -531,8 +531,10 @@ int launch_comp_wgrad(fp4_ctx* ctx, cudaStream_t stream, const fp4_qtensor* a, c
   int* list_short = lists + K;
   int* counts = lists + 2 * K;
   // Columns that at least a quarter of the tokens hit (the outlier channels) form the dense class,
-  // whose product runs on the tensor cores; it needs the CSR.
-  const bool dense = a->csr_rowptr != nullptr;
+  // whose product runs on the tensor cores; it needs the CSR.  It costs three launches, which pay
+  // when the residual is heavy: when it may hold at least 1 % of the activation (alpha <= 0.995).
+  // (No column can reach LONG_COLUMN entries with fewer tokens than that.)
+  const bool dense = a->csr_rowptr != nullptr && a->sparse_cap * 100 >= M * K && M >= LONG_COLUMN;
   const int dense_from = dense ? int(M / 4 > LONG_COLUMN ? M / 4 : LONG_COLUMN) : INT_MAX;
   const unsigned n_blocks = unsigned((N + COMP_COLS - 1) / COMP_COLS);
   KernelScope scope(ctx, stream, KC_COMP_WGRAD, 3 + (dense ? (splits > 1 ? 3 : 2) : 0));
