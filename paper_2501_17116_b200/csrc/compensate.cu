@@ -406,16 +406,25 @@ comp_wgrad_long_kernel(float* __restrict__ comp, const int* __restrict__ colptr,
   }
 }
 
-// Short columns: one warp per (column, 256 outputs), entries in order.
+// Short columns: one warp per (column, 256 outputs), entries in order.  The work items (block of 256
+// outputs, group of 8 columns) are numbered with the block of outputs as the slow index and taken
+// in that order, so that the blocks in flight at any time read one or two 512-byte-wide slabs of dY
+// (tokens x 512 bytes: a few MB, which stay in L2) instead of all of it: every token's piece of a
+// slab is gathered by about 1 % of the columns, and those re-reads then hit L2.
 __global__ void __launch_bounds__(COMP_THREADS)
 comp_wgrad_short_kernel(float* __restrict__ comp, const int* __restrict__ colptr, const int* __restrict__ row,
                         const float* __restrict__ val, const uint4* __restrict__ dy, const int* __restrict__ list,
                         const int* __restrict__ counts, int N) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * COMP_COLS + 8 * lane;
-  if (n0 >= N) return;
   const int n_before = counts[0] + counts[1], n_cols = counts[2];
-  for (int slot = blockIdx.y * 8 + warp; slot < n_cols; slot += gridDim.y * 8) {
+  const int groups = (n_cols + 7) >> 3;
+  const int n_blocks = (N + COMP_COLS - 1) / COMP_COLS;
+  const long long items = (long long)groups * n_blocks;
+  for (long long it = blockIdx.x; it < items; it += gridDim.x) {
+    const int nb = int(it / groups);
+    const int slot = int(it - (long long)nb * groups) * 8 + warp;
+    const int n0 = nb * COMP_COLS + 8 * lane;
+    if (slot >= n_cols || n0 >= N) continue;
     const int k = list[slot];
     float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     strided_entries_times_dense(acc, row, val, colptr[k], colptr[k + 1], 1, dy, N >> 3, n0 >> 3);
@@ -553,10 +562,14 @@ int launch_comp_wgrad(fp4_ctx* ctx, cudaStream_t stream, const fp4_qtensor* a, c
   gy = gy < 1 ? 1 : (gy > unsigned(K) ? unsigned(K) : gy);
   comp_wgrad_long_kernel<<<dim3(n_blocks, gy), LONG_THREADS, 0, stream>>>(comp, a->csc_colptr, a->csc_row, a->csc_val,
                                                                          dy, list_long, counts, int(N));
-  gy = unsigned(32 * ctx->num_sms) / n_blocks;                   // short columns: 8 per block
-  gy = gy < 1 ? 1 : (gy > unsigned((K + 7) / 8) ? unsigned((K + 7) / 8) : gy);
-  comp_wgrad_short_kernel<<<dim3(n_blocks, gy), COMP_THREADS, 0, stream>>>(comp, a->csc_colptr, a->csc_row,
-                                                                           a->csc_val, dy, list_short, counts, int(N));
+  {
+    // short columns: 8 per block; about 32 blocks per SM in all, each taking work items in order
+    const long long max_items = (long long)((K + 7) / 8) * n_blocks;
+    long long g = 32LL * ctx->num_sms;
+    g = g > max_items ? max_items : g;
+    comp_wgrad_short_kernel<<<unsigned(g), COMP_THREADS, 0, stream>>>(comp, a->csc_colptr, a->csc_row, a->csc_val, dy,
+                                                                      list_short, counts, int(N));
+  }
   FP4_CUDA_TRY(cudaGetLastError());
   return FP4_OK;
 }
