@@ -325,6 +325,8 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
   }
   GemmTail tail = {nullptr, nullptr, nullptr};
   const int* hot_slot_of_col = nullptr;
+  const void* kept = nullptr;
+  const int* kept_end = nullptr;
   if (tail_on) {
     // The tail's operands need the CSR, the CSC's column pointers and W's amax: both sparse chains
     // are joined before the GEMM here (without a tail they run beside it).
@@ -333,7 +335,8 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
       FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[7], 0));
     }
     Arena ta(scratch_tail, fwd_tail_scratch_bytes(M, K, N));
-    rc = launch_fwd_tail(ctx, st, savedA, W_bf16, savedW->amax, fp8_max(w8), ta, M, K, N, &tail, &hot_slot_of_col);
+    rc = launch_fwd_tail(ctx, st, savedA, W_bf16, savedW->amax, fp8_max(w8), ta, M, K, N, &tail, &hot_slot_of_col, &kept,
+                         &kept_end);
     if (rc != FP4_OK) return rc;
   }
   rc = launch_gemm_fp4(ctx, st, savedA->codes, savedW->codes_t, M, N, K, savedA->amax, savedW->amax, y1, 1, gemm_kind,
@@ -342,7 +345,7 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
   // Y = store(Y1 + (A - A_c) W): one rounding of the fp32 sum.  Needs the CSR.
   if (!reuse_a && ov) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[3], 0));
   rc = launch_comp_fwd(ctx, st, y1, savedA->csr_rowptr, savedA->csr_col, savedA->csr_val, W_bf16, M, K, N, Y, out_f32,
-                       hot_slot_of_col, tail.count);
+                       hot_slot_of_col, tail.count, kept, kept_end);
   if (rc != FP4_OK) return rc;
   if (!reuse_a && ov) FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[7], 0));  // the CSC too: savedA is complete on return
   return FP4_OK;

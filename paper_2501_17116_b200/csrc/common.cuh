@@ -222,12 +222,13 @@ int launch_quantize_dual(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const 
 int launch_comp_fwd(fp4_ctx* ctx, cudaStream_t stream, const float* y1, const int32_t* rowptr,
                     const int32_t* col, const float* val, const void* w_bf16, int64_t M, int64_t K,
                     int64_t N, void* y, int out_f32, const int* slot_of_col = nullptr,
-                    const int* tail_count = nullptr);
+                    const int* tail_count = nullptr, const void* kept = nullptr, const int* kept_end = nullptr);
 // The forward GEMM's dense tail (see GemmTail): operands built from the saved activation and the weights.
 size_t fwd_tail_scratch_bytes(int64_t M, int64_t K, int64_t N);
+// `kept_out` / `kept_end_out`: per token, the entries the tail does not cover (null for residuals too heavy to list).
 int launch_fwd_tail(fp4_ctx* ctx, cudaStream_t stream, const fp4_qtensor* a, const void* w_bf16, const float* w_amax,
                     float w_div, Arena& scratch, int64_t M, int64_t K, int64_t N, GemmTail* tail,
-                    const int** slot_of_col_out);
+                    const int** slot_of_col_out, const void** kept_out, const int** kept_end_out);
 // Weight-gradient compensation into a compact buffer: for every column k of the residual that
 // holds entries, comp[slot_of_col[k], :] = sum_{entries of column k} val * dy[row, :].
 // Lists, slots and the dense path's buffers are carved from `scratch` (comp_wgrad_scratch_bytes); the slot

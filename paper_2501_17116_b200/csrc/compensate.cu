@@ -147,6 +147,49 @@ comp_fwd_skip_kernel(const float* __restrict__ y1, const int* __restrict__ rowpt
   store8(y, out_f32, off, y8);
 }
 
+// The forward compensation when the dense tail is in use: tail_a has listed, per token, the entries
+// the tail does not cover (`kept`: column and value bits, at the token's own range of the CSR, ending
+// at kept_end[m]), so this kernel walks a plain list: one 8-byte broadcast load per entry, four
+// weight-row gathers in flight.  If the tail was switched off on the device (*tail_count == 0: a value
+// FP16 cannot hold) the list is not valid and the whole CSR row is added instead.
+__global__ void __launch_bounds__(COMP_THREADS)
+comp_fwd_kept_kernel(const float* __restrict__ y1, const int* __restrict__ rowptr, const int* __restrict__ col,
+                     const float* __restrict__ val, const uint2* __restrict__ kept, const int* __restrict__ kept_end,
+                     const uint4* __restrict__ w, int M, int N, void* y, int out_f32,
+                     const int* __restrict__ tail_count) {
+  const int m = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int n0 = blockIdx.y * COMP_COLS + 8 * (threadIdx.x & 31);
+  if (m >= M || n0 >= N) return;
+  const long long off = (long long)m * N + n0;
+  const float4 a = __ldg(reinterpret_cast<const float4*>(y1 + off));
+  const float4 b = __ldg(reinterpret_cast<const float4*>(y1 + off + 4));
+  float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  const int vec_per_row = N >> 3, vcol = n0 >> 3;
+  if (__ldg(tail_count) > 0) {
+    int e = __ldg(&rowptr[m]);
+    const int e1 = __ldg(&kept_end[m]);
+    for (; e + 4 <= e1; e += 4) {
+      uint2 t[4];
+      uint4 d[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) t[u] = __ldg(&kept[e + u]);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) d[u] = __ldg(&w[(long long)t[u].x * vec_per_row + vcol]);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) fma8(acc, __uint_as_float(t[u].y), d[u]);
+    }
+    for (; e < e1; ++e) {
+      const uint2 t = __ldg(&kept[e]);
+      fma8(acc, __uint_as_float(t.y), __ldg(&w[(long long)t.x * vec_per_row + vcol]));
+    }
+  } else {
+    sparse_row_times_dense(acc, col, val, __ldg(&rowptr[m]), __ldg(&rowptr[m + 1]), w, vec_per_row, vcol);
+  }
+  const float y8[8] = {a.x + acc[0], a.y + acc[1], a.z + acc[2], a.w + acc[3],
+                       b.x + acc[4], b.y + acc[5], b.z + acc[6], b.w + acc[7]};
+  store8(y, out_f32, off, y8);
+}
+
 constexpr int LONG_COLUMN = 512;           // entries from which a column gets a whole 1024-thread block
 constexpr int LONG_THREADS = 1024;
 
@@ -215,7 +258,7 @@ __device__ __forceinline__ void split_half(float x, __half& hi, __half& lo) {
 __global__ void __launch_bounds__(COMP_THREADS)
 tail_a_kernel(const int* __restrict__ rowptr, const int* __restrict__ col, const float* __restrict__ val,
               const int* __restrict__ slot_of_col, int* __restrict__ count, const float* __restrict__ amax_row,
-              float row_div, __half* __restrict__ ta, int M) {
+              float row_div, __half* __restrict__ ta, int M, uint2* __restrict__ kept, int* __restrict__ kept_end) {
   const int hot = *count;
   if (hot == 0) return;
   const int lane = threadIdx.x & 31;
@@ -227,10 +270,26 @@ tail_a_kernel(const int* __restrict__ rowptr, const int* __restrict__ col, const
   const float scale = __fdiv_rn(__ldg(&amax_row[m]), row_div) * TAIL_SCALE;
   __half* row = ta + size_t(m) * TAIL_WIDTH;
   bool bad = false;
-  for (int e = rowptr[m] + lane; e < rowptr[m + 1]; e += 32) {
-    const int slot = slot_of_col[col[e]];
-    if (unsigned(slot) >= unsigned(hot)) continue;
-    const float x = __fdiv_rn(val[e], scale);
+  const int e0 = rowptr[m], e1 = rowptr[m + 1];
+  int n_kept = e0;                                       // the kept entries go to this token's own range
+  for (int base = e0; base < e1; base += 32) {
+    const int e = base + lane;
+    int k = 0, slot = -1;
+    float v = 0.0f;
+    if (e < e1) {
+      k = col[e];
+      v = val[e];
+      slot = slot_of_col[k];
+    }
+    const bool is_hot = e < e1 && unsigned(slot) < unsigned(hot);
+    const bool keep = e < e1 && !is_hot;
+    if (kept) {                                          // entries the tail does not cover, in column order
+      const unsigned km = __ballot_sync(0xFFFFFFFFu, keep);
+      if (keep) kept[n_kept + __popc(km & ((1u << lane) - 1u))] = make_uint2(uint32_t(k), __float_as_uint(v));
+      n_kept += __popc(km);
+    }
+    if (!is_hot) continue;
+    const float x = __fdiv_rn(v, scale);
     if (!(fabsf(x) <= 65504.0f)) { bad = true; continue; }         // also catches NaN (0 / 0)
     __half hi, lo;
     split_half(x, hi, lo);
@@ -239,6 +298,7 @@ tail_a_kernel(const int* __restrict__ rowptr, const int* __restrict__ col, const
     row[at + 64] = hi;
     row[at + 128] = lo;
   }
+  if (kept && lane == 0) kept_end[m] = n_kept;
   if (bad) atomicExch(count, 0);
 }
 
@@ -472,10 +532,14 @@ extern "C" int fp4_l2_read_probe(void* stream, const void* buf, size_t bytes, in
 
 int launch_comp_fwd(fp4_ctx* ctx, cudaStream_t stream, const float* y1, const int32_t* rowptr, const int32_t* col,
                     const float* val, const void* w_bf16, int64_t M, int64_t, int64_t N, void* y, int out_f32,
-                    const int* slot_of_col, const int* tail_count) {
+                    const int* slot_of_col, const int* tail_count, const void* kept, const int* kept_end) {
   const dim3 grid(unsigned((M + 7) / 8), unsigned((N + COMP_COLS - 1) / COMP_COLS));
   KernelScope scope(ctx, stream, KC_COMP_FWD, 1);
-  if (slot_of_col && tail_count)
+  if (kept && kept_end && tail_count)
+    comp_fwd_kept_kernel<<<grid, COMP_THREADS, 0, stream>>>(y1, rowptr, col, val, static_cast<const uint2*>(kept),
+                                                            kept_end, static_cast<const uint4*>(w_bf16), int(M), int(N),
+                                                            y, out_f32, tail_count);
+  else if (slot_of_col && tail_count)
     comp_fwd_skip_kernel<<<grid, COMP_THREADS, 0, stream>>>(y1, rowptr, col, val, static_cast<const uint4*>(w_bf16),
                                                             int(M), int(N), y, out_f32, slot_of_col, tail_count);
   else
@@ -492,10 +556,14 @@ size_t comp_wgrad_scratch_bytes(int64_t M, int64_t K, int64_t N) {
   return b;
 }
 
+// Residual entries up to which the forward lists the entries its dense tail does not cover
+// (4 % of the activation: alpha >= 0.98); heavier residuals filter inside the per-entry kernel.
+static int64_t kept_list_capacity(int64_t M, int64_t K) { return M * K / 25; }
+
 size_t fwd_tail_scratch_bytes(int64_t M, int64_t K, int64_t N) {
   auto r256 = [](size_t b) { return (b + 255) & ~size_t(255); };
   return r256(size_t(M) * TAIL_WIDTH * 2) + r256(size_t(N) * TAIL_WIDTH * 2) + r256(size_t(K) * 4) +
-         r256(TAIL_MAX_COLS * 4) + 256;
+         r256(TAIL_MAX_COLS * 4) + 256 + r256(size_t(kept_list_capacity(M, K)) * 8) + r256(size_t(M) * 4);
 }
 
 // Prepares the dense tail of the forward GEMM from the saved activation `a` (CSR, CSC column
@@ -503,19 +571,24 @@ size_t fwd_tail_scratch_bytes(int64_t M, int64_t K, int64_t N) {
 // for the per-entry kernel.  Buffers come from `scratch` (fwd_tail_scratch_bytes).
 int launch_fwd_tail(fp4_ctx* ctx, cudaStream_t stream, const fp4_qtensor* a, const void* w_bf16, const float* w_amax,
                     float w_div, Arena& scratch, int64_t M, int64_t K, int64_t N, GemmTail* tail,
-                    const int** slot_of_col_out) {
+                    const int** slot_of_col_out, const void** kept_out, const int** kept_end_out) {
   __half* ta = scratch.take<__half>(size_t(M) * TAIL_WIDTH);
   __half* tb = scratch.take<__half>(size_t(N) * TAIL_WIDTH);
   int* slot_of_col = scratch.take<int>(size_t(K));
   int* list_hot = scratch.take<int>(TAIL_MAX_COLS);
   int* count = scratch.take<int>(1);
+  const bool list_kept = a->sparse_cap <= kept_list_capacity(M, K);
+  uint2* kept = list_kept ? scratch.take<uint2>(size_t(kept_list_capacity(M, K))) : nullptr;
+  int* kept_end = list_kept ? scratch.take<int>(size_t(M)) : nullptr;
   if (!scratch.ok) return FP4_ERR_WORKSPACE;
+  *kept_out = kept;
+  *kept_end_out = kept_end;
   const int hot_from = int(M / 4 > LONG_COLUMN ? M / 4 : LONG_COLUMN);
   KernelScope scope(ctx, stream, KC_COMP_FWD, 3);
   hot_columns_kernel<<<1, 1024, 0, stream>>>(a->csc_colptr, int(K), hot_from, list_hot, slot_of_col, count);
   FP4_CUDA_TRY(cudaMemsetAsync(tb, 0, size_t(N) * TAIL_WIDTH * 2, stream));
   tail_a_kernel<<<unsigned((M + 7) / 8), COMP_THREADS, 0, stream>>>(a->csr_rowptr, a->csr_col, a->csr_val, slot_of_col,
-                                                                   count, a->amax, 6.0f, ta, int(M));
+                                                                   count, a->amax, 6.0f, ta, int(M), kept, kept_end);
   tail_b_kernel<<<dim3(unsigned((N + 255) / 256), 16), 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(w_bf16),
                                                                         list_hot, count, w_amax, w_div, tb, int(N));
   FP4_CUDA_TRY(cudaGetLastError());
