@@ -53,6 +53,15 @@ NCU_TRAFFIC_PER_LAUNCH = {
         "comp_fwd": 36.1e6,    # profiles/compensation_llama1p3b.md
         "comp_wgrad_dge": 6.5e6,
     },
+    # profiles/compensation_gather_llama7b_mlp.md: captured on the 7B MLP block (same kernels, same
+    # residual density; the 13B layer is too large for a multi-pass capture) and scaled to the mean
+    # launch of this workload by the units processed: comp_fwd_kept moves 6.85 B per output element
+    # (fp32 FP4-branch read, BF16 store, the weight once), comp_wgrad_short reads dY once plus the
+    # entries (1.14 x 2 B per element of dY) and writes its fp32 rows (0.87 x 4 B per weight element).
+    "llama-13b-layer": {
+        "comp_fwd": 6.85 * 124.6e6,
+        "comp_wgrad_dge": 1.14 * 2 * 124.6e6 + 0.87 * 4 * 45.3e6,
+    },
 }
 
 

@@ -30,8 +30,8 @@ Readings of points the paper leaves open (each also listed in the design notes):
   with ``n_tail = round((1 - alpha) * n)``, ``lo = sorted[n_tail]`` and
   ``hi = sorted[n - 1 - n_tail]`` (Section 3.2 gives a residual density of
   2(1 - alpha), Appendix B).
-* The residual is multiplied by the original BF16 weight ("high-precision
-  sparse matrix multiplication", Section 3.2).
+* The residual is multiplied by the original BF16 weight in high precision
+  (Section 3.2 asks for a high-precision product of the sparse residual).
 * Backward GEMMs take E2M1 operands as well (Appendix B counts the backward at
   the FP4 rate) and re-use the forward codes of A and W; the scale vector that
   lies along the contraction is folded into dY before dY is quantised.
@@ -60,7 +60,7 @@ import numpy as np
 # E2M1 format: Table 4, row "e2m1"; sign-magnitude 4-bit codes (Section 2).
 # --------------------------------------------------------------------------- #
 E2M1_MAGNITUDES = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
-FP4_MAX = 6.0  # "MAX_fp4 is calculated to be 6.0", below Eq. 1
+FP4_MAX = 6.0  # the largest E2M1 magnitude: the value the text below Eq. 1 gives for MAX_fp4
 
 # Appendix A: the 14 constants of the comparison chain and the 15 results.
 LUT_THRESHOLDS = np.array(
