@@ -304,7 +304,7 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
     savedA->rows = M;
     savedA->cols = K;
     // CSR on side stream 1, CSC on side stream 0 (behind W's short chain, which has ended by then)
-    const SparseOverlap so = {ctx->side[1], ctx->ev[2], ctx->ev[3], ctx->side[0], ctx->ev[7]};
+    const SparseOverlap so = {ctx->side[1], ctx->ev[2], ctx->ev[3], ctx->side[0], ctx->ev[7], ctx->ev[4]};
     rc = launch_quantize(ctx, st, a, A_bf16, M, K, /*scale_axis=*/0, alpha, nullptr, 0.0f, savedA, status,
                          occ && ov ? &so : nullptr);
     if (rc != FP4_OK) return rc;
@@ -328,11 +328,11 @@ int linear_fwd_impl(fp4_ctx* ctx, cudaStream_t st, Arena arena, const void* A_bf
   const void* kept = nullptr;
   const int* kept_end = nullptr;
   if (tail_on) {
-    // The tail's operands need the CSR, the CSC's column pointers and W's amax: both sparse chains
-    // are joined before the GEMM here (without a tail they run beside it).
+    // The tail's operands need the CSR, the CSC's column pointers and W's amax: the CSR chain and
+    // the first half of the CSC chain are joined before the GEMM here; the CSC's fill runs beside it.
     if (!reuse_a && ov) {
       FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[3], 0));
-      FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[7], 0));
+      FP4_CUDA_TRY(cudaStreamWaitEvent(st, ctx->ev[4], 0));
     }
     Arena ta(scratch_tail, fwd_tail_scratch_bytes(M, K, N));
     rc = launch_fwd_tail(ctx, st, savedA, W_bf16, savedW->amax, fp8_max(w8), ta, M, K, N, &tail, &hot_slot_of_col, &kept,

@@ -188,14 +188,16 @@ int launch_gemm_fp4_two(fp4_ctx* ctx, cudaStream_t stream, const Fp4GemmDesc& fi
 
 // Lets the mask -> CSR / CSC stage of a clamping quantisation run beside the caller's stream: both
 // chains start after `encoded` (recorded on the main stream); the CSR chain runs on `stream` and
-// records `csr_done` there; the CSC chain runs on `stream_csc` and records `csc_done` there (null:
-// it follows the CSR on `stream`).  The caller joins the streams.
+// records `csr_done` there; the CSC chain runs on `stream_csc` and records `colptr_done` after its
+// column pointers and `csc_done` at its end there (null: it follows the CSR on `stream`).  The caller
+// joins the streams.
 struct SparseOverlap {
   cudaStream_t stream;
   cudaEvent_t encoded;
   cudaEvent_t csr_done;
   cudaStream_t stream_csc;
   cudaEvent_t csc_done;
+  cudaEvent_t colptr_done;    // recorded on the CSC chain's stream once csc_colptr is complete (or null)
 };
 
 // Quantiser pieces (quantize.cu)

@@ -1184,6 +1184,7 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
       KernelScope scope(ctx, sc2, KC_SPARSE, 3);
       csc_strip_prefix_kernel<<<(cols + 255) / 256, 256, 0, sc2>>>(sc.strip_cnt, cols, strips, sc.strip_off, sc.col_cnt);
       scan_counts_kernel<<<1, 1024, 0, sc2>>>(sc.col_cnt, cols, out->csc_colptr, nullptr);
+      if (sc2 != sp && overlap->colptr_done) FP4_CUDA_TRY(cudaEventRecord(overlap->colptr_done, sc2));
       const dim3 cgrid((cols / 32 + 7) / 8, strips);
       csc_fill_kernel<<<cgrid, 256, 0, sc2>>>(mask32, xb, rows, cols, out->thresholds, per_token, out->csc_colptr, sc.strip_off,
                                               out->sparse_cap, out->csc_row, out->csc_val);
