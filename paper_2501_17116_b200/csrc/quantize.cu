@@ -622,6 +622,7 @@ struct EncodeArgs {
   uint8_t* mask;                // clamp: [rows x cols/8] bytes
   int* row_cnt;                 // clamp: clamped entries per row (zero-initialised)
   uint8_t* strip_cnt;           // clamp: [rows/64 x cols] clamped entries per (strip, column)
+  int* col_cnt;                 // clamp: clamped entries per column (zero-initialised)
   float fmax;                   // FP8 encoder: the format's largest value (448 or 57344)
   int e5m2;                     // FP8 encoder: E5M2 bytes instead of E4M3 bytes
 };
@@ -766,8 +767,10 @@ encode_kernel(const EncodeArgs a) {
     for (int c = 0; c < 8; ++c) tile_t[(c * 8 + warp) * 32 + lane] = word[c];
   }
   __syncthreads();
-  if (OCC && col0 + tid < a.cols)
+  if (OCC && col0 + tid < a.cols) {
     a.strip_cnt[(long long)blockIdx.y * a.cols + col0 + tid] = uint8_t(s_colcnt[tid]);
+    if (s_colcnt[tid]) atomicAdd(&a.col_cnt[col0 + tid], s_colcnt[tid]);     // integer sums: order-independent
+  }
   if (a.codes_t) {
     // thread (c = warp, j = lane) owns column col0 + 8 j + c: 64 rows = 8 words = 32 bytes
     const int k = col0 + 8 * lane + warp;
@@ -919,26 +922,58 @@ encode_fp8_kernel(const EncodeArgs a) {
 // ------------------------------------------------------------------------------------------
 // 4. mask -> CSR / CSC
 // ------------------------------------------------------------------------------------------
-// Exclusive prefix sum of n counts by one block; ptr[n] = total.  Also publishes nnz.  (The total
-// cannot exceed the caller's capacity: the host refuses capacities below 2 n_tail, and at most
-// n_tail entries lie beyond either threshold.  The fill kernels still guard every write.)
+// The CSR and the CSC of the residual are built from the encoder's mask and counts in three launches
+// (formerly five, two of them single-block scans).
+//
+// Launch 1, sparse_prefix_kernel: block 0 turns the row counts into csr_rowptr (and nnz); every
+// other block owns 1024 columns: their column pointers -- the counts of all earlier columns are
+// summed by the block itself, so no block waits for another -- and, per column, the running offsets
+// of the 64-row strips (strip_off), from which the fill kernel places a strip's entries.
+// (A total cannot exceed the caller's capacity: the host refuses capacities below 2 n_tail, and at
+// most n_tail entries lie beyond either threshold.  The fill kernel still guards every write.)
 __global__ void __launch_bounds__(1024, 1)
-scan_counts_kernel(const int* __restrict__ cnt, int n, int* __restrict__ ptr, int* nnz_out) {
+sparse_prefix_kernel(const int* __restrict__ row_cnt, int rows, int* __restrict__ rowptr, int* __restrict__ nnz_out,
+                     const int* __restrict__ col_cnt, const uint8_t* __restrict__ strip_cnt, int cols, int strips,
+                     int* __restrict__ colptr, int* __restrict__ strip_off) {
   __shared__ long long warp_tot[32];
   const int t = threadIdx.x;
-  const int per = (n + 1023) / 1024;
-  const int b = min(n, t * per), e = min(n, b + per);
-  int s = 0;
-  for (int i = b; i < e; ++i) s += cnt[i];
-  const long long incl = block_scan_1024(s, warp_tot);
-  int run = int(incl) - s;
-  for (int i = b; i < e; ++i) {
-    ptr[i] = run;
-    run += cnt[i];
+  if (blockIdx.x == 0) {
+    const int per = (rows + 1023) / 1024;
+    const int b = min(rows, t * per), e = min(rows, b + per);
+    int s = 0;
+    for (int i = b; i < e; ++i) s += row_cnt[i];
+    const long long incl = block_scan_1024(s, warp_tot);
+    int run = int(incl) - s;
+    for (int i = b; i < e; ++i) {
+      rowptr[i] = run;
+      run += row_cnt[i];
+    }
+    if (t == 1023) {
+      rowptr[rows] = int(incl);
+      if (nnz_out) *nnz_out = int(incl);
+    }
+    return;
   }
-  if (t == 1023) {
-    ptr[n] = int(incl);
-    if (nnz_out) *nnz_out = int(incl);
+  const int c0 = (int(blockIdx.x) - 1) * 1024;
+  // entries of all earlier columns
+  int before = 0;
+  for (int i = t; i < c0; i += 1024) before += col_cnt[i];
+  const long long earlier = block_scan_1024(before, warp_tot);
+  __shared__ long long s_base;
+  if (t == 1023) s_base = earlier;
+  __syncthreads();
+  const int k = c0 + t;
+  const int mine = k < cols ? col_cnt[k] : 0;
+  const long long incl = block_scan_1024(mine, warp_tot);
+  if (k < cols) colptr[k] = int(s_base + incl) - mine;
+  if (k == cols - 1) colptr[cols] = int(s_base + incl);
+  if (k >= cols) return;
+  int run = 0;
+#pragma unroll 8
+  for (int s = 0; s < strips; ++s) {
+    const int c = strip_cnt[(long long)s * cols + k];
+    strip_off[(long long)s * cols + k] = run;
+    run += c;
   }
 }
 
@@ -947,11 +982,14 @@ __device__ __forceinline__ float residual_of(const __nv_bfloat16* x, long long i
   return __fsub_rn(v, v > hi ? hi : lo);
 }
 
-__global__ void __launch_bounds__(256)
-csr_fill_kernel(const uint32_t* __restrict__ mask, const __nv_bfloat16* __restrict__ x, int rows, int cols,
-                const float* __restrict__ thresholds, int thr_per_row, const int* __restrict__ rowptr, long long cap,
-                int* __restrict__ csr_col, float* __restrict__ csr_val) {
-  const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+// CSR: one warp per row sweeps the row's mask words; a warp scan of the words' bit counts gives
+// every marked entry its place, columns ascending.
+__device__ __forceinline__ void csr_fill_block(int block, const uint32_t* __restrict__ mask,
+                                               const __nv_bfloat16* __restrict__ x, int rows, int cols,
+                                               const float* __restrict__ thresholds, int thr_per_row,
+                                               const int* __restrict__ rowptr, long long cap, int* __restrict__ csr_col,
+                                               float* __restrict__ csr_val) {
+  const int row = block * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= rows) return;
   int base = rowptr[row];
@@ -983,43 +1021,27 @@ csr_fill_kernel(const uint32_t* __restrict__ mask, const __nv_bfloat16* __restri
   }
 }
 
-// Per column: running offsets of the strips inside the column, total -> col_cnt.
-__global__ void __launch_bounds__(256)
-csc_strip_prefix_kernel(const uint8_t* __restrict__ strip_cnt, int cols, int strips, int* __restrict__ strip_off,
-                        int* __restrict__ col_cnt) {
-  const int k = blockIdx.x * blockDim.x + threadIdx.x;
-  if (k >= cols) return;
-  int run = 0;
-#pragma unroll 8
-  for (int s = 0; s < strips; ++s) {
-    const int c = strip_cnt[(long long)s * cols + k];
-    strip_off[(long long)s * cols + k] = run;
-    run += c;
-  }
-  col_cnt[k] = run;
-}
-
-// Column direction: one warp per (64-row strip, 32-column word of the mask).  Lane <-> row: each
-// lane keeps the mask word of its row.  For every column of the word that holds a marked entry
-// (usually one or two: the outlier channels), a ballot gives each marked row its rank inside the
-// column, so all gathers of a column are issued at once and the order is by row by construction.
-__global__ void __launch_bounds__(256)
-csc_fill_kernel(const uint32_t* __restrict__ mask, const __nv_bfloat16* __restrict__ x, int rows, int cols,
-                const float* __restrict__ thresholds, int thr_per_row, const int* __restrict__ colptr,
-                const int* __restrict__ strip_off, long long cap, int* __restrict__ csc_row,
-                float* __restrict__ csc_val) {
-  const int q = blockIdx.x * 8 + (threadIdx.x >> 5);
+// CSC: one warp per (64-row strip, 32-column word of the mask).  Lane <-> row: each lane keeps the
+// mask word of its row.  For every column of the word that holds a marked entry (usually one or
+// two: the outlier channels), a ballot gives each marked row its rank inside the column, so all
+// gathers of a column are issued at once and the order is by row by construction.
+__device__ __forceinline__ void csc_fill_block(int bx, int strip, const uint32_t* __restrict__ mask,
+                                               const __nv_bfloat16* __restrict__ x, int rows, int cols,
+                                               const float* __restrict__ thresholds, int thr_per_row,
+                                               const int* __restrict__ colptr, const int* __restrict__ strip_off,
+                                               long long cap, int* __restrict__ csc_row, float* __restrict__ csc_val) {
+  const int q = bx * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   const int words_per_row = cols >> 5;
   if (q >= words_per_row) return;
-  const int r0 = blockIdx.y * ENC_TM;
+  const int r0 = strip * ENC_TM;
   const uint32_t w0 = mask[(long long)(r0 + lane) * words_per_row + q];
   const uint32_t w1 = mask[(long long)(r0 + 32 + lane) * words_per_row + q];
   const uint32_t any0 = __reduce_or_sync(0xFFFFFFFFu, w0);
   const uint32_t any1 = __reduce_or_sync(0xFFFFFFFFu, w1);
   if (!(any0 | any1)) return;
   // lane c holds the next free position of column 32 q + c
-  int next = colptr[32 * q + lane] + strip_off[(long long)blockIdx.y * cols + 32 * q + lane];
+  int next = colptr[32 * q + lane] + strip_off[(long long)strip * cols + 32 * q + lane];
   const uint32_t lt_mask = (1u << lane) - 1u;
 #pragma unroll
   for (int half = 0; half < 2; ++half) {
@@ -1043,6 +1065,25 @@ csc_fill_kernel(const uint32_t* __restrict__ mask, const __nv_bfloat16* __restri
       if (lane == c) next += __popc(b);
     }
   }
+}
+
+// Launches 2 and 3 fill the CSR (8 rows per block) and the CSC (8 mask words of one strip per block).
+// They share only their inputs and run on two streams where the caller offers them: the forward's
+// compensation waits for the CSR alone.
+__global__ void __launch_bounds__(256)
+csr_fill_kernel(const uint32_t* __restrict__ mask, const __nv_bfloat16* __restrict__ x, int rows, int cols,
+                const float* __restrict__ thresholds, int thr_per_row, const int* __restrict__ rowptr, long long cap,
+                int* __restrict__ csr_col, float* __restrict__ csr_val) {
+  csr_fill_block(blockIdx.x, mask, x, rows, cols, thresholds, thr_per_row, rowptr, cap, csr_col, csr_val);
+}
+
+__global__ void __launch_bounds__(256)
+csc_fill_kernel(const uint32_t* __restrict__ mask, const __nv_bfloat16* __restrict__ x, int rows, int cols,
+                const float* __restrict__ thresholds, int thr_per_row, const int* __restrict__ colptr,
+                const int* __restrict__ strip_off, long long cap, int* __restrict__ csc_row,
+                float* __restrict__ csc_val) {
+  csc_fill_block(blockIdx.x, blockIdx.y, mask, x, rows, cols, thresholds, thr_per_row, colptr, strip_off, cap, csc_row,
+                 csc_val);
 }
 
 size_t r256(size_t b) { return (b + 255) & ~size_t(255); }
@@ -1124,6 +1165,7 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
   ea.mask = sc.mask;
   ea.row_cnt = sc.row_cnt;
   ea.strip_cnt = sc.strip_cnt;
+  ea.col_cnt = sc.col_cnt;
   ea.e5m2 = out->format == FP4_FORMAT_E5M2;
   ea.fmax = fp8_max(out->format);
   const dim3 tile_grid((cols + ENC_TK - 1) / ENC_TK, rows / ENC_TM);
@@ -1150,6 +1192,7 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
           x, rows, cols / 8, ctx->occ_hist, parity, sc.row_max, sc.row_min, sc.row_cnt, n, n_tail, out->thresholds,
           parity + 1, status, ctx->quantile_mode == FP4_QUANTILE_ABS);
     }
+    FP4_CUDA_TRY(cudaMemsetAsync(sc.col_cnt, 0, size_t(cols) * 4, stream));     // the encoder adds to it
     {
       KernelScope scope(ctx, stream, KC_ENCODE, 1);
       if (per_token)
@@ -1163,33 +1206,32 @@ int launch_quantize(fp4_ctx* ctx, cudaStream_t stream, Arena& arena, const void*
       FP4_CUDA_TRY(cudaEventRecord(overlap->encoded, stream));
       FP4_CUDA_TRY(cudaStreamWaitEvent(sp, overlap->encoded, 0));
     }
-    // The CSC chain takes a stream of its own where the caller offers one: it shares only the
-    // mask and the counts with the CSR chain.
-    cudaStream_t sc2 = sp;
-    if (sp != stream && overlap->stream_csc) {
-      sc2 = overlap->stream_csc;
-      FP4_CUDA_TRY(cudaStreamWaitEvent(sc2, overlap->encoded, 0));
-    }
     const uint32_t* mask32 = reinterpret_cast<const uint32_t*>(sc.mask);
     const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x_bf16);
     const int strips = rows / ENC_TM;
+    // The CSC's fill takes a stream of its own where the caller offers one.
+    cudaStream_t sc2 = sp;
     {
       KernelScope scope(ctx, sp, KC_SPARSE, 2);
-      scan_counts_kernel<<<1, 1024, 0, sp>>>(sc.row_cnt, rows, out->csr_rowptr, out->nnz);
+      sparse_prefix_kernel<<<1 + (cols + 1023) / 1024, 1024, 0, sp>>>(sc.row_cnt, rows, out->csr_rowptr, out->nnz,
+                                                                    sc.col_cnt, sc.strip_cnt, cols, strips,
+                                                                    out->csc_colptr, sc.strip_off);
+      if (sp != stream && overlap->colptr_done) FP4_CUDA_TRY(cudaEventRecord(overlap->colptr_done, sp));
+      if (sp != stream && overlap->stream_csc && overlap->colptr_done) {
+        sc2 = overlap->stream_csc;
+        FP4_CUDA_TRY(cudaStreamWaitEvent(sc2, overlap->colptr_done, 0));
+      }
       csr_fill_kernel<<<(rows + 7) / 8, 256, 0, sp>>>(mask32, xb, rows, cols, out->thresholds, per_token, out->csr_rowptr,
                                                       out->sparse_cap, out->csr_col, out->csr_val);
     }
     if (sp != stream) FP4_CUDA_TRY(cudaEventRecord(overlap->csr_done, sp));
     {
-      KernelScope scope(ctx, sc2, KC_SPARSE, 3);
-      csc_strip_prefix_kernel<<<(cols + 255) / 256, 256, 0, sc2>>>(sc.strip_cnt, cols, strips, sc.strip_off, sc.col_cnt);
-      scan_counts_kernel<<<1, 1024, 0, sc2>>>(sc.col_cnt, cols, out->csc_colptr, nullptr);
-      if (sc2 != sp && overlap->colptr_done) FP4_CUDA_TRY(cudaEventRecord(overlap->colptr_done, sc2));
+      KernelScope scope(ctx, sc2, KC_SPARSE, 1);
       const dim3 cgrid((cols / 32 + 7) / 8, strips);
       csc_fill_kernel<<<cgrid, 256, 0, sc2>>>(mask32, xb, rows, cols, out->thresholds, per_token, out->csc_colptr, sc.strip_off,
                                               out->sparse_cap, out->csc_row, out->csc_val);
     }
-    if (sc2 != sp) FP4_CUDA_TRY(cudaEventRecord(overlap->csc_done, sc2));
+    if (sp != stream && overlap->csc_done) FP4_CUDA_TRY(cudaEventRecord(overlap->csc_done, sc2));
   } else {
     if (prescale && prescale_div > 0.0f) {
       float* d = scale_axis == 0 ? sc.pre_cols : sc.pre_rows;
