@@ -186,18 +186,18 @@ struct Fp4GemmDesc {
 int launch_gemm_fp4_two(fp4_ctx* ctx, cudaStream_t stream, const Fp4GemmDesc& first, const Fp4GemmDesc& second,
                         int gemm_kind, int32_t* status);
 
-// Lets the mask -> CSR / CSC stage of a clamping quantisation run beside the caller's stream: both
-// chains start after `encoded` (recorded on the main stream); the CSR chain runs on `stream` and
-// records `csr_done` there; the CSC chain runs on `stream_csc` and records `colptr_done` after its
-// column pointers and `csc_done` at its end there (null: it follows the CSR on `stream`).  The caller
-// joins the streams.
+// Lets the mask -> CSR / CSC stage of a clamping quantisation run beside the caller's stream: it
+// starts after `encoded` (recorded on the main stream); the pointers kernel and the CSR fill run on
+// `stream`, which records `colptr_done` once row and column pointers are complete and `csr_done`
+// after the CSR fill; the CSC fill runs on `stream_csc` behind `colptr_done` and records `csc_done`
+// there (null: it follows the CSR fill on `stream`).  The caller joins the streams.
 struct SparseOverlap {
   cudaStream_t stream;
   cudaEvent_t encoded;
   cudaEvent_t csr_done;
   cudaStream_t stream_csc;
   cudaEvent_t csc_done;
-  cudaEvent_t colptr_done;    // recorded on the CSC chain's stream once csc_colptr is complete (or null)
+  cudaEvent_t colptr_done;    // csr_rowptr and csc_colptr are complete (or null: the CSC fill stays on `stream`)
 };
 
 // Quantiser pieces (quantize.cu)
