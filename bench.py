@@ -141,6 +141,27 @@ def layer_inputs(cfg, WL, seed=0):
     return out
 
 
+def fuse_shared(layers_in):
+    """q|k|v and gate|up as one linear each: the group's weights (and output gradients) side by side."""
+    groups = (("q", "k", "v"), ("gate", "up"))
+    by_name = {t[0]: t for t in layers_in}
+    out, done = [], set()
+    for t in layers_in:
+        name = t[0]
+        if name in done:
+            continue
+        grp = next((g for g in groups if name in g and all(n in by_name for n in g)), None)
+        if grp is None:
+            out.append(t)
+            continue
+        members = [by_name[n] for n in grp]
+        done.update(grp)
+        out.append(("|".join(grp), members[0][1], sum(m[2] for m in members), members[0][3],
+                    np.ascontiguousarray(np.concatenate([m[4] for m in members], axis=1)),
+                    np.ascontiguousarray(np.concatenate([m[5] for m in members], axis=1))))
+    return out
+
+
 ORACLE_SAMPLE_TOKENS = 1024         # tokens of the first linear the oracle is timed on (a bounded sample)
 
 
@@ -310,6 +331,9 @@ def main():
                     help="operand formats: w4a4 (the method, default); w4a8 / w8a4: E4M3 activations / weights "
                          "(the ablation settings); w4a4-dy8 / w4a4-dy8e5m2: dY quantised to E4M3 / E5M2.  All but w4a4 need --gemm-kind 1")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fuse-shared", action="store_true",
+                    help="q|k|v and gate|up as one linear each (weights stored side by side): Y and dW are those of the "
+                         "separate linears, dA is the gradient with respect to the shared input")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer measurement (profiling runs)")
     ap.add_argument("--no-isolated", action="store_true", help="skip the single-kernel measurements")
     ap.add_argument("--no-share-activations", action="store_true",
@@ -354,7 +378,10 @@ def main():
     lib = fp4.load_library()
     share = not args.no_share_activations
     owner = {}                                   # id of the host activation array -> first layer that reads it
-    for name, K, N, a_bits, w_bits, dy_bits in layer_inputs(cfg, WL, seed=rank):
+    inputs = layer_inputs(cfg, WL, seed=rank)
+    if args.fuse_shared:
+        inputs = fuse_shared(inputs)
+    for name, K, N, a_bits, w_bits, dy_bits in inputs:
         hA, hW, hG = pinned(a_bits), pinned(w_bits), pinned(dy_bits)
         first = owner.setdefault(id(a_bits), len(layers)) if share else len(layers)
         shared = first != len(layers)
@@ -588,7 +615,9 @@ def main():
                        "precision": args.precision,
                        "l2": f"inputs exceed L2: {resident_bytes / 1e6:.0f} MB touched per step",
                        "launch": "one CUDA graph per step, replayed",
-                       "shared_activations": ("q/k/v and gate/up read one activation tensor: quantised once, re-used"
+                       "shared_activations": ("q|k|v and gate|up run as one linear each (weights side by side)"
+                                              if args.fuse_shared else
+                                              "q/k/v and gate/up read one activation tensor: quantised once, re-used"
                                               if share else "every linear quantises its activation"),
                        "weights": ("codes of the weights cached across the timed steps (micro-batches of one "
                                    "optimizer step)" if args.cache_weights else "quantised in every step"),

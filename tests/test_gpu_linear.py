@@ -230,6 +230,42 @@ def test_reuse_quantised_activation(lib, ctx):
     assert torch.equal(y_shared, y_fresh) and torch.equal(da_s, da_f) and torch.equal(dw_s, dw_f)
 
 
+def test_linears_that_share_an_input_as_one_call(lib, ctx):
+    """q/k/v-style grouping: with the group's weights stored side by side ([K x (N1 + N2 + N3)]) one
+    call does the work of three.  Weights are scaled per output channel and dY for the weight
+    gradient per output channel too, so Y of the fused call is the separate calls' Y bit for bit,
+    column block by column block (heavy residual: dense tail included), and dW the same sums: equal
+    bit for bit except where the tensor-core dense class groups its token ranges differently for a
+    different N (fp32 additions of the same partial products: a few ulp).  dA of the fused call is the gradient with respect to the shared input -- the
+    sum over the group, accumulated in fp32 inside one GEMM with dY quantised token-wise over the
+    whole row -- and is held to the oracle's value for the fused linear."""
+    M, K, alpha = 1024, 512, 0.97
+    a_bits, w1, dy1 = WL.small_case(M, K, 256, seed=41, alpha_outliers=12)
+    _, w2, dy2 = WL.small_case(M, K, 384, seed=42)
+    _, w3, dy3 = WL.small_case(M, K, 128, seed=43)
+    w_cat = np.ascontiguousarray(np.concatenate([w1, w2, w3], axis=1))
+    dy_cat = np.ascontiguousarray(np.concatenate([dy1, dy2, dy3], axis=1))
+    A = _dev(a_bits)
+    ctx.status.zero_()
+    y_cat, sa, sw = lib.fp4_linear_fwd(ctx, A, _dev(w_cat), alpha)
+    da_cat, dw_cat = lib.fp4_linear_bwd(ctx, _dev(dy_cat), _dev(w_cat), sa, sw, out_f32=True)
+    n0 = 0
+    for w_bits, dy_bits in ((w1, dy1), (w2, dy2), (w3, dy3)):
+        n1 = n0 + w_bits.shape[1]
+        y, sa_g, sw_g = lib.fp4_linear_fwd(ctx, A, _dev(w_bits), alpha)
+        _, dw = lib.fp4_linear_bwd(ctx, _dev(dy_bits), _dev(w_bits), sa_g, sw_g, out_f32=True, want_da=False)
+        torch.cuda.synchronize()
+        assert torch.equal(y_cat[:, n0:n1], y)
+        got, want = dw_cat[:, n0:n1].double(), dw.double()
+        assert ((got - want).abs() <= 1e-5 * want.abs().max()).all()
+        assert (got == want).double().mean() > 0.9
+        n0 = n1
+    assert ctx.read_status() == 0
+    f = O.linear_fwd(a_bits, w_cat, alpha)
+    b = O.linear_bwd(dy_cat, w_cat, f)
+    assert_close_f32(da_cat.cpu().numpy(), b.da, b.da, None, "dA of the fused linear")
+
+
 def test_config0_full_layer(lib, ctx):
     """The small configuration in full: X[256 x 1024] with 8 outlier channels, alpha = 0.99, DGE on."""
     cfg = WL.CONFIGS[0]
