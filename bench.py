@@ -381,22 +381,37 @@ def main():
     inputs = layer_inputs(cfg, WL, seed=rank)
     if args.fuse_shared:
         inputs = fuse_shared(inputs)
-    for name, K, N, a_bits, w_bits, dy_bits in inputs:
-        hA, hW, hG = pinned(a_bits), pinned(w_bits), pinned(dy_bits)
+    pinned_a = {}                                # one pinned copy of an activation that several linears read
+    while inputs:
+        name, K, N, a_bits, w_bits, dy_bits = inputs.pop(0)      # the unpinned copies are dropped as we go
+        if id(a_bits) not in pinned_a:
+            pinned_a[id(a_bits)] = pinned(a_bits)
+        hA, hW, hG = pinned_a[id(a_bits)], pinned(w_bits), pinned(dy_bits)
         first = owner.setdefault(id(a_bits), len(layers)) if share else len(layers)
         shared = first != len(layers)
         L = dict(name=name, K=K, N=N, hA=hA, hW=hW, hG=hG, W=hW.to(dev), G=hG.to(dev),
-                 A=layers[first]["A"] if shared else hA.to(dev), reuse_a=shared,
+                 A=layers[first]["A"] if shared else hA.to(dev), reuse_a=shared, keep=a_bits,
                  Y=torch.empty((M, N), dtype=torch.bfloat16, device=dev),
                  dA=torch.empty((M, K), dtype=torch.bfloat16, device=dev),
                  dW=torch.empty((K, N), dtype=torch.bfloat16, device=dev),
                  sa=layers[first]["sa"] if shared else fp4.QTensor(M, K, 0, dev, fp4.tail_capacity(M, K, alpha), fmt=fmt_a),
-                 sw=fp4.QTensor(K, N, 1, dev, fmt=fmt_w),
-                 hY=torch.empty((M, N), dtype=torch.bfloat16).pin_memory(),
-                 hdA=torch.empty((M, K), dtype=torch.bfloat16).pin_memory(),
-                 hdW=torch.empty((K, N), dtype=torch.bfloat16).pin_memory())
+                 sw=fp4.QTensor(K, N, 1, dev, fmt=fmt_w))
+        del w_bits, dy_bits
         layers.append(L)
         ws_bytes = max(ws_bytes, int(lib.fp4_step_host_workspace_bytes(M, K, N, alpha)))
+    for L in layers:
+        L.pop("keep")                            # (held only so that ids of activation arrays stayed unique)
+    # pinned host outputs of the end-to-end measurement: one set, as large as the largest linear
+    # needs, written by every linear in turn (the copies back are ordered on one stream)
+    def host_out(n_elems):
+        return torch.empty(n_elems, dtype=torch.bfloat16).pin_memory()
+    hY_all = host_out(max(M * L["N"] for L in layers))
+    hdA_all = host_out(max(M * L["K"] for L in layers))
+    hdW_all = host_out(max(L["K"] * L["N"] for L in layers))
+    for L in layers:
+        L["hY"] = hY_all[:M * L["N"]].view(M, L["N"])
+        L["hdA"] = hdA_all[:M * L["K"]].view(M, L["K"])
+        L["hdW"] = hdW_all[:L["K"] * L["N"]].view(L["K"], L["N"])
     ctx = fp4.Context(local_rank, ws_bytes)
     flop_step = sum(6.0 * M * L["K"] * L["N"] for L in layers)
     resident_bytes = sum(2 * (M * L["K"] + L["K"] * L["N"] + M * L["N"]) * 2 for L in layers)
