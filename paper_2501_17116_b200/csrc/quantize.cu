@@ -631,7 +631,7 @@ struct EncodeArgs {
 // MODE_DUAL: codes hold the row-scaled tensor x (.) pre_col, codes_t the column-scaled tensor
 // x (.) pre_row.  OCC (clamping) implies MODE_ROWS without prescale.
 template <int MODE, bool OCC, bool PRESCALE, bool PER_TOKEN = false>
-__global__ void __launch_bounds__(ENC_THREADS)
+__global__ void __launch_bounds__(ENC_THREADS, 4)
 encode_kernel(const EncodeArgs a) {
   __shared__ float s_gcol[ENC_TK];
   __shared__ float s_grow[ENC_TM];
