@@ -471,7 +471,7 @@ comp_wgrad_long_kernel(float* __restrict__ comp, const int* __restrict__ colptr,
 // in that order, so that the blocks in flight at any time read one or two 512-byte-wide slabs of dY
 // (tokens x 512 bytes: a few MB, which stay in L2) instead of all of it: every token's piece of a
 // slab is gathered by about 1 % of the columns, and those re-reads then hit L2.
-__global__ void __launch_bounds__(COMP_THREADS)
+__global__ void __launch_bounds__(COMP_THREADS, 4)
 comp_wgrad_short_kernel(float* __restrict__ comp, const int* __restrict__ colptr, const int* __restrict__ row,
                         const float* __restrict__ val, const uint4* __restrict__ dy, const int* __restrict__ list,
                         const int* __restrict__ counts, int N) {
