@@ -211,6 +211,11 @@ int fp4_linear_fwd(fp4_ctx* ctx, void* stream, const void* A_bf16, const void* W
  * multiplication by d_A[m] (wgrad), so that the forward's codes of W and A are re-used.
  *   dY_bf16 [M x N], W_bf16 [K x N], dA [M x K], dW [K x N] (BF16, or float if out_f32).
  *   dA or dW may be NULL to skip that gradient.
+ *   With a heavy residual (same condition as in fp4_linear_fwd, and at least 512 tokens) the
+ *   residual's dense columns -- the same outlier channels -- are multiplied with dY on the tensor
+ *   cores (exact three-term BF16 split of the residual, chunks of 128 tokens added in fp32 in token
+ *   order); the other entries are added per entry in fp32.  That part of dW differs from the
+ *   per-entry sum by at most 4e-6 * sum_m |A - A_c|[m,k] |dY|[m,n] (times the DGE factor).
  *   gemm_kind | FP4_BWD_DY_E4M3 (or FP4_BWD_DY_E5M2) quantises both copies of dY to E4M3 (E5M2)
  *   bytes; the saved operands keep the formats the forward gave them; with an 8-bit weight Q' = 1
  *   whatever dge_on says.
