@@ -499,7 +499,23 @@ comp_wgrad_short_kernel(float* __restrict__ comp, const int* __restrict__ colptr
     if (slot >= n_cols || n0 >= N) continue;
     const int k = list[slot];
     float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    strided_entries_times_dense(acc, row, val, colptr[k], colptr[k + 1], 1, dy, N >> 3, n0 >> 3);
+    {
+      const int vec_per_row = N >> 3, vcol = n0 >> 3;
+      int e = colptr[k];
+      const int e1 = colptr[k + 1];
+      for (; e + 8 <= e1; e += 8) {                 // eight gathers in flight, entries in order
+        int r[8];
+        float v[8];
+        uint4 d[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { r[u] = __ldg(&row[e + u]); v[u] = __ldg(&val[e + u]); }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) d[u] = __ldg(&dy[(long long)r[u] * vec_per_row + vcol]);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) fma8(acc, v[u], d[u]);
+      }
+      for (; e < e1; ++e) fma8(acc, __ldg(&val[e]), __ldg(&dy[(long long)__ldg(&row[e]) * vec_per_row + vcol]));
+    }
     store8_f32(comp + (long long)(n_before + slot) * N + n0, acc);
   }
 }
