@@ -502,7 +502,7 @@ def main():
     if alpha < 1.0:
         probe = torch.empty(32 << 20, dtype=torch.uint8, device=dev)
         sink = torch.zeros(1, dtype=torch.int32, device=dev)
-        blocks, reps = 4 * SM_COUNT, 1
+        blocks, reps = 16 * SM_COUNT, 1             # enough blocks that launch ramp and tail do not show
         best = None
         for _ in range(4):
             q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

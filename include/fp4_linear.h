@@ -270,7 +270,7 @@ int fp4_profile_enable(fp4_ctx* ctx, int on);
 /* Measurement support (no counterpart in the paper): a read-only kernel for measuring the bandwidth
  * of the L2 cache, the bound of the per-entry gathers of the sparse compensation (Section 3.2: one
  * row of the dense matrix per residual entry).  `blocks` blocks of 256 threads each read all of
- * `buf` (`bytes`, a multiple of 16384, at least 65536, 16-byte aligned; choose it smaller than L2)
+ * `buf` (`bytes`, a multiple of 32768, at least 65536, 16-byte aligned; choose it smaller than L2)
  * `repeats` times with 16-byte loads that bypass L1, every block from its own starting offset.
  * Bytes read = blocks * repeats * bytes; the caller times the call.  `sink` is a device word the
  * kernel may write.                                                                          */

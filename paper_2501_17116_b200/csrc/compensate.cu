@@ -527,10 +527,10 @@ l2_read_probe_kernel(const uint4* __restrict__ buf, long long n_vec, int repeats
   unsigned acc = 0;
   const long long start = ((long long)blockIdx.x * 9973 * 256) % n_vec;
   for (int r = 0; r < repeats; ++r) {
-    for (long long i0 = 0; i0 < n_vec; i0 += 4 * 256) {
-      uint4 v[4];
+    for (long long i0 = 0; i0 < n_vec; i0 += 8 * 256) {
+      uint4 v[8];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < 8; ++u) {
         long long i = start + i0 + u * 256 + threadIdx.x;
         if (i >= n_vec) i -= n_vec;
         if (i >= n_vec) i -= n_vec;
@@ -539,7 +539,7 @@ l2_read_probe_kernel(const uint4* __restrict__ buf, long long n_vec, int repeats
                      : "l"(buf + i));
       }
 #pragma unroll
-      for (int u = 0; u < 4; ++u) acc ^= v[u].x ^ v[u].y ^ v[u].z ^ v[u].w;
+      for (int u = 0; u < 8; ++u) acc ^= v[u].x ^ v[u].y ^ v[u].z ^ v[u].w;
     }
   }
   if (acc == 0x9E3779B9u) *sink = acc;               // keeps the loads alive
@@ -549,7 +549,7 @@ l2_read_probe_kernel(const uint4* __restrict__ buf, long long n_vec, int repeats
 
 extern "C" int fp4_l2_read_probe(void* stream, const void* buf, size_t bytes, int repeats, int blocks, unsigned* sink) {
   if (!buf || !sink) return FP4_ERR_NULL;
-  if (bytes < 4096 * 16 || (bytes % (4 * 256 * 16)) || repeats <= 0 || blocks <= 0 ||
+  if (bytes < 4096 * 16 || (bytes % (8 * 256 * 16)) || repeats <= 0 || blocks <= 0 ||
       (reinterpret_cast<uintptr_t>(buf) & 15))
     return FP4_ERR_ARG;
   l2_read_probe_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
