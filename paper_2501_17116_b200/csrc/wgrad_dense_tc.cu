@@ -308,13 +308,21 @@ int make_bf16_map(fp4_ctx* ctx, CUtensorMap* map, const void* base, int64_t rows
 
 }  // namespace
 
-// Ranges of chunks per block of output columns: about one CTA per SM (148 on this GPU).
+// Ranges of chunks per block of output columns: the split (at most 16 ranges) whose CTAs, taken
+// in rounds of one per SM, finish soonest -- rounds x chunks per CTA, plus about one chunk's time per
+// round for filling the pipeline.
 static int splits_for(int sms, int64_t M, int64_t N) {
   const int tiles = int((N + DT_NT - 1) / DT_NT);
   const int chunks = int((M + DT_CHUNK - 1) / DT_CHUNK);
-  int splits = (sms < 148 ? sms : 148) / tiles;
-  splits = splits < 1 ? 1 : splits;
-  return splits > chunks ? chunks : splits;
+  if (sms > 148) sms = 148;
+  int best = 1;
+  long long best_cost = -1;
+  for (int s = 1; s <= 16 && s <= chunks; ++s) {
+    const long long rounds = (tiles * s + sms - 1) / sms;
+    const long long cost = rounds * ((chunks + s - 1) / s + 1);
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
+  }
+  return best;
 }
 
 int dense_tc_splits(const fp4_ctx* ctx, int64_t M, int64_t N) { return splits_for(ctx->num_sms, M, N); }
