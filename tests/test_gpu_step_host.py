@@ -120,3 +120,17 @@ def test_host_step_with_thresholds_per_token(lib):
     assert not torch.equal(Y0, Y)
     for c in (ref, ctx, dflt):
         c.close()
+
+
+def test_l2_probe_runs_and_reads_what_it_says(lib):
+    """Measurement support: the probe reads blocks * repeats * bytes and leaves the device usable."""
+    buf = torch.zeros(4 << 20, dtype=torch.uint8, device="cuda")
+    sink = torch.zeros(1, dtype=torch.int32, device="cuda")
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    lib.fp4_l2_read_probe(buf, 2, 296, sink)
+    b.record()
+    torch.cuda.synchronize()
+    gbs = 296 * 2 * buf.numel() / (a.elapsed_time(b) / 1e3) / 1e9
+    assert 100.0 < gbs < 100000.0
+    assert int(sink.item()) == 0

@@ -99,3 +99,11 @@ def test_sparse_capacity_is_the_librarys_rule(lib):
 
 def test_debug_switches_validate_their_arguments(lib):
     assert lib.fp4_debug_set(None, 1, 1000) == -1
+
+
+def test_l2_probe_validates_its_arguments(lib):
+    dummy = C.c_void_p(4096)
+    assert lib.fp4_l2_read_probe(None, None, 1 << 20, 1, 1, dummy) == -1
+    assert lib.fp4_l2_read_probe(None, dummy, 1000, 1, 1, dummy) == -7           # not a multiple of 32 KB
+    assert lib.fp4_l2_read_probe(None, dummy, 1 << 20, 0, 1, dummy) == -7
+    assert lib.fp4_l2_read_probe(None, C.c_void_p(4100), 1 << 20, 1, 1, dummy) == -7   # misaligned
