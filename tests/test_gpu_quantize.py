@@ -184,6 +184,43 @@ def test_occ_values_outside_the_histogram_window(lib, ctx):
         _check_dense(q, ref)
 
 
+def _occ_equals_oracle(lib, c, bits, alpha):
+    c.status.zero_()
+    q = lib.fp4_quantize(c, _dev(bits), 0, alpha=alpha)
+    torch.cuda.synchronize()
+    assert c.read_status() == 0
+    ref = O.occ_quantize(O.bf16_bits_to_f64(bits), alpha)
+    _check_sparse(q, ref)
+    _check_dense(q, ref)
+
+
+@pytest.mark.parametrize("kind", ["positive", "negative", "relu", "two_scales", "constant", "tiny"])
+def test_selection_on_tensors_whose_bulk_is_not_around_zero(lib, ctx, kind):
+    """One-signed tensors (both thresholds on one side of zero), a tensor with more exact zeros than
+    the clamped share (lo = 0), rows of very different scale, a constant tensor and one no larger than
+    the sample of the selection."""
+    rng = np.random.default_rng(32)
+    a = rng.standard_normal((256, 1024)).astype(np.float32)
+    if kind == "positive":
+        a = np.abs(a) + np.float32(0.5)
+    elif kind == "negative":
+        a = -np.abs(a) * np.float32(100.0) - np.float32(1.0)
+    elif kind == "relu":
+        a = np.maximum(a, np.float32(0.0))
+    elif kind == "two_scales":
+        a[::2] *= np.float32(1e-4)
+        a[1::2] *= np.float32(50.0)
+    elif kind == "constant":
+        a[:] = np.float32(-1.5)
+    else:
+        a = np.ascontiguousarray(a[:128, :128])
+    bits = WL.to_bf16_bits(a)
+    for alpha in (0.99, 0.97, 0.9999):
+        if round((1.0 - alpha) * a.size) < 1:
+            continue
+        _occ_equals_oracle(lib, ctx, bits, alpha)
+
+
 def test_config0_activation_and_weight(lib, ctx):
     cfg = WL.CONFIGS[0]
     a_bits = WL.activations(cfg, 1024)
