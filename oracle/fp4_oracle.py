@@ -399,7 +399,7 @@ def occ_quantize(a, alpha: float, quantile: str = "signed") -> Quantized:
 
 
 # --------------------------------------------------------------------------- #
-# FP4 GEMM: Fig. 2 ("two scaling factors are then applied to the final result")
+# FP4 GEMM: Fig. 2 (both scale vectors are applied to the accumulated result)
 # --------------------------------------------------------------------------- #
 def gemm_codes(codes_a, codes_b) -> np.ndarray:
     """acc[i, j] = sum_c val(codes_a[i, c]) * val(codes_b[j, c]), exact.
