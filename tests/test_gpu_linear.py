@@ -16,6 +16,14 @@ of 64 FP16 columns, 4 instructions each), each off by at most 2^-23 of the runni
 from the two-term FP16 splits, i.e. at most 4e-6 of sum_k |dA[m,k]| |W[k,n]|.  Where both branches
 cancel to a thousandth of their terms that floor can exceed 1e-3 of the branches, so the cases that
 can take the tail add TAIL_FLOOR * (|dA| |W|)[m,n] to the allowance.
+
+Accumulation floor of the per-entry compensation.  The compensation products are accumulated in
+fp32 (one fused multiply-add per residual entry, then the sum with the FP4 branch and the DGE
+factor): by the standard bound for a sum of n terms its error is at most (n + 4) * 2^-24 of the
+sum of the terms' magnitudes.  That is far below 1e-3 of the branches unless the terms cancel
+by more than four orders of magnitude, which the randomised runs do meet (one output in 4e8: 83
+terms of up to 8.5e-3 adding up to 4e-9 beside an FP4 branch of exactly 0, where the GPU's value
+is the fp32 sum to the last bit); `fp32_sum_floor` gives that bound for the cases drawn at random.
 """
 import numpy as np
 import pytest
@@ -32,6 +40,15 @@ TAIL_FLOOR = 4e-6
 def tail_floor(f: "O.Forward", w_bits):
     """Allowance for the tensor cores' accumulation of the dense tail: TAIL_FLOOR * (|dA| |W|)."""
     return TAIL_FLOOR * (np.abs(f.qa.residual) @ np.abs(O.bf16_bits_to_f64(w_bits)))
+
+
+def fp32_sum_floor(residual, dense_abs, transpose=False):
+    """(n + 4) 2^-24 sum |terms| for the fp32-accumulated product of the sparse residual [M x K] with
+    a dense matrix: residual @ dense [M x N] (n = entries of the row), or with `transpose`
+    residual^T @ dense [K x N] (n = entries of the column)."""
+    r = np.abs(residual.T if transpose else residual)
+    n = np.count_nonzero(r, axis=1).astype(np.float64)
+    return (n[:, None] + 4.0) * 2.0 ** -24 * (r @ dense_abs)
 
 
 @pytest.fixture(scope="module")
