@@ -191,7 +191,10 @@ int fp4_gemm(fp4_ctx* ctx, void* stream, const uint8_t* a_codes, const uint8_t* 
  *   residual's columns that at least max(M / 4, 512) tokens hit -- the outlier channels of
  *   Appendix D, up to 128 of them -- are multiplied on the tensor cores inside the GEMM (two-term
  *   FP16 splits of residual and weight); the other entries are added per entry in fp32.  The
- *   result differs from the per-entry sum by at most 4e-6 * sum_k |A - A_c|[m,k] |W|[k,n].
+ *   result differs from the per-entry sum by at most 4e-6 * sum_k |A - A_c|[m,k] |W|[k,n]
+ *   (weights below 2^-12 of their column's largest count as that much).  A residual value
+ *   beyond 43 000 times its token's clamped absmax does not fit the FP16 operand: the call
+ *   then adds every entry per entry.
  */
 #define FP4_REUSE_W 1
 #define FP4_REUSE_A 2

@@ -256,15 +256,18 @@ hot_columns_kernel(const int* __restrict__ colptr, int K, int hot_from, int* __r
   if (t == 0) *count = min(total, TAIL_MAX_COLS);
 }
 
-// Two-term FP16 split of x: hi = RN16(x), lo = RN16(x - hi).
-__device__ __forceinline__ void split_half(float x, __half& hi, __half& lo) {
+// Two-term FP16 split of x: hi = RN16(x), lo = RN16(x - hi), stored for the cross products as
+// hi_small = hi / TAIL_BALANCE and lo_big = TAIL_BALANCE * lo (exact powers of two: see GemmTail).
+__device__ __forceinline__ void split_half(float x, __half& hi, __half& hi_small, __half& lo_big) {
   hi = __float2half_rn(x);
-  lo = __float2half_rn(x - __half2float(hi));
+  const float h = __half2float(hi);
+  hi_small = __float2half_rn(h * (1.0f / TAIL_BALANCE));
+  lo_big = __float2half_rn((x - h) * TAIL_BALANCE);
 }
 
 // A operand of the dense tail: row m holds, for hot column s = 64 j + c, the value
-// x = residual[m, k_s] / (d_A[m] * TAIL_SCALE) as x_hi at columns 192 j + c and 192 j + 64 + c and
-// x_lo at 192 j + 128 + c; zero elsewhere.  One warp per token walks the token's CSR row.  A value
+// x = residual[m, k_s] / (d_A[m] * TAIL_SCALE) as x_hi at column 192 j + c, x_hi / TAIL_BALANCE at
+// 192 j + 64 + c and TAIL_BALANCE x_lo at 192 j + 128 + c; zero elsewhere.  One warp per token walks the token's CSR row.  A value
 // that FP16 cannot hold (or a token whose de-scale is zero) switches the tail off for this call:
 // *count becomes 0 and the per-entry kernel keeps every entry.
 __global__ void __launch_bounds__(COMP_THREADS)
@@ -303,20 +306,21 @@ tail_a_kernel(const int* __restrict__ rowptr, const int* __restrict__ col, const
     if (!is_hot) continue;
     const float x = __fdiv_rn(v, scale);
     if (!(fabsf(x) <= 65504.0f)) { bad = true; continue; }         // also catches NaN (0 / 0)
-    __half hi, lo;
-    split_half(x, hi, lo);
+    __half hi, hi_small, lo_big;
+    split_half(x, hi, hi_small, lo_big);
     const int at = 192 * (slot >> 6) + (slot & 63);
     row[at] = hi;
-    row[at + 64] = hi;
-    row[at + 128] = lo;
+    row[at + 64] = hi_small;
+    row[at + 128] = lo_big;
   }
   if (kept && lane == 0) kept_end[m] = n_kept;
   if (bad) atomicExch(count, 0);
 }
 
 // B operand of the dense tail: row n holds, for hot column s = 64 j + c, the value
-// x = TAIL_SCALE * W[k_s, n] / d_W[n] as x_hi at 192 j + c and 192 j + 128 + c and x_lo at
-// 192 j + 64 + c (|x| <= 6 * 256 for an E2M1 operand: the weight is at most amax in magnitude).  The buffer
+// x = TAIL_SCALE * W[k_s, n] / d_W[n] as x_hi at 192 j + c, TAIL_BALANCE x_lo at 192 j + 64 + c and
+// x_hi / TAIL_BALANCE at 192 j + 128 + c (|x| <= 6 * 4, or 448 * 4 for an FP8 weight: the weight is at
+// most amax in magnitude).  The buffer
 // was cleared before.  One thread per (n, group of hot columns).
 __global__ void __launch_bounds__(256)
 tail_b_kernel(const __nv_bfloat16* __restrict__ w, const int* __restrict__ list_hot, const int* __restrict__ count,
@@ -330,12 +334,12 @@ tail_b_kernel(const __nv_bfloat16* __restrict__ w, const int* __restrict__ list_
   for (int s = blockIdx.y; s < hot; s += gridDim.y) {
     const float wv = __bfloat162float(w[size_t(list_hot[s]) * N + n]);
     const float x = inv_ok != 0.0f ? __fdiv_rn(wv * TAIL_SCALE, d) : 0.0f;
-    __half hi, lo;
-    split_half(x, hi, lo);
+    __half hi, hi_small, lo_big;
+    split_half(x, hi, hi_small, lo_big);
     const int at = 192 * (s >> 6) + (s & 63);
     row[at] = hi;
-    row[at + 64] = lo;
-    row[at + 128] = hi;
+    row[at + 64] = lo_big;
+    row[at + 128] = hi_small;
   }
 }
 
