@@ -4,8 +4,9 @@ Seeded draws over shapes (multiples of 128, ragged against every tile size), cla
 activation distributions, number of outlier channels, GEMM kind and DGE setting.  Every draw checks
 what the fixed cases check: saved operands bit for bit, the three outputs within the bar stated in
 test_gpu_linear.py.  The draws are fixed by the seed, so a failure reproduces; FP4_RANDOM_DRAWS in
-the environment sets how many are made (default 16); FP4_TEST_NO_OVERLAP=1 runs them with the
-library's side streams switched off.
+the environment sets how many are made (default 16), FP4_RANDOM_SEED moves both generators to
+another sequence of cases (default 0); FP4_TEST_NO_OVERLAP=1 runs them with the library's side
+streams switched off.
 """
 import os
 
@@ -18,6 +19,7 @@ from paper_2501_17116_b200 import workloads as WL
 from test_gpu_linear import _dev, _saved_matches, assert_close_f32, fp32_sum_floor, tail_floor
 
 pytestmark = pytest.mark.gpu
+SEED_SHIFT = 100003 * int(os.environ.get("FP4_RANDOM_SEED", "0"))
 
 
 @pytest.fixture(scope="module")
@@ -58,9 +60,9 @@ def _draws(n, seed):
 
 
 @pytest.mark.parametrize("i,M,K,N,alpha,dist,hot,kind,dge,fp8",
-                         _draws(int(os.environ.get("FP4_RANDOM_DRAWS", "16")), seed=2501))
+                         _draws(int(os.environ.get("FP4_RANDOM_DRAWS", "16")), seed=2501 + SEED_SHIFT))
 def test_random_layer_matches_oracle(lib, ctx, i, M, K, N, alpha, dist, hot, kind, dge, fp8):
-    a_bits, w_bits, dy_bits = WL.small_case(M, K, N, seed=1000 + i, alpha_outliers=hot, dist=dist)
+    a_bits, w_bits, dy_bits = WL.small_case(M, K, N, seed=1000 + i + SEED_SHIFT, alpha_outliers=hot, dist=dist)
     fmt_a = {"a8": "e4m3", "a5": "e5m2"}.get(fp8, "e2m1")
     fmt_w = "e4m3" if "w8" in fp8 else "e2m1"
     fmt_dy = "e4m3" if "dy8" in fp8 else ("e5m2" if "dy5" in fp8 else "e2m1")
@@ -122,13 +124,13 @@ def _quantizer_draws(n, seed):
 
 
 @pytest.mark.parametrize("i,rows,cols,alpha,spread,zeros",
-                         _quantizer_draws(int(os.environ.get("FP4_RANDOM_DRAWS", "16")), seed=1711))
+                         _quantizer_draws(int(os.environ.get("FP4_RANDOM_DRAWS", "16")), seed=1711 + SEED_SHIFT))
 def test_random_clamping_quantizer_is_bit_exact(lib, ctx, i, rows, cols, alpha, spread, zeros):
     """Thresholds, codes in both layouts, amax and the sparse residual on tensors whose rows live on
     scales spread over many binades (values outside the histogram kernel's window, subnormals),
     with ties and exact zeros of both signs."""
     from test_gpu_quantize import _check_dense, _check_sparse, _check_token_mode
-    rng = np.random.default_rng(5000 + i)
+    rng = np.random.default_rng(5000 + i + SEED_SHIFT)
     a = rng.standard_normal((rows, cols)).astype(np.float32)
     if spread:
         a *= np.exp2(rng.integers(-spread, spread + 1, size=(rows, 1))).astype(np.float32)
