@@ -16,7 +16,7 @@ import torch
 
 from oracle import fp4_oracle as O
 from paper_2501_17116_b200 import workloads as WL
-from test_gpu_linear import _dev, _saved_matches, assert_close_f32, fp32_sum_floor, tail_floor
+from test_gpu_linear import _dev, _saved_matches, assert_bf16_rounding, assert_close_f32, fp32_sum_floor, tail_floor
 
 pytestmark = pytest.mark.gpu
 SEED_SHIFT = 100003 * int(os.environ.get("FP4_RANDOM_SEED", "0"))
@@ -62,7 +62,40 @@ def _draws(n, seed):
 @pytest.mark.parametrize("i,M,K,N,alpha,dist,hot,kind,dge,fp8",
                          _draws(int(os.environ.get("FP4_RANDOM_DRAWS", "16")), seed=2501 + SEED_SHIFT))
 def test_random_layer_matches_oracle(lib, ctx, i, M, K, N, alpha, dist, hot, kind, dge, fp8):
-    a_bits, w_bits, dy_bits = WL.small_case(M, K, N, seed=1000 + i + SEED_SHIFT, alpha_outliers=hot, dist=dist)
+    _layer_case(lib, ctx, 1000 + i, M, K, N, alpha, dist, hot, kind, dge, fp8, out_f32=True)
+
+
+def _many_tile_draws(n, seed):
+    """Shapes whose GEMMs have more 128 x 240 tiles than the GPU has SMs (forward 176-234, and with the
+    large K the backward's two problems as well), so that CTAs walk several tiles and both
+    accumulator buffers; every other draw stores BF16 outputs."""
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        M = int(rng.choice([2048, 2304]))
+        K = int(rng.choice([256, 640, 2560]))
+        N = int(rng.choice([2560, 2944, 3072]))
+        alpha = float(rng.choice([1.0, 0.999, 0.99, 0.97]))
+        dist = str(rng.choice(["normal", "student_t3", "laplace"]))
+        hot = int(rng.choice([0, 9, 40]))
+        kind = int(rng.integers(0, 2))
+        dge = bool(rng.integers(0, 2))
+        out.append((i, M, K, N, alpha, dist, hot, kind, dge, i % 2 == 0))
+    return out
+
+
+@pytest.mark.parametrize("i,M,K,N,alpha,dist,hot,kind,dge,out_f32",
+                         _many_tile_draws(int(os.environ.get("FP4_RANDOM_BIG_DRAWS", "3")), seed=4099 + SEED_SHIFT))
+def test_random_layer_with_more_tiles_than_sms(lib, i, M, K, N, alpha, dist, hot, kind, dge, out_f32):
+    c = lib.Context(0, int(lib.load_library().fp4_workspace_bytes(M, K, N)))
+    try:
+        _layer_case(lib, c, 700000 + i, M, K, N, alpha, dist, hot, kind, dge, "none", out_f32=out_f32)
+    finally:
+        c.close()
+
+
+def _layer_case(lib, ctx, case_seed, M, K, N, alpha, dist, hot, kind, dge, fp8, out_f32):
+    a_bits, w_bits, dy_bits = WL.small_case(M, K, N, seed=case_seed + SEED_SHIFT, alpha_outliers=hot, dist=dist)
     fmt_a = {"a8": "e4m3", "a5": "e5m2"}.get(fp8, "e2m1")
     fmt_w = "e4m3" if "w8" in fp8 else "e2m1"
     fmt_dy = "e4m3" if "dy8" in fp8 else ("e5m2" if "dy5" in fp8 else "e2m1")
@@ -71,9 +104,9 @@ def test_random_layer_matches_oracle(lib, ctx, i, M, K, N, alpha, dist, hot, kin
     b = O.linear_bwd(dy_bits, w_bits, f, dge_on=dge, fmt_dy=fmt_dy)
     A, W, dY = _dev(a_bits), _dev(w_bits), _dev(dy_bits)
     ctx.status.zero_()
-    y32, sa, sw = lib.fp4_linear_fwd(ctx, A, W, alpha, gemm_kind=kind, out_f32=True, fmt_a=code[fmt_a],
+    y32, sa, sw = lib.fp4_linear_fwd(ctx, A, W, alpha, gemm_kind=kind, out_f32=out_f32, fmt_a=code[fmt_a],
                                      fmt_w=code[fmt_w])
-    da32, dw32 = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, gemm_kind=kind, out_f32=True, dge_on=dge,
+    da32, dw32 = lib.fp4_linear_bwd(ctx, dY, W, sa, sw, gemm_kind=kind, out_f32=out_f32, dge_on=dge,
                                     dy_fmt=code[fmt_dy])
     torch.cuda.synchronize()
     assert ctx.read_status() == 0
@@ -105,6 +138,11 @@ def test_random_layer_matches_oracle(lib, ctx, i, M, K, N, alpha, dist, hot, kin
         # fp32 accumulation of the per-entry compensation (matters only where its terms cancel)
         floor_y = floor_y + fp32_sum_floor(f.qa.residual, np.abs(O.bf16_bits_to_f64(w_bits)))
         floor_dw = floor_dw + fp32_sum_floor(f.qa.residual, np.abs(O.bf16_bits_to_f64(dy_bits)), transpose=True) * np.abs(b.dge)
+    if not out_f32:
+        assert_bf16_rounding(y32, f.y, "Y", f.y_fp4, f.y_comp, floor_y)
+        assert_bf16_rounding(da32, b.da, "dA", None, None, floor_da)
+        assert_bf16_rounding(dw32, b.dw, "dW", b.s_fp4 * b.dge, b.s_comp * b.dge, floor_dw)
+        return
     assert_close_f32(y32.cpu().numpy(), f.y, f.y_fp4, f.y_comp, "Y", floor_y)
     assert_close_f32(da32.cpu().numpy(), b.da, b.da, None, "dA", floor_da)
     assert_close_f32(dw32.cpu().numpy(), b.dw, b.s_fp4 * b.dge, b.s_comp * b.dge, "dW", floor_dw)
