@@ -192,7 +192,9 @@ int fp4_gemm(fp4_ctx* ctx, void* stream, const uint8_t* a_codes, const uint8_t* 
  *   Appendix D, up to 128 of them -- are multiplied on the tensor cores inside the GEMM (two-term
  *   FP16 splits of residual and weight); the other entries are added per entry in fp32.  The
  *   result differs from the per-entry sum by at most 4e-6 * sum_k |A - A_c|[m,k] |W|[k,n]
- *   (weights below 2^-12 of their column's largest count as that much).  A residual value
+ *   + 2e-11 * amax_W[n] * sum_k |A - A_c|[m,k] (the second term is the resolution of W / d_W in
+ *   FP16: it matters only for weights ten orders of magnitude below their column's largest).
+ *   A residual value
  *   beyond 43 000 times its token's clamped absmax does not fit the FP16 operand: the call
  *   then adds every entry per entry.
  */

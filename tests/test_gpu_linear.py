@@ -15,7 +15,10 @@ inside the tensor cores, whose fp32 accumulation rounds toward zero: up to 24 ad
 of 64 FP16 columns, 4 instructions each), each off by at most 2^-23 of the running sum, plus 2^-21
 from the two-term FP16 splits, i.e. at most 4e-6 of sum_k |dA[m,k]| |W[k,n]|.  Where both branches
 cancel to a thousandth of their terms that floor can exceed 1e-3 of the branches, so the cases that
-can take the tail add TAIL_FLOOR * (|dA| |W|)[m,n] to the allowance.
+can take the tail add TAIL_FLOOR * (|dA| |W|)[m,n] to the allowance.  The weight operand of the tail
+is W / d_W in FP16, whose smallest step (with the scaled low half) is 2^-31 of a unit: a weight
+more than ten orders of magnitude below its column's largest is not resolved, hence the second term
+of `tail_floor`, 2^-33 d_W[n] sum_k |dA[m,k]| (1e-9 of the first for ordinary weights).
 
 Accumulation floor of the per-entry compensation.  The compensation products are accumulated in
 fp32 (one fused multiply-add per residual entry, then the sum with the FP4 branch and the DGE
@@ -38,8 +41,13 @@ TAIL_FLOOR = 4e-6
 
 
 def tail_floor(f: "O.Forward", w_bits):
-    """Allowance for the tensor cores' accumulation of the dense tail: TAIL_FLOOR * (|dA| |W|)."""
-    return TAIL_FLOOR * (np.abs(f.qa.residual) @ np.abs(O.bf16_bits_to_f64(w_bits)))
+    """Allowance for the dense tail: TAIL_FLOOR * (|dA| |W|) for the tensor cores' accumulation and the
+    FP16 splits, plus the absolute resolution of the weight operand W / d_W in FP16 (2^-31 of a unit
+    with the scaled low half; the operand is 4 W / d_W against dA / (4 d_A)), which matters only for
+    weights ten orders of magnitude below their column's largest."""
+    r = np.abs(f.qa.residual)
+    return (TAIL_FLOOR * (r @ np.abs(O.bf16_bits_to_f64(w_bits)))
+            + 2.0 ** -33 * r.sum(axis=1)[:, None] * f.qw.descale.astype(np.float64)[None, :])
 
 
 def fp32_sum_floor(residual, dense_abs, transpose=False):

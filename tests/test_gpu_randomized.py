@@ -94,8 +94,38 @@ def test_random_layer_with_more_tiles_than_sms(lib, i, M, K, N, alpha, dist, hot
         c.close()
 
 
-def _layer_case(lib, ctx, case_seed, M, K, N, alpha, dist, hot, kind, dge, fp8, out_f32):
+def _degenerate(bits_list, rng):
+    """Zero rows and columns, rows on scales 2^-20 .. 2^20 and a few huge values in one column of each
+    of the three tensors: vectors whose absmax is 0, de-scales far from 1, residuals near and beyond
+    what the dense tail's FP16 operands hold."""
+    out = []
+    for bits in bits_list:
+        x = O.bf16_bits_to_f64(bits).astype(np.float32)
+        r, c = x.shape
+        if rng.random() < 0.7:
+            x[rng.integers(0, r, size=int(rng.integers(1, 4)))] = 0.0
+        if rng.random() < 0.7:
+            x[:, rng.integers(0, c, size=int(rng.integers(1, 4)))] = 0.0
+        if rng.random() < 0.5:
+            x *= np.exp2(rng.integers(-20, 21, size=(r, 1))).astype(np.float32)
+        if rng.random() < 0.5:
+            rows = rng.integers(0, r, size=int(rng.integers(1, 6)))
+            x[rows, int(rng.integers(0, c))] *= np.float32(10.0 ** rng.integers(3, 9))
+        out.append(WL.to_bf16_bits(x))
+    return out
+
+
+@pytest.mark.parametrize("i,M,K,N,alpha,dist,hot,kind,dge,fp8",
+                         _draws(int(os.environ.get("FP4_RANDOM_DRAWS", "16")), seed=9973 + SEED_SHIFT))
+def test_random_layer_with_degenerate_vectors(lib, ctx, i, M, K, N, alpha, dist, hot, kind, dge, fp8):
+    _layer_case(lib, ctx, 300000 + i, M, K, N, alpha, dist, hot, kind, dge, fp8, out_f32=True,
+                mutate=np.random.default_rng(77000 + i + SEED_SHIFT))
+
+
+def _layer_case(lib, ctx, case_seed, M, K, N, alpha, dist, hot, kind, dge, fp8, out_f32, mutate=None):
     a_bits, w_bits, dy_bits = WL.small_case(M, K, N, seed=case_seed + SEED_SHIFT, alpha_outliers=hot, dist=dist)
+    if mutate is not None:
+        a_bits, w_bits, dy_bits = _degenerate([a_bits, w_bits, dy_bits], mutate)
     fmt_a = {"a8": "e4m3", "a5": "e5m2"}.get(fp8, "e2m1")
     fmt_w = "e4m3" if "w8" in fp8 else "e2m1"
     fmt_dy = "e4m3" if "dy8" in fp8 else ("e5m2" if "dy5" in fp8 else "e2m1")
