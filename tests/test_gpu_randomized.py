@@ -123,7 +123,26 @@ def test_random_layer_with_degenerate_vectors(lib, ctx, i, M, K, N, alpha, dist,
                 mutate=np.random.default_rng(77000 + i + SEED_SHIFT))
 
 
-def _layer_case(lib, ctx, case_seed, M, K, N, alpha, dist, hot, kind, dge, fp8, out_f32, mutate=None):
+@pytest.mark.parametrize("i,M,K,N,alpha,dist,hot,kind,dge,fp8",
+                         _draws(int(os.environ.get("FP4_RANDOM_DRAWS", "16")), seed=31337 + SEED_SHIFT))
+def test_random_layer_in_the_other_quantile_modes(lib, i, M, K, N, alpha, dist, hot, kind, dge, fp8):
+    """The two variants of the clamp (one threshold on |x|; thresholds per token) through the whole
+    layer, forward and backward, FP8 settings and dense tail included where the draw has them."""
+    if alpha >= 1.0:
+        alpha = 0.99
+        if fp8 in ("a8", "a5"):
+            fp8 = "none"
+    quantile = "abs" if i % 2 == 0 else "token"
+    c = lib.Context(0, 1 << 30)
+    c.set_quantile_mode(lib.FP4_QUANTILE_ABS if quantile == "abs" else lib.FP4_QUANTILE_TOKEN)
+    try:
+        _layer_case(lib, c, 500000 + i, M, K, N, alpha, dist, hot, kind, dge, fp8, out_f32=True, quantile=quantile)
+    finally:
+        c.close()
+
+
+def _layer_case(lib, ctx, case_seed, M, K, N, alpha, dist, hot, kind, dge, fp8, out_f32, mutate=None,
+                quantile="signed"):
     a_bits, w_bits, dy_bits = WL.small_case(M, K, N, seed=case_seed + SEED_SHIFT, alpha_outliers=hot, dist=dist)
     if mutate is not None:
         a_bits, w_bits, dy_bits = _degenerate([a_bits, w_bits, dy_bits], mutate)
@@ -131,7 +150,7 @@ def _layer_case(lib, ctx, case_seed, M, K, N, alpha, dist, hot, kind, dge, fp8, 
     fmt_w = "e4m3" if "w8" in fp8 else "e2m1"
     fmt_dy = "e4m3" if "dy8" in fp8 else ("e5m2" if "dy5" in fp8 else "e2m1")
     code = {"e2m1": lib.FP4_FORMAT_E2M1, "e4m3": lib.FP4_FORMAT_E4M3, "e5m2": lib.FP4_FORMAT_E5M2}
-    f = O.linear_fwd(a_bits, w_bits, alpha, fmt_a=fmt_a, fmt_w=fmt_w)
+    f = O.linear_fwd(a_bits, w_bits, alpha, fmt_a=fmt_a, fmt_w=fmt_w, quantile=quantile)
     b = O.linear_bwd(dy_bits, w_bits, f, dge_on=dge, fmt_dy=fmt_dy)
     A, W, dY = _dev(a_bits), _dev(w_bits), _dev(dy_bits)
     ctx.status.zero_()
@@ -149,7 +168,10 @@ def _layer_case(lib, ctx, case_seed, M, K, N, alpha, dist, hot, kind, dge, fp8, 
         np.testing.assert_array_equal(sa.codes.cpu().numpy(), f.qa.packed() if fmt_a == "e2m1" else f.qa.codes)
         np.testing.assert_array_equal(sw.codes_t.cpu().numpy(),
                                       f.qw.packed_t() if fmt_w == "e2m1" else np.ascontiguousarray(f.qw.codes.T))
-    if alpha < 1.0:
+    if alpha < 1.0 and quantile == "token":
+        from test_gpu_quantize import _check_token_mode
+        _check_token_mode(sa, f.qa)
+    elif alpha < 1.0:
         th = sa.thresholds.cpu().numpy()
         assert (float(th[0]), float(th[1])) == (f.qa.lo, f.qa.hi)
         assert int(sa.nnz.item()) == int(np.count_nonzero(f.qa.residual))
